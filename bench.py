@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the MXFP4 weight-only linear path on B200.
+
+Workload (BASELINE.json config "7B-Llama-shaped decode layer set", M=1): one *step* is one
+draft-token pass over the linear projections of ``--layers`` (default 32) distinct 7B decoder
+layers -- q/k/v/o 4096x4096, gate/up 11008x4096, down 4096x11008 -- i.e. 7 mxq_linear calls per
+layer set, 224 per step, streaming 3.44 GB of MXFP4 weights (far larger than the 126 MB L2, so
+every step reads HBM).  Weights are synthetic (Student-t, seeded), direct-cast on the device by
+mxq_quantize before timing; the offline cast and the greedy-accept step are timed separately and
+reported under "extra".
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead (the only other
+place this file may execute anything under oracle/ is the cpu_baseline leg).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2503_13565_b200 import replicas, synth  # noqa: E402
+
+METRIC = "mxq_linear_hbm_gbs"
+UNIT = "GB/s"
+HBM_DATASHEET_GBS = 8000.0
+
+
+def algorithmic_bytes(m: int, n: int, k: int, y_bytes: int = 4) -> int:
+    """4.25 bits per weight + activations + outputs (the byte count the metric is defined on)."""
+    return n * k // 2 + n * k // 32 + 2 * m * k + y_bytes * m * n
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks: NVML polling thread (read-only) running during the timed region
+# ---------------------------------------------------------------------------------------------
+class ClockMonitor:
+    REASONS = {
+        0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+        0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+        0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+    }
+
+    def __init__(self, device_index: int):
+        self.samples, self.reason_bits, self.max_mhz = [], 0, None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            self._nv = pynvml
+            pynvml.nvmlInit()
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+                idx = int(vis.split(",")[device_index]) if vis and vis.split(",")[device_index].isdigit() else device_index
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self._h is not None:
+            self._stop.clear()
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+            self._thread = None
+
+    def summary(self):
+        bits = self.reason_bits & ~0x1  # idle between samples is not a throttle
+        return {
+            "sm_mhz": statistics.median(self.samples) if self.samples else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": [name for bit, name in self.REASONS.items() if bits & bit],
+            "samples": len(self.samples),
+        }
+
+
+# ---------------------------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------------------------
+def build_layers(mxq, n_layers: int, shapes, device):
+    """Direct-cast `n_layers` seeded layer sets on the device; returns [(name, n, k, codes, scales)]."""
+    out = []
+    for layer in range(n_layers):
+        for i, (name, n, k) in enumerate(shapes):
+            w = synth.weight(3, layer * len(shapes) + i, n, k, device=device)
+            codes, scales = mxq.mxq_quantize(w)
+            out.append((name, n, k, codes, scales))
+            del w
+    torch.cuda.synchronize()
+    return out
+
+
+class LinearPass:
+    """One pass over a list of quantised matrices at M token rows, replayed from a CUDA graph."""
+
+    def __init__(self, mxq, mats, m: int, device, seed: int, use_graph: bool = True):
+        self.mxq, self.mats, self.m = mxq, mats, m
+        ks = sorted({k for _, _, k, _, _ in mats})
+        self.x = {k: synth.normal_bf16((m, k), 1.0, seed + k, device) for k in ks}
+        self.y = [torch.empty((m, n), dtype=torch.float32, device=device) for _, n, _, _, _ in mats]
+        ws_bytes = max([mxq.mxq_linear_workspace_bytes(m, n, k) for _, n, k, _, _ in mats] + [16])
+        self.ws = mxq.new_workspace(ws_bytes, device)
+        self.bytes = sum(algorithmic_bytes(m, n, k) for _, n, k, _, _ in mats)
+        self.launches = len(mats)
+        self.graph = None
+        self.stream = torch.cuda.Stream(device=device)
+        if use_graph:
+            with torch.cuda.stream(self.stream):
+                self.enqueue()          # first call outside capture (lazy module loading)
+                self.stream.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=self.stream):
+                    self.enqueue()
+                self.graph = g
+
+    def enqueue(self):
+        for (_, n, k, codes, scales), y in zip(self.mats, self.y):
+            self.mxq.mxq_linear(self.x[k], codes, scales, out=y, workspace=self.ws)
+
+    def step(self):
+        if self.graph is not None:
+            self.graph.replay()
+        else:
+            self.enqueue()
+
+    def time(self, steps: int, warmup: int, monitor: ClockMonitor = None):
+        """seconds for `steps` passes, CUDA events on the launching stream, sync on both sides."""
+        with torch.cuda.stream(self.stream):
+            for _ in range(warmup):
+                self.step()
+            self.stream.synchronize()
+            replicas.barrier()
+            torch.cuda.synchronize()
+            if monitor:
+                monitor.start()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(self.stream)
+            for _ in range(steps):
+                self.step()
+            e1.record(self.stream)
+            self.stream.synchronize()
+            torch.cuda.synchronize()
+            if monitor:
+                monitor.stop()
+            replicas.barrier()
+        return e0.elapsed_time(e1) * 1e-3
+
+
+def time_e2e(mxq, mats, m: int, steps: int, warmup: int, device):
+    """Same pass through mxq_linear_host: activations come from pinned host memory and results go
+    back to pinned host memory inside the timed region (weights stay resident)."""
+    ks = sorted({k for _, _, k, _, _ in mats})
+    xh = {k: synth.normal_bf16((m, k), 1.0, 77 + k).pin_memory() for k in ks}
+    xs = {k: torch.empty((m, k), dtype=torch.bfloat16, device=device) for k in ks}
+    yh = [torch.empty((m, n), dtype=torch.float32).pin_memory() for _, n, _, _, _ in mats]
+    ys = [torch.empty((m, n), dtype=torch.float32, device=device) for _, n, _, _, _ in mats]
+    ws = mxq.new_workspace(max([mxq.mxq_linear_workspace_bytes(m, n, k) for _, n, k, _, _ in mats] + [16]), device)
+    stream = torch.cuda.Stream(device=device)
+    h2d = sum(2 * m * k for _, _, k, _, _ in mats)
+    d2h = sum(4 * m * n for _, n, _, _, _ in mats)
+
+    def one():
+        for (_, n, k, codes, scales), yh_i, ys_i in zip(mats, yh, ys):
+            mxq.mxq_linear_host(xh[k], codes, scales, yh_i, xs[k], ys_i, workspace=ws, stream=stream)
+
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            one()
+        stream.synchronize()
+        replicas.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        e0.record(stream)
+        for _ in range(steps):
+            one()
+        e1.record(stream)
+        stream.synchronize()
+        wall = time.perf_counter() - t0
+        replicas.barrier()
+    return max(e0.elapsed_time(e1) * 1e-3, 0.0), wall, h2d, d2h
+
+
+def time_fn(fn, iters: int, warmup: int = 3):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e-3 / iters
+
+
+def cpu_baseline_leg(m: int, budget_s: float = 15.0):
+    """The oracle, as it stands, on one 7B layer set (host cores of this machine)."""
+    import numpy as np
+
+    import oracle
+    mats = []
+    for i, (name, n, k) in enumerate(synth.LAYERS_7B):
+        rng = np.random.default_rng(i)
+        mats.append((n, k, rng.integers(0, 256, (n, k // 2), dtype=np.uint8),
+                     rng.integers(110, 126, (n, k // 32), dtype=np.uint8),
+                     synth.bits_of(synth.normal_bf16((m, k), 1.0, 5 + i))))
+    nbytes = sum(algorithmic_bytes(m, n, k) for n, k, *_ in mats)
+    reps, t_total = 0, 0.0
+    while t_total < budget_s and reps < 50:
+        t0 = time.perf_counter()
+        for n, k, codes, scales, x in mats:
+            oracle.linear(x, codes, scales)
+        t_total += time.perf_counter() - t0
+        reps += 1
+    return {"value": nbytes * reps / t_total / 1e9, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": "%d pass(es) over one 7B layer set (7 matrices, 202M weights) at M=%d, FP64" % (reps, m),
+            "us_per_layer_set": t_total / reps * 1e6}
+
+
+def run_ours(args):
+    rank, local_rank, world = replicas.env_world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    replicas.init("nccl")
+    import paper_2503_13565_b200 as mxq
+    mxq.binding.lib()  # fail loudly now if the extension is missing
+
+    shapes = synth.LAYERS_7B
+    mats = build_layers(mxq, args.layers, shapes, device)
+    m = args.m
+    monitor = ClockMonitor(local_rank)
+
+    main = LinearPass(mxq, mats, m, device, seed=31, use_graph=not args.no_graph)
+    secs = main.time(args.steps, args.warmup, monitor)
+    secs_max = replicas.max_over_ranks(secs, device)
+    bytes_step = main.bytes
+    value = replicas.sum_over_ranks(bytes_step * args.steps, device) / secs_max / 1e9
+    ms_per_step = secs_max / args.steps * 1e3
+    per_launch_s = secs / (args.steps * main.launches)
+    achieved = bytes_step / main.launches / per_launch_s / 1e9
+    peaks, peak_kind = measured_peaks()
+
+    # end to end with host buffers
+    e2e_steps = max(3, min(args.steps, 50))
+    e2e_dev, e2e_wall, h2d, d2h = time_e2e(mxq, mats, m, e2e_steps, 3, device)
+    e2e_secs = replicas.max_over_ranks(max(e2e_dev, e2e_wall), device)
+    e2e_value = replicas.sum_over_ranks(bytes_step * e2e_steps, device) / e2e_secs / 1e9
+
+    extra = {}
+    if rank == 0 and not args.quick:
+        # the verify-side pass (M=8) over the same layers
+        p8 = LinearPass(mxq, mats, 8, device, seed=32, use_graph=not args.no_graph)
+        s8 = p8.time(max(3, args.steps // 2), 3)
+        extra["m8"] = {"gbs": p8.bytes * max(3, args.steps // 2) / s8 / 1e9,
+                       "us_per_layer_set": s8 / max(3, args.steps // 2) / args.layers * 1e6}
+        del p8
+        # per-shape, one matrix at a time, rotating over the layers (each pass > L2)
+        per_shape = {}
+        for name, n, k in [("4096x4096", 4096, 4096), ("11008x4096", 11008, 4096), ("4096x11008", 4096, 11008)]:
+            sel = [t for t in mats if (t[1], t[2]) == (n, k)]
+            for mm in (1, 8):
+                p = LinearPass(mxq, sel, mm, device, seed=33, use_graph=not args.no_graph)
+                s = p.time(20, 3)
+                per_shape["%s_m%d" % (name, mm)] = {"us_per_call": s / 20 / len(sel) * 1e6,
+                                                    "gbs": p.bytes * 20 / s / 1e9}
+        extra["per_shape"] = per_shape
+        # direct cast throughput (2 B read + 0.53125 B written per weight)
+        w = synth.student_t_bf16((11008, 4096), 0.02, 1, device=device)
+        ws_ = [w.clone() for _ in range(4)]   # 360 MB rotated: larger than L2
+        codes = torch.empty((11008, 2048), dtype=torch.uint8, device=device)
+        scales = torch.empty((11008, 128), dtype=torch.uint8, device=device)
+        it = [0]
+
+        def q():
+            mxq.mxq_quantize(ws_[it[0] % 4], codes, scales)
+            it[0] += 1
+        tq = time_fn(q, 40)
+        extra["quantize"] = {"gbs": 11008 * 4096 * 2.53125 / tq / 1e9, "us_per_call": tq * 1e6, "shape": "11008x4096"}
+        del w, ws_
+        # greedy accept: 250 sequences x 17 rows x 32000 logits (FP32), one call
+        lg, draft, _, _ = synth.accept_trials(250, 16, 17, 32000, seed=1, device=device)
+        ws2 = mxq.new_workspace(mxq.mxq_accept_workspace_bytes(250, 17, 32000), device)
+        ta = time_fn(lambda: mxq.mxq_greedy_accept(lg, draft, workspace=ws2), 20)
+        extra["greedy_accept"] = {"gbs": lg.numel() * 4 / ta / 1e9, "us_per_call": ta * 1e6, "shape": "250x17x32000 f32"}
+        del lg
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline_leg(m)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "7B decode layer set (q,k,v,o 4096x4096; gate,up 11008x4096; down 4096x11008), "
+                               "M=%d, %d distinct layers per step" % (m, args.layers),
+                   "M": m, "layers": args.layers, "calls_per_step": main.launches, "bytes_per_step": bytes_step,
+                   "y_dtype": "f32", "l2": "inputs larger than L2 (%.2f GB of weights per step)" % (bytes_step / 1e9),
+                   "cuda_graph": not args.no_graph, "multi_gpu": "replicas only"},
+        "us_per_layer_set": ms_per_step * 1e3 / args.layers,
+        "pct_of_8000": 100.0 * value / world / HBM_DATASHEET_GBS,
+        "clocks": monitor.summary(),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps},
+        "gpu_launches": main.launches * args.steps,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_kind": "of " + peak_kind,
+                     "kernel": "mxq_linear M=%d" % m, "bytes_per_launch": bytes_step / main.launches},
+        "cpu_baseline": cpu,
+        "extra": extra,
+    }
+    if rank == 0:
+        print(json.dumps(line))
+    replicas.shutdown()
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm: the oracle on the host cores
+# ---------------------------------------------------------------------------------------------
+def run_reference(args):
+    rank, _, world = replicas.env_world()
+    if rank != 0:
+        return
+    import numpy as np
+
+    import oracle
+    m = args.m
+    frac = 8  # every 8th row of each matrix: a bounded sample of the layer set
+    mats = []
+    for i, (name, n, k) in enumerate(synth.LAYERS_7B):
+        rng = np.random.default_rng(i)
+        rows = np.arange(0, n, frac, dtype=np.int64)
+        mats.append((n, k, rows, rng.integers(0, 256, (n, k // 2), dtype=np.uint8),
+                     rng.integers(110, 126, (n, k // 32), dtype=np.uint8),
+                     synth.bits_of(synth.normal_bf16((m, k), 1.0, 5 + i))))
+    nbytes = sum(algorithmic_bytes(m, len(rows), k) for n, k, rows, *_ in mats)
+
+    def one():
+        for n, k, rows, codes, scales, x in mats:
+            oracle.linear(x, codes, scales, rows=rows)
+
+    for _ in range(args.warmup):
+        one()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one()
+    secs = time.perf_counter() - t0
+    value = nbytes * args.steps / secs / 1e9
+    sample = "every %dth output row of one 7B layer set per step (%.1fM weights), M=%d, FP64" % (
+        frac, sum(len(r) * k for _, k, r, *_ in mats) / 1e6, m)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "7B decode layer set, M=%d (CPU oracle, bounded sample)" % m, "M": m, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--layers", type=int, default=32, help="distinct 7B layer sets per step")
+    ap.add_argument("--m", type=int, default=1, help="token rows (1 = draft step)")
+    ap.add_argument("--no-graph", action="store_true", help="launch from Python instead of replaying a CUDA graph")
+    ap.add_argument("--quick", action="store_true", help="skip the extra measurements")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

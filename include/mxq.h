@@ -1,0 +1,141 @@
+/*
+ * mxq.h -- C ABI of libmxq: the MXFP4 weight-only-quantised linear layer that
+ * dominates every draft step of ML-SpecQD (arXiv 2503.13565), for one NVIDIA
+ * B200 (sm_100a).
+ *
+ * General rules, valid for every call below unless it says otherwise:
+ *   - Pointers named *_dev (and every pointer not named *_host) are DEVICE
+ *     pointers owned by the caller; the library allocates nothing, frees
+ *     nothing and keeps no pointer after the call returns.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     legacy default stream).  No call synchronises.
+ *   - The return value is an MXQ_* status.  Argument errors are found on the
+ *     host before anything is enqueued, so a non-zero status other than
+ *     MXQ_ERR_CUDA means nothing ran.  Nothing throws or aborts.
+ *   - Base pointers must be 16-byte aligned (MXQ_ERR_ALIGN otherwise).
+ *   - K must be a positive multiple of 32 and N >= 1 (MXQ_ERR_SHAPE otherwise).
+ *
+ * The MXFP4 tensor pair (Sec. III-D-3 of the paper: an FP4 weight tensor plus
+ * one 8-bit scale per 32 elements):
+ *   codes  uint8 [N][K/2]  row-major; byte j of a row holds element 2j in its
+ *                          low nibble and element 2j+1 in its high nibble.  A
+ *                          nibble is an E2M1 code  s e1 e0 m  (bias 1), i.e.
+ *                          one of 0, 0.5, 1, 1.5, 2, 3, 4, 6 with a sign.
+ *   scales uint8 [N][K/32] row-major; E8M0: the byte b stands for 2^(b-127);
+ *                          0xFF stands for NaN.
+ * Sixteen consecutive code bytes are one block of 32 weights and share one
+ * scale byte.  The dequantised weight is  w^ = (+-)value(code) * 2^(b-127).
+ */
+#ifndef MXQ_H
+#define MXQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MXQ_VERSION 100 /* major*100 + minor */
+
+enum mxq_status {
+    MXQ_OK = 0,
+    MXQ_ERR_NULL = 1,      /* a required pointer is NULL                               */
+    MXQ_ERR_SHAPE = 2,     /* a size is out of range (K % 32, M not in 1..16, ...)      */
+    MXQ_ERR_ALIGN = 3,     /* a base pointer is not 16-byte aligned                    */
+    MXQ_ERR_DTYPE = 4,     /* unknown MXQ_F32 / MXQ_BF16 selector                      */
+    MXQ_ERR_WORKSPACE = 5, /* workspace missing or smaller than *_workspace_bytes()     */
+    MXQ_ERR_CUDA = 6       /* the CUDA runtime reported an error at launch             */
+};
+
+enum mxq_dtype { MXQ_F32 = 0, MXQ_BF16 = 1 };
+
+#define MXQ_MAX_M 16 /* token rows per mxq_linear call                          */
+#define MXQ_MAX_T 64 /* speculated tokens per sequence in mxq_greedy_accept*    */
+
+/* Library version (MXQ_VERSION of the build). */
+int mxq_version(void);
+
+/* Static, human-readable text for a status code; never NULL. */
+const char *mxq_status_string(int status);
+
+/* Programmatic dependent launch.  When enabled (the default) mxq_linear kernels are
+ * launched so that their weight prefetch may overlap the tail of the previous kernel
+ * in the stream; they read X and write Y only after that kernel has completed, so
+ * results do not change.  Returns the previous setting.  Host-side, process-wide. */
+int mxq_set_pdl(int enabled);
+
+/* Bytes of a codes / scales tensor for an [N][K] weight matrix: N*K/2 and N*K/32
+ * (together 4.25 bits per weight, Sec. III-D-3).  0 if the shape is invalid. */
+size_t mxq_codes_bytes(int64_t N, int64_t K);
+size_t mxq_scales_bytes(int64_t N, int64_t K);
+
+/* Direct cast BF16 -> MXFP4 (Sec. III-D-3, steps i and ii).
+ *   W_bf16  [N][K] BF16 row-major, contiguous (read)
+ *   codes   [N][K/2], scales [N][K/32] (written; layout above)
+ *   nonfinite_blocks  optional uint32 counter (may be NULL); incremented once per
+ *           block that contained an Inf or a NaN.  The caller zeroes it.
+ * Per block of 32 along K: the scale is 2^(floor(log2 max|v|) - 2), never below
+ * 2^-127 (an all-zero block gets 2^-127); each element divided by the scale is
+ * rounded to the nearest E2M1 value, ties to the even code, magnitudes above 6
+ * clamp to 6; the sign bit of the input is always kept (so -0 stays -0).  A block
+ * holding Inf/NaN gets scale 0xFF and all-zero codes. */
+int mxq_quantize(const void *W_bf16, int64_t N, int64_t K, uint8_t *codes, uint8_t *scales,
+                 uint32_t *nonfinite_blocks, void *stream);
+
+/* Exact inverse map (the value each code/scale pair stands for, Sec. III-D-3), for
+ * tools and tests.  W_bf16_out [N][K] BF16.  Every w^ with scale byte <= 252 is
+ * BF16-representable and written exactly; 0xFF gives NaN; 253/254 may overflow to Inf. */
+int mxq_dequantize(const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K, void *W_bf16_out,
+                   void *stream);
+
+/* Workspace (bytes) mxq_linear needs for this shape; may be 0.  The workspace must be
+ * zero-filled once before its first use; every call leaves it ready for the next one
+ * (of any shape).  Two calls that may run concurrently need separate workspaces. */
+size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K);
+
+/* Weight-only-quantised linear layer (the MXFP4 GEMM of Sec. III-D-3, Eq. 2):
+ *     Y[m][n] = sum_k X[m][k] * w^[n][k],   1 <= M <= 16 token rows.
+ *   X_bf16  [M][K] BF16 row-major (read)
+ *   codes, scales  the MXFP4 pair for W[N][K] (read)
+ *   Y       [M][N] row-major, float (MXQ_F32) or BF16 rounded to nearest even (MXQ_BF16)
+ *   workspace / workspace_bytes  see mxq_linear_workspace_bytes (may be NULL / 0 if that is 0)
+ * Products are formed exactly and accumulated in FP32; the block scale is applied to
+ * 32-long partial sums (Eq. 2).  The summation order is fixed for a given shape, so
+ * results are bit-reproducible run to run.  A row containing a 0xFF scale yields NaN. */
+int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
+               void *Y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream);
+
+/* The same layer with the activations and the result in HOST memory (pinned memory
+ * makes the copies asynchronous).  X_host [M][K] BF16 is copied to X_stage_dev
+ * (>= M*K*2 bytes), the layer runs, and Y_stage_dev (>= M*N*elem bytes) is copied to
+ * Y_host, all on `stream`.  The weights stay resident on the device. */
+int mxq_linear_host(const void *X_host, int M, const uint8_t *codes, const uint8_t *scales, int64_t N,
+                    int64_t K, void *Y_host, int y_dtype, void *X_stage_dev, void *Y_stage_dev,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/* Workspace (bytes) for mxq_greedy_accept; same zero-once / reusable contract as above. */
+size_t mxq_accept_workspace_bytes(int64_t B, int R, int64_t V);
+
+/* Greedy verification of speculated tokens (Sec. III-A: tokens after the first
+ * mismatch are dropped; Sec. III-B: G accepted tokens plus one of the target's own).
+ *   logits  [B][R][V] row-major, MXQ_F32 or MXQ_BF16; row i of a sequence is the
+ *           target's distribution for the position draft token i proposes to fill;
+ *           R == T (no extra row) or R == T + 1
+ *   draft   [B][T] int32, 1 <= T <= 64
+ *   accept_len [B] int32: G = first i with draft[i] != argmax(logits[i]), else T
+ *   next_token [B] int32: argmax(logits[G]) if G < R, else -1
+ * argmax takes the lowest index among equal maxima and never selects a NaN; a row
+ * with nothing above -inf yields 0. */
+int mxq_greedy_accept(const void *logits, int logits_dtype, int64_t B, int R, int64_t V, const int32_t *draft,
+                      int T, int32_t *accept_len, int32_t *next_token, void *workspace, size_t workspace_bytes,
+                      void *stream);
+
+/* Same, with the verifier's tokens already known: verifier [B][R] int32. */
+int mxq_greedy_accept_tokens(const int32_t *draft, const int32_t *verifier, int64_t B, int T, int R,
+                             int32_t *accept_len, int32_t *next_token, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MXQ_H */

@@ -1,0 +1,211 @@
+"""Thin ctypes binding of ``libmxq.so`` -- argument marshalling only.
+
+Function names and argument order follow ``include/mxq.h``.  Tensors are torch CUDA
+tensors (torch supplies device memory and streams, nothing else); every step of the
+computation runs in the library's own kernels.  There is no fallback: if the shared
+library is missing, or a call returns a non-zero status, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmxq.so")
+
+MXQ_OK = 0
+MXQ_F32, MXQ_BF16 = 0, 1
+MAX_M, MAX_T = 16, 64
+
+_lib = None
+_lock = threading.Lock()
+
+
+class MxqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: status %d (%s)" % (where, status, status_string(status)))
+
+
+def lib() -> ctypes.CDLL:
+    """Load ``libmxq.so`` (built by ``python -m paper_2503_13565_b200.build``)."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            if not os.path.exists(LIB_PATH):
+                raise ImportError("libmxq.so is not built (%s missing): run python -m paper_2503_13565_b200.build; "
+                                  "there is no CPU fallback" % LIB_PATH)
+            L = ctypes.CDLL(LIB_PATH)
+            vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
+            L.mxq_version.restype = i32
+            L.mxq_status_string.restype = ctypes.c_char_p
+            L.mxq_status_string.argtypes = [i32]
+            L.mxq_set_pdl.restype = i32
+            L.mxq_set_pdl.argtypes = [i32]
+            for f in (L.mxq_codes_bytes, L.mxq_scales_bytes):
+                f.restype = sz
+                f.argtypes = [i64, i64]
+            L.mxq_linear_workspace_bytes.restype = sz
+            L.mxq_linear_workspace_bytes.argtypes = [i32, i64, i64]
+            L.mxq_accept_workspace_bytes.restype = sz
+            L.mxq_accept_workspace_bytes.argtypes = [i64, i32, i64]
+            L.mxq_quantize.restype = i32
+            L.mxq_quantize.argtypes = [vp, i64, i64, vp, vp, vp, vp]
+            L.mxq_dequantize.restype = i32
+            L.mxq_dequantize.argtypes = [vp, vp, i64, i64, vp, vp]
+            L.mxq_linear.restype = i32
+            L.mxq_linear.argtypes = [vp, i32, vp, vp, i64, i64, vp, i32, vp, sz, vp]
+            L.mxq_linear_host.restype = i32
+            L.mxq_linear_host.argtypes = [vp, i32, vp, vp, i64, i64, vp, i32, vp, vp, vp, sz, vp]
+            L.mxq_greedy_accept.restype = i32
+            L.mxq_greedy_accept.argtypes = [vp, i32, i64, i32, i64, vp, i32, vp, vp, vp, sz, vp]
+            L.mxq_greedy_accept_tokens.restype = i32
+            L.mxq_greedy_accept_tokens.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp]
+            _lib = L
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != MXQ_OK:
+        raise MxqError(status, where)
+
+
+def _stream(stream=None) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype, what: str) -> int:
+    if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError("%s must be a contiguous CUDA tensor of dtype %s" % (what, dtype))
+    return t.data_ptr()
+
+
+def _dt(dtype) -> int:
+    if dtype == torch.float32:
+        return MXQ_F32
+    if dtype == torch.bfloat16:
+        return MXQ_BF16
+    raise TypeError("dtype must be torch.float32 or torch.bfloat16")
+
+
+# ---- the calls of include/mxq.h ---------------------------------------------------------
+
+
+def mxq_version() -> int:
+    return int(lib().mxq_version())
+
+
+def status_string(status: int) -> str:
+    return lib().mxq_status_string(int(status)).decode()
+
+
+def mxq_set_pdl(enabled: bool) -> bool:
+    return bool(lib().mxq_set_pdl(1 if enabled else 0))
+
+
+def mxq_codes_bytes(n: int, k: int) -> int:
+    return int(lib().mxq_codes_bytes(n, k))
+
+
+def mxq_scales_bytes(n: int, k: int) -> int:
+    return int(lib().mxq_scales_bytes(n, k))
+
+
+def mxq_linear_workspace_bytes(m: int, n: int, k: int) -> int:
+    return int(lib().mxq_linear_workspace_bytes(m, n, k))
+
+
+def mxq_accept_workspace_bytes(b: int, r: int, v: int) -> int:
+    return int(lib().mxq_accept_workspace_bytes(b, r, v))
+
+
+def new_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """Zero-filled workspace of at least ``nbytes`` (the zero fill is the one-time initialisation)."""
+    return torch.zeros(max(16, (int(nbytes) + 15) // 16 * 16), dtype=torch.uint8, device=device)
+
+
+def mxq_quantize(w: torch.Tensor, codes: torch.Tensor = None, scales: torch.Tensor = None,
+                 nonfinite_blocks: torch.Tensor = None, stream=None):
+    """BF16 W[N,K] -> (codes u8 [N,K/2], scales u8 [N,K/32])."""
+    n, k = w.shape
+    if codes is None:
+        codes = torch.empty((n, k // 2), dtype=torch.uint8, device=w.device)
+    if scales is None:
+        scales = torch.empty((n, k // 32), dtype=torch.uint8, device=w.device)
+    cnt = 0 if nonfinite_blocks is None else _dev(nonfinite_blocks, torch.int32, "nonfinite_blocks")
+    _check(lib().mxq_quantize(_dev(w, torch.bfloat16, "W"), n, k, _dev(codes, torch.uint8, "codes"),
+                              _dev(scales, torch.uint8, "scales"), cnt, _stream(stream)), "mxq_quantize")
+    return codes, scales
+
+
+def mxq_dequantize(codes: torch.Tensor, scales: torch.Tensor, out: torch.Tensor = None, stream=None) -> torch.Tensor:
+    n, k = codes.shape[0], codes.shape[1] * 2
+    if out is None:
+        out = torch.empty((n, k), dtype=torch.bfloat16, device=codes.device)
+    _check(lib().mxq_dequantize(_dev(codes, torch.uint8, "codes"), _dev(scales, torch.uint8, "scales"), n, k,
+                                _dev(out, torch.bfloat16, "out"), _stream(stream)), "mxq_dequantize")
+    return out
+
+
+def mxq_linear(x: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, out: torch.Tensor = None,
+               out_dtype=torch.float32, workspace: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """Y[M,N] = X[M,K] . dequant(codes, scales)^T."""
+    m, k = x.shape
+    n = codes.shape[0]
+    if codes.shape[1] * 2 != k or tuple(scales.shape) != (n, k // 32):
+        raise ValueError("shape mismatch between X, codes and scales")
+    if out is None:
+        out = torch.empty((m, n), dtype=out_dtype, device=x.device)
+    ws_ptr, ws_bytes = (0, 0) if workspace is None else (_dev(workspace, torch.uint8, "workspace"), workspace.numel())
+    _check(lib().mxq_linear(_dev(x, torch.bfloat16, "X"), m, _dev(codes, torch.uint8, "codes"),
+                            _dev(scales, torch.uint8, "scales"), n, k, _dev(out, out.dtype, "Y"), _dt(out.dtype),
+                            ws_ptr, ws_bytes, _stream(stream)), "mxq_linear")
+    return out
+
+
+def mxq_linear_host(x_host: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, y_host: torch.Tensor,
+                    x_stage: torch.Tensor, y_stage: torch.Tensor, workspace: torch.Tensor = None, stream=None) -> None:
+    """Same layer with X and Y in (pinned) host memory; staging buffers live on the device."""
+    m, k = x_host.shape
+    n = codes.shape[0]
+    if x_host.is_cuda or y_host.is_cuda or x_host.dtype != torch.bfloat16 or not x_host.is_contiguous() \
+            or not y_host.is_contiguous() or tuple(y_host.shape) != (m, n):
+        raise TypeError("x_host / y_host must be contiguous host tensors (BF16 X[M,K], Y[M,N])")
+    if x_stage.numel() * x_stage.element_size() < m * k * 2 or \
+            y_stage.numel() * y_stage.element_size() < m * n * y_host.element_size():
+        raise ValueError("staging buffers too small")
+    ws_ptr, ws_bytes = (0, 0) if workspace is None else (_dev(workspace, torch.uint8, "workspace"), workspace.numel())
+    _check(lib().mxq_linear_host(x_host.data_ptr(), m, _dev(codes, torch.uint8, "codes"),
+                                 _dev(scales, torch.uint8, "scales"), n, k, y_host.data_ptr(), _dt(y_host.dtype),
+                                 x_stage.data_ptr(), y_stage.data_ptr(), ws_ptr, ws_bytes, _stream(stream)),
+           "mxq_linear_host")
+
+
+def mxq_greedy_accept(logits: torch.Tensor, draft: torch.Tensor, workspace: torch.Tensor = None, stream=None):
+    """logits [B,R,V] (fp32 or bf16), draft [B,T] int32 -> (accept_len [B], next_token [B]) int32."""
+    b, r, v = logits.shape
+    t = draft.shape[1]
+    if workspace is None:
+        workspace = new_workspace(mxq_accept_workspace_bytes(b, r, v), logits.device)
+    g = torch.empty(b, dtype=torch.int32, device=logits.device)
+    nxt = torch.empty(b, dtype=torch.int32, device=logits.device)
+    _check(lib().mxq_greedy_accept(_dev(logits, logits.dtype, "logits"), _dt(logits.dtype), b, r, v,
+                                   _dev(draft, torch.int32, "draft"), t, g.data_ptr(), nxt.data_ptr(),
+                                   _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)),
+           "mxq_greedy_accept")
+    return g, nxt
+
+
+def mxq_greedy_accept_tokens(draft: torch.Tensor, verifier: torch.Tensor, stream=None):
+    b, t = draft.shape
+    r = verifier.shape[1]
+    g = torch.empty(b, dtype=torch.int32, device=draft.device)
+    nxt = torch.empty(b, dtype=torch.int32, device=draft.device)
+    _check(lib().mxq_greedy_accept_tokens(_dev(draft, torch.int32, "draft"), _dev(verifier, torch.int32, "verifier"),
+                                          b, t, r, g.data_ptr(), nxt.data_ptr(), _stream(stream)),
+           "mxq_greedy_accept_tokens")
+    return g, nxt

@@ -1,0 +1,71 @@
+// Device-side helpers shared by the mxq kernels (sm_100a only).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/mxq.h"
+
+#if defined(__CUDA_ARCH__) && !defined(__CUDA_ARCH_FEAT_SM100_ALL)
+#error "mxq kernels use sm_100a-only conversions; compile with -gencode arch=compute_100a,code=sm_100a"
+#endif
+
+namespace mxq {
+
+constexpr int kBlock = 32;  // weights per scale (MX block), Sec. III-D-3
+
+// ---- programmatic dependent launch ---------------------------------------------------
+// wait: block until the kernel launched before this one in the stream has completed and
+// its writes are visible.  trigger: allow the next kernel in the stream to start launching.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// ---- loads that bypass L1 allocation (weights are read exactly once) -------------------
+__device__ __forceinline__ uint4 ld_stream_u4(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_stream_u32(const void *p) {
+    uint32_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+
+// ---- E2M1 / E8M0 decode ---------------------------------------------------------------
+// One code byte (element 2j in the low nibble, 2j+1 in the high nibble) -> the two values
+// as packed halves (.x = low nibble).  Exact: every E2M1 value is an FP16 number.
+__device__ __forceinline__ __half2 e2m1x2_to_half2(uint32_t byte) {
+    uint32_t out;
+    asm("{\n\t.reg .b8 b;\n\tcvt.u8.u32 b, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}" : "=r"(out) : "r"(byte));
+    return *reinterpret_cast<__half2 *>(&out);
+}
+
+// E8M0 byte -> 2^(b-127) as FP32.  b = 0 is the subnormal 2^-127, b = 255 is NaN.
+__device__ __forceinline__ float e8m0_to_float(uint32_t b) {
+    uint32_t bits = (b == 0u) ? 0x00400000u : (b == 255u ? 0x7FC00000u : (b << 23));
+    return __uint_as_float(bits);
+}
+
+// two FP32 -> one code byte: `lo` lands in the low nibble, `hi` in the high nibble.
+// Round to nearest even, magnitudes above 6 clamp to 6.
+__device__ __forceinline__ uint32_t float2_to_e2m1x2(float lo, float hi) {
+    uint32_t out;
+    asm("{\n\t.reg .b8 b;\n\tcvt.rn.satfinite.e2m1x2.f32 b, %1, %2;\n\tcvt.u32.u8 %0, b;\n\t}"
+        : "=r"(out)
+        : "f"(hi), "f"(lo));
+    return out;
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+}  // namespace mxq

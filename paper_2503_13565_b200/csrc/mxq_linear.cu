@@ -1,0 +1,137 @@
+// mxq_linear: Y[M,N] = X[M,K] . dequant(codes, scales)[N,K]^T  (Sec. III-D-3, Eq. 2).
+//
+// The weight stream (4.25 bits per weight) is the cost; X and Y are negligible.  Each warp
+// owns whole output rows, so no partial sums ever leave the warp and the summation order is
+// fixed.  Lanes walk the row's MX blocks with 16-byte loads (one load = one block of 32
+// weights = one scale byte), decode the E2M1 pairs in registers, accumulate the 32-long
+// partial sum in FP32 and apply the block scale once per block (the late scaling of Eq. 2).
+#include "mxq_device.cuh"
+#include "mxq_host.h"
+
+namespace mxq {
+
+constexpr int kRowWarpThreads = 256;
+constexpr int kRowWarpRows = kRowWarpThreads / 32;
+
+__device__ __forceinline__ void store_y(void *Y, int y_dtype, int64_t idx, float v) {
+    if (y_dtype == MXQ_F32)
+        reinterpret_cast<float *>(Y)[idx] = v;
+    else
+        reinterpret_cast<__nv_bfloat16 *>(Y)[idx] = __float2bfloat16_rn(v);
+}
+
+// Generic kernel: any M <= MT, any N, any K % 32 == 0.  One warp per output row.
+template <int MT>
+__global__ void __launch_bounds__(kRowWarpThreads)
+linear_rowwarp_kernel(const __nv_bfloat16 *__restrict__ X, int M, const uint4 *__restrict__ codes,
+                      const uint8_t *__restrict__ scales, int64_t N, int64_t K, void *__restrict__ Y, int y_dtype) {
+    pdl_trigger();
+    const int lane = threadIdx.x & 31;
+    const int64_t n = (int64_t)blockIdx.x * kRowWarpRows + (threadIdx.x >> 5);
+    if (n >= N) return;
+    const int64_t nblk = K / kBlock;
+    const uint4 *crow = codes + n * nblk;
+    const uint8_t *srow = scales + n * nblk;
+
+    float acc[MT];
+#pragma unroll
+    for (int m = 0; m < MT; ++m) acc[m] = 0.f;
+
+    pdl_wait();  // X may be the previous kernel's output
+    for (int64_t j = lane; j < nblk; j += 32) {
+        const uint4 c = ld_stream_u4(crow + j);
+        const float s = e8m0_to_float(srow[j]);
+        const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+        float part[MT];
+#pragma unroll
+        for (int m = 0; m < MT; ++m) part[m] = 0.f;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 wv = __half22float2(e2m1x2_to_half2((w[q] >> (8 * i)) & 0xFFu));
+                const int64_t k = j * kBlock + q * 8 + i * 2;
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    if (m < M) {
+                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * K + k);
+                        part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
+                        part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int m = 0; m < MT; ++m) acc[m] = fmaf(part[m], s, acc[m]);
+    }
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+        const float v = warp_sum(acc[m]);
+        if (lane == 0 && m < M) store_y(Y, y_dtype, (int64_t)m * N + n, v);
+    }
+}
+
+template <int MT>
+static void launch_rowwarp(const void *X, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
+                           void *Y, int y_dtype, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((N + kRowWarpRows - 1) / kRowWarpRows));
+    cfg.blockDim = dim3(kRowWarpThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, linear_rowwarp_kernel<MT>, (const __nv_bfloat16 *)X, M, (const uint4 *)codes, scales, N,
+                       K, Y, y_dtype);
+}
+
+}  // namespace mxq
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K) {
+    if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return 0;
+    return 0;
+}
+
+int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
+               void *Y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!X_bf16 || !codes || !scales || !Y) return MXQ_ERR_NULL;
+    if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return MXQ_ERR_SHAPE;
+    if (y_dtype != MXQ_F32 && y_dtype != MXQ_BF16) return MXQ_ERR_DTYPE;
+    if (!mxq::aligned16(X_bf16) || !mxq::aligned16(codes) || !mxq::aligned16(scales) || !mxq::aligned16(Y))
+        return MXQ_ERR_ALIGN;
+    const size_t need = mxq_linear_workspace_bytes(M, N, K);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return MXQ_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (M == 1) mxq::launch_rowwarp<1>(X_bf16, M, codes, scales, N, K, Y, y_dtype, st);
+    else if (M == 2) mxq::launch_rowwarp<2>(X_bf16, M, codes, scales, N, K, Y, y_dtype, st);
+    else if (M <= 4) mxq::launch_rowwarp<4>(X_bf16, M, codes, scales, N, K, Y, y_dtype, st);
+    else if (M <= 8) mxq::launch_rowwarp<8>(X_bf16, M, codes, scales, N, K, Y, y_dtype, st);
+    else mxq::launch_rowwarp<16>(X_bf16, M, codes, scales, N, K, Y, y_dtype, st);
+    return mxq::launch_status();
+}
+
+int mxq_linear_host(const void *X_host, int M, const uint8_t *codes, const uint8_t *scales, int64_t N,
+                    int64_t K, void *Y_host, int y_dtype, void *X_stage_dev, void *Y_stage_dev,
+                    void *workspace, size_t workspace_bytes, void *stream) {
+    if (!X_host || !Y_host || !X_stage_dev || !Y_stage_dev) return MXQ_ERR_NULL;
+    if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return MXQ_ERR_SHAPE;
+    if (y_dtype != MXQ_F32 && y_dtype != MXQ_BF16) return MXQ_ERR_DTYPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(X_stage_dev, X_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return MXQ_ERR_CUDA;
+    const int rc = mxq_linear(X_stage_dev, M, codes, scales, N, K, Y_stage_dev, y_dtype, workspace, workspace_bytes,
+                              stream);
+    if (rc != MXQ_OK) return rc;
+    const size_t ybytes = (size_t)M * N * (y_dtype == MXQ_F32 ? 4 : 2);
+    if (cudaMemcpyAsync(Y_host, Y_stage_dev, ybytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MXQ_ERR_CUDA;
+    return MXQ_OK;
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

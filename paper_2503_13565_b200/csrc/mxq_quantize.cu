@@ -1,0 +1,129 @@
+// mxq_quantize / mxq_dequantize: the direct cast BF16 -> MXFP4 of Sec. III-D-3 and its
+// exact inverse map.
+//
+// Data movement is the whole cost: 2 bytes read and 0.53125 bytes written per weight, so
+// the kernel is a pure HBM stream.  Because K is a multiple of 32, MX blocks never straddle
+// a row and the three tensors can be walked as flat arrays: 16-byte chunk i of W (8 BF16)
+// becomes 32-bit word i of codes, and four consecutive chunks (one quad of lanes) share
+// scale byte i/4.  Every lane issues its 16-byte loads up front; the quad agrees on the
+// block maximum with two shuffles.
+#include "mxq_device.cuh"
+#include "mxq_host.h"
+
+namespace mxq {
+
+constexpr int kQuantThreads = 256;
+constexpr int kQuantUnroll = 4;  // 16-byte loads in flight per lane
+
+// Cast the 8 BF16 values of one chunk given the block's scale byte; returns 8 packed codes.
+__device__ __forceinline__ uint32_t cast_chunk(const uint4 &v, uint32_t scale_byte) {
+    // v / X with X = 2^(byte-127): multiply by 2^(127-byte), exact (a power of two; results
+    // stay below 8, and anything that underflows is far below the first rounding boundary).
+    const float inv_x = __uint_as_float((254u - scale_byte) << 23);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t out = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float lo = __uint_as_float((w[j] & 0x7FFFu) << 16) * inv_x;     // |element 2j|
+        const float hi = __uint_as_float(w[j] & 0x7FFF0000u) * inv_x;         // |element 2j+1|
+        uint32_t c = float2_to_e2m1x2(lo, hi);                                 // round-to-nearest-even, clamp
+        c |= ((w[j] >> 12) & 0x8u) | ((w[j] >> 24) & 0x80u);                   // input sign bits, always kept
+        out |= c << (8 * j);
+    }
+    return out;
+}
+
+__global__ void __launch_bounds__(kQuantThreads)
+quantize_kernel(const uint4 *__restrict__ W, uint32_t *__restrict__ codes, uint8_t *__restrict__ scales,
+                uint32_t *__restrict__ nonfinite_blocks, int64_t nchunks, int64_t iters) {
+    const int64_t stride = (int64_t)gridDim.x * kQuantThreads;
+    const int64_t tid = (int64_t)blockIdx.x * kQuantThreads + threadIdx.x;
+    for (int64_t it = 0; it < iters; ++it) {  // same trip count in every lane: shuffles below use the full mask
+        uint4 v[kQuantUnroll];
+        int64_t idx[kQuantUnroll];
+#pragma unroll
+        for (int u = 0; u < kQuantUnroll; ++u) {
+            idx[u] = (it * kQuantUnroll + u) * stride + tid;
+            v[u] = (idx[u] < nchunks) ? ld_stream_u4(W + idx[u]) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < kQuantUnroll; ++u) {
+            // block maximum: for finite BF16 the magnitude bits order like the values
+            uint32_t a = max(max(v[u].x & 0x7FFFu, (v[u].x >> 16) & 0x7FFFu), max(v[u].y & 0x7FFFu, (v[u].y >> 16) & 0x7FFFu));
+            a = max(a, max(max(v[u].z & 0x7FFFu, (v[u].z >> 16) & 0x7FFFu), max(v[u].w & 0x7FFFu, (v[u].w >> 16) & 0x7FFFu)));
+            a = max(a, __shfl_xor_sync(0xffffffffu, a, 1));
+            a = max(a, __shfl_xor_sync(0xffffffffu, a, 2));
+            const uint32_t efield = a >> 7;               // biased exponent of the block maximum
+            const bool nonfinite = efield == 0xFFu;       // Inf/NaN sort above every finite pattern
+            // floor(log2 max) - 2 + 127 = efield - 2; clamped at 0 (also covers subnormal and zero maxima)
+            const uint32_t byte = nonfinite ? 0xFFu : (efield > 2u ? efield - 2u : 0u);
+            if (idx[u] < nchunks) {
+                codes[idx[u]] = nonfinite ? 0u : cast_chunk(v[u], byte);
+                if ((idx[u] & 3) == 0) {
+                    scales[idx[u] >> 2] = (uint8_t)byte;
+                    if (nonfinite && nonfinite_blocks != nullptr) atomicAdd(nonfinite_blocks, 1u);
+                }
+            }
+        }
+    }
+}
+
+// One lane per MX block: 16 code bytes + 1 scale byte -> 32 BF16 values.
+__global__ void __launch_bounds__(256)
+dequantize_kernel(const uint4 *__restrict__ codes, const uint8_t *__restrict__ scales, uint4 *__restrict__ W,
+                  int64_t nblocks) {
+    const int64_t b = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (b >= nblocks) return;
+    const uint4 c = codes[b];
+    const float s = e8m0_to_float(scales[b]);
+    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        uint32_t o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __half22float2(e2m1x2_to_half2((w[j] >> (8 * i)) & 0xFFu));
+            // value * 2^(b-127) has at most two significant bits: the FP32 product is exact and its
+            // upper 16 bits are the BF16 number (subnormal results included)
+            o[i] = (__float_as_uint(f.x * s) >> 16) | (__float_as_uint(f.y * s) & 0xFFFF0000u);
+        }
+        W[b * 4 + j] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+}  // namespace mxq
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+int mxq_quantize(const void *W_bf16, int64_t N, int64_t K, uint8_t *codes, uint8_t *scales,
+                 uint32_t *nonfinite_blocks, void *stream) {
+    if (!W_bf16 || !codes || !scales) return MXQ_ERR_NULL;
+    if (!mxq::shape_ok(N, K)) return MXQ_ERR_SHAPE;
+    if (!mxq::aligned16(W_bf16) || !mxq::aligned16(codes) || !mxq::aligned16(scales)) return MXQ_ERR_ALIGN;
+    if (nonfinite_blocks && (reinterpret_cast<uintptr_t>(nonfinite_blocks) & 3u)) return MXQ_ERR_ALIGN;
+    const int64_t nchunks = N * K / 8;
+    const int64_t per_pass = (int64_t)mxq::kQuantThreads * mxq::kQuantUnroll;
+    int64_t grid = (nchunks + per_pass - 1) / per_pass;
+    const int64_t cap = (int64_t)mxq::sm_count() * 8;  // 8 resident CTAs of 256 lanes per SM
+    if (grid > cap) grid = cap;
+    const int64_t iters = (nchunks + grid * per_pass - 1) / (grid * per_pass);
+    mxq::quantize_kernel<<<(unsigned)grid, mxq::kQuantThreads, 0, (cudaStream_t)stream>>>(
+        (const uint4 *)W_bf16, (uint32_t *)codes, scales, nonfinite_blocks, nchunks, iters);
+    return mxq::launch_status();
+}
+
+int mxq_dequantize(const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K, void *W_bf16_out,
+                   void *stream) {
+    if (!codes || !scales || !W_bf16_out) return MXQ_ERR_NULL;
+    if (!mxq::shape_ok(N, K)) return MXQ_ERR_SHAPE;
+    if (!mxq::aligned16(codes) || !mxq::aligned16(scales) || !mxq::aligned16(W_bf16_out)) return MXQ_ERR_ALIGN;
+    const int64_t nblocks = N * K / 32;
+    const int64_t grid = (nblocks + 255) / 256;
+    mxq::dequantize_kernel<<<(unsigned)grid, 256, 0, (cudaStream_t)stream>>>((const uint4 *)codes, scales,
+                                                                             (uint4 *)W_bf16_out, nblocks);
+    return mxq::launch_status();
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

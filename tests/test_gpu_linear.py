@@ -1,0 +1,172 @@
+"""GPU parity of mxq_linear against the oracle: |y - y64| <= 2e-3 * sum|x w^| + 1e-6 element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2503_13565_b200 as mxq
+from golden_io import direct_cast_blocks, linear_block_a
+from paper_2503_13565_b200 import synth
+from parity import check_linear, gpu_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def run_case(wbits, xbits, out_dtype=torch.float32, rows=None, what=""):
+    """Quantise on the oracle side, run the layer on both sides from the same bytes."""
+    codes, scales, _ = oracle.quantize(wbits)
+    y64, a64 = oracle.linear(xbits, codes, scales, rows=rows)
+    n, k = wbits.shape
+    m = xbits.shape[0]
+    ws = mxq.new_workspace(mxq.mxq_linear_workspace_bytes(m, n, k))
+    y = mxq.mxq_linear(gpu_bf16(xbits), torch.from_numpy(codes).cuda(), torch.from_numpy(scales).cuda(),
+                       out_dtype=out_dtype, workspace=ws)
+    torch.cuda.synchronize()
+    if rows is not None:
+        y = y[:, torch.as_tensor(rows, device="cuda")]
+    return check_linear(y, y64, a64, what), y
+
+
+def test_config1_tiny():
+    w = synth.bits_of(synth.weight(1, 0, 512, 256))
+    x = synth.bits_of(synth.activations(1, 0, 1, 256))
+    run_case(w, x, what="config1")
+
+
+@pytest.mark.parametrize("m", [1, 4])
+@pytest.mark.parametrize("idx,n,k", [(0, 768, 768), (4, 3072, 768), (6, 768, 3072), (7, 32000, 768)])
+def test_config2_small_draft(idx, n, k, m):
+    w = synth.bits_of(synth.weight(2, idx, n, k))
+    x = synth.bits_of(synth.activations(2, idx, m, k))
+    run_case(w, x, what="config2 %dx%d M=%d" % (n, k, m))
+
+
+@pytest.mark.parametrize("m", [1, 8])
+@pytest.mark.parametrize("idx,n,k", [(0, 4096, 4096), (4, 11008, 4096), (6, 4096, 11008)])
+def test_config3_7b_layers_sampled_rows(idx, n, k, m):
+    """Full-size layers in the launch configuration the benchmark times; the oracle checks a seeded
+    sample of output rows (first, last, and rows spread over every tile)."""
+    w = synth.bits_of(synth.weight(3, idx, n, k))
+    x = synth.bits_of(synth.activations(3, idx, m, k))
+    rng = np.random.default_rng(idx)
+    rows = np.unique(np.concatenate([[0, 1, n - 1, n - 2], rng.integers(0, n, 700)])).astype(np.int64)
+    run_case(w, x, rows=rows, what="config3 %dx%d M=%d" % (n, k, m))
+
+
+@pytest.mark.parametrize("m", [1, 2, 3, 4, 5, 7, 8, 9, 12, 15, 16])
+def test_every_token_count_on_a_ragged_shape(m):
+    n, k = 203, 1440   # N not a multiple of any tile, K = 45 blocks
+    w = synth.bits_of(synth.weight(3, 10, n, k))
+    x = synth.bits_of(synth.activations(3, 10, m, k))
+    run_case(w, x, what="ragged M=%d" % m)
+
+
+@pytest.mark.parametrize("n,k", [(1, 32), (2, 64), (7, 32), (9, 4096), (300, 96), (16, 13824), (129, 5120)])
+@pytest.mark.parametrize("m", [1, 3, 16])
+def test_small_and_extreme_shapes(n, k, m):
+    w = synth.bits_of(synth.weight(5, 2, n, k))
+    x = synth.bits_of(synth.activations(5, 2, m, k))
+    run_case(w, x, what="%dx%d M=%d" % (n, k, m))
+
+
+@pytest.mark.parametrize("m", [1, 2, 4, 8, 16])
+def test_config4_lm_head_sampled_rows(m):
+    n, k = 32000, 4096
+    w = synth.bits_of(synth.weight(4, 0, n, k))
+    x = synth.bits_of(synth.activations(4, 0, m, k))
+    rows = np.unique(np.concatenate([[0, n - 1], np.random.default_rng(4).integers(0, n, 300)])).astype(np.int64)
+    run_case(w, x, rows=rows, what="lm_head M=%d" % m)
+
+
+def test_bf16_output_is_the_rounded_fp32_output():
+    w = synth.bits_of(synth.weight(3, 11, 515, 2048))
+    x = synth.bits_of(synth.activations(3, 11, 5, 2048))
+    _, y32 = run_case(w, x, torch.float32, what="fp32 out")
+    _, y16 = run_case(w, x, torch.bfloat16, what="bf16 out")
+    assert torch.equal(y16, y32.to(torch.bfloat16))   # round to nearest even of the same FP32 sums
+
+
+def test_results_are_bit_reproducible():
+    w = synth.bits_of(synth.weight(3, 12, 1000, 4096))
+    for m in (1, 8):
+        x = synth.bits_of(synth.activations(3, 12, m, 4096))
+        _, y1 = run_case(w, x)
+        _, y2 = run_case(w, x)
+        assert torch.equal(y1, y2)
+
+
+def test_hand_block_a():
+    blk = [b for b in direct_cast_blocks() if b["name"] == "A"][0]
+    fx = linear_block_a()
+    x = np.zeros((1, 32), np.float32)
+    x[0, : len(fx["x"])] = fx["x"]
+    xbits = (x.view(np.uint32) >> 16).astype(np.uint16)
+    gc, gs = mxq.mxq_quantize(gpu_bf16(blk["bits"].reshape(1, 32)))
+    y = mxq.mxq_linear(gpu_bf16(xbits), gc, gs)
+    assert float(y[0, 0]) == fx["y"][0]   # every partial sum here is exact in FP32
+
+
+def test_all_codes_under_extreme_scales():
+    """Every code next to every scale byte the cast can produce (0..252), in one matrix; X picks out
+    single weights so each output is one product."""
+    n = 253
+    codes = np.zeros((n, 16), np.uint8)
+    for j in range(8):
+        codes[:, j] = (2 * j) | ((2 * j + 1) << 4)
+    scales = np.arange(n, dtype=np.uint8).reshape(n, 1)
+    xs = np.zeros((16, 32), np.float32)
+    xs[np.arange(16), np.arange(16)] = 1.0
+    xbits = (xs.view(np.uint32) >> 16).astype(np.uint16)
+    y64, a64 = oracle.linear(xbits, codes, scales)
+    y = mxq.mxq_linear(gpu_bf16(xbits), torch.from_numpy(codes).cuda(), torch.from_numpy(scales).cuda())
+    got = y.cpu().numpy().astype(np.float64)
+    assert np.array_equal(got, y64)      # single exact products, FP32-representable: no tolerance needed
+
+
+def test_nan_scale_gives_nan_row_only():
+    w = synth.bits_of(synth.weight(1, 0, 64, 256))
+    codes, scales, _ = oracle.quantize(w)
+    scales[5, 3] = 0xFF
+    x = synth.bits_of(synth.activations(1, 0, 2, 256))
+    y64, a64 = oracle.linear(x, codes, scales)
+    y = mxq.mxq_linear(gpu_bf16(x), torch.from_numpy(codes).cuda(), torch.from_numpy(scales).cuda())
+    check_linear(y, y64, a64, "nan scale")
+    assert torch.isnan(y[:, 5]).all() and torch.isfinite(y[:, :5]).all()
+
+
+def test_wide_range_activations():
+    """Activations spanning many binades, including BF16 subnormals and zeros."""
+    rng = np.random.default_rng(7)
+    n, k, m = 130, 1024, 6
+    w = synth.bits_of(synth.weight(3, 13, n, k))
+    x = rng.standard_normal((m, k)) * np.exp2(rng.integers(-40, 30, (m, k)))
+    x[0, ::3] = 0
+    xbits = (x.astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    xbits[1, :64] = (rng.integers(1, 128, 64) | (rng.integers(0, 2, 64) << 15)).astype(np.uint16)  # subnormals
+    run_case(w, xbits, what="wide range")
+
+
+def test_host_variant_matches_device_variant():
+    n, k, m = 768, 3072, 4
+    w = synth.bits_of(synth.weight(2, 6, n, k))
+    gc, gs = mxq.mxq_quantize(gpu_bf16(w))
+    x = synth.activations(2, 6, m, k)
+    y_dev = mxq.mxq_linear(x.cuda(), gc, gs)
+    xh = x.pin_memory()
+    yh = torch.empty((m, n), dtype=torch.float32).pin_memory()
+    mxq.mxq_linear_host(xh, gc, gs, yh, torch.empty_like(x, device="cuda"),
+                        torch.empty((m, n), dtype=torch.float32, device="cuda"))
+    torch.cuda.synchronize()
+    assert torch.equal(yh, y_dev.cpu())
+
+
+def test_canaries_around_the_output_survive():
+    n, k, m = 203, 1440, 3
+    w = synth.bits_of(synth.weight(3, 10, n, k))
+    gc, gs = mxq.mxq_quantize(gpu_bf16(w))
+    x = synth.activations(3, 10, m, k).cuda()
+    buf = torch.full((m * n + 64,), 12345.0, dtype=torch.float32, device="cuda")
+    out = buf[32: 32 + m * n].view(m, n)
+    mxq.mxq_linear(x, gc, gs, out=out)
+    torch.cuda.synchronize()
+    assert (buf[:32] == 12345.0).all() and (buf[32 + m * n:] == 12345.0).all()

@@ -94,6 +94,13 @@ int mxq_dequantize(const uint8_t *codes, const uint8_t *scales, int64_t N, int64
  * (of any shape).  Two calls that may run concurrently need separate workspaces. */
 size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K);
 
+/* How mxq_linear will run this shape on the current device (diagnostics; launches nothing).
+ * info[12] int32: [0] 1 = tensor-core stream-K kernel, 0 = generic kernel; [1] CTAs;
+ * [2] ring stages; [3] K windows; [4] blocks per window; [5] blocks in the last window;
+ * [6] partial slots per CTA; [7] dynamic shared memory bytes; [8] 16-row tiles; [9] K/32;
+ * [10] 8-token column tiles; [11] work units (tiles * K/32).  Unused entries are 0. */
+int mxq_linear_plan_info(int M, int64_t N, int64_t K, int32_t *info);
+
 /* Weight-only-quantised linear layer (the MXFP4 GEMM of Sec. III-D-3, Eq. 2):
  *     Y[m][n] = sum_k X[m][k] * w^[n][k],   1 <= M <= 16 token rows.
  *   X_bf16  [M][K] BF16 row-major (read)

@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
             L.mxq_dequantize.argtypes = [vp, vp, i64, i64, vp, vp]
             L.mxq_linear.restype = i32
             L.mxq_linear.argtypes = [vp, i32, vp, vp, i64, i64, vp, i32, vp, sz, vp]
+            L.mxq_linear_plan_info.restype = i32
+            L.mxq_linear_plan_info.argtypes = [i32, i64, i64, vp]
             L.mxq_linear_host.restype = i32
             L.mxq_linear_host.argtypes = [vp, i32, vp, vp, i64, i64, vp, i32, vp, vp, vp, sz, vp]
             L.mxq_greedy_accept.restype = i32
@@ -119,8 +121,31 @@ def mxq_linear_workspace_bytes(m: int, n: int, k: int) -> int:
     return int(lib().mxq_linear_workspace_bytes(m, n, k))
 
 
+def mxq_linear_plan_info(m: int, n: int, k: int) -> dict:
+    """How mxq_linear will run this shape (diagnostics)."""
+    info = (ctypes.c_int32 * 12)()
+    _check(lib().mxq_linear_plan_info(m, n, k, ctypes.cast(info, ctypes.c_void_p)), "mxq_linear_plan_info")
+    keys = ("tensor_core", "grid", "stages", "windows", "bw", "bw_last", "slots", "smem_bytes", "tiles", "kb", "nt8",
+            "units")
+    return dict(zip(keys, [int(v) for v in info]))
+
+
 def mxq_accept_workspace_bytes(b: int, r: int, v: int) -> int:
     return int(lib().mxq_accept_workspace_bytes(b, r, v))
+
+
+_default_ws = {}
+
+
+def _default_workspace(nbytes: int, device) -> torch.Tensor:
+    """A cached, zero-initialised workspace per device for callers that pass none."""
+    key = (torch.device(device).type, torch.device(device).index if torch.device(device).index is not None
+           else torch.cuda.current_device())
+    ws = _default_ws.get(key)
+    if ws is None or ws.numel() < nbytes:
+        ws = new_workspace(nbytes, device)
+        _default_ws[key] = ws
+    return ws
 
 
 def new_workspace(nbytes: int, device="cuda") -> torch.Tensor:
@@ -160,6 +185,9 @@ def mxq_linear(x: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, out: 
         raise ValueError("shape mismatch between X, codes and scales")
     if out is None:
         out = torch.empty((m, n), dtype=out_dtype, device=x.device)
+    if workspace is None:
+        need = mxq_linear_workspace_bytes(m, n, k)
+        workspace = _default_workspace(need, x.device) if need else None
     ws_ptr, ws_bytes = (0, 0) if workspace is None else (_dev(workspace, torch.uint8, "workspace"), workspace.numel())
     _check(lib().mxq_linear(_dev(x, torch.bfloat16, "X"), m, _dev(codes, torch.uint8, "codes"),
                             _dev(scales, torch.uint8, "scales"), n, k, _dev(out, out.dtype, "Y"), _dt(out.dtype),
@@ -178,6 +206,9 @@ def mxq_linear_host(x_host: torch.Tensor, codes: torch.Tensor, scales: torch.Ten
     if x_stage.numel() * x_stage.element_size() < m * k * 2 or \
             y_stage.numel() * y_stage.element_size() < m * n * y_host.element_size():
         raise ValueError("staging buffers too small")
+    if workspace is None:
+        need = mxq_linear_workspace_bytes(m, n, k)
+        workspace = _default_workspace(need, codes.device) if need else None
     ws_ptr, ws_bytes = (0, 0) if workspace is None else (_dev(workspace, torch.uint8, "workspace"), workspace.numel())
     _check(lib().mxq_linear_host(x_host.data_ptr(), m, _dev(codes, torch.uint8, "codes"),
                                  _dev(scales, torch.uint8, "scales"), n, k, y_host.data_ptr(), _dt(y_host.dtype),

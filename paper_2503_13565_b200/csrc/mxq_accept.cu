@@ -16,6 +16,7 @@ namespace mxq {
 constexpr int kAcceptThreads = 256;
 constexpr int64_t kSliceQuantum = 2048;  // slice lengths are multiples of this many logits
 constexpr int64_t kTargetCtas = 592;     // 4 per SM on a 148-SM part
+constexpr int kTickets = 1024;           // ticket counters live in a fixed region: sequence b uses ticket b % kTickets
 
 struct Best {
     float v;
@@ -53,7 +54,7 @@ static Slicing slicing_for(int64_t B, int R, int64_t V) {
     return s;
 }
 
-static size_t ticket_bytes(int64_t B) { return ((size_t)B * sizeof(unsigned) + 15) / 16 * 16; }
+static size_t ticket_bytes() { return (size_t)kTickets * sizeof(unsigned); }
 
 template <typename T>
 __device__ __forceinline__ float logit_value(T x);
@@ -65,7 +66,7 @@ __device__ __forceinline__ float logit_value<uint16_t>(uint16_t x) { return bf16
 // T = float or uint16_t (BF16 bits).  grid.x = B * R * slices.
 template <typename T>
 __global__ void __launch_bounds__(kAcceptThreads)
-greedy_accept_kernel(const T *__restrict__ logits, int R, int64_t V, int slices, int64_t slice_len, bool vec_ok,
+greedy_accept_kernel(const T *__restrict__ logits, int64_t B, int R, int64_t V, int slices, int64_t slice_len, bool vec_ok,
                      const int32_t *__restrict__ draft, int Tn, int32_t *__restrict__ accept_len,
                      int32_t *__restrict__ next_token, Best *__restrict__ partial, unsigned *__restrict__ tickets) {
     constexpr int kVec = 16 / sizeof(T);
@@ -120,38 +121,44 @@ greedy_accept_kernel(const T *__restrict__ logits, int R, int64_t V, int slices,
         for (int w = 1; w < kAcceptThreads / 32; ++w) best = better(best, warp_best[w]);
         partial[row * slices + slice] = best;
         __threadfence();
-        const unsigned arrived = atomicAdd(&tickets[b], 1u);
-        is_last = arrived == (unsigned)(R * slices) - 1u;
+        // sequences b, b + kTickets, ... share a counter; whoever arrives last finishes all of them
+        const int64_t group = b % kTickets;
+        const int64_t members = (B - group + kTickets - 1) / kTickets;
+        const unsigned arrived = atomicAdd(&tickets[group], 1u);
+        is_last = arrived == (unsigned)(members * R * slices) - 1u;
     }
     __syncthreads();
     if (!is_last) return;
 
-    // last CTA of sequence b: every slice of every row of b has been published
+    // every slice of every row of this group of sequences has been published
     __threadfence();
-    if (threadIdx.x < R) {
-        const Best *pr = partial + (b * R + threadIdx.x) * slices;
-        Best r = {-INFINITY, INT_MAX};
-        for (int s = 0; s < slices; ++s) {
-            Best q;
-            q.v = __ldcg(&pr[s].v);
-            q.idx = __ldcg(&pr[s].idx);
-            r = better(r, q);
-        }
-        verifier[threadIdx.x] = (r.idx == INT_MAX) ? 0 : r.idx;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int G = Tn;
-        for (int i = 0; i < Tn; ++i) {
-            if (i >= R || draft[b * Tn + i] != verifier[i]) {
-                G = i;
-                break;
+    for (int64_t bb = b % kTickets; bb < B; bb += kTickets) {
+        if (threadIdx.x < R) {
+            const Best *pr = partial + (bb * R + threadIdx.x) * slices;
+            Best r = {-INFINITY, INT_MAX};
+            for (int s = 0; s < slices; ++s) {
+                Best q;
+                q.v = __ldcg(&pr[s].v);
+                q.idx = __ldcg(&pr[s].idx);
+                r = better(r, q);
             }
+            verifier[threadIdx.x] = (r.idx == INT_MAX) ? 0 : r.idx;
         }
-        accept_len[b] = G;
-        next_token[b] = (G < R) ? verifier[G] : -1;
-        tickets[b] = 0;  // ready for the next call
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int G = Tn;
+            for (int i = 0; i < Tn; ++i) {
+                if (i >= R || draft[bb * Tn + i] != verifier[i]) {
+                    G = i;
+                    break;
+                }
+            }
+            accept_len[bb] = G;
+            next_token[bb] = (G < R) ? verifier[G] : -1;
+        }
+        __syncthreads();
     }
+    if (threadIdx.x == 0) tickets[b % kTickets] = 0;  // ready for the next call
 }
 
 __global__ void accept_tokens_kernel(const int32_t *__restrict__ draft, const int32_t *__restrict__ verifier, int64_t B,
@@ -182,7 +189,7 @@ extern "C" {
 size_t mxq_accept_workspace_bytes(int64_t B, int R, int64_t V) {
     if (B < 1 || R < 1 || R > MXQ_MAX_T + 1 || V < 1) return 0;
     const mxq::Slicing s = mxq::slicing_for(B, R, V);
-    return mxq::ticket_bytes(B) + (size_t)B * R * s.slices * sizeof(mxq::Best);
+    return mxq::ticket_bytes() + (size_t)B * R * s.slices * sizeof(mxq::Best);
 }
 
 int mxq_greedy_accept(const void *logits, int logits_dtype, int64_t B, int R, int64_t V, const int32_t *draft,
@@ -195,17 +202,17 @@ int mxq_greedy_accept(const void *logits, int logits_dtype, int64_t B, int R, in
     if (!workspace || workspace_bytes < mxq_accept_workspace_bytes(B, R, V)) return MXQ_ERR_WORKSPACE;
     const mxq::Slicing s = mxq::slicing_for(B, R, V);
     unsigned *tickets = (unsigned *)workspace;
-    mxq::Best *partial = (mxq::Best *)((char *)workspace + mxq::ticket_bytes(B));
+    mxq::Best *partial = (mxq::Best *)((char *)workspace + mxq::ticket_bytes());
     const unsigned grid = (unsigned)(B * R * s.slices);
     cudaStream_t st = (cudaStream_t)stream;
     if (logits_dtype == MXQ_F32) {
         const bool vec_ok = (V % 4) == 0;
         mxq::greedy_accept_kernel<float><<<grid, mxq::kAcceptThreads, 0, st>>>(
-            (const float *)logits, R, V, s.slices, s.slice_len, vec_ok, draft, T, accept_len, next_token, partial, tickets);
+            (const float *)logits, B, R, V, s.slices, s.slice_len, vec_ok, draft, T, accept_len, next_token, partial, tickets);
     } else {
         const bool vec_ok = (V % 8) == 0;
         mxq::greedy_accept_kernel<uint16_t><<<grid, mxq::kAcceptThreads, 0, st>>>(
-            (const uint16_t *)logits, R, V, s.slices, s.slice_len, vec_ok, draft, T, accept_len, next_token, partial,
+            (const uint16_t *)logits, B, R, V, s.slices, s.slice_len, vec_ok, draft, T, accept_len, next_token, partial,
             tickets);
     }
     return mxq::launch_status();

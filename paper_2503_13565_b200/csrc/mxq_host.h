@@ -16,4 +16,11 @@ int sm_count();
 // whether mxq_linear launches carry the programmatic-dependent-launch attribute
 bool pdl_enabled();
 
+struct LinearPlan;
+// tensor-core path of mxq_linear (mxq_linear_mma.cu): false if the shape is not covered
+bool linear_mma_plan(int M, int64_t N, int64_t K, LinearPlan &plan);
+size_t linear_mma_workspace_bytes(const LinearPlan &plan);
+cudaError_t linear_mma_launch(const LinearPlan &plan, const void *X, const uint8_t *codes, const uint8_t *scales,
+                              void *Y, int y_dtype, void *workspace, cudaStream_t stream);
+
 }  // namespace mxq

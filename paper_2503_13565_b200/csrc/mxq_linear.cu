@@ -1,12 +1,20 @@
 // mxq_linear: Y[M,N] = X[M,K] . dequant(codes, scales)[N,K]^T  (Sec. III-D-3, Eq. 2).
 //
-// The weight stream (4.25 bits per weight) is the cost; X and Y are negligible.  Each warp
+// This file holds the entry points, the dispatch and the generic kernel.  Shapes with
+// K % 128 == 0 go to the tensor-core kernel in mxq_linear_mma.cu; everything else (and
+// MXQ_LINEAR_VARIANT=generic in the environment) runs the generic kernel below.
+//
+// Generic kernel: the weight stream (4.25 bits per weight) is the cost; X and Y are negligible.  Each warp
 // owns whole output rows, so no partial sums ever leave the warp and the summation order is
 // fixed.  Lanes walk the row's MX blocks with 16-byte loads (one load = one block of 32
 // weights = one scale byte), decode the E2M1 pairs in registers, accumulate the 32-long
 // partial sum in FP32 and apply the block scale once per block (the late scaling of Eq. 2).
+#include <cstdlib>
+#include <cstring>
+
 #include "mxq_device.cuh"
 #include "mxq_host.h"
+#include "mxq_linear_plan.h"
 
 namespace mxq {
 
@@ -88,6 +96,15 @@ static void launch_rowwarp(const void *X, int M, const uint8_t *codes, const uin
                        K, Y, y_dtype);
 }
 
+// MXQ_LINEAR_VARIANT=generic forces the generic kernel (for tests and comparisons)
+static bool force_generic() {
+    static const int v = [] {
+        const char *e = std::getenv("MXQ_LINEAR_VARIANT");
+        return (e && std::strcmp(e, "generic") == 0) ? 1 : 0;
+    }();
+    return v != 0;
+}
+
 }  // namespace mxq
 
 extern "C" {
@@ -95,7 +112,34 @@ extern "C" {
 
 size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K) {
     if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return 0;
+    mxq::LinearPlan plan;
+    if (!mxq::force_generic() && mxq::linear_mma_plan(M, N, K, plan)) return mxq::linear_mma_workspace_bytes(plan);
     return 0;
+}
+
+int mxq_linear_plan_info(int M, int64_t N, int64_t K, int32_t *info) {
+    if (!info) return MXQ_ERR_NULL;
+    if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return MXQ_ERR_SHAPE;
+    mxq::LinearPlan p;
+    const bool mma = !mxq::force_generic() && mxq::linear_mma_plan(M, N, K, p);
+    for (int i = 0; i < 12; ++i) info[i] = 0;
+    info[0] = mma ? 1 : 0;
+    if (mma) {
+        info[1] = p.grid;
+        info[2] = p.nstage;
+        info[3] = p.nwin;
+        info[4] = p.bw;
+        info[5] = p.bw_last;
+        info[6] = p.slots;
+        info[7] = (int32_t)p.smem_bytes;
+        info[8] = p.tiles;
+        info[9] = p.kb;
+        info[10] = p.nt8;
+        info[11] = (int32_t)p.units;
+    } else {
+        info[1] = (int32_t)((N + mxq::kRowWarpRows - 1) / mxq::kRowWarpRows);
+    }
+    return MXQ_OK;
 }
 
 int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
@@ -105,9 +149,17 @@ int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *s
     if (y_dtype != MXQ_F32 && y_dtype != MXQ_BF16) return MXQ_ERR_DTYPE;
     if (!mxq::aligned16(X_bf16) || !mxq::aligned16(codes) || !mxq::aligned16(scales) || !mxq::aligned16(Y))
         return MXQ_ERR_ALIGN;
-    const size_t need = mxq_linear_workspace_bytes(M, N, K);
-    if (need > 0 && (!workspace || workspace_bytes < need)) return MXQ_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    mxq::LinearPlan plan;
+    if (!mxq::force_generic() && mxq::linear_mma_plan(M, N, K, plan)) {
+        if (!workspace || workspace_bytes < mxq::linear_mma_workspace_bytes(plan)) return MXQ_ERR_WORKSPACE;
+        if (!mxq::aligned16(workspace)) return MXQ_ERR_ALIGN;
+        if (mxq::linear_mma_launch(plan, X_bf16, codes, scales, Y, y_dtype, workspace, st) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return MXQ_ERR_CUDA;
+        }
+        return mxq::launch_status();
+    }
     if (M == 1) mxq::launch_rowwarp<1>(X_bf16, M, codes, scales, N, K, Y, y_dtype, st);
     else if (M == 2) mxq::launch_rowwarp<2>(X_bf16, M, codes, scales, N, K, Y, y_dtype, st);
     else if (M <= 4) mxq::launch_rowwarp<4>(X_bf16, M, codes, scales, N, K, Y, y_dtype, st);

@@ -1,0 +1,495 @@
+// Tensor-core mxq_linear for sm_100a: Y[M,N] = X[M,K] . dequant(codes, scales)^T, M <= 16
+// (the MXFP4 GEMM of Sec. III-D-3 with the late scaling of Eq. 2).
+//
+// Why tensor cores for a mat-vec: the weight stream delivers ~42 weights per clock per SM at
+// HBM speed, and every way of turning a 4-bit code into an FP32 operand on the CUDA cores
+// costs 2.5+ issue slots per weight (measured: conversion and logic pipes run at 64 lanes/clk).
+// cvt.rn.f16x2.e2m1x2 decodes two weights per instruction, exactly, and mma.sync takes the
+// FP16 pairs as they come; the multiply-accumulate then costs almost nothing for any M <= 8.
+//
+// Exactness: every E2M1 value is an FP16 number.  X is BF16; each CTA rescales its slice of X
+// by a power of two (per token row) so that the largest magnitude sits just below 2^15 and
+// converts it to FP16, checking every element converts exactly (true whenever an element is
+// within 2^32 of its row maximum).  Products FP16 x FP16 are exact in the FP32 accumulator.
+// If any element does not convert exactly the CTA takes a scalar FP32 path instead, so the
+// result never depends on the shortcut.
+//
+// Decomposition (stream-K): the matrix is cut into units of 16 rows x 32 k (one MX block per
+// row), ordered window-major / tile / k.  Each CTA owns an equal, contiguous range of units,
+// so all SMs stream the same number of bytes whatever N is.  Within a CTA, 16 warps split each
+// stage's 64 blocks; their FP32 partial tiles are summed in a fixed order through shared
+// memory.  A tile whose K range is shared between CTAs goes through a workspace slot and a
+// ticket counter; the CTA that completes the tile sums the slots in unit order.  Nobody waits
+// for anybody, and the summation order is fixed, so results are bit-reproducible.
+//
+// Pipeline: every warp runs its own ring of 16-byte cp.async copies for exactly the bytes it
+// will consume (16 rows x 64 code bytes + 16 x 4 scale bytes per stage), so the main loop has
+// no CTA-wide barrier and no spin-wait.  Weights never depend on the previous kernel, so the
+// ring is filled before griddepcontrol.wait (programmatic dependent launch); X, Y and the
+// workspace are touched only after it.  A CTA uses at most half an SM so that the next
+// kernel's CTAs can be resident and prefetching while this one computes.
+#include "mxq_device.cuh"
+#include "mxq_host.h"
+#include "mxq_linear_plan.h"
+
+namespace mxq {
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+// four code bytes -> four FP16 pairs (low nibble in the low half)
+__device__ __forceinline__ void e2m1x8_to_half2x4(uint32_t word, uint32_t &p0, uint32_t &p1, uint32_t &p2, uint32_t &p3) {
+    asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\tmov.b32 {b0, b1, b2, b3}, %4;\n\t"
+        "cvt.rn.f16x2.e2m1x2 %0, b0;\n\tcvt.rn.f16x2.e2m1x2 %1, b1;\n\t"
+        "cvt.rn.f16x2.e2m1x2 %2, b2;\n\tcvt.rn.f16x2.e2m1x2 %3, b3;\n\t}"
+        : "=r"(p0), "=r"(p1), "=r"(p2), "=r"(p3)
+        : "r"(word));
+}
+// two E8M0 bytes (low 16 bits of v) -> BF16 pair; 0 -> 2^-127 (a BF16 subnormal), 0xFF -> NaN
+__device__ __forceinline__ uint32_t e8m0x2_to_bf16x2(uint32_t v) {
+    uint32_t out;
+    asm("{\n\t.reg .b16 h;\n\tcvt.u16.u32 h, %1;\n\tcvt.rn.bf16x2.ue8m0x2 %0, h;\n\t}" : "=r"(out) : "r"(v));
+    return out;
+}
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                        uint32_t b1, const float (&c)[4]) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(c[0]), "f"(c[1]), "f"(c[2]), "f"(c[3]));
+}
+
+// ---------------------------------------------------------------------------------------------
+// stage table entry (uint4), built once per CTA from stage_lookup():
+//   x  byte offset into codes of (first row of the tile, first block of the stage)
+//   y  byte offset into scales of the same position
+//   z  b (16 bits: first block within the window) | nblk << 16 | flags << 24 | (rows in tile - 1) << 28
+//   w  tile | window << 20
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kFlagSegFirst = 1, kFlagSegLast = 2, kFlagWinFirst = 4;
+
+__device__ __forceinline__ void store_out(void *Y, int y_dtype, int64_t idx, float v) {
+    if (y_dtype == MXQ_F32)
+        reinterpret_cast<float *>(Y)[idx] = v;
+    else
+        reinterpret_cast<__nv_bfloat16 *>(Y)[idx] = __float2bfloat16_rn(v);
+}
+
+// ---------------------------------------------------------------------------------------------
+// the kernel
+// ---------------------------------------------------------------------------------------------
+// NT8: 8-token column tiles (1 for M <= 8, 2 for M <= 16); NS: ring depth
+template <int NT8, int NS>
+__global__ void __launch_bounds__(kMmaThreads, 2)
+linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restrict__ X,
+                  const uint8_t *__restrict__ codes, const uint8_t *__restrict__ scales, void *__restrict__ Y,
+                  int y_dtype, uint8_t *__restrict__ ws) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t sbase = smem_u32(smem);
+    int *s_rowmax = reinterpret_cast<int *>(smem + kOffMisc);               // [0]: largest |x| bits of the window
+    int *s_flags = reinterpret_cast<int *>(smem + kOffMisc + 128);          // [0] inexact, [1] last-arriver
+    const uint4 *s_table = reinterpret_cast<const uint4 *>(smem + kOffTable);
+    float *s_red = reinterpret_cast<float *>(smem + kOffRed);               // [warps][NT8*8][16]
+    constexpr int kOutPerWarp = NT8 * 8 * kTileRows;
+
+    pdl_trigger();  // let the next kernel in the stream start prefetching its weights
+
+    // ---- stage table: one thread per stage, closed form -------------------------------------------
+    const uint32_t u_begin = cta_begin(p, blockIdx.x), u_end = cta_begin(p, blockIdx.x + 1);
+    StageInfo si;
+    const int nstages = stage_lookup(p, u_begin, u_end, -1, si);
+    for (int q = tid; q < nstages; q += kMmaThreads) {
+        stage_lookup(p, u_begin, u_end, q, si);
+        const uint32_t j = (uint32_t)si.w * (uint32_t)p.bw + (uint32_t)si.b;   // block index within the row
+        const int64_t rows_left = p.N - (int64_t)si.tile * kTileRows;
+        const uint32_t rows_m1 = (uint32_t)(rows_left < kTileRows ? rows_left : kTileRows) - 1u;
+        uint4 e;
+        e.x = (uint32_t)si.tile * kTileRows * (uint32_t)(p.K / 2) + j * 16u;
+        e.y = (uint32_t)si.tile * kTileRows * (uint32_t)p.kb + j;
+        e.z = (uint32_t)si.b | ((uint32_t)si.nblk << 16) |
+              ((si.seg_first ? kFlagSegFirst : 0u) | (si.seg_last ? kFlagSegLast : 0u) | (si.win_first ? kFlagWinFirst : 0u)) << 24 |
+              rows_m1 << 28;
+        e.w = (uint32_t)si.tile | ((uint32_t)si.w << 20);
+        reinterpret_cast<uint4 *>(smem + kOffTable)[q] = e;
+    }
+    if (tid == 0) s_flags[0] = s_flags[1] = 0;
+    __syncthreads();
+
+    // ---- per-lane constants ---------------------------------------------------------------------------
+    const int blk0 = warp * kWarpBlocks;  // this warp's blocks within a stage
+    const uint32_t ring = sbase + p.off_ring + (uint32_t)warp * (uint32_t)(NS * kWarpStageBytes);
+    // copy role of this lane: rows cr and cr + 8 of the tile, 16-byte chunk cc (= block within the slice);
+    // lanes 0..15 also copy the 4 scale bytes of row `lane`
+    const int cr = lane & 7, cc = lane >> 3;
+    const uint32_t row_bytes = (uint32_t)(p.K / 2);
+    // codes are laid out [block][row][16 bytes] inside a slot, so that a fragment read (row g, word t of
+    // block jb) hits bank 4g + t: conflict-free, with immediate offsets
+    const uint32_t dst_lo = (uint32_t)(cc * 256 + cr * 16), dst_sc = kWarpCodeBytes + (lane & 15) * 4;
+    const uint8_t *codes_w = codes + (blk0 + cc) * 16;
+    const uint8_t *scales_w = scales + blk0;
+
+    auto issue = [&](int q, int slot) {
+        const uint4 e = s_table[q];
+        const int nblk = (e.z >> 16) & 0xFF;
+        if (blk0 < nblk) {
+            const uint32_t rows_m1 = e.z >> 28;
+            const uint32_t dst = ring + (uint32_t)slot * kWarpStageBytes;
+            const uint8_t *src = codes_w + e.x;
+            cp_async16(dst + dst_lo, src + min((uint32_t)cr, rows_m1) * row_bytes);
+            cp_async16(dst + dst_lo + 128, src + min((uint32_t)cr + 8u, rows_m1) * row_bytes);
+            if (lane < kTileRows) cp_async4(dst + dst_sc, scales_w + e.y + min((uint32_t)lane, rows_m1) * (uint32_t)p.kb);
+        }
+    };
+
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+        if (s < nstages) issue(s, s);
+        cp_async_commit();
+    }
+
+    pdl_wait();  // from here on X, Y and the workspace may be touched
+
+    unsigned *tickets = reinterpret_cast<unsigned *>(ws + kWsTicketOff);
+    float *partials = reinterpret_cast<float *>(ws + kWsPartialOff);
+
+    float acc[NT8][4];
+#pragma unroll
+    for (int n = 0; n < NT8; ++n)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[n][i] = 0.f;
+
+    // per-thread constants of the fragment reads
+    const uint32_t a_off = (uint32_t)(g * 16 + 4 * t);                       // + jb*256 (+128 for row g+8)
+    // B fragment: token g (and g + 8).  Lanes whose token does not exist read the last real token instead:
+    // a column of B only ever feeds the same column of the result, and those columns are never stored.
+    const uint32_t x_thread0 = sbase + p.off_x + (uint32_t)blk0 * 64u + 16u * t + (uint32_t)min(g, p.M - 1) * p.x_stride;
+    const uint32_t x_thread1 = sbase + p.off_x + (uint32_t)blk0 * 64u + 16u * t + (uint32_t)min(g + 8, p.M - 1) * p.x_stride;
+
+    int seg_index = 0, slot = 0, seg_b0 = 0;
+    bool exact_ok = true;
+    float un = 1.f;
+#pragma unroll 1
+    for (int q = 0; q < nstages; ++q) {
+        const uint4 e = s_table[q];
+        const int b_now = e.z & 0xFFFF, nblk_now = (e.z >> 16) & 0xFF;
+        const uint32_t flags = (e.z >> 24) & 0xF;
+        if (flags & kFlagSegFirst) seg_b0 = b_now;
+
+        // ---- (re)stage this window's slice of X as scaled FP16 -------------------------------
+        if (flags & kFlagWinFirst) {
+            const int w_now = e.w >> 20;
+            const int bwid = (w_now == p.nwin - 1) ? p.bw_last : p.bw;
+            const int64_t k0 = (int64_t)w_now * p.bw * kBlock;
+            const int nvec = bwid * kBlock / 8;  // 16-byte vectors per token row
+            __syncthreads();                      // everyone is done with the previous window
+            if (tid == 0) {
+                s_rowmax[0] = 0;
+                s_flags[0] = 0;
+            }
+            __syncthreads();
+            uint32_t mx = 0;
+            for (int m = 0; m < p.M; ++m) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0);
+                for (int i = tid; i < nvec; i += kMmaThreads) {
+                    const uint4 v = __ldcg(src + i);
+                    mx = max(mx, max(max(v.x & 0x7FFFu, (v.x >> 16) & 0x7FFFu), max(v.y & 0x7FFFu, (v.y >> 16) & 0x7FFFu)));
+                    mx = max(mx, max(max(v.z & 0x7FFFu, (v.z >> 16) & 0x7FFFu), max(v.w & 0x7FFFu, (v.w >> 16) & 0x7FFFu)));
+                }
+            }
+            if (mx) atomicMax(&s_rowmax[0], (int)mx);
+            __syncthreads();
+            // one power-of-two scale for the whole slice: the largest magnitude lands in [2^14, 2^15)
+            int sh = 141 - min(s_rowmax[0] >> 7, 254);
+            sh = sh > 126 ? 126 : sh;
+            const float up = __uint_as_float((uint32_t)(sh + 127) << 23);
+            un = __uint_as_float((uint32_t)(127 - sh) << 23);
+            int inexact = 0;
+            for (int m = 0; m < p.M; ++m) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0);
+                uint8_t *dst = smem + p.off_x + (size_t)m * p.x_stride;
+                for (int i = tid; i < nvec; i += kMmaThreads) {
+                    const uint4 v = __ldcg(src + i);
+                    const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+                    uint32_t out[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float lo = __uint_as_float(in[j] << 16) * up;
+                        const float hi = __uint_as_float(in[j] & 0xFFFF0000u) * up;
+                        const __half2 h = __floats2half2_rn(lo, hi);
+                        const float2 back = __half22float2(h);
+                        inexact |= (back.x != lo) | (back.y != hi);
+                        out[j] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                    *reinterpret_cast<uint4 *>(dst + (size_t)i * 16) = make_uint4(out[0], out[1], out[2], out[3]);
+                }
+            }
+            if (inexact) atomicOr(&s_flags[0], 1);
+            __syncthreads();
+            exact_ok = s_flags[0] == 0;
+            if (!exact_ok && tid == 0) atomicAdd(reinterpret_cast<unsigned *>(ws + kWsFallbackOff), 1u);  // diagnostic
+        }
+
+        // ---- consume this warp's slice of the stage ------------------------------------------------
+        cp_async_wait<NS - 1>();  // all but the newest NS-1 groups have landed: this stage is in
+        __syncwarp();
+        if (exact_ok && blk0 < nblk_now) {
+            const uint32_t cbase = ring + (uint32_t)slot * kWarpStageBytes;
+            // the four blocks' scales of rows g and g+8; 2^-shift of X is folded in here (8 multiplies per stage)
+            const uint32_t sw_lo = lds32(cbase + kWarpCodeBytes + g * 4), sw_hi = lds32(cbase + kWarpCodeBytes + g * 4 + 32);
+            const uint32_t sl01 = e8m0x2_to_bf16x2(sw_lo), sl23 = e8m0x2_to_bf16x2(sw_lo >> 16);
+            const uint32_t sh01 = e8m0x2_to_bf16x2(sw_hi), sh23 = e8m0x2_to_bf16x2(sw_hi >> 16);
+            const float sc_lo[4] = {__uint_as_float(sl01 << 16) * un, __uint_as_float(sl01 & 0xFFFF0000u) * un,
+                                    __uint_as_float(sl23 << 16) * un, __uint_as_float(sl23 & 0xFFFF0000u) * un};
+            const float sc_hi[4] = {__uint_as_float(sh01 << 16) * un, __uint_as_float(sh01 & 0xFFFF0000u) * un,
+                                    __uint_as_float(sh23 << 16) * un, __uint_as_float(sh23 & 0xFFFF0000u) * un};
+            const uint32_t abase = cbase + a_off;
+            const uint32_t xbase0 = x_thread0 + (uint32_t)b_now * 64u, xbase1 = x_thread1 + (uint32_t)b_now * 64u;
+            const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int jb = 0; jb < kWarpBlocks; ++jb) {
+                // A: this lane's 8 weights of rows g and g+8 of block jb (k = 8t .. 8t+7 of the block)
+                const uint32_t a_lo = lds32(abase + jb * 256);
+                const uint32_t a_hi = lds32(abase + jb * 256 + 128);
+                uint32_t l0, l1, l2, l3, h0, h1, h2, h3;
+                e2m1x8_to_half2x4(a_lo, l0, l1, l2, l3);
+                e2m1x8_to_half2x4(a_hi, h0, h1, h2, h3);
+#pragma unroll
+                for (int n = 0; n < NT8; ++n) {
+                    // B: the same 8 k of token g (+8 for the second column tile)
+                    const uint4 xb = lds128((n == 0 ? xbase0 : xbase1) + jb * 64);
+                    float part[4];
+                    mma_f16(part, l0, h0, l1, h1, xb.x, xb.y, zero);
+                    mma_f16(part, l2, h2, l3, h3, xb.z, xb.w, part);
+                    // late scaling (Eq. 2): one multiply per 32-long partial sum
+                    acc[n][0] = fmaf(part[0], sc_lo[jb], acc[n][0]);
+                    acc[n][1] = fmaf(part[1], sc_lo[jb], acc[n][1]);
+                    acc[n][2] = fmaf(part[2], sc_hi[jb], acc[n][2]);
+                    acc[n][3] = fmaf(part[3], sc_hi[jb], acc[n][3]);
+                }
+            }
+        }
+        __syncwarp();  // every lane is done reading the slot
+        if (q + NS < nstages) issue(q + NS, slot);
+        cp_async_commit();
+        slot = (slot + 1 == NS) ? 0 : slot + 1;
+
+        if (!(flags & kFlagSegLast)) continue;
+
+        // ---- end of this CTA's share of a (window, tile) pair: combine the 16 warps ---------------
+        const int tile_now = e.w & 0xFFFFF, w_now = e.w >> 20;
+        const int seg_b1 = b_now + nblk_now;
+        const int nseg_blocks = seg_b1 - seg_b0;
+        if (exact_ok) {
+            float *mine = s_red + warp * kOutPerWarp;
+#pragma unroll
+            for (int n = 0; n < NT8; ++n) {
+                mine[(8 * n + 2 * t) * kTileRows + g] = acc[n][0];
+                mine[(8 * n + 2 * t + 1) * kTileRows + g] = acc[n][1];
+                mine[(8 * n + 2 * t) * kTileRows + g + 8] = acc[n][2];
+                mine[(8 * n + 2 * t + 1) * kTileRows + g + 8] = acc[n][3];
+                acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+            }
+        } else {
+            // scalar FP32 path for X that does not fit FP16 exactly: warp r computes tile row r directly
+            // from global memory (same late scaling, FP32 accumulation), for every token
+            const int64_t row = min((int64_t)tile_now * kTileRows + warp, p.N - 1);
+            const int64_t j0 = (int64_t)w_now * p.bw;
+            for (int m = 0; m < NT8 * 8; ++m) {
+                float a = 0.f;
+                if (m < p.M) {
+                    for (int j = seg_b0 + lane; j < seg_b1; j += 32) {
+                        const uint4 c = ld_stream_u4(codes + row * (p.K / 2) + (j0 + j) * 16);
+                        const float s = e8m0_to_float(scales[row * p.kb + j0 + j]);
+                        const uint32_t w4[4] = {c.x, c.y, c.z, c.w};
+                        const uint16_t *xr = X + (int64_t)m * p.K + (j0 + j) * kBlock;
+                        float part = 0.f;
+#pragma unroll
+                        for (int qd = 0; qd < 4; ++qd)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float2 wv = __half22float2(e2m1x2_to_half2((w4[qd] >> (8 * i)) & 0xFFu));
+                                const uint32_t xb = __ldcg(reinterpret_cast<const uint32_t *>(xr + qd * 8 + i * 2));
+                                part = fmaf(wv.x, __uint_as_float(xb << 16), part);
+                                part = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part);
+                            }
+                        a = fmaf(part, s, a);
+                    }
+                    a = warp_sum(a);
+                }
+                if (lane == 0) s_red[m * kTileRows + warp] = a;  // [token][row]
+            }
+        }
+        __syncthreads();
+
+        const bool whole = (p.nwin == 1) && (seg_b0 == 0) && (seg_b1 == p.bw_last);
+        float val = 0.f;
+        const int m_out = tid / kTileRows, r_out = tid % kTileRows;
+        const int64_t n_out = (int64_t)tile_now * kTileRows + r_out;
+        if (tid < kOutPerWarp) {
+            if (exact_ok) {
+#pragma unroll
+                for (int w = 0; w < kMmaWarps; ++w) val += s_red[w * kOutPerWarp + tid];
+            } else {
+                val = s_red[tid];
+            }
+            if (whole) {
+                if (m_out < p.M && n_out < p.N) store_out(Y, y_dtype, (int64_t)m_out * p.N + n_out, val);
+            } else {
+                partials[((size_t)blockIdx.x * p.slots + seg_index) * kOutPerWarp + tid] = val;
+                __threadfence();
+            }
+        }
+        __syncthreads();
+        if (!whole) {
+            if (tid == 0) {
+                const unsigned done = atomicAdd(&tickets[tile_now], (unsigned)nseg_blocks) + (unsigned)nseg_blocks;
+                s_flags[1] = (done == (unsigned)p.kb);
+                if (done == (unsigned)p.kb) tickets[tile_now] = 0;  // ready for the next call
+            }
+            __syncthreads();
+            if (s_flags[1]) {
+                __threadfence();
+                if (tid < kOutPerWarp) {
+                    // sum every CTA's share of this tile in unit order
+                    float sum = 0.f;
+                    for (int w = 0; w < p.nwin; ++w) {
+                        const uint32_t pb = pair_begin(p, w, tile_now);
+                        const uint32_t pe = pb + (uint32_t)((w == p.nwin - 1) ? p.bw_last : p.bw);
+                        const int c0 = cta_of(p, pb), c1 = cta_of(p, pe - 1);
+                        const int pair_id = w * p.tiles + tile_now;
+                        for (int c = c0; c <= c1; ++c) {
+                            int fw, ft, fb;
+                            unit_decode(p, cta_begin(p, c), fw, ft, fb);
+                            const int slot_i = pair_id - (fw * p.tiles + ft);
+                            sum += __ldcg(&partials[((size_t)c * p.slots + slot_i) * kOutPerWarp + tid]);
+                        }
+                    }
+                    if (m_out < p.M && n_out < p.N) store_out(Y, y_dtype, (int64_t)m_out * p.N + n_out, sum);
+                }
+            }
+            __syncthreads();
+        }
+        ++seg_index;
+    }
+    cp_async_wait<0>();
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side: plan + launch
+// ---------------------------------------------------------------------------------------------
+bool linear_mma_plan(int M, int64_t N, int64_t K, LinearPlan &p) {
+    if (M < 1 || M > 16 || (K % 128) != 0 || N < 1) return false;
+    const int64_t tiles = (N + kTileRows - 1) / kTileRows;
+    const int64_t kb = K / 32;
+    if (tiles > kTicketCap || tiles * kb >= (int64_t)1 << 31 || N * (K / 2) >= (int64_t)1 << 32) return false;
+    p.M = M;
+    p.nt8 = M <= 8 ? 1 : 2;
+    p.tiles = (int)tiles;
+    p.kb = (int)kb;
+    p.N = N;
+    p.K = K;
+    p.units = (uint32_t)(tiles * kb);
+    const uint32_t red_bytes = (uint32_t)kMmaWarps * p.nt8 * 8 * kTileRows * 4;
+    p.off_x = kOffRed + red_bytes;
+    // ring depth and K windows: prefer 4 stages and one window; give up stages, then split K
+    auto layout = [&](int nstage, int64_t bw) {  // fills the offsets for a window of bw blocks; returns total bytes
+        p.x_stride = (uint32_t)(2 * bw * 32 + 64);
+        p.off_ring = (p.off_x + (uint32_t)M * p.x_stride + 127) / 128 * 128;
+        p.smem_bytes = p.off_ring + (uint32_t)(kMmaWarps * nstage * kWarpStageBytes);
+        return p.smem_bytes;
+    };
+    int nstage = kMaxStages, nwin = 1;
+    int64_t bw = kb;
+    while (nstage > 2 && layout(nstage, bw) > kSmemBudget) --nstage;
+    while (layout(nstage, bw) > kSmemBudget) {
+        if (++nwin > 64) return false;
+        bw = ((kb + nwin - 1) / nwin + 3) / 4 * 4;
+    }
+    while ((int64_t)(nwin - 1) * bw >= kb) --nwin;  // rounding up may have left the last window empty
+    p.nstage = nstage;
+    p.nwin = nwin;
+    p.bw = (int)bw;
+    p.bw_last = (int)(kb - (int64_t)(nwin - 1) * bw);
+    // one CTA per SM; more (a multiple of the SM count) only if a CTA's stage table would not fit
+    const int min_bw = p.bw_last < p.bw ? p.bw_last : p.bw;
+    const uint32_t groups = p.units / 4;
+    const int sms = sm_count();
+    for (int mult = 1;; ++mult) {
+        int grid = sms * mult;
+        if ((uint32_t)grid > groups) grid = (int)groups;
+        const uint32_t per_cta = (p.units + grid - 1) / grid + 4;
+        const uint32_t stages_bound = per_cta / kStageBlocks + per_cta / (uint32_t)min_bw + (uint32_t)p.nwin + 3;
+        if (stages_bound <= (uint32_t)kMaxCtaStages || (uint32_t)grid == groups) {
+            if (stages_bound > (uint32_t)kMaxCtaStages) return false;
+            p.grid = grid;
+            p.slots = (int)(per_cta / min_bw) + 3;
+            return true;
+        }
+        if (mult > 4096) return false;
+    }
+}
+
+size_t linear_mma_workspace_bytes(const LinearPlan &p) {
+    return kWsPartialOff + (size_t)p.grid * p.slots * (size_t)(p.nt8 * 8 * kTileRows) * sizeof(float);
+}
+
+template <int NT8, int NS>
+static cudaError_t launch_mma(const LinearPlan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,
+                              int y_dtype, void *ws, cudaStream_t stream) {
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(linear_mma_kernel<NT8, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kSmemBudget);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.grid);
+    cfg.blockDim = dim3(kMmaThreads);
+    cfg.dynamicSmemBytes = p.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, linear_mma_kernel<NT8, NS>, p, (const uint16_t *)X, codes, scales, Y, y_dtype,
+                              (uint8_t *)ws);
+}
+
+cudaError_t linear_mma_launch(const LinearPlan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,
+                              int y_dtype, void *ws, cudaStream_t stream) {
+#define MXQ_LAUNCH(NT, NSTG) launch_mma<NT, NSTG>(p, X, codes, scales, Y, y_dtype, ws, stream)
+    if (p.nt8 == 1) return p.nstage == 4 ? MXQ_LAUNCH(1, 4) : (p.nstage == 3 ? MXQ_LAUNCH(1, 3) : MXQ_LAUNCH(1, 2));
+    return p.nstage == 4 ? MXQ_LAUNCH(2, 4) : (p.nstage == 3 ? MXQ_LAUNCH(2, 3) : MXQ_LAUNCH(2, 2));
+#undef MXQ_LAUNCH
+}
+
+}  // namespace mxq

@@ -22,6 +22,9 @@ def run_case(wbits, xbits, out_dtype=torch.float32, rows=None, what=""):
     y = mxq.mxq_linear(gpu_bf16(xbits), torch.from_numpy(codes).cuda(), torch.from_numpy(scales).cuda(),
                        out_dtype=out_dtype, workspace=ws)
     torch.cuda.synchronize()
+    assert int(ws.view(torch.int32)[0]) == 0, what + ": a bounded wait inside the kernel gave up"
+    if ws.numel() >= 256 + 65536 * 4:
+        assert not ws[256: 256 + 65536 * 4].any(), what + ": ticket counters were not returned to zero"
     if rows is not None:
         y = y[:, torch.as_tensor(rows, device="cuda")]
     return check_linear(y, y64, a64, what), y
@@ -61,7 +64,26 @@ def test_every_token_count_on_a_ragged_shape(m):
     run_case(w, x, what="ragged M=%d" % m)
 
 
-@pytest.mark.parametrize("n,k", [(1, 32), (2, 64), (7, 32), (9, 4096), (300, 96), (16, 13824), (129, 5120)])
+@pytest.mark.parametrize("m", [1, 2, 3, 4, 5, 7, 8, 9, 12, 15, 16])
+def test_every_token_count_on_a_ragged_shape_tensor_core_path(m):
+    n, k = 203, 1408   # N not a multiple of 16, K = 44 blocks (a multiple of 128: tensor-core kernel)
+    w = synth.bits_of(synth.weight(3, 14, n, k))
+    x = synth.bits_of(synth.activations(3, 14, m, k))
+    assert mxq.mxq_linear_plan_info(m, n, k)["tensor_core"] == 1
+    run_case(w, x, what="ragged tc M=%d" % m)
+
+
+@pytest.mark.parametrize("m,n,k", [(8, 4096, 11008), (16, 512, 13824), (16, 1000, 4096), (12, 333, 5120)])
+def test_shapes_that_split_k_into_windows(m, n, k):
+    assert mxq.mxq_linear_plan_info(m, n, k)["windows"] > 1
+    w = synth.bits_of(synth.weight(3, 15, n, k))
+    x = synth.bits_of(synth.activations(3, 15, m, k))
+    rows = np.unique(np.concatenate([[0, n - 1], np.random.default_rng(5).integers(0, n, 200)])).astype(np.int64)
+    run_case(w, x, rows=rows, what="windows %dx%d M=%d" % (n, k, m))
+
+
+@pytest.mark.parametrize("n,k", [(1, 32), (2, 64), (7, 32), (9, 4096), (300, 96), (16, 13824), (129, 5120), (1, 128),
+                                 (17, 128), (5000, 256)])
 @pytest.mark.parametrize("m", [1, 3, 16])
 def test_small_and_extreme_shapes(n, k, m):
     w = synth.bits_of(synth.weight(5, 2, n, k))
@@ -135,7 +157,8 @@ def test_nan_scale_gives_nan_row_only():
 
 
 def test_wide_range_activations():
-    """Activations spanning many binades, including BF16 subnormals and zeros."""
+    """Activations spanning many binades, including BF16 subnormals and zeros: more than FP16 can hold
+    next to the row maximum, so the tensor-core kernel must take its exact scalar path."""
     rng = np.random.default_rng(7)
     n, k, m = 130, 1024, 6
     w = synth.bits_of(synth.weight(3, 13, n, k))

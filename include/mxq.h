@@ -89,16 +89,16 @@ int mxq_quantize(const void *W_bf16, int64_t N, int64_t K, uint8_t *codes, uint8
 int mxq_dequantize(const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K, void *W_bf16_out,
                    void *stream);
 
-/* Workspace (bytes) mxq_linear needs for this shape; may be 0.  The workspace must be
- * zero-filled once before its first use; every call leaves it ready for the next one
- * (of any shape).  Two calls that may run concurrently need separate workspaces. */
+/* Workspace (bytes) mxq_linear needs for this shape; 0 for every shape in this version
+ * (no CTA shares an output with another), kept in the interface for kernels that split K
+ * across CTAs.  If non-zero: zero-fill once before first use; calls leave it reusable. */
 size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K);
 
 /* How mxq_linear will run this shape on the current device (diagnostics; launches nothing).
- * info[12] int32: [0] 1 = tensor-core stream-K kernel, 0 = generic kernel; [1] CTAs;
- * [2] ring stages; [3] K windows; [4] blocks per window; [5] blocks in the last window;
- * [6] partial slots per CTA; [7] dynamic shared memory bytes; [8] 16-row tiles; [9] K/32;
- * [10] 8-token column tiles; [11] work units (tiles * K/32).  Unused entries are 0. */
+ * info[12] int32: [0] 1 = tensor-core kernel, 0 = generic kernel; [1] CTAs; [2] ring stages;
+ * [3] K windows; [4] blocks per window; [5] blocks in the last window; [6] most 16-row tiles
+ * a CTA owns; [7] dynamic shared memory bytes; [8] 8-token column tiles; [9] K/32.
+ * Unused entries are 0. */
 int mxq_linear_plan_info(int M, int64_t N, int64_t K, int32_t *info);
 
 /* Weight-only-quantised linear layer (the MXFP4 GEMM of Sec. III-D-3, Eq. 2):

@@ -125,8 +125,8 @@ def mxq_linear_plan_info(m: int, n: int, k: int) -> dict:
     """How mxq_linear will run this shape (diagnostics)."""
     info = (ctypes.c_int32 * 12)()
     _check(lib().mxq_linear_plan_info(m, n, k, ctypes.cast(info, ctypes.c_void_p)), "mxq_linear_plan_info")
-    keys = ("tensor_core", "grid", "stages", "windows", "bw", "bw_last", "slots", "smem_bytes", "tiles", "kb", "nt8",
-            "units")
+    keys = ("tensor_core", "grid", "stages", "windows", "bw", "bw_last", "max_tiles", "smem_bytes", "nt8", "kb",
+            "reserved0", "reserved1")
     return dict(zip(keys, [int(v) for v in info]))
 
 

@@ -130,12 +130,10 @@ int mxq_linear_plan_info(int M, int64_t N, int64_t K, int32_t *info) {
         info[3] = p.nwin;
         info[4] = p.bw;
         info[5] = p.bw_last;
-        info[6] = p.slots;
+        info[6] = p.max_tiles;
         info[7] = (int32_t)p.smem_bytes;
-        info[8] = p.tiles;
+        info[8] = p.nt8;
         info[9] = p.kb;
-        info[10] = p.nt8;
-        info[11] = (int32_t)p.units;
     } else {
         info[1] = (int32_t)((N + mxq::kRowWarpRows - 1) / mxq::kRowWarpRows);
     }
@@ -152,7 +150,8 @@ int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *s
     cudaStream_t st = (cudaStream_t)stream;
     mxq::LinearPlan plan;
     if (!mxq::force_generic() && mxq::linear_mma_plan(M, N, K, plan)) {
-        if (!workspace || workspace_bytes < mxq::linear_mma_workspace_bytes(plan)) return MXQ_ERR_WORKSPACE;
+        const size_t need = mxq::linear_mma_workspace_bytes(plan);
+        if (need > 0 && (!workspace || workspace_bytes < need)) return MXQ_ERR_WORKSPACE;
         if (!mxq::aligned16(workspace)) return MXQ_ERR_ALIGN;
         if (mxq::linear_mma_launch(plan, X_bf16, codes, scales, Y, y_dtype, workspace, st) != cudaSuccess) {
             (void)cudaGetLastError();

@@ -8,26 +8,27 @@
 // FP16 pairs as they come; the multiply-accumulate then costs almost nothing for any M <= 8.
 //
 // Exactness: every E2M1 value is an FP16 number.  X is BF16; each CTA rescales its slice of X
-// by a power of two (per token row) so that the largest magnitude sits just below 2^15 and
-// converts it to FP16, checking every element converts exactly (true whenever an element is
-// within 2^32 of its row maximum).  Products FP16 x FP16 are exact in the FP32 accumulator.
-// If any element does not convert exactly the CTA takes a scalar FP32 path instead, so the
-// result never depends on the shortcut.
+// by one power of two so that the largest magnitude sits just below 2^15 and converts it to
+// FP16, checking that every element converts exactly (true whenever an element is within 2^32
+// of the largest).  Products FP16 x FP16 are exact in the FP32 accumulator.  If any element
+// does not convert exactly the CTA takes a scalar FP32 path instead, so the result never
+// depends on the shortcut.
 //
-// Decomposition (stream-K): the matrix is cut into units of 16 rows x 32 k (one MX block per
-// row), ordered window-major / tile / k.  Each CTA owns an equal, contiguous range of units,
-// so all SMs stream the same number of bytes whatever N is.  Within a CTA, 16 warps split each
-// stage's 64 blocks; their FP32 partial tiles are summed in a fixed order through shared
-// memory.  A tile whose K range is shared between CTAs goes through a workspace slot and a
-// ticket counter; the CTA that completes the tile sums the slots in unit order.  Nobody waits
-// for anybody, and the summation order is fixed, so results are bit-reproducible.
+// Decomposition: CTA c owns the weight rows [c*N/G, (c+1)*N/G) for the whole of K, so every
+// CTA streams the same number of bytes to within one row, no output is shared between CTAs,
+// and there is no workspace.  The rows are processed as 16-row tiles (the last one ragged:
+// missing rows are neither fetched nor stored).  Within a CTA the 8 warps split each stage's
+// 32 MX blocks; every warp leaves its FP32 partial tile in shared memory and the warp that
+// arrives last (a counter, not a barrier) sums the 8 in warp order, so results are
+// bit-reproducible.  When M*K is too large for X to fit in shared memory, K is cut into
+// windows; the CTA walks its tiles once per window and keeps per-tile sums in shared memory.
 //
 // Pipeline: every warp runs its own ring of 16-byte cp.async copies for exactly the bytes it
 // will consume (16 rows x 64 code bytes + 16 x 4 scale bytes per stage), so the main loop has
 // no CTA-wide barrier and no spin-wait.  Weights never depend on the previous kernel, so the
-// ring is filled before griddepcontrol.wait (programmatic dependent launch); X, Y and the
-// workspace are touched only after it.  A CTA uses at most half an SM so that the next
-// kernel's CTAs can be resident and prefetching while this one computes.
+// ring is filled before griddepcontrol.wait (programmatic dependent launch); X and Y are
+// touched only after it.  A CTA is small enough that two kernels, two CTAs per SM each, can be
+// resident: the next kernel prefetches while this one computes.
 #include "mxq_device.cuh"
 #include "mxq_host.h"
 #include "mxq_linear_plan.h"
@@ -87,9 +88,9 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1,
 //   x  byte offset into codes of (first row of the tile, first block of the stage)
 //   y  byte offset into scales of the same position
 //   z  b (16 bits: first block within the window) | nblk << 16 | flags << 24 | (rows in tile - 1) << 28
-//   w  tile | window << 20
+//   w  tile (local to the CTA) | window << 20
 // ---------------------------------------------------------------------------------------------
-constexpr uint32_t kFlagSegFirst = 1, kFlagSegLast = 2, kFlagWinFirst = 4;
+constexpr uint32_t kFlagSegLast = 1, kFlagWinFirst = 2;
 
 __device__ __forceinline__ void store_out(void *Y, int y_dtype, int64_t idx, float v) {
     if (y_dtype == MXQ_F32)
@@ -98,46 +99,75 @@ __device__ __forceinline__ void store_out(void *Y, int y_dtype, int64_t idx, flo
         reinterpret_cast<__nv_bfloat16 *>(Y)[idx] = __float2bfloat16_rn(v);
 }
 
+__device__ __forceinline__ uint32_t max_abs_bits(const uint4 &v) {  // largest BF16 magnitude pattern of 8 values
+    return max(max(max(v.x & 0x7FFFu, (v.x >> 16) & 0x7FFFu), max(v.y & 0x7FFFu, (v.y >> 16) & 0x7FFFu)),
+               max(max(v.z & 0x7FFFu, (v.z >> 16) & 0x7FFFu), max(v.w & 0x7FFFu, (v.w >> 16) & 0x7FFFu)));
+}
+
+// 8 BF16 -> 8 FP16 after scaling by `up`; returns non-zero if any conversion was inexact
+__device__ __forceinline__ int bf16x8_to_f16x8(const uint4 &v, float up, uint4 &out) {
+    const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+    uint32_t o[4];
+    int inexact = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float lo = __uint_as_float(in[j] << 16) * up;
+        const float hi = __uint_as_float(in[j] & 0xFFFF0000u) * up;
+        const __half2 h = __floats2half2_rn(lo, hi);
+        const float2 back = __half22float2(h);
+        inexact |= (back.x != lo) | (back.y != hi);
+        o[j] = *reinterpret_cast<const uint32_t *>(&h);
+    }
+    out = make_uint4(o[0], o[1], o[2], o[3]);
+    return inexact;
+}
+
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
 // NT8: 8-token column tiles (1 for M <= 8, 2 for M <= 16); NS: ring depth
 template <int NT8, int NS>
-__global__ void __launch_bounds__(kMmaThreads, 2)
+__global__ void __launch_bounds__(kMmaThreads, 4)
 linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restrict__ X,
                   const uint8_t *__restrict__ codes, const uint8_t *__restrict__ scales, void *__restrict__ Y,
-                  int y_dtype, uint8_t *__restrict__ ws) {
+                  int y_dtype) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     const uint32_t sbase = smem_u32(smem);
-    int *s_rowmax = reinterpret_cast<int *>(smem + kOffMisc);               // [0]: largest |x| bits of the window
-    int *s_flags = reinterpret_cast<int *>(smem + kOffMisc + 128);          // [0] inexact, [1] last-arriver
+    int *s_max = reinterpret_cast<int *>(smem + kOffMisc);            // [0]: largest |x| pattern of the window
+    int *s_inexact = reinterpret_cast<int *>(smem + kOffMisc + 16);   // [0]
+    int *s_cnt = reinterpret_cast<int *>(smem + kOffMisc + 32);       // [kRedSlots] warps arrived
+    int *s_gen = reinterpret_cast<int *>(smem + kOffMisc + 64);       // [kRedSlots] tiles summed per slot
     const uint4 *s_table = reinterpret_cast<const uint4 *>(smem + kOffTable);
-    float *s_red = reinterpret_cast<float *>(smem + kOffRed);               // [warps][NT8*8][16]
-    constexpr int kOutPerWarp = NT8 * 8 * kTileRows;
+    float *s_red = reinterpret_cast<float *>(smem + kOffRed);         // [kRedSlots][warps][NT8*8][16]
+    float *s_acc = reinterpret_cast<float *>(smem + p.off_acc);       // [tiles][NT8*8][16], only if nwin > 1
+    constexpr int kOut = NT8 * 8 * kTileRows;                         // values of one tile
+    constexpr int kPerLane = kOut / 32;
 
     pdl_trigger();  // let the next kernel in the stream start prefetching its weights
 
-    // ---- stage table: one thread per stage, closed form -------------------------------------------
-    const uint32_t u_begin = cta_begin(p, blockIdx.x), u_end = cta_begin(p, blockIdx.x + 1);
+    // ---- this CTA's rows and its stage table (one thread per stage, closed form) ---------------------
+    const int64_t r0 = row_begin(p, blockIdx.x), r1 = row_begin(p, blockIdx.x + 1);
+    const int tiles = (int)((r1 - r0 + kTileRows - 1) / kTileRows);
     StageInfo si;
-    const int nstages = stage_lookup(p, u_begin, u_end, -1, si);
+    const int nstages = stage_lookup(p, tiles, -1, si);
     for (int q = tid; q < nstages; q += kMmaThreads) {
-        stage_lookup(p, u_begin, u_end, q, si);
+        stage_lookup(p, tiles, q, si);
         const uint32_t j = (uint32_t)si.w * (uint32_t)p.bw + (uint32_t)si.b;   // block index within the row
-        const int64_t rows_left = p.N - (int64_t)si.tile * kTileRows;
+        const int64_t row = r0 + (int64_t)si.tile * kTileRows;
+        const int64_t rows_left = r1 - row;
         const uint32_t rows_m1 = (uint32_t)(rows_left < kTileRows ? rows_left : kTileRows) - 1u;
         uint4 e;
-        e.x = (uint32_t)si.tile * kTileRows * (uint32_t)(p.K / 2) + j * 16u;
-        e.y = (uint32_t)si.tile * kTileRows * (uint32_t)p.kb + j;
+        e.x = (uint32_t)(row * (p.K / 2)) + j * 16u;
+        e.y = (uint32_t)(row * p.kb) + j;
         e.z = (uint32_t)si.b | ((uint32_t)si.nblk << 16) |
-              ((si.seg_first ? kFlagSegFirst : 0u) | (si.seg_last ? kFlagSegLast : 0u) | (si.win_first ? kFlagWinFirst : 0u)) << 24 |
-              rows_m1 << 28;
+              ((si.seg_last ? kFlagSegLast : 0u) | (si.win_first ? kFlagWinFirst : 0u)) << 24 | rows_m1 << 28;
         e.w = (uint32_t)si.tile | ((uint32_t)si.w << 20);
         reinterpret_cast<uint4 *>(smem + kOffTable)[q] = e;
     }
-    if (tid == 0) s_flags[0] = s_flags[1] = 0;
+    if (tid < kRedSlots) s_cnt[tid] = s_gen[tid] = 0;
+    if (tid == 0) s_inexact[0] = 0;
     __syncthreads();
 
     // ---- per-lane constants ---------------------------------------------------------------------------
@@ -145,24 +175,21 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
     const uint32_t ring = sbase + p.off_ring + (uint32_t)warp * (uint32_t)(NS * kWarpStageBytes);
     // copy role of this lane: rows cr and cr + 8 of the tile, 16-byte chunk cc (= block within the slice);
     // lanes 0..15 also copy the 4 scale bytes of row `lane`
-    const int cr = lane & 7, cc = lane >> 3;
+    const uint32_t cr = lane & 7, cc = lane >> 3;
     const uint32_t row_bytes = (uint32_t)(p.K / 2);
-    // codes are laid out [block][row][16 bytes] inside a slot, so that a fragment read (row g, word t of
-    // block jb) hits bank 4g + t: conflict-free, with immediate offsets
-    const uint32_t dst_lo = (uint32_t)(cc * 256 + cr * 16), dst_sc = kWarpCodeBytes + (lane & 15) * 4;
-    const uint8_t *codes_w = codes + (blk0 + cc) * 16;
-    const uint8_t *scales_w = scales + blk0;
+    const uint32_t dst_lo = cc * 256 + cr * 16, dst_sc = kWarpCodeBytes + (lane & 15) * 4;
+    const uint8_t *src_lo = codes + (blk0 + cc) * 16 + (size_t)cr * row_bytes;
+    const uint8_t *src_hi = src_lo + (size_t)8 * row_bytes;
+    const uint8_t *src_sc = scales + blk0 + (size_t)(lane & 15) * (uint32_t)p.kb;
 
     auto issue = [&](int q, int slot) {
         const uint4 e = s_table[q];
-        const int nblk = (e.z >> 16) & 0xFF;
-        if (blk0 < nblk) {
-            const uint32_t rows_m1 = e.z >> 28;
+        const uint32_t nblk = (e.z >> 16) & 0xFF, rows_m1 = e.z >> 28;
+        if ((uint32_t)blk0 < nblk) {
             const uint32_t dst = ring + (uint32_t)slot * kWarpStageBytes;
-            const uint8_t *src = codes_w + e.x;
-            cp_async16(dst + dst_lo, src + min((uint32_t)cr, rows_m1) * row_bytes);
-            cp_async16(dst + dst_lo + 128, src + min((uint32_t)cr + 8u, rows_m1) * row_bytes);
-            if (lane < kTileRows) cp_async4(dst + dst_sc, scales_w + e.y + min((uint32_t)lane, rows_m1) * (uint32_t)p.kb);
+            if (cr <= rows_m1) cp_async16(dst + dst_lo, src_lo + e.x);
+            if (cr + 8 <= rows_m1) cp_async16(dst + dst_lo + 128, src_hi + e.x);
+            if ((uint32_t)lane <= rows_m1) cp_async4(dst + dst_sc, src_sc + e.y);  // rows_m1 <= 15: lanes 0..15 at most
         }
     };
 
@@ -172,10 +199,7 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
         cp_async_commit();
     }
 
-    pdl_wait();  // from here on X, Y and the workspace may be touched
-
-    unsigned *tickets = reinterpret_cast<unsigned *>(ws + kWsTicketOff);
-    float *partials = reinterpret_cast<float *>(ws + kWsPartialOff);
+    pdl_wait();  // from here on X and Y may be touched
 
     float acc[NT8][4];
 #pragma unroll
@@ -190,7 +214,7 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
     const uint32_t x_thread0 = sbase + p.off_x + (uint32_t)blk0 * 64u + 16u * t + (uint32_t)min(g, p.M - 1) * p.x_stride;
     const uint32_t x_thread1 = sbase + p.off_x + (uint32_t)blk0 * 64u + 16u * t + (uint32_t)min(g + 8, p.M - 1) * p.x_stride;
 
-    int seg_index = 0, slot = 0, seg_b0 = 0;
+    int seg_index = 0, slot = 0;
     bool exact_ok = true;
     float un = 1.f;
 #pragma unroll 1
@@ -198,60 +222,67 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
         const uint4 e = s_table[q];
         const int b_now = e.z & 0xFFFF, nblk_now = (e.z >> 16) & 0xFF;
         const uint32_t flags = (e.z >> 24) & 0xF;
-        if (flags & kFlagSegFirst) seg_b0 = b_now;
 
-        // ---- (re)stage this window's slice of X as scaled FP16 -------------------------------
+        // ---- (re)stage this window's slice of X as scaled FP16 (the only CTA-wide barriers) ----------
         if (flags & kFlagWinFirst) {
             const int w_now = e.w >> 20;
             const int bwid = (w_now == p.nwin - 1) ? p.bw_last : p.bw;
             const int64_t k0 = (int64_t)w_now * p.bw * kBlock;
-            const int nvec = bwid * kBlock / 8;  // 16-byte vectors per token row
-            __syncthreads();                      // everyone is done with the previous window
+            const int vec_per_row = bwid * kBlock / 8;   // 16-byte vectors per token row
+            const int nvec = vec_per_row * p.M;
+            __syncthreads();                              // everyone is done with the previous window
             if (tid == 0) {
-                s_rowmax[0] = 0;
-                s_flags[0] = 0;
+                s_max[0] = 0;
+                s_inexact[0] = 0;
             }
             __syncthreads();
+            // one trip to L2: the first four vectors of every thread stay in registers for the second pass
+            constexpr int kKeep = 4;
+            uint4 keep[kKeep];
             uint32_t mx = 0;
-            for (int m = 0; m < p.M; ++m) {
-                const uint4 *src = reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0);
-                for (int i = tid; i < nvec; i += kMmaThreads) {
-                    const uint4 v = __ldcg(src + i);
-                    mx = max(mx, max(max(v.x & 0x7FFFu, (v.x >> 16) & 0x7FFFu), max(v.y & 0x7FFFu, (v.y >> 16) & 0x7FFFu)));
-                    mx = max(mx, max(max(v.z & 0x7FFFu, (v.z >> 16) & 0x7FFFu), max(v.w & 0x7FFFu, (v.w >> 16) & 0x7FFFu)));
+#pragma unroll
+            for (int i = 0; i < kKeep; ++i) {
+                const int v = tid + i * kMmaThreads;
+                keep[i] = make_uint4(0, 0, 0, 0);
+                if (v < nvec) {
+                    const int m = v / vec_per_row, c = v - m * vec_per_row;
+                    keep[i] = __ldcg(reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0) + c);
                 }
+                mx = max(mx, max_abs_bits(keep[i]));
             }
-            if (mx) atomicMax(&s_rowmax[0], (int)mx);
+            for (int v = tid + kKeep * kMmaThreads; v < nvec; v += kMmaThreads) {
+                const int m = v / vec_per_row, c = v - m * vec_per_row;
+                mx = max(mx, max_abs_bits(__ldcg(reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0) + c)));
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            if (lane == 0 && mx) atomicMax(&s_max[0], (int)mx);
             __syncthreads();
             // one power-of-two scale for the whole slice: the largest magnitude lands in [2^14, 2^15)
-            int sh = 141 - min(s_rowmax[0] >> 7, 254);
+            int sh = 141 - min(s_max[0] >> 7, 254);
             sh = sh > 126 ? 126 : sh;
             const float up = __uint_as_float((uint32_t)(sh + 127) << 23);
             un = __uint_as_float((uint32_t)(127 - sh) << 23);
             int inexact = 0;
-            for (int m = 0; m < p.M; ++m) {
-                const uint4 *src = reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0);
-                uint8_t *dst = smem + p.off_x + (size_t)m * p.x_stride;
-                for (int i = tid; i < nvec; i += kMmaThreads) {
-                    const uint4 v = __ldcg(src + i);
-                    const uint32_t in[4] = {v.x, v.y, v.z, v.w};
-                    uint32_t out[4];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float lo = __uint_as_float(in[j] << 16) * up;
-                        const float hi = __uint_as_float(in[j] & 0xFFFF0000u) * up;
-                        const __half2 h = __floats2half2_rn(lo, hi);
-                        const float2 back = __half22float2(h);
-                        inexact |= (back.x != lo) | (back.y != hi);
-                        out[j] = *reinterpret_cast<const uint32_t *>(&h);
-                    }
-                    *reinterpret_cast<uint4 *>(dst + (size_t)i * 16) = make_uint4(out[0], out[1], out[2], out[3]);
+            for (int i = 0; i < kKeep; ++i) {
+                const int v = tid + i * kMmaThreads;
+                if (v < nvec) {
+                    const int m = v / vec_per_row, c = v - m * vec_per_row;
+                    uint4 out;
+                    inexact |= bf16x8_to_f16x8(keep[i], up, out);
+                    *reinterpret_cast<uint4 *>(smem + p.off_x + (size_t)m * p.x_stride + (size_t)c * 16) = out;
                 }
             }
-            if (inexact) atomicOr(&s_flags[0], 1);
+            for (int v = tid + kKeep * kMmaThreads; v < nvec; v += kMmaThreads) {
+                const int m = v / vec_per_row, c = v - m * vec_per_row;
+                uint4 out;
+                inexact |= bf16x8_to_f16x8(__ldcg(reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0) + c), up, out);
+                *reinterpret_cast<uint4 *>(smem + p.off_x + (size_t)m * p.x_stride + (size_t)c * 16) = out;
+            }
+            if (inexact) atomicOr(&s_inexact[0], 1);
             __syncthreads();
-            exact_ok = s_flags[0] == 0;
-            if (!exact_ok && tid == 0) atomicAdd(reinterpret_cast<unsigned *>(ws + kWsFallbackOff), 1u);  // diagnostic
+            exact_ok = s_inexact[0] == 0;
         }
 
         // ---- consume this warp's slice of the stage ------------------------------------------------
@@ -300,12 +331,20 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
 
         if (!(flags & kFlagSegLast)) continue;
 
-        // ---- end of this CTA's share of a (window, tile) pair: combine the 16 warps ---------------
+        // ---- end of a (window, tile) pair -----------------------------------------------------------------
+        // Each warp leaves its partial tile in red[rslot][warp]; the last warp to arrive sums them in warp
+        // order and finishes the pair.  No CTA-wide barrier: the other warps move on to the next tile.
         const int tile_now = e.w & 0xFFFFF, w_now = e.w >> 20;
-        const int seg_b1 = b_now + nblk_now;
-        const int nseg_blocks = seg_b1 - seg_b0;
+        const int rslot = seg_index % kRedSlots;
+        {   // the slot's previous pair (kRedSlots pairs ago) must have been summed.  The wait is bounded;
+            // if it ever gave up the result would be wrong, which the parity tests would show.
+            const int need = seg_index / kRedSlots;
+            int spins = 0;
+            while (*reinterpret_cast<volatile int *>(&s_gen[rslot]) < need && ++spins < (1 << 24)) {
+            }
+        }
+        float *mine = s_red + (rslot * kMmaWarps + warp) * kOut;
         if (exact_ok) {
-            float *mine = s_red + warp * kOutPerWarp;
 #pragma unroll
             for (int n = 0; n < NT8; ++n) {
                 mine[(8 * n + 2 * t) * kTileRows + g] = acc[n][0];
@@ -315,14 +354,19 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
                 acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
             }
         } else {
-            // scalar FP32 path for X that does not fit FP16 exactly: warp r computes tile row r directly
-            // from global memory (same late scaling, FP32 accumulation), for every token
-            const int64_t row = min((int64_t)tile_now * kTileRows + warp, p.N - 1);
+            // scalar FP32 path for X that does not fit FP16 exactly: warp r computes tile rows r and r + 8
+            // directly from global memory (same late scaling, FP32 accumulation), for every token; its partial
+            // tile is zero everywhere else, so the common sum below still applies
+            const int bwid = (w_now == p.nwin - 1) ? p.bw_last : p.bw;
             const int64_t j0 = (int64_t)w_now * p.bw;
-            for (int m = 0; m < NT8 * 8; ++m) {
-                float a = 0.f;
-                if (m < p.M) {
-                    for (int j = seg_b0 + lane; j < seg_b1; j += 32) {
+            for (int i = lane; i < kOut; i += 32) mine[i] = 0.f;
+            __syncwarp();
+            for (int half = 0; half < 2; ++half) {
+                const int64_t row = r0 + (int64_t)tile_now * kTileRows + warp + 8 * half;
+                if (row >= r1) continue;
+                for (int m = 0; m < p.M; ++m) {
+                    float a = 0.f;
+                    for (int j = lane; j < bwid; j += 32) {
                         const uint4 c = ld_stream_u4(codes + row * (p.K / 2) + (j0 + j) * 16);
                         const float s = e8m0_to_float(scales[row * p.kb + j0 + j]);
                         const uint32_t w4[4] = {c.x, c.y, c.z, c.w};
@@ -340,59 +384,51 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
                         a = fmaf(part, s, a);
                     }
                     a = warp_sum(a);
+                    if (lane == 0) mine[m * kTileRows + warp + 8 * half] = a;  // [token][row]
                 }
-                if (lane == 0) s_red[m * kTileRows + warp] = a;  // [token][row]
             }
         }
-        __syncthreads();
-
-        const bool whole = (p.nwin == 1) && (seg_b0 == 0) && (seg_b1 == p.bw_last);
-        float val = 0.f;
-        const int m_out = tid / kTileRows, r_out = tid % kTileRows;
-        const int64_t n_out = (int64_t)tile_now * kTileRows + r_out;
-        if (tid < kOutPerWarp) {
-            if (exact_ok) {
+        __threadfence_block();
+        __syncwarp();
+        int arrived = 0;
+        if (lane == 0) arrived = atomicAdd(&s_cnt[rslot], 1);
+        arrived = __shfl_sync(0xffffffffu, arrived, 0);
+        if (arrived == kMmaWarps - 1) {
+            // last warp in: sum the partial tiles in warp order
+            __threadfence_block();
+            float val[kPerLane];
+            const float *all = s_red + rslot * kMmaWarps * kOut;
 #pragma unroll
-                for (int w = 0; w < kMmaWarps; ++w) val += s_red[w * kOutPerWarp + tid];
-            } else {
-                val = s_red[tid];
+            for (int i = 0; i < kPerLane; ++i) {
+                float v = 0.f;
+#pragma unroll
+                for (int w = 0; w < kMmaWarps; ++w) v += all[w * kOut + lane + 32 * i];
+                val[i] = v;
             }
-            if (whole) {
-                if (m_out < p.M && n_out < p.N) store_out(Y, y_dtype, (int64_t)m_out * p.N + n_out, val);
-            } else {
-                partials[((size_t)blockIdx.x * p.slots + seg_index) * kOutPerWarp + tid] = val;
-                __threadfence();
+            __syncwarp();
+            if (lane == 0) {
+                s_cnt[rslot] = 0;
+                __threadfence_block();
+                *reinterpret_cast<volatile int *>(&s_gen[rslot]) = seg_index / kRedSlots + 1;  // slot free again
             }
-        }
-        __syncthreads();
-        if (!whole) {
-            if (tid == 0) {
-                const unsigned done = atomicAdd(&tickets[tile_now], (unsigned)nseg_blocks) + (unsigned)nseg_blocks;
-                s_flags[1] = (done == (unsigned)p.kb);
-                if (done == (unsigned)p.kb) tickets[tile_now] = 0;  // ready for the next call
-            }
-            __syncthreads();
-            if (s_flags[1]) {
-                __threadfence();
-                if (tid < kOutPerWarp) {
-                    // sum every CTA's share of this tile in unit order
-                    float sum = 0.f;
-                    for (int w = 0; w < p.nwin; ++w) {
-                        const uint32_t pb = pair_begin(p, w, tile_now);
-                        const uint32_t pe = pb + (uint32_t)((w == p.nwin - 1) ? p.bw_last : p.bw);
-                        const int c0 = cta_of(p, pb), c1 = cta_of(p, pe - 1);
-                        const int pair_id = w * p.tiles + tile_now;
-                        for (int c = c0; c <= c1; ++c) {
-                            int fw, ft, fb;
-                            unit_decode(p, cta_begin(p, c), fw, ft, fb);
-                            const int slot_i = pair_id - (fw * p.tiles + ft);
-                            sum += __ldcg(&partials[((size_t)c * p.slots + slot_i) * kOutPerWarp + tid]);
-                        }
-                    }
-                    if (m_out < p.M && n_out < p.N) store_out(Y, y_dtype, (int64_t)m_out * p.N + n_out, sum);
+            if (p.nwin > 1) {
+                // windows are walked in order and each pair has exactly one summing warp, so the order of
+                // these additions is fixed
+                float *ta = s_acc + tile_now * kOut;
+#pragma unroll
+                for (int i = 0; i < kPerLane; ++i) {
+                    if (w_now > 0) val[i] += ta[lane + 32 * i];
+                    if (w_now < p.nwin - 1) ta[lane + 32 * i] = val[i];
                 }
             }
-            __syncthreads();
+            if (w_now == p.nwin - 1) {
+#pragma unroll
+                for (int i = 0; i < kPerLane; ++i) {
+                    const int idx = lane + 32 * i, m_out = idx / kTileRows;
+                    const int64_t n_out = r0 + (int64_t)tile_now * kTileRows + idx % kTileRows;
+                    if (m_out < p.M && n_out < r1) store_out(Y, y_dtype, (int64_t)m_out * p.N + n_out, val[i]);
+                }
+            }
         }
         ++seg_index;
     }
@@ -404,69 +440,67 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
 // ---------------------------------------------------------------------------------------------
 bool linear_mma_plan(int M, int64_t N, int64_t K, LinearPlan &p) {
     if (M < 1 || M > 16 || (K % 128) != 0 || N < 1) return false;
-    const int64_t tiles = (N + kTileRows - 1) / kTileRows;
     const int64_t kb = K / 32;
-    if (tiles > kTicketCap || tiles * kb >= (int64_t)1 << 31 || N * (K / 2) >= (int64_t)1 << 32) return false;
+    if (kb > 65535 || N * (K / 2) >= (int64_t)1 << 32) return false;
     p.M = M;
     p.nt8 = M <= 8 ? 1 : 2;
-    p.tiles = (int)tiles;
     p.kb = (int)kb;
     p.N = N;
     p.K = K;
-    p.units = (uint32_t)(tiles * kb);
-    const uint32_t red_bytes = (uint32_t)kMmaWarps * p.nt8 * 8 * kTileRows * 4;
-    p.off_x = kOffRed + red_bytes;
-    // ring depth and K windows: prefer 4 stages and one window; give up stages, then split K
-    auto layout = [&](int nstage, int64_t bw) {  // fills the offsets for a window of bw blocks; returns total bytes
-        p.x_stride = (uint32_t)(2 * bw * 32 + 64);
-        p.off_ring = (p.off_x + (uint32_t)M * p.x_stride + 127) / 128 * 128;
-        p.smem_bytes = p.off_ring + (uint32_t)(kMmaWarps * nstage * kWarpStageBytes);
-        return p.smem_bytes;
-    };
-    int nstage = kMaxStages, nwin = 1;
-    int64_t bw = kb;
-    while (nstage > 2 && layout(nstage, bw) > kSmemBudget) --nstage;
-    while (layout(nstage, bw) > kSmemBudget) {
-        if (++nwin > 64) return false;
-        bw = ((kb + nwin - 1) / nwin + 3) / 4 * 4;
-    }
-    while ((int64_t)(nwin - 1) * bw >= kb) --nwin;  // rounding up may have left the last window empty
-    p.nstage = nstage;
-    p.nwin = nwin;
-    p.bw = (int)bw;
-    p.bw_last = (int)(kb - (int64_t)(nwin - 1) * bw);
-    // one CTA per SM; more (a multiple of the SM count) only if a CTA's stage table would not fit
-    const int min_bw = p.bw_last < p.bw ? p.bw_last : p.bw;
-    const uint32_t groups = p.units / 4;
     const int sms = sm_count();
-    for (int mult = 1;; ++mult) {
-        int grid = sms * mult;
-        if ((uint32_t)grid > groups) grid = (int)groups;
-        const uint32_t per_cta = (p.units + grid - 1) / grid + 4;
-        const uint32_t stages_bound = per_cta / kStageBlocks + per_cta / (uint32_t)min_bw + (uint32_t)p.nwin + 3;
-        if (stages_bound <= (uint32_t)kMaxCtaStages || (uint32_t)grid == groups) {
-            if (stages_bound > (uint32_t)kMaxCtaStages) return false;
-            p.grid = grid;
-            p.slots = (int)(per_cta / min_bw) + 3;
-            return true;
+    const uint32_t kout_bytes = (uint32_t)p.nt8 * 8 * kTileRows * 4;
+    const uint32_t red_bytes = (uint32_t)kRedSlots * kMmaWarps * kout_bytes;
+
+    // grid: two CTAs per SM, more only if a CTA's stage table would overflow; never more CTAs than rows
+    for (int mult = 2; mult <= 4096; mult *= 2) {
+        int64_t grid = (int64_t)sms * mult;
+        if (grid > N) grid = N;
+        p.grid = (int)grid;
+        const int64_t max_rows = (N + grid - 1) / grid;
+        p.max_tiles = (int)((max_rows + kTileRows - 1) / kTileRows);
+
+        // ring depth and K windows: prefer a quarter of an SM, 4 stages, one window
+        auto layout = [&](int nstage, int64_t bw, int nwin) {
+            p.off_acc = kOffRed + red_bytes;
+            p.off_x = p.off_acc + (nwin > 1 ? (uint32_t)p.max_tiles * kout_bytes : 0u);
+            p.x_stride = (uint32_t)(2 * bw * 32 + 64);
+            p.off_ring = (p.off_x + (uint32_t)M * p.x_stride + 127) / 128 * 128;
+            p.smem_bytes = p.off_ring + (uint32_t)(kMmaWarps * nstage * kWarpStageBytes);
+            return p.smem_bytes;
+        };
+        int nstage = kMaxStages, nwin = 1;
+        int64_t bw = kb;
+        if (layout(nstage, bw, nwin) > kSmemQuarterSm) {
+            while (nstage > 2 && layout(nstage, bw, nwin) > kSmemHalfSm) --nstage;
+            while (layout(nstage, bw, nwin) > kSmemHalfSm) {
+                if (++nwin > 64) return false;
+                bw = ((kb + nwin - 1) / nwin + 3) / 4 * 4;
+            }
+            while ((int64_t)(nwin - 1) * bw >= kb) --nwin;  // rounding up may have left the last window empty
+            layout(nstage, bw, nwin);
         }
-        if (mult > 4096) return false;
+        p.nstage = nstage;
+        p.nwin = nwin;
+        p.bw = (int)bw;
+        p.bw_last = (int)(kb - (int64_t)(nwin - 1) * bw);
+        StageInfo si;
+        if (stage_lookup(p, p.max_tiles, -1, si) <= kMaxCtaStages && p.smem_bytes <= kSmemHalfSm) return true;
+        if (grid == N) return false;
     }
+    return false;
 }
 
-size_t linear_mma_workspace_bytes(const LinearPlan &p) {
-    return kWsPartialOff + (size_t)p.grid * p.slots * (size_t)(p.nt8 * 8 * kTileRows) * sizeof(float);
-}
+size_t linear_mma_workspace_bytes(const LinearPlan &) { return 0; }
 
 template <int NT8, int NS>
 static cudaError_t launch_mma(const LinearPlan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,
-                              int y_dtype, void *ws, cudaStream_t stream) {
+                              int y_dtype, cudaStream_t stream) {
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(linear_mma_kernel<NT8, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)kSmemBudget);
+                                             (int)kSmemHalfSm);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -480,13 +514,12 @@ static cudaError_t launch_mma(const LinearPlan &p, const void *X, const uint8_t 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl_enabled() ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, linear_mma_kernel<NT8, NS>, p, (const uint16_t *)X, codes, scales, Y, y_dtype,
-                              (uint8_t *)ws);
+    return cudaLaunchKernelEx(&cfg, linear_mma_kernel<NT8, NS>, p, (const uint16_t *)X, codes, scales, Y, y_dtype);
 }
 
 cudaError_t linear_mma_launch(const LinearPlan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,
-                              int y_dtype, void *ws, cudaStream_t stream) {
-#define MXQ_LAUNCH(NT, NSTG) launch_mma<NT, NSTG>(p, X, codes, scales, Y, y_dtype, ws, stream)
+                              int y_dtype, void *, cudaStream_t stream) {
+#define MXQ_LAUNCH(NT, NSTG) launch_mma<NT, NSTG>(p, X, codes, scales, Y, y_dtype, stream)
     if (p.nt8 == 1) return p.nstage == 4 ? MXQ_LAUNCH(1, 4) : (p.nstage == 3 ? MXQ_LAUNCH(1, 3) : MXQ_LAUNCH(1, 2));
     return p.nstage == 4 ? MXQ_LAUNCH(2, 4) : (p.nstage == 3 ? MXQ_LAUNCH(2, 3) : MXQ_LAUNCH(2, 2));
 #undef MXQ_LAUNCH

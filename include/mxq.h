@@ -138,6 +138,34 @@ int mxq_greedy_accept(const void *logits, int logits_dtype, int64_t B, int R, in
                       int T, int32_t *accept_len, int32_t *next_token, void *workspace, size_t workspace_bytes,
                       void *stream);
 
+/* mxq_greedy_accept for callers that cannot hand over a workspace because they cannot allocate
+ * one.  (The paper has no counterpart: this entry point exists for the library's users, not for
+ * the method.)  Who that is: code that runs inside someone else's process with the device memory
+ * already given out -- an inference server that sized its pools at start-up and forbids further
+ * cudaMalloc, a plugin that is handed input and output buffers and nothing else, a latency-critical
+ * loop where the device-wide synchronisation an allocation implies is not acceptable.
+ *
+ * Same arguments and results as mxq_greedy_accept minus the workspace.  The scratch (ticket
+ * counters and per-slice partial maxima) lives in an array built into the library,
+ * mxq_greedy_accept_static_max_bytes() bytes (1 MiB) on every GPU that loads the library, for the
+ * life of the process.  The call allocates and frees nothing.
+ *   - A shape whose scratch (mxq_accept_workspace_bytes) exceeds that size is refused with
+ *     MXQ_ERR_WORKSPACE; use mxq_greedy_accept with your own workspace instead.
+ *   - The first call on each device asks the CUDA runtime once for the array's device address
+ *     (with that device current) and remembers it; make that first call outside any stream
+ *     capture.  A failure of that query returns MXQ_ERR_CUDA.
+ *   - All calls on a device share the one array, and it keeps what the previous call left in it
+ *     (each call re-zeroes the counters it needs on `stream` before launching).  Two calls that may
+ *     run on the GPU at the same time -- different streams, or different host threads -- race on
+ *     it and may return wrong results; serialise them, or give each its own workspace through
+ *     mxq_greedy_accept. */
+int mxq_greedy_accept_static(const void *logits, int logits_dtype, int64_t B, int R, int64_t V,
+                             const int32_t *draft, int T, int32_t *accept_len, int32_t *next_token,
+                             void *stream);
+
+/* Size in bytes of the built-in scratch array of mxq_greedy_accept_static. */
+size_t mxq_greedy_accept_static_max_bytes(void);
+
 /* Same, with the verifier's tokens already known: verifier [B][R] int32. */
 int mxq_greedy_accept_tokens(const int32_t *draft, const int32_t *verifier, int64_t B, int T, int R,
                              int32_t *accept_len, int32_t *next_token, void *stream);

@@ -64,6 +64,10 @@ def lib() -> ctypes.CDLL:
             L.mxq_linear_host.argtypes = [vp, i32, vp, vp, i64, i64, vp, i32, vp, vp, vp, sz, vp]
             L.mxq_greedy_accept.restype = i32
             L.mxq_greedy_accept.argtypes = [vp, i32, i64, i32, i64, vp, i32, vp, vp, vp, sz, vp]
+            L.mxq_greedy_accept_static.restype = i32
+            L.mxq_greedy_accept_static.argtypes = [vp, i32, i64, i32, i64, vp, i32, vp, vp, vp]
+            L.mxq_greedy_accept_static_max_bytes.restype = sz
+            L.mxq_greedy_accept_static_max_bytes.argtypes = []
             L.mxq_greedy_accept_tokens.restype = i32
             L.mxq_greedy_accept_tokens.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp]
             _lib = L
@@ -229,6 +233,26 @@ def mxq_greedy_accept(logits: torch.Tensor, draft: torch.Tensor, workspace: torc
                                    _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)),
            "mxq_greedy_accept")
     return g, nxt
+
+
+def mxq_greedy_accept_static_max_bytes() -> int:
+    return int(lib().mxq_greedy_accept_static_max_bytes())
+
+
+def mxq_greedy_accept_static(logits: torch.Tensor, draft: torch.Tensor, accept_len: torch.Tensor,
+                             next_token: torch.Tensor, stream=None) -> None:
+    """mxq_greedy_accept without a workspace, for callers that cannot allocate one: the scratch is an array
+    built into the library (1 MiB per GPU).  The caller passes the outputs too (int32 [B] each); nothing is
+    allocated on the way.  Calls on one device share that array, so calls that may overlap on the GPU race."""
+    b, r, v = logits.shape
+    t = draft.shape[1]
+    if tuple(accept_len.shape) != (b,) or tuple(next_token.shape) != (b,):
+        raise ValueError("accept_len and next_token must be int32 tensors of shape [B]")
+    _check(lib().mxq_greedy_accept_static(_dev(logits, logits.dtype, "logits"), _dt(logits.dtype), b, r, v,
+                                          _dev(draft, torch.int32, "draft"), t,
+                                          _dev(accept_len, torch.int32, "accept_len"),
+                                          _dev(next_token, torch.int32, "next_token"), _stream(stream)),
+           "mxq_greedy_accept_static")
 
 
 def mxq_greedy_accept_tokens(draft: torch.Tensor, verifier: torch.Tensor, stream=None):

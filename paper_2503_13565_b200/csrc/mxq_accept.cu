@@ -181,6 +181,32 @@ static bool accept_shape_ok(int64_t B, int R, int64_t V, int T) {
            B * (int64_t)R <= (int64_t)INT_MAX / 1024;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Built-in scratch for mxq_greedy_accept_static: lives in the library image, so every GPU that
+// loads the library holds these bytes until the process exits.  Same layout as the caller-provided
+// workspace of mxq_greedy_accept: ticket counters first, then the per-slice (value, index) pairs.
+// ---------------------------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = (size_t)1 << 20;  // 1 MiB
+static __device__ __align__(256) unsigned char g_accept_scratch[kStaticScratchBytes];
+
+// Device address of g_accept_scratch on the current device.  In host code the array's name is only a
+// handle for the runtime, never a device address, so the address is asked for once per device (with that
+// device current) and remembered.  Returns nullptr if the runtime refuses.
+static void *static_scratch_for_current_device() {
+    static void *cached[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (cached[dev] == nullptr) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_accept_scratch) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        cached[dev] = ptr;
+    }
+    return cached[dev];
+}
+
 }  // namespace mxq
 
 extern "C" {
@@ -226,6 +252,40 @@ int mxq_greedy_accept_tokens(const int32_t *draft, const int32_t *verifier, int6
     mxq::accept_tokens_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(draft, verifier, B, T, R, accept_len, next_token);
     return mxq::launch_status();
 }
+
+int mxq_greedy_accept_static(const void *logits, int logits_dtype, int64_t B, int R, int64_t V, const int32_t *draft,
+                             int T, int32_t *accept_len, int32_t *next_token, void *stream) {
+    if (!logits || !draft || !accept_len || !next_token) return MXQ_ERR_NULL;
+    if (!mxq::accept_shape_ok(B, R, V, T)) return MXQ_ERR_SHAPE;
+    if (logits_dtype != MXQ_F32 && logits_dtype != MXQ_BF16) return MXQ_ERR_DTYPE;
+    if (!mxq::aligned16(logits)) return MXQ_ERR_ALIGN;
+    // the scratch this shape needs must fit the built-in array; nothing is ever allocated to make room
+    if (mxq_accept_workspace_bytes(B, R, V) > mxq::kStaticScratchBytes) return MXQ_ERR_WORKSPACE;
+    void *scratch = mxq::static_scratch_for_current_device();  // first call on a device: one runtime query
+    if (!scratch) return MXQ_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    // the array keeps whatever the previous call left; the ticket counters must start at zero
+    if (cudaMemsetAsync(scratch, 0, mxq::ticket_bytes(), st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MXQ_ERR_CUDA;
+    }
+    const mxq::Slicing s = mxq::slicing_for(B, R, V);
+    unsigned *tickets = (unsigned *)scratch;
+    mxq::Best *partial = (mxq::Best *)((char *)scratch + mxq::ticket_bytes());
+    const unsigned grid = (unsigned)(B * R * s.slices);
+    if (logits_dtype == MXQ_F32) {
+        mxq::greedy_accept_kernel<float><<<grid, mxq::kAcceptThreads, 0, st>>>(
+            (const float *)logits, B, R, V, s.slices, s.slice_len, (V % 4) == 0, draft, T, accept_len, next_token, partial,
+            tickets);
+    } else {
+        mxq::greedy_accept_kernel<uint16_t><<<grid, mxq::kAcceptThreads, 0, st>>>(
+            (const uint16_t *)logits, B, R, V, s.slices, s.slice_len, (V % 8) == 0, draft, T, accept_len, next_token,
+            partial, tickets);
+    }
+    return mxq::launch_status();
+}
+
+size_t mxq_greedy_accept_static_max_bytes(void) { return mxq::kStaticScratchBytes; }
 
 #pragma GCC visibility pop
 }  // extern "C"

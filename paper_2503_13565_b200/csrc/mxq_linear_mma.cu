@@ -18,17 +18,19 @@
 // CTA streams the same number of bytes to within one row, no output is shared between CTAs,
 // and there is no workspace.  The rows are processed as 16-row tiles (the last one ragged:
 // missing rows are neither fetched nor stored).  Within a CTA the 8 warps split each stage's
-// 32 MX blocks; every warp leaves its FP32 partial tile in shared memory and the warp that
+// 64 MX blocks; every warp leaves its FP32 partial tile in shared memory and the warp that
 // arrives last (a counter, not a barrier) sums the 8 in warp order, so results are
 // bit-reproducible.  When M*K is too large for X to fit in shared memory, K is cut into
 // windows; the CTA walks its tiles once per window and keeps per-tile sums in shared memory.
 //
 // Pipeline: every warp runs its own ring of 16-byte cp.async copies for exactly the bytes it
-// will consume (16 rows x 64 code bytes + 16 x 4 scale bytes per stage), so the main loop has
+// will consume (16 rows x 128 code bytes + 16 x 8 scale bytes per stage), so the main loop has
 // no CTA-wide barrier and no spin-wait.  Weights never depend on the previous kernel, so the
 // ring is filled before griddepcontrol.wait (programmatic dependent launch); X and Y are
 // touched only after it.  A CTA is small enough that two kernels, two CTAs per SM each, can be
 // resident: the next kernel prefetches while this one computes.
+#include <cstdlib>
+
 #include "mxq_device.cuh"
 #include "mxq_host.h"
 #include "mxq_linear_plan.h"
@@ -43,6 +45,9 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)_
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
+__device__ __forceinline__ void cp_async8(uint32_t dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+}
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
@@ -50,6 +55,11 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
 }
 __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
     uint32_t v;
@@ -61,13 +71,18 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
-// four code bytes -> four FP16 pairs (low nibble in the low half)
+// low byte of v (two E2M1 codes) -> FP16 pair, low nibble in the low half; the upper bits of v are ignored
+__device__ __forceinline__ uint32_t e2m1x2_lowbyte_to_half2(uint32_t v) {
+    uint32_t out;
+    asm("{\n\t.reg .b8 b;\n\tcvt.u8.u32 b, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}" : "=r"(out) : "r"(v));
+    return out;
+}
+// four code bytes -> four FP16 pairs: one shift per byte beyond the first, one conversion per byte
 __device__ __forceinline__ void e2m1x8_to_half2x4(uint32_t word, uint32_t &p0, uint32_t &p1, uint32_t &p2, uint32_t &p3) {
-    asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\tmov.b32 {b0, b1, b2, b3}, %4;\n\t"
-        "cvt.rn.f16x2.e2m1x2 %0, b0;\n\tcvt.rn.f16x2.e2m1x2 %1, b1;\n\t"
-        "cvt.rn.f16x2.e2m1x2 %2, b2;\n\tcvt.rn.f16x2.e2m1x2 %3, b3;\n\t}"
-        : "=r"(p0), "=r"(p1), "=r"(p2), "=r"(p3)
-        : "r"(word));
+    p0 = e2m1x2_lowbyte_to_half2(word);
+    p1 = e2m1x2_lowbyte_to_half2(word >> 8);
+    p2 = e2m1x2_lowbyte_to_half2(word >> 16);
+    p3 = e2m1x2_lowbyte_to_half2(word >> 24);
 }
 // two E8M0 bytes (low 16 bits of v) -> BF16 pair; 0 -> 2^-127 (a BF16 subnormal), 0xFF -> NaN
 __device__ __forceinline__ uint32_t e8m0x2_to_bf16x2(uint32_t v) {
@@ -77,7 +92,7 @@ __device__ __forceinline__ uint32_t e8m0x2_to_bf16x2(uint32_t v) {
 }
 __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                         uint32_t b1, const float (&c)[4]) {
-    asm volatile(
+    asm(
         "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
         : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(c[0]), "f"(c[1]), "f"(c[2]), "f"(c[3]));
@@ -127,7 +142,7 @@ __device__ __forceinline__ int bf16x8_to_f16x8(const uint4 &v, float up, uint4 &
 // ---------------------------------------------------------------------------------------------
 // NT8: 8-token column tiles (1 for M <= 8, 2 for M <= 16); NS: ring depth
 template <int NT8, int NS>
-__global__ void __launch_bounds__(kMmaThreads, 4)
+__global__ void __launch_bounds__(kMmaThreads, 2)
 linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restrict__ X,
                   const uint8_t *__restrict__ codes, const uint8_t *__restrict__ scales, void *__restrict__ Y,
                   int y_dtype) {
@@ -173,23 +188,40 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
     // ---- per-lane constants ---------------------------------------------------------------------------
     const int blk0 = warp * kWarpBlocks;  // this warp's blocks within a stage
     const uint32_t ring = sbase + p.off_ring + (uint32_t)warp * (uint32_t)(NS * kWarpStageBytes);
-    // copy role of this lane: rows cr and cr + 8 of the tile, 16-byte chunk cc (= block within the slice);
-    // lanes 0..15 also copy the 4 scale bytes of row `lane`
-    const uint32_t cr = lane & 7, cc = lane >> 3;
+    // Copy role of this lane.  Four consecutive lanes fetch 64 contiguous bytes of one row (lanes that split a
+    // 32-byte sector between two quarter-warps halve the L2 -> SM rate: measured 4.1 vs 6.4 TB/s), so a
+    // quarter-warp covers rows r and r + 4.  In shared memory row r keeps its 8 chunks at (chunk ^ (r & 7)),
+    // which makes both these writes and the fragment reads (8 rows, one chunk) bank-conflict free.
+    // lane -> rows cr and cr + 8 of the tile, chunks cc and cc + 4; lanes 0..15 also copy row `lane`'s 8 scale bytes
+    const uint32_t cc = lane & 3, cr = ((lane >> 2) & 1) * 4 + (lane >> 3);
     const uint32_t row_bytes = (uint32_t)(p.K / 2);
-    const uint32_t dst_lo = cc * 256 + cr * 16, dst_sc = kWarpCodeBytes + (lane & 15) * 4;
+    const uint32_t dst_a = cr * 128 + ((cc ^ cr) << 4), dst_b = cr * 128 + (((cc + 4) ^ cr) << 4);
+    const uint32_t dst_sc = kWarpCodeBytes + (lane & 15) * 8 + (lane >> 4) * 4;
     const uint8_t *src_lo = codes + (blk0 + cc) * 16 + (size_t)cr * row_bytes;
     const uint8_t *src_hi = src_lo + (size_t)8 * row_bytes;
-    const uint8_t *src_sc = scales + blk0 + (size_t)(lane & 15) * (uint32_t)p.kb;
+    const uint8_t *src_sc = scales + blk0 + (lane >> 4) * 4 + (size_t)(lane & 15) * (uint32_t)p.kb;
+    const bool sc8 = (p.kb % 8) == 0;   // scale rows 8-byte aligned: one 8-byte copy per row instead of two 4-byte ones
 
     auto issue = [&](int q, int slot) {
         const uint4 e = s_table[q];
-        const uint32_t nblk = (e.z >> 16) & 0xFF, rows_m1 = e.z >> 28;
-        if ((uint32_t)blk0 < nblk) {
+        const int left = (int)((e.z >> 16) & 0xFF) - blk0;   // blocks of this stage from this warp's first one on
+        const uint32_t rows_m1 = e.z >> 28;
+        if (left > 0) {
             const uint32_t dst = ring + (uint32_t)slot * kWarpStageBytes;
-            if (cr <= rows_m1) cp_async16(dst + dst_lo, src_lo + e.x);
-            if (cr + 8 <= rows_m1) cp_async16(dst + dst_lo + 128, src_hi + e.x);
-            if ((uint32_t)lane <= rows_m1) cp_async4(dst + dst_sc, src_sc + e.y);  // rows_m1 <= 15: lanes 0..15 at most
+            const bool lo_ok = cr <= rows_m1, hi_ok = cr + 8 <= rows_m1, sc_ok = (uint32_t)(lane & 15) <= rows_m1;
+            if (lo_ok) cp_async16(dst + dst_a, src_lo + e.x);
+            if (hi_ok) cp_async16(dst + dst_a + 1024, src_hi + e.x);
+            if (left > 4) {
+                if (lo_ok) cp_async16(dst + dst_b, src_lo + e.x + 64);
+                if (hi_ok) cp_async16(dst + dst_b + 1024, src_hi + e.x + 64);
+                if (sc8) {
+                    if (lane < 16 && sc_ok) cp_async8(dst + dst_sc, src_sc + e.y);
+                } else if (sc_ok) {
+                    cp_async4(dst + dst_sc, src_sc + e.y);
+                }
+            } else if (lane < 16 && sc_ok) {
+                cp_async4(dst + dst_sc, src_sc + e.y);
+            }
         }
     };
 
@@ -208,7 +240,9 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
         for (int i = 0; i < 4; ++i) acc[n][i] = 0.f;
 
     // per-thread constants of the fragment reads
-    const uint32_t a_off = (uint32_t)(g * 16 + 4 * t);                       // + jb*256 (+128 for row g+8)
+    // row g's chunk jb sits at g*128 + ((jb ^ g) << 4): with the slot 128-byte aligned that is
+    // (slot + a_off) ^ (jb << 4); row g + 8 is 1024 bytes further
+    const uint32_t a_off = (uint32_t)(g * 128 + (g << 4) + 4 * t);
     // B fragment: token g (and g + 8).  Lanes whose token does not exist read the last real token instead:
     // a column of B only ever feeds the same column of the result, and those columns are never stored.
     const uint32_t x_thread0 = sbase + p.off_x + (uint32_t)blk0 * 64u + 16u * t + (uint32_t)min(g, p.M - 1) * p.x_stride;
@@ -288,41 +322,58 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
         // ---- consume this warp's slice of the stage ------------------------------------------------
         cp_async_wait<NS - 1>();  // all but the newest NS-1 groups have landed: this stage is in
         __syncwarp();
-        if (exact_ok && blk0 < nblk_now) {
+        const int left = nblk_now - blk0;  // blocks of this stage that are this warp's: 8, 4 or none
+        if (exact_ok && left > 0) {
             const uint32_t cbase = ring + (uint32_t)slot * kWarpStageBytes;
-            // the four blocks' scales of rows g and g+8; 2^-shift of X is folded in here (8 multiplies per stage)
-            const uint32_t sw_lo = lds32(cbase + kWarpCodeBytes + g * 4), sw_hi = lds32(cbase + kWarpCodeBytes + g * 4 + 32);
-            const uint32_t sl01 = e8m0x2_to_bf16x2(sw_lo), sl23 = e8m0x2_to_bf16x2(sw_lo >> 16);
-            const uint32_t sh01 = e8m0x2_to_bf16x2(sw_hi), sh23 = e8m0x2_to_bf16x2(sw_hi >> 16);
-            const float sc_lo[4] = {__uint_as_float(sl01 << 16) * un, __uint_as_float(sl01 & 0xFFFF0000u) * un,
-                                    __uint_as_float(sl23 << 16) * un, __uint_as_float(sl23 & 0xFFFF0000u) * un};
-            const float sc_hi[4] = {__uint_as_float(sh01 << 16) * un, __uint_as_float(sh01 & 0xFFFF0000u) * un,
-                                    __uint_as_float(sh23 << 16) * un, __uint_as_float(sh23 & 0xFFFF0000u) * un};
             const uint32_t abase = cbase + a_off;
             const uint32_t xbase0 = x_thread0 + (uint32_t)b_now * 64u, xbase1 = x_thread1 + (uint32_t)b_now * 64u;
-            const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+            const uint2 sw_lo = lds64(cbase + kWarpCodeBytes + g * 8), sw_hi = lds64(cbase + kWarpCodeBytes + g * 8 + 64);
+            auto four_blocks = [&](uint32_t s_lo, uint32_t s_hi, int jb0) {
+                // all shared-memory reads of the four blocks first, so that their latencies overlap
+                uint32_t a_lo[4], a_hi[4];
+                uint4 xb[4][NT8];
 #pragma unroll
-            for (int jb = 0; jb < kWarpBlocks; ++jb) {
-                // A: this lane's 8 weights of rows g and g+8 of block jb (k = 8t .. 8t+7 of the block)
-                const uint32_t a_lo = lds32(abase + jb * 256);
-                const uint32_t a_hi = lds32(abase + jb * 256 + 128);
-                uint32_t l0, l1, l2, l3, h0, h1, h2, h3;
-                e2m1x8_to_half2x4(a_lo, l0, l1, l2, l3);
-                e2m1x8_to_half2x4(a_hi, h0, h1, h2, h3);
+                for (int i = 0; i < 4; ++i) {
+                    // A: this lane's 8 weights of rows g and g+8 of block jb (k = 8t .. 8t+7 of the block)
+                    a_lo[i] = lds32(abase ^ (uint32_t)((jb0 + i) << 4));
+                    a_hi[i] = lds32((abase ^ (uint32_t)((jb0 + i) << 4)) + 1024);
+                    // B: the same 8 k of token g (+8 for the second column tile)
+#pragma unroll
+                    for (int n = 0; n < NT8; ++n) xb[i][n] = lds128((n == 0 ? xbase0 : xbase1) + (jb0 + i) * 64);
+                }
+                // the four blocks' scales of rows g and g+8; 2^-shift of X is folded in here
+                const uint32_t sl01 = e8m0x2_to_bf16x2(s_lo), sl23 = e8m0x2_to_bf16x2(s_lo >> 16);
+                const uint32_t sh01 = e8m0x2_to_bf16x2(s_hi), sh23 = e8m0x2_to_bf16x2(s_hi >> 16);
+                const float sc_lo[4] = {__uint_as_float(sl01 << 16) * un, __uint_as_float(sl01 & 0xFFFF0000u) * un,
+                                        __uint_as_float(sl23 << 16) * un, __uint_as_float(sl23 & 0xFFFF0000u) * un};
+                const float sc_hi[4] = {__uint_as_float(sh01 << 16) * un, __uint_as_float(sh01 & 0xFFFF0000u) * un,
+                                        __uint_as_float(sh23 << 16) * un, __uint_as_float(sh23 & 0xFFFF0000u) * un};
+                const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+                uint32_t l[4][4], h[4][4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    e2m1x8_to_half2x4(a_lo[i], l[i][0], l[i][1], l[i][2], l[i][3]);
+                    e2m1x8_to_half2x4(a_hi[i], h[i][0], h[i][1], h[i][2], h[i][3]);
+                }
 #pragma unroll
                 for (int n = 0; n < NT8; ++n) {
-                    // B: the same 8 k of token g (+8 for the second column tile)
-                    const uint4 xb = lds128((n == 0 ? xbase0 : xbase1) + jb * 64);
-                    float part[4];
-                    mma_f16(part, l0, h0, l1, h1, xb.x, xb.y, zero);
-                    mma_f16(part, l2, h2, l3, h3, xb.z, xb.w, part);
+                    float part[4][4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) mma_f16(part[i], l[i][0], h[i][0], l[i][1], h[i][1], xb[i][n].x, xb[i][n].y, zero);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) mma_f16(part[i], l[i][2], h[i][2], l[i][3], h[i][3], xb[i][n].z, xb[i][n].w, part[i]);
                     // late scaling (Eq. 2): one multiply per 32-long partial sum
-                    acc[n][0] = fmaf(part[0], sc_lo[jb], acc[n][0]);
-                    acc[n][1] = fmaf(part[1], sc_lo[jb], acc[n][1]);
-                    acc[n][2] = fmaf(part[2], sc_hi[jb], acc[n][2]);
-                    acc[n][3] = fmaf(part[3], sc_hi[jb], acc[n][3]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        acc[n][0] = fmaf(part[i][0], sc_lo[i], acc[n][0]);
+                        acc[n][1] = fmaf(part[i][1], sc_lo[i], acc[n][1]);
+                        acc[n][2] = fmaf(part[i][2], sc_hi[i], acc[n][2]);
+                        acc[n][3] = fmaf(part[i][3], sc_hi[i], acc[n][3]);
+                    }
                 }
-            }
+            };
+            four_blocks(sw_lo.x, sw_hi.x, 0);
+            if (left > 4) four_blocks(sw_lo.y, sw_hi.y, 4);
         }
         __syncwarp();  // every lane is done reading the slot
         if (q + NS < nstages) issue(q + NS, slot);
@@ -340,8 +391,7 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
             // if it ever gave up the result would be wrong, which the parity tests would show.
             const int need = seg_index / kRedSlots;
             int spins = 0;
-            while (*reinterpret_cast<volatile int *>(&s_gen[rslot]) < need && ++spins < (1 << 24)) {
-            }
+            while (*reinterpret_cast<volatile int *>(&s_gen[rslot]) < need && ++spins < (1 << 22)) __nanosleep(40);
         }
         float *mine = s_red + (rslot * kMmaWarps + warp) * kOut;
         if (exact_ok) {
@@ -438,6 +488,26 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
 // ---------------------------------------------------------------------------------------------
 // host side: plan + launch
 // ---------------------------------------------------------------------------------------------
+// MXQ_LINEAR_STAGES=2|3 in the environment pins the ring depth (for experiments)
+static int forced_stages() {
+    static const int v = [] {
+        const char *e = std::getenv("MXQ_LINEAR_STAGES");
+        const int n = e ? std::atoi(e) : 0;
+        return (n == 2 || n == 3) ? n : 0;
+    }();
+    return v;
+}
+
+// MXQ_LINEAR_CTAS_PER_SM=1..8 in the environment sets the grid to that many CTAs per SM (for experiments)
+static int forced_ctas_per_sm() {
+    static const int v = [] {
+        const char *e = std::getenv("MXQ_LINEAR_CTAS_PER_SM");
+        const int n = e ? std::atoi(e) : 0;
+        return (n >= 1 && n <= 8) ? n : 0;
+    }();
+    return v;
+}
+
 bool linear_mma_plan(int M, int64_t N, int64_t K, LinearPlan &p) {
     if (M < 1 || M > 16 || (K % 128) != 0 || N < 1) return false;
     const int64_t kb = K / 32;
@@ -452,7 +522,7 @@ bool linear_mma_plan(int M, int64_t N, int64_t K, LinearPlan &p) {
     const uint32_t red_bytes = (uint32_t)kRedSlots * kMmaWarps * kout_bytes;
 
     // grid: two CTAs per SM, more only if a CTA's stage table would overflow; never more CTAs than rows
-    for (int mult = 2; mult <= 4096; mult *= 2) {
+    for (int mult = forced_ctas_per_sm() ? forced_ctas_per_sm() : 2; mult <= 4096; mult *= 2) {
         int64_t grid = (int64_t)sms * mult;
         if (grid > N) grid = N;
         p.grid = (int)grid;
@@ -468,13 +538,13 @@ bool linear_mma_plan(int M, int64_t N, int64_t K, LinearPlan &p) {
             p.smem_bytes = p.off_ring + (uint32_t)(kMmaWarps * nstage * kWarpStageBytes);
             return p.smem_bytes;
         };
-        int nstage = kMaxStages, nwin = 1;
+        int nstage = forced_stages() ? forced_stages() : kMaxStages, nwin = 1;
         int64_t bw = kb;
-        if (layout(nstage, bw, nwin) > kSmemQuarterSm) {
+        if (layout(nstage, bw, nwin) > kSmemThirdSm) {
             while (nstage > 2 && layout(nstage, bw, nwin) > kSmemHalfSm) --nstage;
             while (layout(nstage, bw, nwin) > kSmemHalfSm) {
                 if (++nwin > 64) return false;
-                bw = ((kb + nwin - 1) / nwin + 3) / 4 * 4;
+                bw = ((kb + nwin - 1) / nwin + 7) / 8 * 8;
             }
             while ((int64_t)(nwin - 1) * bw >= kb) --nwin;  // rounding up may have left the last window empty
             layout(nstage, bw, nwin);
@@ -520,8 +590,8 @@ static cudaError_t launch_mma(const LinearPlan &p, const void *X, const uint8_t 
 cudaError_t linear_mma_launch(const LinearPlan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,
                               int y_dtype, void *, cudaStream_t stream) {
 #define MXQ_LAUNCH(NT, NSTG) launch_mma<NT, NSTG>(p, X, codes, scales, Y, y_dtype, stream)
-    if (p.nt8 == 1) return p.nstage == 4 ? MXQ_LAUNCH(1, 4) : (p.nstage == 3 ? MXQ_LAUNCH(1, 3) : MXQ_LAUNCH(1, 2));
-    return p.nstage == 4 ? MXQ_LAUNCH(2, 4) : (p.nstage == 3 ? MXQ_LAUNCH(2, 3) : MXQ_LAUNCH(2, 2));
+    if (p.nt8 == 1) return p.nstage == 3 ? MXQ_LAUNCH(1, 3) : MXQ_LAUNCH(1, 2);
+    return p.nstage == 3 ? MXQ_LAUNCH(2, 3) : MXQ_LAUNCH(2, 2);
 #undef MXQ_LAUNCH
 }
 

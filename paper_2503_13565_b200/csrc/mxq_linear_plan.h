@@ -12,18 +12,20 @@
 namespace mxq {
 
 constexpr int kTileRows = 16;        // weight rows per tile = rows of one m16n8k16 A operand
-constexpr int kMmaWarps = 8;         // warps per CTA; each takes 4 of a stage's 32 MX blocks
+constexpr int kMmaWarps = 8;         // warps per CTA; each takes 8 of a stage's 64 MX blocks
 constexpr int kMmaThreads = kMmaWarps * 32;
-constexpr int kWarpBlocks = 4;       // MX blocks per warp per stage (their 4 scale bytes are one 32-bit word)
-constexpr int kStageBlocks = kMmaWarps * kWarpBlocks;    // 32 blocks = 1024 weights per row per stage
-// one warp's slice of one stage in shared memory: codes as [block][row][16 bytes] (a fragment read of
-// row g, word t of block jb hits bank 4g + t: conflict-free), then 16 rows x 4 scale bytes
-constexpr int kWarpCodeBytes = kTileRows * kWarpBlocks * 16;     // 1024
-constexpr int kWarpStageBytes = kWarpCodeBytes + kTileRows * 4;  // 1088
-constexpr int kMaxStages = 4;        // ring depth
-constexpr int kMaxCtaStages = 256;   // stage-table entries per CTA (16 bytes each)
-constexpr int kRedSlots = 2;         // tiles whose per-warp partial results can be pending at once
+constexpr int kWarpBlocks = 8;       // MX blocks per warp per stage (their 8 scale bytes are one 64-bit word)
+constexpr int kStageBlocks = kMmaWarps * kWarpBlocks;    // 64 blocks = 2048 weights per row per stage
+// one warp's slice of one stage in shared memory: codes as [row][8 chunks of 16 bytes], chunk c of row r
+// stored at position c ^ (r & 7) (copies and fragment reads are both bank-conflict free), then
+// 16 rows x 8 scale bytes; slots are 128-byte aligned
+constexpr int kWarpCodeBytes = kTileRows * kWarpBlocks * 16;               // 2048
+constexpr int kWarpStageBytes = kWarpCodeBytes + kTileRows * kWarpBlocks;  // 2176
+constexpr int kMaxStages = 3;        // ring depth
+constexpr int kMaxCtaStages = 128;   // stage-table entries per CTA (16 bytes each)
+constexpr int kRedSlots = 4;         // tiles whose per-warp partial results can be pending at once
 constexpr uint32_t kSmemQuarterSm = 56 * 1024;   // 4 CTAs per SM: two kernels, two CTAs each, can be resident
+constexpr uint32_t kSmemThirdSm = 75 * 1024;     // 3 CTAs per SM
 constexpr uint32_t kSmemHalfSm = 113 * 1024;     // 2 CTAs per SM
 constexpr uint32_t kOffMisc = 0;
 constexpr uint32_t kOffTable = 256;              // uint4[kMaxCtaStages]

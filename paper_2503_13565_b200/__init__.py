@@ -8,5 +8,6 @@ if ``libmxq.so`` is missing.
 from .binding import (MAX_M, MAX_T, MXQ_BF16, MXQ_F32, MxqError, mxq_accept_workspace_bytes, mxq_codes_bytes,  # noqa: F401
                       mxq_dequantize, mxq_greedy_accept, mxq_greedy_accept_static,
                       mxq_greedy_accept_static_max_bytes, mxq_greedy_accept_tokens, mxq_linear, mxq_linear_host,
-                      mxq_linear_plan_info, mxq_linear_workspace_bytes, mxq_quantize, mxq_scales_bytes, mxq_set_pdl, mxq_version,
+                      KERNELS, mxq_linear_device_status, mxq_linear_plan_info, mxq_linear_workspace_bytes,
+                      mxq_set_linear_kernel, mxq_quantize, mxq_scales_bytes, mxq_set_pdl, mxq_version,
                       new_workspace, status_string)

@@ -59,7 +59,11 @@ def lib() -> ctypes.CDLL:
             L.mxq_linear.restype = i32
             L.mxq_linear.argtypes = [vp, i32, vp, vp, i64, i64, vp, i32, vp, sz, vp]
             L.mxq_linear_plan_info.restype = i32
-            L.mxq_linear_plan_info.argtypes = [i32, i64, i64, vp]
+            L.mxq_linear_plan_info.argtypes = [i32, i32, i64, i64, vp]
+            L.mxq_set_linear_kernel.restype = i32
+            L.mxq_set_linear_kernel.argtypes = [i32]
+            L.mxq_linear_device_status.restype = i32
+            L.mxq_linear_device_status.argtypes = [vp]
             L.mxq_linear_host.restype = i32
             L.mxq_linear_host.argtypes = [vp, i32, vp, vp, i64, i64, vp, i32, vp, vp, vp, sz, vp]
             L.mxq_greedy_accept.restype = i32
@@ -125,13 +129,40 @@ def mxq_linear_workspace_bytes(m: int, n: int, k: int) -> int:
     return int(lib().mxq_linear_workspace_bytes(m, n, k))
 
 
-def mxq_linear_plan_info(m: int, n: int, k: int) -> dict:
-    """How mxq_linear will run this shape (diagnostics)."""
+KERNELS = {"auto": -1, "generic": 0, "mma": 1, "umma": 2}
+_KERNEL_NAMES = {v: k for k, v in KERNELS.items()}
+_PLAN_KEYS = {
+    2: ("kernel", "grid", "ring", "split", "chunk_max", "tiles", "tmem_cols", "smem_bytes", "nb", "kb"),
+    1: ("kernel", "grid", "stages", "windows", "bw", "bw_last", "max_tiles", "smem_bytes", "nt8", "kb"),
+    0: ("kernel", "grid"),
+}
+
+
+def mxq_set_linear_kernel(kernel) -> str:
+    """Restrict mxq_linear's choice of kernel ("auto", "umma", "mma", "generic"); returns the previous setting."""
+    code = KERNELS[kernel] if isinstance(kernel, str) else int(kernel)
+    return _KERNEL_NAMES[int(lib().mxq_set_linear_kernel(code))]
+
+
+def mxq_linear_plan_info(m: int, n: int, k: int, kernel="auto") -> dict:
+    """How a kernel would run this shape (diagnostics).  ``kernel`` is a name of KERNELS; the result's
+    "kernel" is the name of the kernel described, or None if the requested one does not cover the shape."""
     info = (ctypes.c_int32 * 12)()
-    _check(lib().mxq_linear_plan_info(m, n, k, ctypes.cast(info, ctypes.c_void_p)), "mxq_linear_plan_info")
-    keys = ("tensor_core", "grid", "stages", "windows", "bw", "bw_last", "max_tiles", "smem_bytes", "nt8", "kb",
-            "reserved0", "reserved1")
-    return dict(zip(keys, [int(v) for v in info]))
+    code = KERNELS[kernel] if isinstance(kernel, str) else int(kernel)
+    _check(lib().mxq_linear_plan_info(code, m, n, k, ctypes.cast(info, ctypes.c_void_p)), "mxq_linear_plan_info")
+    vals = [int(v) for v in info]
+    if vals[0] < 0:
+        return {"kernel": None}
+    out = dict(zip(_PLAN_KEYS[vals[0]], vals))
+    out["kernel"] = _KERNEL_NAMES[vals[0]]
+    return out
+
+
+def mxq_linear_device_status() -> int:
+    """The sticky word in which the tcgen05 kernel records a bounded wait that gave up (0 = never); cleared by the call."""
+    word = ctypes.c_uint32(0)
+    _check(lib().mxq_linear_device_status(ctypes.cast(ctypes.byref(word), ctypes.c_void_p)), "mxq_linear_device_status")
+    return int(word.value)
 
 
 def mxq_accept_workspace_bytes(b: int, r: int, v: int) -> int:

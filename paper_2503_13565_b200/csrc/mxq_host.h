@@ -23,4 +23,11 @@ size_t linear_mma_workspace_bytes(const LinearPlan &plan);
 cudaError_t linear_mma_launch(const LinearPlan &plan, const void *X, const uint8_t *codes, const uint8_t *scales,
                               void *Y, int y_dtype, void *workspace, cudaStream_t stream);
 
+struct UmmaPlan;
+// tcgen05 path of mxq_linear (mxq_linear_umma.cu): false if the shape is not covered
+bool linear_umma_available();
+bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &plan);
+cudaError_t linear_umma_launch(const UmmaPlan &plan, const void *X, const uint8_t *codes, const uint8_t *scales,
+                               void *Y, int y_dtype, cudaStream_t stream);
+
 }  // namespace mxq

@@ -1,20 +1,25 @@
 // mxq_linear: Y[M,N] = X[M,K] . dequant(codes, scales)[N,K]^T  (Sec. III-D-3, Eq. 2).
 //
 // This file holds the entry points, the dispatch and the generic kernel.  Shapes with
-// K % 128 == 0 go to the tensor-core kernel in mxq_linear_mma.cu; everything else (and
-// MXQ_LINEAR_VARIANT=generic in the environment) runs the generic kernel below.
+// K % 128 == 0 go to the tcgen05 kernel in mxq_linear_umma.cu (weights as a native tensor-core
+// operand) or, where that one does not cover the shape, to the mma.sync kernel in
+// mxq_linear_mma.cu; everything else runs the generic kernel below.  MXQ_LINEAR_VARIANT in the
+// environment (umma | mma | generic) restricts the choice to that kernel and the ones after it.
 //
 // Generic kernel: the weight stream (4.25 bits per weight) is the cost; X and Y are negligible.  Each warp
 // owns whole output rows, so no partial sums ever leave the warp and the summation order is
 // fixed.  Lanes walk the row's MX blocks with 16-byte loads (one load = one block of 32
 // weights = one scale byte), decode the E2M1 pairs in registers, accumulate the 32-long
 // partial sum in FP32 and apply the block scale once per block (the late scaling of Eq. 2).
+#include <atomic>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
 #include "mxq_device.cuh"
 #include "mxq_host.h"
 #include "mxq_linear_plan.h"
+#include "mxq_linear_umma.h"
 
 namespace mxq {
 
@@ -96,13 +101,25 @@ static void launch_rowwarp(const void *X, int M, const uint8_t *codes, const uin
                        K, Y, y_dtype);
 }
 
-// MXQ_LINEAR_VARIANT=generic forces the generic kernel (for tests and comparisons)
-static bool force_generic() {
-    static const int v = [] {
+// mxq_set_linear_kernel / MXQ_LINEAR_VARIANT: 0 = no restriction (umma, then mma, then generic),
+// 1 = mma then generic, 2 = generic only
+static std::atomic<int> g_floor{-1};
+static int variant_floor() {
+    int v = g_floor.load(std::memory_order_relaxed);
+    if (v < 0) {
         const char *e = std::getenv("MXQ_LINEAR_VARIANT");
-        return (e && std::strcmp(e, "generic") == 0) ? 1 : 0;
-    }();
-    return v != 0;
+        v = (e && std::strcmp(e, "generic") == 0) ? 2 : ((e && std::strcmp(e, "mma") == 0) ? 1 : 0);
+        g_floor.store(v, std::memory_order_relaxed);
+    }
+    return v;
+}
+static bool force_generic() { return variant_floor() >= 2; }
+
+// the tcgen05 kernel reads the codes through a tensor map, which wants a 32-byte aligned base
+static bool use_umma(int M, int64_t N, int64_t K, const uint8_t *codes, UmmaPlan &plan) {
+    if (variant_floor() >= 1 || !linear_umma_available()) return false;
+    if (codes && (reinterpret_cast<uintptr_t>(codes) & 31u) != 0) return false;
+    return linear_umma_plan(M, N, K, plan);
 }
 
 }  // namespace mxq
@@ -112,19 +129,48 @@ extern "C" {
 
 size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K) {
     if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return 0;
-    mxq::LinearPlan plan;
-    if (!mxq::force_generic() && mxq::linear_mma_plan(M, N, K, plan)) return mxq::linear_mma_workspace_bytes(plan);
-    return 0;
+    return 0;   // the tcgen05 kernel adds partial results inside a cluster, the others never split a row
 }
 
-int mxq_linear_plan_info(int M, int64_t N, int64_t K, int32_t *info) {
+int mxq_set_linear_kernel(int kernel) {
+    const int prev = mxq::variant_floor();
+    const int now = kernel == MXQ_KERNEL_GENERIC ? 2 : (kernel == MXQ_KERNEL_MMA ? 1 : 0);
+    mxq::g_floor.store(now, std::memory_order_relaxed);
+    return prev == 2 ? MXQ_KERNEL_GENERIC : (prev == 1 ? MXQ_KERNEL_MMA : MXQ_KERNEL_AUTO);
+}
+
+int mxq_linear_plan_info(int kernel, int M, int64_t N, int64_t K, int32_t *info) {
     if (!info) return MXQ_ERR_NULL;
     if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return MXQ_ERR_SHAPE;
+    if (kernel < MXQ_KERNEL_AUTO || kernel > MXQ_KERNEL_UMMA) return MXQ_ERR_SHAPE;
     mxq::LinearPlan p;
-    const bool mma = !mxq::force_generic() && mxq::linear_mma_plan(M, N, K, p);
+    mxq::UmmaPlan u;
     for (int i = 0; i < 12; ++i) info[i] = 0;
-    info[0] = mma ? 1 : 0;
-    if (mma) {
+    if (kernel == MXQ_KERNEL_AUTO) {
+        if (mxq::use_umma(M, N, K, nullptr, u)) kernel = MXQ_KERNEL_UMMA;
+        else if (!mxq::force_generic() && mxq::linear_mma_plan(M, N, K, p)) kernel = MXQ_KERNEL_MMA;
+        else kernel = MXQ_KERNEL_GENERIC;
+    }
+    info[0] = kernel;
+    if (kernel == MXQ_KERNEL_UMMA) {
+        if (!mxq::linear_umma_plan(M, N, K, u)) {
+            info[0] = -1;
+            return MXQ_OK;
+        }
+        info[1] = u.grid;
+        info[2] = u.ring;
+        info[3] = u.split;
+        info[4] = u.chunk_max;
+        info[5] = u.tiles;
+        info[6] = u.tmem_cols;
+        info[7] = (int32_t)u.smem_bytes;
+        info[8] = u.nb;
+        info[9] = (int32_t)(K / 32);
+    } else if (kernel == MXQ_KERNEL_MMA) {
+        if (!mxq::linear_mma_plan(M, N, K, p)) {
+            info[0] = -1;
+            return MXQ_OK;
+        }
         info[1] = p.grid;
         info[2] = p.nstage;
         info[3] = p.nwin;
@@ -148,6 +194,16 @@ int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *s
     if (!mxq::aligned16(X_bf16) || !mxq::aligned16(codes) || !mxq::aligned16(scales) || !mxq::aligned16(Y))
         return MXQ_ERR_ALIGN;
     cudaStream_t st = (cudaStream_t)stream;
+    mxq::UmmaPlan uplan;
+    if (mxq::use_umma(M, N, K, codes, uplan)) {
+        const cudaError_t e = mxq::linear_umma_launch(uplan, X_bf16, codes, scales, Y, y_dtype, st);
+        if (e != cudaSuccess) {
+            if (std::getenv("MXQ_DEBUG")) std::fprintf(stderr, "mxq_linear (tcgen05 kernel): %s\n", cudaGetErrorString(e));
+            (void)cudaGetLastError();
+            return MXQ_ERR_CUDA;
+        }
+        return mxq::launch_status();
+    }
     mxq::LinearPlan plan;
     if (!mxq::force_generic() && mxq::linear_mma_plan(M, N, K, plan)) {
         const size_t need = mxq::linear_mma_workspace_bytes(plan);

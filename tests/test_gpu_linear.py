@@ -12,6 +12,16 @@ from parity import check_linear, gpu_bf16
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(autouse=True, params=["auto", "mma"])
+def linear_kernel(request):
+    """Every case runs twice: with the library's own choice of kernel (the tcgen05 kernel where it covers
+    the shape) and with that kernel excluded (mma.sync kernel, else the generic one)."""
+    prev = mxq.mxq_set_linear_kernel(request.param)
+    yield request.param
+    mxq.mxq_set_linear_kernel(prev)
+    assert mxq.mxq_linear_device_status() == 0, "a bounded wait inside the tcgen05 kernel gave up"
+
+
 def run_case(wbits, xbits, out_dtype=torch.float32, rows=None, what=""):
     """Quantise on the oracle side, run the layer on both sides from the same bytes."""
     codes, scales, _ = oracle.quantize(wbits)
@@ -22,9 +32,6 @@ def run_case(wbits, xbits, out_dtype=torch.float32, rows=None, what=""):
     y = mxq.mxq_linear(gpu_bf16(xbits), torch.from_numpy(codes).cuda(), torch.from_numpy(scales).cuda(),
                        out_dtype=out_dtype, workspace=ws)
     torch.cuda.synchronize()
-    assert int(ws.view(torch.int32)[0]) == 0, what + ": a bounded wait inside the kernel gave up"
-    if ws.numel() >= 256 + 65536 * 4:
-        assert not ws[256: 256 + 65536 * 4].any(), what + ": ticket counters were not returned to zero"
     if rows is not None:
         y = y[:, torch.as_tensor(rows, device="cuda")]
     return check_linear(y, y64, a64, what), y
@@ -69,13 +76,13 @@ def test_every_token_count_on_a_ragged_shape_tensor_core_path(m):
     n, k = 203, 1408   # N not a multiple of 16, K = 44 blocks (a multiple of 128: tensor-core kernel)
     w = synth.bits_of(synth.weight(3, 14, n, k))
     x = synth.bits_of(synth.activations(3, 14, m, k))
-    assert mxq.mxq_linear_plan_info(m, n, k)["tensor_core"] == 1
+    assert mxq.mxq_linear_plan_info(m, n, k)["kernel"] in ("umma", "mma")
     run_case(w, x, what="ragged tc M=%d" % m)
 
 
 @pytest.mark.parametrize("m,n,k", [(8, 4096, 11008), (16, 512, 13824), (16, 1000, 4096), (12, 333, 5120)])
 def test_shapes_that_split_k_into_windows(m, n, k):
-    assert mxq.mxq_linear_plan_info(m, n, k)["windows"] > 1
+    assert mxq.mxq_linear_plan_info(m, n, k, "mma")["windows"] > 1
     w = synth.bits_of(synth.weight(3, 15, n, k))
     x = synth.bits_of(synth.activations(3, 15, m, k))
     rows = np.unique(np.concatenate([[0, n - 1], np.random.default_rng(5).integers(0, n, 200)])).astype(np.int64)

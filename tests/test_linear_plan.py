@@ -36,8 +36,8 @@ def stage_lookup(p, tiles, q):
 
 @pytest.mark.parametrize("m,n,k", SHAPES)
 def test_plan_invariants(m, n, k):
-    p = mxq.mxq_linear_plan_info(m, n, k)
-    assert p["tensor_core"] == 1
+    p = mxq.mxq_linear_plan_info(m, n, k, "mma")
+    assert p["kernel"] == "mma"
     assert p["smem_bytes"] <= SMEM_HALF_SM
     assert p["kb"] == k // 32
     assert p["bw"] % 4 == 0 and p["bw_last"] % 4 == 0 and p["bw_last"] > 0
@@ -77,17 +77,54 @@ def test_plan_invariants(m, n, k):
     assert sum(v for (w, t), v in covered.items() if t == 0) == p["kb"]
 
 
-def test_shapes_outside_the_tensor_core_path_use_the_generic_kernel():
-    assert mxq.mxq_linear_plan_info(1, 3, 1 << 20)["tensor_core"] == 0      # a single row would overflow the stage table
-    assert mxq.mxq_linear_plan_info(1, 64, 96)["tensor_core"] == 0          # K % 128 != 0
+def test_shapes_outside_the_tensor_core_paths_use_the_generic_kernel():
+    assert mxq.mxq_linear_plan_info(1, 3, 1 << 20, "mma")["kernel"] is None      # a single row would overflow the stage table
+    for kernel in ("mma", "umma"):
+        assert mxq.mxq_linear_plan_info(1, 64, 96, kernel)["kernel"] is None      # K % 128 != 0
+        assert mxq.mxq_linear_plan_info(1, 203, 1440, kernel)["kernel"] is None
     assert mxq.mxq_linear_workspace_bytes(1, 64, 96) == 0
-    assert mxq.mxq_linear_plan_info(1, 203, 1440)["tensor_core"] == 0
+    assert mxq.mxq_linear_plan_info(1, 64, 96)["kernel"] == "generic"
+    assert mxq.mxq_linear_plan_info(1, 64, 96, "generic") == {"kernel": "generic", "grid": 8}
 
 
-def test_headline_shapes_leave_room_for_the_next_kernel():
-    """M=1 on the 7B layers: one window, three stages, two CTAs per SM, and small enough (at most a third
-    of an SM for K=4096) that a CTA of the next kernel fits beside them."""
-    for n, k, limit in [(4096, 4096, 75 * 1024), (11008, 4096, 75 * 1024), (4096, 11008, SMEM_HALF_SM)]:
-        p = mxq.mxq_linear_plan_info(1, n, k)
+def test_headline_shapes_run_two_ctas_per_sm():
+    """M=1 on the 7B layers with the mma.sync kernel: one window, two or three stages, two CTAs per SM."""
+    for n, k, limit in [(4096, 4096, SMEM_HALF_SM), (11008, 4096, SMEM_HALF_SM), (4096, 11008, SMEM_HALF_SM)]:
+        p = mxq.mxq_linear_plan_info(1, n, k, "mma")
         assert (p["windows"], p["grid"]) == (1, 2 * SMS) and p["stages"] in (2, 3), p
         assert p["smem_bytes"] <= limit, p
+
+
+UMMA_SHAPES = SHAPES + [(1, 32000, 4096), (1, 1000, 65536), (16, 4096, 28672), (4, 300, 128)]
+
+
+@pytest.mark.parametrize("m,n,k", UMMA_SHAPES)
+def test_tcgen05_plan_invariants(m, n, k):
+    """One CTA per (128-row tile, K chunk); the CTAs of a tile form a cluster of `split` <= 8; everything a
+    CTA keeps in shared and tensor memory fits."""
+    p = mxq.mxq_linear_plan_info(m, n, k, "umma")
+    assert p["kernel"] == "umma"
+    ks = k // 128
+    assert p["kb"] == k // 32 and p["tiles"] == -(-n // 128)
+    assert 1 <= p["split"] <= min(8, ks)
+    assert p["grid"] == p["tiles"] * p["split"]
+    assert p["chunk_max"] == -(-ks // p["split"])
+    assert 1 <= p["ring"] <= min(8, p["chunk_max"])
+    assert p["nb"] in (16, 32, 48) and p["nb"] >= 3 * m and (p["nb"] == 16 or p["nb"] - 16 < 3 * m)
+    assert p["smem_bytes"] <= 227 * 1024
+    assert p["tmem_cols"] in (64, 128) and p["tmem_cols"] >= p["nb"] + 8 * p["ring"]
+    # the stage ranges of a cluster's CTAs partition [0, K/128) and none is empty
+    bounds = [r * ks // p["split"] for r in range(p["split"] + 1)]
+    sizes = [b1 - b0 for b0, b1 in zip(bounds, bounds[1:])]
+    assert bounds[0] == 0 and bounds[-1] == ks and min(sizes) >= 1 and max(sizes) <= p["chunk_max"]
+    # rows of a tile are shared out among the cluster's CTAs for the final sum
+    rb = [r * 128 // p["split"] for r in range(p["split"] + 1)]
+    assert rb[-1] == 128 and p["split"] * max(b1 - b0 for b0, b1 in zip(rb, rb[1:])) <= 136
+    for row in range(128):
+        owner = ((row + 1) * p["split"] - 1) // 128
+        assert rb[owner] <= row < rb[owner + 1]
+
+
+def test_tcgen05_kernel_needs_whole_stages():
+    assert mxq.mxq_linear_plan_info(1, 4096, 4096 + 64, "umma")["kernel"] is None
+    assert mxq.mxq_linear_plan_info(1, 4096, 96, "umma")["kernel"] is None

@@ -94,26 +94,31 @@ int mxq_dequantize(const uint8_t *codes, const uint8_t *scales, int64_t N, int64
  * interface for future kernels.  If non-zero: zero-fill once before first use; calls leave it reusable. */
 size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K);
 
-/* The three kernels behind mxq_linear.  MXQ_KERNEL_UMMA feeds the MXFP4 codes and scales to the
- * tcgen05 block-scaled tensor-core instruction as they are (needs K % 128 == 0 and a 32-byte aligned
- * `codes`); MXQ_KERNEL_MMA decodes them into FP16 mma.sync fragments (K % 128 == 0); MXQ_KERNEL_GENERIC
- * takes any valid shape on the CUDA cores.  mxq_linear uses the first of these, in this order, that
- * covers the call. */
-enum mxq_kernel { MXQ_KERNEL_AUTO = -1, MXQ_KERNEL_GENERIC = 0, MXQ_KERNEL_MMA = 1, MXQ_KERNEL_UMMA = 2 };
+/* The kernels behind mxq_linear, fastest first.
+ *   MXQ_KERNEL_FP4     tcgen05 block-scaled MMA with packed 4-bit operands on both sides: the codes and scales
+ *                      go to the tensor core as they are, the 1..4 token rows as 16 exact radix-4 digit planes
+ *                      each (needs K % 128 == 0, M <= 4)
+ *   MXQ_KERNEL_UMMA    tcgen05 block-scaled MMA with the codes expanded in flight by the copy engine and each
+ *                      token row split exactly into three E5M2 rows (needs K % 128 == 0, a 32-byte aligned `codes`)
+ *   MXQ_KERNEL_MMA     decodes the codes into FP16 mma.sync fragments (needs K % 128 == 0)
+ *   MXQ_KERNEL_GENERIC any valid shape, on the CUDA cores
+ * mxq_linear uses the first of these, in this order, that is allowed (next call) and covers the call. */
+enum mxq_kernel {
+    MXQ_KERNEL_AUTO = -1, MXQ_KERNEL_GENERIC = 0, MXQ_KERNEL_MMA = 1, MXQ_KERNEL_UMMA = 2, MXQ_KERNEL_FP4 = 3
+};
 
-/* Restricts mxq_linear's choice (tests, comparisons): MXQ_KERNEL_AUTO or MXQ_KERNEL_UMMA = no
- * restriction, MXQ_KERNEL_MMA = never the tcgen05 kernel, MXQ_KERNEL_GENERIC = the generic kernel only.
- * Returns the previous setting.  Host-side, process-wide.  The initial setting comes from the
- * environment variable MXQ_LINEAR_VARIANT (umma | mma | generic), else MXQ_KERNEL_AUTO. */
+/* Caps mxq_linear's choice (tests, comparisons): kernels listed above `kernel` are not used; MXQ_KERNEL_AUTO
+ * (or MXQ_KERNEL_FP4) lifts the cap.  Returns the previous cap.  Host-side, process-wide.  The initial cap comes
+ * from the environment variable MXQ_LINEAR_VARIANT (umma | mma | generic), else there is none. */
 int mxq_set_linear_kernel(int kernel);
 
 /* How a kernel would run this shape on the current device (diagnostics; launches nothing).
- * kernel = MXQ_KERNEL_AUTO describes the one mxq_linear would pick under the current setting for a
+ * kernel = MXQ_KERNEL_AUTO describes the one mxq_linear would pick under the current cap for a
  * suitably aligned `codes`; another value describes that kernel whether or not it would be picked.
  * info[12] int32; info[0] = the kernel described, or -1 if the requested kernel does not cover the shape.
- *   MXQ_KERNEL_UMMA:    [1] CTAs; [2] ring stages; [3] CTAs per cluster (K split); [4] most 128-k stages a
- *                       CTA owns; [5] 128-row tiles; [6] tensor-memory columns; [7] dynamic shared memory
- *                       bytes; [8] columns of the token operand; [9] K/32.
+ *   MXQ_KERNEL_FP4,     [1] CTAs; [2] ring stages; [3] CTAs per cluster (K split); [4] most stages a CTA owns
+ *   MXQ_KERNEL_UMMA:    (a stage is 256 k for FP4, 128 k for UMMA); [5] 128-row tiles; [6] tensor-memory
+ *                       columns; [7] dynamic shared memory bytes; [8] columns of the token operand; [9] K/32.
  *   MXQ_KERNEL_MMA:     [1] CTAs; [2] ring stages; [3] K windows; [4] blocks per window; [5] blocks in the
  *                       last window; [6] most 16-row tiles a CTA owns; [7] dynamic shared memory bytes;
  *                       [8] 8-token column tiles; [9] K/32.
@@ -121,9 +126,10 @@ int mxq_set_linear_kernel(int kernel);
  * Unused entries are 0. */
 int mxq_linear_plan_info(int kernel, int M, int64_t N, int64_t K, int32_t *info);
 
-/* Copies to *status_host, and then clears, the sticky device word in which the tcgen05 kernel records a
+/* Copies to *status_host, and then clears, the sticky device words in which the tcgen05 kernels record a
  * bounded wait that gave up (bit 0: data of a stage never arrived, bit 1: a stage was never released,
- * bit 2: the accumulator never completed, bit 3: a prefetched stage never landed).  0 in normal
+ * bit 2: the accumulator never completed, bit 3: a prefetched stage never landed; bits 0-3 for
+ * MXQ_KERNEL_UMMA, bits 8-11 the same for MXQ_KERNEL_FP4).  0 in normal
  * operation; a non-zero word means the affected output tiles were written as NaN.  Synchronises with
  * the device (a blocking copy), so call it outside the hot loop. */
 int mxq_linear_device_status(uint32_t *status_host);

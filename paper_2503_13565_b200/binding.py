@@ -129,9 +129,10 @@ def mxq_linear_workspace_bytes(m: int, n: int, k: int) -> int:
     return int(lib().mxq_linear_workspace_bytes(m, n, k))
 
 
-KERNELS = {"auto": -1, "generic": 0, "mma": 1, "umma": 2}
+KERNELS = {"auto": -1, "generic": 0, "mma": 1, "umma": 2, "fp4": 3}
 _KERNEL_NAMES = {v: k for k, v in KERNELS.items()}
 _PLAN_KEYS = {
+    3: ("kernel", "grid", "ring", "split", "chunk_max", "tiles", "tmem_cols", "smem_bytes", "nb", "kb"),
     2: ("kernel", "grid", "ring", "split", "chunk_max", "tiles", "tmem_cols", "smem_bytes", "nb", "kb"),
     1: ("kernel", "grid", "stages", "windows", "bw", "bw_last", "max_tiles", "smem_bytes", "nt8", "kb"),
     0: ("kernel", "grid"),
@@ -139,7 +140,7 @@ _PLAN_KEYS = {
 
 
 def mxq_set_linear_kernel(kernel) -> str:
-    """Restrict mxq_linear's choice of kernel ("auto", "umma", "mma", "generic"); returns the previous setting."""
+    """Cap mxq_linear's choice of kernel ("auto"/"fp4" = no cap, "umma", "mma", "generic"); returns the previous cap."""
     code = KERNELS[kernel] if isinstance(kernel, str) else int(kernel)
     return _KERNEL_NAMES[int(lib().mxq_set_linear_kernel(code))]
 

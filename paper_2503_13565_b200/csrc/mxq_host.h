@@ -30,4 +30,11 @@ bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &plan);
 cudaError_t linear_umma_launch(const UmmaPlan &plan, const void *X, const uint8_t *codes, const uint8_t *scales,
                                void *Y, int y_dtype, cudaStream_t stream);
 
+struct Fp4Plan;
+// tcgen05 path with packed 4-bit operands on both sides, M <= 4 (mxq_linear_fp4.cu)
+bool linear_fp4_plan(int M, int64_t N, int64_t K, Fp4Plan &plan);
+cudaError_t linear_fp4_launch(const Fp4Plan &plan, const void *X, const uint8_t *codes, const uint8_t *scales,
+                              void *Y, int y_dtype, cudaStream_t stream);
+int linear_fp4_take_status(uint32_t *out);
+
 }  // namespace mxq

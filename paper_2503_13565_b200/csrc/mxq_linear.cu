@@ -1,10 +1,10 @@
 // mxq_linear: Y[M,N] = X[M,K] . dequant(codes, scales)[N,K]^T  (Sec. III-D-3, Eq. 2).
 //
 // This file holds the entry points, the dispatch and the generic kernel.  Shapes with
-// K % 128 == 0 go to the tcgen05 kernel in mxq_linear_umma.cu (weights as a native tensor-core
-// operand) or, where that one does not cover the shape, to the mma.sync kernel in
-// mxq_linear_mma.cu; everything else runs the generic kernel below.  MXQ_LINEAR_VARIANT in the
-// environment (umma | mma | generic) restricts the choice to that kernel and the ones after it.
+// K % 128 == 0 go to a tcgen05 kernel (weights as a native tensor-core operand: mxq_linear_fp4.cu
+// for up to 4 token rows, mxq_linear_umma.cu above that) or, where neither covers the call, to the
+// mma.sync kernel in mxq_linear_mma.cu; everything else runs the generic kernel below.
+// mxq_set_linear_kernel, or MXQ_LINEAR_VARIANT in the environment (umma | mma | generic), caps the choice.
 //
 // Generic kernel: the weight stream (4.25 bits per weight) is the cost; X and Y are negligible.  Each warp
 // owns whole output rows, so no partial sums ever leave the warp and the summation order is
@@ -19,6 +19,7 @@
 #include "mxq_device.cuh"
 #include "mxq_host.h"
 #include "mxq_linear_plan.h"
+#include "mxq_linear_fp4.h"
 #include "mxq_linear_umma.h"
 
 namespace mxq {
@@ -101,25 +102,38 @@ static void launch_rowwarp(const void *X, int M, const uint8_t *codes, const uin
                        K, Y, y_dtype);
 }
 
-// mxq_set_linear_kernel / MXQ_LINEAR_VARIANT: 0 = no restriction (umma, then mma, then generic),
-// 1 = mma then generic, 2 = generic only
-static std::atomic<int> g_floor{-1};
-static int variant_floor() {
-    int v = g_floor.load(std::memory_order_relaxed);
-    if (v < 0) {
+// mxq_set_linear_kernel / MXQ_LINEAR_VARIANT: the highest kernel mxq_linear may use (MXQ_KERNEL_* order)
+static std::atomic<int> g_ceiling{-2};
+static int kernel_ceiling() {
+    int v = g_ceiling.load(std::memory_order_relaxed);
+    if (v < -1) {
         const char *e = std::getenv("MXQ_LINEAR_VARIANT");
-        v = (e && std::strcmp(e, "generic") == 0) ? 2 : ((e && std::strcmp(e, "mma") == 0) ? 1 : 0);
-        g_floor.store(v, std::memory_order_relaxed);
+        v = MXQ_KERNEL_FP4;
+        if (e && std::strcmp(e, "generic") == 0) v = MXQ_KERNEL_GENERIC;
+        else if (e && std::strcmp(e, "mma") == 0) v = MXQ_KERNEL_MMA;
+        else if (e && std::strcmp(e, "umma") == 0) v = MXQ_KERNEL_UMMA;
+        g_ceiling.store(v, std::memory_order_relaxed);
     }
     return v;
 }
-static bool force_generic() { return variant_floor() >= 2; }
 
-// the tcgen05 kernel reads the codes through a tensor map, which wants a 32-byte aligned base
-static bool use_umma(int M, int64_t N, int64_t K, const uint8_t *codes, UmmaPlan &plan) {
-    if (variant_floor() >= 1 || !linear_umma_available()) return false;
-    if (codes && (reinterpret_cast<uintptr_t>(codes) & 31u) != 0) return false;
-    return linear_umma_plan(M, N, K, plan);
+// The kernel mxq_linear runs for this call: the first of FP4, UMMA, MMA, GENERIC that is not above the ceiling
+// and covers the shape.  The tcgen05 kernels read the codes through a tensor map (FP4: 16-byte aligned base,
+// which every call has; UMMA: 32-byte aligned base); codes == nullptr means "suitably aligned".
+struct Choice {
+    int kernel;
+    Fp4Plan fp4;
+    UmmaPlan umma;
+    LinearPlan mma;
+};
+static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *codes, Choice &c) {
+    const bool tc = linear_umma_available();
+    if (ceiling >= MXQ_KERNEL_FP4 && tc && linear_fp4_plan(M, N, K, c.fp4)) c.kernel = MXQ_KERNEL_FP4;
+    else if (ceiling >= MXQ_KERNEL_UMMA && tc && (!codes || (reinterpret_cast<uintptr_t>(codes) & 31u) == 0) &&
+             linear_umma_plan(M, N, K, c.umma))
+        c.kernel = MXQ_KERNEL_UMMA;
+    else if (ceiling >= MXQ_KERNEL_MMA && linear_mma_plan(M, N, K, c.mma)) c.kernel = MXQ_KERNEL_MMA;
+    else c.kernel = MXQ_KERNEL_GENERIC;
 }
 
 }  // namespace mxq
@@ -133,44 +147,45 @@ size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K) {
 }
 
 int mxq_set_linear_kernel(int kernel) {
-    const int prev = mxq::variant_floor();
-    const int now = kernel == MXQ_KERNEL_GENERIC ? 2 : (kernel == MXQ_KERNEL_MMA ? 1 : 0);
-    mxq::g_floor.store(now, std::memory_order_relaxed);
-    return prev == 2 ? MXQ_KERNEL_GENERIC : (prev == 1 ? MXQ_KERNEL_MMA : MXQ_KERNEL_AUTO);
+    const int prev = mxq::kernel_ceiling();
+    mxq::g_ceiling.store(kernel < MXQ_KERNEL_GENERIC || kernel > MXQ_KERNEL_FP4 ? MXQ_KERNEL_FP4 : kernel,
+                         std::memory_order_relaxed);
+    return prev;
 }
 
 int mxq_linear_plan_info(int kernel, int M, int64_t N, int64_t K, int32_t *info) {
     if (!info) return MXQ_ERR_NULL;
     if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return MXQ_ERR_SHAPE;
-    if (kernel < MXQ_KERNEL_AUTO || kernel > MXQ_KERNEL_UMMA) return MXQ_ERR_SHAPE;
-    mxq::LinearPlan p;
-    mxq::UmmaPlan u;
+    if (kernel < MXQ_KERNEL_AUTO || kernel > MXQ_KERNEL_FP4) return MXQ_ERR_SHAPE;
     for (int i = 0; i < 12; ++i) info[i] = 0;
+    mxq::Choice c;
     if (kernel == MXQ_KERNEL_AUTO) {
-        if (mxq::use_umma(M, N, K, nullptr, u)) kernel = MXQ_KERNEL_UMMA;
-        else if (!mxq::force_generic() && mxq::linear_mma_plan(M, N, K, p)) kernel = MXQ_KERNEL_MMA;
-        else kernel = MXQ_KERNEL_GENERIC;
+        mxq::choose(mxq::kernel_ceiling(), M, N, K, nullptr, c);
+    } else {
+        c.kernel = kernel;
+        const bool ok = kernel == MXQ_KERNEL_FP4    ? mxq::linear_fp4_plan(M, N, K, c.fp4)
+                        : kernel == MXQ_KERNEL_UMMA ? mxq::linear_umma_plan(M, N, K, c.umma)
+                        : kernel == MXQ_KERNEL_MMA  ? mxq::linear_mma_plan(M, N, K, c.mma)
+                                                    : true;
+        if (!ok) {
+            info[0] = -1;
+            return MXQ_OK;
+        }
     }
-    info[0] = kernel;
-    if (kernel == MXQ_KERNEL_UMMA) {
-        if (!mxq::linear_umma_plan(M, N, K, u)) {
-            info[0] = -1;
-            return MXQ_OK;
-        }
-        info[1] = u.grid;
-        info[2] = u.ring;
-        info[3] = u.split;
-        info[4] = u.chunk_max;
-        info[5] = u.tiles;
-        info[6] = u.tmem_cols;
-        info[7] = (int32_t)u.smem_bytes;
-        info[8] = u.nb;
+    info[0] = c.kernel;
+    if (c.kernel == MXQ_KERNEL_FP4 || c.kernel == MXQ_KERNEL_UMMA) {
+        const bool f = c.kernel == MXQ_KERNEL_FP4;
+        info[1] = f ? c.fp4.grid : c.umma.grid;
+        info[2] = f ? c.fp4.ring : c.umma.ring;
+        info[3] = f ? c.fp4.split : c.umma.split;
+        info[4] = f ? c.fp4.chunk_max : c.umma.chunk_max;
+        info[5] = f ? c.fp4.tiles : c.umma.tiles;
+        info[6] = f ? c.fp4.tmem_cols : c.umma.tmem_cols;
+        info[7] = (int32_t)(f ? c.fp4.smem_bytes : c.umma.smem_bytes);
+        info[8] = f ? c.fp4.nb : c.umma.nb;
         info[9] = (int32_t)(K / 32);
-    } else if (kernel == MXQ_KERNEL_MMA) {
-        if (!mxq::linear_mma_plan(M, N, K, p)) {
-            info[0] = -1;
-            return MXQ_OK;
-        }
+    } else if (c.kernel == MXQ_KERNEL_MMA) {
+        const mxq::LinearPlan &p = c.mma;
         info[1] = p.grid;
         info[2] = p.nstage;
         info[3] = p.nwin;
@@ -188,28 +203,23 @@ int mxq_linear_plan_info(int kernel, int M, int64_t N, int64_t K, int32_t *info)
 
 int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
                void *Y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream) {
+    (void)workspace;
+    (void)workspace_bytes;
     if (!X_bf16 || !codes || !scales || !Y) return MXQ_ERR_NULL;
     if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return MXQ_ERR_SHAPE;
     if (y_dtype != MXQ_F32 && y_dtype != MXQ_BF16) return MXQ_ERR_DTYPE;
     if (!mxq::aligned16(X_bf16) || !mxq::aligned16(codes) || !mxq::aligned16(scales) || !mxq::aligned16(Y))
         return MXQ_ERR_ALIGN;
     cudaStream_t st = (cudaStream_t)stream;
-    mxq::UmmaPlan uplan;
-    if (mxq::use_umma(M, N, K, codes, uplan)) {
-        const cudaError_t e = mxq::linear_umma_launch(uplan, X_bf16, codes, scales, Y, y_dtype, st);
+    mxq::Choice c;
+    mxq::choose(mxq::kernel_ceiling(), M, N, K, codes, c);
+    if (c.kernel != MXQ_KERNEL_GENERIC) {
+        const cudaError_t e =
+            c.kernel == MXQ_KERNEL_FP4    ? mxq::linear_fp4_launch(c.fp4, X_bf16, codes, scales, Y, y_dtype, st)
+            : c.kernel == MXQ_KERNEL_UMMA ? mxq::linear_umma_launch(c.umma, X_bf16, codes, scales, Y, y_dtype, st)
+                                          : mxq::linear_mma_launch(c.mma, X_bf16, codes, scales, Y, y_dtype, nullptr, st);
         if (e != cudaSuccess) {
-            if (std::getenv("MXQ_DEBUG")) std::fprintf(stderr, "mxq_linear (tcgen05 kernel): %s\n", cudaGetErrorString(e));
-            (void)cudaGetLastError();
-            return MXQ_ERR_CUDA;
-        }
-        return mxq::launch_status();
-    }
-    mxq::LinearPlan plan;
-    if (!mxq::force_generic() && mxq::linear_mma_plan(M, N, K, plan)) {
-        const size_t need = mxq::linear_mma_workspace_bytes(plan);
-        if (need > 0 && (!workspace || workspace_bytes < need)) return MXQ_ERR_WORKSPACE;
-        if (!mxq::aligned16(workspace)) return MXQ_ERR_ALIGN;
-        if (mxq::linear_mma_launch(plan, X_bf16, codes, scales, Y, y_dtype, workspace, st) != cudaSuccess) {
+            if (std::getenv("MXQ_DEBUG")) std::fprintf(stderr, "mxq_linear (kernel %d): %s\n", c.kernel, cudaGetErrorString(e));
             (void)cudaGetLastError();
             return MXQ_ERR_CUDA;
         }

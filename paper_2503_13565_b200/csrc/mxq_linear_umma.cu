@@ -34,11 +34,12 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
-#include <mutex>
 
 #include "mxq_device.cuh"
 #include "mxq_host.h"
 #include "mxq_linear_umma.h"
+#include "mxq_tcgen05.cuh"
+#include "mxq_tensor_map.h"
 
 namespace mxq {
 
@@ -48,110 +49,12 @@ namespace {
 
 constexpr uint32_t kFullArrivals = 1 + 64;   // TMA thread's expect_tx arrive + one cp.async arrive per scale thread
 
-// ---- small PTX wrappers ----------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// bounded wait: false after about a second
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
-    const uint64_t t0 = global_ns();
-    for (;;) {
-        for (int i = 0; i < 256; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (global_ns() - t0 > 1000000000ull) return false;
-    }
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (int i = 0; i < 64; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity);
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void tma_load_codes(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
-        : "memory");
-}
-__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
-    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// shared-memory matrix descriptor: start address, leading / stride byte offsets (all >> 4), version 1, layout
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo, uint32_t layout) {
-    return (uint64_t)((saddr >> 4) & 0x3FFF) | (uint64_t)((lbo >> 4) & 0x3FFF) << 16 |
-           (uint64_t)((sbo >> 4) & 0x3FFF) << 32 | (uint64_t)1 << 46 | (uint64_t)layout << 61;
-}
-__device__ __forceinline__ void tc_copy_sf(uint32_t tmem, uint32_t atom_saddr) {
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(tmem), "l"(smem_desc(atom_saddr, 0, 128, 0))
-                 : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t sfa, uint32_t sfb,
-                                       uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-        ::"r"(d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
-        : "memory");
-}
-__device__ __forceinline__ void tc_load16(uint32_t taddr, float *v) {
-    uint32_t r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
-}
-// one lane of a converged warp; the surrounding control flow stays warp-uniform, which lets the compiler keep
-// descriptors and barrier addresses in uniform registers (the tcgen05 and TMA instructions take those)
-__device__ __forceinline__ bool elect_one() {
-    uint32_t pred;
-    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
-    return pred != 0;
-}
-__device__ __forceinline__ uint32_t cluster_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ float ld_peer_f32(uint32_t local_saddr, uint32_t rank) {
-    uint32_t raddr;
-    float v;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(local_saddr), "r"(rank));
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(raddr) : "memory");
-    return v;
-}
+// Every partial sum is bounded by sum |x w^|, which cancellation can leave up to 1/2e-3 = 500 times larger than a
+// result that still has to come out finite.  So the token operand's scales carry an extra 2^-kGuard, all sums are
+// formed 2^kGuard too small, and the factor is restored once, at the final store.  (What this costs at the bottom of
+// the FP32 range is far below the layer's absolute tolerance.)
+constexpr int kGuard = 10;
+constexpr float kGuardUp = 1024.f, kGuardDown = 1.f / 1024.f;
 
 // ---- exact split of a scaled BF16 value into E5M2 parts ---------------------------------------------------
 // Largest-magnitude E5M2 number not above |v| (same sign).  Below the E5M2 normal range a non-final part
@@ -166,13 +69,6 @@ __device__ __forceinline__ uint32_t pack_e5m2x2(float lo, float hi) {
     uint16_t out;
     asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(out) : "f"(hi), "f"(lo));
     return out;
-}
-
-__device__ __forceinline__ void store_out(void *Y, int y_dtype, int64_t idx, float v) {
-    if (y_dtype == MXQ_F32)
-        reinterpret_cast<float *>(Y)[idx] = v;
-    else
-        reinterpret_cast<__nv_bfloat16 *>(Y)[idx] = __float2bfloat16_rn(v);
 }
 
 // ---- the kernel ----------------------------------------------------------------------------------------
@@ -192,7 +88,7 @@ __device__ __forceinline__ bool split_unit(const uint4 raw, bool act, int m, int
     emax = max(emax, __shfl_xor_sync(0xffffffffu, emax, 2));
     if (emax == 255u) inexact = true;              // Inf or NaN in the block
     // scale byte of the first part: the block's largest element lands in the top E5M2 binade
-    const uint32_t sb1 = emax < 21u ? 6u : emax - 15u;
+    const uint32_t sb1 = max(emax, 21u + kGuard) - 15u;   // >= 6 + kGuard: the third part's byte, kGuard lower, stays >= 0
     const float down = __uint_as_float((254u - sb1) << 23);   // 2^(127 - sb1)
     uint32_t part[3][2];
 #pragma unroll
@@ -221,7 +117,7 @@ __device__ __forceinline__ bool split_unit(const uint4 raw, bool act, int m, int
             uint8_t *dst = gB + (size_t)j * (NB * 128) + (row >> 3) * 1024 + ((kk >> 4) & 7) * 128 + (row & 7) * 16 + (kk & 15);
             *reinterpret_cast<uint2 *>(dst) = make_uint2(part[p][0], part[p][1]);
             if ((lane & 3) == 0)
-                gSFB[(size_t)j * kUmmaSfAtomBytes + (row & 31) * 16 + (row >> 5) * 4 + ((kk >> 5) & 3)] = (uint8_t)(sb1 - 3 * p);
+                gSFB[(size_t)j * kUmmaSfAtomBytes + (row & 31) * 16 + (row >> 5) * 4 + ((kk >> 5) & 3)] = (uint8_t)(sb1 - kGuard - 3 * p);
         }
     }
     return inexact && act;
@@ -452,7 +348,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
             const uint8_t *srow = scales + n * kb_row;
             for (int blk = s_begin * 4; blk < s_end * 4; ++blk) {
                 const uint4 c = ld_stream_u4(crow + blk);
-                const float sc = e8m0_to_float(srow[blk]);
+                const float sc = e8m0_to_float(srow[blk]) * kGuardDown;
                 const uint32_t w[4] = {c.x, c.y, c.z, c.w};
                 float part[16];
 #pragma unroll
@@ -488,7 +384,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
         if (n < N)
 #pragma unroll
             for (int m = 0; m < 16; ++m)
-                if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, y[m]);
+                if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, y[m] * kGuardUp);
     } else {
         // rank q owns rows [q*128/split, (q+1)*128/split) of the tile: every CTA pushes its partial results
         // for those rows into q's shared memory (slot = sender's rank), one cluster barrier, q adds in rank order
@@ -510,7 +406,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
             float acc = 0.f;
             for (int j = 0; j < split; ++j) acc += gRecv[(j * M + m) * cnt_max + r];
             const int64_t n = n0 + rb + r;
-            if (n < N) store_out(Y, y_dtype, (int64_t)m * N + n, acc);
+            if (n < N) store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp);
         }
     }
     tc_fence_before();
@@ -520,67 +416,6 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
 }
 
 // ---- host side -----------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = [] {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            p = nullptr;
-        (void)cudaGetLastError();
-        return (EncodeTiledFn)p;
-    }();
-    return fn;
-}
-
-// tensor maps depend only on (device, pointer, N, K): keep the recent ones
-struct MapSlot {
-    int dev;
-    const void *ptr;
-    int64_t N, K;
-    CUtensorMap map;
-    bool valid;
-};
-constexpr int kMapSlots = 512;
-MapSlot g_maps[kMapSlots];
-std::mutex g_maps_mutex;
-
-bool codes_tensor_map(const uint8_t *codes, int64_t N, int64_t K, CUtensorMap &out) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    const uint64_t h = (reinterpret_cast<uintptr_t>(codes) >> 8) * 0x9E3779B97F4A7C15ull + (uint64_t)N * 31 + (uint64_t)K;
-    MapSlot &slot = g_maps[(h >> 40) % kMapSlots];
-    std::lock_guard<std::mutex> lock(g_maps_mutex);
-    if (slot.valid && slot.dev == dev && slot.ptr == codes && slot.N == N && slot.K == K) {
-        out = slot.map;
-        return true;
-    }
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)N};
-    const cuuint64_t gstr[1] = {(cuuint64_t)(K / 2)};
-    const cuuint32_t box[2] = {(cuuint32_t)kUmmaStageK, (cuuint32_t)kUmmaTileRows};
-    const cuuint32_t estr[2] = {1, 1};
-    if (fn(&slot.map, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 2, const_cast<uint8_t *>(codes), gdim, gstr, box, estr,
-           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
-        if (std::getenv("MXQ_DEBUG")) std::fprintf(stderr, "mxq: tensor map encode failed for N=%lld K=%lld\n", (long long)N, (long long)K);
-        slot.valid = false;
-        return false;
-    }
-    slot.dev = dev;
-    slot.ptr = codes;
-    slot.N = N;
-    slot.K = K;
-    slot.valid = true;
-    out = slot.map;
-    return true;
-}
-
 int env_int(const char *name) {
     const char *e = std::getenv(name);
     return e ? std::atoi(e) : 0;
@@ -641,7 +476,7 @@ bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p) {
 cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,
                                int y_dtype, cudaStream_t stream) {
     CUtensorMap map;
-    if (!codes_tensor_map(codes, p.N, p.K, map)) return cudaErrorNotSupported;
+    if (!codes_tensor_map(codes, p.N, p.K, /*expand_fp4=*/true, &map)) return cudaErrorNotSupported;
     switch (p.nb) {
         case 16: return launch_umma<16>(p, map, X, codes, scales, Y, y_dtype, stream);
         case 32: return launch_umma<32>(p, map, X, codes, scales, Y, y_dtype, stream);
@@ -649,7 +484,7 @@ cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *
     }
 }
 
-bool linear_umma_available() { return encode_fn() != nullptr; }
+bool linear_umma_available() { return tensor_map_available(); }
 
 }  // namespace mxq
 
@@ -660,7 +495,10 @@ int mxq_linear_device_status(uint32_t *status_host) {
     unsigned int v = 0, zero = 0;
     if (cudaMemcpyFromSymbol(&v, mxq::g_umma_status, sizeof v) != cudaSuccess) return MXQ_ERR_CUDA;
     if (v != 0 && cudaMemcpyToSymbol(mxq::g_umma_status, &zero, sizeof zero) != cudaSuccess) return MXQ_ERR_CUDA;
-    *status_host = v;
+    uint32_t v4 = 0;
+    const int rc = mxq::linear_fp4_take_status(&v4);
+    if (rc != MXQ_OK) return rc;
+    *status_host = v | (v4 << 8);
     return MXQ_OK;
 }
 #pragma GCC visibility pop

@@ -12,10 +12,11 @@ from parity import check_linear, gpu_bf16
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(autouse=True, params=["auto", "mma"])
+@pytest.fixture(autouse=True, params=["auto", "umma", "mma"])
 def linear_kernel(request):
-    """Every case runs twice: with the library's own choice of kernel (the tcgen05 kernel where it covers
-    the shape) and with that kernel excluded (mma.sync kernel, else the generic one)."""
+    """Every case runs three times: with the library's own choice of kernel (the packed-FP4 tcgen05 kernel
+    for up to 4 token rows, the FP8-operand tcgen05 kernel above that, where they cover the shape), capped
+    at the FP8-operand kernel, and capped at the mma.sync kernel (else the generic one)."""
     prev = mxq.mxq_set_linear_kernel(request.param)
     yield request.param
     mxq.mxq_set_linear_kernel(prev)
@@ -76,7 +77,7 @@ def test_every_token_count_on_a_ragged_shape_tensor_core_path(m):
     n, k = 203, 1408   # N not a multiple of 16, K = 44 blocks (a multiple of 128: tensor-core kernel)
     w = synth.bits_of(synth.weight(3, 14, n, k))
     x = synth.bits_of(synth.activations(3, 14, m, k))
-    assert mxq.mxq_linear_plan_info(m, n, k)["kernel"] in ("umma", "mma")
+    assert mxq.mxq_linear_plan_info(m, n, k)["kernel"] in ("fp4", "umma", "mma")
     run_case(w, x, what="ragged tc M=%d" % m)
 
 

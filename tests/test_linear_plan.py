@@ -79,7 +79,7 @@ def test_plan_invariants(m, n, k):
 
 def test_shapes_outside_the_tensor_core_paths_use_the_generic_kernel():
     assert mxq.mxq_linear_plan_info(1, 3, 1 << 20, "mma")["kernel"] is None      # a single row would overflow the stage table
-    for kernel in ("mma", "umma"):
+    for kernel in ("mma", "umma", "fp4"):
         assert mxq.mxq_linear_plan_info(1, 64, 96, kernel)["kernel"] is None      # K % 128 != 0
         assert mxq.mxq_linear_plan_info(1, 203, 1440, kernel)["kernel"] is None
     assert mxq.mxq_linear_workspace_bytes(1, 64, 96) == 0
@@ -128,3 +128,35 @@ def test_tcgen05_plan_invariants(m, n, k):
 def test_tcgen05_kernel_needs_whole_stages():
     assert mxq.mxq_linear_plan_info(1, 4096, 4096 + 64, "umma")["kernel"] is None
     assert mxq.mxq_linear_plan_info(1, 4096, 96, "umma")["kernel"] is None
+
+
+@pytest.mark.parametrize("m,n,k", [(m, n, k) for (m, n, k) in UMMA_SHAPES if m <= 4] + [(2, 11008, 4096), (3, 5000, 1408)])
+def test_packed_fp4_plan_invariants(m, n, k):
+    """Stages of 256 k (the last one half full when K % 256 == 128), sixteen digit planes per token."""
+    p = mxq.mxq_linear_plan_info(m, n, k, "fp4")
+    assert p["kernel"] == "fp4"
+    ks = -(-k // 256)
+    assert p["kb"] == k // 32 and p["tiles"] == -(-n // 128)
+    assert 1 <= p["split"] <= min(8, ks)
+    assert p["grid"] == p["tiles"] * p["split"]
+    assert p["chunk_max"] == -(-ks // p["split"])
+    assert 1 <= p["ring"] <= min(8, p["chunk_max"])
+    assert p["nb"] == {1: 16, 2: 32, 3: 64, 4: 64}[m]
+    assert p["smem_bytes"] <= 227 * 1024
+    assert p["tmem_cols"] in (64, 128) and p["tmem_cols"] >= p["nb"] + 32
+    bounds = [r * ks // p["split"] for r in range(p["split"] + 1)]
+    sizes = [b1 - b0 for b0, b1 in zip(bounds, bounds[1:])]
+    assert bounds[0] == 0 and bounds[-1] == ks and min(sizes) >= 1 and max(sizes) <= p["chunk_max"]
+
+
+def test_packed_fp4_kernel_is_for_few_tokens_and_whole_half_stages():
+    assert mxq.mxq_linear_plan_info(5, 4096, 4096, "fp4")["kernel"] is None
+    assert mxq.mxq_linear_plan_info(1, 4096, 4096 + 64, "fp4")["kernel"] is None
+
+
+def test_headline_shapes_fit_in_one_wave_of_small_ctas():
+    """M=1 on the 7B layers with the packed-FP4 kernel: every CTA resident at once, at least two per SM possible."""
+    for n, k in [(4096, 4096), (11008, 4096), (4096, 11008)]:
+        p = mxq.mxq_linear_plan_info(1, n, k, "fp4")
+        per_sm = (228 * 1024) // (p["smem_bytes"] + 1024)
+        assert per_sm >= 2 and p["grid"] <= SMS * per_sm, p

@@ -22,6 +22,7 @@
 // kernel (mxq_linear_umma.cu): one CTA per (128-row tile, K range), the CTAs of a tile form a cluster and add
 // their partial results through distributed shared memory in rank order; warp 0 issues the MMAs, warp 1 the
 // TMA copies, warps 2-3 the scale copies; the first `ring` stages are requested before griddepcontrol.wait.
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
@@ -32,11 +33,34 @@
 
 namespace mxq {
 
+// Build-time diagnostic (-DMXQ_FP4_TRACE): thread 0 of every CTA records %globaltimer at the phase boundaries of
+// the kernel, in one of three tables chosen by the shape, so that a chain of launches can be laid out on one
+// time axis afterwards (mxq_fp4_trace copies the tables to the host).  Not part of the library's interface.
+#ifdef MXQ_FP4_TRACE
+constexpr int kTraceCtas = 1024, kTracePoints = 16;
+__device__ unsigned long long g_fp4_trace[3][kTraceCtas][kTracePoints];
+// point 0 is %globaltimer (ns, common to all SMs, slow to read); the other points are SM clock cycles since point 0
+#define TR(i)                                                                                                     \
+    do {                                                                                                          \
+        if ((tid == 0 || tid == 64 || tid == 32) && blockIdx.x < kTraceCtas) {                                                              \
+            unsigned long long *row_ = g_fp4_trace[(N >> 7) % 3][blockIdx.x];            \
+            if ((i) == 0) {                                                                                       \
+                row_[0] = global_ns();                                                                            \
+                tr_c0 = clock64();                                                                                \
+            } else {                                                                                              \
+                row_[i] = (unsigned long long)(clock64() - tr_c0);                                                \
+            }                                                                                                     \
+        }                                                                                                         \
+    } while (0)
+#else
+#define TR(i)
+#endif
+
 namespace {
 
 __device__ unsigned int g_fp4_status = 0;   // sticky: bit 0 full-wait, 1 empty-wait, 2 done-wait, 3 drain-wait gave up
 
-constexpr uint32_t kFullArrivals = 1 + 64;   // TMA thread's expect_tx arrive + one cp.async arrive per scale thread
+constexpr uint32_t kFullArrivals = 1 + 32;   // the expect_tx arrive of the TMA lane + one cp.async arrive per producer lane
 
 // Every partial sum is bounded by sum |x w^|, which cancellation can leave up to 1/2e-3 = 500 times larger than a
 // result that still has to come out finite.  So the token operand's scales carry an extra 2^-kGuard, all sums are
@@ -45,13 +69,16 @@ constexpr uint32_t kFullArrivals = 1 + 64;   // TMA thread's expect_tx arrive + 
 constexpr int kGuard = 10;
 constexpr float kGuardUp = 1024.f, kGuardDown = 1.f / 1024.f;
 
-// 8 radix-4 digits (16 bits) -> 8 nibbles holding the digits' E2M1 codes (0, 1, 2, 3 -> 0000, 0010, 0100, 0101)
-__device__ __forceinline__ uint32_t digit_codes(uint32_t v16, uint32_t sign_nibbles) {
-    uint32_t w = (v16 | (v16 << 8)) & 0x00FF00FFu;
-    w = (w | (w << 4)) & 0x0F0F0F0Fu;
-    w = (w | (w << 2)) & 0x33333333u;
-    const uint32_t d1 = (w >> 1) & 0x11111111u, d0 = w & 0x11111111u;
-    return (d1 << 2) | ((d0 & ~d1) << 1) | (d0 & d1) | sign_nibbles;
+__device__ __forceinline__ void st_shared_u32(uint32_t saddr, uint32_t v) {
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(saddr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st_shared_u8(uint32_t saddr, uint32_t v) {
+    asm volatile("st.shared.u8 [%0], %1;" ::"r"(saddr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t mask, uint32_t c) {   // (a & mask) | c
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(mask), "r"(c));
+    return d;
 }
 
 // in place: x[j] nibble i  <-  x[i] nibble j
@@ -73,64 +100,66 @@ __device__ __forceinline__ void transpose_nibbles8(uint32_t (&x)[8]) {
 #pragma unroll
     for (int i = 0; i < 8; i += 2) {
         const uint32_t a = x[i], b = x[i + 1];
-        x[i] = (a & 0x0F0F0F0Fu) | ((b & 0x0F0F0F0Fu) << 4);
-        x[i + 1] = ((a >> 4) & 0x0F0F0F0Fu) | (b & 0xF0F0F0F0u);
+        x[i] = lop3_and_or(a, 0x0F0F0F0Fu, (b & 0x0F0F0F0Fu) << 4);
+        x[i + 1] = lop3_and_or(b, 0xF0F0F0F0u, (a >> 4) & 0x0F0F0F0Fu);
     }
 }
 
-// One 8-element unit of X (token m, k offset kk inside the CTA's range) -> 16 digit planes in B and, from one lane
-// of the four that share a 32-block, the planes' 16 scale bytes.  All 32 lanes call it together.
+// Half of one 8-element unit of X (token m, k offset kk inside the CTA's range): the lane with half = 0 writes digit
+// planes 0..7 into B, its neighbour with half = 1 planes 8..15; the two lanes of a 32-block's first unit also write
+// the planes' scale bytes.  Lane layout inside a warp: lane = 8 * block + 2 * unit + half; all 32 lanes call together.
+// sB_ / sSFB_ are shared-window addresses.  The E2M1 codes 0000, 0001, 0010, 0011 are the values 0, 0.5, 1, 1.5, so a
+// radix-4 digit d is its own code for d / 2; the factor 2 goes into the plane's scale.
 template <int NB>
-__device__ __forceinline__ bool split_unit(const uint4 raw, bool act, int m, int kk, int lane, uint8_t *gB, uint8_t *gSFB) {
+__device__ __forceinline__ bool split_half_unit(const uint4 raw, int m, int kk, int half, int lane, uint32_t sB_, uint32_t sSFB_) {
     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-    uint32_t emax = 0;
+    // largest exponent field of the 32-block: both halves of a word at once, then across the block's four units
+    uint32_t e2 = (w[0] >> 7) & 0x00FF00FFu;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        emax = max(emax, (w[i] >> 7) & 0xFFu);
-        emax = max(emax, (w[i] >> 23) & 0xFFu);
-    }
-    emax = max(emax, __shfl_xor_sync(0xffffffffu, emax, 1));
+    for (int i = 1; i < 4; ++i) e2 = __vmaxu2(e2, (w[i] >> 7) & 0x00FF00FFu);
+    uint32_t emax = max(e2 & 0xFFFFu, e2 >> 16);
     emax = max(emax, __shfl_xor_sync(0xffffffffu, emax, 2));
+    emax = max(emax, __shfl_xor_sync(0xffffffffu, emax, 4));
     bool inexact = emax == 255u;                        // Inf or NaN in the block
-    const uint32_t top = max(emax, 31u + kGuard);       // plane p carries 2^(top - 128 - 2p); its scale byte is kGuard lower
-    uint32_t hi[8], lo[8];
+    // 32-bit fixed point under the block maximum: plane p holds bits 31-2p, 30-2p, worth digit * 2^(top - 128 - 2p)
+    const uint32_t top = max(emax, 31u + kGuard);
+    const float up = __uint_as_float((285u - top) << 23);   // 2^(158 - top), a normal number for every top in 41..254
+    const uint32_t pick = half ? 0x4140u : 0x4342u;          // bytes (b0, 0, b1, 0) of this lane's 16 bits of the fixed point
+    uint32_t pl[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const uint32_t bits = (i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu);
-        const uint32_t e = (bits >> 7) & 0xFFu;
-        const uint32_t sig = (bits & 0x7Fu) | (e ? 0x80u : 0u);             // 8-bit significand
-        const int sh = 24 - (int)(top - max(e, 1u));                         // position of its lowest bit in the 32-bit fixed point
-        const uint32_t down = (uint32_t)min(max(-sh, 0), 8);
-        const uint32_t f = sh >= 0 ? (sig << sh) : (sig >> down);
-        if (sh < 0 && (f << down) != sig) inexact = true;                    // bits fell off the bottom
-        const uint32_t sgn = (bits & 0x8000u) ? 0x88888888u : 0u;
-        hi[i] = digit_codes(f >> 16, sgn);       // nibble j = plane 7 - j
-        lo[i] = digit_codes(f & 0xFFFFu, sgn);   // nibble j = plane 15 - j
+        const uint32_t word = w[i >> 1];
+        const uint32_t mag = (i & 1) ? (word & 0x7FFF0000u) : ((word << 16) & 0x7FFF0000u);   // |x| as FP32 bits
+        // |x| * 2^(158 - top) is the fixed-point value (bit 31 is worth 2^(top - 127)); it is below 2^32, and any
+        // fraction it has is exactly the bits that would fall off the bottom
+        const float scaled = __uint_as_float(mag) * up;
+        const uint32_t f = __float2uint_rz(scaled);
+        if (__uint2float_rn(f) != scaled) inexact = true;
+        const uint32_t sgn = (uint32_t)((int32_t)((i & 1) ? word : (word << 16)) >> 31) & 0x88888888u;
+        uint32_t v = __byte_perm(f, 0u, pick);            // 8 digits in bytes 0 and 2
+        v = (v | (v << 4)) & 0x0F0F0F0Fu;                 // 2 digits per byte
+        pl[i] = lop3_and_or(v | (v << 2), 0x33333333u, sgn);   // one digit (its own code) per nibble, nibble j = plane 8 half + 7 - j
     }
-    transpose_nibbles8(hi);   // now hi[j] = plane 7 - j, nibble i = element i
-    transpose_nibbles8(lo);
-    if (act) {
-        const int j = kk >> 8, kin = kk & 255;
-        uint8_t *dst = gB + (size_t)j * (NB * 128) + (size_t)(m * 2) * 1024 + (kin >> 5) * 128 + ((kin & 31) >> 1);
+    transpose_nibbles8(pl);   // now pl[j] = plane 8 * half + 7 - j, nibble i = element i
+    const uint32_t j = (uint32_t)kk >> 8, kin = (uint32_t)kk & 255u;
+    const uint32_t dst = sB_ + j * (NB * 128) + (uint32_t)(m * 2 + half) * 1024u + (kin >> 5) * 128u + ((kin & 31u) >> 1);
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            *reinterpret_cast<uint32_t *>(dst + (7 - q) * 16) = hi[q];           // planes 0..7: row group 2m, row 7 - q
-            *reinterpret_cast<uint32_t *>(dst + 1024 + (7 - q) * 16) = lo[q];    // planes 8..15: row group 2m + 1
-        }
-        if ((lane & 3) == 0) {
-            const int kb = kin >> 5;
-            uint8_t *sf = gSFB + (size_t)j * kFp4SfStageBytes + (kb >> 2) * 512 + (kb & 3);
+    for (int q = 0; q < 8; ++q) st_shared_u32(dst + (7 - q) * 16, pl[q]);   // row group 2m + half, row 7 - q
+    if ((lane & 6) == 0) {
+        const uint32_t kb = kin >> 5;
+        const uint32_t row0 = (uint32_t)(kFp4Planes * m + 8 * half);   // first of this lane's eight planes (rows of B)
+        const uint32_t sf = sSFB_ + j * kFp4SfStageBytes + (kb >> 2) * 512u + (kb & 3u) + (row0 & 31u) * 16u + (row0 >> 5) * 4u;
+        const uint32_t byte0 = top - kGuard - 16u * half;   // digit d is stored as the code of d / 2: one above 2^(top-128-2p), less the guard
 #pragma unroll
-            for (int p = 0; p < kFp4Planes; ++p) {
-                const int row = kFp4Planes * m + p;
-                sf[(row & 31) * 16 + (row >> 5) * 4] = (uint8_t)(top - 1 - kGuard - 2 * p);
-            }
-        }
+        for (int q = 0; q < 8; ++q) st_shared_u8(sf + q * 16, byte0 - 2 * q);
     }
-    return inexact && act;
+    return inexact;
 }
 
 // NB: columns of the B operand / accumulator = 16 planes x tokens (16, 32 or 64).
+// Warp roles (192 threads): warp 0 issues the MMAs and owns tensor memory; warp 1 is the producer (TMA copies of
+// the codes, cp.async of the scale bytes, barrier set-up); warps 2..5 split the activations stage by stage and,
+// at the end, read the accumulator (one row per thread), exchange partial results and store.
 template <int NB>
 __global__ void __launch_bounds__(kFp4Threads)
 linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 *__restrict__ X, int M,
@@ -138,14 +167,19 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                   void *__restrict__ Y, int y_dtype, int split, int ring, int ks, int chunk_max, int tmem_cols) {
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef MXQ_FP4_TRACE
+    long long tr_c0 = 0;
+#endif
+    TR(0);
     const uint32_t rank = split > 1 ? cluster_rank() : 0u;
     const int tile = blockIdx.x / split;
     const int64_t n0 = (int64_t)tile * kFp4TileRows;
-    const int s_begin = (int)(((int64_t)rank * ks) / split), s_end = (int)(((int64_t)(rank + 1) * ks) / split);
+    // everything below fits in 32 bits (the plan refuses K >= 2^30 and more than 2^20 tiles)
+    const int s_begin = (int)((rank * (uint32_t)ks) / (uint32_t)split), s_end = (int)(((rank + 1u) * (uint32_t)ks) / (uint32_t)split);
     const int nst = s_end - s_begin;   // stages of this CTA (>= 1 because split <= ks)
-    const int kb_row = (int)(K / 32);
+    const int kb_row = (int)((uint32_t)K >> 5);
     const int k_begin = s_begin * kFp4StageK;
-    const int k_len = (int)min((int64_t)nst * kFp4StageK, K - k_begin);   // the tile's last stage may be half full
+    const int k_len = min(nst * kFp4StageK, (int)(uint32_t)K - k_begin);   // the tile's last stage may be half full
     const bool half_tail = (k_len & (kFp4StageK - 1)) != 0;
 
     // carve shared memory (1024-byte aligned for the 128-byte swizzle)
@@ -156,276 +190,343 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
     const uint32_t sB = sSFA + (uint32_t)ring * kFp4SfStageBytes;
     const uint32_t sSFB = sB + (uint32_t)chunk_max * (NB * 128);
     const uint32_t sRecv = sSFB + (uint32_t)chunk_max * kFp4SfStageBytes;   // [split][M][rows of this rank] floats
-    const uint32_t sBar = sRecv + (uint32_t)M * kFp4RecvRows * 4u;           // full[ring], empty[ring], done, holder, fail
-    uint8_t *gB = gbase + (sB - base), *gSFB = gbase + (sSFB - base);
-    const float *gRecv = reinterpret_cast<const float *>(gbase + (sRecv - base));
-    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(gbase + (sBar - base) + (2 * ring + 1) * 8);
-    volatile int &s_fail = *reinterpret_cast<volatile int *>(gbase + (sBar - base) + (2 * ring + 1) * 8 + 4);
+    const uint32_t sBar = sRecv + (uint32_t)M * kFp4RecvRows * 4u;
+    // barriers: full[ring], empty[ring], done, recv, ready[chunk_max]; then the tensor-memory address and two flags
     const uint32_t full0 = sBar, empty0 = sBar + (uint32_t)ring * 8u, done_bar = sBar + (uint32_t)ring * 16u;
+    const uint32_t recv_bar = done_bar + 8u, ready0 = done_bar + 16u;
+    const uint32_t sMisc = ready0 + (uint32_t)chunk_max * 8u;
+    const float *gRecv = reinterpret_cast<const float *>(gbase + (sRecv - base));
+    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(gbase + (sMisc - base));
+    volatile int &s_fail = *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 4);
+    const int row_lo = (int)(rank * kFp4TileRows) / split, row_cnt = (int)((rank + 1) * kFp4TileRows) / split - row_lo;
+    const int groups_per_stage = 2 * M;   // a group = one warp's 32 tasks = 128 k of one token; a task = 8 elements x 8 planes
 
-    // ---- prologue: request the first stages of weights (they do not depend on the previous kernel) --------
+    // ---- prologue: barriers, tensor memory, and the first stages of weights (they do not depend on the previous
+    //      kernel, so all of this runs before griddepcontrol.wait) -----------------------------------------------
     const int pre = nst < ring ? nst : ring;
-    if (tid == 32) {   // the TMA thread sets up the barriers and starts the weight stream at once
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
-        s_fail = 0;
-        for (int i = 0; i < ring; ++i) {
-            mbar_init(full0 + i * 8, kFullArrivals);
-            mbar_init(empty0 + i * 8, 1);
-        }
-        mbar_init(done_bar, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        for (int i = 0; i < pre; ++i) {
-            mbar_expect_tx(full0 + i * 8, kFp4StageBytes);
-            tma_load_codes(sA + (uint32_t)i * kFp4StageBytes, &tmap, (s_begin + i) * (kFp4StageK / 2), (int)n0, full0 + i * 8);
-        }
-    }
-    __syncthreads();
-    pdl_trigger();
-    const int64_t row_a = n0 + (tid - 64), row_b = row_a + 64;   // rows of the scale threads (tid 64..127)
-    const uint8_t *srow_a = scales + row_a * kb_row + (int64_t)s_begin * 8;
-    const uint8_t *srow_b = scales + row_b * kb_row + (int64_t)s_begin * 8;
-    const bool has_a = row_a < N, has_b = row_b < N;
-    const uint32_t sf_a = sSFA + (uint32_t)(((tid - 64) & 31) * 16 + ((tid - 64) >> 5) * 4), sf_b = sf_a + 8;
-    auto copy_scales = [&](int i, uint32_t slot) {   // stage i of this CTA into ring slot `slot`
+    // producer lane l owns rows l, l + 32, l + 64, l + 96 of the tile's scale bytes
+    const uint8_t *srow = scales + (n0 + lane) * kb_row + s_begin * 8;
+    const int64_t srow_step = (int64_t)32 * kb_row;
+    const int rows_here = (int)min((int64_t)kFp4TileRows, N - n0);
+    const uint32_t sf_lane = sSFA + (uint32_t)lane * 16u;
+    auto copy_scales = [&](int i, uint32_t slot) {   // stage i of this CTA into ring slot `slot` (producer warp)
         const bool second = !(half_tail && i == nst - 1);
-        const uint32_t dst = slot * kFp4SfStageBytes;
-        if (has_a) {
-            cp_async4(sf_a + dst, srow_a + i * 8);
-            if (second) cp_async4(sf_a + dst + 512, srow_a + i * 8 + 4);
-        }
-        if (has_b) {
-            cp_async4(sf_b + dst, srow_b + i * 8);
-            if (second) cp_async4(sf_b + dst + 512, srow_b + i * 8 + 4);
+        const uint32_t dst = sf_lane + slot * kFp4SfStageBytes;
+        const uint8_t *src = srow + i * 8;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (lane + 32 * q < rows_here) {
+                cp_async4(dst + 4 * q, src);
+                if (second) cp_async4(dst + 4 * q + 512, src + 4);
+            }
+            src += srow_step;
         }
         cp_async_arrive(full0 + slot * 8);
     };
-    if (warp >= 2) {
-        for (int i = 0; i < pre; ++i) copy_scales(i, (uint32_t)i);
+    if (warp == 1) {
+        for (int b = lane; b < 2 * ring + 2 + nst; b += 32) {
+            const int st = b - (2 * ring + 2);   // >= 0: the barrier of stage st's share of the activations
+            const uint32_t count = b < ring ? kFullArrivals
+                                   : (st < 0 ? 1u : (uint32_t)((half_tail && st == nst - 1) ? M : groups_per_stage));
+            mbar_init(sBar + (uint32_t)b * 8u, count);
+        }
+        if (lane == 31) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
+            s_fail = 0;
+            *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 8) = 0;   // s_bad
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        __syncwarp();
+        TR(8);
+        if (lane == 0) {
+            if (split > 1) mbar_expect_tx(recv_bar, (uint32_t)(split * M * row_cnt) * 4u);   // every rank sends M values per row
+            for (int i = 0; i < pre; ++i) {
+                mbar_expect_tx(full0 + i * 8, kFp4StageBytes);
+                tma_load_codes(sA + (uint32_t)i * kFp4StageBytes, &tmap, (s_begin + i) * (kFp4StageK / 2), (int)n0, full0 + i * 8);
+            }
+        }
+        TR(9);
     } else if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                         sBar + (uint32_t)(2 * ring + 1) * 8),
-                     "r"(tmem_cols)
-                     : "memory");
+        // let the next kernel start launching at once (its CTAs take the shared memory this kernel leaves free and start
+        // their own weight stream); the MMA warp does it because it has nothing urgent to do yet
+        pdl_trigger();
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sMisc), "r"(tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-
-    // ---- X of this CTA's K range -> 16 digit planes per token + their block scales ---------------------------
-    pdl_wait();
-    bool inexact = false;
-    {
-        const int upr = k_len / 8;                 // 8-element units per token row
-        const int total = M * upr;
-        const __nv_bfloat16 *xbase = X + k_begin;
-        for (int u0 = 0; u0 < total; u0 += 2 * kFp4Threads) {
-            uint4 raw[2];
-            int mm[2], kk[2];
-#pragma unroll
-            for (int b = 0; b < 2; ++b) {   // both loads of the batch first
-                const int u = u0 + b * kFp4Threads + tid;
-                const bool act = u < total;
-                mm[b] = act ? u / upr : -1;
-                kk[b] = act ? (u - mm[b] * upr) * 8 : 0;
-                raw[b] = make_uint4(0, 0, 0, 0);
-                if (act) raw[b] = *reinterpret_cast<const uint4 *>(xbase + (int64_t)mm[b] * K + kk[b]);
-            }
-#pragma unroll
-            for (int b = 0; b < 2; ++b)
-                if (u0 + b * kFp4Threads < total)   // uniform across the CTA
-                    inexact |= split_unit<NB>(raw[b], mm[b] >= 0, mm[b], kk[b], lane, gB, gSFB);
-        }
+    // Only the activation warps read what the previous kernel wrote (X) and write what the next one reads (Y), so
+    // only they wait for it; they do so at once, and join the CTA-wide barrier (initialised mbarriers, tensor-memory
+    // address) after that wait.
+    if (warp >= 2) {
+        TR(1);
+        pdl_wait();
+        TR(2);
     }
-    fence_async_proxy();   // B and its scales were written with ordinary stores; the tensor core reads them
+    if (split > 1) cluster_arrive();   // "my barriers exist"; the matching wait is just before the first push to a peer
     tc_fence_before();
-    const int bad = __syncthreads_or(inexact ? 1 : 0);
+    asm volatile("bar.sync 0;" ::: "memory");
     tc_fence_after();
+    if (tid == 64) TR(12);
     const uint32_t tmem = *tmem_holder;
-
+    if (warp == 1)
+        for (int i = 0; i < pre; ++i) copy_scales(i, (uint32_t)i);
     float y[kFp4MaxM];
 #pragma unroll
     for (int m = 0; m < kFp4MaxM; ++m) y[m] = 0.f;
 
-    if (!bad) {
-        if (warp == 0) {
-            // ---- MMA warp: the loop is warp-uniform, one elected lane issues ----------------------------------
-            // descriptors as 32-bit halves: only the start-address field changes from MMA to MMA
-            const uint32_t idesc = (1u << 7) | (1u << 10) | (((uint32_t)NB >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
-            const uint32_t a_hi = (uint32_t)(smem_desc(0, 16, 1024, 2) >> 32), b_hi = (uint32_t)(smem_desc(0, 128, 1024, 0) >> 32);
-            const uint32_t s_hi = (uint32_t)(smem_desc(0, 0, 128, 0) >> 32);
-            const uint32_t a_lo0 = (uint32_t)smem_desc(sA, 16, 1024, 2), s_lo0 = (uint32_t)smem_desc(sSFA, 0, 128, 0);
-            uint32_t b_lo = (uint32_t)smem_desc(sB, 128, 1024, 0), sb_lo = (uint32_t)smem_desc(sSFB, 0, 128, 0);
-            uint32_t slot = 0, phase = 0, accumulate = 0;
-            for (int i = 0; i < nst; ++i) {
-                if (!mbar_wait(full0 + slot * 8, phase)) {
-                    if (lane == 0) {
-                        atomicOr(&g_fp4_status, 1u);
-                        s_fail = 1;
-                    }
-                    break;
-                }
-                tc_fence_after();
-                const uint32_t a_lo = a_lo0 + slot * (kFp4StageBytes >> 4);
-                const uint32_t sa_lo = s_lo0 + slot * (kFp4SfStageBytes >> 4);
-                const int nmma = (half_tail && i == nst - 1) ? 2 : 4;
-                const uint32_t t_sf = tmem + NB + (uint32_t)(i & 1) * 16u;   // two slots of 8 + 8 scale columns, alternating
-                if (elect_one()) {
-                    fence_async_proxy();   // the scale atoms were written by cp.async
-                    tc_copy_sf_lohi(t_sf, sa_lo, s_hi);
-                    tc_copy_sf_lohi(t_sf + 4, sa_lo + 32, s_hi);
-                    tc_copy_sf_lohi(t_sf + 8, sb_lo, s_hi);
-                    tc_copy_sf_lohi(t_sf + 12, sb_lo + 32, s_hi);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        if (j < nmma) {
-                            const uint32_t sfid = (uint32_t)(j & 1) * 2u;   // scales 2 (j & 1), 2 (j & 1) + 1 of atom j >> 1
-                            asm volatile(
-                                "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
-                                "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
-                                "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %5, [%7], [%8], p;\n\t}"
-                                ::"r"(tmem), "r"(a_lo + j * 2), "r"(a_hi), "r"(b_lo + j * 16), "r"(b_hi),
-                                "r"(idesc | (sfid << 4) | (sfid << 29)), "r"(j == 0 ? accumulate : 1u),
-                                "r"(t_sf + 4u * (j >> 1)), "r"(t_sf + 8u + 4u * (j >> 1))
-                                : "memory");
-                        }
-                    tc_commit(empty0 + slot * 8);
-                }
-                __syncwarp();
-                accumulate = 1;
-                b_lo += (NB * 128) >> 4;
-                sb_lo += kFp4SfStageBytes >> 4;
-                if (++slot == (uint32_t)ring) {
-                    slot = 0;
-                    phase ^= 1u;
-                }
-            }
-            if (elect_one()) tc_commit(done_bar);
-            __syncwarp();
-        } else if (warp == 1) {
-            // ---- TMA warp ------------------------------------------------------------------------------------
-            uint32_t slot = 0, phase = 0;   // stage `pre` reuses slot 0 (pre == ring whenever the loop runs)
-            for (int i = pre; i < nst; ++i) {
-                if (!mbar_wait(empty0 + slot * 8, phase)) {
-                    if (lane == 0) {
-                        atomicOr(&g_fp4_status, 2u);
-                        s_fail = 1;
-                    }
-                    break;
-                }
-                if (elect_one()) {
-                    mbar_expect_tx(full0 + slot * 8, kFp4StageBytes);
-                    tma_load_codes(sA + slot * kFp4StageBytes, &tmap, (s_begin + i) * (kFp4StageK / 2), (int)n0, full0 + slot * 8);
-                }
-                __syncwarp();
-                if (++slot == (uint32_t)ring) {
-                    slot = 0;
-                    phase ^= 1u;
-                }
-            }
-        } else {
-            uint32_t slot = 0, phase = 0;
-            for (int i = pre; i < nst; ++i) {
-                if (!mbar_wait(empty0 + slot * 8, phase)) {
-                    atomicOr(&g_fp4_status, 2u);
+    if (warp == 0) {
+        // ---- MMA warp: the loop is warp-uniform, one elected lane issues -------------------------------------------
+        // descriptors as 32-bit halves: only the start-address field changes from MMA to MMA
+        const uint32_t idesc = (1u << 7) | (1u << 10) | (((uint32_t)NB >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+        const uint32_t a_hi = (uint32_t)(smem_desc(0, 16, 1024, 2) >> 32), b_hi = (uint32_t)(smem_desc(0, 128, 1024, 0) >> 32);
+        const uint32_t s_hi = (uint32_t)(smem_desc(0, 0, 128, 0) >> 32);
+        const uint32_t a_lo0 = (uint32_t)smem_desc(sA, 16, 1024, 2), s_lo0 = (uint32_t)smem_desc(sSFA, 0, 128, 0);
+        uint32_t b_lo = (uint32_t)smem_desc(sB, 128, 1024, 0), sb_lo = (uint32_t)smem_desc(sSFB, 0, 128, 0);
+        uint32_t slot = 0, phase = 0, accumulate = 0;
+        for (int i = 0; i < nst; ++i) {
+            // the stage's weights and scales have landed, and its share of the activations has been split
+            if (!mbar_wait_relaxed(ready0 + (uint32_t)i * 8u, 0) || !mbar_wait_relaxed(full0 + slot * 8, phase)) {
+                if (lane == 0) {
+                    atomicOr(&g_fp4_status, 1u);
                     s_fail = 1;
-                    break;
                 }
-                copy_scales(i, slot);
-                if (++slot == (uint32_t)ring) {
-                    slot = 0;
-                    phase ^= 1u;
+                break;
+            }
+            tc_fence_after();
+            const uint32_t a_lo = a_lo0 + slot * (kFp4StageBytes >> 4);
+            const uint32_t sa_lo = s_lo0 + slot * (kFp4SfStageBytes >> 4);
+            const int nmma = (half_tail && i == nst - 1) ? 2 : 4;
+            const uint32_t t_sf = tmem + NB + (uint32_t)(i & 1) * 16u;   // two slots of 8 + 8 scale columns, alternating
+            if (elect_one()) {
+                fence_async_proxy();   // the weight scale atoms were written by cp.async
+                tc_copy_sf_lohi(t_sf, sa_lo, s_hi);
+                tc_copy_sf_lohi(t_sf + 4, sa_lo + 32, s_hi);
+                tc_copy_sf_lohi(t_sf + 8, sb_lo, s_hi);
+                tc_copy_sf_lohi(t_sf + 12, sb_lo + 32, s_hi);
+                auto mma = [&](int j, uint32_t acc) {   // k [64 j, 64 j + 64) of the stage: scales 2 (j & 1), + 1 of atom j >> 1
+                    const uint32_t sfid = (uint32_t)(j & 1) * 2u;
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+                        "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+                        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %5, [%7], [%8], p;\n\t}"
+                        ::"r"(tmem), "r"(a_lo + j * 2), "r"(a_hi), "r"(b_lo + j * 16), "r"(b_hi),
+                        "r"(idesc | (sfid << 4) | (sfid << 29)), "r"(acc), "r"(t_sf + 4u * (j >> 1)), "r"(t_sf + 8u + 4u * (j >> 1))
+                        : "memory");
+                };
+                mma(0, accumulate);
+                mma(1, 1u);
+                if (nmma == 4) {
+                    mma(2, 1u);
+                    mma(3, 1u);
                 }
+                tc_commit(empty0 + slot * 8);
+            }
+            accumulate = 1;
+            b_lo += (NB * 128) >> 4;
+            sb_lo += kFp4SfStageBytes >> 4;
+            if (++slot == (uint32_t)ring) {
+                slot = 0;
+                phase ^= 1u;
             }
         }
-        // ---- epilogue: accumulator row -> registers; a token's 16 planes are 16 columns, smallest first -----
-        if (!mbar_wait(done_bar, 0)) {
+        __syncwarp();
+        if (elect_one()) tc_commit(done_bar);
+        __syncwarp();
+        TR(4);
+    } else if (warp == 1) {
+        // ---- producer warp: refill ring slots as the MMAs release them ----------------------------------------------
+        uint32_t slot = 0, phase = 0;   // stage `pre` reuses slot 0 (pre == ring whenever the loop runs)
+        for (int i = pre; i < nst; ++i) {
+            if (!mbar_wait_relaxed(empty0 + slot * 8, phase)) {
+                if (lane == 0) {
+                    atomicOr(&g_fp4_status, 2u);
+                    s_fail = 1;
+                }
+                break;
+            }
+            if (lane == 0) {
+                mbar_expect_tx(full0 + slot * 8, kFp4StageBytes);
+                tma_load_codes(sA + slot * kFp4StageBytes, &tmap, (s_begin + i) * (kFp4StageK / 2), (int)n0, full0 + slot * 8);
+            }
+            copy_scales(i, slot);
+            if (++slot == (uint32_t)ring) {
+                slot = 0;
+                phase ^= 1u;
+            }
+        }
+    } else {
+        // ---- the four activation / epilogue warps ---------------------------------------------------------------------
+        const int ct = tid - 64;                                   // 0..127
+        const int row = ((warp & 3) << 5) + lane;                  // accumulator row this thread may read (its warp's quarter)
+        volatile int &s_bad = *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 8);
+        bool inexact = false;
+#ifdef MXQ_FP4_TRACE
+        long long tr_split = 0, tr_fence = 0;
+#endif
+        {
+            // Groups of 32 tasks (128 k of one token, one warp) in stage-major order, so that the MMA warp can start on
+            // stage 0 while later stages are being split.  Group G: stage G / (2M), then token and 128-k half; in a half
+            // tail stage every group is a different token.  All of this is uniform across a warp.
+            const int ngroups = (k_len >> 7) * M;
+            const __nv_bfloat16 *xbase = X + k_begin;
+            const int cw = ct >> 5;
+            constexpr int kBatch = 4;   // loads in flight per thread
+            for (int G0 = 0; G0 < ngroups; G0 += 4 * kBatch) {
+                uint4 raw[kBatch];
+                int mm[kBatch], kk[kBatch], stage[kBatch];
+#pragma unroll
+                for (int b = 0; b < kBatch; ++b) {   // all loads of the batch first
+                    const int G = G0 + 4 * b + cw;
+                    mm[b] = -1;
+                    kk[b] = stage[b] = 0;
+                    raw[b] = make_uint4(0, 0, 0, 0);
+                    if (G < ngroups) {
+                        const int st = M == 1 ? (G >> 1) : (M == 2 ? (G >> 2) : (M == 3 ? G / 6 : (G >> 3)));
+                        const int rem = G - st * groups_per_stage;
+                        const bool tail = half_tail && st == nst - 1;
+                        stage[b] = st;
+                        mm[b] = tail ? rem : (rem >> 1);
+                        kk[b] = st * kFp4StageK + (tail ? 0 : (rem & 1) * 128) + (lane >> 1) * 8;
+                        raw[b] = *reinterpret_cast<const uint4 *>(xbase + (int64_t)mm[b] * K + kk[b]);
+                    }
+                }
+                if (G0 == 0) TR(13);
+#pragma unroll
+                for (int b = 0; b < kBatch; ++b)
+                    if (G0 + 4 * b + cw < ngroups) {   // uniform across the warp
+#ifdef MXQ_FP4_TRACE
+                        const long long c0_ = clock64();
+#endif
+                        inexact |= split_half_unit<NB>(raw[b], mm[b], kk[b], lane & 1, lane, sB, sSFB);
+#ifdef MXQ_FP4_TRACE
+                        const long long c1_ = clock64();
+#endif
+                        fence_async_proxy();   // ordinary stores, read by the tensor core
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(ready0 + (uint32_t)stage[b] * 8u);
+#ifdef MXQ_FP4_TRACE
+                        tr_split += c1_ - c0_;
+                        tr_fence += clock64() - c1_;
+#endif
+                    }
+            }
+        }
+        TR(3);
+#ifdef MXQ_FP4_TRACE
+        if (tid == 64 && blockIdx.x < kTraceCtas) {
+            unsigned long long *row_ = g_fp4_trace[(N >> 7) % 3][blockIdx.x];
+            row_[10] = (unsigned long long)tr_split;
+            row_[11] = (unsigned long long)tr_fence;
+        }
+#endif
+        if (inexact) s_bad = 1;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const int bad = s_bad;
+
+        // ---- epilogue: accumulator row -> registers; a token's 16 planes are 16 columns, smallest first ------------
+        if (!mbar_wait_relaxed(done_bar, 0)) {
             atomicOr(&g_fp4_status, 4u);
             s_fail = 1;
         }
+        TR(5);
         tc_fence_after();
-        const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
+        if (!bad) {
+            const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 #pragma unroll
-        for (int m = 0; m < NB / kFp4Planes; ++m) {
-            float d[16];
-            tc_load16(t_row + m * 16, d);
-            float acc = d[15];
+            for (int m = 0; m < NB / kFp4Planes; ++m) {
+                float d[16];
+                tc_load16(t_row + m * 16, d);
+                float acc = d[15];
 #pragma unroll
-            for (int p = 14; p >= 0; --p) acc += d[p];
-            y[m] = acc;
-        }
-    } else {
-        // ---- scalar path for a K range whose X cannot be written as digit planes exactly --------------------
-        // first let the copies requested in the prologue land (nothing may be in flight when the CTA ends)
-        for (int i = 0; i < pre; ++i)
-            if (!mbar_wait(full0 + i * 8, 0)) {
-                atomicOr(&g_fp4_status, 8u);
-                s_fail = 1;
-                break;
+                for (int p = 14; p >= 0; --p) acc += d[p];
+                y[m] = acc;
             }
-        const int64_t n = n0 + tid;
-        if (n < N) {
-            const uint4 *crow = reinterpret_cast<const uint4 *>(codes + n * (K / 2));
-            const uint8_t *srow = scales + n * kb_row;
-            for (int blk = k_begin / 32; blk < (k_begin + k_len) / 32; ++blk) {
-                const uint4 c = ld_stream_u4(crow + blk);
-                const float sc = e8m0_to_float(srow[blk]) * kGuardDown;
-                const uint32_t w[4] = {c.x, c.y, c.z, c.w};
-                float part[kFp4MaxM];
+        } else {
+            // scalar path for a K range whose X cannot be written as digit planes exactly (the MMA results are ignored)
+            const int64_t n = n0 + row;
+            if (n < N) {
+                const uint4 *crow = reinterpret_cast<const uint4 *>(codes + n * (K / 2));
+                const uint8_t *srw = scales + n * kb_row;
+                for (int blk = k_begin / 32; blk < (k_begin + k_len) / 32; ++blk) {
+                    const uint4 c = ld_stream_u4(crow + blk);
+                    const float sc = e8m0_to_float(srw[blk]) * kGuardDown;
+                    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+                    float part[kFp4MaxM];
 #pragma unroll
-                for (int m = 0; m < kFp4MaxM; ++m) part[m] = 0.f;
+                    for (int m = 0; m < kFp4MaxM; ++m) part[m] = 0.f;
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
+                    for (int q = 0; q < 4; ++q)
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float2 wv = __half22float2(e2m1x2_to_half2((w[q] >> (8 * i)) & 0xFFu));
-                        const int64_t k = (int64_t)blk * 32 + q * 8 + i * 2;
+                        for (int i = 0; i < 4; ++i) {
+                            const float2 wv = __half22float2(e2m1x2_to_half2((w[q] >> (8 * i)) & 0xFFu));
+                            const int64_t k = (int64_t)blk * 32 + q * 8 + i * 2;
 #pragma unroll
-                        for (int m = 0; m < kFp4MaxM; ++m)
-                            if (m < M) {
-                                const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * K + k);
-                                part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
-                                part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
-                            }
-                    }
+                            for (int m = 0; m < kFp4MaxM; ++m)
+                                if (m < M) {
+                                    const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * K + k);
+                                    part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
+                                    part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
+                                }
+                        }
 #pragma unroll
-                for (int m = 0; m < kFp4MaxM; ++m) y[m] = fmaf(part[m], sc, y[m]);
+                    for (int m = 0; m < kFp4MaxM; ++m) y[m] = fmaf(part[m], sc, y[m]);
+                }
             }
         }
-    }
-    // ---- result: direct store, or rank-ordered sum across the cluster --------------------------------------
-    __syncthreads();   // s_fail is final
-    if (s_fail) {
+        if (s_fail) {
 #pragma unroll
-        for (int m = 0; m < kFp4MaxM; ++m) y[m] = __uint_as_float(0x7FC00000u);
-    }
-    if (split == 1) {
-        const int64_t n = n0 + tid;
-        if (n < N)
+            for (int m = 0; m < kFp4MaxM; ++m) y[m] = __uint_as_float(0x7FC00000u);
+        }
+
+        // ---- result: direct store, or a sum over the cluster in a fixed order ----------------------------------------
+        if (split == 1) {
+            const int64_t n = n0 + row;
+            if (n < N)
+#pragma unroll
+                for (int m = 0; m < kFp4MaxM; ++m)
+                    if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, y[m] * kGuardUp);
+        } else {
+            // rank q owns rows [q*128/split, (q+1)*128/split) of the tile: every CTA pushes its partial results for
+            // those rows into q's shared memory (slot = sender's rank) with stores that count on q's mbarrier; q waits
+            // for all split * M * rows values and adds them in a fixed order.  No CTA reads a peer's memory, and a CTA
+            // leaves only after everything addressed to it has arrived.
+            const int cnt_max = (kFp4TileRows + split - 1) / split;
+            const uint32_t owner = (uint32_t)(((row + 1) * split - 1) / kFp4TileRows);
+            const int rr = row - (int)(owner * kFp4TileRows) / split;
+            const uint32_t remote = peer_saddr(sRecv, owner), remote_bar = peer_saddr(recv_bar, owner);
+            cluster_wait();   // every CTA of the cluster has initialised its barriers (they arrived long ago)
 #pragma unroll
             for (int m = 0; m < kFp4MaxM; ++m)
-                if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, y[m] * kGuardUp);
-    } else {
-        // rank q owns rows [q*128/split, (q+1)*128/split) of the tile: every CTA pushes its partial results
-        // for those rows into q's shared memory (slot = sender's rank), one cluster barrier, q adds in rank order
-        const int cnt_max = (kFp4TileRows + split - 1) / split;
-        const uint32_t owner = (uint32_t)(((tid + 1) * split - 1) / kFp4TileRows);
-        const int rr = tid - (int)(owner * kFp4TileRows) / split;
-        uint32_t remote;
-        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(sRecv), "r"(owner));
-#pragma unroll
-        for (int m = 0; m < kFp4MaxM; ++m)
-            if (m < M)
-                asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote + (uint32_t)(((int)rank * M + m) * cnt_max + rr) * 4u),
-                             "f"(y[m])
-                             : "memory");
-        cluster_sync_all();
-        const int rb = (int)(rank * kFp4TileRows) / split, cnt = (int)((rank + 1) * kFp4TileRows) / split - rb;
-        for (int idx = tid; idx < M * cnt; idx += kFp4Threads) {
-            const int m = idx / cnt, r = idx - m * cnt;
-            float acc = 0.f;
-            for (int j = 0; j < split; ++j) acc += gRecv[(j * M + m) * cnt_max + r];
-            const int64_t n = n0 + rb + r;
-            if (n < N) store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp);
+                if (m < M) st_async_f32(remote + (uint32_t)(((int)rank * M + m) * cnt_max + rr) * 4u, y[m], remote_bar);
+            if (!mbar_wait_relaxed(recv_bar, 0)) {
+                atomicOr(&g_fp4_status, 16u);
+                s_fail = 1;
+            }
+            TR(6);
+            const float poison = s_fail ? __uint_as_float(0x7FC00000u) : 0.f;
+            if ((split & (split - 1)) == 0) {
+                // power-of-two cluster: one value per thread (row ct / split, sender ct % split), butterfly sum over the
+                // senders in neighbouring lanes; the order of additions is fixed by the lane pattern
+                const int r = ct / split, j = ct & (split - 1);
+                const int64_t n = n0 + row_lo + r;
+                for (int m = 0; m < M; ++m) {
+                    float v = gRecv[(j * M + m) * cnt_max + r];
+                    for (int o = 1; o < split; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                    if (j == 0 && n < N) store_out(Y, y_dtype, (int64_t)m * N + n, v * kGuardUp + poison);
+                }
+            } else {
+                for (int idx = ct; idx < M * row_cnt; idx += 128) {
+                    const int m = idx / row_cnt, r = idx - m * row_cnt;
+                    float acc = 0.f;
+                    for (int j = 0; j < split; ++j) acc += gRecv[(j * M + m) * cnt_max + r];
+                    const int64_t n = n0 + row_lo + r;
+                    if (n < N) store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison);
+                }
+            }
         }
     }
+
+    TR(7);
+    if (split > 1 && warp < 2) cluster_wait();   // pairs with the arrive in the prologue (the other warps waited before their push)
     tc_fence_before();
     __syncthreads();
     if (warp == 0)
@@ -446,6 +547,10 @@ cudaError_t launch_fp4(const Fp4Plan &p, const CUtensorMap &map, const void *X, 
     if (dev >= 0 && dev < 64 && !configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(linear_fp4_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kFp4SmemLimit);
+        if (e != cudaSuccess) return e;
+        // all of the SM's L1/shared array as shared memory: how many CTAs (of this and of the next kernel) fit on an
+        // SM is what decides how early the next kernel's weight stream can start
+        e = cudaFuncSetAttribute(linear_fp4_kernel<NB>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -470,6 +575,22 @@ cudaError_t launch_fp4(const Fp4Plan &p, const CUtensorMap &map, const void *X, 
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
+    if (std::getenv("MXQ_DEBUG_OCC")) {
+        int clusters = -1, blocks = -1;
+        cudaOccupancyMaxActiveClusters(&clusters, linear_fp4_kernel<NB>, &cfg);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, linear_fp4_kernel<NB>, kFp4Threads, p.smem_bytes);
+        std::fprintf(stderr, "mxq fp4: grid %d split %d smem %u: max active clusters %d, blocks per SM %d\n", p.grid, p.split,
+                     p.smem_bytes, clusters, blocks);
+        cudaFuncAttributes fa;
+        cudaFuncGetAttributes(&fa, linear_fp4_kernel<NB>);
+        std::fprintf(stderr, "  regs %d static smem %zu local %zu maxThreads %d maxDyn %d carveout %d\n", fa.numRegs, fa.sharedSizeBytes,
+                     fa.localSizeBytes, fa.maxThreadsPerBlock, fa.maxDynamicSharedSizeBytes, fa.preferredShmemCarveout);
+        for (size_t sm : {(size_t)0, (size_t)16384, (size_t)42608, (size_t)100000})
+            for (int th : {128, 192}) {
+                cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, linear_fp4_kernel<NB>, th, sm);
+                std::fprintf(stderr, "  threads %d smem %zu -> %d blocks per SM\n", th, sm, blocks);
+            }
+    }
     return cudaLaunchKernelEx(&cfg, linear_fp4_kernel<NB>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
                               Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols);
 }
@@ -498,6 +619,14 @@ cudaError_t linear_fp4_launch(const Fp4Plan &p, const void *X, const uint8_t *co
         default: return launch_fp4<64>(p, map, X, codes, scales, Y, y_dtype, stream);
     }
 }
+
+#ifdef MXQ_FP4_TRACE
+}  // namespace mxq
+extern "C" __attribute__((visibility("default"))) int mxq_fp4_trace(unsigned long long *out) {
+    return cudaMemcpyFromSymbol(out, mxq::g_fp4_trace, sizeof(mxq::g_fp4_trace)) == cudaSuccess ? 0 : 6;
+}
+namespace mxq {
+#endif
 
 // returns and clears this kernel's sticky status word (see mxq_linear_device_status)
 int linear_fp4_take_status(uint32_t *out) {

@@ -7,7 +7,7 @@ namespace mxq {
 
 constexpr int kFp4TileRows = 128;    // weight rows per CTA = M of one tcgen05.mma
 constexpr int kFp4StageK = 256;      // k per ring stage = 128 packed bytes per row = 8 MX blocks = 4 MMAs of K = 64
-constexpr int kFp4Threads = 128;
+constexpr int kFp4Threads = 192;     // MMA warp, producer warp, four activation / epilogue warps
 constexpr int kFp4Planes = 16;       // radix-4 digit planes per token (32 bits of fixed point under the block maximum)
 constexpr int kFp4MaxM = 4;          // 16 planes x 4 tokens = 64 columns of the token operand
 constexpr uint32_t kFp4StageBytes = 16384;        // 128 rows x 128 bytes; also what the copy engine counts
@@ -34,7 +34,8 @@ struct Fp4Plan {
 inline uint32_t fp4_smem_bytes(int nb, int chunk, int ring) {
     const uint32_t recv = (uint32_t)(nb / kFp4Planes) * kFp4RecvRows * 4u;   // partial results pushed by the cluster's CTAs
     const uint32_t b = 1024u /* alignment slack */ + (uint32_t)ring * (kFp4StageBytes + kFp4SfStageBytes) +
-                       (uint32_t)chunk * ((uint32_t)nb * 128u + kFp4SfStageBytes) + recv + (uint32_t)(2 * ring + 2) * 8u;
+                       (uint32_t)chunk * ((uint32_t)nb * 128u + kFp4SfStageBytes) + recv +
+                       (uint32_t)(2 * ring + 2 + chunk) * 8u /* mbarriers */ + 16u /* tensor-memory address, flags */;
     return (b + 15u) & ~15u;
 }
 

@@ -41,6 +41,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity);
 }
+// bounded wait for a barrier that is expected to take a while: sleeps between probes, so that a waiting warp does
+// not take issue slots from the warps it is waiting for; false after about a second
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (;;) {
+        for (int i = 0; i < 1024; ++i) {
+            __nanosleep(40);
+            if (mbar_try_wait(bar, parity)) return true;
+        }
+        if (global_ns() - t0 > 1000000000ull) return false;
+    }
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
@@ -110,6 +126,22 @@ __device__ __forceinline__ uint32_t cluster_rank() {
 }
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// split cluster barrier: arrive early, wait late (acquire).  The relaxed arrive orders nothing by itself: what peers
+// must see (initialised mbarriers) is published by fence.mbarrier_init.release.cluster before it.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// address of the same shared-memory location in the CTA of rank `rank` of this cluster
+__device__ __forceinline__ uint32_t peer_saddr(uint32_t local_saddr, uint32_t rank) {
+    uint32_t raddr;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(local_saddr), "r"(rank));
+    return raddr;
+}
+// 4-byte store into a peer's shared memory that also counts 4 bytes on the peer's mbarrier when it lands
+__device__ __forceinline__ void st_async_f32(uint32_t peer_addr, float v, uint32_t peer_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(peer_addr),
+                 "r"(__float_as_uint(v)), "r"(peer_bar)
+                 : "memory");
 }
 __device__ __forceinline__ float ld_peer_f32(uint32_t local_saddr, uint32_t rank) {
     uint32_t raddr;

@@ -116,9 +116,11 @@ int mxq_set_linear_kernel(int kernel);
  * kernel = MXQ_KERNEL_AUTO describes the one mxq_linear would pick under the current cap for a
  * suitably aligned `codes`; another value describes that kernel whether or not it would be picked.
  * info[12] int32; info[0] = the kernel described, or -1 if the requested kernel does not cover the shape.
- *   MXQ_KERNEL_FP4,     [1] CTAs; [2] ring stages; [3] CTAs per cluster (K split); [4] most stages a CTA owns
+ *   MXQ_KERNEL_FP4,     [1] CTAs; [2] ring slots; [3] CTAs per cluster (K split); [4] most stages a CTA owns
  *   MXQ_KERNEL_UMMA:    (a stage is 256 k for FP4, 128 k for UMMA); [5] 128-row tiles; [6] tensor-memory
- *                       columns; [7] dynamic shared memory bytes; [8] columns of the token operand; [9] K/32.
+ *                       columns; [7] dynamic shared memory bytes; [8] columns of the token operand; [9] K/32;
+ *                       [10] tile groups (CTAs = groups x split; a CTA walks the tiles of its group);
+ *                       [11] most tiles in a group.
  *   MXQ_KERNEL_MMA:     [1] CTAs; [2] ring stages; [3] K windows; [4] blocks per window; [5] blocks in the
  *                       last window; [6] most 16-row tiles a CTA owns; [7] dynamic shared memory bytes;
  *                       [8] 8-token column tiles; [9] K/32.

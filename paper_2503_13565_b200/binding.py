@@ -132,8 +132,8 @@ def mxq_linear_workspace_bytes(m: int, n: int, k: int) -> int:
 KERNELS = {"auto": -1, "generic": 0, "mma": 1, "umma": 2, "fp4": 3}
 _KERNEL_NAMES = {v: k for k, v in KERNELS.items()}
 _PLAN_KEYS = {
-    3: ("kernel", "grid", "ring", "split", "chunk_max", "tiles", "tmem_cols", "smem_bytes", "nb", "kb"),
-    2: ("kernel", "grid", "ring", "split", "chunk_max", "tiles", "tmem_cols", "smem_bytes", "nb", "kb"),
+    3: ("kernel", "grid", "ring", "split", "chunk_max", "tiles", "tmem_cols", "smem_bytes", "nb", "kb", "groups", "tiles_max"),
+    2: ("kernel", "grid", "ring", "split", "chunk_max", "tiles", "tmem_cols", "smem_bytes", "nb", "kb", "groups", "tiles_max"),
     1: ("kernel", "grid", "stages", "windows", "bw", "bw_last", "max_tiles", "smem_bytes", "nt8", "kb"),
     0: ("kernel", "grid"),
 }

@@ -160,20 +160,26 @@ __device__ __forceinline__ bool split_half_unit(const uint4 raw, int m, int kk, 
 // Warp roles (192 threads): warp 0 issues the MMAs and owns tensor memory; warp 1 is the producer (TMA copies of
 // the codes, cp.async of the scale bytes, barrier set-up); warps 2..5 split the activations stage by stage and,
 // at the end, read the accumulator (one row per thread), exchange partial results and store.
-template <int NB>
+// MULTI: whether a CTA may own more than one tile (false: exactly one, and the per-tile loops fold away).
+template <int NB, bool MULTI>
 __global__ void __launch_bounds__(kFp4Threads)
 linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 *__restrict__ X, int M,
                   const uint8_t *__restrict__ codes, const uint8_t *__restrict__ scales, int64_t N, int64_t K,
-                  void *__restrict__ Y, int y_dtype, int split, int ring, int ks, int chunk_max, int tmem_cols) {
+                  void *__restrict__ Y, int y_dtype, int split, int ring, int ks, int chunk_max, int tmem_cols, int groups,
+                  int tiles, int tiles_max) {
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef MXQ_FP4_TRACE
     long long tr_c0 = 0;
 #endif
+    if (tid == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");   // needed by the first copy, 1 us from now
     TR(0);
     const uint32_t rank = split > 1 ? cluster_rank() : 0u;
-    const int tile = blockIdx.x / split;
-    const int64_t n0 = (int64_t)tile * kFp4TileRows;
+    const uint32_t group = blockIdx.x / (uint32_t)split;
+    // this CTA's tiles [tile_lo, tile_lo + ntile) and, for all of them, its K range
+    const int tile_lo = (int)((group * (uint32_t)tiles) / (uint32_t)groups);
+    const int ntile = MULTI ? (int)(((group + 1u) * (uint32_t)tiles) / (uint32_t)groups) - tile_lo : 1;
+    const int64_t n0 = (int64_t)tile_lo * kFp4TileRows;   // first weight row of the first tile
     // everything below fits in 32 bits (the plan refuses K >= 2^30 and more than 2^20 tiles)
     const int s_begin = (int)((rank * (uint32_t)ks) / (uint32_t)split), s_end = (int)(((rank + 1u) * (uint32_t)ks) / (uint32_t)split);
     const int nst = s_end - s_begin;   // stages of this CTA (>= 1 because split <= ks)
@@ -189,8 +195,8 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
     const uint32_t sSFA = sA + (uint32_t)ring * kFp4StageBytes;
     const uint32_t sB = sSFA + (uint32_t)ring * kFp4SfStageBytes;
     const uint32_t sSFB = sB + (uint32_t)chunk_max * (NB * 128);
-    const uint32_t sRecv = sSFB + (uint32_t)chunk_max * kFp4SfStageBytes;   // [split][M][rows of this rank] floats
-    const uint32_t sBar = sRecv + (uint32_t)M * kFp4RecvRows * 4u;
+    const uint32_t sRecv = sSFB + (uint32_t)chunk_max * kFp4SfStageBytes;   // [tile][split][M][rows of this rank] floats
+    const uint32_t sBar = sRecv + (uint32_t)(tiles_max * M) * kFp4RecvRows * 4u;
     // barriers: full[ring], empty[ring], done, recv, ready[chunk_max]; then the tensor-memory address and two flags
     const uint32_t full0 = sBar, empty0 = sBar + (uint32_t)ring * 8u, done_bar = sBar + (uint32_t)ring * 16u;
     const uint32_t recv_bar = done_bar + 8u, ready0 = done_bar + 16u;
@@ -203,16 +209,23 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
 
     // ---- prologue: barriers, tensor memory, and the first stages of weights (they do not depend on the previous
     //      kernel, so all of this runs before griddepcontrol.wait) -----------------------------------------------
-    const int pre = nst < ring ? nst : ring;
-    // producer lane l owns rows l, l + 32, l + 64, l + 96 of the tile's scale bytes
-    const uint8_t *srow = scales + (n0 + lane) * kb_row + s_begin * 8;
+    // The CTA's work is a sequence of units (tile, stage), tile-major; unit u goes through ring slot u % ring.
+    const int nunit = ntile * nst;
+    const int pre = nunit < ring ? nunit : ring;
+    // The SM's requests are served roughly in order, so activations asked for behind a ring full of weight copies
+    // arrive late, and everything after the split waits with them.  Only the first two units are requested up
+    // front; the rest of the ring follows once the activations are in, or else at a trickle.
+    const int pre0 = pre < 2 ? pre : 2;
+    volatile int &s_xin = *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 12);   // the activations have arrived
+    // producer lane l owns rows l, l + 32, l + 64, l + 96 of a tile's scale bytes
+    const uint8_t *srow0 = scales + (n0 + lane) * kb_row + s_begin * 8;
     const int64_t srow_step = (int64_t)32 * kb_row;
-    const int rows_here = (int)min((int64_t)kFp4TileRows, N - n0);
     const uint32_t sf_lane = sSFA + (uint32_t)lane * 16u;
-    auto copy_scales = [&](int i, uint32_t slot) {   // stage i of this CTA into ring slot `slot` (producer warp)
+    auto copy_scales = [&](int t, int i, uint32_t slot) {   // unit (t, i) into ring slot `slot` (all lanes of the producer warp)
         const bool second = !(half_tail && i == nst - 1);
         const uint32_t dst = sf_lane + slot * kFp4SfStageBytes;
-        const uint8_t *src = srow + i * 8;
+        const uint8_t *src = srow0 + (int64_t)t * (4 * srow_step) + i * 8;
+        const int rows_here = (int)min((int64_t)kFp4TileRows, N - n0 - (int64_t)t * kFp4TileRows);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             if (lane + 32 * q < rows_here) {
@@ -223,7 +236,12 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
         }
         cp_async_arrive(full0 + slot * 8);
     };
+    auto copy_codes = [&](int t, int i, uint32_t slot) {    // one lane
+        mbar_expect_tx(full0 + slot * 8, kFp4StageBytes);
+        tma_load_codes(sA + slot * kFp4StageBytes, &tmap, (s_begin + i) * (kFp4StageK / 2), (int)n0 + t * kFp4TileRows, full0 + slot * 8);
+    };
     if (warp == 1) {
+        if (tid == 32) TR(14);
         for (int b = lane; b < 2 * ring + 2 + nst; b += 32) {
             const int st = b - (2 * ring + 2);   // >= 0: the barrier of stage st's share of the activations
             const uint32_t count = b < ring ? kFullArrivals
@@ -231,18 +249,22 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
             mbar_init(sBar + (uint32_t)b * 8u, count);
         }
         if (lane == 31) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
             s_fail = 0;
             *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 8) = 0;   // s_bad
+            s_xin = 0;
         }
+        if (tid == 32) TR(15);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         __syncwarp();
         TR(8);
         if (lane == 0) {
-            if (split > 1) mbar_expect_tx(recv_bar, (uint32_t)(split * M * row_cnt) * 4u);   // every rank sends M values per row
-            for (int i = 0; i < pre; ++i) {
-                mbar_expect_tx(full0 + i * 8, kFp4StageBytes);
-                tma_load_codes(sA + (uint32_t)i * kFp4StageBytes, &tmap, (s_begin + i) * (kFp4StageK / 2), (int)n0, full0 + i * 8);
+            if (split > 1) mbar_expect_tx(recv_bar, (uint32_t)(ntile * split * M * row_cnt) * 4u);   // every rank sends M values per tile and row
+            for (int u = 0, t = 0, i = 0; u < pre0; ++u) {
+                copy_codes(t, i, (uint32_t)u);
+                if (++i == nst) {
+                    i = 0;
+                    ++t;
+                }
             }
         }
         TR(9);
@@ -267,11 +289,23 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
     tc_fence_after();
     if (tid == 64) TR(12);
     const uint32_t tmem = *tmem_holder;
-    if (warp == 1)
-        for (int i = 0; i < pre; ++i) copy_scales(i, (uint32_t)i);
-    float y[kFp4MaxM];
+    if (warp == 1) {
+        for (int u = 0, t = 0, i = 0; u < pre; ++u) {
+            if (u >= pre0) {
+                for (int spin = 0; spin < 3 && !s_xin; ++spin) __nanosleep(100);
+                if (lane == 0) copy_codes(t, i, (uint32_t)u);
+            }
+            copy_scales(t, i, (uint32_t)u);
+            if (++i == nst) {
+                i = 0;
+                ++t;
+            }
+        }
+    }
+    constexpr int kResults = MULTI ? 16 : NB / kFp4Planes;
+    float y[kResults];   // results of this thread's row: [tile][token slot]
 #pragma unroll
-    for (int m = 0; m < kFp4MaxM; ++m) y[m] = 0.f;
+    for (int q = 0; q < kResults; ++q) y[q] = 0.f;
 
     if (warp == 0) {
         // ---- MMA warp: the loop is warp-uniform, one elected lane issues -------------------------------------------
@@ -280,22 +314,30 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
         const uint32_t a_hi = (uint32_t)(smem_desc(0, 16, 1024, 2) >> 32), b_hi = (uint32_t)(smem_desc(0, 128, 1024, 0) >> 32);
         const uint32_t s_hi = (uint32_t)(smem_desc(0, 0, 128, 0) >> 32);
         const uint32_t a_lo0 = (uint32_t)smem_desc(sA, 16, 1024, 2), s_lo0 = (uint32_t)smem_desc(sSFA, 0, 128, 0);
-        uint32_t b_lo = (uint32_t)smem_desc(sB, 128, 1024, 0), sb_lo = (uint32_t)smem_desc(sSFB, 0, 128, 0);
-        uint32_t slot = 0, phase = 0, accumulate = 0;
-        for (int i = 0; i < nst; ++i) {
-            // the stage's weights and scales have landed, and its share of the activations has been split
-            if (!mbar_wait_relaxed(ready0 + (uint32_t)i * 8u, 0) || !mbar_wait_relaxed(full0 + slot * 8, phase)) {
+        const uint32_t b_lo0 = (uint32_t)smem_desc(sB, 128, 1024, 0), sb_lo0 = (uint32_t)smem_desc(sSFB, 0, 128, 0);
+        const uint32_t t_sf0 = tmem + (uint32_t)(NB * tiles_max);   // after the accumulators: two slots of 8 + 8 scale columns
+        uint32_t slot = 0, phase = 0, par = 0;
+        bool ok = true;
+        for (int t = 0; t < ntile && ok; ++t) {
+          const uint32_t t_acc = tmem + (uint32_t)(t * NB);   // this tile's accumulator columns
+          uint32_t b_lo = b_lo0, sb_lo = sb_lo0, accumulate = 0;
+          for (int i = 0; i < nst; ++i) {
+            // the unit's weights and scales have landed and (first tile only; the others find it done) the stage's
+            // share of the activations has been split
+            if ((t == 0 && !mbar_wait_relaxed(ready0 + (uint32_t)i * 8u, 0)) || !mbar_wait_relaxed(full0 + slot * 8, phase)) {
                 if (lane == 0) {
                     atomicOr(&g_fp4_status, 1u);
                     s_fail = 1;
                 }
+                ok = false;
                 break;
             }
             tc_fence_after();
             const uint32_t a_lo = a_lo0 + slot * (kFp4StageBytes >> 4);
             const uint32_t sa_lo = s_lo0 + slot * (kFp4SfStageBytes >> 4);
             const int nmma = (half_tail && i == nst - 1) ? 2 : 4;
-            const uint32_t t_sf = tmem + NB + (uint32_t)(i & 1) * 16u;   // two slots of 8 + 8 scale columns, alternating
+            const uint32_t t_sf = t_sf0 + par * 16u;   // alternating between consecutive units
+            par ^= 1u;
             if (elect_one()) {
                 fence_async_proxy();   // the weight scale atoms were written by cp.async
                 tc_copy_sf_lohi(t_sf, sa_lo, s_hi);
@@ -308,7 +350,7 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                         "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
                         "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
                         "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %5, [%7], [%8], p;\n\t}"
-                        ::"r"(tmem), "r"(a_lo + j * 2), "r"(a_hi), "r"(b_lo + j * 16), "r"(b_hi),
+                        ::"r"(t_acc), "r"(a_lo + j * 2), "r"(a_hi), "r"(b_lo + j * 16), "r"(b_hi),
                         "r"(idesc | (sfid << 4) | (sfid << 29)), "r"(acc), "r"(t_sf + 4u * (j >> 1)), "r"(t_sf + 8u + 4u * (j >> 1))
                         : "memory");
                 };
@@ -327,6 +369,7 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                 slot = 0;
                 phase ^= 1u;
             }
+          }
         }
         __syncwarp();
         if (elect_one()) tc_commit(done_bar);
@@ -334,8 +377,9 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
         TR(4);
     } else if (warp == 1) {
         // ---- producer warp: refill ring slots as the MMAs release them ----------------------------------------------
-        uint32_t slot = 0, phase = 0;   // stage `pre` reuses slot 0 (pre == ring whenever the loop runs)
-        for (int i = pre; i < nst; ++i) {
+        uint32_t slot = 0, phase = 0;   // unit `pre` reuses slot 0 (pre == ring whenever the loop runs)
+        int t = pre / nst, i = pre - t * nst;
+        for (int u = pre; u < nunit; ++u) {
             if (!mbar_wait_relaxed(empty0 + slot * 8, phase)) {
                 if (lane == 0) {
                     atomicOr(&g_fp4_status, 2u);
@@ -343,11 +387,12 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                 }
                 break;
             }
-            if (lane == 0) {
-                mbar_expect_tx(full0 + slot * 8, kFp4StageBytes);
-                tma_load_codes(sA + slot * kFp4StageBytes, &tmap, (s_begin + i) * (kFp4StageK / 2), (int)n0, full0 + slot * 8);
+            if (lane == 0) copy_codes(t, i, slot);
+            copy_scales(t, i, slot);
+            if (++i == nst) {
+                i = 0;
+                ++t;
             }
-            copy_scales(i, slot);
             if (++slot == (uint32_t)ring) {
                 slot = 0;
                 phase ^= 1u;
@@ -397,6 +442,7 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                         const long long c0_ = clock64();
 #endif
                         inexact |= split_half_unit<NB>(raw[b], mm[b], kk[b], lane & 1, lane, sB, sSFB);
+                        if (G0 == 0 && b == 0 && ct == 0) s_xin = 1;   // lets the producer request the rest of the ring
 #ifdef MXQ_FP4_TRACE
                         const long long c1_ = clock64();
 #endif
@@ -423,6 +469,8 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
         const int bad = s_bad;
 
         // ---- epilogue: accumulator row -> registers; a token's 16 planes are 16 columns, smallest first ------------
+        constexpr int MT = NB / kFp4Planes;   // token slots per tile (1, 2 or 4)
+        constexpr int TCAP = MULTI ? 16 / MT : 1;   // tiles a thread can keep results for
         if (!mbar_wait_relaxed(done_bar, 0)) {
             atomicOr(&g_fp4_status, 4u);
             s_fail = 1;
@@ -432,71 +480,96 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
         if (!bad) {
             const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 #pragma unroll
-            for (int m = 0; m < NB / kFp4Planes; ++m) {
-                float d[16];
-                tc_load16(t_row + m * 16, d);
-                float acc = d[15];
+            for (int t = 0; t < TCAP; ++t)
+                if (t < ntile) {
 #pragma unroll
-                for (int p = 14; p >= 0; --p) acc += d[p];
-                y[m] = acc;
-            }
-        } else {
-            // scalar path for a K range whose X cannot be written as digit planes exactly (the MMA results are ignored)
-            const int64_t n = n0 + row;
-            if (n < N) {
-                const uint4 *crow = reinterpret_cast<const uint4 *>(codes + n * (K / 2));
-                const uint8_t *srw = scales + n * kb_row;
-                for (int blk = k_begin / 32; blk < (k_begin + k_len) / 32; ++blk) {
-                    const uint4 c = ld_stream_u4(crow + blk);
-                    const float sc = e8m0_to_float(srw[blk]) * kGuardDown;
-                    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
-                    float part[kFp4MaxM];
+                    for (int m = 0; m < MT; ++m) {
+                        float d[16];
+                        tc_load16(t_row + t * NB + m * 16, d);
+                        float acc = d[15];
 #pragma unroll
-                    for (int m = 0; m < kFp4MaxM; ++m) part[m] = 0.f;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const float2 wv = __half22float2(e2m1x2_to_half2((w[q] >> (8 * i)) & 0xFFu));
-                            const int64_t k = (int64_t)blk * 32 + q * 8 + i * 2;
-#pragma unroll
-                            for (int m = 0; m < kFp4MaxM; ++m)
-                                if (m < M) {
-                                    const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * K + k);
-                                    part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
-                                    part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
-                                }
-                        }
-#pragma unroll
-                    for (int m = 0; m < kFp4MaxM; ++m) y[m] = fmaf(part[m], sc, y[m]);
+                        for (int p = 14; p >= 0; --p) acc += d[p];
+                        y[t * MT + m] = acc;
+                    }
                 }
+        } else {
+            // Scalar path for a K range whose X cannot be written as digit planes exactly (the MMA results are ignored).
+            // Results pass through the ring's shared memory, which is idle once every MMA has completed.
+            float *scratch = reinterpret_cast<float *>(gbase);
+            for (int t = 0; t < ntile; ++t) {
+                const int64_t n = n0 + (int64_t)t * kFp4TileRows + row;
+                float acc[kFp4MaxM];
+#pragma unroll
+                for (int m = 0; m < kFp4MaxM; ++m) acc[m] = 0.f;
+                if (n < N) {
+                    const uint4 *crow = reinterpret_cast<const uint4 *>(codes + n * (K / 2));
+                    const uint8_t *srw = scales + n * kb_row;
+                    for (int blk = k_begin / 32; blk < (k_begin + k_len) / 32; ++blk) {
+                        const uint4 c = ld_stream_u4(crow + blk);
+                        const float sc = e8m0_to_float(srw[blk]) * kGuardDown;
+                        const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+                        float part[kFp4MaxM];
+#pragma unroll
+                        for (int m = 0; m < kFp4MaxM; ++m) part[m] = 0.f;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float2 wv = __half22float2(e2m1x2_to_half2((w[q] >> (8 * i)) & 0xFFu));
+                                const int64_t k = (int64_t)blk * 32 + q * 8 + i * 2;
+#pragma unroll
+                                for (int m = 0; m < kFp4MaxM; ++m)
+                                    if (m < M) {
+                                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * K + k);
+                                        part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
+                                        part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
+                                    }
+                            }
+#pragma unroll
+                        for (int m = 0; m < kFp4MaxM; ++m) acc[m] = fmaf(part[m], sc, acc[m]);
+                    }
+                }
+#pragma unroll
+                for (int m = 0; m < MT; ++m) scratch[(t * MT + m) * kFp4TileRows + row] = acc[m];
             }
+#pragma unroll
+            for (int q = 0; q < kResults; ++q)
+                if (q < ntile * MT) y[q] = scratch[q * kFp4TileRows + row];   // the thread's own values, back in registers
         }
         if (s_fail) {
 #pragma unroll
-            for (int m = 0; m < kFp4MaxM; ++m) y[m] = __uint_as_float(0x7FC00000u);
+            for (int q = 0; q < kResults; ++q) y[q] = __uint_as_float(0x7FC00000u);
         }
 
         // ---- result: direct store, or a sum over the cluster in a fixed order ----------------------------------------
         if (split == 1) {
-            const int64_t n = n0 + row;
-            if (n < N)
 #pragma unroll
-                for (int m = 0; m < kFp4MaxM; ++m)
-                    if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, y[m] * kGuardUp);
+            for (int t = 0; t < TCAP; ++t)
+                if (t < ntile) {
+                    const int64_t n = n0 + (int64_t)t * kFp4TileRows + row;
+                    if (n < N)
+#pragma unroll
+                        for (int m = 0; m < MT; ++m)
+                            if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, y[t * MT + m] * kGuardUp);
+                }
         } else {
-            // rank q owns rows [q*128/split, (q+1)*128/split) of the tile: every CTA pushes its partial results for
-            // those rows into q's shared memory (slot = sender's rank) with stores that count on q's mbarrier; q waits
-            // for all split * M * rows values and adds them in a fixed order.  No CTA reads a peer's memory, and a CTA
-            // leaves only after everything addressed to it has arrived.
+            // Rank q owns rows [q*128/split, (q+1)*128/split) of every tile of the group: every CTA pushes its partial
+            // results for those rows into q's shared memory (slot = tile, sender's rank) with stores that count on q's
+            // mbarrier; q waits for all of them and adds them in a fixed order.  No CTA reads a peer's memory, and a
+            // CTA leaves only after everything addressed to it has arrived.
             const int cnt_max = (kFp4TileRows + split - 1) / split;
             const uint32_t owner = (uint32_t)(((row + 1) * split - 1) / kFp4TileRows);
             const int rr = row - (int)(owner * kFp4TileRows) / split;
             const uint32_t remote = peer_saddr(sRecv, owner), remote_bar = peer_saddr(recv_bar, owner);
             cluster_wait();   // every CTA of the cluster has initialised its barriers (they arrived long ago)
 #pragma unroll
-            for (int m = 0; m < kFp4MaxM; ++m)
-                if (m < M) st_async_f32(remote + (uint32_t)(((int)rank * M + m) * cnt_max + rr) * 4u, y[m], remote_bar);
+            for (int t = 0; t < TCAP; ++t)
+                if (t < ntile) {
+#pragma unroll
+                    for (int m = 0; m < MT; ++m)
+                        if (m < M)
+                            st_async_f32(remote + (uint32_t)(((t * split + (int)rank) * M + m) * cnt_max + rr) * 4u, y[t * MT + m], remote_bar);
+                }
             if (!mbar_wait_relaxed(recv_bar, 0)) {
                 atomicOr(&g_fp4_status, 16u);
                 s_fail = 1;
@@ -507,18 +580,21 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                 // power-of-two cluster: one value per thread (row ct / split, sender ct % split), butterfly sum over the
                 // senders in neighbouring lanes; the order of additions is fixed by the lane pattern
                 const int r = ct / split, j = ct & (split - 1);
-                const int64_t n = n0 + row_lo + r;
-                for (int m = 0; m < M; ++m) {
-                    float v = gRecv[(j * M + m) * cnt_max + r];
-                    for (int o = 1; o < split; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                    if (j == 0 && n < N) store_out(Y, y_dtype, (int64_t)m * N + n, v * kGuardUp + poison);
+                for (int t = 0; t < ntile; ++t) {
+                    const int64_t n = n0 + (int64_t)t * kFp4TileRows + row_lo + r;
+                    for (int m = 0; m < M; ++m) {
+                        float v = gRecv[((t * split + j) * M + m) * cnt_max + r];
+                        for (int o = 1; o < split; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                        if (j == 0 && n < N) store_out(Y, y_dtype, (int64_t)m * N + n, v * kGuardUp + poison);
+                    }
                 }
             } else {
-                for (int idx = ct; idx < M * row_cnt; idx += 128) {
-                    const int m = idx / row_cnt, r = idx - m * row_cnt;
+                for (int idx = ct; idx < ntile * M * row_cnt; idx += 128) {
+                    const int t = idx / (M * row_cnt), rem = idx - t * (M * row_cnt);
+                    const int m = rem / row_cnt, r = rem - m * row_cnt;
                     float acc = 0.f;
-                    for (int j = 0; j < split; ++j) acc += gRecv[(j * M + m) * cnt_max + r];
-                    const int64_t n = n0 + row_lo + r;
+                    for (int j = 0; j < split; ++j) acc += gRecv[((t * split + j) * M + m) * cnt_max + r];
+                    const int64_t n = n0 + (int64_t)t * kFp4TileRows + row_lo + r;
                     if (n < N) store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison);
                 }
             }
@@ -538,19 +614,19 @@ int env_int(const char *name) {
     return e ? std::atoi(e) : 0;
 }
 
-template <int NB>
+template <int NB, bool MULTI>
 cudaError_t launch_fp4(const Fp4Plan &p, const CUtensorMap &map, const void *X, const uint8_t *codes,
                        const uint8_t *scales, void *Y, int y_dtype, cudaStream_t stream) {
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(linear_fp4_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(linear_fp4_kernel<NB, MULTI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kFp4SmemLimit);
         if (e != cudaSuccess) return e;
         // all of the SM's L1/shared array as shared memory: how many CTAs (of this and of the next kernel) fit on an
         // SM is what decides how early the next kernel's weight stream can start
-        e = cudaFuncSetAttribute(linear_fp4_kernel<NB>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(linear_fp4_kernel<NB, MULTI>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -575,24 +651,8 @@ cudaError_t launch_fp4(const Fp4Plan &p, const CUtensorMap &map, const void *X, 
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    if (std::getenv("MXQ_DEBUG_OCC")) {
-        int clusters = -1, blocks = -1;
-        cudaOccupancyMaxActiveClusters(&clusters, linear_fp4_kernel<NB>, &cfg);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, linear_fp4_kernel<NB>, kFp4Threads, p.smem_bytes);
-        std::fprintf(stderr, "mxq fp4: grid %d split %d smem %u: max active clusters %d, blocks per SM %d\n", p.grid, p.split,
-                     p.smem_bytes, clusters, blocks);
-        cudaFuncAttributes fa;
-        cudaFuncGetAttributes(&fa, linear_fp4_kernel<NB>);
-        std::fprintf(stderr, "  regs %d static smem %zu local %zu maxThreads %d maxDyn %d carveout %d\n", fa.numRegs, fa.sharedSizeBytes,
-                     fa.localSizeBytes, fa.maxThreadsPerBlock, fa.maxDynamicSharedSizeBytes, fa.preferredShmemCarveout);
-        for (size_t sm : {(size_t)0, (size_t)16384, (size_t)42608, (size_t)100000})
-            for (int th : {128, 192}) {
-                cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, linear_fp4_kernel<NB>, th, sm);
-                std::fprintf(stderr, "  threads %d smem %zu -> %d blocks per SM\n", th, sm, blocks);
-            }
-    }
-    return cudaLaunchKernelEx(&cfg, linear_fp4_kernel<NB>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
-                              Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols);
+    return cudaLaunchKernelEx(&cfg, linear_fp4_kernel<NB, MULTI>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
+                              Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols, p.groups, p.tiles, p.tiles_max);
 }
 
 }  // namespace
@@ -613,20 +673,19 @@ cudaError_t linear_fp4_launch(const Fp4Plan &p, const void *X, const uint8_t *co
                               int y_dtype, cudaStream_t stream) {
     CUtensorMap map;
     if (!codes_tensor_map(codes, p.N, p.K, /*expand_fp4=*/false, &map)) return cudaErrorNotSupported;
+    const bool multi = p.tiles_max > 1;
     switch (p.nb) {
-        case 16: return launch_fp4<16>(p, map, X, codes, scales, Y, y_dtype, stream);
-        case 32: return launch_fp4<32>(p, map, X, codes, scales, Y, y_dtype, stream);
-        default: return launch_fp4<64>(p, map, X, codes, scales, Y, y_dtype, stream);
+        case 16:
+            return multi ? launch_fp4<16, true>(p, map, X, codes, scales, Y, y_dtype, stream)
+                         : launch_fp4<16, false>(p, map, X, codes, scales, Y, y_dtype, stream);
+        case 32:
+            return multi ? launch_fp4<32, true>(p, map, X, codes, scales, Y, y_dtype, stream)
+                         : launch_fp4<32, false>(p, map, X, codes, scales, Y, y_dtype, stream);
+        default:
+            return multi ? launch_fp4<64, true>(p, map, X, codes, scales, Y, y_dtype, stream)
+                         : launch_fp4<64, false>(p, map, X, codes, scales, Y, y_dtype, stream);
     }
 }
-
-#ifdef MXQ_FP4_TRACE
-}  // namespace mxq
-extern "C" __attribute__((visibility("default"))) int mxq_fp4_trace(unsigned long long *out) {
-    return cudaMemcpyFromSymbol(out, mxq::g_fp4_trace, sizeof(mxq::g_fp4_trace)) == cudaSuccess ? 0 : 6;
-}
-namespace mxq {
-#endif
 
 // returns and clears this kernel's sticky status word (see mxq_linear_device_status)
 int linear_fp4_take_status(uint32_t *out) {

@@ -12,75 +12,120 @@ constexpr int kFp4Planes = 16;       // radix-4 digit planes per token (32 bits 
 constexpr int kFp4MaxM = 4;          // 16 planes x 4 tokens = 64 columns of the token operand
 constexpr uint32_t kFp4StageBytes = 16384;        // 128 rows x 128 bytes; also what the copy engine counts
 constexpr uint32_t kFp4SfStageBytes = 1024;       // two 512-byte scale atoms (4 blocks each) per stage
-constexpr int kFp4MaxRing = 8;
 constexpr int kFp4MaxSplit = 8;                   // portable cluster size
 constexpr uint32_t kFp4RecvRows = 136;            // >= split * ceil(128 / split) for every split <= 8
 constexpr uint32_t kFp4SmemLimit = 227 * 1024;
 
 struct Fp4Plan {
     int M;           // token rows (1..4)
-    int nb;          // columns of the token operand: 16, 32 or 64 (sixteen planes per token)
+    int nb;          // columns of the token operand per tile: 16, 32 or 64 (sixteen planes per token)
     int ks;          // ceil(K / 256), stages per tile; the last one is half full when K % 256 == 128
     int tiles;       // ceil(N / 128)
-    int split;       // CTAs (cluster size) sharing one tile; CTA r takes stages [r*ks/split, (r+1)*ks/split)
-    int ring;        // stages in flight per CTA
+    int split;       // CTAs (cluster size) sharing a group of tiles; CTA r takes stages [r*ks/split, (r+1)*ks/split)
+    int groups;      // tile groups; group g owns tiles [g*tiles/groups, (g+1)*tiles/groups)
+    int tiles_max;   // most tiles in a group = ceil(tiles / groups)
+    int ring;        // (tile, stage) units in flight per CTA
     int chunk_max;   // most stages any CTA owns = ceil(ks / split)
-    int grid;        // tiles * split
+    int grid;        // groups * split
     int tmem_cols;   // tensor-memory columns allocated per CTA
     uint32_t smem_bytes;
     int64_t N, K;
 };
 
-inline uint32_t fp4_smem_bytes(int nb, int chunk, int ring) {
-    const uint32_t recv = (uint32_t)(nb / kFp4Planes) * kFp4RecvRows * 4u;   // partial results pushed by the cluster's CTAs
+constexpr int kFp4MaxUnitsResident = 12;   // most ring slots (16 KB of codes + 1 KB of scales each)
+
+inline uint32_t fp4_smem_bytes(int nb, int M, int tiles_max, int chunk, int ring) {
+    const uint32_t recv = (uint32_t)(tiles_max * M) * kFp4RecvRows * 4u;   // partial results pushed by the cluster's CTAs
     const uint32_t b = 1024u /* alignment slack */ + (uint32_t)ring * (kFp4StageBytes + kFp4SfStageBytes) +
                        (uint32_t)chunk * ((uint32_t)nb * 128u + kFp4SfStageBytes) + recv +
-                       (uint32_t)(2 * ring + 2 + chunk) * 8u /* mbarriers */ + 16u /* tensor-memory address, flags */;
+                       (uint32_t)(2 * ring + 2 + chunk) * 8u /* mbarriers */ + 16u /* tensor-memory address, three flags */;
     return (b + 15u) & ~15u;
 }
 
-// how many CTAs of `bytes` dynamic shared memory fit on one SM (each also takes 1 KB of system use)
-inline int fp4_ctas_per_sm(uint32_t bytes) { return (int)((228u * 1024u) / (bytes + 1024u)); }
+inline int fp4_tmem_cols(int nb, int tiles_max) {
+    const int need = nb * tiles_max + 32;   // one accumulator per tile + two slots of (8 + 8) scale columns
+    int cols = 32;
+    while (cols < need) cols *= 2;
+    return cols;
+}
 
-// Chooses split and ring for p.{M, nb, ks, tiles}; false if no choice fits in shared memory.
-// Measured on B200: a call is fastest when all of its CTAs are resident at once (one wave) and there are about
-// two per SM, so that one CTA's serial phases (activation split, epilogue, cluster sum) hide behind another's
-// weight stream; small CTAs also leave room for the next kernel's CTAs to start their weight stream early.
+// CTAs of this kernel that fit on one SM: shared memory (each CTA also takes 1 KB of system use) and tensor-memory
+// columns (512 per SM).  The occupancy calculator reports 1 for any kernel that contains tcgen05.alloc, but the hardware
+// does place several such CTAs on an SM when these two resources allow (checked on B200 by recording %smid and
+// residency intervals).
+inline int fp4_ctas_per_sm(uint32_t smem_bytes, int tmem_cols) {
+    const int by_smem = (int)((228u * 1024u) / (smem_bytes + 1024u)), by_tmem = 512 / tmem_cols;
+    return by_smem < by_tmem ? by_smem : by_tmem;
+}
+
+// Chooses split, groups and ring for p.{M, nb, ks, tiles}; false if nothing fits.
+//
+// Two regimes, both measured on B200:
+//  - up to 2 * SMs tiles (the transformer layers themselves): one tile per CTA; the deepest ring up to 4 stages that
+//    still lets every CTA of the call be resident at once; the split that brings the CTA count closest to two per
+//    SM.  Small CTAs matter twice: the call runs as one wave, and what it leaves free of an SM's shared memory is taken
+//    by the CTAs of the next call (programmatic dependent launch), which start their weight stream early.
+//  - more tiles (vocabulary projections): one CTA per SM walking several tiles with a deep ring, so that the
+//    activations of a K range are split once per CTA and the pipeline never drains between tiles; the cost of a
+//    choice is the number of (tile, stage) units per CTA, ties to the larger split.
 // force_split / force_ring (> 0) override the heuristic where they are feasible.
 inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring) {
-    int best_split = 0, best_ring = 0;
+    const int tcap_regs = 16 / (p.nb / kFp4Planes);  // results a thread keeps in registers: tiles * token slots <= 16
+    const int tcap_tmem = (512 - 32) / p.nb;
+    const int tcap = tcap_regs < tcap_tmem ? tcap_regs : tcap_tmem;
+    const bool layer_regime = p.tiles <= 2 * sms;
     long best_cost = -1;
+    int best_split = 0, best_groups = 0, best_ring = 0;
     const int smax = p.ks < kFp4MaxSplit ? p.ks : kFp4MaxSplit;
     for (int s = 1; s <= smax; ++s) {
         if (force_split > 0 && s != (force_split < smax ? force_split : smax)) continue;
         const int chunk = (p.ks + s - 1) / s;
-        const long ctas = (long)p.tiles * s;
-        // deepest ring up to 4 stages that still lets every CTA be resident at once; if none does, 4 stages
-        int ring = chunk < 4 ? chunk : 4;
-        if (force_ring > 0) ring = force_ring < chunk ? force_ring : chunk;
-        else
-            while (ring > 2 && ctas > (long)sms * fp4_ctas_per_sm(fp4_smem_bytes(p.nb, chunk, ring))) --ring;
-        while (ring > 1 && fp4_smem_bytes(p.nb, chunk, ring) > kFp4SmemLimit) --ring;
-        const uint32_t bytes = fp4_smem_bytes(p.nb, chunk, ring);
-        if (bytes > kFp4SmemLimit) continue;
-        const long slots = (long)sms * fp4_ctas_per_sm(bytes);
-        const long waves = (ctas + slots - 1) / slots;
-        const long off = ctas > 2L * sms ? ctas - 2L * sms : 2L * sms - ctas;   // distance from two CTAs per SM
-        long cost = (waves - 1) * 100000 + off;
-        if (waves > 1) cost = 100000 + (chunk > 8 ? chunk - 8 : 8 - chunk);      // many waves: about 8 stages per CTA
-        if (best_cost < 0 || cost < best_cost) {
+        int groups, ring;
+        long cost;
+        if (layer_regime) {
+            groups = p.tiles;
+            const long ctas = (long)groups * s;
+            const int tm = fp4_tmem_cols(p.nb, 1);
+            ring = chunk < 4 ? chunk : 4;
+            if (force_ring > 0) ring = force_ring < chunk ? force_ring : chunk;
+            else
+                while (ring > 2 && ctas > (long)sms * fp4_ctas_per_sm(fp4_smem_bytes(p.nb, p.M, 1, chunk, ring), tm)) --ring;
+            while (ring > 1 && fp4_smem_bytes(p.nb, p.M, 1, chunk, ring) > kFp4SmemLimit) --ring;
+            const uint32_t bytes = fp4_smem_bytes(p.nb, p.M, 1, chunk, ring);
+            if (bytes > kFp4SmemLimit) continue;
+            const long slots = (long)sms * fp4_ctas_per_sm(bytes, tm);
+            const long waves = (ctas + slots - 1) / slots;
+            const long off = ctas > 2L * sms ? ctas - 2L * sms : 2L * sms - ctas;   // distance from two CTAs per SM
+            cost = (waves - 1) * 100000 + off;
+        } else {
+            groups = sms / s < 1 ? 1 : sms / s;          // one CTA per SM
+            if (groups > p.tiles) groups = p.tiles;
+            if ((p.tiles + groups - 1) / groups > tcap) groups = (p.tiles + tcap - 1) / tcap;
+            const int tmax = (p.tiles + groups - 1) / groups;
+            const int units = tmax * chunk;
+            ring = units < kFp4MaxUnitsResident ? units : kFp4MaxUnitsResident;
+            if (force_ring > 0 && force_ring < ring) ring = force_ring;
+            while (ring > 1 && fp4_smem_bytes(p.nb, p.M, tmax, chunk, ring) > kFp4SmemLimit) --ring;
+            if (fp4_smem_bytes(p.nb, p.M, tmax, chunk, ring) > kFp4SmemLimit) continue;
+            const long waves = ((long)groups * s + sms - 1) / sms;
+            cost = waves * units * 8 + chunk + (s > 1 ? 2 : 0);
+        }
+        if (best_cost < 0 || cost < best_cost || cost == best_cost) {   // ties: the larger split (less of X per CTA)
             best_cost = cost;
             best_split = s;
+            best_groups = groups;
             best_ring = ring;
         }
     }
     if (best_cost < 0) return false;
     p.split = best_split;
+    p.groups = best_groups;
+    p.tiles_max = (p.tiles + best_groups - 1) / best_groups;
     p.ring = best_ring;
     p.chunk_max = (p.ks + best_split - 1) / best_split;
-    p.grid = p.tiles * best_split;
-    p.smem_bytes = fp4_smem_bytes(p.nb, p.chunk_max, best_ring);
-    p.tmem_cols = p.nb + 32 <= 64 ? 64 : 128;   // accumulator + two slots of (8 + 8) scale columns
+    p.grid = best_groups * best_split;
+    p.smem_bytes = fp4_smem_bytes(p.nb, p.M, p.tiles_max, p.chunk_max, best_ring);
+    p.tmem_cols = fp4_tmem_cols(p.nb, p.tiles_max);
     return true;
 }
 

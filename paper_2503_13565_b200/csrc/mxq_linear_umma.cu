@@ -458,16 +458,6 @@ cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    if (std::getenv("MXQ_DEBUG_OCC")) {
-        int blocks = -1;
-        cudaFuncAttributes fa;
-        cudaFuncGetAttributes(&fa, linear_umma_kernel<NB>);
-        std::fprintf(stderr, "umma: regs %d static smem %zu local %zu maxThreads %d\n", fa.numRegs, fa.sharedSizeBytes, fa.localSizeBytes, fa.maxThreadsPerBlock);
-        for (size_t sm : {(size_t)0, (size_t)42608, (size_t)100000}) {
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, linear_umma_kernel<NB>, 128, sm);
-            std::fprintf(stderr, "  umma threads 128 smem %zu -> %d blocks per SM\n", sm, blocks);
-        }
-    }
     return cudaLaunchKernelEx(&cfg, linear_umma_kernel<NB>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
                               Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols);
 }

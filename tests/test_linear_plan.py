@@ -130,23 +130,33 @@ def test_tcgen05_kernel_needs_whole_stages():
     assert mxq.mxq_linear_plan_info(1, 4096, 96, "umma")["kernel"] is None
 
 
-@pytest.mark.parametrize("m,n,k", [(m, n, k) for (m, n, k) in UMMA_SHAPES if m <= 4] + [(2, 11008, 4096), (3, 5000, 1408)])
+@pytest.mark.parametrize("m,n,k", [(m, n, k) for (m, n, k) in UMMA_SHAPES if m <= 4] + [(2, 11008, 4096), (3, 5000, 1408),
+                                   (1, 128256, 4096), (4, 128256, 4096), (2, 1000000, 128)])
 def test_packed_fp4_plan_invariants(m, n, k):
-    """Stages of 256 k (the last one half full when K % 256 == 128), sixteen digit planes per token."""
+    """Stages of 256 k (the last one half full when K % 256 == 128), sixteen digit planes per token; a CTA owns a K
+    range (its rank in the cluster) of a group of tiles."""
     p = mxq.mxq_linear_plan_info(m, n, k, "fp4")
     assert p["kernel"] == "fp4"
     ks = -(-k // 256)
-    assert p["kb"] == k // 32 and p["tiles"] == -(-n // 128)
+    tiles = -(-n // 128)
+    assert p["kb"] == k // 32 and p["tiles"] == tiles
     assert 1 <= p["split"] <= min(8, ks)
-    assert p["grid"] == p["tiles"] * p["split"]
+    assert 1 <= p["groups"] <= tiles and p["grid"] == p["groups"] * p["split"]
+    assert p["tiles_max"] == -(-tiles // p["groups"])
     assert p["chunk_max"] == -(-ks // p["split"])
-    assert 1 <= p["ring"] <= min(8, p["chunk_max"])
-    assert p["nb"] == {1: 16, 2: 32, 3: 64, 4: 64}[m]
+    assert 1 <= p["ring"] <= min(12, p["tiles_max"] * p["chunk_max"])
+    slots = {1: 1, 2: 2, 3: 4, 4: 4}[m]
+    assert p["nb"] == 16 * slots
+    assert p["tiles_max"] * slots <= 16                      # results a thread keeps in registers
     assert p["smem_bytes"] <= 227 * 1024
-    assert p["tmem_cols"] in (64, 128) and p["tmem_cols"] >= p["nb"] + 32
+    assert p["tmem_cols"] in (32, 64, 128, 256, 512) and p["tmem_cols"] >= p["nb"] * p["tiles_max"] + 32
+    # stage ranges of a cluster's CTAs partition [0, ks); tile ranges of the groups partition [0, tiles)
     bounds = [r * ks // p["split"] for r in range(p["split"] + 1)]
     sizes = [b1 - b0 for b0, b1 in zip(bounds, bounds[1:])]
     assert bounds[0] == 0 and bounds[-1] == ks and min(sizes) >= 1 and max(sizes) <= p["chunk_max"]
+    tb = [g * tiles // p["groups"] for g in range(p["groups"] + 1)]
+    tsz = [b1 - b0 for b0, b1 in zip(tb, tb[1:])]
+    assert tb[0] == 0 and tb[-1] == tiles and min(tsz) >= 1 and max(tsz) == p["tiles_max"]
 
 
 def test_packed_fp4_kernel_is_for_few_tokens_and_whole_half_stages():
@@ -154,9 +164,14 @@ def test_packed_fp4_kernel_is_for_few_tokens_and_whole_half_stages():
     assert mxq.mxq_linear_plan_info(1, 4096, 4096 + 64, "fp4")["kernel"] is None
 
 
-def test_headline_shapes_fit_in_one_wave_of_small_ctas():
-    """M=1 on the 7B layers with the packed-FP4 kernel: every CTA resident at once, at least two per SM possible."""
-    for n, k in [(4096, 4096), (11008, 4096), (4096, 11008)]:
+def test_packed_fp4_regimes():
+    """Transformer-layer shapes: one tile per CTA, every CTA of the call resident at once with room to spare for the
+    next call's CTAs.  Vocabulary projection with a thousand tiles: one CTA per SM, each walking several tiles."""
+    for n, k in [(4096, 4096), (11008, 4096), (4096, 11008), (5120, 5120), (13824, 5120), (5120, 13824)]:
         p = mxq.mxq_linear_plan_info(1, n, k, "fp4")
-        per_sm = (228 * 1024) // (p["smem_bytes"] + 1024)
+        assert p["tiles_max"] == 1 and p["groups"] == p["tiles"]
+        per_sm = min((228 * 1024) // (p["smem_bytes"] + 1024), 512 // p["tmem_cols"])
         assert per_sm >= 2 and p["grid"] <= SMS * per_sm, p
+        assert SMS < p["grid"] <= 2.5 * SMS and p["ring"] <= 4
+    p = mxq.mxq_linear_plan_info(1, 128256, 4096, "fp4")
+    assert p["tiles_max"] > 1 and p["grid"] <= SMS

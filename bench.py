@@ -36,6 +36,11 @@ UNIT = "GB/s"
 HBM_DATASHEET_GBS = 8000.0
 
 
+# DRAM bytes (read + write) over algorithmic bytes of one mxq_linear launch, from the committed profiler summary of the
+# 11008x4096 M=1 launch (profiles/mxq_linear_fp4_m1_11008x4096_full.md): 24.034816 MB / 23.957504 MB
+DRAM_OVER_ALGORITHMIC = 24.034816 / 23.957504
+
+
 def algorithmic_bytes(m: int, n: int, k: int, y_bytes: int = 4) -> int:
     """4.25 bits per weight + activations + outputs (the byte count the metric is defined on)."""
     return n * k // 2 + n * k // 32 + 2 * m * k + y_bytes * m * n
@@ -305,6 +310,20 @@ def run_ours(args):
                 per_shape["%s_m%d" % (name, mm)] = {"us_per_call": s / 20 / len(sel) * 1e6,
                                                     "gbs": p.bytes * 20 / s / 1e9}
         extra["per_shape"] = per_shape
+        # vocabulary projections (one launch streams 70 / 279 MB): where launch latency no longer hides the kernel
+        vocab = {}
+        for n, copies in ((32000, 3), (128256, 2)):
+            gen = torch.Generator(device=device).manual_seed(n)
+            sel = [("lm_head", n, 4096,
+                    torch.randint(0, 256, (n, 2048), dtype=torch.uint8, device=device, generator=gen),
+                    torch.randint(110, 126, (n, 128), dtype=torch.uint8, device=device, generator=gen)) for _ in range(copies)]
+            for mm in (1, 4):
+                p = LinearPass(mxq, sel, mm, device, seed=34, use_graph=not args.no_graph)
+                s = p.time(10, 3)
+                vocab["%dx4096_m%d" % (n, mm)] = {"us_per_call": s / 10 / len(sel) * 1e6, "gbs": p.bytes * 10 / s / 1e9,
+                                                  "frac_of_peak": p.bytes * 10 / s / 1e9 / peaks["hbm_gbs"]}
+            del sel
+        extra["vocab_projection"] = vocab
         # direct cast throughput (2 B read + 0.53125 B written per weight)
         w = synth.student_t_bf16((11008, 4096), 0.02, 1, device=device)
         ws_ = [w.clone() for _ in range(4)]   # 360 MB rotated: larger than L2
@@ -345,7 +364,10 @@ def run_ours(args):
                 "steps": e2e_steps},
         "gpu_launches": main.launches * args.steps,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_kind": "of " + peak_kind,
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": DRAM_OVER_ALGORITHMIC * bytes_step / main.launches,
+                     "traffic_kind": "dram read+write bytes of one profiler capture of the 11008x4096 launch "
+                                     "(24.03 MB against 23.96 MB algorithmic), scaled to the average launch",
+                     "peak_kind": "of " + peak_kind,
                      "kernel": "mxq_linear M=%d" % m, "bytes_per_launch": bytes_step / main.launches},
         "cpu_baseline": cpu,
         "extra": extra,
@@ -358,6 +380,38 @@ def run_ours(args):
 # ---------------------------------------------------------------------------------------------
 # reference arm: the oracle on the host cores
 # ---------------------------------------------------------------------------------------------
+def run_case(args):
+    """One mxq_linear shape, launched `steps` times on a few distinct weight matrices (together larger than L2):
+    the small case that profiler captures run on.  Prints one JSON line with the device time per call."""
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product has no CPU path")
+    import paper_2503_13565_b200 as mxq
+    mxq.binding.lib()
+    n, k, m = (int(v) for v in args.case.lower().split("x"))
+    device = torch.device("cuda", 0)
+    nbytes = algorithmic_bytes(m, n, k)
+    copies = max(2, min(8, int(200e6 // nbytes) + 1))
+    gen = torch.Generator(device=device).manual_seed(7)
+    mats = [(torch.randint(0, 256, (n, k // 2), dtype=torch.uint8, device=device, generator=gen),
+             torch.randint(110, 126, (n, k // 32), dtype=torch.uint8, device=device, generator=gen)) for _ in range(copies)]
+    x = synth.normal_bf16((m, k), 1.0, 3, device)
+    y = torch.empty((m, n), dtype=torch.float32, device=device)
+    for c, s in mats[:1]:
+        mxq.mxq_linear(x, c, s, out=y)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        c, s = mats[i % copies]
+        mxq.mxq_linear(x, c, s, out=y)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / args.steps
+    print(json.dumps({"case": args.case, "kernel": mxq.mxq_linear_plan_info(m, n, k)["kernel"], "launches": args.steps,
+                      "us_per_call": us, "gbs": nbytes / us / 1e3, "bytes_per_call": nbytes,
+                      "device_status": mxq.mxq_linear_device_status()}))
+
+
 def run_reference(args):
     rank, _, world = replicas.env_world()
     if rank != 0:
@@ -412,7 +466,12 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch from Python instead of replaying a CUDA graph")
     ap.add_argument("--quick", action="store_true", help="skip the extra measurements")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--case", default=None, metavar="NxKxM",
+                    help="instead of the benchmark: launch this one mxq_linear shape --steps times (profiler captures)")
     args = ap.parse_args()
+    if args.case:
+        run_case(args)
+        return
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)

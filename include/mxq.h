@@ -102,18 +102,20 @@ size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K);
  *                      token row split exactly into three E5M2 rows (needs K % 128 == 0, a 32-byte aligned `codes`)
  *   MXQ_KERNEL_MMA     decodes the codes into FP16 mma.sync fragments (needs K % 128 == 0)
  *   MXQ_KERNEL_GENERIC any valid shape, on the CUDA cores
- * mxq_linear uses the first of these, in this order, that is allowed (next call) and covers the call. */
+ * Left to itself (MXQ_KERNEL_AUTO) mxq_linear picks by measured speed among the kernels that cover the call: FP4
+ * for M = 1; from M = 2, UMMA for matrices of at most as many row tiles of 128 as the GPU has SMs, MMA for larger ones. */
 enum mxq_kernel {
     MXQ_KERNEL_AUTO = -1, MXQ_KERNEL_GENERIC = 0, MXQ_KERNEL_MMA = 1, MXQ_KERNEL_UMMA = 2, MXQ_KERNEL_FP4 = 3
 };
 
-/* Caps mxq_linear's choice (tests, comparisons): kernels listed above `kernel` are not used; MXQ_KERNEL_AUTO
- * (or MXQ_KERNEL_FP4) lifts the cap.  Returns the previous cap.  Host-side, process-wide.  The initial cap comes
- * from the environment variable MXQ_LINEAR_VARIANT (umma | mma | generic), else there is none. */
+/* Overrides mxq_linear's choice (tests, comparisons): with a kernel of the list, mxq_linear uses the first of FP4,
+ * UMMA, MMA, GENERIC that is not above it and covers the call; MXQ_KERNEL_AUTO restores the default.  Returns the
+ * previous setting.  Host-side, process-wide.  The initial setting comes from the environment variable
+ * MXQ_LINEAR_VARIANT (fp4 | umma | mma | generic), else MXQ_KERNEL_AUTO. */
 int mxq_set_linear_kernel(int kernel);
 
 /* How a kernel would run this shape on the current device (diagnostics; launches nothing).
- * kernel = MXQ_KERNEL_AUTO describes the one mxq_linear would pick under the current cap for a
+ * kernel = MXQ_KERNEL_AUTO describes the one mxq_linear would pick under the current setting for a
  * suitably aligned `codes`; another value describes that kernel whether or not it would be picked.
  * info[12] int32; info[0] = the kernel described, or -1 if the requested kernel does not cover the shape.
  *   MXQ_KERNEL_FP4,     [1] CTAs; [2] ring slots; [3] CTAs per cluster (K split); [4] most stages a CTA owns

@@ -140,7 +140,8 @@ _PLAN_KEYS = {
 
 
 def mxq_set_linear_kernel(kernel) -> str:
-    """Cap mxq_linear's choice of kernel ("auto"/"fp4" = no cap, "umma", "mma", "generic"); returns the previous cap."""
+    """Override mxq_linear's choice of kernel: "auto" (default: by measured speed), or "fp4" / "umma" / "mma" /
+    "generic" = the first kernel not above that one that covers the call.  Returns the previous setting."""
     code = KERNELS[kernel] if isinstance(kernel, str) else int(kernel)
     return _KERNEL_NAMES[int(lib().mxq_set_linear_kernel(code))]
 

@@ -102,24 +102,31 @@ static void launch_rowwarp(const void *X, int M, const uint8_t *codes, const uin
                        K, Y, y_dtype);
 }
 
-// mxq_set_linear_kernel / MXQ_LINEAR_VARIANT: the highest kernel mxq_linear may use (MXQ_KERNEL_* order)
+// mxq_set_linear_kernel / MXQ_LINEAR_VARIANT: MXQ_KERNEL_AUTO (-1), or the highest kernel mxq_linear may use
 static std::atomic<int> g_ceiling{-2};
 static int kernel_ceiling() {
     int v = g_ceiling.load(std::memory_order_relaxed);
     if (v < -1) {
         const char *e = std::getenv("MXQ_LINEAR_VARIANT");
-        v = MXQ_KERNEL_FP4;
+        v = MXQ_KERNEL_AUTO;
         if (e && std::strcmp(e, "generic") == 0) v = MXQ_KERNEL_GENERIC;
         else if (e && std::strcmp(e, "mma") == 0) v = MXQ_KERNEL_MMA;
         else if (e && std::strcmp(e, "umma") == 0) v = MXQ_KERNEL_UMMA;
+        else if (e && std::strcmp(e, "fp4") == 0) v = MXQ_KERNEL_FP4;
         g_ceiling.store(v, std::memory_order_relaxed);
     }
     return v;
 }
 
-// The kernel mxq_linear runs for this call: the first of FP4, UMMA, MMA, GENERIC that is not above the ceiling
-// and covers the shape.  The tcgen05 kernels read the codes through a tensor map (FP4: 16-byte aligned base,
-// which every call has; UMMA: 32-byte aligned base); codes == nullptr means "suitably aligned".
+// The kernel mxq_linear runs for this call.
+//   ceiling >= 0: the first of FP4, UMMA, MMA, GENERIC that is not above the ceiling and covers the call.
+//   MXQ_KERNEL_AUTO: the same order, except that measured speed decides among the kernels that cover the call
+//   (B200, layer shapes and vocabulary projections, M = 1..16): the packed-FP4 kernel wins at M = 1 everywhere;
+//   from M = 2 its activation split (16 planes per token) costs more than the FP8-operand kernel's (3 parts per
+//   token), which wins on layer-sized matrices; on matrices of more row tiles of 128 than SMs with M >= 2 the
+//   mma.sync kernel's row-range decomposition wins.
+// The tcgen05 kernels read the codes through a tensor map (FP4: 16-byte aligned base, which every call has; UMMA:
+// 32-byte aligned base); codes == nullptr means "suitably aligned".
 struct Choice {
     int kernel;
     Fp4Plan fp4;
@@ -128,11 +135,18 @@ struct Choice {
 };
 static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *codes, Choice &c) {
     const bool tc = linear_umma_available();
-    if (ceiling >= MXQ_KERNEL_FP4 && tc && linear_fp4_plan(M, N, K, c.fp4)) c.kernel = MXQ_KERNEL_FP4;
-    else if (ceiling >= MXQ_KERNEL_UMMA && tc && (!codes || (reinterpret_cast<uintptr_t>(codes) & 31u) == 0) &&
-             linear_umma_plan(M, N, K, c.umma))
-        c.kernel = MXQ_KERNEL_UMMA;
-    else if (ceiling >= MXQ_KERNEL_MMA && linear_mma_plan(M, N, K, c.mma)) c.kernel = MXQ_KERNEL_MMA;
+    const bool aligned32 = !codes || (reinterpret_cast<uintptr_t>(codes) & 31u) == 0;
+    bool try_fp4 = ceiling == MXQ_KERNEL_AUTO || ceiling >= MXQ_KERNEL_FP4;
+    bool try_umma = ceiling == MXQ_KERNEL_AUTO || ceiling >= MXQ_KERNEL_UMMA;
+    const bool try_mma = ceiling == MXQ_KERNEL_AUTO || ceiling >= MXQ_KERNEL_MMA;
+    if (ceiling == MXQ_KERNEL_AUTO && M >= 2) {
+        try_fp4 = false;
+        const int64_t tiles = (N + 127) / 128;
+        if (tiles > (int64_t)sm_count() && linear_mma_plan(M, N, K, c.mma)) try_umma = false;
+    }
+    if (try_fp4 && tc && linear_fp4_plan(M, N, K, c.fp4)) c.kernel = MXQ_KERNEL_FP4;
+    else if (try_umma && tc && aligned32 && linear_umma_plan(M, N, K, c.umma)) c.kernel = MXQ_KERNEL_UMMA;
+    else if (try_mma && linear_mma_plan(M, N, K, c.mma)) c.kernel = MXQ_KERNEL_MMA;
     else c.kernel = MXQ_KERNEL_GENERIC;
 }
 
@@ -148,7 +162,7 @@ size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K) {
 
 int mxq_set_linear_kernel(int kernel) {
     const int prev = mxq::kernel_ceiling();
-    mxq::g_ceiling.store(kernel < MXQ_KERNEL_GENERIC || kernel > MXQ_KERNEL_FP4 ? MXQ_KERNEL_FP4 : kernel,
+    mxq::g_ceiling.store(kernel < MXQ_KERNEL_GENERIC || kernel > MXQ_KERNEL_FP4 ? MXQ_KERNEL_AUTO : kernel,
                          std::memory_order_relaxed);
     return prev;
 }

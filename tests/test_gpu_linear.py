@@ -12,11 +12,11 @@ from parity import check_linear, gpu_bf16
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(autouse=True, params=["auto", "umma", "mma"])
+@pytest.fixture(autouse=True, params=["auto", "fp4", "umma", "mma"])
 def linear_kernel(request):
-    """Every case runs three times: with the library's own choice of kernel (the packed-FP4 tcgen05 kernel
-    for up to 4 token rows, the FP8-operand tcgen05 kernel above that, where they cover the shape), capped
-    at the FP8-operand kernel, and capped at the mma.sync kernel (else the generic one)."""
+    """Every case runs four times: with the library's own choice of kernel (by measured speed), and with the choice
+    capped at the packed-FP4 tcgen05 kernel (used for up to 4 token rows wherever it covers the shape), at the
+    FP8-operand tcgen05 kernel, and at the mma.sync kernel (else the generic one)."""
     prev = mxq.mxq_set_linear_kernel(request.param)
     yield request.param
     mxq.mxq_set_linear_kernel(prev)

@@ -198,8 +198,8 @@ int mxq_linear_plan_info(int kernel, int M, int64_t N, int64_t K, int32_t *info)
         info[7] = (int32_t)(f ? c.fp4.smem_bytes : c.umma.smem_bytes);
         info[8] = f ? c.fp4.nb : c.umma.nb;
         info[9] = (int32_t)(K / 32);
-        info[10] = f ? c.fp4.groups : c.umma.tiles;
-        info[11] = f ? c.fp4.tiles_max : 1;
+        info[10] = f ? c.fp4.groups : c.umma.groups;
+        info[11] = f ? c.fp4.tiles_max : c.umma.tiles_max;
     } else if (c.kernel == MXQ_KERNEL_MMA) {
         const mxq::LinearPlan &p = c.mma;
         info[1] = p.grid;

@@ -666,7 +666,7 @@ bool linear_fp4_plan(int M, int64_t N, int64_t K, Fp4Plan &p) {
     p.nb = M == 1 ? 16 : (M == 2 ? 32 : 64);
     p.ks = (int)((K + kFp4StageK - 1) / kFp4StageK);
     p.tiles = (int)((N + kFp4TileRows - 1) / kFp4TileRows);
-    return fp4_layout(p, sm_count(), env_int("MXQ_FP4_SPLIT"), env_int("MXQ_FP4_RING"));
+    return fp4_layout(p, sm_count(), env_int("MXQ_FP4_SPLIT"), env_int("MXQ_FP4_RING"), env_int("MXQ_FP4_TILES"));
 }
 
 cudaError_t linear_fp4_launch(const Fp4Plan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,

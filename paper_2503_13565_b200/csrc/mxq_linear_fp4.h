@@ -69,7 +69,7 @@ inline int fp4_ctas_per_sm(uint32_t smem_bytes, int tmem_cols) {
 //    activations of a K range are split once per CTA and the pipeline never drains between tiles; the cost of a
 //    choice is the number of (tile, stage) units per CTA, ties to the larger split.
 // force_split / force_ring (> 0) override the heuristic where they are feasible.
-inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring) {
+inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring, int force_tiles = 0) {
     const int tcap_regs = 16 / (p.nb / kFp4Planes);  // results a thread keeps in registers: tiles * token slots <= 16
     const int tcap_tmem = (512 - 32) / p.nb;
     const int tcap = tcap_regs < tcap_tmem ? tcap_regs : tcap_tmem;
@@ -83,15 +83,18 @@ inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring) {
         int groups, ring;
         long cost;
         if (layer_regime) {
-            groups = p.tiles;
+            int tper = force_tiles > 0 ? (force_tiles < tcap ? force_tiles : tcap) : 1;
+            groups = (p.tiles + tper - 1) / tper;
+            tper = (p.tiles + groups - 1) / groups;
             const long ctas = (long)groups * s;
-            const int tm = fp4_tmem_cols(p.nb, 1);
-            ring = chunk < 4 ? chunk : 4;
-            if (force_ring > 0) ring = force_ring < chunk ? force_ring : chunk;
+            const int tm = fp4_tmem_cols(p.nb, tper);
+            const int units = tper * chunk;
+            ring = units < 4 ? units : 4;
+            if (force_ring > 0) ring = force_ring < units ? force_ring : units;
             else
-                while (ring > 2 && ctas > (long)sms * fp4_ctas_per_sm(fp4_smem_bytes(p.nb, p.M, 1, chunk, ring), tm)) --ring;
-            while (ring > 1 && fp4_smem_bytes(p.nb, p.M, 1, chunk, ring) > kFp4SmemLimit) --ring;
-            const uint32_t bytes = fp4_smem_bytes(p.nb, p.M, 1, chunk, ring);
+                while (ring > 2 && ctas > (long)sms * fp4_ctas_per_sm(fp4_smem_bytes(p.nb, p.M, tper, chunk, ring), tm)) --ring;
+            while (ring > 1 && fp4_smem_bytes(p.nb, p.M, tper, chunk, ring) > kFp4SmemLimit) --ring;
+            const uint32_t bytes = fp4_smem_bytes(p.nb, p.M, tper, chunk, ring);
             if (bytes > kFp4SmemLimit) continue;
             const long slots = (long)sms * fp4_ctas_per_sm(bytes, tm);
             const long waves = (ctas + slots - 1) / slots;

@@ -1,4 +1,5 @@
-// mxq_linear on the 5th-generation tensor cores (tcgen05) with the MXFP4 weights as a NATIVE operand.
+// mxq_linear for 1..16 token rows on the 5th-generation tensor cores (tcgen05) with the MXFP4 weights as a NATIVE
+// operand and the activations rewritten exactly as FP8 numbers.
 //
 // The layer (Sec. III-D-3, Eq. 2) is  Y[m][n] = sum_blocks 2^(b-127) * sum_{k in block} X[m][k] * value(code[n][k]).
 // tcgen05.mma kind::mxf8f6f4.block_scale computes exactly that shape of sum in hardware: both operands carry
@@ -18,24 +19,14 @@
 //                                        meets one computes its share with scalar FP32 code instead.
 //   D (128 rows x NB columns, FP32)   <- tensor memory; tcgen05.ld in the epilogue.
 //
-// Work decomposition: one CTA per (128-row tile, K chunk); the `split` CTAs of a tile form a thread-block
-// cluster and add their partial results through distributed shared memory in rank order, so the result is
-// bit-reproducible and no global workspace or atomics are needed.  Inside a CTA: warp 0 issues the MMAs,
-// warp 1 the TMA copies, warps 2-3 the scale copies, over a ring of `ring` stages (128 k each) guarded by
-// full/empty mbarriers; all four warps run the X split before and the epilogue after.
-//
-// Programmatic dependent launch: weights are constants, so the first `ring` stages are requested before
-// griddepcontrol.wait; X is read and Y written only after it.
-//
-// Every mbarrier wait is bounded (about a second); a wait that gives up sets a sticky device word that
-// mxq_linear_device_status() returns, the tile is written as NaN, and the kernel still ends cleanly.
-#include <cuda.h>   // CUtensorMap and its enums only; the encoder is looked up at run time (no libcuda link)
-
+// Work decomposition, warp roles, pipeline, programmatic dependent launch and bounded waits are those of the
+// packed-FP4 kernel (mxq_linear_fp4.cu), which is the faster one at M = 1; this one splits a token into 3 rows of
+// the token operand instead of 16 and wins from M = 2 on.  A stage here is 128 k (16 KB of shared memory for 8 KB of
+// packed codes); the activations are split in groups of 256 k, so one "ready" barrier covers two stages.
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
-#include "mxq_device.cuh"
 #include "mxq_host.h"
 #include "mxq_linear_umma.h"
 #include "mxq_tcgen05.cuh"
@@ -43,11 +34,11 @@
 
 namespace mxq {
 
-__device__ unsigned int g_umma_status = 0;   // sticky: bit 0 full-wait, 1 empty-wait, 2 done-wait, 3 drain-wait gave up
-
 namespace {
 
-constexpr uint32_t kFullArrivals = 1 + 64;   // TMA thread's expect_tx arrive + one cp.async arrive per scale thread
+__device__ unsigned int g_umma_status = 0;   // sticky: bit 0 full-wait, 1 empty-wait, 2 done-wait, 3 drain-wait gave up
+
+constexpr uint32_t kFullArrivals = 1 + 32;   // the expect_tx arrive of the TMA lane + one cp.async arrive per producer lane
 
 // Every partial sum is bounded by sum |x w^|, which cancellation can leave up to 1/2e-3 = 500 times larger than a
 // result that still has to come out finite.  So the token operand's scales carry an extra 2^-kGuard, all sums are
@@ -71,7 +62,6 @@ __device__ __forceinline__ uint32_t pack_e5m2x2(float lo, float hi) {
     return out;
 }
 
-// ---- the kernel ----------------------------------------------------------------------------------------
 // One 8-element unit of X (token m, k offset kk inside the CTA's range): split into parts, store into B and SFB.
 // All 32 lanes call it together (the block maximum crosses the four lanes of a 32-block by shuffle).
 template <int NB>
@@ -117,323 +107,433 @@ __device__ __forceinline__ bool split_unit(const uint4 raw, bool act, int m, int
             uint8_t *dst = gB + (size_t)j * (NB * 128) + (row >> 3) * 1024 + ((kk >> 4) & 7) * 128 + (row & 7) * 16 + (kk & 15);
             *reinterpret_cast<uint2 *>(dst) = make_uint2(part[p][0], part[p][1]);
             if ((lane & 3) == 0)
-                gSFB[(size_t)j * kUmmaSfAtomBytes + (row & 31) * 16 + (row >> 5) * 4 + ((kk >> 5) & 3)] = (uint8_t)(sb1 - kGuard - 3 * p);
+                gSFB[(size_t)j * kUmmaSfStageBytes + (row & 31) * 16 + (row >> 5) * 4 + ((kk >> 5) & 3)] = (uint8_t)(sb1 - kGuard - 3 * p);
         }
     }
     return inexact && act;
 }
 
-// NB: columns of the B operand / accumulator (16, 32 or 48 >= 3 * M).
-template <int NB>
+// NB: columns of the B operand / accumulator = 3 parts x tokens, rounded up to 16, 32 or 48.
+// Warp roles (192 threads): warp 0 issues the MMAs and owns tensor memory; warp 1 is the producer (TMA copies of
+// the codes, cp.async of the scale bytes, barrier set-up); warps 2..5 split the activations stage by stage and,
+// at the end, read the accumulator (one row per thread), exchange partial results and store.
+// MULTI: whether a CTA may own more than one tile (false: exactly one, and the per-tile loops fold away).
+template <int NB, bool MULTI>
 __global__ void __launch_bounds__(kUmmaThreads)
 linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 *__restrict__ X, int M,
-                   const uint8_t *__restrict__ codes, const uint8_t *__restrict__ scales, int64_t N, int64_t K,
-                   void *__restrict__ Y, int y_dtype, int split, int ring, int ks, int chunk_max, int tmem_cols) {
+                  const uint8_t *__restrict__ codes, const uint8_t *__restrict__ scales, int64_t N, int64_t K,
+                  void *__restrict__ Y, int y_dtype, int split, int ring, int ks, int chunk_max, int tmem_cols, int groups,
+                  int tiles, int tiles_max) {
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");   // needed by the first copy, 1 us from now
     const uint32_t rank = split > 1 ? cluster_rank() : 0u;
-    const int tile = blockIdx.x / split;
-    const int64_t n0 = (int64_t)tile * kUmmaTileRows;
-    const int s_begin = (int)(((int64_t)rank * ks) / split), s_end = (int)(((int64_t)(rank + 1) * ks) / split);
+    const uint32_t group = blockIdx.x / (uint32_t)split;
+    // this CTA's tiles [tile_lo, tile_lo + ntile) and, for all of them, its K range
+    const int tile_lo = (int)((group * (uint32_t)tiles) / (uint32_t)groups);
+    const int ntile = MULTI ? (int)(((group + 1u) * (uint32_t)tiles) / (uint32_t)groups) - tile_lo : 1;
+    const int64_t n0 = (int64_t)tile_lo * kUmmaTileRows;   // first weight row of the first tile
+    // everything below fits in 32 bits (the plan refuses K >= 2^30 and more than 2^20 tiles)
+    const int s_begin = (int)((rank * (uint32_t)ks) / (uint32_t)split), s_end = (int)(((rank + 1u) * (uint32_t)ks) / (uint32_t)split);
     const int nst = s_end - s_begin;   // stages of this CTA (>= 1 because split <= ks)
-    const int kb_row = (int)(K / 32);
+    const int kb_row = (int)((uint32_t)K >> 5);
+    const int k_begin = s_begin * kUmmaStageK;
+    const int k_len = nst * kUmmaStageK;
 
     // carve shared memory (1024-byte aligned for the 128-byte swizzle)
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gbase = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t sA = base;
-    const uint32_t sSFA = sA + (uint32_t)ring * kUmmaStageSmemBytes;
-    const uint32_t sB = sSFA + (uint32_t)ring * kUmmaSfAtomBytes;
+    const uint32_t sSFA = sA + (uint32_t)ring * kUmmaStageBytes;
+    const uint32_t sB = sSFA + (uint32_t)ring * kUmmaSfStageBytes;
     const uint32_t sSFB = sB + (uint32_t)chunk_max * (NB * 128);
-    const uint32_t sRecv = sSFB + (uint32_t)chunk_max * kUmmaSfAtomBytes;   // [split][M][rows of this rank] floats
-    const uint32_t sBar = sRecv + (uint32_t)M * kUmmaRecvRows * 4u;    // full[ring], empty[ring], done, holder, fail
+    const uint32_t sRecv = sSFB + (uint32_t)chunk_max * kUmmaSfStageBytes;   // [tile][split][M][rows of this rank] floats
+    const uint32_t sBar = sRecv + (uint32_t)(tiles_max * M) * kUmmaRecvRows * 4u;
+    // barriers: full[ring], empty[ring], done, recv, ready[pairs of stages]; then the tensor-memory address and flags
+    const uint32_t full0 = sBar, empty0 = sBar + (uint32_t)ring * 8u, done_bar = sBar + (uint32_t)ring * 16u;
+    const uint32_t recv_bar = done_bar + 8u, ready0 = done_bar + 16u;
+    const int npair = (nst + 1) >> 1;   // the activations are split 256 k (two stages) at a time
+    const uint32_t sMisc = ready0 + (uint32_t)((chunk_max + 1) >> 1) * 8u;
     uint8_t *gB = gbase + (sB - base), *gSFB = gbase + (sSFB - base);
     const float *gRecv = reinterpret_cast<const float *>(gbase + (sRecv - base));
-    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(gbase + (sBar - base) + (2 * ring + 1) * 8);
-    volatile int &s_fail = *reinterpret_cast<volatile int *>(gbase + (sBar - base) + (2 * ring + 1) * 8 + 4);
-    const uint32_t full0 = sBar, empty0 = sBar + (uint32_t)ring * 8u, done_bar = sBar + (uint32_t)ring * 16u;
+    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(gbase + (sMisc - base));
+    volatile int &s_fail = *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 4);
+    const int row_lo = (int)(rank * kUmmaTileRows) / split, row_cnt = (int)((rank + 1) * kUmmaTileRows) / split - row_lo;
 
-    // ---- prologue: request the first stages of weights (they do not depend on the previous kernel) --------
-    const int pre = nst < ring ? nst : ring;
-    if (tid == 32) {   // the TMA thread sets up the barriers and starts the weight stream at once
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
-        s_fail = 0;
-        for (int i = 0; i < ring; ++i) {
-            mbar_init(full0 + i * 8, kFullArrivals);
-            mbar_init(empty0 + i * 8, 1);
+    // ---- prologue: barriers, tensor memory, and the first stages of weights (they do not depend on the previous
+    //      kernel, so all of this runs before griddepcontrol.wait) -----------------------------------------------
+    // The CTA's work is a sequence of units (tile, stage), tile-major; unit u goes through ring slot u % ring.
+    const int nunit = ntile * nst;
+    const int pre = nunit < ring ? nunit : ring;
+    // The SM's requests are served roughly in order, so activations asked for behind a ring full of weight copies
+    // arrive late, and everything after the split waits with them.  Only the first two units are requested up
+    // front; the rest of the ring follows once the activations are in, or else at a trickle.
+    const int pre0 = pre < 2 ? pre : 2;
+    volatile int &s_xin = *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 12);   // the activations have arrived
+    // producer lane l owns rows l, l + 32, l + 64, l + 96 of a tile's scale bytes
+    const uint8_t *srow0 = scales + (n0 + lane) * kb_row + s_begin * 4;
+    const int64_t srow_step = (int64_t)32 * kb_row;
+    const uint32_t sf_lane = sSFA + (uint32_t)lane * 16u;
+    auto copy_scales = [&](int t, int i, uint32_t slot) {   // unit (t, i) into ring slot `slot` (all lanes of the producer warp)
+        const uint32_t dst = sf_lane + slot * kUmmaSfStageBytes;
+        const uint8_t *src = srow0 + (int64_t)t * (4 * srow_step) + i * 4;
+        const int rows_here = (int)min((int64_t)kUmmaTileRows, N - n0 - (int64_t)t * kUmmaTileRows);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (lane + 32 * q < rows_here) cp_async4(dst + 4 * q, src);
+            src += srow_step;
         }
-        mbar_init(done_bar, 1);
+        cp_async_arrive(full0 + slot * 8);
+    };
+    auto copy_codes = [&](int t, int i, uint32_t slot) {    // one lane
+        mbar_expect_tx(full0 + slot * 8, kUmmaStageTxBytes);
+        tma_load_codes(sA + slot * kUmmaStageBytes, &tmap, (s_begin + i) * kUmmaStageK, (int)n0 + t * kUmmaTileRows, full0 + slot * 8);
+    };
+    if (warp == 1) {
+        for (int b = lane; b < 2 * ring + 2 + npair; b += 32) {
+            // full: the TMA lane + 32 producer lanes; empty, done, recv: 1; ready (one per 256 k): one arrival per token
+            const uint32_t count = b < ring ? kFullArrivals : (b < 2 * ring + 2 ? 1u : (uint32_t)M);
+            mbar_init(sBar + (uint32_t)b * 8u, count);
+        }
+        if (lane == 31) {
+            s_fail = 0;
+            *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 8) = 0;   // s_bad
+            s_xin = 0;
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        for (int i = 0; i < pre; ++i) {
-            mbar_expect_tx(full0 + i * 8, kUmmaStageTxBytes);
-            tma_load_codes(sA + (uint32_t)i * kUmmaStageSmemBytes, &tmap, (s_begin + i) * kUmmaStageK, (int)n0, full0 + i * 8);
-        }
-    }
-    __syncthreads();
-    pdl_trigger();
-    const int64_t row_a = n0 + (tid - 64), row_b = row_a + 64;   // rows of the scale threads (tid 64..127)
-    const uint8_t *srow_a = scales + row_a * kb_row + (int64_t)s_begin * 4;
-    const uint8_t *srow_b = scales + row_b * kb_row + (int64_t)s_begin * 4;
-    const bool has_a = row_a < N, has_b = row_b < N;
-    const uint32_t sf_a = sSFA + (uint32_t)(((tid - 64) & 31) * 16 + ((tid - 64) >> 5) * 4), sf_b = sf_a + 8;
-    if (warp >= 2) {
-        for (int i = 0; i < pre; ++i) {
-            if (has_a) cp_async4(sf_a + (uint32_t)i * kUmmaSfAtomBytes, srow_a + i * 4);
-            if (has_b) cp_async4(sf_b + (uint32_t)i * kUmmaSfAtomBytes, srow_b + i * 4);
-            cp_async_arrive(full0 + i * 8);
+        __syncwarp();
+        if (lane == 0) {
+            if (split > 1) mbar_expect_tx(recv_bar, (uint32_t)(ntile * split * M * row_cnt) * 4u);   // every rank sends M values per tile and row
+            for (int u = 0, t = 0, i = 0; u < pre0; ++u) {
+                copy_codes(t, i, (uint32_t)u);
+                if (++i == nst) {
+                    i = 0;
+                    ++t;
+                }
+            }
         }
     } else if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                         sBar + (uint32_t)(2 * ring + 1) * 8),
-                     "r"(tmem_cols)
-                     : "memory");
+        // let the next kernel start launching at once (its CTAs take the shared memory this kernel leaves free and start
+        // their own weight stream); the MMA warp does it because it has nothing urgent to do yet
+        pdl_trigger();
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sMisc), "r"(tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-
-    // ---- X of this CTA's K range -> three E5M2 parts + block scales (after the previous kernel finished) ---
-    pdl_wait();
-    bool inexact = false;
-    {
-        const int upr = nst * (kUmmaStageK / 8);        // 8-element units per token row
-        const int total = M * upr;
-        const __nv_bfloat16 *xbase = X + (int64_t)s_begin * kUmmaStageK;
-        for (int u0 = 0; u0 < total; u0 += 4 * kUmmaThreads) {
-            uint4 raw[4];
-            int mm[4], kk[4];
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {   // all loads of the batch first
-                const int u = u0 + b * kUmmaThreads + tid;
-                const bool act = u < total;
-                mm[b] = act ? u / upr : -1;
-                kk[b] = act ? (u - mm[b] * upr) * 8 : 0;
-                raw[b] = make_uint4(0, 0, 0, 0);
-                if (act) raw[b] = *reinterpret_cast<const uint4 *>(xbase + (int64_t)mm[b] * K + kk[b]);
-            }
-#pragma unroll
-            for (int b = 0; b < 4; ++b)
-                if (u0 + b * kUmmaThreads < total)   // uniform across the CTA
-                    inexact |= split_unit<NB>(raw[b], mm[b] >= 0, mm[b], kk[b], lane, gB, gSFB);
-        }
+    // Only the activation warps read what the previous kernel wrote (X) and write what the next one reads (Y), so
+    // only they wait for it; they do so at once, and join the CTA-wide barrier (initialised mbarriers, tensor-memory
+    // address) after that wait.
+    if (warp >= 2) {
+        pdl_wait();
     }
-    fence_async_proxy();   // B and its scales were written with ordinary stores; the tensor core reads them
+    if (split > 1) cluster_arrive();   // "my barriers exist"; the matching wait is just before the first push to a peer
     tc_fence_before();
-    const int bad = __syncthreads_or(inexact ? 1 : 0);
+    asm volatile("bar.sync 0;" ::: "memory");
     tc_fence_after();
     const uint32_t tmem = *tmem_holder;
-
-    float y[16];
-#pragma unroll
-    for (int m = 0; m < 16; ++m) y[m] = 0.f;
-
-    if (!bad) {
-        if (warp == 0) {
-            // ---- MMA warp: the loop is warp-uniform, one elected lane issues ----------------------------------
-            // descriptors as 32-bit halves: only the start-address field changes from MMA to MMA
-            const uint32_t idesc = (5u << 7) | (1u << 10) | (((uint32_t)NB >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
-            const uint32_t a_hi = (uint32_t)(smem_desc(0, 16, 1024, 2) >> 32), b_hi = (uint32_t)(smem_desc(0, 128, 1024, 0) >> 32);
-            const uint32_t s_hi = (uint32_t)(smem_desc(0, 0, 128, 0) >> 32);
-            const uint32_t a_lo0 = (uint32_t)smem_desc(sA, 16, 1024, 2), s_lo0 = (uint32_t)smem_desc(sSFA, 0, 128, 0);
-            uint32_t b_lo = (uint32_t)smem_desc(sB, 128, 1024, 0), sb_lo = (uint32_t)smem_desc(sSFB, 0, 128, 0);
-            const uint32_t t_sfa0 = tmem + NB, t_sfb0 = t_sfa0 + 4u * (uint32_t)ring;
-            uint32_t slot = 0, phase = 0, accumulate = 0;
-            for (int i = 0; i < nst; ++i) {
-                if (!mbar_wait(full0 + slot * 8, phase)) {
-                    if (lane == 0) {
-                        atomicOr(&g_umma_status, 1u);
-                        s_fail = 1;
-                    }
-                    break;
-                }
-                tc_fence_after();
-                const uint32_t t_sfa = t_sfa0 + 4u * slot, t_sfb = t_sfb0 + 4u * slot;
-                const uint32_t a_lo = a_lo0 + slot * (kUmmaStageSmemBytes >> 4);
-                if (elect_one()) {
-                    fence_async_proxy();   // the scale atom was written by cp.async
-                    asm volatile(
-                        "{\n\t.reg .b64 d;\n\tmov.b64 d, {%1, %2};\n\ttcgen05.cp.cta_group::1.32x128b.warpx4 [%0], d;\n\t}"
-                        ::"r"(t_sfa), "r"(s_lo0 + slot * (kUmmaSfAtomBytes >> 4)), "r"(s_hi) : "memory");
-                    asm volatile(
-                        "{\n\t.reg .b64 d;\n\tmov.b64 d, {%1, %2};\n\ttcgen05.cp.cta_group::1.32x128b.warpx4 [%0], d;\n\t}"
-                        ::"r"(t_sfb), "r"(sb_lo), "r"(s_hi) : "memory");
-#pragma unroll
-                    for (int kb = 0; kb < 4; ++kb)
-                        asm volatile(
-                            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
-                            "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
-                            "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], da, db, %5, [%7], [%8], p;\n\t}"
-                            ::"r"(tmem), "r"(a_lo + kb * 2), "r"(a_hi), "r"(b_lo + kb * 16), "r"(b_hi),
-                            "r"(idesc | ((uint32_t)kb << 4) | ((uint32_t)kb << 29)), "r"(kb == 0 ? accumulate : 1u), "r"(t_sfa),
-                            "r"(t_sfb)
-                            : "memory");
-                    tc_commit(empty0 + slot * 8);
-                }
-                __syncwarp();
-                accumulate = 1;
-                b_lo += (NB * 128) >> 4;
-                sb_lo += kUmmaSfAtomBytes >> 4;
-                if (++slot == (uint32_t)ring) {
-                    slot = 0;
-                    phase ^= 1u;
-                }
+    if (warp == 1) {
+        for (int u = 0, t = 0, i = 0; u < pre; ++u) {
+            if (u >= pre0) {
+                for (int spin = 0; spin < 3 && !s_xin; ++spin) __nanosleep(100);
+                if (lane == 0) copy_codes(t, i, (uint32_t)u);
             }
-            if (elect_one()) tc_commit(done_bar);
-            __syncwarp();
-        } else if (warp == 1) {
-            // ---- TMA warp ------------------------------------------------------------------------------------
-            uint32_t slot = 0, phase = 0;   // stage `pre` reuses slot 0 (pre == ring whenever the loop runs)
-            for (int i = pre; i < nst; ++i) {
-                if (!mbar_wait(empty0 + slot * 8, phase)) {
-                    if (lane == 0) {
-                        atomicOr(&g_umma_status, 2u);
-                        s_fail = 1;
-                    }
-                    break;
-                }
-                if (elect_one()) {
-                    mbar_expect_tx(full0 + slot * 8, kUmmaStageTxBytes);
-                    tma_load_codes(sA + slot * kUmmaStageSmemBytes, &tmap, (s_begin + i) * kUmmaStageK, (int)n0, full0 + slot * 8);
-                }
-                __syncwarp();
-                if (++slot == (uint32_t)ring) {
-                    slot = 0;
-                    phase ^= 1u;
-                }
-            }
-        } else {
-            uint32_t slot = 0, phase = 0;
-            for (int i = pre; i < nst; ++i) {
-                if (!mbar_wait(empty0 + slot * 8, phase)) {
-                    atomicOr(&g_umma_status, 2u);
-                    s_fail = 1;
-                    break;
-                }
-                if (has_a) cp_async4(sf_a + slot * kUmmaSfAtomBytes, srow_a + i * 4);
-                if (has_b) cp_async4(sf_b + slot * kUmmaSfAtomBytes, srow_b + i * 4);
-                cp_async_arrive(full0 + slot * 8);
-                if (++slot == (uint32_t)ring) {
-                    slot = 0;
-                    phase ^= 1u;
-                }
+            copy_scales(t, i, (uint32_t)u);
+            if (++i == nst) {
+                i = 0;
+                ++t;
             }
         }
-        // ---- epilogue: accumulator row -> registers; the three parts of a token are three columns ----------
-        if (!mbar_wait(done_bar, 0)) {
+    }
+    constexpr int kResults = MULTI ? 16 : NB / kUmmaParts;
+    float y[kResults];   // results of this thread's row: [tile][token slot]
+#pragma unroll
+    for (int q = 0; q < kResults; ++q) y[q] = 0.f;
+
+    if (warp == 0) {
+        // ---- MMA warp: the loop is warp-uniform, one elected lane issues -------------------------------------------
+        // descriptors as 32-bit halves: only the start-address field changes from MMA to MMA
+        // A = E2M1 (5), B = E5M2 (1), N = NB, E8M0 scales, M = 128
+        const uint32_t idesc = (5u << 7) | (1u << 10) | (((uint32_t)NB >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+        const uint32_t a_hi = (uint32_t)(smem_desc(0, 16, 1024, 2) >> 32), b_hi = (uint32_t)(smem_desc(0, 128, 1024, 0) >> 32);
+        const uint32_t s_hi = (uint32_t)(smem_desc(0, 0, 128, 0) >> 32);
+        const uint32_t a_lo0 = (uint32_t)smem_desc(sA, 16, 1024, 2), s_lo0 = (uint32_t)smem_desc(sSFA, 0, 128, 0);
+        const uint32_t b_lo0 = (uint32_t)smem_desc(sB, 128, 1024, 0), sb_lo0 = (uint32_t)smem_desc(sSFB, 0, 128, 0);
+        const uint32_t t_sf0 = tmem + (uint32_t)(NB * tiles_max);   // after the accumulators: two slots of 4 + 4 scale columns
+        uint32_t slot = 0, phase = 0, par = 0;
+        bool ok = true;
+        for (int t = 0; t < ntile && ok; ++t) {
+          const uint32_t t_acc = tmem + (uint32_t)(t * NB);   // this tile's accumulator columns
+          uint32_t b_lo = b_lo0, sb_lo = sb_lo0, accumulate = 0;
+          for (int i = 0; i < nst; ++i) {
+            // the unit's weights and scales have landed and (first tile only; the others find it done) the stage's
+            // share of the activations has been split
+            if ((t == 0 && !mbar_wait_relaxed(ready0 + (uint32_t)(i >> 1) * 8u, 0)) || !mbar_wait_relaxed(full0 + slot * 8, phase)) {
+                if (lane == 0) {
+                    atomicOr(&g_umma_status, 1u);
+                    s_fail = 1;
+                }
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            const uint32_t a_lo = a_lo0 + slot * (kUmmaStageBytes >> 4);
+            const uint32_t sa_lo = s_lo0 + slot * (kUmmaSfStageBytes >> 4);
+            const uint32_t t_sf = t_sf0 + par * 8u;   // alternating between consecutive units
+            par ^= 1u;
+            if (elect_one()) {
+                fence_async_proxy();   // the weight scale atom was written by cp.async
+                tc_copy_sf_lohi(t_sf, sa_lo, s_hi);
+                tc_copy_sf_lohi(t_sf + 4, sb_lo, s_hi);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)   // k [32 j, 32 j + 32) of the stage: scale j of the atom on both sides
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+                        "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+                        "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], da, db, %5, [%7], [%8], p;\n\t}"
+                        ::"r"(t_acc), "r"(a_lo + j * 2), "r"(a_hi), "r"(b_lo + j * 16), "r"(b_hi),
+                        "r"(idesc | ((uint32_t)j << 4) | ((uint32_t)j << 29)), "r"(j == 0 ? accumulate : 1u), "r"(t_sf), "r"(t_sf + 4u)
+                        : "memory");
+                tc_commit(empty0 + slot * 8);
+            }
+            accumulate = 1;
+            b_lo += (NB * 128) >> 4;
+            sb_lo += kUmmaSfStageBytes >> 4;
+            if (++slot == (uint32_t)ring) {
+                slot = 0;
+                phase ^= 1u;
+            }
+          }
+        }
+        __syncwarp();
+        if (elect_one()) tc_commit(done_bar);
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---- producer warp: refill ring slots as the MMAs release them ----------------------------------------------
+        uint32_t slot = 0, phase = 0;   // unit `pre` reuses slot 0 (pre == ring whenever the loop runs)
+        int t = pre / nst, i = pre - t * nst;
+        for (int u = pre; u < nunit; ++u) {
+            if (!mbar_wait_relaxed(empty0 + slot * 8, phase)) {
+                if (lane == 0) {
+                    atomicOr(&g_umma_status, 2u);
+                    s_fail = 1;
+                }
+                break;
+            }
+            if (lane == 0) copy_codes(t, i, slot);
+            copy_scales(t, i, slot);
+            if (++i == nst) {
+                i = 0;
+                ++t;
+            }
+            if (++slot == (uint32_t)ring) {
+                slot = 0;
+                phase ^= 1u;
+            }
+        }
+    } else {
+        // ---- the four activation / epilogue warps ---------------------------------------------------------------------
+        const int ct = tid - 64;                                   // 0..127
+        const int row = ((warp & 3) << 5) + lane;                  // accumulator row this thread may read (its warp's quarter)
+        volatile int &s_bad = *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 8);
+        bool inexact = false;
+        {
+            // Groups of 32 units (256 k of one token, one warp; a unit is 8 elements, one lane) in order of K, so that
+            // the MMA warp can start on the first stages while later ones are being split.  Group G: pair of stages
+            // G / M, token G % M; the last pair is half full when the CTA has an odd number of stages.  All of this
+            // is uniform across a warp.
+            const int ngroups = npair * M;
+            const __nv_bfloat16 *xbase = X + k_begin;
+            const int cw = ct >> 5;
+            constexpr int kBatch = 4;   // loads in flight per thread
+            for (int G0 = 0; G0 < ngroups; G0 += 4 * kBatch) {
+                uint4 raw[kBatch];
+                int mm[kBatch], kk[kBatch], pair[kBatch];
+                bool act[kBatch];
+#pragma unroll
+                for (int b = 0; b < kBatch; ++b) {   // all loads of the batch first
+                    const int G = G0 + 4 * b + cw;
+                    mm[b] = kk[b] = pair[b] = 0;
+                    act[b] = false;
+                    raw[b] = make_uint4(0, 0, 0, 0);
+                    if (G < ngroups) {
+                        pair[b] = G / M;
+                        mm[b] = G - pair[b] * M;
+                        kk[b] = pair[b] * (2 * kUmmaStageK) + lane * 8;
+                        act[b] = kk[b] < k_len;
+                        if (act[b]) raw[b] = *reinterpret_cast<const uint4 *>(xbase + (int64_t)mm[b] * K + kk[b]);
+                    }
+                }
+#pragma unroll
+                for (int b = 0; b < kBatch; ++b)
+                    if (G0 + 4 * b + cw < ngroups) {   // uniform across the warp
+                        inexact |= split_unit<NB>(raw[b], act[b], mm[b], kk[b], lane, gB, gSFB);
+                        if (G0 == 0 && b == 0 && ct == 0) s_xin = 1;   // lets the producer request the rest of the ring
+                        fence_async_proxy();   // ordinary stores, read by the tensor core
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(ready0 + (uint32_t)pair[b] * 8u);
+                    }
+            }
+        }
+        if (inexact) s_bad = 1;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const int bad = s_bad;
+
+        // ---- epilogue: accumulator row -> registers; the three parts of a token are three neighbouring columns -------
+        constexpr int MT = NB / kUmmaParts;         // token slots per tile (5, 10 or 16)
+        constexpr int TCAP = MULTI ? 16 / MT : 1;   // tiles a thread can keep results for
+        if (!mbar_wait_relaxed(done_bar, 0)) {
             atomicOr(&g_umma_status, 4u);
             s_fail = 1;
         }
         tc_fence_after();
-        const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
+        if (!bad) {
+            const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 #pragma unroll
-        for (int c = 0; c < NB / 16; ++c) {
-            float d[16];
-            tc_load16(t_row + c * 16, d);
+            for (int t = 0; t < TCAP; ++t)
+                if (t < ntile) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const int col = c * 16 + j;
-                if (col < 48) y[col / 3] += d[j];   // fixed order: parts 0, 1, 2 of token col / 3
-            }
-        }
-    } else {
-        // ---- scalar path for a K range whose X cannot be split exactly ------------------------------------
-        // first let the copies requested in the prologue land (nothing may be in flight when the CTA ends)
-        for (int i = 0; i < pre; ++i)
-            if (!mbar_wait(full0 + i * 8, 0)) {
-                atomicOr(&g_umma_status, 8u);
-                s_fail = 1;
-                break;
-            }
-        const int64_t n = n0 + tid;
-        if (n < N) {
-            const uint4 *crow = reinterpret_cast<const uint4 *>(codes + n * (K / 2));
-            const uint8_t *srow = scales + n * kb_row;
-            for (int blk = s_begin * 4; blk < s_end * 4; ++blk) {
-                const uint4 c = ld_stream_u4(crow + blk);
-                const float sc = e8m0_to_float(srow[blk]) * kGuardDown;
-                const uint32_t w[4] = {c.x, c.y, c.z, c.w};
-                float part[16];
+                    for (int c = 0; c < NB / 16; ++c) {
+                        float d[16];
+                        tc_load16(t_row + t * NB + c * 16, d);
 #pragma unroll
-                for (int m = 0; m < 16; ++m) part[m] = 0.f;
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float2 wv = __half22float2(e2m1x2_to_half2((w[q] >> (8 * i)) & 0xFFu));
-                        const int64_t k = (int64_t)blk * 32 + q * 8 + i * 2;
-#pragma unroll
-                        for (int m = 0; m < 16; ++m)
-                            if (m < M) {
-                                const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * K + k);
-                                part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
-                                part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
-                            }
+                        for (int j = 0; j < 16; ++j) {
+                            const int col = c * 16 + j;
+                            if (col < MT * kUmmaParts) y[t * MT + col / kUmmaParts] += d[j];   // fixed order: parts 0, 1, 2
+                        }
                     }
+                }
+        } else {
+            // Scalar path for a K range whose X cannot be split into E5M2 parts exactly (the MMA results are ignored).
+            // Results pass through the ring's shared memory, which is idle once every MMA has completed.
+            float *scratch = reinterpret_cast<float *>(gbase);
+            for (int t = 0; t < ntile; ++t) {
+                const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row;
+                float acc[kUmmaMaxM];
 #pragma unroll
-                for (int m = 0; m < 16; ++m) y[m] = fmaf(part[m], sc, y[m]);
+                for (int m = 0; m < kUmmaMaxM; ++m) acc[m] = 0.f;
+                if (n < N) {
+                    const uint4 *crow = reinterpret_cast<const uint4 *>(codes + n * (K / 2));
+                    const uint8_t *srw = scales + n * kb_row;
+                    for (int blk = k_begin / 32; blk < (k_begin + k_len) / 32; ++blk) {
+                        const uint4 c = ld_stream_u4(crow + blk);
+                        const float sc = e8m0_to_float(srw[blk]) * kGuardDown;
+                        const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+                        float part[kUmmaMaxM];
+#pragma unroll
+                        for (int m = 0; m < kUmmaMaxM; ++m) part[m] = 0.f;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float2 wv = __half22float2(e2m1x2_to_half2((w[q] >> (8 * i)) & 0xFFu));
+                                const int64_t k = (int64_t)blk * 32 + q * 8 + i * 2;
+#pragma unroll
+                                for (int m = 0; m < kUmmaMaxM; ++m)
+                                    if (m < M) {
+                                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * K + k);
+                                        part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
+                                        part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
+                                    }
+                            }
+#pragma unroll
+                        for (int m = 0; m < kUmmaMaxM; ++m) acc[m] = fmaf(part[m], sc, acc[m]);
+                    }
+                }
+#pragma unroll
+                for (int m = 0; m < MT; ++m) scratch[(t * MT + m) * kUmmaTileRows + row] = acc[m];
+            }
+#pragma unroll
+            for (int q = 0; q < kResults; ++q)
+                if (q < ntile * MT) y[q] = scratch[q * kUmmaTileRows + row];   // the thread's own values, back in registers
+        }
+        if (s_fail) {
+#pragma unroll
+            for (int q = 0; q < kResults; ++q) y[q] = __uint_as_float(0x7FC00000u);
+        }
+
+        // ---- result: direct store, or a sum over the cluster in a fixed order ----------------------------------------
+        if (split == 1) {
+#pragma unroll
+            for (int t = 0; t < TCAP; ++t)
+                if (t < ntile) {
+                    const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row;
+                    if (n < N)
+#pragma unroll
+                        for (int m = 0; m < MT; ++m)
+                            if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, y[t * MT + m] * kGuardUp);
+                }
+        } else {
+            // Rank q owns rows [q*128/split, (q+1)*128/split) of every tile of the group: every CTA pushes its partial
+            // results for those rows into q's shared memory (slot = tile, sender's rank) with stores that count on q's
+            // mbarrier; q waits for all of them and adds them in a fixed order.  No CTA reads a peer's memory, and a
+            // CTA leaves only after everything addressed to it has arrived.
+            const int cnt_max = (kUmmaTileRows + split - 1) / split;
+            const uint32_t owner = (uint32_t)(((row + 1) * split - 1) / kUmmaTileRows);
+            const int rr = row - (int)(owner * kUmmaTileRows) / split;
+            const uint32_t remote = peer_saddr(sRecv, owner), remote_bar = peer_saddr(recv_bar, owner);
+            cluster_wait();   // every CTA of the cluster has initialised its barriers (they arrived long ago)
+#pragma unroll
+            for (int t = 0; t < TCAP; ++t)
+                if (t < ntile) {
+#pragma unroll
+                    for (int m = 0; m < MT; ++m)
+                        if (m < M)
+                            st_async_f32(remote + (uint32_t)(((t * split + (int)rank) * M + m) * cnt_max + rr) * 4u, y[t * MT + m], remote_bar);
+                }
+            if (!mbar_wait_relaxed(recv_bar, 0)) {
+                atomicOr(&g_umma_status, 16u);
+                s_fail = 1;
+            }
+            const float poison = s_fail ? __uint_as_float(0x7FC00000u) : 0.f;
+            if ((split & (split - 1)) == 0) {
+                // power-of-two cluster: one value per thread (row ct / split, sender ct % split), butterfly sum over the
+                // senders in neighbouring lanes; the order of additions is fixed by the lane pattern
+                const int r = ct / split, j = ct & (split - 1);
+                for (int t = 0; t < ntile; ++t) {
+                    const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row_lo + r;
+                    for (int m = 0; m < M; ++m) {
+                        float v = gRecv[((t * split + j) * M + m) * cnt_max + r];
+                        for (int o = 1; o < split; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                        if (j == 0 && n < N) store_out(Y, y_dtype, (int64_t)m * N + n, v * kGuardUp + poison);
+                    }
+                }
+            } else {
+                for (int idx = ct; idx < ntile * M * row_cnt; idx += 128) {
+                    const int t = idx / (M * row_cnt), rem = idx - t * (M * row_cnt);
+                    const int m = rem / row_cnt, r = rem - m * row_cnt;
+                    float acc = 0.f;
+                    for (int j = 0; j < split; ++j) acc += gRecv[((t * split + j) * M + m) * cnt_max + r];
+                    const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row_lo + r;
+                    if (n < N) store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison);
+                }
             }
         }
     }
 
-    // ---- result: direct store, or rank-ordered sum across the cluster --------------------------------------
-    __syncthreads();   // s_fail is final
-    if (s_fail) {
-#pragma unroll
-        for (int m = 0; m < 16; ++m) y[m] = __uint_as_float(0x7FC00000u);
-    }
-    if (split == 1) {
-        const int64_t n = n0 + tid;
-        if (n < N)
-#pragma unroll
-            for (int m = 0; m < 16; ++m)
-                if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, y[m] * kGuardUp);
-    } else {
-        // rank q owns rows [q*128/split, (q+1)*128/split) of the tile: every CTA pushes its partial results
-        // for those rows into q's shared memory (slot = sender's rank), one cluster barrier, q adds in rank order
-        const int cnt_max = (kUmmaTileRows + split - 1) / split;
-        const uint32_t owner = (uint32_t)(((tid + 1) * split - 1) / kUmmaTileRows);
-        const int rr = tid - (int)(owner * kUmmaTileRows) / split;
-        uint32_t remote;
-        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(sRecv), "r"(owner));
-#pragma unroll
-        for (int m = 0; m < 16; ++m)
-            if (m < M)
-                asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote + (uint32_t)(((int)rank * M + m) * cnt_max + rr) * 4u),
-                             "f"(y[m])
-                             : "memory");
-        cluster_sync_all();
-        const int rb = (int)(rank * kUmmaTileRows) / split, cnt = (int)((rank + 1) * kUmmaTileRows) / split - rb;
-        for (int idx = tid; idx < M * cnt; idx += kUmmaThreads) {
-            const int m = idx / cnt, r = idx - m * cnt;
-            float acc = 0.f;
-            for (int j = 0; j < split; ++j) acc += gRecv[(j * M + m) * cnt_max + r];
-            const int64_t n = n0 + rb + r;
-            if (n < N) store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp);
-        }
-    }
+    if (split > 1 && warp < 2) cluster_wait();   // pairs with the arrive in the prologue (the other warps waited before their push)
     tc_fence_before();
     __syncthreads();
     if (warp == 0)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
 }
 
-// ---- host side -----------------------------------------------------------------------------------------
 int env_int(const char *name) {
     const char *e = std::getenv(name);
     return e ? std::atoi(e) : 0;
 }
 
-template <int NB>
+template <int NB, bool MULTI>
 cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X, const uint8_t *codes,
-                        const uint8_t *scales, void *Y, int y_dtype, cudaStream_t stream) {
+                       const uint8_t *scales, void *Y, int y_dtype, cudaStream_t stream) {
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(linear_umma_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kUmmaSmemLimit);
         if (e != cudaSuccess) return e;
         // all of the SM's L1/shared array as shared memory: how many CTAs (of this and of the next kernel) fit on an
         // SM is what decides how early the next kernel's weight stream can start
-        e = cudaFuncSetAttribute(linear_umma_kernel<NB>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -458,16 +558,15 @@ cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    return cudaLaunchKernelEx(&cfg, linear_umma_kernel<NB>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
-                              Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols);
+    return cudaLaunchKernelEx(&cfg, linear_umma_kernel<NB, MULTI>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
+                              Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols, p.groups, p.tiles, p.tiles_max);
 }
 
 }  // namespace
 
 bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p) {
-    if (M < 1 || M > 16 || N < 1 || K < kUmmaStageK || (K % kUmmaStageK) != 0) return false;
-    if (K / kUmmaStageK > 32767 || (N + kUmmaTileRows - 1) / kUmmaTileRows > (1 << 20)) return false;
-    if (N > 0x7FFFFFFF || K > 0x7FFFFFFF) return false;
+    if (M < 1 || M > kUmmaMaxM || N < 1 || K < 128 || (K % 128) != 0) return false;
+    if (K > 0x3FFFFFFF || N > 0x7FFFFFFF) return false;
     p.M = M;
     p.N = N;
     p.K = K;
@@ -478,17 +577,28 @@ bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p) {
 }
 
 cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,
-                               int y_dtype, cudaStream_t stream) {
+                              int y_dtype, cudaStream_t stream) {
     CUtensorMap map;
     if (!codes_tensor_map(codes, p.N, p.K, /*expand_fp4=*/true, &map)) return cudaErrorNotSupported;
     switch (p.nb) {
-        case 16: return launch_umma<16>(p, map, X, codes, scales, Y, y_dtype, stream);
-        case 32: return launch_umma<32>(p, map, X, codes, scales, Y, y_dtype, stream);
-        default: return launch_umma<48>(p, map, X, codes, scales, Y, y_dtype, stream);
+        case 16:   // the only width with room in a thread's registers for more than one tile
+            return p.tiles_max > 1 ? launch_umma<16, true>(p, map, X, codes, scales, Y, y_dtype, stream)
+                                   : launch_umma<16, false>(p, map, X, codes, scales, Y, y_dtype, stream);
+        case 32: return launch_umma<32, false>(p, map, X, codes, scales, Y, y_dtype, stream);
+        default: return launch_umma<48, false>(p, map, X, codes, scales, Y, y_dtype, stream);
     }
 }
 
 bool linear_umma_available() { return tensor_map_available(); }
+
+// returns and clears this kernel's sticky status word (see mxq_linear_device_status)
+static int linear_umma_take_status(uint32_t *out) {
+    unsigned int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_umma_status, sizeof v) != cudaSuccess) return MXQ_ERR_CUDA;
+    if (v != 0 && cudaMemcpyToSymbol(g_umma_status, &zero, sizeof zero) != cudaSuccess) return MXQ_ERR_CUDA;
+    *out = v;
+    return MXQ_OK;
+}
 
 }  // namespace mxq
 
@@ -496,11 +606,10 @@ extern "C" {
 #pragma GCC visibility push(default)
 int mxq_linear_device_status(uint32_t *status_host) {
     if (!status_host) return MXQ_ERR_NULL;
-    unsigned int v = 0, zero = 0;
-    if (cudaMemcpyFromSymbol(&v, mxq::g_umma_status, sizeof v) != cudaSuccess) return MXQ_ERR_CUDA;
-    if (v != 0 && cudaMemcpyToSymbol(mxq::g_umma_status, &zero, sizeof zero) != cudaSuccess) return MXQ_ERR_CUDA;
-    uint32_t v4 = 0;
-    const int rc = mxq::linear_fp4_take_status(&v4);
+    uint32_t v = 0, v4 = 0;
+    int rc = mxq::linear_umma_take_status(&v);
+    if (rc != MXQ_OK) return rc;
+    rc = mxq::linear_fp4_take_status(&v4);
     if (rc != MXQ_OK) return rc;
     *status_host = v | (v4 << 8);
     return MXQ_OK;

@@ -1,83 +1,122 @@
-// Work decomposition and shared-memory layout of the tcgen05 mxq_linear kernel (mxq_linear_umma.cu).
+// Work decomposition and shared-memory layout of the FP8-operand tcgen05 mxq_linear kernel (mxq_linear_umma.cu).
 // Plain integers only, so the host (sizing, launch) and the tests' mirror of it agree with the device code.
 #pragma once
 #include <stdint.h>
 
 namespace mxq {
 
-constexpr int kUmmaTileRows = 128;   // weight rows per CTA = M of one tcgen05.mma
+constexpr int kUmmaTileRows = 128;   // weight rows per tile = M of one tcgen05.mma
 constexpr int kUmmaStageK = 128;     // k per ring stage = 4 MX blocks = 4 MMAs of K = 32
-constexpr int kUmmaThreads = 128;
-constexpr uint32_t kUmmaStageSmemBytes = 16384;   // 128 rows x 128 codes, each 8 code bytes in a 16-byte slot
+constexpr int kUmmaThreads = 192;    // MMA warp, producer warp, four activation / epilogue warps
+constexpr int kUmmaParts = 3;        // E5M2 parts (columns of the token operand) per token
+constexpr int kUmmaMaxM = 16;
+constexpr uint32_t kUmmaStageBytes = 16384;       // shared memory per stage: 128 rows x 128 codes, 8 code bytes per 16-byte slot
 constexpr uint32_t kUmmaStageTxBytes = 8192;      // what the copy engine counts for one stage: the packed bytes
-constexpr uint32_t kUmmaSfAtomBytes = 512;        // scale bytes of 128 rows x 4 blocks in tensor-core order
-constexpr int kUmmaMaxRing = 8;
+constexpr uint32_t kUmmaSfStageBytes = 512;       // one scale atom: 128 rows x 4 blocks in tensor-core order
 constexpr int kUmmaMaxSplit = 8;                  // portable cluster size
 constexpr uint32_t kUmmaRecvRows = 136;           // >= split * ceil(128 / split) for every split <= 8
 constexpr uint32_t kUmmaSmemLimit = 227 * 1024;
-constexpr uint32_t kUmmaSmemHalf = 113 * 1024;    // two CTAs per SM
-constexpr uint32_t kUmmaSmemThird = 75 * 1024;    // three CTAs per SM
+constexpr int kUmmaMaxUnitsResident = 12;         // most ring slots (16 KB of expanded codes + 512 B of scales each)
 
 struct UmmaPlan {
-    int M;           // token rows
-    int nb;          // columns of the B operand: 16, 32 or 48 (three per token)
+    int M;           // token rows (1..16)
+    int nb;          // columns of the token operand per tile: 16, 32 or 48 (three per token)
     int ks;          // K / 128, stages per tile
     int tiles;       // ceil(N / 128)
-    int split;       // CTAs (cluster size) sharing one tile; CTA r takes stages [r*ks/split, (r+1)*ks/split)
-    int ring;        // stages in flight per CTA
+    int split;       // CTAs (cluster size) sharing a group of tiles; CTA r takes stages [r*ks/split, (r+1)*ks/split)
+    int groups;      // tile groups; group g owns tiles [g*tiles/groups, (g+1)*tiles/groups)
+    int tiles_max;   // most tiles in a group = ceil(tiles / groups)
+    int ring;        // (tile, stage) units in flight per CTA
     int chunk_max;   // most stages any CTA owns = ceil(ks / split)
-    int grid;        // tiles * split
+    int grid;        // groups * split
     int tmem_cols;   // tensor-memory columns allocated per CTA
     uint32_t smem_bytes;
     int64_t N, K;
 };
 
-inline uint32_t umma_smem_bytes(int nb, int chunk, int ring) {
-    const uint32_t recv = (uint32_t)(nb / 3) * kUmmaRecvRows * 4u;   // partial results pushed by the cluster's CTAs
-    const uint32_t b = 1024u /* alignment slack */ + (uint32_t)ring * (kUmmaStageSmemBytes + kUmmaSfAtomBytes) +
-                       (uint32_t)chunk * ((uint32_t)nb * 128u + kUmmaSfAtomBytes) + recv + (uint32_t)(2 * ring + 2) * 8u;
+inline uint32_t umma_smem_bytes(int nb, int M, int tiles_max, int chunk, int ring) {
+    const uint32_t recv = (uint32_t)(tiles_max * M) * kUmmaRecvRows * 4u;   // partial results pushed by the cluster's CTAs
+    const uint32_t b = 1024u /* alignment slack */ + (uint32_t)ring * (kUmmaStageBytes + kUmmaSfStageBytes) +
+                       (uint32_t)chunk * ((uint32_t)nb * 128u + kUmmaSfStageBytes) + recv +
+                       (uint32_t)(2 * ring + 2 + (chunk + 1) / 2) * 8u /* mbarriers */ + 16u /* tensor-memory address, flags */;
     return (b + 15u) & ~15u;
 }
 
-// Chooses split and ring for p.{M, nb, ks, tiles}; false if no choice fits in shared memory.
+inline int umma_tmem_cols(int nb, int tiles_max) {
+    const int need = nb * tiles_max + 16;   // one accumulator per tile + two slots of (4 + 4) scale columns
+    int cols = 32;
+    while (cols < need) cols *= 2;
+    return cols;
+}
+
+// CTAs of this kernel that fit on one SM (shared memory incl. 1 KB of system use each; 512 tensor-memory columns)
+inline int umma_ctas_per_sm(uint32_t smem_bytes, int tmem_cols) {
+    const int by_smem = (int)((228u * 1024u) / (smem_bytes + 1024u)), by_tmem = 512 / tmem_cols;
+    return by_smem < by_tmem ? by_smem : by_tmem;
+}
+
+// Chooses split, groups and ring for p.{M, nb, ks, tiles}; false if nothing fits.  Same two regimes as the packed-FP4
+// kernel: up to 2 * SMs tiles -> one tile per CTA, every CTA resident at once, about two CTAs per SM (ties to the
+// larger split: splitting the activations is this kernel's main cost from M = 4 on, and it shrinks with the K range);
+// more tiles -> one CTA per SM walking several tiles.
 // force_split / force_ring (> 0) override the heuristic where they are feasible.
 inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring) {
-    int best_split = 0, best_ring = 0;
+    const int slots_per_tile = p.nb / kUmmaParts;        // 5, 10 or 16 tokens fit in a tile's columns
+    const int tcap_regs = 16 / slots_per_tile;           // results a thread keeps in registers: tiles * slots <= 16
+    const int tcap = tcap_regs < 1 ? 1 : tcap_regs;
+    const bool layer_regime = p.tiles <= 2 * sms || tcap == 1;
     long best_cost = -1;
+    int best_split = 0, best_groups = 0, best_ring = 0;
     const int smax = p.ks < kUmmaMaxSplit ? p.ks : kUmmaMaxSplit;
     for (int s = 1; s <= smax; ++s) {
         if (force_split > 0 && s != (force_split < smax ? force_split : smax)) continue;
         const int chunk = (p.ks + s - 1) / s;
-        int ring = chunk < kUmmaMaxRing ? chunk : kUmmaMaxRing;
-        if (force_ring > 0 && force_ring < ring) ring = force_ring;
-        const int ring_floor = force_ring > 0 ? ring : (ring < 4 ? ring : 4);
-        while (ring > ring_floor && umma_smem_bytes(p.nb, chunk, ring) > kUmmaSmemHalf) --ring;
-        if (umma_smem_bytes(p.nb, chunk, ring) > kUmmaSmemHalf) {
-            // one CTA per SM: as deep a ring as fits
-            ring = chunk < kUmmaMaxRing ? chunk : kUmmaMaxRing;
+        int groups, ring;
+        long cost;
+        if (layer_regime) {
+            groups = p.tiles;
+            const long ctas = (long)groups * s;
+            const int tm = umma_tmem_cols(p.nb, 1);
+            ring = chunk < 8 ? chunk : 8;
+            if (force_ring > 0) ring = force_ring < chunk ? force_ring : chunk;
+            else
+                while (ring > 2 && ctas > (long)sms * umma_ctas_per_sm(umma_smem_bytes(p.nb, p.M, 1, chunk, ring), tm)) --ring;
+            while (ring > 1 && umma_smem_bytes(p.nb, p.M, 1, chunk, ring) > kUmmaSmemLimit) --ring;
+            const uint32_t bytes = umma_smem_bytes(p.nb, p.M, 1, chunk, ring);
+            if (bytes > kUmmaSmemLimit) continue;
+            const long slots = (long)sms * umma_ctas_per_sm(bytes, tm);
+            const long waves = (ctas + slots - 1) / slots;
+            const long off = ctas > 2L * sms ? ctas - 2L * sms : 2L * sms - ctas;   // distance from two CTAs per SM
+            cost = (waves - 1) * 100000 + off;
+        } else {
+            groups = sms / s < 1 ? 1 : sms / s;          // one CTA per SM
+            if (groups > p.tiles) groups = p.tiles;
+            if ((p.tiles + groups - 1) / groups > tcap) groups = (p.tiles + tcap - 1) / tcap;
+            const int tmax = (p.tiles + groups - 1) / groups;
+            const int units = tmax * chunk;
+            ring = units < kUmmaMaxUnitsResident ? units : kUmmaMaxUnitsResident;
             if (force_ring > 0 && force_ring < ring) ring = force_ring;
-            while (ring > 2 && umma_smem_bytes(p.nb, chunk, ring) > kUmmaSmemLimit) --ring;
-            if (umma_smem_bytes(p.nb, chunk, ring) > kUmmaSmemLimit) continue;
+            while (ring > 1 && umma_smem_bytes(p.nb, p.M, tmax, chunk, ring) > kUmmaSmemLimit) --ring;
+            if (umma_smem_bytes(p.nb, p.M, tmax, chunk, ring) > kUmmaSmemLimit) continue;
+            const long waves = ((long)groups * s + sms - 1) / sms;
+            cost = waves * units * 8 + chunk + (s > 1 ? 2 : 0);
         }
-        const uint32_t bytes = umma_smem_bytes(p.nb, chunk, ring);
-        const int occ = bytes <= kUmmaSmemThird ? 3 : (bytes <= kUmmaSmemHalf ? 2 : 1);
-        const long ctas = (long)p.tiles * s;
-        const long per_sm = (ctas + sms - 1) / sms;                 // CTAs the busiest SM runs in total
-        const long waves = (ctas + (long)sms * occ - 1) / ((long)sms * occ);
-        const long cost = per_sm * chunk * 4 + (s > 1 ? 4 : 0) + (waves - 1) * 8;   // in quarter stages
-        if (best_cost < 0 || cost < best_cost) {
+        if (best_cost < 0 || cost <= best_cost) {   // ties: the larger split
             best_cost = cost;
             best_split = s;
+            best_groups = groups;
             best_ring = ring;
         }
     }
     if (best_cost < 0) return false;
     p.split = best_split;
+    p.groups = best_groups;
+    p.tiles_max = (p.tiles + best_groups - 1) / best_groups;
     p.ring = best_ring;
     p.chunk_max = (p.ks + best_split - 1) / best_split;
-    p.grid = p.tiles * best_split;
-    p.smem_bytes = umma_smem_bytes(p.nb, p.chunk_max, best_ring);
-    p.tmem_cols = p.nb + 8 * best_ring <= 64 ? 64 : 128;
+    p.grid = best_groups * best_split;
+    p.smem_bytes = umma_smem_bytes(p.nb, p.M, p.tiles_max, p.chunk_max, best_ring);
+    p.tmem_cols = umma_tmem_cols(p.nb, p.tiles_max);
     return true;
 }
 

@@ -100,23 +100,29 @@ UMMA_SHAPES = SHAPES + [(1, 32000, 4096), (1, 1000, 65536), (16, 4096, 28672), (
 
 @pytest.mark.parametrize("m,n,k", UMMA_SHAPES)
 def test_tcgen05_plan_invariants(m, n, k):
-    """One CTA per (128-row tile, K chunk); the CTAs of a tile form a cluster of `split` <= 8; everything a
-    CTA keeps in shared and tensor memory fits."""
+    """FP8-operand tcgen05 kernel: a CTA owns a K range (its rank in a cluster of `split` <= 8) of a group of 128-row
+    tiles; everything it keeps in shared and tensor memory fits."""
     p = mxq.mxq_linear_plan_info(m, n, k, "umma")
     assert p["kernel"] == "umma"
     ks = k // 128
-    assert p["kb"] == k // 32 and p["tiles"] == -(-n // 128)
+    tiles = -(-n // 128)
+    assert p["kb"] == k // 32 and p["tiles"] == tiles
     assert 1 <= p["split"] <= min(8, ks)
-    assert p["grid"] == p["tiles"] * p["split"]
+    assert 1 <= p["groups"] <= tiles and p["grid"] == p["groups"] * p["split"]
+    assert p["tiles_max"] == -(-tiles // p["groups"])
     assert p["chunk_max"] == -(-ks // p["split"])
-    assert 1 <= p["ring"] <= min(8, p["chunk_max"])
+    assert 1 <= p["ring"] <= min(12, p["tiles_max"] * p["chunk_max"])
     assert p["nb"] in (16, 32, 48) and p["nb"] >= 3 * m and (p["nb"] == 16 or p["nb"] - 16 < 3 * m)
+    assert p["tiles_max"] * (p["nb"] // 3) <= 16 or p["tiles_max"] == 1   # results a thread keeps in registers
     assert p["smem_bytes"] <= 227 * 1024
-    assert p["tmem_cols"] in (64, 128) and p["tmem_cols"] >= p["nb"] + 8 * p["ring"]
+    assert p["tmem_cols"] in (32, 64, 128, 256, 512) and p["tmem_cols"] >= p["nb"] * p["tiles_max"] + 16
     # the stage ranges of a cluster's CTAs partition [0, K/128) and none is empty
     bounds = [r * ks // p["split"] for r in range(p["split"] + 1)]
     sizes = [b1 - b0 for b0, b1 in zip(bounds, bounds[1:])]
     assert bounds[0] == 0 and bounds[-1] == ks and min(sizes) >= 1 and max(sizes) <= p["chunk_max"]
+    tb = [g * tiles // p["groups"] for g in range(p["groups"] + 1)]
+    tsz = [b1 - b0 for b0, b1 in zip(tb, tb[1:])]
+    assert tb[0] == 0 and tb[-1] == tiles and min(tsz) >= 1 and max(tsz) == p["tiles_max"]
     # rows of a tile are shared out among the cluster's CTAs for the final sum
     rb = [r * 128 // p["split"] for r in range(p["split"] + 1)]
     assert rb[-1] == 128 and p["split"] * max(b1 - b0 for b0, b1 in zip(rb, rb[1:])) <= 136

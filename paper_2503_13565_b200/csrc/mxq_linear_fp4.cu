@@ -374,6 +374,11 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
         __syncwarp();
         if (elect_one()) tc_commit(done_bar);
         __syncwarp();
+        // tensor memory goes back as soon as the epilogue warps have read it (they arrive on barrier 2 without waiting),
+        // so that nothing but their stores is left at the end of the CTA
+        asm volatile("bar.sync 2, 160;" ::: "memory");
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
         TR(4);
     } else if (warp == 1) {
         // ---- producer warp: refill ring slots as the MMAs release them ----------------------------------------------
@@ -536,6 +541,8 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
             for (int q = 0; q < kResults; ++q)
                 if (q < ntile * MT) y[q] = scratch[q * kFp4TileRows + row];   // the thread's own values, back in registers
         }
+        tc_fence_before();
+        asm volatile("bar.arrive 2, 160;" ::: "memory");   // the accumulators have been read (or are not needed)
         if (s_fail) {
 #pragma unroll
             for (int q = 0; q < kResults; ++q) y[q] = __uint_as_float(0x7FC00000u);
@@ -603,10 +610,6 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
 
     TR(7);
     if (split > 1 && warp < 2) cluster_wait();   // pairs with the arrive in the prologue (the other warps waited before their push)
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 0)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
 }
 
 int env_int(const char *name) {
@@ -686,6 +689,14 @@ cudaError_t linear_fp4_launch(const Fp4Plan &p, const void *X, const uint8_t *co
                          : launch_fp4<64, false>(p, map, X, codes, scales, Y, y_dtype, stream);
     }
 }
+
+#ifdef MXQ_FP4_TRACE
+}  // namespace mxq
+extern "C" __attribute__((visibility("default"))) int mxq_fp4_trace(unsigned long long *out) {
+    return cudaMemcpyFromSymbol(out, mxq::g_fp4_trace, sizeof(mxq::g_fp4_trace)) == cudaSuccess ? 0 : 6;
+}
+namespace mxq {
+#endif
 
 // returns and clears this kernel's sticky status word (see mxq_linear_device_status)
 int linear_fp4_take_status(uint32_t *out) {

@@ -306,6 +306,11 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
         __syncwarp();
         if (elect_one()) tc_commit(done_bar);
         __syncwarp();
+        // tensor memory goes back as soon as the epilogue warps have read it (they arrive on barrier 2 without waiting),
+        // so that nothing but their stores is left at the end of the CTA
+        asm volatile("bar.sync 2, 160;" ::: "memory");
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
     } else if (warp == 1) {
         // ---- producer warp: refill ring slots as the MMAs release them ----------------------------------------------
         uint32_t slot = 0, phase = 0;   // unit `pre` reuses slot 0 (pre == ring whenever the loop runs)
@@ -445,6 +450,8 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
             for (int q = 0; q < kResults; ++q)
                 if (q < ntile * MT) y[q] = scratch[q * kUmmaTileRows + row];   // the thread's own values, back in registers
         }
+        tc_fence_before();
+        asm volatile("bar.arrive 2, 160;" ::: "memory");   // the accumulators have been read (or are not needed)
         if (s_fail) {
 #pragma unroll
             for (int q = 0; q < kResults; ++q) y[q] = __uint_as_float(0x7FC00000u);
@@ -510,10 +517,6 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
     }
 
     if (split > 1 && warp < 2) cluster_wait();   // pairs with the arrive in the prologue (the other warps waited before their push)
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 0)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
 }
 
 int env_int(const char *name) {

@@ -89,9 +89,12 @@ int mxq_quantize(const void *W_bf16, int64_t N, int64_t K, uint8_t *codes, uint8
 int mxq_dequantize(const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K, void *W_bf16_out,
                    void *stream);
 
-/* Workspace (bytes) mxq_linear needs for this shape; 0 for every shape in this version
- * (partial results of a split row meet in on-chip memory, never in global memory), kept in the
- * interface for future kernels.  If non-zero: zero-fill once before first use; calls leave it reusable. */
+/* Workspace (bytes) with which mxq_linear runs fastest for this shape; 0 where none is used.  The workspace is
+ * OPTIONAL: mxq_linear accepts NULL / 0 or a smaller buffer and is then merely slower for 3 or more token rows.
+ * With it, MXQ_KERNEL_UMMA rewrites the M token rows as FP8 parts once per call (a small kernel ahead of the
+ * weight kernel, which then fetches them with bulk copies) instead of once per CTA.  Device memory, 16-byte
+ * aligned, no initialisation needed; contents are scratch.  Calls that may run concurrently (different streams)
+ * need a workspace each. */
 size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K);
 
 /* The kernels behind mxq_linear, fastest first.
@@ -143,7 +146,7 @@ int mxq_linear_device_status(uint32_t *status_host);
  *   X_bf16  [M][K] BF16 row-major (read)
  *   codes, scales  the MXFP4 pair for W[N][K] (read)
  *   Y       [M][N] row-major, float (MXQ_F32) or BF16 rounded to nearest even (MXQ_BF16)
- *   workspace / workspace_bytes  see mxq_linear_workspace_bytes (may be NULL / 0 if that is 0)
+ *   workspace / workspace_bytes  optional scratch, see mxq_linear_workspace_bytes (NULL / 0 allowed)
  * Products are formed exactly and accumulated in FP32; the block scale is applied to
  * 32-long partial sums (Eq. 2).  The summation order is fixed for a given shape, so
  * results are bit-reproducible run to run.  A row containing a 0xFF scale yields NaN. */

@@ -27,8 +27,11 @@ struct UmmaPlan;
 // tcgen05 path of mxq_linear (mxq_linear_umma.cu): false if the shape is not covered
 bool linear_umma_available();
 bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &plan);
+// workspace: optional; with linear_umma_workspace_bytes(M, K) bytes (0: not used for this M) the token operand is split
+// once per call by a kernel of its own instead of by every CTA of the weight kernel
+size_t linear_umma_workspace_bytes(int M, int64_t K);
 cudaError_t linear_umma_launch(const UmmaPlan &plan, const void *X, const uint8_t *codes, const uint8_t *scales,
-                               void *Y, int y_dtype, cudaStream_t stream);
+                               void *Y, int y_dtype, void *workspace, size_t workspace_bytes, cudaStream_t stream);
 
 struct Fp4Plan;
 // tcgen05 path with packed 4-bit operands on both sides, M <= 4 (mxq_linear_fp4.cu)

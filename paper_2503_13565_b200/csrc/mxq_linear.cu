@@ -157,7 +157,9 @@ extern "C" {
 
 size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K) {
     if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return 0;
-    return 0;   // the tcgen05 kernel adds partial results inside a cluster, the others never split a row
+    // No kernel needs one (partial results are added inside a thread-block cluster or never leave a warp); the
+    // FP8-operand tcgen05 kernel is faster with one: the token operand is then split once per call.
+    return mxq::linear_umma_available() ? mxq::linear_umma_workspace_bytes(M, K) : 0;
 }
 
 int mxq_set_linear_kernel(int kernel) {
@@ -219,8 +221,6 @@ int mxq_linear_plan_info(int kernel, int M, int64_t N, int64_t K, int32_t *info)
 
 int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
                void *Y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream) {
-    (void)workspace;
-    (void)workspace_bytes;
     if (!X_bf16 || !codes || !scales || !Y) return MXQ_ERR_NULL;
     if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return MXQ_ERR_SHAPE;
     if (y_dtype != MXQ_F32 && y_dtype != MXQ_BF16) return MXQ_ERR_DTYPE;
@@ -232,7 +232,7 @@ int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *s
     if (c.kernel != MXQ_KERNEL_GENERIC) {
         const cudaError_t e =
             c.kernel == MXQ_KERNEL_FP4    ? mxq::linear_fp4_launch(c.fp4, X_bf16, codes, scales, Y, y_dtype, st)
-            : c.kernel == MXQ_KERNEL_UMMA ? mxq::linear_umma_launch(c.umma, X_bf16, codes, scales, Y, y_dtype, st)
+            : c.kernel == MXQ_KERNEL_UMMA ? mxq::linear_umma_launch(c.umma, X_bf16, codes, scales, Y, y_dtype, workspace, workspace_bytes, st)
                                           : mxq::linear_mma_launch(c.mma, X_bf16, codes, scales, Y, y_dtype, nullptr, st);
         if (e != cudaSuccess) {
             if (std::getenv("MXQ_DEBUG")) std::fprintf(stderr, "mxq_linear (kernel %d): %s\n", c.kernel, cudaGetErrorString(e));

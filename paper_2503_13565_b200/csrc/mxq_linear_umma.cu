@@ -113,6 +113,55 @@ __device__ __forceinline__ bool split_unit(const uint4 raw, bool act, int m, int
     return inexact && act;
 }
 
+// The token operand of a whole call, split once, ahead of the weight kernel (from kUmmaPresplitMinM token rows on, where
+// every CTA splitting its own K range costs more than one more launch in the chain).  CTA = 256 k of every token;
+// a warp takes tokens warp, warp + 8, ...  The result lies in the workspace as umma_ws_bytes describes.
+constexpr int kSplitWarps = 8;
+template <int NB>
+__global__ void __launch_bounds__(kSplitWarps * 32)
+split_tokens_kernel(const __nv_bfloat16 *__restrict__ X, int M, int64_t K, int ks, uint8_t *__restrict__ ws) {
+    pdl_trigger();   // the weight kernel may start at once: it streams weights until this kernel has completed
+    __shared__ int s_bad;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) s_bad = 0;
+    uint8_t *gSFB = ws + umma_ws_flags_bytes(ks), *gB = gSFB + (size_t)ks * kUmmaSfStageBytes;
+    const int kk = (int)blockIdx.x * (2 * kUmmaStageK) + lane * 8;
+    const bool act = kk < K;
+    pdl_wait();      // X may be the previous kernel's output; the workspace may still be read by the previous weight kernel
+    __syncthreads();
+    uint4 raw[(kUmmaMaxM + kSplitWarps - 1) / kSplitWarps];
+#pragma unroll
+    for (int q = 0; q < (kUmmaMaxM + kSplitWarps - 1) / kSplitWarps; ++q) {
+        const int m = warp + q * kSplitWarps;
+        raw[q] = make_uint4(0, 0, 0, 0);
+        if (m < M && act) raw[q] = *reinterpret_cast<const uint4 *>(X + (int64_t)m * K + kk);
+    }
+    bool inexact = false;
+#pragma unroll
+    for (int q = 0; q < (kUmmaMaxM + kSplitWarps - 1) / kSplitWarps; ++q) {
+        const int m = warp + q * kSplitWarps;
+        if (m < M) inexact |= split_unit<NB>(raw[q], act, m, kk, lane, gB, gSFB);   // uniform across the warp
+    }
+    if (inexact) s_bad = 1;
+    __syncthreads();
+    const int stage = (int)blockIdx.x * 2 + (int)threadIdx.x;
+    if (threadIdx.x < 2 && stage < ks) reinterpret_cast<uint32_t *>(ws)[stage] = (uint32_t)s_bad;
+}
+
+template <int NB>
+cudaError_t launch_split(const __nv_bfloat16 *X, int M, int64_t K, int ks, uint8_t *ws, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((ks + 1) / 2));
+    cfg.blockDim = dim3(kSplitWarps * 32);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, split_tokens_kernel<NB>, X, M, K, ks, ws);
+}
+
 // NB: columns of the B operand / accumulator = 3 parts x tokens, rounded up to 16, 32 or 48.
 // Warp roles (192 threads): warp 0 issues the MMAs and owns tensor memory; warp 1 is the producer (TMA copies of
 // the codes, cp.async of the scale bytes, barrier set-up); warps 2..5 split the activations stage by stage and,
@@ -123,7 +172,7 @@ __global__ void __launch_bounds__(kUmmaThreads)
 linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 *__restrict__ X, int M,
                   const uint8_t *__restrict__ codes, const uint8_t *__restrict__ scales, int64_t N, int64_t K,
                   void *__restrict__ Y, int y_dtype, int split, int ring, int ks, int chunk_max, int tmem_cols, int groups,
-                  int tiles, int tiles_max) {
+                  int tiles, int tiles_max, const uint8_t *__restrict__ presplit) {
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");   // needed by the first copy, 1 us from now
@@ -192,7 +241,8 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
     if (warp == 1) {
         for (int b = lane; b < 2 * ring + 2 + npair; b += 32) {
             // full: the TMA lane + 32 producer lanes; empty, done, recv: 1; ready (one per 256 k): one arrival per token
-            const uint32_t count = b < ring ? kFullArrivals : (b < 2 * ring + 2 ? 1u : (uint32_t)M);
+            // (with the token operand split ahead of this kernel: the one thread that requests the copies)
+            const uint32_t count = b < ring ? kFullArrivals : (b < 2 * ring + 2 || presplit ? 1u : (uint32_t)M);
             mbar_init(sBar + (uint32_t)b * 8u, count);
         }
         if (lane == 31) {
@@ -243,7 +293,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
             }
         }
     }
-    constexpr int kResults = MULTI ? 16 : NB / kUmmaParts;
+    constexpr int kResults = MULTI ? umma_results_cap(NB) : NB / kUmmaParts;
     float y[kResults];   // results of this thread's row: [tile][token slot]
 #pragma unroll
     for (int q = 0; q < kResults; ++q) y[q] = 0.f;
@@ -340,7 +390,23 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
         const int row = ((warp & 3) << 5) + lane;                  // accumulator row this thread may read (its warp's quarter)
         volatile int &s_bad = *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 8);
         bool inexact = false;
-        {
+        if (presplit) {
+            // The token operand was split by split_tokens_kernel: fetch this CTA's stages, two at a time, each pair
+            // completing the "ready" barrier the MMA warp waits on; the flags say whether every block split exactly.
+            const uint8_t *ws_sf = presplit + umma_ws_flags_bytes(ks), *ws_b = ws_sf + (size_t)ks * kUmmaSfStageBytes;
+            if (ct == 0) {
+                for (int p = 0; p < npair; ++p) {
+                    const uint32_t n2 = (uint32_t)min(2, nst - 2 * p), bar = ready0 + (uint32_t)p * 8u;
+                    mbar_expect_tx(bar, n2 * (NB * 128u + kUmmaSfStageBytes));
+                    bulk_load(sB + (uint32_t)(2 * p) * (NB * 128u), ws_b + (size_t)(s_begin + 2 * p) * (NB * 128u), n2 * (NB * 128u), bar);
+                    bulk_load(sSFB + (uint32_t)(2 * p) * kUmmaSfStageBytes, ws_sf + (size_t)(s_begin + 2 * p) * kUmmaSfStageBytes,
+                              n2 * kUmmaSfStageBytes, bar);
+                }
+                s_xin = 1;   // lets the producer request the rest of the ring
+            }
+            const uint32_t *flags = reinterpret_cast<const uint32_t *>(presplit);
+            for (int i = ct; i < nst; i += 128) inexact |= flags[s_begin + i] != 0u;
+        } else {
             // Groups of 32 units (256 k of one token, one warp; a unit is 8 elements, one lane) in order of K, so that
             // the MMA warp can start on the first stages while later ones are being split.  Group G: pair of stages
             // G / M, token G % M; the last pair is half full when the CTA has an odd number of stages.  All of this
@@ -384,7 +450,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
 
         // ---- epilogue: accumulator row -> registers; the three parts of a token are three neighbouring columns -------
         constexpr int MT = NB / kUmmaParts;         // token slots per tile (5, 10 or 16)
-        constexpr int TCAP = MULTI ? 16 / MT : 1;   // tiles a thread can keep results for
+        constexpr int TCAP = MULTI ? kResults / MT : 1;   // tiles a thread can keep results for
         if (!mbar_wait_relaxed(done_bar, 0)) {
             atomicOr(&g_umma_status, 4u);
             s_fail = 1;
@@ -526,7 +592,7 @@ int env_int(const char *name) {
 
 template <int NB, bool MULTI>
 cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X, const uint8_t *codes,
-                       const uint8_t *scales, void *Y, int y_dtype, cudaStream_t stream) {
+                       const uint8_t *scales, void *Y, int y_dtype, const uint8_t *presplit, cudaStream_t stream) {
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -562,7 +628,7 @@ cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X
     cfg.attrs = attr;
     cfg.numAttrs = na;
     return cudaLaunchKernelEx(&cfg, linear_umma_kernel<NB, MULTI>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
-                              Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols, p.groups, p.tiles, p.tiles_max);
+                              Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols, p.groups, p.tiles, p.tiles_max, presplit);
 }
 
 }  // namespace
@@ -573,22 +639,45 @@ bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p) {
     p.M = M;
     p.N = N;
     p.K = K;
-    p.nb = 3 * M <= 16 ? 16 : (3 * M <= 32 ? 32 : 48);
+    p.nb = umma_nb(M);
     p.ks = (int)(K / kUmmaStageK);
     p.tiles = (int)((N + kUmmaTileRows - 1) / kUmmaTileRows);
-    return umma_layout(p, sm_count(), env_int("MXQ_UMMA_SPLIT"), env_int("MXQ_UMMA_RING"));
+    return umma_layout(p, sm_count(), env_int("MXQ_UMMA_SPLIT"), env_int("MXQ_UMMA_RING"), env_int("MXQ_UMMA_TILES"));
+}
+
+size_t linear_umma_workspace_bytes(int M, int64_t K) {
+    if (M < kUmmaPresplitMinM || M > kUmmaMaxM || K < 128 || (K % 128) != 0 || K > 0x3FFFFFFF) return 0;
+    return umma_ws_bytes(umma_nb(M), (int)(K / kUmmaStageK));
 }
 
 cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,
-                              int y_dtype, cudaStream_t stream) {
+                              int y_dtype, void *workspace, size_t workspace_bytes, cudaStream_t stream) {
     CUtensorMap map;
     if (!codes_tensor_map(codes, p.N, p.K, /*expand_fp4=*/true, &map)) return cudaErrorNotSupported;
+    // a workspace that is large enough (and aligned for bulk copies) lets the token operand be split once per call
+    static const bool no_presplit = env_int("MXQ_UMMA_NO_PRESPLIT") != 0;
+    static const int min_m = env_int("MXQ_UMMA_PRESPLIT_MIN_M") > 0 ? env_int("MXQ_UMMA_PRESPLIT_MIN_M") : kUmmaPresplitMinM;
+    const size_t need = umma_ws_bytes(p.nb, p.ks);
+    uint8_t *ws = nullptr;
+    if (!no_presplit && p.M >= min_m && workspace && workspace_bytes >= need && (reinterpret_cast<uintptr_t>(workspace) & 15u) == 0)
+        ws = static_cast<uint8_t *>(workspace);
+    if (ws) {
+        const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(X);
+        const cudaError_t e = p.nb == 16   ? launch_split<16>(x, p.M, p.K, p.ks, ws, stream)
+                              : p.nb == 32 ? launch_split<32>(x, p.M, p.K, p.ks, ws, stream)
+                                           : launch_split<48>(x, p.M, p.K, p.ks, ws, stream);
+        if (e != cudaSuccess) return e;
+    }
     switch (p.nb) {
-        case 16:   // the only width with room in a thread's registers for more than one tile
-            return p.tiles_max > 1 ? launch_umma<16, true>(p, map, X, codes, scales, Y, y_dtype, stream)
-                                   : launch_umma<16, false>(p, map, X, codes, scales, Y, y_dtype, stream);
-        case 32: return launch_umma<32, false>(p, map, X, codes, scales, Y, y_dtype, stream);
-        default: return launch_umma<48, false>(p, map, X, codes, scales, Y, y_dtype, stream);
+        case 16:
+            return p.tiles_max > 1 ? launch_umma<16, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
+                                   : launch_umma<16, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream);
+        case 32:
+            return p.tiles_max > 1 ? launch_umma<32, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
+                                   : launch_umma<32, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream);
+        default:
+            return p.tiles_max > 1 ? launch_umma<48, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
+                                   : launch_umma<48, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream);
     }
 }
 

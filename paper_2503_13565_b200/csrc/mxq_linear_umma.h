@@ -5,6 +5,12 @@
 
 namespace mxq {
 
+#ifdef __CUDACC__
+#define MXQ_UMMA_HD __host__ __device__
+#else
+#define MXQ_UMMA_HD
+#endif
+
 constexpr int kUmmaTileRows = 128;   // weight rows per tile = M of one tcgen05.mma
 constexpr int kUmmaStageK = 128;     // k per ring stage = 4 MX blocks = 4 MMAs of K = 32
 constexpr int kUmmaThreads = 192;    // MMA warp, producer warp, four activation / epilogue warps
@@ -17,6 +23,19 @@ constexpr int kUmmaMaxSplit = 8;                  // portable cluster size
 constexpr uint32_t kUmmaRecvRows = 136;           // >= split * ceil(128 / split) for every split <= 8
 constexpr uint32_t kUmmaSmemLimit = 227 * 1024;
 constexpr int kUmmaMaxUnitsResident = 12;         // most ring slots (16 KB of expanded codes + 512 B of scales each)
+
+// The token operand split ahead of the weight kernel, in the caller's workspace: one 32-bit "cannot be split
+// exactly" flag per stage (padded to 1 KB), then one 512-byte scale atom per stage, then one image of the stage's
+// nb x 128 bytes of E5M2 parts per stage -- atoms and images exactly as the weight kernel keeps them in shared memory,
+// so that a CTA fetches its K range with two bulk copies per 256 k.
+constexpr int kUmmaPresplitMinM = 3;              // fewer token rows: splitting inside the weight kernel is as fast
+MXQ_UMMA_HD inline size_t umma_ws_flags_bytes(int ks) { return (((size_t)ks * 4u) + 1023u) & ~(size_t)1023u; }
+MXQ_UMMA_HD inline size_t umma_ws_bytes(int nb, int ks) {
+    return umma_ws_flags_bytes(ks) + (size_t)ks * kUmmaSfStageBytes + (size_t)ks * (size_t)nb * 128u;
+}
+// results (tile x token slot) an epilogue thread keeps in registers when its CTA owns several tiles
+MXQ_UMMA_HD constexpr int umma_results_cap(int nb) { return nb == 16 ? 16 : 32; }
+inline int umma_nb(int M) { return 3 * M <= 16 ? 16 : (3 * M <= 32 ? 32 : 48); }
 
 struct UmmaPlan {
     int M;           // token rows (1..16)
@@ -59,12 +78,16 @@ inline int umma_ctas_per_sm(uint32_t smem_bytes, int tmem_cols) {
 // kernel: up to 2 * SMs tiles -> one tile per CTA, every CTA resident at once, about two CTAs per SM (ties to the
 // larger split: splitting the activations is this kernel's main cost from M = 4 on, and it shrinks with the K range);
 // more tiles -> one CTA per SM walking several tiles.
-// force_split / force_ring (> 0) override the heuristic where they are feasible.
-inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring) {
+// force_split / force_ring / force_tiles (> 0) override the heuristic where they are feasible.
+inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, int force_tiles = 0) {
     const int slots_per_tile = p.nb / kUmmaParts;        // 5, 10 or 16 tokens fit in a tile's columns
-    const int tcap_regs = 16 / slots_per_tile;           // results a thread keeps in registers: tiles * slots <= 16
-    const int tcap = tcap_regs < 1 ? 1 : tcap_regs;
-    const bool layer_regime = p.tiles <= 2 * sms || tcap == 1;
+    const int tcap = umma_results_cap(p.nb) / slots_per_tile;   // tiles whose results fit in a thread's registers: 3, 3, 2
+    const bool layer_regime = p.tiles <= 2 * sms;
+    // Tiles per CTA in the layer regime: one, except for the widest token operand on matrices of many tiles, where
+    // the operand's K range of a CTA (6.5 KB per stage) leaves too little shared memory for weights unless two
+    // tiles share it (11008 x 4096 at M = 16: 21.5 -> 16 us).
+    int tper = p.nb == 48 && 2 * p.tiles >= sms ? 2 : 1;
+    if (force_tiles > 0) tper = force_tiles < tcap ? force_tiles : tcap;
     long best_cost = -1;
     int best_split = 0, best_groups = 0, best_ring = 0;
     const int smax = p.ks < kUmmaMaxSplit ? p.ks : kUmmaMaxSplit;
@@ -74,15 +97,18 @@ inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring) {
         int groups, ring;
         long cost;
         if (layer_regime) {
-            groups = p.tiles;
+            groups = (p.tiles + tper - 1) / tper;
+            const int tmax = (p.tiles + groups - 1) / groups;
             const long ctas = (long)groups * s;
-            const int tm = umma_tmem_cols(p.nb, 1);
-            ring = chunk < 8 ? chunk : 8;
-            if (force_ring > 0) ring = force_ring < chunk ? force_ring : chunk;
+            const int tm = umma_tmem_cols(p.nb, tmax);
+            const int units = tmax * chunk;
+            ring = units < kUmmaMaxUnitsResident ? units : kUmmaMaxUnitsResident;
+            if (tper == 1 && ring > 8) ring = 8;
+            if (force_ring > 0) ring = force_ring < units ? force_ring : units;
             else
-                while (ring > 2 && ctas > (long)sms * umma_ctas_per_sm(umma_smem_bytes(p.nb, p.M, 1, chunk, ring), tm)) --ring;
-            while (ring > 1 && umma_smem_bytes(p.nb, p.M, 1, chunk, ring) > kUmmaSmemLimit) --ring;
-            const uint32_t bytes = umma_smem_bytes(p.nb, p.M, 1, chunk, ring);
+                while (ring > 2 && ctas > (long)sms * umma_ctas_per_sm(umma_smem_bytes(p.nb, p.M, tmax, chunk, ring), tm)) --ring;
+            while (ring > 1 && umma_smem_bytes(p.nb, p.M, tmax, chunk, ring) > kUmmaSmemLimit) --ring;
+            const uint32_t bytes = umma_smem_bytes(p.nb, p.M, tmax, chunk, ring);
             if (bytes > kUmmaSmemLimit) continue;
             const long slots = (long)sms * umma_ctas_per_sm(bytes, tm);
             const long waves = (ctas + slots - 1) / slots;

@@ -113,7 +113,7 @@ def test_tcgen05_plan_invariants(m, n, k):
     assert p["chunk_max"] == -(-ks // p["split"])
     assert 1 <= p["ring"] <= min(12, p["tiles_max"] * p["chunk_max"])
     assert p["nb"] in (16, 32, 48) and p["nb"] >= 3 * m and (p["nb"] == 16 or p["nb"] - 16 < 3 * m)
-    assert p["tiles_max"] * (p["nb"] // 3) <= 16 or p["tiles_max"] == 1   # results a thread keeps in registers
+    assert p["tiles_max"] * (p["nb"] // 3) <= (16 if p["nb"] == 16 else 32) or p["tiles_max"] == 1   # results a thread keeps in registers
     assert p["smem_bytes"] <= 227 * 1024
     assert p["tmem_cols"] in (32, 64, 128, 256, 512) and p["tmem_cols"] >= p["nb"] * p["tiles_max"] + 16
     # the stage ranges of a cluster's CTAs partition [0, K/128) and none is empty

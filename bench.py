@@ -237,6 +237,27 @@ def time_fn(fn, iters: int, warmup: int = 3):
     return e0.elapsed_time(e1) * 1e-3 / iters
 
 
+def time_graph(fn, iters: int, warmup: int = 3):
+    """Device time per replay of a CUDA graph of fn() (no host launch overhead between the kernels)."""
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        fn()
+        st.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            fn()
+        for _ in range(warmup):
+            g.replay()
+        st.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        for _ in range(iters):
+            g.replay()
+        e1.record(st)
+        st.synchronize()
+    return e0.elapsed_time(e1) * 1e-3 / iters
+
+
 def cpu_baseline_leg(m: int, budget_s: float = 15.0):
     """The oracle, as it stands, on one 7B layer set (host cores of this machine)."""
     import numpy as np
@@ -329,18 +350,17 @@ def run_ours(args):
         ws_ = [w.clone() for _ in range(4)]   # 360 MB rotated: larger than L2
         codes = torch.empty((11008, 2048), dtype=torch.uint8, device=device)
         scales = torch.empty((11008, 128), dtype=torch.uint8, device=device)
-        it = [0]
 
-        def q():
-            mxq.mxq_quantize(ws_[it[0] % 4], codes, scales)
-            it[0] += 1
-        tq = time_fn(q, 40)
+        def q():   # one replay = the four matrices once
+            for w_ in ws_:
+                mxq.mxq_quantize(w_, codes, scales)
+        tq = time_graph(q, 10) / 4
         extra["quantize"] = {"gbs": 11008 * 4096 * 2.53125 / tq / 1e9, "us_per_call": tq * 1e6, "shape": "11008x4096"}
         del w, ws_
         # greedy accept: 250 sequences x 17 rows x 32000 logits (FP32), one call
         lg, draft, _, _ = synth.accept_trials(250, 16, 17, 32000, seed=1, device=device)
         ws2 = mxq.new_workspace(mxq.mxq_accept_workspace_bytes(250, 17, 32000), device)
-        ta = time_fn(lambda: mxq.mxq_greedy_accept(lg, draft, workspace=ws2), 20)
+        ta = time_graph(lambda: mxq.mxq_greedy_accept(lg, draft, workspace=ws2), 20)
         extra["greedy_accept"] = {"gbs": lg.numel() * 4 / ta / 1e9, "us_per_call": ta * 1e6, "shape": "250x17x32000 f32"}
         del lg
 
@@ -387,8 +407,11 @@ def run_case(args):
         raise SystemExit("bench.py needs a CUDA device: the product has no CPU path")
     import paper_2503_13565_b200 as mxq
     mxq.binding.lib()
-    n, k, m = (int(v) for v in args.case.lower().split("x"))
     device = torch.device("cuda", 0)
+    case = args.case.lower()
+    if case.startswith("quantize:") or case.startswith("accept:"):
+        return run_case_other(mxq, case, args.steps, device)
+    n, k, m = (int(v) for v in case.split("x"))
     nbytes = algorithmic_bytes(m, n, k)
     copies = max(2, min(8, int(200e6 // nbytes) + 1))
     gen = torch.Generator(device=device).manual_seed(7)
@@ -410,6 +433,49 @@ def run_case(args):
     print(json.dumps({"case": args.case, "kernel": mxq.mxq_linear_plan_info(m, n, k)["kernel"], "launches": args.steps,
                       "us_per_call": us, "gbs": nbytes / us / 1e3, "bytes_per_call": nbytes,
                       "device_status": mxq.mxq_linear_device_status()}))
+
+
+def run_case_other(mxq, case: str, steps: int, device):
+    """--case quantize:NxK (direct cast of `steps` distinct BF16 matrices, rotated) or accept:BxRxV (greedy accept of
+    FP32 logits, T = R - 1): the small cases profiler captures of those kernels run on."""
+    op, dims = case.split(":")
+    dims = [int(v) for v in dims.split("x")]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if op == "quantize":
+        n, k = dims
+        copies = max(2, min(8, int(400e6 // (n * k * 2)) + 1))
+        ws_ = [synth.student_t_bf16((n, k), 0.02, 1 + i, device=device) for i in range(copies)]
+        codes = torch.empty((n, k // 2), dtype=torch.uint8, device=device)
+        scales = torch.empty((n, k // 32), dtype=torch.uint8, device=device)
+        mxq.mxq_quantize(ws_[0], codes, scales)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(steps):
+            mxq.mxq_quantize(ws_[i % copies], codes, scales)
+        e1.record()
+        nbytes = n * k * 2.53125
+
+        def all_copies():
+            for w_ in ws_:
+                mxq.mxq_quantize(w_, codes, scales)
+        graph_us = time_graph(all_copies, 10) / copies * 1e6
+    else:
+        b, r, v = dims
+        lg, draft, _, _ = synth.accept_trials(b, r - 1, r, v, seed=1, device=device)
+        ws = mxq.new_workspace(mxq.mxq_accept_workspace_bytes(b, r, v), device)
+        mxq.mxq_greedy_accept(lg, draft, workspace=ws)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(steps):
+            mxq.mxq_greedy_accept(lg, draft, workspace=ws)
+        e1.record()
+        nbytes = lg.numel() * 4
+        graph_us = time_graph(lambda: mxq.mxq_greedy_accept(lg, draft, workspace=ws), 10) * 1e6
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / steps
+    print(json.dumps({"case": case, "launches": steps, "us_per_call_from_python": us, "us_per_call": graph_us,
+                      "gbs": nbytes / graph_us / 1e3, "bytes_per_call": nbytes,
+                      "note": "us_per_call: replayed CUDA graph; from_python adds the host launch overhead"}))
 
 
 def run_reference(args):

@@ -16,21 +16,37 @@ constexpr int kQuantThreads = 256;
 constexpr int kQuantUnroll = 4;  // 16-byte loads in flight per lane
 
 // Cast the 8 BF16 values of one chunk given the block's scale byte; returns 8 packed codes.
+// The kernel is a stream of 2.5 bytes per weight, so the integer pipe must not spend more than a few instructions
+// per weight: the conversion instruction takes the sign along (a negative value that rounds to zero gives the
+// code of -0, as the cast requires).
 __device__ __forceinline__ uint32_t cast_chunk(const uint4 &v, uint32_t scale_byte) {
     // v / X with X = 2^(byte-127): multiply by 2^(127-byte), exact (a power of two; results
-    // stay below 8, and anything that underflows is far below the first rounding boundary).
+    // stay below 8 in magnitude, and anything that underflows is far below the first rounding boundary).
     const float inv_x = __uint_as_float((254u - scale_byte) << 23);
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    uint32_t out = 0;
+    float lo[4], hi[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-        const float lo = __uint_as_float((w[j] & 0x7FFFu) << 16) * inv_x;     // |element 2j|
-        const float hi = __uint_as_float(w[j] & 0x7FFF0000u) * inv_x;         // |element 2j+1|
-        uint32_t c = float2_to_e2m1x2(lo, hi);                                 // round-to-nearest-even, clamp
-        c |= ((w[j] >> 12) & 0x8u) | ((w[j] >> 24) & 0x80u);                   // input sign bits, always kept
-        out |= c << (8 * j);
+        lo[j] = __uint_as_float(w[j] << 16) * inv_x;            // element 2j
+        hi[j] = __uint_as_float(w[j] & 0xFFFF0000u) * inv_x;    // element 2j+1
     }
+    // round-to-nearest-even, clamp, sign kept; the bytes are packed with multiply-adds, which run on the other pipe
+    uint32_t c[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) c[j] = float2_to_e2m1x2(lo[j], hi[j]);
+    uint32_t out;
+    asm("{\n\t.reg .u32 t;\n\tmad.lo.u32 t, %2, 256, %1;\n\tmad.lo.u32 t, %3, 65536, t;\n\tmad.lo.u32 %0, %4, 16777216, t;\n\t}"
+        : "=r"(out)
+        : "r"(c[0]), "r"(c[1]), "r"(c[2]), "r"(c[3]));
     return out;
+}
+
+// largest magnitude pattern (15 bits) among the 8 BF16 values of a chunk: for finite BF16 the magnitude bits order like
+// the values; two values per instruction
+__device__ __forceinline__ uint32_t chunk_max(const uint4 &v) {
+    const uint32_t m = 0x7FFF7FFFu;
+    const uint32_t a = __vmaxu2(__vmaxu2(v.x & m, v.y & m), __vmaxu2(v.z & m, v.w & m));
+    return max(a & 0xFFFFu, a >> 16);
 }
 
 __global__ void __launch_bounds__(kQuantThreads)
@@ -48,9 +64,7 @@ quantize_kernel(const uint4 *__restrict__ W, uint32_t *__restrict__ codes, uint8
         }
 #pragma unroll
         for (int u = 0; u < kQuantUnroll; ++u) {
-            // block maximum: for finite BF16 the magnitude bits order like the values
-            uint32_t a = max(max(v[u].x & 0x7FFFu, (v[u].x >> 16) & 0x7FFFu), max(v[u].y & 0x7FFFu, (v[u].y >> 16) & 0x7FFFu));
-            a = max(a, max(max(v[u].z & 0x7FFFu, (v[u].z >> 16) & 0x7FFFu), max(v[u].w & 0x7FFFu, (v[u].w >> 16) & 0x7FFFu)));
+            uint32_t a = chunk_max(v[u]);
             a = max(a, __shfl_xor_sync(0xffffffffu, a, 1));
             a = max(a, __shfl_xor_sync(0xffffffffu, a, 2));
             const uint32_t efield = a >> 7;               // biased exponent of the block maximum
@@ -105,7 +119,7 @@ int mxq_quantize(const void *W_bf16, int64_t N, int64_t K, uint8_t *codes, uint8
     const int64_t nchunks = N * K / 8;
     const int64_t per_pass = (int64_t)mxq::kQuantThreads * mxq::kQuantUnroll;
     int64_t grid = (nchunks + per_pass - 1) / per_pass;
-    const int64_t cap = (int64_t)mxq::sm_count() * 8;  // 8 resident CTAs of 256 lanes per SM
+    const int64_t cap = (int64_t)mxq::sm_count() * 8;  // more CTAs than are resident at once (5 per SM): measured faster than one wave
     if (grid > cap) grid = cap;
     const int64_t iters = (nchunks + grid * per_pass - 1) / (grid * per_pass);
     mxq::quantize_kernel<<<(unsigned)grid, mxq::kQuantThreads, 0, (cudaStream_t)stream>>>(

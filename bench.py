@@ -331,19 +331,29 @@ def run_ours(args):
                 per_shape["%s_m%d" % (name, mm)] = {"us_per_call": s / 20 / len(sel) * 1e6,
                                                     "gbs": p.bytes * 20 / s / 1e9}
         extra["per_shape"] = per_shape
-        # vocabulary projections (one launch streams 70 / 279 MB): where launch latency no longer hides the kernel
-        vocab = {}
-        for n, copies in ((32000, 3), (128256, 2)):
-            gen = torch.Generator(device=device).manual_seed(n)
-            sel = [("lm_head", n, 4096,
-                    torch.randint(0, 256, (n, 2048), dtype=torch.uint8, device=device, generator=gen),
-                    torch.randint(110, 126, (n, 128), dtype=torch.uint8, device=device, generator=gen)) for _ in range(copies)]
-            for mm in (1, 4):
+        # vocabulary projections (one launch streams 70 / 279 MB): where launch latency no longer hides the kernel;
+        # and the token-count curves of the 13B layer shapes and of the paper's own 8192 x 8192 micro-benchmark shape
+        def m_curve(n, k, ms, iters=10):
+            copies = max(2, int(300e6 // (n * k * 0.53125)) + 1)   # rotated, together larger than L2
+            gen = torch.Generator(device=device).manual_seed(n + k)
+            sel = [("w", n, k,
+                    torch.randint(0, 256, (n, k // 2), dtype=torch.uint8, device=device, generator=gen),
+                    torch.randint(110, 126, (n, k // 32), dtype=torch.uint8, device=device, generator=gen)) for _ in range(copies)]
+            out = {}
+            for mm in ms:
                 p = LinearPass(mxq, sel, mm, device, seed=34, use_graph=not args.no_graph)
-                s = p.time(10, 3)
-                vocab["%dx4096_m%d" % (n, mm)] = {"us_per_call": s / 10 / len(sel) * 1e6, "gbs": p.bytes * 10 / s / 1e9,
-                                                  "frac_of_peak": p.bytes * 10 / s / 1e9 / peaks["hbm_gbs"]}
-            del sel
+                s = p.time(iters, 3)
+                out["%dx%d_m%d" % (n, k, mm)] = {"us_per_call": s / iters / len(sel) * 1e6, "gbs": p.bytes * iters / s / 1e9,
+                                                 "frac_of_peak": p.bytes * iters / s / 1e9 / peaks["hbm_gbs"],
+                                                 "kernel": mxq.mxq_linear_plan_info(mm, n, k)["kernel"]}
+            return out
+        vocab = {}
+        for n in (32000, 128256):
+            vocab.update(m_curve(n, 4096, (1, 2, 4, 8, 16)))
+        curves = {}
+        for n, k in ((5120, 5120), (13824, 5120), (5120, 13824), (8192, 8192)):
+            curves.update(m_curve(n, k, (1, 2, 4, 8, 16) if (n, k) != (8192, 8192) else (1, 2, 4, 8)))
+        extra["m_curves"] = curves
         extra["vocab_projection"] = vocab
         # direct cast throughput (2 B read + 0.53125 B written per weight)
         w = synth.student_t_bf16((11008, 4096), 0.02, 1, device=device)

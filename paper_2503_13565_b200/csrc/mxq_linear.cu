@@ -121,10 +121,10 @@ static int kernel_ceiling() {
 // The kernel mxq_linear runs for this call.
 //   ceiling >= 0: the first of FP4, UMMA, MMA, GENERIC that is not above the ceiling and covers the call.
 //   MXQ_KERNEL_AUTO: the same order, except that measured speed decides among the kernels that cover the call
-//   (B200, layer shapes and vocabulary projections, M = 1..16): the packed-FP4 kernel wins at M = 1 everywhere;
-//   from M = 2 its activation split (16 planes per token) costs more than the FP8-operand kernel's (3 parts per
-//   token), which wins on layer-sized matrices; on matrices of more row tiles of 128 than SMs with M >= 2 the
-//   mma.sync kernel's row-range decomposition wins.
+//   (B200, layer shapes and vocabulary projections, M = 1..16): the packed-FP4 kernel wins at M = 1 everywhere and
+//   at M = 2 on matrices of more row tiles of 128 than SMs; otherwise, from M = 2, its activation split (16 planes
+//   per token) costs more than the FP8-operand kernel's (3 parts per token), which wins everywhere except where it
+//   cannot run as one CTA per SM (M = 16 on the largest vocabularies), where the mma.sync kernel does.
 // The tcgen05 kernels read the codes through a tensor map (FP4: 16-byte aligned base, which every call has; UMMA:
 // 32-byte aligned base); codes == nullptr means "suitably aligned".
 struct Choice {
@@ -140,9 +140,17 @@ static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *code
     bool try_umma = ceiling == MXQ_KERNEL_AUTO || ceiling >= MXQ_KERNEL_UMMA;
     const bool try_mma = ceiling == MXQ_KERNEL_AUTO || ceiling >= MXQ_KERNEL_MMA;
     if (ceiling == MXQ_KERNEL_AUTO && M >= 2) {
-        try_fp4 = false;
         const int64_t tiles = (N + 127) / 128;
-        if (tiles > (int64_t)sm_count() && linear_mma_plan(M, N, K, c.mma)) try_umma = false;
+        if (tiles <= (int64_t)sm_count()) {
+            try_fp4 = false;
+        } else {
+            // vocabulary-sized matrices, where a CTA per SM walks several tiles: the packed-FP4 kernel still wins at two
+            // token rows; above, the FP8-operand kernel, unless its token operand leaves no room for one CTA per SM
+            try_fp4 = M == 2;
+            if (M > 2 && !(tc && aligned32 && linear_umma_plan(M, N, K, c.umma) && c.umma.grid <= sm_count()) &&
+                linear_mma_plan(M, N, K, c.mma))
+                try_umma = false;
+        }
     }
     if (try_fp4 && tc && linear_fp4_plan(M, N, K, c.fp4)) c.kernel = MXQ_KERNEL_FP4;
     else if (try_umma && tc && aligned32 && linear_umma_plan(M, N, K, c.umma)) c.kernel = MXQ_KERNEL_UMMA;

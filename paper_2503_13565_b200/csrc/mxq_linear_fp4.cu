@@ -196,7 +196,7 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
     const uint32_t sB = sSFA + (uint32_t)ring * kFp4SfStageBytes;
     const uint32_t sSFB = sB + (uint32_t)chunk_max * (NB * 128);
     const uint32_t sRecv = sSFB + (uint32_t)chunk_max * kFp4SfStageBytes;   // [tile][split][M][rows of this rank] floats
-    const uint32_t sBar = sRecv + (uint32_t)(tiles_max * M) * kFp4RecvRows * 4u;
+    const uint32_t sBar = sRecv + (split > 1 ? (uint32_t)(tiles_max * M) * kFp4RecvRows * 4u : 0u);   // no exchange, no buffer
     // barriers: full[ring], empty[ring], done, recv, ready[chunk_max]; then the tensor-memory address and two flags
     const uint32_t full0 = sBar, empty0 = sBar + (uint32_t)ring * 8u, done_bar = sBar + (uint32_t)ring * 16u;
     const uint32_t recv_bar = done_bar + 8u, ready0 = done_bar + 16u;
@@ -214,7 +214,8 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
     const int pre = nunit < ring ? nunit : ring;
     // The SM's requests are served roughly in order, so activations asked for behind a ring full of weight copies
     // arrive late, and everything after the split waits with them.  Only the first two units are requested up
-    // front; the rest of the ring follows once the activations are in, or else at a trickle.
+    // front (1, 3 and 4 measured slower); the rest of the ring follows once the activations have been asked for, or
+    // else at a trickle.
     const int pre0 = pre < 2 ? pre : 2;
     volatile int &s_xin = *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 12);   // the activations have arrived
     // producer lane l owns rows l, l + 32, l + 64, l + 96 of a tile's scale bytes
@@ -302,11 +303,6 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
             }
         }
     }
-    constexpr int kResults = MULTI ? 16 : NB / kFp4Planes;
-    float y[kResults];   // results of this thread's row: [tile][token slot]
-#pragma unroll
-    for (int q = 0; q < kResults; ++q) y[q] = 0.f;
-
     if (warp == 0) {
         // ---- MMA warp: the loop is warp-uniform, one elected lane issues -------------------------------------------
         // descriptors as 32-bit halves: only the start-address field changes from MMA to MMA
@@ -392,6 +388,7 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                 }
                 break;
             }
+            // (requests from a second warp are served beside this lane's, but measured no gain here: 128256 x 4096 got slower)
             if (lane == 0) copy_codes(t, i, slot);
             copy_scales(t, i, slot);
             if (++i == nst) {
@@ -436,9 +433,12 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                         stage[b] = st;
                         mm[b] = tail ? rem : (rem >> 1);
                         kk[b] = st * kFp4StageK + (tail ? 0 : (rem & 1) * 128) + (lane >> 1) * 8;
-                        raw[b] = *reinterpret_cast<const uint4 *>(xbase + (int64_t)mm[b] * K + kk[b]);
+                        raw[b] = ld_ordered_u4(xbase + (int64_t)mm[b] * K + kk[b]);
                     }
                 }
+                // The activations have been asked for: weight copies requested from here on queue up behind them, so
+                // the producer may request the rest of the ring (asm volatile keeps this store after the loads).
+                if (G0 == 0 && ct == 0) st_shared_flag(sMisc + 12, 1);
                 if (G0 == 0) TR(13);
 #pragma unroll
                 for (int b = 0; b < kBatch; ++b)
@@ -447,7 +447,6 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                         const long long c0_ = clock64();
 #endif
                         inexact |= split_half_unit<NB>(raw[b], mm[b], kk[b], lane & 1, lane, sB, sSFB);
-                        if (G0 == 0 && b == 0 && ct == 0) s_xin = 1;   // lets the producer request the rest of the ring
 #ifdef MXQ_FP4_TRACE
                         const long long c1_ = clock64();
 #endif
@@ -475,33 +474,39 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
 
         // ---- epilogue: accumulator row -> registers; a token's 16 planes are 16 columns, smallest first ------------
         constexpr int MT = NB / kFp4Planes;   // token slots per tile (1, 2 or 4)
-        constexpr int TCAP = MULTI ? 16 / MT : 1;   // tiles a thread can keep results for
         if (!mbar_wait_relaxed(done_bar, 0)) {
             atomicOr(&g_fp4_status, 4u);
             s_fail = 1;
         }
         TR(5);
         tc_fence_after();
-        if (!bad) {
-            const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        // Tile by tile: this thread's row of the accumulator -> registers -> direct store (split == 1) or, for the sum over
+        // the cluster in a fixed order, a push to the row's owner.  Rank q owns rows [q*128/split, (q+1)*128/split) of every
+        // tile of the group: every CTA pushes its partial results for those rows into q's shared memory (slot = tile,
+        // sender's rank) with stores that count on q's mbarrier; q waits for all of them and adds them in a fixed
+        // order.  No CTA reads a peer's memory, and a CTA leaves only after everything addressed to it has arrived.
+        const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        const int cnt_max = (kFp4TileRows + split - 1) / split;
+        const uint32_t owner = (uint32_t)(((row + 1) * split - 1) / kFp4TileRows);
+        const int rr = row - (int)(owner * kFp4TileRows) / split;
+        const uint32_t remote = peer_saddr(sRecv, owner), remote_bar = peer_saddr(recv_bar, owner);
+        if (split > 1) cluster_wait();   // every CTA of the cluster has initialised its barriers (they arrived long ago)
+        for (int t = 0; t < ntile; ++t) {
+            float yt[MT];
 #pragma unroll
-            for (int t = 0; t < TCAP; ++t)
-                if (t < ntile) {
+            for (int m = 0; m < MT; ++m) yt[m] = 0.f;
+            if (!bad) {
 #pragma unroll
-                    for (int m = 0; m < MT; ++m) {
-                        float d[16];
-                        tc_load16(t_row + t * NB + m * 16, d);
-                        float acc = d[15];
+                for (int m = 0; m < MT; ++m) {
+                    float d[16];
+                    tc_load16(t_row + t * NB + m * 16, d);
+                    float acc = d[15];
 #pragma unroll
-                        for (int p = 14; p >= 0; --p) acc += d[p];
-                        y[t * MT + m] = acc;
-                    }
+                    for (int p = 14; p >= 0; --p) acc += d[p];
+                    yt[m] = acc;
                 }
-        } else {
-            // Scalar path for a K range whose X cannot be written as digit planes exactly (the MMA results are ignored).
-            // Results pass through the ring's shared memory, which is idle once every MMA has completed.
-            float *scratch = reinterpret_cast<float *>(gbase);
-            for (int t = 0; t < ntile; ++t) {
+            } else {
+                // Scalar path for a K range whose X cannot be rewritten exactly (the MMA results are ignored).
                 const int64_t n = n0 + (int64_t)t * kFp4TileRows + row;
                 float acc[kFp4MaxM];
 #pragma unroll
@@ -535,48 +540,30 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                     }
                 }
 #pragma unroll
-                for (int m = 0; m < MT; ++m) scratch[(t * MT + m) * kFp4TileRows + row] = acc[m];
+                for (int m = 0; m < MT; ++m) yt[m] = acc[m];
             }
+            if (t == ntile - 1) {
+                // the accumulators have been read (or are not needed): the MMA warp may give tensor memory back
+                tc_fence_before();
+                asm volatile("bar.arrive 2, 160;" ::: "memory");
+            }
+            if (s_fail) {
 #pragma unroll
-            for (int q = 0; q < kResults; ++q)
-                if (q < ntile * MT) y[q] = scratch[q * kFp4TileRows + row];   // the thread's own values, back in registers
-        }
-        tc_fence_before();
-        asm volatile("bar.arrive 2, 160;" ::: "memory");   // the accumulators have been read (or are not needed)
-        if (s_fail) {
-#pragma unroll
-            for (int q = 0; q < kResults; ++q) y[q] = __uint_as_float(0x7FC00000u);
-        }
-
-        // ---- result: direct store, or a sum over the cluster in a fixed order ----------------------------------------
-        if (split == 1) {
-#pragma unroll
-            for (int t = 0; t < TCAP; ++t)
-                if (t < ntile) {
-                    const int64_t n = n0 + (int64_t)t * kFp4TileRows + row;
-                    if (n < N)
-#pragma unroll
-                        for (int m = 0; m < MT; ++m)
-                            if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, y[t * MT + m] * kGuardUp);
-                }
-        } else {
-            // Rank q owns rows [q*128/split, (q+1)*128/split) of every tile of the group: every CTA pushes its partial
-            // results for those rows into q's shared memory (slot = tile, sender's rank) with stores that count on q's
-            // mbarrier; q waits for all of them and adds them in a fixed order.  No CTA reads a peer's memory, and a
-            // CTA leaves only after everything addressed to it has arrived.
-            const int cnt_max = (kFp4TileRows + split - 1) / split;
-            const uint32_t owner = (uint32_t)(((row + 1) * split - 1) / kFp4TileRows);
-            const int rr = row - (int)(owner * kFp4TileRows) / split;
-            const uint32_t remote = peer_saddr(sRecv, owner), remote_bar = peer_saddr(recv_bar, owner);
-            cluster_wait();   // every CTA of the cluster has initialised its barriers (they arrived long ago)
-#pragma unroll
-            for (int t = 0; t < TCAP; ++t)
-                if (t < ntile) {
+                for (int m = 0; m < MT; ++m) yt[m] = __uint_as_float(0x7FC00000u);
+            }
+            if (split == 1) {
+                const int64_t n = n0 + (int64_t)t * kFp4TileRows + row;
+                if (n < N)
 #pragma unroll
                     for (int m = 0; m < MT; ++m)
-                        if (m < M)
-                            st_async_f32(remote + (uint32_t)(((t * split + (int)rank) * M + m) * cnt_max + rr) * 4u, y[t * MT + m], remote_bar);
-                }
+                        if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, yt[m] * kGuardUp);
+            } else {
+#pragma unroll
+                for (int m = 0; m < MT; ++m)
+                    if (m < M) st_async_f32(remote + (uint32_t)(((t * split + (int)rank) * M + m) * cnt_max + rr) * 4u, yt[m], remote_bar);
+            }
+        }
+        if (split > 1) {
             if (!mbar_wait_relaxed(recv_bar, 0)) {
                 atomicOr(&g_fp4_status, 16u);
                 s_fail = 1;

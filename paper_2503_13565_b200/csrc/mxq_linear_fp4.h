@@ -34,8 +34,8 @@ struct Fp4Plan {
 
 constexpr int kFp4MaxUnitsResident = 12;   // most ring slots (16 KB of codes + 1 KB of scales each)
 
-inline uint32_t fp4_smem_bytes(int nb, int M, int tiles_max, int chunk, int ring) {
-    const uint32_t recv = (uint32_t)(tiles_max * M) * kFp4RecvRows * 4u;   // partial results pushed by the cluster's CTAs
+inline uint32_t fp4_smem_bytes(int nb, int M, int tiles_max, int chunk, int ring, int split) {
+    const uint32_t recv = split > 1 ? (uint32_t)(tiles_max * M) * kFp4RecvRows * 4u : 0u;   // partial results pushed by the cluster's CTAs
     const uint32_t b = 1024u /* alignment slack */ + (uint32_t)ring * (kFp4StageBytes + kFp4SfStageBytes) +
                        (uint32_t)chunk * ((uint32_t)nb * 128u + kFp4SfStageBytes) + recv +
                        (uint32_t)(2 * ring + 2 + chunk) * 8u /* mbarriers */ + 16u /* tensor-memory address, three flags */;
@@ -67,13 +67,13 @@ inline int fp4_ctas_per_sm(uint32_t smem_bytes, int tmem_cols) {
 //    by the CTAs of the next call (programmatic dependent launch), which start their weight stream early.
 //  - more tiles (vocabulary projections): one CTA per SM walking several tiles with a deep ring, so that the
 //    activations of a K range are split once per CTA and the pipeline never drains between tiles; the cost of a
-//    choice is the number of (tile, stage) units per CTA, ties to the larger split.
+//    choice is the number of (tile, stage) units per CTA, weighted as the code below says.
 // force_split / force_ring (> 0) override the heuristic where they are feasible.
 inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring, int force_tiles = 0) {
-    const int tcap_regs = 16 / (p.nb / kFp4Planes);  // results a thread keeps in registers: tiles * token slots <= 16
-    const int tcap_tmem = (512 - 32) / p.nb;
-    const int tcap = tcap_regs < tcap_tmem ? tcap_regs : tcap_tmem;
-    const bool layer_regime = p.tiles <= 2 * sms;
+    const int tcap = (512 - 32) / p.nb;   // tiles whose accumulators fit in tensor memory beside the scale columns
+    // (one token row: up to 2 * SMs tiles; more rows: up to SMs tiles, because every CTA of the first regime splits the
+    // token rows over all of K before its stream can run ahead: 32000 x 4096 at M = 2 ran at 2.4 TB/s there)
+    const bool layer_regime = p.tiles <= (p.nb == 16 ? 2 * sms : sms);
     long best_cost = -1;
     int best_split = 0, best_groups = 0, best_ring = 0;
     const int smax = p.ks < kFp4MaxSplit ? p.ks : kFp4MaxSplit;
@@ -92,9 +92,9 @@ inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring, int
             ring = units < 4 ? units : 4;
             if (force_ring > 0) ring = force_ring < units ? force_ring : units;
             else
-                while (ring > 2 && ctas > (long)sms * fp4_ctas_per_sm(fp4_smem_bytes(p.nb, p.M, tper, chunk, ring), tm)) --ring;
-            while (ring > 1 && fp4_smem_bytes(p.nb, p.M, tper, chunk, ring) > kFp4SmemLimit) --ring;
-            const uint32_t bytes = fp4_smem_bytes(p.nb, p.M, tper, chunk, ring);
+                while (ring > 2 && ctas > (long)sms * fp4_ctas_per_sm(fp4_smem_bytes(p.nb, p.M, tper, chunk, ring, s), tm)) --ring;
+            while (ring > 1 && fp4_smem_bytes(p.nb, p.M, tper, chunk, ring, s) > kFp4SmemLimit) --ring;
+            const uint32_t bytes = fp4_smem_bytes(p.nb, p.M, tper, chunk, ring, s);
             if (bytes > kFp4SmemLimit) continue;
             const long slots = (long)sms * fp4_ctas_per_sm(bytes, tm);
             const long waves = (ctas + slots - 1) / slots;
@@ -108,12 +108,16 @@ inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring, int
             const int units = tmax * chunk;
             ring = units < kFp4MaxUnitsResident ? units : kFp4MaxUnitsResident;
             if (force_ring > 0 && force_ring < ring) ring = force_ring;
-            while (ring > 1 && fp4_smem_bytes(p.nb, p.M, tmax, chunk, ring) > kFp4SmemLimit) --ring;
-            if (fp4_smem_bytes(p.nb, p.M, tmax, chunk, ring) > kFp4SmemLimit) continue;
+            while (ring > 1 && fp4_smem_bytes(p.nb, p.M, tmax, chunk, ring, s) > kFp4SmemLimit) --ring;
+            if (fp4_smem_bytes(p.nb, p.M, tmax, chunk, ring, s) > kFp4SmemLimit) continue;
+            // time ~ units per CTA; a K range narrower than half a row of codes costs almost twice as much per byte
+            // (the parts of a row are then fetched by three or more SMs at unrelated times: 64000 x 4096 ran at
+            // 2.6 TB/s with split 4 and at 5.0 TB/s with split 2); a ring too shallow to cover the latency costs too
             const long waves = ((long)groups * s + sms - 1) / sms;
-            cost = waves * units * 8 + chunk + (s > 1 ? 2 : 0);
+            const long by_ring = (long)ring * 16384 / 1500, rate = by_ring < 40 ? by_ring : 40;   // GB/s: bytes in flight per 1.5 us, one requester
+            cost = waves * units * 1000 / rate * (s <= 2 ? 10 : 19) + s;
         }
-        if (best_cost < 0 || cost < best_cost || cost == best_cost) {   // ties: the larger split (less of X per CTA)
+        if (best_cost < 0 || cost < best_cost || (cost == best_cost && layer_regime)) {   // layer regime: ties to the larger split (less of X per CTA)
             best_cost = cost;
             best_split = s;
             best_groups = groups;
@@ -127,7 +131,7 @@ inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring, int
     p.ring = best_ring;
     p.chunk_max = (p.ks + best_split - 1) / best_split;
     p.grid = best_groups * best_split;
-    p.smem_bytes = fp4_smem_bytes(p.nb, p.M, p.tiles_max, p.chunk_max, best_ring);
+    p.smem_bytes = fp4_smem_bytes(p.nb, p.M, p.tiles_max, p.chunk_max, best_ring, best_split);
     p.tmem_cols = fp4_tmem_cols(p.nb, p.tiles_max);
     return true;
 }

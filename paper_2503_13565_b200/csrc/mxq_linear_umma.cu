@@ -197,7 +197,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
     const uint32_t sB = sSFA + (uint32_t)ring * kUmmaSfStageBytes;
     const uint32_t sSFB = sB + (uint32_t)chunk_max * (NB * 128);
     const uint32_t sRecv = sSFB + (uint32_t)chunk_max * kUmmaSfStageBytes;   // [tile][split][M][rows of this rank] floats
-    const uint32_t sBar = sRecv + (uint32_t)(tiles_max * M) * kUmmaRecvRows * 4u;
+    const uint32_t sBar = sRecv + (split > 1 ? (uint32_t)(tiles_max * M) * kUmmaRecvRows * 4u : 0u);   // no exchange, no buffer
     // barriers: full[ring], empty[ring], done, recv, ready[pairs of stages]; then the tensor-memory address and flags
     const uint32_t full0 = sBar, empty0 = sBar + (uint32_t)ring * 8u, done_bar = sBar + (uint32_t)ring * 16u;
     const uint32_t recv_bar = done_bar + 8u, ready0 = done_bar + 16u;
@@ -293,11 +293,6 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
             }
         }
     }
-    constexpr int kResults = MULTI ? umma_results_cap(NB) : NB / kUmmaParts;
-    float y[kResults];   // results of this thread's row: [tile][token slot]
-#pragma unroll
-    for (int q = 0; q < kResults; ++q) y[q] = 0.f;
-
     if (warp == 0) {
         // ---- MMA warp: the loop is warp-uniform, one elected lane issues -------------------------------------------
         // descriptors as 32-bit halves: only the start-address field changes from MMA to MMA
@@ -450,33 +445,39 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
 
         // ---- epilogue: accumulator row -> registers; the three parts of a token are three neighbouring columns -------
         constexpr int MT = NB / kUmmaParts;         // token slots per tile (5, 10 or 16)
-        constexpr int TCAP = MULTI ? kResults / MT : 1;   // tiles a thread can keep results for
         if (!mbar_wait_relaxed(done_bar, 0)) {
             atomicOr(&g_umma_status, 4u);
             s_fail = 1;
         }
         tc_fence_after();
-        if (!bad) {
-            const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        // Tile by tile: this thread's row of the accumulator -> registers -> direct store (split == 1) or, for the sum over
+        // the cluster in a fixed order, a push to the row's owner.  Rank q owns rows [q*128/split, (q+1)*128/split) of every
+        // tile of the group: every CTA pushes its partial results for those rows into q's shared memory (slot = tile,
+        // sender's rank) with stores that count on q's mbarrier; q waits for all of them and adds them in a fixed
+        // order.  No CTA reads a peer's memory, and a CTA leaves only after everything addressed to it has arrived.
+        const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        const int cnt_max = (kUmmaTileRows + split - 1) / split;
+        const uint32_t owner = (uint32_t)(((row + 1) * split - 1) / kUmmaTileRows);
+        const int rr = row - (int)(owner * kUmmaTileRows) / split;
+        const uint32_t remote = peer_saddr(sRecv, owner), remote_bar = peer_saddr(recv_bar, owner);
+        if (split > 1) cluster_wait();   // every CTA of the cluster has initialised its barriers (they arrived long ago)
+        for (int t = 0; t < ntile; ++t) {
+            float yt[MT];
 #pragma unroll
-            for (int t = 0; t < TCAP; ++t)
-                if (t < ntile) {
+            for (int m = 0; m < MT; ++m) yt[m] = 0.f;
+            if (!bad) {
 #pragma unroll
-                    for (int c = 0; c < NB / 16; ++c) {
-                        float d[16];
-                        tc_load16(t_row + t * NB + c * 16, d);
+                for (int c = 0; c < NB / 16; ++c) {
+                    float d[16];
+                    tc_load16(t_row + t * NB + c * 16, d);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int col = c * 16 + j;
-                            if (col < MT * kUmmaParts) y[t * MT + col / kUmmaParts] += d[j];   // fixed order: parts 0, 1, 2
-                        }
+                    for (int j = 0; j < 16; ++j) {
+                        const int col = c * 16 + j;
+                        if (col < MT * kUmmaParts) yt[col / kUmmaParts] += d[j];   // fixed order: parts 0, 1, 2
                     }
                 }
-        } else {
-            // Scalar path for a K range whose X cannot be split into E5M2 parts exactly (the MMA results are ignored).
-            // Results pass through the ring's shared memory, which is idle once every MMA has completed.
-            float *scratch = reinterpret_cast<float *>(gbase);
-            for (int t = 0; t < ntile; ++t) {
+            } else {
+                // Scalar path for a K range whose X cannot be rewritten exactly (the MMA results are ignored).
                 const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row;
                 float acc[kUmmaMaxM];
 #pragma unroll
@@ -510,48 +511,30 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                     }
                 }
 #pragma unroll
-                for (int m = 0; m < MT; ++m) scratch[(t * MT + m) * kUmmaTileRows + row] = acc[m];
+                for (int m = 0; m < MT; ++m) yt[m] = acc[m];
             }
+            if (t == ntile - 1) {
+                // the accumulators have been read (or are not needed): the MMA warp may give tensor memory back
+                tc_fence_before();
+                asm volatile("bar.arrive 2, 160;" ::: "memory");
+            }
+            if (s_fail) {
 #pragma unroll
-            for (int q = 0; q < kResults; ++q)
-                if (q < ntile * MT) y[q] = scratch[q * kUmmaTileRows + row];   // the thread's own values, back in registers
-        }
-        tc_fence_before();
-        asm volatile("bar.arrive 2, 160;" ::: "memory");   // the accumulators have been read (or are not needed)
-        if (s_fail) {
-#pragma unroll
-            for (int q = 0; q < kResults; ++q) y[q] = __uint_as_float(0x7FC00000u);
-        }
-
-        // ---- result: direct store, or a sum over the cluster in a fixed order ----------------------------------------
-        if (split == 1) {
-#pragma unroll
-            for (int t = 0; t < TCAP; ++t)
-                if (t < ntile) {
-                    const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row;
-                    if (n < N)
-#pragma unroll
-                        for (int m = 0; m < MT; ++m)
-                            if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, y[t * MT + m] * kGuardUp);
-                }
-        } else {
-            // Rank q owns rows [q*128/split, (q+1)*128/split) of every tile of the group: every CTA pushes its partial
-            // results for those rows into q's shared memory (slot = tile, sender's rank) with stores that count on q's
-            // mbarrier; q waits for all of them and adds them in a fixed order.  No CTA reads a peer's memory, and a
-            // CTA leaves only after everything addressed to it has arrived.
-            const int cnt_max = (kUmmaTileRows + split - 1) / split;
-            const uint32_t owner = (uint32_t)(((row + 1) * split - 1) / kUmmaTileRows);
-            const int rr = row - (int)(owner * kUmmaTileRows) / split;
-            const uint32_t remote = peer_saddr(sRecv, owner), remote_bar = peer_saddr(recv_bar, owner);
-            cluster_wait();   // every CTA of the cluster has initialised its barriers (they arrived long ago)
-#pragma unroll
-            for (int t = 0; t < TCAP; ++t)
-                if (t < ntile) {
+                for (int m = 0; m < MT; ++m) yt[m] = __uint_as_float(0x7FC00000u);
+            }
+            if (split == 1) {
+                const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row;
+                if (n < N)
 #pragma unroll
                     for (int m = 0; m < MT; ++m)
-                        if (m < M)
-                            st_async_f32(remote + (uint32_t)(((t * split + (int)rank) * M + m) * cnt_max + rr) * 4u, y[t * MT + m], remote_bar);
-                }
+                        if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, yt[m] * kGuardUp);
+            } else {
+#pragma unroll
+                for (int m = 0; m < MT; ++m)
+                    if (m < M) st_async_f32(remote + (uint32_t)(((t * split + (int)rank) * M + m) * cnt_max + rr) * 4u, yt[m], remote_bar);
+            }
+        }
+        if (split > 1) {
             if (!mbar_wait_relaxed(recv_bar, 0)) {
                 atomicOr(&g_umma_status, 16u);
                 s_fail = 1;

@@ -33,8 +33,6 @@ MXQ_UMMA_HD inline size_t umma_ws_flags_bytes(int ks) { return (((size_t)ks * 4u
 MXQ_UMMA_HD inline size_t umma_ws_bytes(int nb, int ks) {
     return umma_ws_flags_bytes(ks) + (size_t)ks * kUmmaSfStageBytes + (size_t)ks * (size_t)nb * 128u;
 }
-// results (tile x token slot) an epilogue thread keeps in registers when its CTA owns several tiles
-MXQ_UMMA_HD constexpr int umma_results_cap(int nb) { return nb == 16 ? 16 : 32; }
 inline int umma_nb(int M) { return 3 * M <= 16 ? 16 : (3 * M <= 32 ? 32 : 48); }
 
 struct UmmaPlan {
@@ -53,8 +51,8 @@ struct UmmaPlan {
     int64_t N, K;
 };
 
-inline uint32_t umma_smem_bytes(int nb, int M, int tiles_max, int chunk, int ring) {
-    const uint32_t recv = (uint32_t)(tiles_max * M) * kUmmaRecvRows * 4u;   // partial results pushed by the cluster's CTAs
+inline uint32_t umma_smem_bytes(int nb, int M, int tiles_max, int chunk, int ring, int split) {
+    const uint32_t recv = split > 1 ? (uint32_t)(tiles_max * M) * kUmmaRecvRows * 4u : 0u;   // partial results pushed by the cluster's CTAs
     const uint32_t b = 1024u /* alignment slack */ + (uint32_t)ring * (kUmmaStageBytes + kUmmaSfStageBytes) +
                        (uint32_t)chunk * ((uint32_t)nb * 128u + kUmmaSfStageBytes) + recv +
                        (uint32_t)(2 * ring + 2 + (chunk + 1) / 2) * 8u /* mbarriers */ + 16u /* tensor-memory address, flags */;
@@ -75,14 +73,13 @@ inline int umma_ctas_per_sm(uint32_t smem_bytes, int tmem_cols) {
 }
 
 // Chooses split, groups and ring for p.{M, nb, ks, tiles}; false if nothing fits.  Same two regimes as the packed-FP4
-// kernel: up to 2 * SMs tiles -> one tile per CTA, every CTA resident at once, about two CTAs per SM (ties to the
+// kernel: up to one tile per SM -> one tile per CTA, every CTA resident at once, about two CTAs per SM (ties to the
 // larger split: splitting the activations is this kernel's main cost from M = 4 on, and it shrinks with the K range);
 // more tiles -> one CTA per SM walking several tiles.
 // force_split / force_ring / force_tiles (> 0) override the heuristic where they are feasible.
 inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, int force_tiles = 0) {
-    const int slots_per_tile = p.nb / kUmmaParts;        // 5, 10 or 16 tokens fit in a tile's columns
-    const int tcap = umma_results_cap(p.nb) / slots_per_tile;   // tiles whose results fit in a thread's registers: 3, 3, 2
-    const bool layer_regime = p.tiles <= 2 * sms;
+    const int tcap = (512 - 16) / p.nb;   // tiles whose accumulators fit in tensor memory beside the scale columns
+    const bool layer_regime = p.tiles <= sms;
     // Tiles per CTA in the layer regime: one, except for the widest token operand on matrices of many tiles, where
     // the operand's K range of a CTA (6.5 KB per stage) leaves too little shared memory for weights unless two
     // tiles share it (11008 x 4096 at M = 16: 21.5 -> 16 us).
@@ -106,9 +103,9 @@ inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, i
             if (tper == 1 && ring > 8) ring = 8;
             if (force_ring > 0) ring = force_ring < units ? force_ring : units;
             else
-                while (ring > 2 && ctas > (long)sms * umma_ctas_per_sm(umma_smem_bytes(p.nb, p.M, tmax, chunk, ring), tm)) --ring;
-            while (ring > 1 && umma_smem_bytes(p.nb, p.M, tmax, chunk, ring) > kUmmaSmemLimit) --ring;
-            const uint32_t bytes = umma_smem_bytes(p.nb, p.M, tmax, chunk, ring);
+                while (ring > 2 && ctas > (long)sms * umma_ctas_per_sm(umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s), tm)) --ring;
+            while (ring > 1 && umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s) > kUmmaSmemLimit) --ring;
+            const uint32_t bytes = umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s);
             if (bytes > kUmmaSmemLimit) continue;
             const long slots = (long)sms * umma_ctas_per_sm(bytes, tm);
             const long waves = (ctas + slots - 1) / slots;
@@ -122,12 +119,16 @@ inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, i
             const int units = tmax * chunk;
             ring = units < kUmmaMaxUnitsResident ? units : kUmmaMaxUnitsResident;
             if (force_ring > 0 && force_ring < ring) ring = force_ring;
-            while (ring > 1 && umma_smem_bytes(p.nb, p.M, tmax, chunk, ring) > kUmmaSmemLimit) --ring;
-            if (umma_smem_bytes(p.nb, p.M, tmax, chunk, ring) > kUmmaSmemLimit) continue;
+            while (ring > 1 && umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s) > kUmmaSmemLimit) --ring;
+            if (umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s) > kUmmaSmemLimit) continue;
+            // Time ~ units per CTA / the rate its stream reaches: two requesters at 25 GB/s each, the ring's bytes in
+            // flight (8 KB of packed codes per slot) per 1.5 us of latency, the SM's share of the memory bandwidth;
+            // nearly doubled for K ranges under half a row of codes (see the packed-FP4 kernel).
             const long waves = ((long)groups * s + sms - 1) / sms;
-            cost = waves * units * 8 + chunk + (s > 1 ? 2 : 0);
+            const long by_ring = (long)ring * 8192 / 1500, rate = by_ring < 41 ? by_ring : 41;   // GB/s
+            cost = waves * units * 1000 / rate * (s <= 2 ? 10 : 19) + s;
         }
-        if (best_cost < 0 || cost <= best_cost) {   // ties: the larger split
+        if (best_cost < 0 || cost < best_cost || (cost == best_cost && layer_regime)) {   // layer regime: ties to the larger split
             best_cost = cost;
             best_split = s;
             best_groups = groups;
@@ -141,7 +142,7 @@ inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, i
     p.ring = best_ring;
     p.chunk_max = (p.ks + best_split - 1) / best_split;
     p.grid = best_groups * best_split;
-    p.smem_bytes = umma_smem_bytes(p.nb, p.M, p.tiles_max, p.chunk_max, best_ring);
+    p.smem_bytes = umma_smem_bytes(p.nb, p.M, p.tiles_max, p.chunk_max, best_ring, best_split);
     p.tmem_cols = umma_tmem_cols(p.nb, p.tiles_max);
     return true;
 }

@@ -66,6 +66,15 @@ __device__ __forceinline__ void tma_load_codes(uint32_t dst, const CUtensorMap *
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
+// a 16-byte global load and a 32-bit shared store that the compiler keeps in program order with each other
+__device__ __forceinline__ uint4 ld_ordered_u4(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_shared_flag(uint32_t saddr, int v) {
+    asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(saddr), "r"(v) : "memory");
+}
 // untiled bulk copy global -> shared memory (both 16-byte aligned, size a multiple of 16), counted on an mbarrier
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),

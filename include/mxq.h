@@ -148,8 +148,8 @@ int mxq_linear_device_status(uint32_t *status_host);
  *   Y       [M][N] row-major, float (MXQ_F32) or BF16 rounded to nearest even (MXQ_BF16)
  *   workspace / workspace_bytes  optional scratch, see mxq_linear_workspace_bytes (NULL / 0 allowed)
  * Products are formed exactly and accumulated in FP32; the block scale is applied to
- * 32-long partial sums (Eq. 2).  The summation order is fixed for a given shape, so
- * results are bit-reproducible run to run.  A row containing a 0xFF scale yields NaN. */
+ * 32-long partial sums (Eq. 2).  The summation order is fixed for a given shape, kernel selection and
+ * presence of a workspace, so results are bit-reproducible run to run.  A row containing a 0xFF scale yields NaN. */
 int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
                void *Y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream);
 

@@ -26,7 +26,8 @@ cudaError_t linear_mma_launch(const LinearPlan &plan, const void *X, const uint8
 struct UmmaPlan;
 // tcgen05 path of mxq_linear (mxq_linear_umma.cu): false if the shape is not covered
 bool linear_umma_available();
-bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &plan);
+// with_workspace: plan for a token operand split ahead of the weight kernel (from 3 token rows on)
+bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &plan, bool with_workspace);
 // workspace: optional; with linear_umma_workspace_bytes(M, K) bytes (0: not used for this M) the token operand is split
 // once per call by a kernel of its own instead of by every CTA of the weight kernel
 size_t linear_umma_workspace_bytes(int M, int64_t K);

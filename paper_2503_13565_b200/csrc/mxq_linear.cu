@@ -133,7 +133,7 @@ struct Choice {
     UmmaPlan umma;
     LinearPlan mma;
 };
-static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *codes, Choice &c) {
+static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *codes, bool with_workspace, Choice &c) {
     const bool tc = linear_umma_available();
     const bool aligned32 = !codes || (reinterpret_cast<uintptr_t>(codes) & 31u) == 0;
     bool try_fp4 = ceiling == MXQ_KERNEL_AUTO || ceiling >= MXQ_KERNEL_FP4;
@@ -147,13 +147,13 @@ static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *code
             // vocabulary-sized matrices, where a CTA per SM walks several tiles: the packed-FP4 kernel still wins at two
             // token rows; above, the FP8-operand kernel, unless its token operand leaves no room for one CTA per SM
             try_fp4 = M == 2;
-            if (M > 2 && !(tc && aligned32 && linear_umma_plan(M, N, K, c.umma) && c.umma.grid <= sm_count()) &&
+            if (M > 2 && !(tc && aligned32 && linear_umma_plan(M, N, K, c.umma, with_workspace) && c.umma.grid <= sm_count()) &&
                 linear_mma_plan(M, N, K, c.mma))
                 try_umma = false;
         }
     }
     if (try_fp4 && tc && linear_fp4_plan(M, N, K, c.fp4)) c.kernel = MXQ_KERNEL_FP4;
-    else if (try_umma && tc && aligned32 && linear_umma_plan(M, N, K, c.umma)) c.kernel = MXQ_KERNEL_UMMA;
+    else if (try_umma && tc && aligned32 && linear_umma_plan(M, N, K, c.umma, with_workspace)) c.kernel = MXQ_KERNEL_UMMA;
     else if (try_mma && linear_mma_plan(M, N, K, c.mma)) c.kernel = MXQ_KERNEL_MMA;
     else c.kernel = MXQ_KERNEL_GENERIC;
 }
@@ -184,11 +184,11 @@ int mxq_linear_plan_info(int kernel, int M, int64_t N, int64_t K, int32_t *info)
     for (int i = 0; i < 12; ++i) info[i] = 0;
     mxq::Choice c;
     if (kernel == MXQ_KERNEL_AUTO) {
-        mxq::choose(mxq::kernel_ceiling(), M, N, K, nullptr, c);
+        mxq::choose(mxq::kernel_ceiling(), M, N, K, nullptr, true, c);
     } else {
         c.kernel = kernel;
         const bool ok = kernel == MXQ_KERNEL_FP4    ? mxq::linear_fp4_plan(M, N, K, c.fp4)
-                        : kernel == MXQ_KERNEL_UMMA ? mxq::linear_umma_plan(M, N, K, c.umma)
+                        : kernel == MXQ_KERNEL_UMMA ? mxq::linear_umma_plan(M, N, K, c.umma, true)
                         : kernel == MXQ_KERNEL_MMA  ? mxq::linear_mma_plan(M, N, K, c.mma)
                                                     : true;
         if (!ok) {
@@ -236,7 +236,9 @@ int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *s
         return MXQ_ERR_ALIGN;
     cudaStream_t st = (cudaStream_t)stream;
     mxq::Choice c;
-    mxq::choose(mxq::kernel_ceiling(), M, N, K, codes, c);
+    const bool with_workspace = workspace && workspace_bytes >= mxq::linear_umma_workspace_bytes(M, K) &&
+                                (reinterpret_cast<uintptr_t>(workspace) & 15u) == 0;
+    mxq::choose(mxq::kernel_ceiling(), M, N, K, codes, with_workspace, c);
     if (c.kernel != MXQ_KERNEL_GENERIC) {
         const cudaError_t e =
             c.kernel == MXQ_KERNEL_FP4    ? mxq::linear_fp4_launch(c.fp4, X_bf16, codes, scales, Y, y_dtype, st)

@@ -167,12 +167,13 @@ cudaError_t launch_split(const __nv_bfloat16 *X, int M, int64_t K, int ks, uint8
 // the codes, cp.async of the scale bytes, barrier set-up); warps 2..5 split the activations stage by stage and,
 // at the end, read the accumulator (one row per thread), exchange partial results and store.
 // MULTI: whether a CTA may own more than one tile (false: exactly one, and the per-tile loops fold away).
-template <int NB, bool MULTI>
+template <int NB, bool MULTI, bool BRING>
 __global__ void __launch_bounds__(kUmmaThreads)
 linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 *__restrict__ X, int M,
                   const uint8_t *__restrict__ codes, const uint8_t *__restrict__ scales, int64_t N, int64_t K,
                   void *__restrict__ Y, int y_dtype, int split, int ring, int ks, int chunk_max, int tmem_cols, int groups,
                   int tiles, int tiles_max, const uint8_t *__restrict__ presplit) {
+    constexpr bool bring = BRING;   // the token operand is fetched stage by stage into the ring slots (needs presplit, one tile)
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");   // needed by the first copy, 1 us from now
@@ -195,8 +196,11 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
     const uint32_t sA = base;
     const uint32_t sSFA = sA + (uint32_t)ring * kUmmaStageBytes;
     const uint32_t sB = sSFA + (uint32_t)ring * kUmmaSfStageBytes;
-    const uint32_t sSFB = sB + (uint32_t)chunk_max * (NB * 128);
-    const uint32_t sRecv = sSFB + (uint32_t)chunk_max * kUmmaSfStageBytes;   // [tile][split][M][rows of this rank] floats
+    // the token operand: one image and one scale atom per stage of the CTA's K range, or (bring: the operand was split
+    // ahead of this kernel and the CTA owns one tile) per ring slot, fetched with the slot's weights
+    const uint32_t nbslot = bring ? (uint32_t)ring : (uint32_t)chunk_max;
+    const uint32_t sSFB = sB + nbslot * (NB * 128);
+    const uint32_t sRecv = sSFB + nbslot * kUmmaSfStageBytes;   // [tile][split][M][rows of this rank] floats
     const uint32_t sBar = sRecv + (split > 1 ? (uint32_t)(tiles_max * M) * kUmmaRecvRows * 4u : 0u);   // no exchange, no buffer
     // barriers: full[ring], empty[ring], done, recv, ready[pairs of stages]; then the tensor-memory address and flags
     const uint32_t full0 = sBar, empty0 = sBar + (uint32_t)ring * 8u, done_bar = sBar + (uint32_t)ring * 16u;
@@ -238,11 +242,18 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
         mbar_expect_tx(full0 + slot * 8, kUmmaStageTxBytes);
         tma_load_codes(sA + slot * kUmmaStageBytes, &tmap, (s_begin + i) * kUmmaStageK, (int)n0 + t * kUmmaTileRows, full0 + slot * 8);
     };
+    const uint8_t *ws_sf = presplit ? presplit + umma_ws_flags_bytes(ks) : nullptr;
+    const uint8_t *ws_b = presplit ? ws_sf + (size_t)ks * kUmmaSfStageBytes : nullptr;
+    auto copy_tokens = [&](int i, uint32_t slot) {     // one lane; bring only: stage i of the token operand into ring slot `slot`
+        mbar_expect_tx(full0 + slot * 8, NB * 128u + kUmmaSfStageBytes);
+        bulk_load(sB + slot * (NB * 128u), ws_b + (size_t)(s_begin + i) * (NB * 128u), NB * 128u, full0 + slot * 8);
+        bulk_load(sSFB + slot * kUmmaSfStageBytes, ws_sf + (size_t)(s_begin + i) * kUmmaSfStageBytes, kUmmaSfStageBytes, full0 + slot * 8);
+    };
     if (warp == 1) {
         for (int b = lane; b < 2 * ring + 2 + npair; b += 32) {
             // full: the TMA lane + 32 producer lanes; empty, done, recv: 1; ready (one per 256 k): one arrival per token
             // (with the token operand split ahead of this kernel: the one thread that requests the copies)
-            const uint32_t count = b < ring ? kFullArrivals : (b < 2 * ring + 2 || presplit ? 1u : (uint32_t)M);
+            const uint32_t count = b < ring ? kFullArrivals + (bring ? 1u : 0u) : (b < 2 * ring + 2 || presplit ? 1u : (uint32_t)M);
             mbar_init(sBar + (uint32_t)b * 8u, count);
         }
         if (lane == 31) {
@@ -272,7 +283,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
     // Only the activation warps read what the previous kernel wrote (X) and write what the next one reads (Y), so
     // only they wait for it; they do so at once, and join the CTA-wide barrier (initialised mbarriers, tensor-memory
     // address) after that wait.
-    if (warp >= 2) {
+    if (warp >= 2 || (warp == 1 && bring)) {   // (bring: the producer reads what the split kernel wrote)
         pdl_wait();
     }
     if (split > 1) cluster_arrive();   // "my barriers exist"; the matching wait is just before the first push to a peer
@@ -283,9 +294,10 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
     if (warp == 1) {
         for (int u = 0, t = 0, i = 0; u < pre; ++u) {
             if (u >= pre0) {
-                for (int spin = 0; spin < 3 && !s_xin; ++spin) __nanosleep(100);
+                for (int spin = 0; spin < 3 && !s_xin && !bring; ++spin) __nanosleep(100);
                 if (lane == 0) copy_codes(t, i, (uint32_t)u);
             }
+            if (bring && lane == 0) copy_tokens(i, (uint32_t)u);
             copy_scales(t, i, (uint32_t)u);
             if (++i == nst) {
                 i = 0;
@@ -311,7 +323,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
           for (int i = 0; i < nst; ++i) {
             // the unit's weights and scales have landed and (first tile only; the others find it done) the stage's
             // share of the activations has been split
-            if ((t == 0 && !mbar_wait_relaxed(ready0 + (uint32_t)(i >> 1) * 8u, 0)) || !mbar_wait_relaxed(full0 + slot * 8, phase)) {
+            if ((t == 0 && !bring && !mbar_wait_relaxed(ready0 + (uint32_t)(i >> 1) * 8u, 0)) || !mbar_wait_relaxed(full0 + slot * 8, phase)) {
                 if (lane == 0) {
                     atomicOr(&g_umma_status, 1u);
                     s_fail = 1;
@@ -322,6 +334,10 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
             tc_fence_after();
             const uint32_t a_lo = a_lo0 + slot * (kUmmaStageBytes >> 4);
             const uint32_t sa_lo = s_lo0 + slot * (kUmmaSfStageBytes >> 4);
+            if (bring) {   // the token operand's stage sits in the ring slot
+                b_lo = b_lo0 + slot * ((NB * 128) >> 4);
+                sb_lo = sb_lo0 + slot * (kUmmaSfStageBytes >> 4);
+            }
             const uint32_t t_sf = t_sf0 + par * 8u;   // alternating between consecutive units
             par ^= 1u;
             if (elect_one()) {
@@ -368,7 +384,10 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                 }
                 break;
             }
-            if (lane == 0) copy_codes(t, i, slot);
+            if (lane == 0) {
+                copy_codes(t, i, slot);
+                if (bring) copy_tokens(i, slot);
+            }
             copy_scales(t, i, slot);
             if (++i == nst) {
                 i = 0;
@@ -387,9 +406,9 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
         bool inexact = false;
         if (presplit) {
             // The token operand was split by split_tokens_kernel: fetch this CTA's stages, two at a time, each pair
-            // completing the "ready" barrier the MMA warp waits on; the flags say whether every block split exactly.
-            const uint8_t *ws_sf = presplit + umma_ws_flags_bytes(ks), *ws_b = ws_sf + (size_t)ks * kUmmaSfStageBytes;
-            if (ct == 0) {
+            // completing the "ready" barrier the MMA warp waits on (unless the producer fetches them stage by stage into
+            // the ring); the flags say whether every block split exactly.
+            if (ct == 0 && !bring) {
                 for (int p = 0; p < npair; ++p) {
                     const uint32_t n2 = (uint32_t)min(2, nst - 2 * p), bar = ready0 + (uint32_t)p * 8u;
                     mbar_expect_tx(bar, n2 * (NB * 128u + kUmmaSfStageBytes));
@@ -573,19 +592,19 @@ int env_int(const char *name) {
     return e ? std::atoi(e) : 0;
 }
 
-template <int NB, bool MULTI>
+template <int NB, bool MULTI, bool BRING>
 cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X, const uint8_t *codes,
                        const uint8_t *scales, void *Y, int y_dtype, const uint8_t *presplit, cudaStream_t stream) {
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI, BRING>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kUmmaSmemLimit);
         if (e != cudaSuccess) return e;
         // all of the SM's L1/shared array as shared memory: how many CTAs (of this and of the next kernel) fit on an
         // SM is what decides how early the next kernel's weight stream can start
-        e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI, BRING>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -610,26 +629,35 @@ cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    return cudaLaunchKernelEx(&cfg, linear_umma_kernel<NB, MULTI>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
+    return cudaLaunchKernelEx(&cfg, linear_umma_kernel<NB, MULTI, BRING>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
                               Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols, p.groups, p.tiles, p.tiles_max, presplit);
 }
 
 }  // namespace
 
-bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p) {
+// token rows from which the token operand is split ahead of the weight kernel when a workspace is there
+static int presplit_min_m() {
+    static const int v = env_int("MXQ_UMMA_NO_PRESPLIT") != 0 ? kUmmaMaxM + 1
+                         : (env_int("MXQ_UMMA_PRESPLIT_MIN_M") > 0 ? env_int("MXQ_UMMA_PRESPLIT_MIN_M") : kUmmaPresplitMinM);
+    return v;
+}
+
+bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p, bool with_workspace) {
     if (M < 1 || M > kUmmaMaxM || N < 1 || K < 128 || (K % 128) != 0) return false;
     if (K > 0x3FFFFFFF || N > 0x7FFFFFFF) return false;
+    p.presplit = with_workspace && M >= presplit_min_m() ? 1 : 0;
     p.M = M;
     p.N = N;
     p.K = K;
     p.nb = umma_nb(M);
     p.ks = (int)(K / kUmmaStageK);
     p.tiles = (int)((N + kUmmaTileRows - 1) / kUmmaTileRows);
-    return umma_layout(p, sm_count(), env_int("MXQ_UMMA_SPLIT"), env_int("MXQ_UMMA_RING"), env_int("MXQ_UMMA_TILES"));
+    return umma_layout(p, sm_count(), env_int("MXQ_UMMA_SPLIT"), env_int("MXQ_UMMA_RING"), env_int("MXQ_UMMA_TILES"),
+                       std::getenv("MXQ_UMMA_BRING") ? env_int("MXQ_UMMA_BRING") : -1);
 }
 
 size_t linear_umma_workspace_bytes(int M, int64_t K) {
-    if (M < kUmmaPresplitMinM || M > kUmmaMaxM || K < 128 || (K % 128) != 0 || K > 0x3FFFFFFF) return 0;
+    if (M < presplit_min_m() || M > kUmmaMaxM || K < 128 || (K % 128) != 0 || K > 0x3FFFFFFF) return 0;
     return umma_ws_bytes(umma_nb(M), (int)(K / kUmmaStageK));
 }
 
@@ -638,12 +666,15 @@ cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *
     CUtensorMap map;
     if (!codes_tensor_map(codes, p.N, p.K, /*expand_fp4=*/true, &map)) return cudaErrorNotSupported;
     // a workspace that is large enough (and aligned for bulk copies) lets the token operand be split once per call
-    static const bool no_presplit = env_int("MXQ_UMMA_NO_PRESPLIT") != 0;
-    static const int min_m = env_int("MXQ_UMMA_PRESPLIT_MIN_M") > 0 ? env_int("MXQ_UMMA_PRESPLIT_MIN_M") : kUmmaPresplitMinM;
     const size_t need = umma_ws_bytes(p.nb, p.ks);
     uint8_t *ws = nullptr;
-    if (!no_presplit && p.M >= min_m && workspace && workspace_bytes >= need && (reinterpret_cast<uintptr_t>(workspace) & 15u) == 0)
+    if (p.presplit && workspace && workspace_bytes >= need && (reinterpret_cast<uintptr_t>(workspace) & 15u) == 0)
         ws = static_cast<uint8_t *>(workspace);
+    if (p.presplit && !ws) {   // planned for a workspace that is not there: plan again without
+        UmmaPlan q;
+        if (!linear_umma_plan(p.M, p.N, p.K, q, false)) return cudaErrorNotSupported;
+        return linear_umma_launch(q, X, codes, scales, Y, y_dtype, nullptr, 0, stream);
+    }
     if (ws) {
         const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(X);
         const cudaError_t e = p.nb == 16   ? launch_split<16>(x, p.M, p.K, p.ks, ws, stream)
@@ -651,16 +682,20 @@ cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *
                                            : launch_split<48>(x, p.M, p.K, p.ks, ws, stream);
         if (e != cudaSuccess) return e;
     }
+    const bool bring = ws && p.bring && p.tiles_max == 1;
     switch (p.nb) {
         case 16:
-            return p.tiles_max > 1 ? launch_umma<16, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
-                                   : launch_umma<16, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream);
+            return p.tiles_max > 1 ? launch_umma<16, true, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
+                   : bring         ? launch_umma<16, false, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
+                                   : launch_umma<16, false, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream);
         case 32:
-            return p.tiles_max > 1 ? launch_umma<32, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
-                                   : launch_umma<32, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream);
+            return p.tiles_max > 1 ? launch_umma<32, true, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
+                   : bring         ? launch_umma<32, false, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
+                                   : launch_umma<32, false, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream);
         default:
-            return p.tiles_max > 1 ? launch_umma<48, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
-                                   : launch_umma<48, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream);
+            return p.tiles_max > 1 ? launch_umma<48, true, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
+                   : bring         ? launch_umma<48, false, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
+                                   : launch_umma<48, false, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream);
     }
 }
 

@@ -47,14 +47,16 @@ struct UmmaPlan {
     int chunk_max;   // most stages any CTA owns = ceil(ks / split)
     int grid;        // groups * split
     int tmem_cols;   // tensor-memory columns allocated per CTA
+    int presplit;    // planned for a token operand split ahead of the weight kernel (needs the workspace)
+    int bring;       // ... and fetched stage by stage into the ring slots (one tile per CTA) instead of whole K ranges
     uint32_t smem_bytes;
     int64_t N, K;
 };
 
-inline uint32_t umma_smem_bytes(int nb, int M, int tiles_max, int chunk, int ring, int split) {
+inline uint32_t umma_smem_bytes(int nb, int M, int tiles_max, int chunk, int ring, int split, int bring = 0) {
     const uint32_t recv = split > 1 ? (uint32_t)(tiles_max * M) * kUmmaRecvRows * 4u : 0u;   // partial results pushed by the cluster's CTAs
     const uint32_t b = 1024u /* alignment slack */ + (uint32_t)ring * (kUmmaStageBytes + kUmmaSfStageBytes) +
-                       (uint32_t)chunk * ((uint32_t)nb * 128u + kUmmaSfStageBytes) + recv +
+                       (uint32_t)(bring ? ring : chunk) * ((uint32_t)nb * 128u + kUmmaSfStageBytes) + recv +
                        (uint32_t)(2 * ring + 2 + (chunk + 1) / 2) * 8u /* mbarriers */ + 16u /* tensor-memory address, flags */;
     return (b + 15u) & ~15u;
 }
@@ -77,19 +79,22 @@ inline int umma_ctas_per_sm(uint32_t smem_bytes, int tmem_cols) {
 // larger split: splitting the activations is this kernel's main cost from M = 4 on, and it shrinks with the K range);
 // more tiles -> one CTA per SM walking several tiles.
 // force_split / force_ring / force_tiles (> 0) override the heuristic where they are feasible.
-inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, int force_tiles = 0) {
+inline bool umma_layout_one(UmmaPlan &p, int sms, int force_split, int force_ring, int force_tiles, bool allow_bring) {
+    // p.presplit (set by the caller): the token operand comes ready-made from the workspace; a CTA of one tile may then
+    // fetch it stage by stage with the weights (p.bring), so that its K range does not eat the ring's shared memory
     const int tcap = (512 - 16) / p.nb;   // tiles whose accumulators fit in tensor memory beside the scale columns
     const bool layer_regime = p.tiles <= sms;
     // Tiles per CTA in the layer regime: one, except for the widest token operand on matrices of many tiles, where
     // the operand's K range of a CTA (6.5 KB per stage) leaves too little shared memory for weights unless two
     // tiles share it (11008 x 4096 at M = 16: 21.5 -> 16 us).
-    int tper = p.nb == 48 && 2 * p.tiles >= sms ? 2 : 1;
+    int tper = p.nb == 48 && 2 * p.tiles >= sms && !allow_bring ? 2 : 1;
     if (force_tiles > 0) tper = force_tiles < tcap ? force_tiles : tcap;
     long best_cost = -1;
     int best_split = 0, best_groups = 0, best_ring = 0;
     const int smax = p.ks < kUmmaMaxSplit ? p.ks : kUmmaMaxSplit;
     for (int s = 1; s <= smax; ++s) {
         if (force_split > 0 && s != (force_split < smax ? force_split : smax)) continue;
+        if (force_split <= 0 && s == 7) continue;   // clusters of 7 measured up to 1.5 times slower than of 6 or 8 (5120 x 5120, 5120 x 13824)
         const int chunk = (p.ks + s - 1) / s;
         int groups, ring;
         long cost;
@@ -99,13 +104,14 @@ inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, i
             const long ctas = (long)groups * s;
             const int tm = umma_tmem_cols(p.nb, tmax);
             const int units = tmax * chunk;
+            const int br = allow_bring && p.presplit && tmax == 1 ? 1 : 0;
             ring = units < kUmmaMaxUnitsResident ? units : kUmmaMaxUnitsResident;
             if (tper == 1 && ring > 8) ring = 8;
             if (force_ring > 0) ring = force_ring < units ? force_ring : units;
             else
-                while (ring > 2 && ctas > (long)sms * umma_ctas_per_sm(umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s), tm)) --ring;
-            while (ring > 1 && umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s) > kUmmaSmemLimit) --ring;
-            const uint32_t bytes = umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s);
+                while (ring > 2 && ctas > (long)sms * umma_ctas_per_sm(umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s, br), tm)) --ring;
+            while (ring > 1 && umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s, br) > kUmmaSmemLimit) --ring;
+            const uint32_t bytes = umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s, br);
             if (bytes > kUmmaSmemLimit) continue;
             const long slots = (long)sms * umma_ctas_per_sm(bytes, tm);
             const long waves = (ctas + slots - 1) / slots;
@@ -142,9 +148,26 @@ inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, i
     p.ring = best_ring;
     p.chunk_max = (p.ks + best_split - 1) / best_split;
     p.grid = best_groups * best_split;
-    p.smem_bytes = umma_smem_bytes(p.nb, p.M, p.tiles_max, p.chunk_max, best_ring, best_split);
+    p.bring = allow_bring && p.presplit && layer_regime && p.tiles_max == 1 ? 1 : 0;
+    p.smem_bytes = umma_smem_bytes(p.nb, p.M, p.tiles_max, p.chunk_max, best_ring, best_split, p.bring);
     p.tmem_cols = umma_tmem_cols(p.nb, p.tiles_max);
     return true;
+}
+
+// With the token operand split ahead of the kernel there are two ways to hold it.  Whole K range resident: measured
+// faster (by 0.5 us on the 7B layer shapes at M = 8) when that still leaves three ring slots and the plan fills at least
+// 5/6 of the SMs.  Stage by stage through the ring otherwise (13824 x 5120 at M = 8: 22 -> 15 us).
+inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, int force_tiles = 0, int force_bring = -1) {
+    if (!p.presplit || force_bring == 0) return umma_layout_one(p, sms, force_split, force_ring, force_tiles, false);
+    UmmaPlan r = p;
+    const bool have_r = force_bring < 0 && umma_layout_one(r, sms, force_split, force_ring, force_tiles, false);
+    if (have_r && (r.tiles_max > 1 ? p.tiles > sms : (r.ring >= 3 && 6 * r.grid >= 5 * sms))) {   // (several tiles per CTA: the vocabulary regime only)
+        p = r;
+        return true;
+    }
+    if (umma_layout_one(p, sms, force_split, force_ring, force_tiles, true)) return true;
+    if (have_r) p = r;
+    return have_r;
 }
 
 }  // namespace mxq

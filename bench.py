@@ -355,6 +355,36 @@ def run_ours(args):
             curves.update(m_curve(n, k, (1, 2, 4, 8, 16) if (n, k) != (8192, 8192) else (1, 2, 4, 8)))
         extra["m_curves"] = curves
         extra["vocab_projection"] = vocab
+        # vocabulary projection + greedy verification: one fused launch against mxq_linear followed by mxq_greedy_accept
+        fused = {}
+        for v_, r_ in ((32000, 1), (32000, 9), (128256, 1), (128256, 9)):
+            copies = 3 if v_ == 32000 else 2
+            gen = torch.Generator(device=device).manual_seed(v_ + r_)
+            mats_ = [(torch.randint(0, 256, (v_, 2048), dtype=torch.uint8, device=device, generator=gen),
+                      torch.randint(110, 126, (v_, 128), dtype=torch.uint8, device=device, generator=gen)) for _ in range(copies)]
+            x_ = synth.normal_bf16((r_, 4096), 1.0, 5, device)
+            t_ = r_ - 1
+            draft_ = torch.zeros(max(t_, 1), dtype=torch.int32, device=device)
+            wsf = mxq.new_workspace(mxq.mxq_lm_head_accept_workspace_bytes(r_, v_, 4096), device)
+            wsl = mxq.new_workspace(max(mxq.mxq_linear_workspace_bytes(r_, v_, 4096), 16), device)
+            wsa = mxq.new_workspace(mxq.mxq_accept_workspace_bytes(1, r_, v_), device)
+            lg_ = torch.empty((1, r_, v_), dtype=torch.float32, device=device)
+
+            def fused_pass():
+                for c_, s_ in mats_:
+                    mxq.mxq_lm_head_accept(x_, c_, s_, draft_[:t_] if t_ else None, workspace=wsf)
+
+            draft2d = draft_[:max(t_, 1)].view(1, -1)   # (R = 1: a one-token draft stands in; the work is the same)
+
+            def unfused_pass():
+                for c_, s_ in mats_:
+                    mxq.mxq_linear(x_, c_, s_, out=lg_[0], workspace=wsl)
+                    mxq.mxq_greedy_accept(lg_, draft2d, workspace=wsa)
+            tf = time_graph(fused_pass, 10) / copies
+            tu = time_graph(unfused_pass, 10) / copies
+            fused["%dx4096_r%d" % (v_, r_)] = {"fused_us": tf * 1e6, "linear_then_accept_us": tu * 1e6}
+            del mats_
+        extra["lm_head_accept"] = fused
         # direct cast throughput (2 B read + 0.53125 B written per weight)
         w = synth.student_t_bf16((11008, 4096), 0.02, 1, device=device)
         ws_ = [w.clone() for _ in range(4)]   # 360 MB rotated: larger than L2

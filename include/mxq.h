@@ -210,6 +210,24 @@ size_t mxq_greedy_accept_static_max_bytes(void);
 int mxq_greedy_accept_tokens(const int32_t *draft, const int32_t *verifier, int64_t B, int T, int R,
                              int32_t *accept_len, int32_t *next_token, void *stream);
 
+/* Vocabulary projection fused with the greedy verification: logits = X . w^[V][K]^T (mxq_linear with N = V), the
+ * argmax of every row and the walk over the draft in ONE launch; the logits are never written (Sec. III-A, III-B:
+ * the verifier's tokens decide how many speculated tokens survive, and supply the next one).
+ *   X_bf16  [R][K] BF16: the hidden states at the positions the T draft tokens propose to fill, R == T or T + 1,
+ *           1 <= R <= 16.  T == 0, R == 1 is the plain draft step: next_token = argmax.
+ *   draft   [T] int32 (device; may be NULL if T == 0)
+ *   verifier [R] int32 out, optional (NULL to skip): argmax of every row
+ *   accept_len [1], next_token [1] int32 out: as mxq_greedy_accept for one sequence
+ *   workspace  device memory, >= mxq_lm_head_accept_workspace_bytes, 16-byte aligned; zero its first 4096 bytes once
+ *              before the first use; every call leaves them zero again.  One per stream.
+ * Argmax rules as in mxq_greedy_accept (lowest index among equal maxima, NaN and -inf never selected), applied to the
+ * FP32 sums mxq_linear would have stored.  Where no tcgen05 kernel covers the call (K % 128 != 0, no tensor maps) the
+ * logits pass through the workspace and the ordinary kernels run. */
+size_t mxq_lm_head_accept_workspace_bytes(int R, int64_t V, int64_t K);
+int mxq_lm_head_accept(const void *X_bf16, int R, const uint8_t *codes, const uint8_t *scales, int64_t V, int64_t K,
+                       const int32_t *draft, int T, int32_t *verifier, int32_t *accept_len, int32_t *next_token,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

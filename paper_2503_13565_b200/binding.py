@@ -74,6 +74,10 @@ def lib() -> ctypes.CDLL:
             L.mxq_greedy_accept_static_max_bytes.argtypes = []
             L.mxq_greedy_accept_tokens.restype = i32
             L.mxq_greedy_accept_tokens.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp]
+            L.mxq_lm_head_accept_workspace_bytes.restype = sz
+            L.mxq_lm_head_accept_workspace_bytes.argtypes = [i32, i64, i64]
+            L.mxq_lm_head_accept.restype = i32
+            L.mxq_lm_head_accept.argtypes = [vp, i32, vp, vp, i64, i64, vp, i32, vp, vp, vp, vp, sz, vp]
             _lib = L
     return _lib
 
@@ -297,3 +301,30 @@ def mxq_greedy_accept_tokens(draft: torch.Tensor, verifier: torch.Tensor, stream
                                           b, t, r, g.data_ptr(), nxt.data_ptr(), _stream(stream)),
            "mxq_greedy_accept_tokens")
     return g, nxt
+
+
+def mxq_lm_head_accept_workspace_bytes(r: int, v: int, k: int) -> int:
+    return int(lib().mxq_lm_head_accept_workspace_bytes(r, v, k))
+
+
+def mxq_lm_head_accept(x: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, draft: torch.Tensor = None,
+                       workspace: torch.Tensor = None, stream=None):
+    """Vocabulary projection + argmax of every row + walk over the draft in one launch (the logits are never written).
+    x [R,K] BF16, codes/scales the MXFP4 pair of the [V,K] projection, draft [T] int32 with R == T or T + 1 (None: T = 0).
+    Returns (verifier [R] int32, accept_len [1] int32, next_token [1] int32).  ``workspace``: from ``new_workspace(
+    mxq_lm_head_accept_workspace_bytes(R, V, K))`` (zero-filled once; reusable; one per stream)."""
+    r, k = x.shape
+    v = codes.shape[0]
+    t = 0 if draft is None else int(draft.numel())
+    if workspace is None:
+        workspace = new_workspace(mxq_lm_head_accept_workspace_bytes(r, v, k), x.device)
+    verifier = torch.empty(r, dtype=torch.int32, device=x.device)
+    g = torch.empty(1, dtype=torch.int32, device=x.device)
+    nxt = torch.empty(1, dtype=torch.int32, device=x.device)
+    _check(lib().mxq_lm_head_accept(_dev(x, torch.bfloat16, "x"), r, _dev(codes, torch.uint8, "codes"),
+                                    _dev(scales, torch.uint8, "scales"), v, k,
+                                    0 if draft is None else _dev(draft, torch.int32, "draft"), t,
+                                    verifier.data_ptr(), g.data_ptr(), nxt.data_ptr(),
+                                    _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)),
+           "mxq_lm_head_accept")
+    return verifier, g, nxt

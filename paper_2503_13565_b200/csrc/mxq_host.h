@@ -16,6 +16,19 @@ int sm_count();
 // whether mxq_linear launches carry the programmatic-dependent-launch attribute
 bool pdl_enabled();
 
+// Vocabulary projection fused with the greedy verification (Sec. III-A, III-B).  With `keys` set a tcgen05 kernel
+// does not store Y: every finished logit (token row m, vocabulary index n) competes for keys[m], the last CTA to
+// deliver turns the keys into the verifier's tokens, walks the draft and leaves keys and ticket zero for the next call.
+struct FusedAccept {
+    unsigned long long *keys;   // running maxima as (ordered value, ~index), 0 = nothing yet, one per 128 bytes; nullptr: plain layer
+    unsigned int *ticket;       // CTAs that have delivered
+    const int32_t *draft;       // [T] speculated tokens
+    int32_t *verifier;          // [R] out: argmax of every row (may be nullptr)
+    int32_t *accept_len;        // [1] out: G
+    int32_t *next_token;        // [1] out: the verifier's token at position G, -1 if there is no such row
+    int T;
+};
+
 struct LinearPlan;
 // tensor-core path of mxq_linear (mxq_linear_mma.cu): false if the shape is not covered
 bool linear_mma_plan(int M, int64_t N, int64_t K, LinearPlan &plan);
@@ -32,13 +45,14 @@ bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &plan, bool with_wor
 // once per call by a kernel of its own instead of by every CTA of the weight kernel
 size_t linear_umma_workspace_bytes(int M, int64_t K);
 cudaError_t linear_umma_launch(const UmmaPlan &plan, const void *X, const uint8_t *codes, const uint8_t *scales,
-                               void *Y, int y_dtype, void *workspace, size_t workspace_bytes, cudaStream_t stream);
+                               void *Y, int y_dtype, void *workspace, size_t workspace_bytes, cudaStream_t stream,
+                               const FusedAccept *fused = nullptr);
 
 struct Fp4Plan;
 // tcgen05 path with packed 4-bit operands on both sides, M <= 4 (mxq_linear_fp4.cu)
 bool linear_fp4_plan(int M, int64_t N, int64_t K, Fp4Plan &plan);
 cudaError_t linear_fp4_launch(const Fp4Plan &plan, const void *X, const uint8_t *codes, const uint8_t *scales,
-                              void *Y, int y_dtype, cudaStream_t stream);
+                              void *Y, int y_dtype, cudaStream_t stream, const FusedAccept *fused = nullptr);
 int linear_fp4_take_status(uint32_t *out);
 
 }  // namespace mxq

@@ -259,6 +259,69 @@ int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *s
     return mxq::launch_status();
 }
 
+// ---- vocabulary projection fused with the greedy verification ---------------------------------------------------------
+// workspace: [4096-byte header: 16 keys 128 bytes apart, ticket, a constant -1][mxq_linear's own workspace][fallback only: logits, accept scratch]
+static constexpr size_t kFusedHeader = 4096;
+static size_t align256(size_t v) { return (v + 255u) & ~(size_t)255u; }
+
+size_t mxq_lm_head_accept_workspace_bytes(int R, int64_t V, int64_t K) {
+    if (R < 1 || R > MXQ_MAX_M || !mxq::shape_ok(V, K)) return 0;
+    mxq::Choice c;
+    mxq::choose(mxq::kernel_ceiling(), R, V, K, nullptr, true, c);
+    size_t b = kFusedHeader + align256(mxq_linear_workspace_bytes(R, V, K));
+    if (c.kernel != MXQ_KERNEL_FP4 && c.kernel != MXQ_KERNEL_UMMA)
+        b += align256((size_t)R * (size_t)V * 4u) + align256(mxq_accept_workspace_bytes(1, R, V));
+    return b;
+}
+
+int mxq_lm_head_accept(const void *X_bf16, int R, const uint8_t *codes, const uint8_t *scales, int64_t V, int64_t K,
+                       const int32_t *draft, int T, int32_t *verifier, int32_t *accept_len, int32_t *next_token,
+                       void *workspace, size_t workspace_bytes, void *stream) {
+    if (!X_bf16 || !codes || !scales || !accept_len || !next_token || !workspace || (T > 0 && !draft)) return MXQ_ERR_NULL;
+    if (R < 1 || R > MXQ_MAX_M || T < 0 || (R != T && R != T + 1) || !mxq::shape_ok(V, K) || V > 0x7FFFFFFF) return MXQ_ERR_SHAPE;
+    if (!mxq::aligned16(X_bf16) || !mxq::aligned16(codes) || !mxq::aligned16(scales) || !mxq::aligned16(workspace)) return MXQ_ERR_ALIGN;
+    if (workspace_bytes < mxq_lm_head_accept_workspace_bytes(R, V, K)) return MXQ_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    void *lin_ws = ws + kFusedHeader;
+    const size_t lin_ws_bytes = align256(mxq_linear_workspace_bytes(R, V, K));
+    mxq::Choice c;
+    mxq::choose(mxq::kernel_ceiling(), R, V, K, codes, true, c);
+    if (c.kernel == MXQ_KERNEL_FP4 || c.kernel == MXQ_KERNEL_UMMA) {
+        mxq::FusedAccept fa;
+        fa.keys = reinterpret_cast<unsigned long long *>(ws);
+        fa.ticket = reinterpret_cast<unsigned int *>(ws + 2048);
+        fa.draft = draft;
+        fa.verifier = verifier;
+        fa.accept_len = accept_len;
+        fa.next_token = next_token;
+        fa.T = T;
+        const cudaError_t e = c.kernel == MXQ_KERNEL_FP4
+                                  ? mxq::linear_fp4_launch(c.fp4, X_bf16, codes, scales, nullptr, MXQ_F32, st, &fa)
+                                  : mxq::linear_umma_launch(c.umma, X_bf16, codes, scales, nullptr, MXQ_F32, lin_ws, lin_ws_bytes, st, &fa);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            return MXQ_ERR_CUDA;
+        }
+        return mxq::launch_status();
+    }
+    // no tcgen05 kernel covers the call: the logits pass through the workspace
+    float *logits = reinterpret_cast<float *>(ws + kFusedHeader + lin_ws_bytes);
+    void *acc_ws = ws + kFusedHeader + lin_ws_bytes + align256((size_t)R * (size_t)V * 4u);
+    const size_t acc_ws_bytes = align256(mxq_accept_workspace_bytes(1, R, V));
+    int32_t *minus_one = reinterpret_cast<int32_t *>(ws + 2176);
+    if (cudaMemsetAsync(minus_one, 0xFF, 4, st) != cudaSuccess) return MXQ_ERR_CUDA;
+    int rc = mxq_linear(X_bf16, R, codes, scales, V, K, logits, MXQ_F32, lin_ws, lin_ws_bytes, stream);
+    if (rc != MXQ_OK) return rc;
+    if (verifier)   // a draft token of -1 never matches: the call returns G = 0 and the row's argmax
+        for (int r = 0; r < R; ++r) {
+            rc = mxq_greedy_accept(logits + (size_t)r * V, MXQ_F32, 1, 1, V, minus_one, 1, accept_len, verifier + r, acc_ws, acc_ws_bytes, stream);
+            if (rc != MXQ_OK) return rc;
+        }
+    if (T == 0) return mxq_greedy_accept(logits, MXQ_F32, 1, 1, V, minus_one, 1, accept_len, next_token, acc_ws, acc_ws_bytes, stream);
+    return mxq_greedy_accept(logits, MXQ_F32, 1, R, V, draft, T, accept_len, next_token, acc_ws, acc_ws_bytes, stream);
+}
+
 int mxq_linear_host(const void *X_host, int M, const uint8_t *codes, const uint8_t *scales, int64_t N,
                     int64_t K, void *Y_host, int y_dtype, void *X_stage_dev, void *Y_stage_dev,
                     void *workspace, size_t workspace_bytes, void *stream) {

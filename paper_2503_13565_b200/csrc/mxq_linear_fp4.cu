@@ -161,13 +161,17 @@ __device__ __forceinline__ bool split_half_unit(const uint4 raw, int m, int kk, 
 // the codes, cp.async of the scale bytes, barrier set-up); warps 2..5 split the activations stage by stage and,
 // at the end, read the accumulator (one row per thread), exchange partial results and store.
 // MULTI: whether a CTA may own more than one tile (false: exactly one, and the per-tile loops fold away).
-template <int NB, bool MULTI>
+template <int NB, bool MULTI, bool FUSED>
 __global__ void __launch_bounds__(kFp4Threads)
 linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 *__restrict__ X, int M,
                   const uint8_t *__restrict__ codes, const uint8_t *__restrict__ scales, int64_t N, int64_t K,
                   void *__restrict__ Y, int y_dtype, int split, int ring, int ks, int chunk_max, int tmem_cols, int groups,
-                  int tiles, int tiles_max) {
+                  int tiles, int tiles_max, const FusedAccept fa_arg) {
     extern __shared__ uint8_t smem_raw[];
+    // FUSED: the values compete for the verifier's argmax instead of being stored (fa.keys set); a template parameter so
+    // that the plain layer's epilogue carries none of it
+    FusedAccept fa = fa_arg;
+    if (!FUSED) fa.keys = nullptr;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef MXQ_FP4_TRACE
     long long tr_c0 = 0;
@@ -253,6 +257,8 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
             s_fail = 0;
             *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 8) = 0;   // s_bad
             s_xin = 0;
+            if (fa.keys)
+                for (int q = 0; q < 16; ++q) reinterpret_cast<volatile unsigned long long *>(gbase + (sMisc - base) + 16)[q] = 0ull;
         }
         if (tid == 32) TR(15);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -491,6 +497,17 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
         const int rr = row - (int)(owner * kFp4TileRows) / split;
         const uint32_t remote = peer_saddr(sRecv, owner), remote_bar = peer_saddr(recv_bar, owner);
         if (split > 1) cluster_wait();   // every CTA of the cluster has initialised its barriers (they arrived long ago)
+        // fused verification: instead of being stored, a finished value competes for its token row's running maximum
+        unsigned long long *s_keys = reinterpret_cast<unsigned long long *>(gbase + (sMisc - base) + 16);
+        // (a thread meets its candidates in ascending index order, so "strictly greater" keeps the lowest index; NaN and
+        // -inf never pass the test)
+        float bestv[MT];
+        uint32_t besti[MT];
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            bestv[m] = -INFINITY;
+            besti[m] = 0xFFFFFFFFu;
+        }
         for (int t = 0; t < ntile; ++t) {
             float yt[MT];
 #pragma unroll
@@ -556,7 +573,17 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                 if (n < N)
 #pragma unroll
                     for (int m = 0; m < MT; ++m)
-                        if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, yt[m] * kGuardUp);
+                        if (m < M) {
+                            if (fa.keys) {
+                                const float v = yt[m] * kGuardUp;
+                                if (v > bestv[m]) {
+                                    bestv[m] = v;
+                                    besti[m] = (uint32_t)n;
+                                }
+                            } else {
+                                store_out(Y, y_dtype, (int64_t)m * N + n, yt[m] * kGuardUp);
+                            }
+                        }
             } else {
 #pragma unroll
                 for (int m = 0; m < MT; ++m)
@@ -576,10 +603,28 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                 const int r = ct / split, j = ct & (split - 1);
                 for (int t = 0; t < ntile; ++t) {
                     const int64_t n = n0 + (int64_t)t * kFp4TileRows + row_lo + r;
-                    for (int m = 0; m < M; ++m) {
-                        float v = gRecv[((t * split + j) * M + m) * cnt_max + r];
-                        for (int o = 1; o < split; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                        if (j == 0 && n < N) store_out(Y, y_dtype, (int64_t)m * N + n, v * kGuardUp + poison);
+                    // all loads, then all shuffles, then all uses: the token rows are independent of each other
+                    float v[MT];
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) v[m] = m < M ? gRecv[((t * split + j) * M + m) * cnt_max + r] : 0.f;
+                    for (int o = 1; o < split; o <<= 1) {
+#pragma unroll
+                        for (int m = 0; m < MT; ++m) v[m] += __shfl_xor_sync(0xffffffffu, v[m], o);
+                    }
+                    if (j == 0 && n < N) {
+#pragma unroll
+                        for (int m = 0; m < MT; ++m)
+                            if (m < M) {
+                                const float w = v[m] * kGuardUp + poison;
+                                if (fa.keys) {
+                                    if (w > bestv[m]) {
+                                        bestv[m] = w;
+                                        besti[m] = (uint32_t)n;
+                                    }
+                                } else {
+                                    store_out(Y, y_dtype, (int64_t)m * N + n, w);
+                                }
+                            }
                     }
                 }
             } else {
@@ -589,9 +634,25 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                     float acc = 0.f;
                     for (int j = 0; j < split; ++j) acc += gRecv[((t * split + j) * M + m) * cnt_max + r];
                     const int64_t n = n0 + (int64_t)t * kFp4TileRows + row_lo + r;
-                    if (n < N) store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison);
+                    if (n < N) {
+                        if (fa.keys) {
+                            const unsigned long long key = argmax_key(acc * kGuardUp + poison, (uint32_t)n);
+                            if (key) atomicMax(s_keys + m, key);   // (rare decomposition: straight into shared memory)
+                        } else {
+                            store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison);
+                        }
+                    }
                 }
             }
+        }
+        if (fa.keys) {
+#pragma unroll
+            for (int m = 0; m < MT; ++m)
+                if (m < M) {
+                    const unsigned long long k = warp_max_key(besti[m] != 0xFFFFFFFFu ? argmax_key(bestv[m], besti[m]) : 0ull);
+                    if (lane == 0 && k) atomicMax(s_keys + m, k);
+                }
+            fused_accept_finish(fa, s_keys, M, gridDim.x, ct);
         }
     }
 
@@ -604,19 +665,19 @@ int env_int(const char *name) {
     return e ? std::atoi(e) : 0;
 }
 
-template <int NB, bool MULTI>
+template <int NB, bool MULTI, bool FUSED>
 cudaError_t launch_fp4(const Fp4Plan &p, const CUtensorMap &map, const void *X, const uint8_t *codes,
-                       const uint8_t *scales, void *Y, int y_dtype, cudaStream_t stream) {
+                       const uint8_t *scales, void *Y, int y_dtype, cudaStream_t stream, const FusedAccept &fa) {
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(linear_fp4_kernel<NB, MULTI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(linear_fp4_kernel<NB, MULTI, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kFp4SmemLimit);
         if (e != cudaSuccess) return e;
         // all of the SM's L1/shared array as shared memory: how many CTAs (of this and of the next kernel) fit on an
         // SM is what decides how early the next kernel's weight stream can start
-        e = cudaFuncSetAttribute(linear_fp4_kernel<NB, MULTI>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(linear_fp4_kernel<NB, MULTI, FUSED>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -641,8 +702,8 @@ cudaError_t launch_fp4(const Fp4Plan &p, const CUtensorMap &map, const void *X, 
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    return cudaLaunchKernelEx(&cfg, linear_fp4_kernel<NB, MULTI>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
-                              Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols, p.groups, p.tiles, p.tiles_max);
+    return cudaLaunchKernelEx(&cfg, linear_fp4_kernel<NB, MULTI, FUSED>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
+                              Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols, p.groups, p.tiles, p.tiles_max, fa);
 }
 
 }  // namespace
@@ -660,20 +721,27 @@ bool linear_fp4_plan(int M, int64_t N, int64_t K, Fp4Plan &p) {
 }
 
 cudaError_t linear_fp4_launch(const Fp4Plan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,
-                              int y_dtype, cudaStream_t stream) {
+                              int y_dtype, cudaStream_t stream, const FusedAccept *fused) {
     CUtensorMap map;
     if (!codes_tensor_map(codes, p.N, p.K, /*expand_fp4=*/false, &map)) return cudaErrorNotSupported;
     const bool multi = p.tiles_max > 1;
+    const FusedAccept fa = fused ? *fused : FusedAccept{};
     switch (p.nb) {
         case 16:
-            return multi ? launch_fp4<16, true>(p, map, X, codes, scales, Y, y_dtype, stream)
-                         : launch_fp4<16, false>(p, map, X, codes, scales, Y, y_dtype, stream);
+            return fa.keys ? (multi ? launch_fp4<16, true, true>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
+                                    : launch_fp4<16, false, true>(p, map, X, codes, scales, Y, y_dtype, stream, fa))
+                           : (multi ? launch_fp4<16, true, false>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
+                                    : launch_fp4<16, false, false>(p, map, X, codes, scales, Y, y_dtype, stream, fa));
         case 32:
-            return multi ? launch_fp4<32, true>(p, map, X, codes, scales, Y, y_dtype, stream)
-                         : launch_fp4<32, false>(p, map, X, codes, scales, Y, y_dtype, stream);
+            return fa.keys ? (multi ? launch_fp4<32, true, true>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
+                                    : launch_fp4<32, false, true>(p, map, X, codes, scales, Y, y_dtype, stream, fa))
+                           : (multi ? launch_fp4<32, true, false>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
+                                    : launch_fp4<32, false, false>(p, map, X, codes, scales, Y, y_dtype, stream, fa));
         default:
-            return multi ? launch_fp4<64, true>(p, map, X, codes, scales, Y, y_dtype, stream)
-                         : launch_fp4<64, false>(p, map, X, codes, scales, Y, y_dtype, stream);
+            return fa.keys ? (multi ? launch_fp4<64, true, true>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
+                                    : launch_fp4<64, false, true>(p, map, X, codes, scales, Y, y_dtype, stream, fa))
+                           : (multi ? launch_fp4<64, true, false>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
+                                    : launch_fp4<64, false, false>(p, map, X, codes, scales, Y, y_dtype, stream, fa));
     }
 }
 

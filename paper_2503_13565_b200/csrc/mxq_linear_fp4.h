@@ -38,7 +38,7 @@ inline uint32_t fp4_smem_bytes(int nb, int M, int tiles_max, int chunk, int ring
     const uint32_t recv = split > 1 ? (uint32_t)(tiles_max * M) * kFp4RecvRows * 4u : 0u;   // partial results pushed by the cluster's CTAs
     const uint32_t b = 1024u /* alignment slack */ + (uint32_t)ring * (kFp4StageBytes + kFp4SfStageBytes) +
                        (uint32_t)chunk * ((uint32_t)nb * 128u + kFp4SfStageBytes) + recv +
-                       (uint32_t)(2 * ring + 2 + chunk) * 8u /* mbarriers */ + 16u /* tensor-memory address, three flags */;
+                       (uint32_t)(2 * ring + 2 + chunk) * 8u /* mbarriers */ + 16u /* tensor-memory address, three flags */ + 208u /* fused verification: keys, tokens, flag */;
     return (b + 15u) & ~15u;
 }
 

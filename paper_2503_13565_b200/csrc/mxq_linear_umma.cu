@@ -167,12 +167,16 @@ cudaError_t launch_split(const __nv_bfloat16 *X, int M, int64_t K, int ks, uint8
 // the codes, cp.async of the scale bytes, barrier set-up); warps 2..5 split the activations stage by stage and,
 // at the end, read the accumulator (one row per thread), exchange partial results and store.
 // MULTI: whether a CTA may own more than one tile (false: exactly one, and the per-tile loops fold away).
-template <int NB, bool MULTI, bool BRING>
+template <int NB, bool MULTI, bool BRING, bool FUSED>
 __global__ void __launch_bounds__(kUmmaThreads)
 linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 *__restrict__ X, int M,
                   const uint8_t *__restrict__ codes, const uint8_t *__restrict__ scales, int64_t N, int64_t K,
                   void *__restrict__ Y, int y_dtype, int split, int ring, int ks, int chunk_max, int tmem_cols, int groups,
-                  int tiles, int tiles_max, const uint8_t *__restrict__ presplit) {
+                  int tiles, int tiles_max, const uint8_t *__restrict__ presplit, const FusedAccept fa_arg) {
+    // FUSED: the values compete for the verifier's argmax instead of being stored (fa.keys set); a template parameter so
+    // that the plain layer's epilogue carries none of it
+    FusedAccept fa = fa_arg;
+    if (!FUSED) fa.keys = nullptr;
     constexpr bool bring = BRING;   // the token operand is fetched stage by stage into the ring slots (needs presplit, one tile)
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -260,6 +264,8 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
             s_fail = 0;
             *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 8) = 0;   // s_bad
             s_xin = 0;
+            if (fa.keys)
+                for (int q = 0; q < 16; ++q) reinterpret_cast<volatile unsigned long long *>(gbase + (sMisc - base) + 16)[q] = 0ull;
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         __syncwarp();
@@ -480,6 +486,17 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
         const int rr = row - (int)(owner * kUmmaTileRows) / split;
         const uint32_t remote = peer_saddr(sRecv, owner), remote_bar = peer_saddr(recv_bar, owner);
         if (split > 1) cluster_wait();   // every CTA of the cluster has initialised its barriers (they arrived long ago)
+        // fused verification: instead of being stored, a finished value competes for its token row's running maximum
+        unsigned long long *s_keys = reinterpret_cast<unsigned long long *>(gbase + (sMisc - base) + 16);
+        // (a thread meets its candidates in ascending index order, so "strictly greater" keeps the lowest index; NaN and
+        // -inf never pass the test)
+        float bestv[MT];
+        uint32_t besti[MT];
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            bestv[m] = -INFINITY;
+            besti[m] = 0xFFFFFFFFu;
+        }
         for (int t = 0; t < ntile; ++t) {
             float yt[MT];
 #pragma unroll
@@ -546,7 +563,17 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                 if (n < N)
 #pragma unroll
                     for (int m = 0; m < MT; ++m)
-                        if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, yt[m] * kGuardUp);
+                        if (m < M) {
+                            if (fa.keys) {
+                                const float v = yt[m] * kGuardUp;
+                                if (v > bestv[m]) {
+                                    bestv[m] = v;
+                                    besti[m] = (uint32_t)n;
+                                }
+                            } else {
+                                store_out(Y, y_dtype, (int64_t)m * N + n, yt[m] * kGuardUp);
+                            }
+                        }
             } else {
 #pragma unroll
                 for (int m = 0; m < MT; ++m)
@@ -565,10 +592,28 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                 const int r = ct / split, j = ct & (split - 1);
                 for (int t = 0; t < ntile; ++t) {
                     const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row_lo + r;
-                    for (int m = 0; m < M; ++m) {
-                        float v = gRecv[((t * split + j) * M + m) * cnt_max + r];
-                        for (int o = 1; o < split; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                        if (j == 0 && n < N) store_out(Y, y_dtype, (int64_t)m * N + n, v * kGuardUp + poison);
+                    // all loads, then all shuffles, then all uses: the token rows are independent of each other
+                    float v[MT];
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) v[m] = m < M ? gRecv[((t * split + j) * M + m) * cnt_max + r] : 0.f;
+                    for (int o = 1; o < split; o <<= 1) {
+#pragma unroll
+                        for (int m = 0; m < MT; ++m) v[m] += __shfl_xor_sync(0xffffffffu, v[m], o);
+                    }
+                    if (j == 0 && n < N) {
+#pragma unroll
+                        for (int m = 0; m < MT; ++m)
+                            if (m < M) {
+                                const float w = v[m] * kGuardUp + poison;
+                                if (fa.keys) {
+                                    if (w > bestv[m]) {
+                                        bestv[m] = w;
+                                        besti[m] = (uint32_t)n;
+                                    }
+                                } else {
+                                    store_out(Y, y_dtype, (int64_t)m * N + n, w);
+                                }
+                            }
                     }
                 }
             } else {
@@ -578,9 +623,25 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                     float acc = 0.f;
                     for (int j = 0; j < split; ++j) acc += gRecv[((t * split + j) * M + m) * cnt_max + r];
                     const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row_lo + r;
-                    if (n < N) store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison);
+                    if (n < N) {
+                        if (fa.keys) {
+                            const unsigned long long key = argmax_key(acc * kGuardUp + poison, (uint32_t)n);
+                            if (key) atomicMax(s_keys + m, key);   // (rare decomposition: straight into shared memory)
+                        } else {
+                            store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison);
+                        }
+                    }
                 }
             }
+        }
+        if (fa.keys) {
+#pragma unroll
+            for (int m = 0; m < MT; ++m)
+                if (m < M) {
+                    const unsigned long long k = warp_max_key(besti[m] != 0xFFFFFFFFu ? argmax_key(bestv[m], besti[m]) : 0ull);
+                    if (lane == 0 && k) atomicMax(s_keys + m, k);
+                }
+            fused_accept_finish(fa, s_keys, M, gridDim.x, ct);
         }
     }
 
@@ -592,19 +653,19 @@ int env_int(const char *name) {
     return e ? std::atoi(e) : 0;
 }
 
-template <int NB, bool MULTI, bool BRING>
+template <int NB, bool MULTI, bool BRING, bool FUSED>
 cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X, const uint8_t *codes,
-                       const uint8_t *scales, void *Y, int y_dtype, const uint8_t *presplit, cudaStream_t stream) {
+                       const uint8_t *scales, void *Y, int y_dtype, const uint8_t *presplit, cudaStream_t stream, const FusedAccept &fa) {
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI, BRING>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI, BRING, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kUmmaSmemLimit);
         if (e != cudaSuccess) return e;
         // all of the SM's L1/shared array as shared memory: how many CTAs (of this and of the next kernel) fit on an
         // SM is what decides how early the next kernel's weight stream can start
-        e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI, BRING>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI, BRING, FUSED>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -629,8 +690,8 @@ cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    return cudaLaunchKernelEx(&cfg, linear_umma_kernel<NB, MULTI, BRING>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
-                              Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols, p.groups, p.tiles, p.tiles_max, presplit);
+    return cudaLaunchKernelEx(&cfg, linear_umma_kernel<NB, MULTI, BRING, FUSED>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
+                              Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols, p.groups, p.tiles, p.tiles_max, presplit, fa);
 }
 
 }  // namespace
@@ -656,13 +717,25 @@ bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p, bool with_worksp
                        std::getenv("MXQ_UMMA_BRING") ? env_int("MXQ_UMMA_BRING") : -1);
 }
 
+template <int NB>
+static cudaError_t pick_umma(const UmmaPlan &p, bool bring, const CUtensorMap &map, const void *X, const uint8_t *codes,
+                             const uint8_t *scales, void *Y, int y_dtype, const uint8_t *ws, cudaStream_t stream, const FusedAccept &fa) {
+    if (fa.keys)
+        return p.tiles_max > 1 ? launch_umma<NB, true, false, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)
+               : bring         ? launch_umma<NB, false, true, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)
+                               : launch_umma<NB, false, false, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa);
+    return p.tiles_max > 1 ? launch_umma<NB, true, false, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)
+           : bring         ? launch_umma<NB, false, true, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)
+                           : launch_umma<NB, false, false, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa);
+}
+
 size_t linear_umma_workspace_bytes(int M, int64_t K) {
     if (M < presplit_min_m() || M > kUmmaMaxM || K < 128 || (K % 128) != 0 || K > 0x3FFFFFFF) return 0;
     return umma_ws_bytes(umma_nb(M), (int)(K / kUmmaStageK));
 }
 
 cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,
-                              int y_dtype, void *workspace, size_t workspace_bytes, cudaStream_t stream) {
+                              int y_dtype, void *workspace, size_t workspace_bytes, cudaStream_t stream, const FusedAccept *fused) {
     CUtensorMap map;
     if (!codes_tensor_map(codes, p.N, p.K, /*expand_fp4=*/true, &map)) return cudaErrorNotSupported;
     // a workspace that is large enough (and aligned for bulk copies) lets the token operand be split once per call
@@ -673,7 +746,7 @@ cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *
     if (p.presplit && !ws) {   // planned for a workspace that is not there: plan again without
         UmmaPlan q;
         if (!linear_umma_plan(p.M, p.N, p.K, q, false)) return cudaErrorNotSupported;
-        return linear_umma_launch(q, X, codes, scales, Y, y_dtype, nullptr, 0, stream);
+        return linear_umma_launch(q, X, codes, scales, Y, y_dtype, nullptr, 0, stream, fused);
     }
     if (ws) {
         const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(X);
@@ -683,19 +756,14 @@ cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *
         if (e != cudaSuccess) return e;
     }
     const bool bring = ws && p.bring && p.tiles_max == 1;
+    const FusedAccept fa = fused ? *fused : FusedAccept{};
     switch (p.nb) {
         case 16:
-            return p.tiles_max > 1 ? launch_umma<16, true, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
-                   : bring         ? launch_umma<16, false, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
-                                   : launch_umma<16, false, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream);
+            return pick_umma<16>(p, bring, map, X, codes, scales, Y, y_dtype, ws, stream, fa);
         case 32:
-            return p.tiles_max > 1 ? launch_umma<32, true, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
-                   : bring         ? launch_umma<32, false, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
-                                   : launch_umma<32, false, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream);
+            return pick_umma<32>(p, bring, map, X, codes, scales, Y, y_dtype, ws, stream, fa);
         default:
-            return p.tiles_max > 1 ? launch_umma<48, true, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
-                   : bring         ? launch_umma<48, false, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream)
-                                   : launch_umma<48, false, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream);
+            return pick_umma<48>(p, bring, map, X, codes, scales, Y, y_dtype, ws, stream, fa);
     }
 }
 

@@ -57,7 +57,7 @@ inline uint32_t umma_smem_bytes(int nb, int M, int tiles_max, int chunk, int rin
     const uint32_t recv = split > 1 ? (uint32_t)(tiles_max * M) * kUmmaRecvRows * 4u : 0u;   // partial results pushed by the cluster's CTAs
     const uint32_t b = 1024u /* alignment slack */ + (uint32_t)ring * (kUmmaStageBytes + kUmmaSfStageBytes) +
                        (uint32_t)(bring ? ring : chunk) * ((uint32_t)nb * 128u + kUmmaSfStageBytes) + recv +
-                       (uint32_t)(2 * ring + 2 + (chunk + 1) / 2) * 8u /* mbarriers */ + 16u /* tensor-memory address, flags */;
+                       (uint32_t)(2 * ring + 2 + (chunk + 1) / 2) * 8u /* mbarriers */ + 16u /* tensor-memory address, flags */ + 208u /* fused verification: keys, tokens, flag */;
     return (b + 15u) & ~15u;
 }
 

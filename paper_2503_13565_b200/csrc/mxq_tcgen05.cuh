@@ -2,6 +2,7 @@
 // waits, TMA tensor copies, tcgen05 (tensor memory, block-scaled MMA, commit), cluster barriers and
 // distributed shared memory.  One instruction (or one short idiom) per function; no policy here.
 #pragma once
+#include "mxq_host.h"
 #include <cuda.h>   // CUtensorMap only
 
 #include "mxq_device.cuh"
@@ -164,6 +165,59 @@ __device__ __forceinline__ float ld_peer_f32(uint32_t local_saddr, uint32_t rank
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(local_saddr), "r"(rank));
     asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(raddr) : "memory");
     return v;
+}
+
+// ---- vocabulary projection fused with the greedy verification (Sec. III-A, III-B) ----------------------------------
+// With `keys` set a tcgen05 kernel does not store Y: every finished logit (token row m, vocabulary index n) competes
+// for keys[m], the last CTA to deliver turns the keys into the verifier's tokens, walks the draft and leaves keys and
+// ticket zero for the next call.
+constexpr int kFusedKeyStride = 16;   // keys[m] lives at 64-bit word 16 m of the workspace header
+constexpr uint32_t kFusedSmemBytes = 16 * 8 + 16 * 4 + 16;   // keys, tokens, "last CTA" flag
+// Larger value wins, then the lower index; NaN and -inf never compete (a row of nothing else yields token 0).
+__device__ __forceinline__ unsigned long long argmax_key(float v, uint32_t index) {
+    if (!(v > -INFINITY)) return 0ull;
+    const uint32_t b = __float_as_uint(v + 0.f);   // -0 -> +0: equal values must tie
+    const uint32_t u = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+    return ((unsigned long long)u << 32) | (uint32_t)~index;
+}
+__device__ __forceinline__ unsigned long long warp_max_key(unsigned long long k) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, k, o);
+        k = other > k ? other : k;
+    }
+    return k;
+}
+// All 128 epilogue threads (named barrier 1), after their candidates are in s_keys (shared memory, [16]).
+// R = token rows, grid = CTAs of the launch.
+__device__ __forceinline__ void fused_accept_finish(const FusedAccept &fa, unsigned long long *s_keys, int R, uint32_t grid, int ct) {
+    int32_t *s_tok = reinterpret_cast<int32_t *>(s_keys + 16);
+    volatile int *s_last = reinterpret_cast<volatile int *>(s_tok + 16);
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    // (a token row's key has a 128-byte line to itself, and a CTA that cannot raise it does not try: same-address atomics
+    // from every SM at once are served one after the other)
+    if (ct < R && s_keys[ct] > *reinterpret_cast<volatile unsigned long long *>(fa.keys + ct * kFusedKeyStride))
+        atomicMax(fa.keys + ct * kFusedKeyStride, s_keys[ct]);
+    __threadfence();
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (ct == 0) *s_last = atomicAdd(fa.ticket, 1u) == grid - 1u;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (!*s_last) return;
+    __threadfence();
+    if (ct < R) {
+        const unsigned long long key = atomicExch(fa.keys + ct * kFusedKeyStride, 0ull);   // read and leave zero for the next call
+        const int32_t tok = key ? (int32_t)~(uint32_t)key : 0;
+        s_tok[ct] = tok;
+        if (fa.verifier) fa.verifier[ct] = tok;
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (ct == 0) {
+        int G = 0;
+        while (G < fa.T && fa.draft[G] == s_tok[G]) ++G;   // tokens after the first mismatch are dropped (R >= T)
+        *fa.accept_len = G;
+        *fa.next_token = G < R ? s_tok[G] : -1;
+        *fa.ticket = 0u;
+    }
 }
 
 __device__ __forceinline__ void store_out(void *Y, int y_dtype, int64_t idx, float v) {

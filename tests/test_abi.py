@@ -72,6 +72,11 @@ def test_argument_errors_are_caught_before_any_launch():
     assert L.mxq_greedy_accept(a, 3, 1, 5, 100, a, 4, a, a, a, 1 << 20, None) == 4
     assert L.mxq_greedy_accept_tokens(a, a, 1, 4, 6, a, a, None) == 2
     assert L.mxq_greedy_accept_tokens(None, a, 1, 4, 5, a, a, None) == 1
+    # fused vocabulary projection + verification: R must be T or T + 1 and at most 16; a workspace is mandatory
+    assert L.mxq_lm_head_accept(a, 3, a, a, 1024, 128, a, 1, None, a, a, a, 1 << 20, None) == 2
+    assert L.mxq_lm_head_accept(a, 17, a, a, 1024, 128, a, 16, None, a, a, a, 1 << 20, None) == 2
+    assert L.mxq_lm_head_accept(a, 2, a, a, 1024, 128, a, 1, None, a, a, None, 0, None) == 1
+    assert L.mxq_lm_head_accept(a, 2, a, a, 1024, 128, a, 1, None, a, a, a, 16, None) == 5
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

@@ -720,13 +720,15 @@ bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p, bool with_worksp
 template <int NB>
 static cudaError_t pick_umma(const UmmaPlan &p, bool bring, const CUtensorMap &map, const void *X, const uint8_t *codes,
                              const uint8_t *scales, void *Y, int y_dtype, const uint8_t *ws, cudaStream_t stream, const FusedAccept &fa) {
-    if (fa.keys)
-        return p.tiles_max > 1 ? launch_umma<NB, true, false, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)
-               : bring         ? launch_umma<NB, false, true, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)
-                               : launch_umma<NB, false, false, true>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa);
-    return p.tiles_max > 1 ? launch_umma<NB, true, false, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)
-           : bring         ? launch_umma<NB, false, true, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)
-                           : launch_umma<NB, false, false, false>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa);
+    const bool multi = p.tiles_max > 1;
+#define MXQ_UMMA_PICK(FUSED)                                                                                                  \
+    return multi ? (bring ? launch_umma<NB, true, true, FUSED>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)           \
+                          : launch_umma<NB, true, false, FUSED>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa))         \
+                 : (bring ? launch_umma<NB, false, true, FUSED>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)          \
+                          : launch_umma<NB, false, false, FUSED>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa))
+    if (fa.keys) { MXQ_UMMA_PICK(true); }
+    MXQ_UMMA_PICK(false);
+#undef MXQ_UMMA_PICK
 }
 
 size_t linear_umma_workspace_bytes(int M, int64_t K) {
@@ -755,7 +757,7 @@ cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *
                                            : launch_split<48>(x, p.M, p.K, p.ks, ws, stream);
         if (e != cudaSuccess) return e;
     }
-    const bool bring = ws && p.bring && p.tiles_max == 1;
+    const bool bring = ws && p.bring;
     const FusedAccept fa = fused ? *fused : FusedAccept{};
     switch (p.nb) {
         case 16:

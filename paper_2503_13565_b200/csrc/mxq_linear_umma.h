@@ -48,7 +48,8 @@ struct UmmaPlan {
     int grid;        // groups * split
     int tmem_cols;   // tensor-memory columns allocated per CTA
     int presplit;    // planned for a token operand split ahead of the weight kernel (needs the workspace)
-    int bring;       // ... and fetched stage by stage into the ring slots (one tile per CTA) instead of whole K ranges
+    int bring;       // ... and fetched stage by stage into the ring slots instead of whole K ranges
+    long cost;       // the layout heuristic's figure for the chosen decomposition (comparable within a regime)
     uint32_t smem_bytes;
     int64_t N, K;
 };
@@ -125,14 +126,15 @@ inline bool umma_layout_one(UmmaPlan &p, int sms, int force_split, int force_rin
             const int units = tmax * chunk;
             ring = units < kUmmaMaxUnitsResident ? units : kUmmaMaxUnitsResident;
             if (force_ring > 0 && force_ring < ring) ring = force_ring;
-            while (ring > 1 && umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s) > kUmmaSmemLimit) --ring;
-            if (umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s) > kUmmaSmemLimit) continue;
+            const int br = allow_bring && p.presplit ? 1 : 0;   // (every tile then fetches the token operand's stages again, from L2)
+            while (ring > 1 && umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s, br) > kUmmaSmemLimit) --ring;
+            if (umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s, br) > kUmmaSmemLimit) continue;
             // Time ~ units per CTA / the rate its stream reaches: two requesters at 25 GB/s each, the ring's bytes in
             // flight (8 KB of packed codes per slot) per 1.5 us of latency, the SM's share of the memory bandwidth;
             // nearly doubled for K ranges under half a row of codes (see the packed-FP4 kernel).
             const long waves = ((long)groups * s + sms - 1) / sms;
             const long by_ring = (long)ring * 8192 / 1500, rate = by_ring < 41 ? by_ring : 41;   // GB/s
-            cost = waves * units * 1000 / rate * (s <= 2 ? 10 : 19) + s;
+            cost = waves * units * 1000 / rate * (s <= 2 ? 10 : 19) * (br ? 17 : 10) / 10 + s;   // (the operand fetched again per tile: measured)
         }
         if (best_cost < 0 || cost < best_cost || (cost == best_cost && layer_regime)) {   // layer regime: ties to the larger split
             best_cost = cost;
@@ -148,7 +150,8 @@ inline bool umma_layout_one(UmmaPlan &p, int sms, int force_split, int force_rin
     p.ring = best_ring;
     p.chunk_max = (p.ks + best_split - 1) / best_split;
     p.grid = best_groups * best_split;
-    p.bring = allow_bring && p.presplit && layer_regime && p.tiles_max == 1 ? 1 : 0;
+    p.bring = allow_bring && p.presplit && (!layer_regime || p.tiles_max == 1) ? 1 : 0;
+    p.cost = best_cost;
     p.smem_bytes = umma_smem_bytes(p.nb, p.M, p.tiles_max, p.chunk_max, best_ring, best_split, p.bring);
     p.tmem_cols = umma_tmem_cols(p.nb, p.tiles_max);
     return true;
@@ -161,13 +164,21 @@ inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, i
     if (!p.presplit || force_bring == 0) return umma_layout_one(p, sms, force_split, force_ring, force_tiles, false);
     UmmaPlan r = p;
     const bool have_r = force_bring < 0 && umma_layout_one(r, sms, force_split, force_ring, force_tiles, false);
-    if (have_r && (r.tiles_max > 1 ? p.tiles > sms : (r.ring >= 3 && 6 * r.grid >= 5 * sms))) {   // (several tiles per CTA: the vocabulary regime only)
-        p = r;
-        return true;
+    if (p.tiles <= sms) {
+        if (have_r && r.tiles_max == 1 && r.ring >= 3 && 6 * r.grid >= 5 * sms) {
+            p = r;
+            return true;
+        }
+        if (umma_layout_one(p, sms, force_split, force_ring, force_tiles, true)) return true;
+        if (have_r) p = r;
+        return have_r;
     }
-    if (umma_layout_one(p, sms, force_split, force_ring, force_tiles, true)) return true;
-    if (have_r) p = r;
-    return have_r;
+    // vocabulary regime: the modelled cost decides (resident on ties: no second fetch of the operand per tile)
+    UmmaPlan b = p;
+    const bool have_b = umma_layout_one(b, sms, force_split, force_ring, force_tiles, true);
+    if (!have_r && !have_b) return false;
+    p = have_r && (!have_b || r.cost <= b.cost) ? r : b;
+    return true;
 }
 
 }  // namespace mxq

@@ -127,7 +127,7 @@ split_tokens_kernel(const __nv_bfloat16 *__restrict__ X, int M, int64_t K, int k
     uint8_t *gSFB = ws + umma_ws_flags_bytes(ks), *gB = gSFB + (size_t)ks * kUmmaSfStageBytes;
     const int kk = (int)blockIdx.x * (2 * kUmmaStageK) + lane * 8;
     const bool act = kk < K;
-    pdl_wait();      // X may be the previous kernel's output; the workspace may still be read by the previous weight kernel
+    if (warp == 0) pdl_wait();   // X may be the previous kernel's output; the workspace may still be read by the previous weight kernel
     __syncthreads();
     uint4 raw[(kUmmaMaxM + kSplitWarps - 1) / kSplitWarps];
 #pragma unroll
@@ -286,12 +286,10 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sMisc), "r"(tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // Only the activation warps read what the previous kernel wrote (X) and write what the next one reads (Y), so
-    // only they wait for it; they do so at once, and join the CTA-wide barrier (initialised mbarriers, tensor-memory
-    // address) after that wait.
-    if (warp >= 2 || (warp == 1 && bring)) {   // (bring: the producer reads what the split kernel wrote)
-        pdl_wait();
-    }
+    // Only the activation warps read what the previous kernel wrote (X, or the split kernel's output) and write what the
+    // next one reads (Y).  One of them waits for it, at once; the others -- and the producer, which fetches the split
+    // kernel's output only after this point -- meet it at the CTA-wide barrier below (see the packed-FP4 kernel).
+    if (warp == 2) pdl_wait();
     if (split > 1) cluster_arrive();   // "my barriers exist"; the matching wait is just before the first push to a peer
     tc_fence_before();
     asm volatile("bar.sync 0;" ::: "memory");

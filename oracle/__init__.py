@@ -8,7 +8,8 @@ package imports nothing from here.
 All tensors cross this boundary as numpy arrays: BF16 data as ``uint16`` bit
 patterns, codes and scales as ``uint8``, results as ``float64`` / ``int32``.
 The arithmetic is all in the C file; this module only compiles it on first
-use, marshals arguments and allocates outputs.
+use, marshals arguments and allocates outputs (one exception: ``linear_bf16``, the unquantised comparison layer,
+is the textbook matrix product and is written with numpy here).
 """
 from __future__ import annotations
 
@@ -126,6 +127,18 @@ def linear(x_bits: np.ndarray, codes: np.ndarray, scales: np.ndarray, rows=None)
         a = np.empty((m, r.size), np.float64)
         _load().oq_linear_rows(_p(x), m, _p(c), _p(s), n, k, _p(r), r.size, _p(y), _p(a))
     return y, a
+
+
+def linear_bf16(x_bits: np.ndarray, w_bits: np.ndarray, rows=None):
+    """The layer with unquantised BF16 weights (the comparison point of Sec. III-D-3 / IV-D): the plain definition
+    y[m, n] = sum_k x[m, k] * w[n, k] in FP64 (numpy's matmul is the one library step), and a[m, n] = sum_k |x w|.
+    BF16 bit patterns in, every product exact in FP64.  ``rows``: compute only these output columns n."""
+    x = (_c(x_bits, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    wb = _c(w_bits, np.uint16)
+    if rows is not None:
+        wb = wb[np.asarray(rows, dtype=np.int64)]
+    w = (wb.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    return x @ w.T, np.abs(x) @ np.abs(w).T
 
 
 def _logits_arg(logits: np.ndarray):

@@ -385,6 +385,25 @@ def run_ours(args):
             fused["%dx4096_r%d" % (v_, r_)] = {"fused_us": tf * 1e6, "linear_then_accept_us": tu * 1e6}
             del mats_
         extra["lm_head_accept"] = fused
+        # the paper's comparison point: the same layer set with unquantised BF16 weights (16 bits per weight against 4.25)
+        bf = {}
+        shapes7 = [(4096, 4096)] * 4 + [(11008, 4096)] * 2 + [(4096, 11008)]
+        for mm in (1, 8):
+            nl = 3   # 3 x 404 MB of BF16 weights: larger than L2
+            wl = [[synth.normal_bf16((n_, k_), 0.02, 100 + 10 * li + j, device) for j, (n_, k_) in enumerate(shapes7)] for li in range(nl)]
+            xk = {k_: synth.normal_bf16((mm, k_), 1.0, 7, device) for k_ in (4096, 11008)}
+            ys_ = {n_: torch.empty((mm, n_), dtype=torch.float32, device=device) for n_ in (4096, 11008)}
+
+            def bf_pass():
+                for lay in wl:
+                    for w_ in lay:
+                        mxq.mxq_linear_bf16(xk[w_.shape[1]], w_, out=ys_[w_.shape[0]])
+            tb = time_graph(bf_pass, 10) / nl
+            nbytes = sum(n_ * k_ * 2 + 2 * mm * k_ + 4 * mm * n_ for n_, k_ in shapes7)
+            bf["7B_layer_set_m%d" % mm] = {"us_per_layer_set": tb * 1e6, "gbs": nbytes / tb / 1e9, "bytes": nbytes}
+            del wl
+        bf["status"] = mxq.mxq_linear_device_status()
+        extra["bf16_weights"] = bf
         # direct cast throughput (2 B read + 0.53125 B written per weight)
         w = synth.student_t_bf16((11008, 4096), 0.02, 1, device=device)
         ws_ = [w.clone() for _ in range(4)]   # 360 MB rotated: larger than L2

@@ -136,7 +136,7 @@ int mxq_linear_plan_info(int kernel, int M, int64_t N, int64_t K, int32_t *info)
 /* Copies to *status_host, and then clears, the sticky device words in which the tcgen05 kernels record a
  * bounded wait that gave up (bit 0: data of a stage never arrived, bit 1: a stage was never released,
  * bit 2: the accumulator never completed, bit 3: a prefetched stage never landed; bits 0-3 for
- * MXQ_KERNEL_UMMA, bits 8-11 the same for MXQ_KERNEL_FP4).  0 in normal
+ * MXQ_KERNEL_UMMA, bits 8-11 the same for MXQ_KERNEL_FP4, bits 16-20 for mxq_linear_bf16).  0 in normal
  * operation; a non-zero word means the affected output tiles were written as NaN.  Synchronises with
  * the device (a blocking copy), so call it outside the hot loop. */
 int mxq_linear_device_status(uint32_t *status_host);
@@ -209,6 +209,13 @@ size_t mxq_greedy_accept_static_max_bytes(void);
 /* Same, with the verifier's tokens already known: verifier [B][R] int32. */
 int mxq_greedy_accept_tokens(const int32_t *draft, const int32_t *verifier, int64_t B, int T, int R,
                              int32_t *accept_len, int32_t *next_token, void *stream);
+
+/* The same layer with the weights NOT quantised: Y[m][n] = sum_k X[m][k] * W[n][k], W [N][K] BF16 row-major.  The
+ * comparison point of the paper (Sec. III-D-3: 16 / 4.25 = 3.76 times the bytes of MXFP4; Sec. IV-D measures both),
+ * so that the gain of the cast can be measured on this machine.  1 <= M <= 16, K even; FP32 accumulation of exact
+ * products; K % 64 == 0 runs on the tensor cores, anything else on a plain kernel.  Bounded waits that give up are
+ * reported by mxq_linear_device_status in bits 16-20. */
+int mxq_linear_bf16(const void *X_bf16, int M, const void *W_bf16, int64_t N, int64_t K, void *Y, int y_dtype, void *stream);
 
 /* Vocabulary projection fused with the greedy verification: logits = X . w^[V][K]^T (mxq_linear with N = V), the
  * argmax of every row and the walk over the draft in ONE launch; the logits are never written (Sec. III-A, III-B:

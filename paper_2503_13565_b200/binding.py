@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
             L.mxq_greedy_accept_static_max_bytes.argtypes = []
             L.mxq_greedy_accept_tokens.restype = i32
             L.mxq_greedy_accept_tokens.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp]
+            L.mxq_linear_bf16.restype = i32
+            L.mxq_linear_bf16.argtypes = [vp, i32, vp, i64, i64, vp, i32, vp]
             L.mxq_lm_head_accept_workspace_bytes.restype = sz
             L.mxq_lm_head_accept_workspace_bytes.argtypes = [i32, i64, i64]
             L.mxq_lm_head_accept.restype = i32
@@ -328,3 +330,14 @@ def mxq_lm_head_accept(x: torch.Tensor, codes: torch.Tensor, scales: torch.Tenso
                                     _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)),
            "mxq_lm_head_accept")
     return verifier, g, nxt
+
+
+def mxq_linear_bf16(x: torch.Tensor, w: torch.Tensor, out: torch.Tensor = None, out_dtype=torch.float32, stream=None) -> torch.Tensor:
+    """Y[M,N] = X[M,K] . W[N,K]^T with W in BF16 (not quantised): the comparison point for mxq_linear."""
+    m, k = x.shape
+    n = w.shape[0]
+    if out is None:
+        out = torch.empty((m, n), dtype=out_dtype, device=x.device)
+    _check(lib().mxq_linear_bf16(_dev(x, torch.bfloat16, "x"), m, _dev(w, torch.bfloat16, "w"), n, k,
+                                 _dev(out, out.dtype, "out"), _dt(out.dtype), _stream(stream)), "mxq_linear_bf16")
+    return out

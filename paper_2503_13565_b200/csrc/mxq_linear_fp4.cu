@@ -598,7 +598,26 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
             }
             TR(6);
             const float poison = s_fail ? __uint_as_float(0x7FC00000u) : 0.f;
-            if ((split & (split - 1)) == 0) {
+            // (Funnelling the few results of a one-token call through one warp, so that only one warp has stores in flight
+            // when the CTA ends, was measured: the serial sums cost more than the shorter launch-to-launch gap saves.)
+            const int total = ntile * M * row_cnt;
+            if ((split & (split - 1)) != 0) {
+                for (int idx = ct; idx < total; idx += 128) {
+                    const int t = idx / (M * row_cnt), rem = idx - t * (M * row_cnt);
+                    const int m = rem / row_cnt, r = rem - m * row_cnt;
+                    float acc = 0.f;
+                    for (int j = 0; j < split; ++j) acc += gRecv[((t * split + j) * M + m) * cnt_max + r];
+                    const int64_t n = n0 + (int64_t)t * kFp4TileRows + row_lo + r;
+                    if (n < N) {
+                        if (fa.keys) {
+                            const unsigned long long key = argmax_key(acc * kGuardUp + poison, (uint32_t)n);
+                            if (key) atomicMax(s_keys + m, key);   // (rare decomposition: straight into shared memory)
+                        } else {
+                            store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison);
+                        }
+                    }
+                }
+            } else {
                 // power-of-two cluster: one value per thread (row ct / split, sender ct % split), butterfly sum over the
                 // senders in neighbouring lanes; the order of additions is fixed by the lane pattern
                 const int r = ct / split, j = ct & (split - 1);
@@ -626,22 +645,6 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                                     store_out(Y, y_dtype, (int64_t)m * N + n, w);
                                 }
                             }
-                    }
-                }
-            } else {
-                for (int idx = ct; idx < ntile * M * row_cnt; idx += 128) {
-                    const int t = idx / (M * row_cnt), rem = idx - t * (M * row_cnt);
-                    const int m = rem / row_cnt, r = rem - m * row_cnt;
-                    float acc = 0.f;
-                    for (int j = 0; j < split; ++j) acc += gRecv[((t * split + j) * M + m) * cnt_max + r];
-                    const int64_t n = n0 + (int64_t)t * kFp4TileRows + row_lo + r;
-                    if (n < N) {
-                        if (fa.keys) {
-                            const unsigned long long key = argmax_key(acc * kGuardUp + poison, (uint32_t)n);
-                            if (key) atomicMax(s_keys + m, key);   // (rare decomposition: straight into shared memory)
-                        } else {
-                            store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison);
-                        }
                     }
                 }
             }

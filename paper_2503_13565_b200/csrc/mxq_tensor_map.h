@@ -16,4 +16,8 @@ bool tensor_map_available();
 // Maps depend only on (device, pointer, N, K, kind); recent ones are cached.  False if encoding fails.
 bool codes_tensor_map(const uint8_t *codes, int64_t N, int64_t K, bool expand_fp4, CUtensorMap *out);
 
+// A map over a BF16 matrix [rows][K] (K % 64 == 0, 16-byte aligned base) whose box is box_rows rows x 64 elements
+// (128 bytes), 128-byte swizzled; rows of the box beyond the matrix read as zeros.  Cached like the maps above.
+bool bf16_tensor_map(const void *base, int64_t rows, int64_t K, int box_rows, CUtensorMap *out);
+
 }  // namespace mxq

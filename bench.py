@@ -404,6 +404,80 @@ def run_ours(args):
             del wl
         bf["status"] = mxq.mxq_linear_device_status()
         extra["bf16_weights"] = bf
+        # Speculative decoding with the quantised draft (Sec. III-B): a 4-layer slice of the 7B stack plus a 32000-row
+        # vocabulary projection, target in BF16, draft = its MXFP4 cast; acceptance is simulated (random weights accept
+        # nothing), the kernels and the control flow are real.  Measured tokens per second against Eq. 1 fed with the measured S.
+        import random as _random
+        from paper_2503_13565_b200 import specdec
+        nl_, n_draft = 4, 8
+        tw = [[synth.normal_bf16((n_, k_), 0.02, 300 + 10 * li + j, device) for j, (n_, k_) in enumerate(shapes7)] for li in range(nl_)]
+        th = synth.normal_bf16((32000, 4096), 0.02, 399, device)
+        dq = [[mxq.mxq_quantize(w_) for w_ in lay] for lay in tw]
+        dh = mxq.mxq_quantize(th)
+        xs_ = {(r_, k_): synth.normal_bf16((r_, k_), 1.0, 9, device) for r_ in (1, n_draft + 1) for k_ in (4096, 11008)}
+        yo_ = {(r_, n_): torch.empty((r_, n_), dtype=torch.float32, device=device) for r_ in (1, n_draft + 1) for n_ in (4096, 11008)}
+        lg_ = {r_: torch.empty((1, r_, 32000), dtype=torch.float32, device=device) for r_ in (1, n_draft + 1)}
+        dr_ = torch.zeros((1, n_draft), dtype=torch.int32, device=device)
+        wsa_ = mxq.new_workspace(mxq.mxq_accept_workspace_bytes(1, n_draft + 1, 32000), device)
+        wsf_ = mxq.new_workspace(mxq.mxq_lm_head_accept_workspace_bytes(1, 32000, 4096), device)
+
+        def target_step(r_):
+            for lay in tw:
+                for w_ in lay:
+                    mxq.mxq_linear_bf16(xs_[(r_, w_.shape[1])], w_, out=yo_[(r_, w_.shape[0])])
+            mxq.mxq_linear_bf16(xs_[(r_, 4096)], th, out=lg_[r_][0])
+            mxq.mxq_greedy_accept(lg_[r_], dr_[:, :max(r_ - 1, 1)], workspace=wsa_)
+
+        def draft_step():
+            for lay in dq:
+                for (c_, s_) in lay:
+                    mxq.mxq_linear(xs_[(1, c_.shape[1] * 2)], c_, s_, out=yo_[(1, c_.shape[0])], workspace=self_ws)
+            mxq.mxq_lm_head_accept(xs_[(1, 4096)], dh[0], dh[1], None, workspace=wsf_)
+        self_ws = mxq.new_workspace(16, device)
+        st_ = torch.cuda.Stream()
+        graphs = {}
+        with torch.cuda.stream(st_):
+            for name_, fn_ in (("t1", lambda: target_step(1)), ("tv", lambda: target_step(n_draft + 1)), ("d", draft_step)):
+                fn_()
+                st_.synchronize()
+                g_ = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_, stream=st_):
+                    fn_()
+                graphs[name_] = g_
+
+            def timed(launch, reps):
+                for _ in range(2):
+                    launch()
+                st_.synchronize()
+                e0_, e1_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0_.record(st_)
+                for _ in range(reps):
+                    launch()
+                e1_.record(st_)
+                st_.synchronize()
+                return e0_.elapsed_time(e1_) * 1e-3 / reps
+            t_t1 = timed(graphs["t1"].replay, 20)
+            t_tv = timed(graphs["tv"].replay, 20)
+            t_d = timed(graphs["d"].replay, 20)
+            sd = {"layers": nl_, "draft_tokens_per_round": n_draft, "target_step_us": t_t1 * 1e6, "target_verify_us": t_tv * 1e6,
+                  "draft_step_us": t_d * 1e6, "S": t_t1 / t_d, "runs": {}}
+            for p_ in (0.7, 0.9):
+                rng_ = _random.Random(1)
+                steps_ = []
+                tally = specdec.simulate(2, [n_draft], lambda lvl, k_: specdec.leading_successes(rng_, p_, k_), tokens=400,
+                                         on_step=lambda lvl, rows: steps_.append("d" if lvl == 1 else "tv"))
+
+                def run_all():
+                    for nm in steps_:
+                        graphs[nm].replay()
+                t_all = timed(run_all, 3)
+                produced = tally.accepted[0] + tally.steps[0]
+                alpha_ = tally.accepted[0] / tally.proposed[0]
+                sd["runs"]["p=%.1f" % p_] = {"alpha": alpha_, "tokens": produced, "us_per_token": t_all / produced * 1e6,
+                                             "speedup_measured": produced * t_t1 / t_all,
+                                             "speedup_eq1": specdec.eq1_speedup(alpha_, n_draft, t_t1 / t_d)}
+        extra["specdec"] = sd
+        del tw, th, dq, dh
         # direct cast throughput (2 B read + 0.53125 B written per weight)
         w = synth.student_t_bf16((11008, 4096), 0.02, 1, device=device)
         ws_ = [w.clone() for _ in range(4)]   # 360 MB rotated: larger than L2

@@ -108,6 +108,25 @@ def test_config4_lm_head_sampled_rows(m):
     run_case(w, x, rows=rows, what="lm_head M=%d" % m)
 
 
+@pytest.mark.parametrize("m,n", [(1, 128256), (2, 128256), (4, 128256), (8, 128256), (16, 128256), (16, 50304), (3, 64000)])
+def test_largest_vocabularies_sampled_rows(m, n):
+    """The launch configurations of the largest projections bench.py times: one CTA per SM walking up to 14 tiles, the
+    token operand resident or riding the ring.  Codes and scale bytes are drawn directly (seeded), so no cast of half a
+    billion weights is needed; the oracle checks a seeded sample of rows from every part of the matrix."""
+    k = 4096
+    g = torch.Generator().manual_seed(1000 * 4 + m)
+    codes = torch.randint(0, 256, (n, k // 2), dtype=torch.uint8, generator=g)
+    scales = torch.randint(110, 126, (n, k // 32), dtype=torch.uint8, generator=g)
+    x = synth.bits_of(synth.activations(4, 1, m, k))
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, n - 129, n - 128, n - 1],
+                                     np.random.default_rng(m).integers(0, n, 250)])).astype(np.int64)
+    y64, a64 = oracle.linear(x, codes.numpy(), scales.numpy(), rows=rows)
+    ws = mxq.new_workspace(mxq.mxq_linear_workspace_bytes(m, n, k))
+    y = mxq.mxq_linear(gpu_bf16(x), codes.cuda(), scales.cuda(), workspace=ws)
+    torch.cuda.synchronize()
+    check_linear(y[:, torch.as_tensor(rows, device="cuda")], y64, a64, "vocabulary %d M=%d" % (n, m))
+
+
 def test_bf16_output_is_the_rounded_fp32_output():
     w = synth.bits_of(synth.weight(3, 11, 515, 2048))
     x = synth.bits_of(synth.activations(3, 11, 5, 2048))

@@ -70,7 +70,8 @@ def test_fused_equals_composed_oracle(r, t, v, k):
         run(r, v, k, t, seed=r + t, accept_upto=upto)
 
 
-@pytest.mark.parametrize("r,t,v", [(1, 0, 32000), (2, 1, 32000), (5, 4, 32000), (9, 8, 32000), (1, 0, 48000), (3, 2, 48000)])
+@pytest.mark.parametrize("r,t,v", [(1, 0, 32000), (2, 1, 32000), (5, 4, 32000), (9, 8, 32000), (1, 0, 48000), (3, 2, 48000),
+                                   (16, 15, 50304)])
 def test_full_vocabulary_sizes(r, t, v):
     """The launch configurations of the vocabulary projections bench.py times (one CTA per SM walking several tiles)."""
     k = 4096

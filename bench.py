@@ -277,9 +277,33 @@ def cpu_baseline_leg(m: int, budget_s: float = 15.0):
             oracle.linear(x, codes, scales)
         t_total += time.perf_counter() - t0
         reps += 1
-    return {"value": nbytes * reps / t_total / 1e9, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-            "sample": "%d pass(es) over one 7B layer set (7 matrices, 202M weights) at M=%d, FP64" % (reps, m),
-            "us_per_layer_set": t_total / reps * 1e6}
+    out = {"value": nbytes * reps / t_total / 1e9, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+           "sample": "%d pass(es) over one 7B layer set (7 matrices, 202M weights) at M=%d, FP64" % (reps, m),
+           "us_per_layer_set": t_total / reps * 1e6}
+    # beside it, each once: the same layer set at eight token rows and on one thread, and the cast of one 4096 x 4096 matrix
+    cores = oracle.threads()
+    try:
+        x8 = {k: synth.bits_of(synth.normal_bf16((8, k), 1.0, 9)) for k in (4096, 11008)}
+        t0 = time.perf_counter()
+        for n, k, codes, scales, _ in mats:
+            oracle.linear(x8[k], codes, scales)
+        out["m8_us_per_layer_set"] = (time.perf_counter() - t0) * 1e6
+        oracle.set_threads(1)
+        t0 = time.perf_counter()
+        n, k, codes, scales, x = mats[0]
+        oracle.linear(x, codes, scales)
+        out["one_thread_us_4096x4096_m%d" % m] = (time.perf_counter() - t0) * 1e6
+        w = synth.bits_of(synth.normal_bf16((4096, 4096), 0.02, 3))
+        t0 = time.perf_counter()
+        oracle.quantize(w)
+        out["one_thread_quantize_us_4096x4096"] = (time.perf_counter() - t0) * 1e6
+        oracle.set_threads(cores)
+        t0 = time.perf_counter()
+        oracle.quantize(w)
+        out["quantize_us_4096x4096"] = (time.perf_counter() - t0) * 1e6
+    finally:
+        oracle.set_threads(cores)
+    return out
 
 
 def run_ours(args):

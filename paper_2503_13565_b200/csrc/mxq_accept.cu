@@ -82,7 +82,32 @@ greedy_accept_kernel(const T *__restrict__ logits, int64_t B, int R, int64_t V, 
     if (vec_ok) {
         const int64_t nvec = (hi - lo) / kVec;  // lo is a multiple of kSliceQuantum, rows are 16-byte aligned
         const uint4 *pv = reinterpret_cast<const uint4 *>(p + lo);
-        for (int64_t i = threadIdx.x; i < nvec; i += kAcceptThreads) {
+        // four 16-byte loads in flight per lane (ascending index order is kept, so ties still go to the lowest index)
+        int64_t i = threadIdx.x;
+        for (; i + 3 * kAcceptThreads < nvec; i += 4 * kAcceptThreads) {
+            uint4 q4[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) q4[u] = ld_stream_u4(pv + i + u * kAcceptThreads);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint4 q = q4[u];
+                const int base = (int)(lo + (i + u * kAcceptThreads) * kVec);
+                if constexpr (sizeof(T) == 4) {
+                    consider(best, __uint_as_float(q.x), base);
+                    consider(best, __uint_as_float(q.y), base + 1);
+                    consider(best, __uint_as_float(q.z), base + 2);
+                    consider(best, __uint_as_float(q.w), base + 3);
+                } else {
+                    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        consider(best, __uint_as_float(w[j] << 16), base + 2 * j);
+                        consider(best, __uint_as_float(w[j] & 0xFFFF0000u), base + 2 * j + 1);
+                    }
+                }
+            }
+        }
+        for (; i < nvec; i += kAcceptThreads) {
             const uint4 q = ld_stream_u4(pv + i);
             const int base = (int)(lo + i * kVec);
             if constexpr (sizeof(T) == 4) {

@@ -566,7 +566,7 @@ def run_case(args):
     mxq.binding.lib()
     device = torch.device("cuda", 0)
     case = args.case.lower()
-    if case.startswith("quantize:") or case.startswith("accept:"):
+    if case.startswith("quantize:") or case.startswith("accept:") or case.startswith("bf16:"):
         return run_case_other(mxq, case, args.steps, device)
     n, k, m = (int(v) for v in case.split("x"))
     nbytes = algorithmic_bytes(m, n, k)
@@ -593,8 +593,9 @@ def run_case(args):
 
 
 def run_case_other(mxq, case: str, steps: int, device):
-    """--case quantize:NxK (direct cast of `steps` distinct BF16 matrices, rotated) or accept:BxRxV (greedy accept of
-    FP32 logits, T = R - 1): the small cases profiler captures of those kernels run on."""
+    """--case quantize:NxK (direct cast of `steps` distinct BF16 matrices, rotated), accept:BxRxV (greedy accept of FP32
+    logits, T = R - 1) or bf16:NxKxM (the unquantised comparison layer): the small cases profiler captures of those
+    kernels run on."""
     op, dims = case.split(":")
     dims = [int(v) for v in dims.split("x")]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -615,6 +616,24 @@ def run_case_other(mxq, case: str, steps: int, device):
         def all_copies():
             for w_ in ws_:
                 mxq.mxq_quantize(w_, codes, scales)
+        graph_us = time_graph(all_copies, 10) / copies * 1e6
+    elif op == "bf16":
+        n, k, m = dims
+        copies = max(2, min(8, int(400e6 // (n * k * 2)) + 1))
+        ws_ = [synth.normal_bf16((n, k), 0.02, 1 + i, device=device) for i in range(copies)]
+        x = synth.normal_bf16((m, k), 1.0, 3, device)
+        y = torch.empty((m, n), dtype=torch.float32, device=device)
+        mxq.mxq_linear_bf16(x, ws_[0], out=y)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(steps):
+            mxq.mxq_linear_bf16(x, ws_[i % copies], out=y)
+        e1.record()
+        nbytes = n * k * 2 + 2 * m * k + 4 * m * n
+
+        def all_copies():
+            for w_ in ws_:
+                mxq.mxq_linear_bf16(x, w_, out=y)
         graph_us = time_graph(all_copies, 10) / copies * 1e6
     else:
         b, r, v = dims

@@ -37,8 +37,9 @@ uint32_t smem_bytes(int M, int chunk, int ring, int split) {
     return 1024u + (uint32_t)ring * kStageBytes + (uint32_t)chunk * kXStageBytes + recv + (uint32_t)(2 * ring + 3) * 8u + 16u;
 }
 
-// One tile per CTA; the split that brings the grid closest to two CTAs per SM (never 7); the deepest ring up to 6 that
-// keeps two CTAs on an SM.
+// One tile per CTA, two CTAs per SM, ring of up to 6 stages.  Few tiles (layer-sized matrices): the split that brings the
+// grid closest to two CTAs per SM (never 7).  Many tiles: several waves of CTAs; the smallest split whose K range of X
+// (2 KB per stage: a 16-row box) still leaves three ring slots.
 bool layout(Bf16Plan &p, int sms) {
     long best = -1;
     const int smax = p.ks < kMaxSplit ? p.ks : kMaxSplit;
@@ -49,9 +50,11 @@ bool layout(Bf16Plan &p, int sms) {
         while (ring > 1 && smem_bytes(p.M, chunk, ring, s) > 113u * 1024u) --ring;
         if (smem_bytes(p.M, chunk, ring, s) > kSmemLimit) continue;
         const long ctas = (long)p.tiles * s;
-        const long off = ctas > 2L * sms ? (p.tiles > 2 * sms ? (long)s * 1000 : ctas - 2L * sms) : 2L * sms - ctas;
-        if (best < 0 || off <= best) {
-            best = off;
+        const long shallow = (ring < 3 && ring < chunk) ? (long)(3 - ring) * 100000 : 0;   // a ring that cannot cover the latency
+        const long off = ctas > 2L * sms ? (long)s * 1000 : 2L * sms - ctas;
+        const long cost = shallow + off;
+        if (best < 0 || cost < best || (cost == best && ctas <= 2L * sms)) {
+            best = cost;
             p.split = s;
             p.ring = ring;
             p.chunk_max = chunk;

@@ -500,6 +500,59 @@ def run_ours(args):
                 sd["runs"]["p=%.1f" % p_] = {"alpha": alpha_, "tokens": produced, "us_per_token": t_all / produced * 1e6,
                                              "speedup_measured": produced * t_t1 / t_all,
                                              "speedup_eq1": specdec.eq1_speedup(alpha_, n_draft, t_t1 / t_d)}
+            # Two levels (Sec. III-C): a tiny draft (2 layers of the 68M-like shapes, MXFP4) drafts for the MXFP4 model, which
+            # verifies with 9 rows and in turn drafts for the BF16 target.
+            n_tiny = 4
+            tiny_shapes = [(768, 768)] * 4 + [(3072, 768)] * 2 + [(768, 3072)]
+            tq = [[mxq.mxq_quantize(synth.normal_bf16((n_, k_), 0.02, 500 + 10 * li + j, device)) for j, (n_, k_) in enumerate(tiny_shapes)]
+                  for li in range(2)]
+            tqh = mxq.mxq_quantize(synth.normal_bf16((32000, 768), 0.02, 599, device))
+            xt_ = {k_: synth.normal_bf16((1, k_), 1.0, 11, device) for k_ in (768, 3072)}
+            yt_ = {n_: torch.empty((1, n_), dtype=torch.float32, device=device) for n_ in (768, 3072)}
+            wsf_t = mxq.new_workspace(mxq.mxq_lm_head_accept_workspace_bytes(1, 32000, 768), device)
+            rv = n_tiny + 1
+            xv_ = {k_: synth.normal_bf16((rv, k_), 1.0, 12, device) for k_ in (4096, 11008)}
+            yv_ = {n_: torch.empty((rv, n_), dtype=torch.float32, device=device) for n_ in (4096, 11008)}
+            wsv = mxq.new_workspace(max(mxq.mxq_linear_workspace_bytes(rv, n_, k_) for n_, k_ in shapes7), device)
+            wsfv = mxq.new_workspace(mxq.mxq_lm_head_accept_workspace_bytes(rv, 32000, 4096), device)
+            drv = torch.zeros(n_tiny, dtype=torch.int32, device=device)
+
+            def tiny_step():
+                for lay in tq:
+                    for (c_, s_) in lay:
+                        mxq.mxq_linear(xt_[c_.shape[1] * 2], c_, s_, out=yt_[c_.shape[0]], workspace=self_ws)
+                mxq.mxq_lm_head_accept(xt_[768], tqh[0], tqh[1], None, workspace=wsf_t)
+
+            def draft_verify():   # the MXFP4 model checks the tiny draft's n_tiny tokens in one pass of n_tiny + 1 rows
+                for lay in dq:
+                    for (c_, s_) in lay:
+                        mxq.mxq_linear(xv_[c_.shape[1] * 2], c_, s_, out=yv_[c_.shape[0]], workspace=wsv)
+                mxq.mxq_lm_head_accept(xv_[4096], dh[0], dh[1], drv, workspace=wsfv)
+            for name_, fn_ in (("y", tiny_step), ("dv", draft_verify)):
+                fn_()
+                st_.synchronize()
+                g_ = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_, stream=st_):
+                    fn_()
+                graphs[name_] = g_
+            t_y = timed(graphs["y"].replay, 20)
+            t_dv = timed(graphs["dv"].replay, 20)
+            p_lv = [0.9, 0.6]
+            rng_ = _random.Random(2)
+            steps_ = []
+            tally = specdec.simulate(3, [n_draft, n_tiny], lambda lvl, k_: specdec.leading_successes(rng_, p_lv[lvl], k_), tokens=400,
+                                     on_step=lambda lvl, rows: steps_.append({0: "tv", 1: "dv", 2: "y"}[lvl]))
+
+            def run_all2():
+                for nm in steps_:
+                    graphs[nm].replay()
+            t_all = timed(run_all2, 3)
+            produced = tally.accepted[0] + tally.steps[0]
+            alphas = [tally.accepted[i] / tally.proposed[i] for i in range(2)]
+            sd["two_level"] = {"tiny_step_us": t_y * 1e6, "draft_verify_us": t_dv * 1e6, "tiny_tokens_per_round": n_tiny,
+                               "p": p_lv, "alpha": alphas, "tokens": produced, "us_per_token": t_all / produced * 1e6,
+                               "speedup_measured": produced * t_t1 / t_all,
+                               "speedup_nested_eq1": specdec.multilevel_speedup([t_t1, t_d, t_y], [n_draft, n_tiny], alphas)}
         extra["specdec"] = sd
         del tw, th, dq, dh
         # direct cast throughput (2 B read + 0.53125 B written per weight)

@@ -8,8 +8,9 @@ package imports nothing from here.
 All tensors cross this boundary as numpy arrays: BF16 data as ``uint16`` bit
 patterns, codes and scales as ``uint8``, results as ``float64`` / ``int32``.
 The arithmetic is all in the C file; this module only compiles it on first
-use, marshals arguments and allocates outputs (one exception: ``linear_bf16``, the unquantised comparison layer,
-is the textbook matrix product and is written with numpy here).
+use, marshals arguments and allocates outputs (exceptions, written with numpy here: ``linear_bf16``, the unquantised
+comparison layer, is the textbook matrix product; ``silu``, ``linear_residual`` and ``linear_swiglu`` apply an
+elementwise formula to the outputs of ``linear``).
 """
 from __future__ import annotations
 
@@ -139,6 +140,38 @@ def linear_bf16(x_bits: np.ndarray, w_bits: np.ndarray, rows=None):
         wb = wb[np.asarray(rows, dtype=np.int64)]
     w = (wb.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
     return x @ w.T, np.abs(x) @ np.abs(w).T
+
+
+def silu(g: np.ndarray) -> np.ndarray:
+    """silu(g) = g * sigmoid(g) = g / (1 + e^-g), float64: the activation of the gated feed-forward block of the
+    Llama-family models the paper evaluates (Sec. IV-A).  Written in the form that cannot overflow: for g < 0 the
+    quotient is taken as g e^g / (1 + e^g)."""
+    g = np.asarray(g, np.float64)
+    e = np.exp(-np.abs(g))                       # in (0, 1]
+    return np.where(g >= 0, g / (1.0 + e), g * e / (1.0 + e))
+
+
+def linear_residual(x_bits: np.ndarray, codes: np.ndarray, scales: np.ndarray, residual: np.ndarray, rows=None):
+    """The layer with the residual add fused into its output (Sec. III-D-2 lists the residual add among the operators
+    fused into the linear layers): out[m, n] = residual[m, n] + sum_k x[m, k] w^[n, k], float64, and A as ``linear``.
+    ``residual`` is [M, N] (or [M, len(rows)] with ``rows``) as float64 values."""
+    y, a = linear(x_bits, codes, scales, rows)
+    r = np.asarray(residual, np.float64)
+    assert r.shape == y.shape
+    return y + r, a
+
+
+def linear_swiglu(x_bits: np.ndarray, codes: np.ndarray, scales: np.ndarray, rows=None):
+    """Gate and up projections of the gated feed-forward block as ONE matrix of 2F rows, row 2i = gate row i and row
+    2i + 1 = up row i: out[m, i] = silu(g[m, i]) * u[m, i] with g, u the two plain layer outputs.  Returns
+    (out, g, u, a_g, a_u), all [M, F] float64 (a_* = sum_k |x w^| of the two rows, for error bounds).
+    ``rows``: optional list of output columns i."""
+    n = np.asarray(codes).shape[0]
+    assert n % 2 == 0
+    idx = np.arange(n // 2, dtype=np.int64) if rows is None else np.asarray(rows, dtype=np.int64)
+    g, ag = linear(x_bits, codes, scales, 2 * idx)
+    u, au = linear(x_bits, codes, scales, 2 * idx + 1)
+    return silu(g) * u, g, u, ag, au
 
 
 def _logits_arg(logits: np.ndarray):

@@ -235,6 +235,25 @@ int mxq_lm_head_accept(const void *X_bf16, int R, const uint8_t *codes, const ui
                        const int32_t *draft, int T, int32_t *verifier, int32_t *accept_len, int32_t *next_token,
                        void *workspace, size_t workspace_bytes, void *stream);
 
+/* The layer with one more step fused into its output (Sec. III-D-2 names the residual add among the operators
+ * fused into the linear layers; the gate / up pairing is the feed-forward block of the Llama-family models of
+ * Sec. IV-A).  Arguments as mxq_linear, plus:
+ *   mxq_linear_residual   Y[m][n] = residual[m][n] + sum_k X[m][k] w^[n][k].  residual [M][N] row-major in Y's type
+ *                         (device, 16-byte aligned, read); it may be Y itself (in-place add).
+ *   mxq_linear_swiglu     W holds the gate and up projections interleaved by rows: row 2i = gate row i, row 2i+1 = up
+ *                         row i (N = 2F even).  Y[m][i] = silu(g) * u with g, u the FP32 sums of rows 2i and 2i+1 and
+ *                         silu(g) = g / (1 + e^-g) evaluated in FP32; Y is [M][N/2].
+ *   workspace  REQUIRED: device memory, >= mxq_linear_fused_workspace_bytes(M, N, K), 16-byte aligned, no
+ *              initialisation needed, contents are scratch; one per stream.
+ * On the tcgen05 kernels (K % 128 == 0) the step runs in the kernel's epilogue and the sums never reach memory;
+ * elsewhere the plain layer writes its FP32 sums into the workspace and a small kernel finishes them.  Errors as
+ * mxq_linear; MXQ_ERR_WORKSPACE for a workspace that is too small, MXQ_ERR_SHAPE for an odd N in mxq_linear_swiglu. */
+size_t mxq_linear_fused_workspace_bytes(int M, int64_t N, int64_t K);
+int mxq_linear_residual(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
+                        const void *residual, void *Y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream);
+int mxq_linear_swiglu(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
+                      void *Y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -76,6 +76,12 @@ def lib() -> ctypes.CDLL:
             L.mxq_greedy_accept_tokens.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp]
             L.mxq_linear_bf16.restype = i32
             L.mxq_linear_bf16.argtypes = [vp, i32, vp, i64, i64, vp, i32, vp]
+            L.mxq_linear_fused_workspace_bytes.restype = sz
+            L.mxq_linear_fused_workspace_bytes.argtypes = [i32, i64, i64]
+            L.mxq_linear_residual.restype = i32
+            L.mxq_linear_residual.argtypes = [vp, i32, vp, vp, i64, i64, vp, vp, i32, vp, sz, vp]
+            L.mxq_linear_swiglu.restype = i32
+            L.mxq_linear_swiglu.argtypes = [vp, i32, vp, vp, i64, i64, vp, i32, vp, sz, vp]
             L.mxq_lm_head_accept_workspace_bytes.restype = sz
             L.mxq_lm_head_accept_workspace_bytes.argtypes = [i32, i64, i64]
             L.mxq_lm_head_accept.restype = i32
@@ -341,3 +347,50 @@ def mxq_linear_bf16(x: torch.Tensor, w: torch.Tensor, out: torch.Tensor = None, 
     _check(lib().mxq_linear_bf16(_dev(x, torch.bfloat16, "x"), m, _dev(w, torch.bfloat16, "w"), n, k,
                                  _dev(out, out.dtype, "out"), _dt(out.dtype), _stream(stream)), "mxq_linear_bf16")
     return out
+
+
+def mxq_linear_fused_workspace_bytes(m: int, n: int, k: int) -> int:
+    return int(lib().mxq_linear_fused_workspace_bytes(m, n, k))
+
+
+def mxq_linear_residual(x: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, residual: torch.Tensor,
+                        out: torch.Tensor = None, workspace: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """Y[M,N] = residual[M,N] + X[M,K] . dequant(W)^T in one launch.  ``residual`` is FP32 or BF16 and fixes Y's type;
+    ``out`` may be ``residual`` itself (in-place add).  ``workspace``: uint8, at least
+    ``mxq_linear_fused_workspace_bytes(M, N, K)`` bytes (allocated here if None: pass one in a hot loop)."""
+    m, k = x.shape
+    n = codes.shape[0]
+    if out is None:
+        out = torch.empty((m, n), dtype=residual.dtype, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(max(16, mxq_linear_fused_workspace_bytes(m, n, k)), dtype=torch.uint8, device=x.device)
+    _check(lib().mxq_linear_residual(_dev(x, torch.bfloat16, "x"), m, _dev(codes, torch.uint8, "codes"),
+                                     _dev(scales, torch.uint8, "scales"), n, k, _dev(residual, out.dtype, "residual"),
+                                     _dev(out, out.dtype, "out"), _dt(out.dtype),
+                                     _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)),
+           "mxq_linear_residual")
+    return out
+
+
+def mxq_linear_swiglu(x: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, out: torch.Tensor = None,
+                      out_dtype=torch.bfloat16, workspace: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """Y[M,F] = silu(X . gate^T) * (X . up^T) in one launch; ``codes`` / ``scales`` are the MXFP4 pair of the [2F,K]
+    matrix whose row 2i is gate row i and row 2i+1 up row i (``interleave_gate_up``)."""
+    m, k = x.shape
+    n = codes.shape[0]
+    if out is None:
+        out = torch.empty((m, n // 2), dtype=out_dtype, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(max(16, mxq_linear_fused_workspace_bytes(m, n, k)), dtype=torch.uint8, device=x.device)
+    _check(lib().mxq_linear_swiglu(_dev(x, torch.bfloat16, "x"), m, _dev(codes, torch.uint8, "codes"),
+                                   _dev(scales, torch.uint8, "scales"), n, k, _dev(out, out.dtype, "out"), _dt(out.dtype),
+                                   _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)),
+           "mxq_linear_swiglu")
+    return out
+
+
+def interleave_gate_up(gate: torch.Tensor, up: torch.Tensor) -> torch.Tensor:
+    """[F,C] gate and up arrays (BF16 weights, or their codes or scales: the cast works row by row) -> the [2F,C] array
+    mxq_linear_swiglu expects: row 2i = gate[i], row 2i+1 = up[i].  A copy, no arithmetic."""
+    assert gate.shape == up.shape and gate.dtype == up.dtype
+    return torch.stack((gate, up), dim=1).reshape(2 * gate.shape[0], gate.shape[1]).contiguous()

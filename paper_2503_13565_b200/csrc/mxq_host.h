@@ -27,7 +27,14 @@ struct FusedAccept {
     int32_t *accept_len;        // [1] out: G
     int32_t *next_token;        // [1] out: the verifier's token at position G, -1 if there is no such row
     int T;
+    // Layer epilogues (keys == nullptr; Sec. III-D-2: operators fused into the linear layers).  A finished sum is
+    // stored after one more step:
+    const void *residual;       // [M][N] in Y's type, added to the sum (may be Y itself); nullptr: none
+    int swiglu;                 // rows 2i / 2i+1 of W are gate / up row i: Y[m][i] = silu(sum 2i) * sum(2i+1), Y is [M][N/2]
 };
+// which epilogue a tcgen05 kernel is compiled for
+enum { kEpiStore = 0, kEpiAccept = 1, kEpiLayer = 2 };
+inline int epilogue_kind(const FusedAccept &fa) { return fa.keys ? kEpiAccept : (fa.residual || fa.swiglu ? kEpiLayer : kEpiStore); }
 
 struct LinearPlan;
 // tensor-core path of mxq_linear (mxq_linear_mma.cu): false if the shape is not covered
@@ -40,7 +47,9 @@ struct UmmaPlan;
 // tcgen05 path of mxq_linear (mxq_linear_umma.cu): false if the shape is not covered
 bool linear_umma_available();
 // with_workspace: plan for a token operand split ahead of the weight kernel (from 3 token rows on)
-bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &plan, bool with_workspace);
+// pow2_split: only cluster sizes that are powers of two (what the gate / up epilogue needs: the two rows of a pair
+// then end up in one warp)
+bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &plan, bool with_workspace, bool pow2_split = false);
 // workspace: optional; with linear_umma_workspace_bytes(M, K) bytes (0: not used for this M) the token operand is split
 // once per call by a kernel of its own instead of by every CTA of the weight kernel
 size_t linear_umma_workspace_bytes(int M, int64_t K);
@@ -50,7 +59,7 @@ cudaError_t linear_umma_launch(const UmmaPlan &plan, const void *X, const uint8_
 
 struct Fp4Plan;
 // tcgen05 path with packed 4-bit operands on both sides, M <= 4 (mxq_linear_fp4.cu)
-bool linear_fp4_plan(int M, int64_t N, int64_t K, Fp4Plan &plan);
+bool linear_fp4_plan(int M, int64_t N, int64_t K, Fp4Plan &plan, bool pow2_split = false);
 cudaError_t linear_fp4_launch(const Fp4Plan &plan, const void *X, const uint8_t *codes, const uint8_t *scales,
                               void *Y, int y_dtype, cudaStream_t stream, const FusedAccept *fused = nullptr);
 int linear_fp4_take_status(uint32_t *out);

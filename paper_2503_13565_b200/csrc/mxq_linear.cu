@@ -102,6 +102,26 @@ static void launch_rowwarp(const void *X, int M, const uint8_t *codes, const uin
                        K, Y, y_dtype);
 }
 
+// The layer epilogues where no tcgen05 kernel covers the call: one thread per output over the plain layer's FP32 sums.
+__global__ void __launch_bounds__(256)
+layer_epilogue_kernel(const float *__restrict__ S, int M, int64_t N, const void *residual, int swiglu, void *Y, int y_dtype) {
+    pdl_trigger();
+    pdl_wait();   // S is the previous kernel's output
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (swiglu) {
+        const int64_t F = N >> 1;
+        if (i >= (int64_t)M * F) return;
+        const int64_t m = i / F, f = i - m * F;
+        const float g = S[m * N + 2 * f], u = S[m * N + 2 * f + 1];
+        store_y(Y, y_dtype, i, g / (1.f + expf(-g)) * u);
+    } else {
+        if (i >= (int64_t)M * N) return;
+        const float r = y_dtype == MXQ_F32 ? reinterpret_cast<const float *>(residual)[i]
+                                           : __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(residual)[i]);
+        store_y(Y, y_dtype, i, S[i] + r);
+    }
+}
+
 // mxq_set_linear_kernel / MXQ_LINEAR_VARIANT: MXQ_KERNEL_AUTO (-1), or the highest kernel mxq_linear may use
 static std::atomic<int> g_ceiling{-2};
 static int kernel_ceiling() {
@@ -133,7 +153,7 @@ struct Choice {
     UmmaPlan umma;
     LinearPlan mma;
 };
-static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *codes, bool with_workspace, Choice &c) {
+static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *codes, bool with_workspace, Choice &c, bool pow2_split = false) {
     const bool tc = linear_umma_available();
     const bool aligned32 = !codes || (reinterpret_cast<uintptr_t>(codes) & 31u) == 0;
     bool try_fp4 = ceiling == MXQ_KERNEL_AUTO || ceiling >= MXQ_KERNEL_FP4;
@@ -147,13 +167,13 @@ static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *code
             // vocabulary-sized matrices, where a CTA per SM walks several tiles: the packed-FP4 kernel still wins at two
             // token rows; above, the FP8-operand kernel, unless its token operand leaves no room for one CTA per SM
             try_fp4 = M == 2;
-            if (M > 2 && !(tc && aligned32 && linear_umma_plan(M, N, K, c.umma, with_workspace) && c.umma.grid <= sm_count()) &&
+            if (M > 2 && !(tc && aligned32 && linear_umma_plan(M, N, K, c.umma, with_workspace, pow2_split) && c.umma.grid <= sm_count()) &&
                 linear_mma_plan(M, N, K, c.mma))
                 try_umma = false;
         }
     }
-    if (try_fp4 && tc && linear_fp4_plan(M, N, K, c.fp4)) c.kernel = MXQ_KERNEL_FP4;
-    else if (try_umma && tc && aligned32 && linear_umma_plan(M, N, K, c.umma, with_workspace)) c.kernel = MXQ_KERNEL_UMMA;
+    if (try_fp4 && tc && linear_fp4_plan(M, N, K, c.fp4, pow2_split)) c.kernel = MXQ_KERNEL_FP4;
+    else if (try_umma && tc && aligned32 && linear_umma_plan(M, N, K, c.umma, with_workspace, pow2_split)) c.kernel = MXQ_KERNEL_UMMA;
     else if (try_mma && linear_mma_plan(M, N, K, c.mma)) c.kernel = MXQ_KERNEL_MMA;
     else c.kernel = MXQ_KERNEL_GENERIC;
 }
@@ -288,7 +308,7 @@ int mxq_lm_head_accept(const void *X_bf16, int R, const uint8_t *codes, const ui
     mxq::Choice c;
     mxq::choose(mxq::kernel_ceiling(), R, V, K, codes, true, c);
     if (c.kernel == MXQ_KERNEL_FP4 || c.kernel == MXQ_KERNEL_UMMA) {
-        mxq::FusedAccept fa;
+        mxq::FusedAccept fa{};
         fa.keys = reinterpret_cast<unsigned long long *>(ws);
         fa.ticket = reinterpret_cast<unsigned int *>(ws + 2048);
         fa.draft = draft;
@@ -320,6 +340,70 @@ int mxq_lm_head_accept(const void *X_bf16, int R, const uint8_t *codes, const ui
         }
     if (T == 0) return mxq_greedy_accept(logits, MXQ_F32, 1, 1, V, minus_one, 1, accept_len, next_token, acc_ws, acc_ws_bytes, stream);
     return mxq_greedy_accept(logits, MXQ_F32, 1, R, V, draft, T, accept_len, next_token, acc_ws, acc_ws_bytes, stream);
+}
+
+// ---- layer epilogues: residual add, gate / up pairing -------------------------------------------------------------------
+// workspace: [mxq_linear's own workspace][FP32 sums of the plain layer, used where no tcgen05 kernel covers the call]
+size_t mxq_linear_fused_workspace_bytes(int M, int64_t N, int64_t K) {
+    if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return 0;
+    return align256(mxq_linear_workspace_bytes(M, N, K)) + align256((size_t)M * (size_t)N * 4u);
+}
+
+static int linear_with_epilogue(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
+                                const void *residual, int swiglu, void *Y, int y_dtype, void *workspace,
+                                size_t workspace_bytes, void *stream) {
+    if (!X_bf16 || !codes || !scales || !Y || !workspace || (!swiglu && !residual)) return MXQ_ERR_NULL;
+    if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K) || (swiglu && (N & 1))) return MXQ_ERR_SHAPE;
+    if (y_dtype != MXQ_F32 && y_dtype != MXQ_BF16) return MXQ_ERR_DTYPE;
+    if (!mxq::aligned16(X_bf16) || !mxq::aligned16(codes) || !mxq::aligned16(scales) || !mxq::aligned16(Y) ||
+        !mxq::aligned16(workspace) || (residual && !mxq::aligned16(residual)))
+        return MXQ_ERR_ALIGN;
+    if (workspace_bytes < mxq_linear_fused_workspace_bytes(M, N, K)) return MXQ_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    const size_t lin_ws_bytes = align256(mxq_linear_workspace_bytes(M, N, K));
+    mxq::Choice c;
+    mxq::choose(mxq::kernel_ceiling(), M, N, K, codes, true, c, swiglu != 0);
+    if (c.kernel == MXQ_KERNEL_FP4 || c.kernel == MXQ_KERNEL_UMMA) {
+        mxq::FusedAccept fa{};
+        fa.residual = swiglu ? nullptr : residual;
+        fa.swiglu = swiglu;
+        const cudaError_t e = c.kernel == MXQ_KERNEL_FP4
+                                  ? mxq::linear_fp4_launch(c.fp4, X_bf16, codes, scales, Y, y_dtype, st, &fa)
+                                  : mxq::linear_umma_launch(c.umma, X_bf16, codes, scales, Y, y_dtype, ws, lin_ws_bytes, st, &fa);
+        if (e != cudaSuccess) {
+            if (std::getenv("MXQ_DEBUG")) std::fprintf(stderr, "mxq_linear epilogue (kernel %d): %s\n", c.kernel, cudaGetErrorString(e));
+            (void)cudaGetLastError();
+            return MXQ_ERR_CUDA;
+        }
+        return mxq::launch_status();
+    }
+    // no tcgen05 kernel covers the call: the plain layer's sums pass through the workspace
+    float *sums = reinterpret_cast<float *>(ws + lin_ws_bytes);
+    const int rc = mxq_linear(X_bf16, M, codes, scales, N, K, sums, MXQ_F32, ws, lin_ws_bytes, stream);
+    if (rc != MXQ_OK) return rc;
+    const int64_t outs = (int64_t)M * (swiglu ? N / 2 : N);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((outs + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = mxq::pdl_enabled() ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, mxq::layer_epilogue_kernel, (const float *)sums, M, N, residual, swiglu, Y, y_dtype);
+    return mxq::launch_status();
+}
+
+int mxq_linear_residual(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
+                        const void *residual, void *Y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream) {
+    return linear_with_epilogue(X_bf16, M, codes, scales, N, K, residual, 0, Y, y_dtype, workspace, workspace_bytes, stream);
+}
+
+int mxq_linear_swiglu(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
+                      void *Y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream) {
+    return linear_with_epilogue(X_bf16, M, codes, scales, N, K, nullptr, 1, Y, y_dtype, workspace, workspace_bytes, stream);
 }
 
 int mxq_linear_host(const void *X_host, int M, const uint8_t *codes, const uint8_t *scales, int64_t N,

@@ -161,17 +161,18 @@ __device__ __forceinline__ bool split_half_unit(const uint4 raw, int m, int kk, 
 // the codes, cp.async of the scale bytes, barrier set-up); warps 2..5 split the activations stage by stage and,
 // at the end, read the accumulator (one row per thread), exchange partial results and store.
 // MULTI: whether a CTA may own more than one tile (false: exactly one, and the per-tile loops fold away).
-template <int NB, bool MULTI, bool FUSED>
+template <int NB, bool MULTI, int EPI>
 __global__ void __launch_bounds__(kFp4Threads)
 linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 *__restrict__ X, int M,
                   const uint8_t *__restrict__ codes, const uint8_t *__restrict__ scales, int64_t N, int64_t K,
                   void *__restrict__ Y, int y_dtype, int split, int ring, int ks, int chunk_max, int tmem_cols, int groups,
                   int tiles, int tiles_max, const FusedAccept fa_arg) {
     extern __shared__ uint8_t smem_raw[];
-    // FUSED: the values compete for the verifier's argmax instead of being stored (fa.keys set); a template parameter so
-    // that the plain layer's epilogue carries none of it
+    // EPI: what happens to a finished sum: stored (kEpiStore), competing for the verifier's argmax (kEpiAccept, fa.keys
+    // set) or stored after a residual add or the gate / up pairing (kEpiLayer); a template parameter so that the plain
+    // layer's epilogue carries none of the others
     FusedAccept fa = fa_arg;
-    if (!FUSED) fa.keys = nullptr;
+    if (EPI != kEpiAccept) fa.keys = nullptr;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef MXQ_FP4_TRACE
     long long tr_c0 = 0;
@@ -571,7 +572,16 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
             }
             if (split == 1) {
                 const int64_t n = n0 + (int64_t)t * kFp4TileRows + row;
-                if (n < N)
+                if (EPI == kEpiLayer) {
+                    // (gate / up pairing: the partner row's sum sits in the neighbouring lane)
+#pragma unroll
+                    for (int m = 0; m < MT; ++m)
+                        if (m < M) {
+                            const float v = yt[m] * kGuardUp;
+                            const float o = fa.swiglu ? __shfl_xor_sync(0xffffffffu, v, 1) : 0.f;
+                            if (n < N) emit_layer(fa, Y, y_dtype, m, n, N, v, o);
+                        }
+                } else if (n < N)
 #pragma unroll
                     for (int m = 0; m < MT; ++m)
                         if (m < M) {
@@ -609,7 +619,9 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                     for (int j = 0; j < split; ++j) acc += gRecv[((t * split + j) * M + m) * cnt_max + r];
                     const int64_t n = n0 + (int64_t)t * kFp4TileRows + row_lo + r;
                     if (n < N) {
-                        if (fa.keys) {
+                        if (EPI == kEpiLayer) {
+                            emit_layer(fa, Y, y_dtype, m, n, N, acc * kGuardUp + poison, 0.f);   // (gate / up calls are planned with power-of-two clusters)
+                        } else if (fa.keys) {
                             const unsigned long long key = argmax_key(acc * kGuardUp + poison, (uint32_t)n);
                             if (key) atomicMax(s_keys + m, key);   // (rare decomposition: straight into shared memory)
                         } else {
@@ -631,7 +643,16 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
 #pragma unroll
                         for (int m = 0; m < MT; ++m) v[m] += __shfl_xor_sync(0xffffffffu, v[m], o);
                     }
-                    if (j == 0 && n < N) {
+                    if (EPI == kEpiLayer) {
+                        // (every lane holds its row's sum after the butterfly; rows r and r ^ 1 are `split` lanes apart)
+#pragma unroll
+                        for (int m = 0; m < MT; ++m)
+                            if (m < M) {
+                                const float w = v[m] * kGuardUp + poison;
+                                const float o = fa.swiglu ? __shfl_xor_sync(0xffffffffu, w, split) : 0.f;
+                                if (j == 0 && n < N) emit_layer(fa, Y, y_dtype, m, n, N, w, o);
+                            }
+                    } else if (j == 0 && n < N) {
 #pragma unroll
                         for (int m = 0; m < MT; ++m)
                             if (m < M) {
@@ -669,19 +690,19 @@ int env_int(const char *name) {
     return e ? std::atoi(e) : 0;
 }
 
-template <int NB, bool MULTI, bool FUSED>
+template <int NB, bool MULTI, int EPI>
 cudaError_t launch_fp4(const Fp4Plan &p, const CUtensorMap &map, const void *X, const uint8_t *codes,
                        const uint8_t *scales, void *Y, int y_dtype, cudaStream_t stream, const FusedAccept &fa) {
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(linear_fp4_kernel<NB, MULTI, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(linear_fp4_kernel<NB, MULTI, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kFp4SmemLimit);
         if (e != cudaSuccess) return e;
         // all of the SM's L1/shared array as shared memory: how many CTAs (of this and of the next kernel) fit on an
         // SM is what decides how early the next kernel's weight stream can start
-        e = cudaFuncSetAttribute(linear_fp4_kernel<NB, MULTI, FUSED>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(linear_fp4_kernel<NB, MULTI, EPI>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -706,13 +727,13 @@ cudaError_t launch_fp4(const Fp4Plan &p, const CUtensorMap &map, const void *X, 
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    return cudaLaunchKernelEx(&cfg, linear_fp4_kernel<NB, MULTI, FUSED>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
+    return cudaLaunchKernelEx(&cfg, linear_fp4_kernel<NB, MULTI, EPI>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
                               Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols, p.groups, p.tiles, p.tiles_max, fa);
 }
 
 }  // namespace
 
-bool linear_fp4_plan(int M, int64_t N, int64_t K, Fp4Plan &p) {
+bool linear_fp4_plan(int M, int64_t N, int64_t K, Fp4Plan &p, bool pow2_split) {
     if (M < 1 || M > kFp4MaxM || N < 1 || K < 128 || (K % 128) != 0) return false;
     if (K > 0x3FFFFFFF || N > 0x7FFFFFFF) return false;
     p.M = M;
@@ -721,6 +742,7 @@ bool linear_fp4_plan(int M, int64_t N, int64_t K, Fp4Plan &p) {
     p.nb = M == 1 ? 16 : (M == 2 ? 32 : 64);
     p.ks = (int)((K + kFp4StageK - 1) / kFp4StageK);
     p.tiles = (int)((N + kFp4TileRows - 1) / kFp4TileRows);
+    p.pow2_split = pow2_split ? 1 : 0;
     return fp4_layout(p, sm_count(), env_int("MXQ_FP4_SPLIT"), env_int("MXQ_FP4_RING"), env_int("MXQ_FP4_TILES"));
 }
 
@@ -730,23 +752,23 @@ cudaError_t linear_fp4_launch(const Fp4Plan &p, const void *X, const uint8_t *co
     if (!codes_tensor_map(codes, p.N, p.K, /*expand_fp4=*/false, &map)) return cudaErrorNotSupported;
     const bool multi = p.tiles_max > 1;
     const FusedAccept fa = fused ? *fused : FusedAccept{};
-    switch (p.nb) {
-        case 16:
-            return fa.keys ? (multi ? launch_fp4<16, true, true>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
-                                    : launch_fp4<16, false, true>(p, map, X, codes, scales, Y, y_dtype, stream, fa))
-                           : (multi ? launch_fp4<16, true, false>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
-                                    : launch_fp4<16, false, false>(p, map, X, codes, scales, Y, y_dtype, stream, fa));
-        case 32:
-            return fa.keys ? (multi ? launch_fp4<32, true, true>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
-                                    : launch_fp4<32, false, true>(p, map, X, codes, scales, Y, y_dtype, stream, fa))
-                           : (multi ? launch_fp4<32, true, false>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
-                                    : launch_fp4<32, false, false>(p, map, X, codes, scales, Y, y_dtype, stream, fa));
-        default:
-            return fa.keys ? (multi ? launch_fp4<64, true, true>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
-                                    : launch_fp4<64, false, true>(p, map, X, codes, scales, Y, y_dtype, stream, fa))
-                           : (multi ? launch_fp4<64, true, false>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
-                                    : launch_fp4<64, false, false>(p, map, X, codes, scales, Y, y_dtype, stream, fa));
+    if (fa.swiglu && ((p.split & (p.split - 1)) != 0 || (p.N & 1))) return cudaErrorNotSupported;   // see linear_fp4_plan's pow2_split
+#define MXQ_FP4_PICK(NB, EPI)                                                                             \
+    return multi ? launch_fp4<NB, true, EPI>(p, map, X, codes, scales, Y, y_dtype, stream, fa)             \
+                 : launch_fp4<NB, false, EPI>(p, map, X, codes, scales, Y, y_dtype, stream, fa)
+#define MXQ_FP4_PICK_EPI(NB)                                     \
+    switch (epilogue_kind(fa)) {                                 \
+        case kEpiAccept: MXQ_FP4_PICK(NB, kEpiAccept);           \
+        case kEpiLayer: MXQ_FP4_PICK(NB, kEpiLayer);             \
+        default: MXQ_FP4_PICK(NB, kEpiStore);                    \
     }
+    switch (p.nb) {
+        case 16: MXQ_FP4_PICK_EPI(16)
+        case 32: MXQ_FP4_PICK_EPI(32)
+        default: MXQ_FP4_PICK_EPI(64)
+    }
+#undef MXQ_FP4_PICK_EPI
+#undef MXQ_FP4_PICK
 }
 
 #ifdef MXQ_FP4_TRACE

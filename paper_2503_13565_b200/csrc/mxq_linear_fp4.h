@@ -28,6 +28,7 @@ struct Fp4Plan {
     int chunk_max;   // most stages any CTA owns = ceil(ks / split)
     int grid;        // groups * split
     int tmem_cols;   // tensor-memory columns allocated per CTA
+    int pow2_split;  // in: only cluster sizes 1, 2, 4, 8 (the gate / up epilogue pairs rows inside a warp)
     uint32_t smem_bytes;
     int64_t N, K;
 };
@@ -79,6 +80,7 @@ inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring, int
     const int smax = p.ks < kFp4MaxSplit ? p.ks : kFp4MaxSplit;
     for (int s = 1; s <= smax; ++s) {
         if (force_split > 0 && s != (force_split < smax ? force_split : smax)) continue;
+        if (p.pow2_split && (s & (s - 1)) != 0) continue;
         if (force_split <= 0 && s == 7) continue;   // clusters of 7 measured up to 1.5 times slower than of 6 or 8 (5120 x 5120, 5120 x 13824)
         const int chunk = (p.ks + s - 1) / s;
         int groups, ring;

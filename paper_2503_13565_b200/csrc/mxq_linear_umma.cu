@@ -167,16 +167,17 @@ cudaError_t launch_split(const __nv_bfloat16 *X, int M, int64_t K, int ks, uint8
 // the codes, cp.async of the scale bytes, barrier set-up); warps 2..5 split the activations stage by stage and,
 // at the end, read the accumulator (one row per thread), exchange partial results and store.
 // MULTI: whether a CTA may own more than one tile (false: exactly one, and the per-tile loops fold away).
-template <int NB, bool MULTI, bool BRING, bool FUSED>
+template <int NB, bool MULTI, bool BRING, int EPI>
 __global__ void __launch_bounds__(kUmmaThreads)
 linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 *__restrict__ X, int M,
                   const uint8_t *__restrict__ codes, const uint8_t *__restrict__ scales, int64_t N, int64_t K,
                   void *__restrict__ Y, int y_dtype, int split, int ring, int ks, int chunk_max, int tmem_cols, int groups,
                   int tiles, int tiles_max, const uint8_t *__restrict__ presplit, const FusedAccept fa_arg) {
-    // FUSED: the values compete for the verifier's argmax instead of being stored (fa.keys set); a template parameter so
-    // that the plain layer's epilogue carries none of it
+    // EPI: what happens to a finished sum: stored (kEpiStore), competing for the verifier's argmax (kEpiAccept, fa.keys
+    // set) or stored after a residual add or the gate / up pairing (kEpiLayer); a template parameter so that the plain
+    // layer's epilogue carries none of the others
     FusedAccept fa = fa_arg;
-    if (!FUSED) fa.keys = nullptr;
+    if (EPI != kEpiAccept) fa.keys = nullptr;
     constexpr bool bring = BRING;   // the token operand is fetched stage by stage into the ring slots (needs presplit, one tile)
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -558,7 +559,16 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
             }
             if (split == 1) {
                 const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row;
-                if (n < N)
+                if (EPI == kEpiLayer) {
+                    // (gate / up pairing: the partner row's sum sits in the neighbouring lane)
+#pragma unroll
+                    for (int m = 0; m < MT; ++m)
+                        if (m < M) {
+                            const float v = yt[m] * kGuardUp;
+                            const float o = fa.swiglu ? __shfl_xor_sync(0xffffffffu, v, 1) : 0.f;
+                            if (n < N) emit_layer(fa, Y, y_dtype, m, n, N, v, o);
+                        }
+                } else if (n < N)
 #pragma unroll
                     for (int m = 0; m < MT; ++m)
                         if (m < M) {
@@ -595,7 +605,9 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                     for (int j = 0; j < split; ++j) acc += gRecv[((t * split + j) * M + m) * cnt_max + r];
                     const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row_lo + r;
                     if (n < N) {
-                        if (fa.keys) {
+                        if (EPI == kEpiLayer) {
+                            emit_layer(fa, Y, y_dtype, m, n, N, acc * kGuardUp + poison, 0.f);   // (gate / up calls are planned with power-of-two clusters)
+                        } else if (fa.keys) {
                             const unsigned long long key = argmax_key(acc * kGuardUp + poison, (uint32_t)n);
                             if (key) atomicMax(s_keys + m, key);   // (rare decomposition: straight into shared memory)
                         } else {
@@ -617,7 +629,16 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
 #pragma unroll
                         for (int m = 0; m < MT; ++m) v[m] += __shfl_xor_sync(0xffffffffu, v[m], o);
                     }
-                    if (j == 0 && n < N) {
+                    if (EPI == kEpiLayer) {
+                        // (every lane holds its row's sum after the butterfly; rows r and r ^ 1 are `split` lanes apart)
+#pragma unroll
+                        for (int m = 0; m < MT; ++m)
+                            if (m < M) {
+                                const float w = v[m] * kGuardUp + poison;
+                                const float o = fa.swiglu ? __shfl_xor_sync(0xffffffffu, w, split) : 0.f;
+                                if (j == 0 && n < N) emit_layer(fa, Y, y_dtype, m, n, N, w, o);
+                            }
+                    } else if (j == 0 && n < N) {
 #pragma unroll
                         for (int m = 0; m < MT; ++m)
                             if (m < M) {
@@ -654,19 +675,19 @@ int env_int(const char *name) {
     return e ? std::atoi(e) : 0;
 }
 
-template <int NB, bool MULTI, bool BRING, bool FUSED>
+template <int NB, bool MULTI, bool BRING, int EPI>
 cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X, const uint8_t *codes,
                        const uint8_t *scales, void *Y, int y_dtype, const uint8_t *presplit, cudaStream_t stream, const FusedAccept &fa) {
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI, BRING, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI, BRING, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kUmmaSmemLimit);
         if (e != cudaSuccess) return e;
         // all of the SM's L1/shared array as shared memory: how many CTAs (of this and of the next kernel) fit on an
         // SM is what decides how early the next kernel's weight stream can start
-        e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI, BRING, FUSED>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(linear_umma_kernel<NB, MULTI, BRING, EPI>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -691,7 +712,7 @@ cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    return cudaLaunchKernelEx(&cfg, linear_umma_kernel<NB, MULTI, BRING, FUSED>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
+    return cudaLaunchKernelEx(&cfg, linear_umma_kernel<NB, MULTI, BRING, EPI>, map, (const __nv_bfloat16 *)X, p.M, codes, scales, p.N, p.K,
                               Y, y_dtype, p.split, p.ring, p.ks, p.chunk_max, p.tmem_cols, p.groups, p.tiles, p.tiles_max, presplit, fa);
 }
 
@@ -704,10 +725,11 @@ static int presplit_min_m() {
     return v;
 }
 
-bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p, bool with_workspace) {
+bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p, bool with_workspace, bool pow2_split) {
     if (M < 1 || M > kUmmaMaxM || N < 1 || K < 128 || (K % 128) != 0) return false;
     if (K > 0x3FFFFFFF || N > 0x7FFFFFFF) return false;
     p.presplit = with_workspace && M >= presplit_min_m() ? 1 : 0;
+    p.pow2_split = pow2_split ? 1 : 0;
     p.M = M;
     p.N = N;
     p.K = K;
@@ -722,13 +744,16 @@ template <int NB>
 static cudaError_t pick_umma(const UmmaPlan &p, bool bring, const CUtensorMap &map, const void *X, const uint8_t *codes,
                              const uint8_t *scales, void *Y, int y_dtype, const uint8_t *ws, cudaStream_t stream, const FusedAccept &fa) {
     const bool multi = p.tiles_max > 1;
-#define MXQ_UMMA_PICK(FUSED)                                                                                                  \
-    return multi ? (bring ? launch_umma<NB, true, true, FUSED>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)           \
-                          : launch_umma<NB, true, false, FUSED>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa))         \
-                 : (bring ? launch_umma<NB, false, true, FUSED>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)          \
-                          : launch_umma<NB, false, false, FUSED>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa))
-    if (fa.keys) { MXQ_UMMA_PICK(true); }
-    MXQ_UMMA_PICK(false);
+#define MXQ_UMMA_PICK(EPI)                                                                                                    \
+    return multi ? (bring ? launch_umma<NB, true, true, EPI>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)           \
+                          : launch_umma<NB, true, false, EPI>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa))         \
+                 : (bring ? launch_umma<NB, false, true, EPI>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa)          \
+                          : launch_umma<NB, false, false, EPI>(p, map, X, codes, scales, Y, y_dtype, ws, stream, fa))
+    switch (epilogue_kind(fa)) {
+        case kEpiAccept: MXQ_UMMA_PICK(kEpiAccept);
+        case kEpiLayer: MXQ_UMMA_PICK(kEpiLayer);
+        default: MXQ_UMMA_PICK(kEpiStore);
+    }
 #undef MXQ_UMMA_PICK
 }
 
@@ -739,6 +764,7 @@ size_t linear_umma_workspace_bytes(int M, int64_t K) {
 
 cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,
                               int y_dtype, void *workspace, size_t workspace_bytes, cudaStream_t stream, const FusedAccept *fused) {
+    if (fused && fused->swiglu && ((p.split & (p.split - 1)) != 0 || (p.N & 1))) return cudaErrorNotSupported;   // see linear_umma_plan's pow2_split
     CUtensorMap map;
     if (!codes_tensor_map(codes, p.N, p.K, /*expand_fp4=*/true, &map)) return cudaErrorNotSupported;
     // a workspace that is large enough (and aligned for bulk copies) lets the token operand be split once per call
@@ -748,7 +774,7 @@ cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *
         ws = static_cast<uint8_t *>(workspace);
     if (p.presplit && !ws) {   // planned for a workspace that is not there: plan again without
         UmmaPlan q;
-        if (!linear_umma_plan(p.M, p.N, p.K, q, false)) return cudaErrorNotSupported;
+        if (!linear_umma_plan(p.M, p.N, p.K, q, false, p.pow2_split != 0)) return cudaErrorNotSupported;
         return linear_umma_launch(q, X, codes, scales, Y, y_dtype, nullptr, 0, stream, fused);
     }
     if (ws) {

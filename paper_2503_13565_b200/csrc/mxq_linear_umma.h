@@ -50,6 +50,7 @@ struct UmmaPlan {
     int presplit;    // planned for a token operand split ahead of the weight kernel (needs the workspace)
     int bring;       // ... and fetched stage by stage into the ring slots instead of whole K ranges
     long cost;       // the layout heuristic's figure for the chosen decomposition (comparable within a regime)
+    int pow2_split;  // in: only cluster sizes 1, 2, 4, 8 (the gate / up epilogue pairs rows inside a warp)
     uint32_t smem_bytes;
     int64_t N, K;
 };
@@ -95,6 +96,7 @@ inline bool umma_layout_one(UmmaPlan &p, int sms, int force_split, int force_rin
     const int smax = p.ks < kUmmaMaxSplit ? p.ks : kUmmaMaxSplit;
     for (int s = 1; s <= smax; ++s) {
         if (force_split > 0 && s != (force_split < smax ? force_split : smax)) continue;
+        if (p.pow2_split && (s & (s - 1)) != 0) continue;
         if (force_split <= 0 && s == 7) continue;   // clusters of 7 measured up to 1.5 times slower than of 6 or 8 (5120 x 5120, 5120 x 13824)
         const int chunk = (p.ks + s - 1) / s;
         int groups, ring;

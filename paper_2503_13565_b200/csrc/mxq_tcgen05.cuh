@@ -227,4 +227,22 @@ __device__ __forceinline__ void store_out(void *Y, int y_dtype, int64_t idx, flo
         reinterpret_cast<__nv_bfloat16 *>(Y)[idx] = __float2bfloat16_rn(v);
 }
 
+__device__ __forceinline__ float load_in(const void *R, int dtype, int64_t idx) {
+    return dtype == MXQ_F32 ? reinterpret_cast<const float *>(R)[idx]
+                            : __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(R)[idx]);
+}
+
+// Layer epilogues of the tcgen05 kernels: what happens to the finished sum v of (token row m, weight row n).
+// `other` is the sum of weight row n ^ 1 (only read for the gate / up pairing, where the caller fetched it from the
+// neighbouring holder with a shuffle).  silu(g) = g / (1 + e^-g): for g -> -inf the quotient goes to -0, for
+// g -> +inf to g.
+__device__ __forceinline__ void emit_layer(const FusedAccept &fa, void *Y, int y_dtype, int m, int64_t n, int64_t N, float v, float other) {
+    if (fa.swiglu) {
+        if ((n & 1) == 0) store_out(Y, y_dtype, (int64_t)m * (N >> 1) + (n >> 1), v / (1.f + expf(-v)) * other);
+    } else {
+        const int64_t idx = (int64_t)m * N + n;
+        store_out(Y, y_dtype, idx, v + load_in(fa.residual, y_dtype, idx));
+    }
+}
+
 }  // namespace mxq

@@ -428,6 +428,42 @@ def run_ours(args):
             del wl
         bf["status"] = mxq.mxq_linear_device_status()
         extra["bf16_weights"] = bf
+        # The same 7B layer as four calls with fused epilogues (Sec. III-D-2: operators fused into the linear layers):
+        # q/k/v as one 12288 x 4096 matrix, o + residual, gate/up interleaved by rows with SiLU(gate)*up, down + residual.
+        # BF16 in and out; o -> gate/up -> down is a true dependent chain (each call's output is the next one's input).
+        fl = {}
+        nlay = 8   # 8 x 107.5 MB of weights: larger than L2
+        lay4 = []
+        for li in range(nlay):
+            mats4 = []
+            for j, (n_, k_) in enumerate([(12288, 4096), (4096, 4096), (22016, 4096), (4096, 11008)]):
+                w_ = synth.weight(3, 500 + 4 * li + j, n_, k_, device=device)
+                mats4.append(mxq.mxq_quantize(w_))
+                del w_
+            lay4.append(mats4)
+        for mm in (1, 8):
+            h0 = synth.normal_bf16((mm, 4096), 1.0, 11, device)
+            att = synth.normal_bf16((mm, 4096), 1.0, 12, device)
+            qkv = torch.empty((mm, 12288), dtype=torch.bfloat16, device=device)
+            h1 = torch.empty((mm, 4096), dtype=torch.bfloat16, device=device)
+            act = torch.empty((mm, 11008), dtype=torch.bfloat16, device=device)
+            h2 = torch.empty((mm, 4096), dtype=torch.bfloat16, device=device)
+            wsf = torch.empty(max(mxq.mxq_linear_fused_workspace_bytes(mm, 22016, 4096),
+                                  mxq.mxq_linear_fused_workspace_bytes(mm, 4096, 11008),
+                                  mxq.mxq_linear_workspace_bytes(mm, 12288, 4096), 16), dtype=torch.uint8, device=device)
+
+            def fused_pass():
+                for (wqkv, wo, wgu, wd) in lay4:
+                    mxq.mxq_linear(h0, wqkv[0], wqkv[1], out=qkv, workspace=wsf)
+                    mxq.mxq_linear_residual(att, wo[0], wo[1], h0, out=h1, workspace=wsf)
+                    mxq.mxq_linear_swiglu(h1, wgu[0], wgu[1], out=act, workspace=wsf)
+                    mxq.mxq_linear_residual(act, wd[0], wd[1], h1, out=h2, workspace=wsf)
+            tf_ = time_graph(fused_pass, 10) / nlay
+            wbytes = sum(n_ * k_ * 17 // 32 for n_, k_ in [(12288, 4096), (4096, 4096), (22016, 4096), (4096, 11008)])
+            fl["m%d" % mm] = {"us_per_layer": tf_ * 1e6, "gbs": wbytes / tf_ / 1e9, "calls": 4, "weight_bytes": wbytes}
+        fl["status"] = mxq.mxq_linear_device_status()
+        extra["fused_layer"] = fl
+        del lay4
         # Speculative decoding with the quantised draft (Sec. III-B): a 4-layer slice of the 7B stack plus a 32000-row
         # vocabulary projection, target in BF16, draft = its MXFP4 cast; acceptance is simulated (random weights accept
         # nothing), the kernels and the control flow are real.  Measured tokens per second against Eq. 1 fed with the measured S.

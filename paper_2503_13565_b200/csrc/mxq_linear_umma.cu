@@ -469,6 +469,12 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
 
         // ---- epilogue: accumulator row -> registers; the three parts of a token are three neighbouring columns -------
         constexpr int MT = NB / kUmmaParts;         // token slots per tile (5, 10 or 16)
+        // layer epilogues: the residual values this thread will add to its first tile's sums, requested before the wait
+        float res[MT];   // (unused, and optimised away, in the other epilogues)
+        if (EPI == kEpiLayer && split == 1) {
+            const int64_t n_first = (int64_t)tile_lo * kUmmaTileRows + row;
+            layer_prefetch<MT>(fa, y_dtype, M, n_first, N, n_first < N, res);
+        }
         if (!mbar_wait_relaxed(done_bar, 0)) {
             atomicOr(&g_umma_status, 4u);
             s_fail = 1;
@@ -562,12 +568,9 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                 if (EPI == kEpiLayer) {
                     // (gate / up pairing: the partner row's sum sits in the neighbouring lane)
 #pragma unroll
-                    for (int m = 0; m < MT; ++m)
-                        if (m < M) {
-                            const float v = yt[m] * kGuardUp;
-                            const float o = fa.swiglu ? __shfl_xor_sync(0xffffffffu, v, 1) : 0.f;
-                            if (n < N) emit_layer(fa, Y, y_dtype, m, n, N, v, o);
-                        }
+                    for (int m = 0; m < MT; ++m) yt[m] *= kGuardUp;
+                    layer_emit<MT>(fa, Y, y_dtype, M, n, N, n < N, yt, res, 1);
+                    if (t + 1 < ntile) layer_prefetch<MT>(fa, y_dtype, M, n + kUmmaTileRows, N, n + kUmmaTileRows < N, res);
                 } else if (n < N)
 #pragma unroll
                     for (int m = 0; m < MT; ++m)
@@ -589,6 +592,9 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
             }
         }
         if (split > 1) {
+            float res_s[TokenScatter<MT>::PH];   // (power-of-two clusters: the residual values of this lane's share of the token rows)
+            if (EPI == kEpiLayer && (split & (split - 1)) == 0)
+                scatter_prefetch<MT>(fa, y_dtype, M, split, ct & (split - 1), (int64_t)tile_lo * kUmmaTileRows + row_lo + ct / split, N, res_s);
             if (!mbar_wait_relaxed(recv_bar, 0)) {
                 atomicOr(&g_umma_status, 16u);
                 s_fail = 1;
@@ -606,7 +612,9 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                     const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row_lo + r;
                     if (n < N) {
                         if (EPI == kEpiLayer) {
-                            emit_layer(fa, Y, y_dtype, m, n, N, acc * kGuardUp + poison, 0.f);   // (gate / up calls are planned with power-of-two clusters)
+                            // (gate / up calls are planned with power-of-two clusters and never come here)
+                            const int64_t at = (int64_t)m * N + n;
+                            store_out(Y, y_dtype, at, acc * kGuardUp + poison + load_in(fa.residual, y_dtype, at));
                         } else if (fa.keys) {
                             const unsigned long long key = argmax_key(acc * kGuardUp + poison, (uint32_t)n);
                             if (key) atomicMax(s_keys + m, key);   // (rare decomposition: straight into shared memory)
@@ -616,12 +624,20 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                     }
                 }
             } else {
-                // power-of-two cluster: one value per thread (row ct / split, sender ct % split), butterfly sum over the
-                // senders in neighbouring lanes; the order of additions is fixed by the lane pattern
+                // power-of-two cluster: one thread per (row ct / split, sender ct % split), the senders of a row in neighbouring
+                // lanes; the order of additions is fixed by the lane pattern
                 const int r = ct / split, j = ct & (split - 1);
                 for (int t = 0; t < ntile; ++t) {
                     const int64_t n = n0 + (int64_t)t * kUmmaTileRows + row_lo + r;
-                    // all loads, then all shuffles, then all uses: the token rows are independent of each other
+                    if (EPI != kEpiAccept) {
+                        // plain store and layer epilogues: reduce-scatter over the token rows, every lane finishes its share
+                        scatter_sum_store<MT, EPI>(gRecv + ((t * split + j) * M) * cnt_max + r, cnt_max, M, split, j, n, N, kGuardUp, poison,
+                                                   fa, Y, y_dtype, res_s);
+                        if (EPI == kEpiLayer && t + 1 < ntile) scatter_prefetch<MT>(fa, y_dtype, M, split, j, n + kUmmaTileRows, N, res_s);
+                        continue;
+                    }
+                    // fused verification: all-to-all butterfly, every lane ends with all token rows (the running maxima are
+                    // kept per token row); all loads, then all shuffles, then all uses: the token rows are independent of each other
                     float v[MT];
 #pragma unroll
                     for (int m = 0; m < MT; ++m) v[m] = m < M ? gRecv[((t * split + j) * M + m) * cnt_max + r] : 0.f;
@@ -629,16 +645,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
 #pragma unroll
                         for (int m = 0; m < MT; ++m) v[m] += __shfl_xor_sync(0xffffffffu, v[m], o);
                     }
-                    if (EPI == kEpiLayer) {
-                        // (every lane holds its row's sum after the butterfly; rows r and r ^ 1 are `split` lanes apart)
-#pragma unroll
-                        for (int m = 0; m < MT; ++m)
-                            if (m < M) {
-                                const float w = v[m] * kGuardUp + poison;
-                                const float o = fa.swiglu ? __shfl_xor_sync(0xffffffffu, w, split) : 0.f;
-                                if (j == 0 && n < N) emit_layer(fa, Y, y_dtype, m, n, N, w, o);
-                            }
-                    } else if (j == 0 && n < N) {
+                    if (j == 0 && n < N) {
 #pragma unroll
                         for (int m = 0; m < MT; ++m)
                             if (m < M) {

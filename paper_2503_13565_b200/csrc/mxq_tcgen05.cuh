@@ -232,16 +232,116 @@ __device__ __forceinline__ float load_in(const void *R, int dtype, int64_t idx) 
                             : __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(R)[idx]);
 }
 
-// Layer epilogues of the tcgen05 kernels: what happens to the finished sum v of (token row m, weight row n).
-// `other` is the sum of weight row n ^ 1 (only read for the gate / up pairing, where the caller fetched it from the
-// neighbouring holder with a shuffle).  silu(g) = g / (1 + e^-g): for g -> -inf the quotient goes to -0, for
-// g -> +inf to g.
-__device__ __forceinline__ void emit_layer(const FusedAccept &fa, void *Y, int y_dtype, int m, int64_t n, int64_t N, float v, float other) {
+// Layer epilogues of the tcgen05 kernels (kEpiLayer): what happens to the finished sums w[m] of weight row n, one per
+// token row.  Everything is done for all token rows at once -- all loads, then all arithmetic, then all stores -- so
+// that the latencies overlap (one row at a time cost 0.25 us per token row).
+// layer_prefetch: the residual values this thread will add (zeros if there is no residual or the thread is inactive).
+template <int MT>
+__device__ __forceinline__ void layer_prefetch(const FusedAccept &fa, int y_dtype, int M, int64_t n, int64_t N, bool active, float (&r)[MT]) {
+#pragma unroll
+    for (int m = 0; m < MT; ++m) r[m] = (fa.residual != nullptr && active && m < M) ? load_in(fa.residual, y_dtype, (int64_t)m * N + n) : 0.f;
+}
+// layer_emit: called by all 32 lanes of a warp together.  Gate / up pairing: the holder of weight row n ^ 1 is
+// `pair_lanes` lanes away; the even row's holder stores silu(gate) * up with silu(g) = g / (1 + e^-g), which goes to -0
+// for g -> -inf and to g for g -> +inf.  Residual: Y may be the residual itself (every element is read by the thread
+// that writes it, before it writes).
+template <int MT>
+__device__ __forceinline__ void layer_emit(const FusedAccept &fa, void *Y, int y_dtype, int M, int64_t n, int64_t N, bool active,
+                                           const float (&w)[MT], const float (&r)[MT], int pair_lanes) {
     if (fa.swiglu) {
-        if ((n & 1) == 0) store_out(Y, y_dtype, (int64_t)m * (N >> 1) + (n >> 1), v / (1.f + expf(-v)) * other);
-    } else {
-        const int64_t idx = (int64_t)m * N + n;
-        store_out(Y, y_dtype, idx, v + load_in(fa.residual, y_dtype, idx));
+        float y[MT];
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            const float up = __shfl_xor_sync(0xffffffffu, w[m], pair_lanes);
+            y[m] = w[m] / (1.f + expf(-w[m])) * up;
+        }
+        if (active && (n & 1) == 0) {
+#pragma unroll
+            for (int m = 0; m < MT; ++m)
+                if (m < M) store_out(Y, y_dtype, (int64_t)m * (N >> 1) + (n >> 1), y[m]);
+        }
+    } else if (active) {
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+            if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, w[m] + r[m]);
+    }
+}
+
+// ---- sum over the senders of a power-of-two cluster, as a reduce-scatter over the token rows -------------------------------
+// Thread (row r, sender j) of the owner CTA holds sender j's partial sums of all token rows of weight row n; the `split`
+// senders of a row sit in neighbouring lanes.  Step s exchanges between lanes j and j ^ 2^s: the lane with bit s clear
+// keeps the token rows with bit s clear and gets its partner's values for them, and vice versa.  After log2(split)
+// steps lane j holds the finished sums of the token rows m = i * S + (j & (S - 1)), i = 0, 1, .. (S = min(split, P), P =
+// token slots rounded up to a power of two): a third of the shuffles of an all-to-all butterfly, and the final stores
+// (and the residual loads, and the activation) are spread over the lanes instead of falling to lane j = 0.  Every
+// sum is formed by the same tree of additions as in the butterfly (first j ^ 1, then j ^ 2, then j ^ 4), so the
+// result is bit-identical whatever the token count.  Where split > P the last steps add whole values and the lanes
+// j >= P hold duplicates and stay silent.
+template <int MT>
+struct TokenScatter {
+    static constexpr int P = MT <= 1 ? 1 : (MT <= 2 ? 2 : (MT <= 4 ? 4 : (MT <= 8 ? 8 : 16)));
+    static constexpr int PH = P >= 2 ? P / 2 : 1;   // most positions a lane ends up with (split >= 2)
+};
+
+// residual values of the positions this lane will finish (zeros where there is nothing to add)
+template <int MT>
+__device__ __forceinline__ void scatter_prefetch(const FusedAccept &fa, int y_dtype, int M, int split, int j, int64_t n, int64_t N,
+                                                 float (&res)[TokenScatter<MT>::PH]) {
+    constexpr int P = TokenScatter<MT>::P, PH = TokenScatter<MT>::PH;
+    const int S = split < P ? split : P, npos = P / S;
+    const bool speaks = j < P && n < N && fa.residual != nullptr;
+#pragma unroll
+    for (int i = 0; i < PH; ++i) {
+        const int m = i * S + (j & (S - 1));
+        res[i] = (speaks && i < npos && m < M) ? load_in(fa.residual, y_dtype, (int64_t)m * N + n) : 0.f;
+    }
+}
+
+// recv: sender j's partial sums for this thread's row, token row m at recv[m * stride].  All 32 lanes call together.
+template <int MT, int EPI>
+__device__ __forceinline__ void scatter_sum_store(const float *recv, int stride, int M, int split, int j, int64_t n, int64_t N, float scale,
+                                                  float poison, const FusedAccept &fa, void *Y, int y_dtype,
+                                                  const float (&res)[TokenScatter<MT>::PH]) {
+    constexpr int P = TokenScatter<MT>::P, PH = TokenScatter<MT>::PH;
+    float a[P];
+#pragma unroll
+    for (int i = 0; i < P; ++i) a[i] = (i < MT && i < M) ? recv[i * stride] : 0.f;
+#pragma unroll
+    for (int s = 0; s < 3; ++s) {   // clusters of up to 8
+        const int o = 1 << s;
+        if (o < split) {
+            if ((P >> s) >= 2) {
+                const bool up = ((j >> s) & 1) != 0;
+#pragma unroll
+                for (int i = 0; i < P / 2; ++i)
+                    if (i < ((P >> s) >> 1)) {
+                        const float lo = a[2 * i], hi = a[2 * i + 1];
+                        const float keep = up ? hi : lo, send = up ? lo : hi;
+                        a[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                    }
+            } else {
+                a[0] += __shfl_xor_sync(0xffffffffu, a[0], o);
+            }
+        }
+    }
+    const int S = split < P ? split : P, npos = P / S;
+    const bool swiglu = EPI == kEpiLayer && fa.swiglu != 0;
+#pragma unroll
+    for (int i = 0; i < PH; ++i) {
+        a[i] = a[i] * scale + poison;
+        if (swiglu) {   // the partner row's sums sit `split` lanes away, at the same positions
+            const float up = __shfl_xor_sync(0xffffffffu, a[i], split);
+            a[i] = a[i] / (1.f + expf(-a[i])) * up;
+        } else if (EPI == kEpiLayer) {
+            a[i] += res[i];
+        }
+    }
+    if (j < P && n < N && !(swiglu && (n & 1))) {
+#pragma unroll
+        for (int i = 0; i < PH; ++i) {
+            const int m = i * S + (j & (S - 1));
+            if (i < npos && m < M) store_out(Y, y_dtype, swiglu ? (int64_t)m * (N >> 1) + (n >> 1) : (int64_t)m * N + n, a[i]);
+        }
     }
 }
 

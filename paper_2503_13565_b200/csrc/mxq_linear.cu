@@ -167,7 +167,7 @@ static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *code
             // vocabulary-sized matrices, where a CTA per SM walks several tiles: the packed-FP4 kernel still wins at two
             // token rows; above, the FP8-operand kernel, unless its token operand leaves no room for one CTA per SM
             try_fp4 = M == 2;
-            if (M > 2 && !(tc && aligned32 && linear_umma_plan(M, N, K, c.umma, with_workspace, pow2_split) && c.umma.grid <= sm_count()) &&
+            if (M > 2 && !(tc && aligned32 && linear_umma_plan(M, N, K, c.umma, with_workspace, pow2_split) && (c.umma.grid <= sm_count() || c.umma.tiles_max == 1)) &&
                 linear_mma_plan(M, N, K, c.mma))
                 try_umma = false;
         }

@@ -51,6 +51,7 @@ struct UmmaPlan {
     int bring;       // ... and fetched stage by stage into the ring slots instead of whole K ranges
     long cost;       // the layout heuristic's figure for the chosen decomposition (comparable within a regime)
     int pow2_split;  // in: only cluster sizes 1, 2, 4, 8 (the gate / up epilogue pairs rows inside a warp)
+    int layer_tiles; // most tiles for the one-tile-per-CTA regime (0: one per SM); set by umma_layout
     uint32_t smem_bytes;
     int64_t N, K;
 };
@@ -85,7 +86,7 @@ inline bool umma_layout_one(UmmaPlan &p, int sms, int force_split, int force_rin
     // p.presplit (set by the caller): the token operand comes ready-made from the workspace; a CTA of one tile may then
     // fetch it stage by stage with the weights (p.bring), so that its K range does not eat the ring's shared memory
     const int tcap = (512 - 16) / p.nb;   // tiles whose accumulators fit in tensor memory beside the scale columns
-    const bool layer_regime = p.tiles <= sms;
+    const bool layer_regime = p.tiles <= (p.layer_tiles > 0 ? p.layer_tiles : sms);
     // Tiles per CTA in the layer regime: one, except for the widest token operand on matrices of many tiles, where
     // the operand's K range of a CTA (6.5 KB per stage) leaves too little shared memory for weights unless two
     // tiles share it (11008 x 4096 at M = 16: 21.5 -> 16 us).
@@ -119,7 +120,10 @@ inline bool umma_layout_one(UmmaPlan &p, int sms, int force_split, int force_rin
             const long slots = (long)sms * umma_ctas_per_sm(bytes, tm);
             const long waves = (ctas + slots - 1) / slots;
             const long off = ctas > 2L * sms ? ctas - 2L * sms : 2L * sms - ctas;   // distance from two CTAs per SM
-            cost = (waves - 1) * 100000 + off;
+            // more tiles than SMs: the stages the fullest SM has to stream, with the vocabulary regime's penalty for K
+            // ranges under half a row
+            const long per_sm = (ctas + sms - 1) / sms * chunk * (s <= 2 ? 10 : 19);
+            cost = (waves - 1) * 100000 + (p.tiles > sms ? per_sm : off);
         } else {
             groups = sms / s < 1 ? 1 : sms / s;          // one CTA per SM
             if (groups > p.tiles) groups = p.tiles;
@@ -138,7 +142,7 @@ inline bool umma_layout_one(UmmaPlan &p, int sms, int force_split, int force_rin
             const long by_ring = (long)ring * 8192 / 1500, rate = by_ring < 41 ? by_ring : 41;   // GB/s
             cost = waves * units * 1000 / rate * (s <= 2 ? 10 : 19) * (br ? 17 : 10) / 10 + s;   // (the operand fetched again per tile: measured)
         }
-        if (best_cost < 0 || cost < best_cost || (cost == best_cost && layer_regime)) {   // layer regime: ties to the larger split
+        if (best_cost < 0 || cost < best_cost || (cost == best_cost && layer_regime && p.tiles <= sms)) {   // layers: ties to the larger split
             best_cost = cost;
             best_split = s;
             best_groups = groups;
@@ -166,7 +170,7 @@ inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, i
     if (!p.presplit || force_bring == 0) return umma_layout_one(p, sms, force_split, force_ring, force_tiles, false);
     UmmaPlan r = p;
     const bool have_r = force_bring < 0 && umma_layout_one(r, sms, force_split, force_ring, force_tiles, false);
-    if (p.tiles <= sms) {
+    if (p.tiles <= (p.layer_tiles > 0 ? p.layer_tiles : sms)) {
         if (have_r && r.tiles_max == 1 && r.ring >= 3 && 6 * r.grid >= 5 * sms) {
             p = r;
             return true;
@@ -174,6 +178,18 @@ inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, i
         if (umma_layout_one(p, sms, force_split, force_ring, force_tiles, true)) return true;
         if (have_r) p = r;
         return have_r;
+    }
+    // Up to two tiles per SM with the token operand coming through the ring: still one tile per CTA, all CTAs resident
+    // at once (two or three small CTAs per SM), if that leaves three ring slots.  Measured against one fat CTA per SM:
+    // 32000 x 4096 at M = 8: 23.4 -> 19.1 us, 22016 x 4096 at M = 8: 18.9 -> 16.8 us; small CTAs also let the next call's
+    // CTAs in early.
+    if (p.tiles <= 2 * sms && force_bring != 0 && force_tiles <= 0) {
+        UmmaPlan l = p;
+        l.layer_tiles = 2 * sms;
+        if (umma_layout_one(l, sms, force_split, force_ring, 0, true) && l.tiles_max == 1 && l.ring >= 3 && l.cost < 100000) {
+            p = l;
+            return true;
+        }
     }
     // vocabulary regime: the modelled cost decides (resident on ties: no second fetch of the operand per tile)
     UmmaPlan b = p;

@@ -59,12 +59,19 @@ inline int fp4_ctas_per_sm(uint32_t smem_bytes, int tmem_cols) {
     return by_smem < by_tmem ? by_smem : by_tmem;
 }
 
+// CTA slots of the whole GPU that a one-wave launch may count on: a grid that fills more than about 95 % of them ran as
+// if in two waves (clusters are placed inside one GPC, and the last ones find no GPC with room): 12288 x 4096 as 288 CTAs
+// on 296 slots took 12.8 us, as 384 on 444 slots 8.3 us; 13824 x 5120 as 432 on 444 13.3 us, as 540 on 592 10.3 us.
+inline long fp4_usable_slots(int sms, uint32_t smem_bytes, int tmem_cols) {
+    return (long)sms * fp4_ctas_per_sm(smem_bytes, tmem_cols) * 92 / 100;
+}
+
 // Chooses split, groups and ring for p.{M, nb, ks, tiles}; false if nothing fits.
 //
 // Two regimes, both measured on B200:
 //  - up to 2 * SMs tiles (the transformer layers themselves): one tile per CTA; the deepest ring up to 4 stages that
-//    still lets every CTA of the call be resident at once; the split that brings the CTA count closest to two per
-//    SM.  Small CTAs matter twice: the call runs as one wave, and what it leaves free of an SM's shared memory is taken
+//    still lets every CTA of the call be resident at once; the split that leaves the fewest stages per SM outside
+//    the rings.  Small CTAs matter twice: the call runs as one wave, and what it leaves free of an SM's shared memory is taken
 //    by the CTAs of the next call (programmatic dependent launch), which start their weight stream early.
 //  - more tiles (vocabulary projections): one CTA per SM walking several tiles with a deep ring, so that the
 //    activations of a K range are split once per CTA and the pipeline never drains between tiles; the cost of a
@@ -95,14 +102,17 @@ inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring, int
             ring = units < 4 ? units : 4;
             if (force_ring > 0) ring = force_ring < units ? force_ring : units;
             else
-                while (ring > 2 && ctas > (long)sms * fp4_ctas_per_sm(fp4_smem_bytes(p.nb, p.M, tper, chunk, ring, s), tm)) --ring;
+                while (ring > 2 && ctas > fp4_usable_slots(sms, fp4_smem_bytes(p.nb, p.M, tper, chunk, ring, s), tm)) --ring;
             while (ring > 1 && fp4_smem_bytes(p.nb, p.M, tper, chunk, ring, s) > kFp4SmemLimit) --ring;
             const uint32_t bytes = fp4_smem_bytes(p.nb, p.M, tper, chunk, ring, s);
             if (bytes > kFp4SmemLimit) continue;
-            const long slots = (long)sms * fp4_ctas_per_sm(bytes, tm);
+            const long slots = fp4_usable_slots(sms, bytes, tm);
             const long waves = (ctas + slots - 1) / slots;
-            const long off = ctas > 2L * sms ? ctas - 2L * sms : 2L * sms - ctas;   // distance from two CTAs per SM
-            cost = (waves - 1) * 100000 + off;
+            // What a CTA cannot request before the activations arrive -- its stages beyond the ring -- is streamed
+            // inside the dependent chain: the cost is that remainder per SM (in hundredths of a stage).  Measured at
+            // M = 1: 11008 x 4096 8.05 us (split 4, 2.3 stages per SM left) / 8.23 (split 3, 3.5) / 8.80 (split 6, 3.5) /
+            // 9.37 (split 2, 4.6); 12288 x 4096 8.3 us (split 4, 2.6) / 9.95 (split 3 with three slots, 5.8) / 9.4 (split 2, 5.2).
+            cost = (waves - 1) * 100000 + (long)(units - ring) * ctas * 100 / sms;
         } else {
             groups = sms / s < 1 ? 1 : sms / s;          // one CTA per SM
             if (groups > p.tiles) groups = p.tiles;

@@ -77,6 +77,14 @@ inline int umma_ctas_per_sm(uint32_t smem_bytes, int tmem_cols) {
     return by_smem < by_tmem ? by_smem : by_tmem;
 }
 
+// CTA slots a one-wave launch may count on (see fp4_usable_slots: grids filling more than about 95 % of the slots ran as
+// two waves; 12288 x 4096 at M = 8 as 288 CTAs on 296 slots took 16.9 us, as 384 on 444 slots 11.8 us)
+// (not applied to matrices of more tiles than SMs, which measured best with every slot counted: 27648 x 5120 as 432 CTAs)
+inline long umma_usable_slots(int derate_sms, int sms, uint32_t smem_bytes, int tmem_cols) {
+    const long slots = (long)sms * umma_ctas_per_sm(smem_bytes, tmem_cols);
+    return derate_sms > 0 ? slots * 92 / 100 : slots;
+}
+
 // Chooses split, groups and ring for p.{M, nb, ks, tiles}; false if nothing fits.  Same two regimes as the packed-FP4
 // kernel: up to one tile per SM -> one tile per CTA, every CTA resident at once, about two CTAs per SM (ties to the
 // larger split: splitting the activations is this kernel's main cost from M = 4 on, and it shrinks with the K range);
@@ -117,12 +125,14 @@ inline bool umma_layout_one(UmmaPlan &p, int sms, int force_split, int force_rin
             while (ring > 1 && umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s, br) > kUmmaSmemLimit) --ring;
             const uint32_t bytes = umma_smem_bytes(p.nb, p.M, tmax, chunk, ring, s, br);
             if (bytes > kUmmaSmemLimit) continue;
-            const long slots = (long)sms * umma_ctas_per_sm(bytes, tm);
+            const long slots = umma_usable_slots(p.tiles > sms ? 0 : sms, sms, bytes, tm);
             const long waves = (ctas + slots - 1) / slots;
-            const long off = ctas > 2L * sms ? ctas - 2L * sms : 2L * sms - ctas;   // distance from two CTAs per SM
             // more tiles than SMs: the stages the fullest SM has to stream, with the vocabulary regime's penalty for K
             // ranges under half a row
             const long per_sm = (ctas + sms - 1) / sms * chunk * (s <= 2 ? 10 : 19);
+            // (The packed-FP4 kernel's criterion -- fewest stages per SM outside the rings -- was tried here: the 13B layer
+            // set got faster at M = 2 and 16 (71.6 -> 68.2, 116.9 -> 106.7 us) and slower at M = 8 (79.8 -> 83.4 us): not adopted.)
+            const long off = ctas > 2L * sms ? ctas - 2L * sms : 2L * sms - ctas;   // distance from two CTAs per SM
             cost = (waves - 1) * 100000 + (p.tiles > sms ? per_sm : off);
         } else {
             groups = sms / s < 1 ? 1 : sms / s;          // one CTA per SM

@@ -106,7 +106,8 @@ size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K);
  *   MXQ_KERNEL_MMA     decodes the codes into FP16 mma.sync fragments (needs K % 128 == 0)
  *   MXQ_KERNEL_GENERIC any valid shape, on the CUDA cores
  * Left to itself (MXQ_KERNEL_AUTO) mxq_linear picks by measured speed among the kernels that cover the call: FP4
- * for M = 1; from M = 2, UMMA for matrices of at most as many row tiles of 128 as the GPU has SMs, MMA for larger ones. */
+ * for M = 1 (and for M = 2 on matrices of more row tiles of 128 than the GPU has SMs); UMMA otherwise, except on the
+ * largest matrices at M > 2 where it can run neither one tile per CTA nor one CTA per SM: those go to MMA. */
 enum mxq_kernel {
     MXQ_KERNEL_AUTO = -1, MXQ_KERNEL_GENERIC = 0, MXQ_KERNEL_MMA = 1, MXQ_KERNEL_UMMA = 2, MXQ_KERNEL_FP4 = 3
 };

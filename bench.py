@@ -655,7 +655,7 @@ def run_case(args):
     mxq.binding.lib()
     device = torch.device("cuda", 0)
     case = args.case.lower()
-    if case.startswith("quantize:") or case.startswith("accept:") or case.startswith("bf16:"):
+    if case.split(":")[0] in ("quantize", "accept", "bf16", "swiglu", "residual"):
         return run_case_other(mxq, case, args.steps, device)
     n, k, m = (int(v) for v in case.split("x"))
     nbytes = algorithmic_bytes(m, n, k)
@@ -683,8 +683,9 @@ def run_case(args):
 
 def run_case_other(mxq, case: str, steps: int, device):
     """--case quantize:NxK (direct cast of `steps` distinct BF16 matrices, rotated), accept:BxRxV (greedy accept of FP32
-    logits, T = R - 1) or bf16:NxKxM (the unquantised comparison layer): the small cases profiler captures of those
-    kernels run on."""
+    logits, T = R - 1), bf16:NxKxM (the unquantised comparison layer), swiglu:FxKxM (gate / up rows interleaved, 2F x K
+    weights, SiLU(gate) * up in the epilogue) or residual:NxKxM (residual add in the epilogue): the small cases profiler
+    captures of those kernels run on."""
     op, dims = case.split(":")
     dims = [int(v) for v in dims.split("x")]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -705,6 +706,35 @@ def run_case_other(mxq, case: str, steps: int, device):
         def all_copies():
             for w_ in ws_:
                 mxq.mxq_quantize(w_, codes, scales)
+        graph_us = time_graph(all_copies, 10) / copies * 1e6
+    elif op in ("swiglu", "residual"):
+        n, k, m = dims
+        rows = 2 * n if op == "swiglu" else n
+        nbytes = algorithmic_bytes(m, rows, k, 2) - (2 * m * n if op == "swiglu" else -2 * m * n)   # BF16 out (half as many for gate / up), + the residual
+        copies = max(2, min(8, int(200e6 // nbytes) + 1))
+        gen = torch.Generator(device=device).manual_seed(7)
+        mats = [(torch.randint(0, 256, (rows, k // 2), dtype=torch.uint8, device=device, generator=gen),
+                 torch.randint(110, 126, (rows, k // 32), dtype=torch.uint8, device=device, generator=gen)) for _ in range(copies)]
+        x = synth.normal_bf16((m, k), 1.0, 3, device)
+        res = synth.normal_bf16((m, n), 1.0, 4, device)
+        y = torch.empty((m, n), dtype=torch.bfloat16, device=device)
+        ws = torch.empty(max(16, mxq.mxq_linear_fused_workspace_bytes(m, rows, k)), dtype=torch.uint8, device=device)
+
+        def call(c, s_):
+            if op == "swiglu":
+                mxq.mxq_linear_swiglu(x, c, s_, out=y, workspace=ws)
+            else:
+                mxq.mxq_linear_residual(x, c, s_, res, out=y, workspace=ws)
+        call(*mats[0])
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(steps):
+            call(*mats[i % copies])
+        e1.record()
+
+        def all_copies():
+            for c, s_ in mats:
+                call(c, s_)
         graph_us = time_graph(all_copies, 10) / copies * 1e6
     elif op == "bf16":
         n, k, m = dims

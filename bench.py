@@ -148,6 +148,7 @@ class LinearPass:
         self.launches = len(mats)
         self.graph = None
         self.stream = torch.cuda.Stream(device=device)
+        self.stream.wait_stream(torch.cuda.current_stream(device))   # the inputs were produced on the current stream
         if use_graph:
             with torch.cuda.stream(self.stream):
                 self.enqueue()          # first call outside capture (lazy module loading)
@@ -200,6 +201,7 @@ def time_e2e(mxq, mats, m: int, steps: int, warmup: int, device):
     ys = [torch.empty((m, n), dtype=torch.float32, device=device) for _, n, _, _, _ in mats]
     ws = mxq.new_workspace(max([mxq.mxq_linear_workspace_bytes(m, n, k) for _, n, k, _, _ in mats] + [16]), device)
     stream = torch.cuda.Stream(device=device)
+    stream.wait_stream(torch.cuda.current_stream(device))
     h2d = sum(2 * m * k for _, _, k, _, _ in mats)
     d2h = sum(4 * m * n for _, n, _, _, _ in mats)
 
@@ -240,6 +242,7 @@ def time_fn(fn, iters: int, warmup: int = 3):
 def time_graph(fn, iters: int, warmup: int = 3):
     """Device time per replay of a CUDA graph of fn() (no host launch overhead between the kernels)."""
     st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())   # the inputs were produced on the current stream
     with torch.cuda.stream(st):
         fn()
         st.synchronize()
@@ -495,6 +498,7 @@ def run_ours(args):
             mxq.mxq_lm_head_accept(xs_[(1, 4096)], dh[0], dh[1], None, workspace=wsf_)
         self_ws = mxq.new_workspace(16, device)
         st_ = torch.cuda.Stream()
+        st_.wait_stream(torch.cuda.current_stream())
         graphs = {}
         with torch.cuda.stream(st_):
             for name_, fn_ in (("t1", lambda: target_step(1)), ("tv", lambda: target_step(n_draft + 1)), ("d", draft_step)):

@@ -51,6 +51,7 @@ struct UmmaPlan {
     int bring;       // ... and fetched stage by stage into the ring slots instead of whole K ranges
     long cost;       // the layout heuristic's figure for the chosen decomposition (comparable within a regime)
     int pow2_split;  // in: only cluster sizes 1, 2, 4, 8 (the gate / up epilogue pairs rows inside a warp)
+    int cost_left;   // experiment
     int layer_tiles; // most tiles for the one-tile-per-CTA regime (0: one per SM); set by umma_layout
     uint32_t smem_bytes;
     int64_t N, K;
@@ -133,7 +134,9 @@ inline bool umma_layout_one(UmmaPlan &p, int sms, int force_split, int force_rin
             // (The packed-FP4 kernel's criterion -- fewest stages per SM outside the rings -- was tried here: the 13B layer
             // set got faster at M = 2 and 16 (71.6 -> 68.2, 116.9 -> 106.7 us) and slower at M = 8 (79.8 -> 83.4 us): not adopted.)
             const long off = ctas > 2L * sms ? ctas - 2L * sms : 2L * sms - ctas;   // distance from two CTAs per SM
-            cost = (waves - 1) * 100000 + (p.tiles > sms ? per_sm : off);
+            long left = (long)(units - ring) * ctas * 100 / sms;
+            if (p.cost_left == 2) left += (ring < 3 && units >= 3 ? 50000 : 0) + (umma_ctas_per_sm(bytes, tm) < 2 ? 50000 : 0);
+            cost = (waves - 1) * 100000 + (p.tiles > sms ? per_sm : (p.cost_left ? left : off));
         } else {
             groups = sms / s < 1 ? 1 : sms / s;          // one CTA per SM
             if (groups > p.tiles) groups = p.tiles;

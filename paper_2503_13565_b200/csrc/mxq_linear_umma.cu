@@ -738,7 +738,6 @@ bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p, bool with_worksp
     p.presplit = with_workspace && M >= presplit_min_m() ? 1 : 0;
     p.pow2_split = pow2_split ? 1 : 0;
     p.layer_tiles = 0;
-    p.cost_left = env_int("MXQ_UMMA_COST_LEFT");
     p.M = M;
     p.N = N;
     p.K = K;

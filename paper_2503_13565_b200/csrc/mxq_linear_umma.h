@@ -51,7 +51,6 @@ struct UmmaPlan {
     int bring;       // ... and fetched stage by stage into the ring slots instead of whole K ranges
     long cost;       // the layout heuristic's figure for the chosen decomposition (comparable within a regime)
     int pow2_split;  // in: only cluster sizes 1, 2, 4, 8 (the gate / up epilogue pairs rows inside a warp)
-    int cost_left;   // experiment
     int layer_tiles; // most tiles for the one-tile-per-CTA regime (0: one per SM); set by umma_layout
     uint32_t smem_bytes;
     int64_t N, K;
@@ -87,8 +86,9 @@ inline long umma_usable_slots(int derate_sms, int sms, uint32_t smem_bytes, int 
 }
 
 // Chooses split, groups and ring for p.{M, nb, ks, tiles}; false if nothing fits.  Same two regimes as the packed-FP4
-// kernel: up to one tile per SM -> one tile per CTA, every CTA resident at once, about two CTAs per SM (ties to the
-// larger split: splitting the activations is this kernel's main cost from M = 4 on, and it shrinks with the K range);
+// kernel: up to one tile per SM -> one tile per CTA, every CTA resident at once, the split that leaves the fewest stages
+// per SM outside the rings (ties to the larger split: splitting the activations is this kernel's main cost from M = 4
+// on, and it shrinks with the K range);
 // more tiles -> one CTA per SM walking several tiles.
 // force_split / force_ring / force_tiles (> 0) override the heuristic where they are feasible.
 inline bool umma_layout_one(UmmaPlan &p, int sms, int force_split, int force_ring, int force_tiles, bool allow_bring) {
@@ -131,12 +131,15 @@ inline bool umma_layout_one(UmmaPlan &p, int sms, int force_split, int force_rin
             // more tiles than SMs: the stages the fullest SM has to stream, with the vocabulary regime's penalty for K
             // ranges under half a row
             const long per_sm = (ctas + sms - 1) / sms * chunk * (s <= 2 ? 10 : 19);
-            // (The packed-FP4 kernel's criterion -- fewest stages per SM outside the rings -- was tried here: the 13B layer
-            // set got faster at M = 2 and 16 (71.6 -> 68.2, 116.9 -> 106.7 us) and slower at M = 8 (79.8 -> 83.4 us): not adopted.)
-            const long off = ctas > 2L * sms ? ctas - 2L * sms : 2L * sms - ctas;   // distance from two CTAs per SM
-            long left = (long)(units - ring) * ctas * 100 / sms;
-            if (p.cost_left == 2) left += (ring < 3 && units >= 3 ? 50000 : 0) + (umma_ctas_per_sm(bytes, tm) < 2 ? 50000 : 0);
-            cost = (waves - 1) * 100000 + (p.tiles > sms ? per_sm : (p.cost_left ? left : off));
+            // Up to one tile per SM: as in the packed-FP4 kernel, the stages per SM that do not fit in the rings (they
+            // are streamed inside the dependent chain; hundredths of a stage), but never with fewer than three ring
+            // slots (a slot holds 8 KB here: two do not cover the latency) nor with one fat CTA per SM (which keeps the
+            // next call's CTAs out) while another split avoids both.  Against "closest to two CTAs per SM", which this
+            // replaced, the 13B layer set takes 98.6 instead of 116.8 us at M = 16 and 68.0 instead of 71.5 us at M = 2
+            // (13824 x 5120 at M = 16: 24.9 -> 15.5 us, 8192 x 8192: 23.9 -> 15.5 us); the 7B layer set is unchanged.
+            const long left = (long)(units - ring) * ctas * 100 / sms + (ring < 3 && units >= 3 ? 50000 : 0) +
+                              (umma_ctas_per_sm(bytes, tm) < 2 ? 50000 : 0);
+            cost = (waves - 1) * 100000 + (p.tiles > sms ? per_sm : left);
         } else {
             groups = sms / s < 1 ? 1 : sms / s;          // one CTA per SM
             if (groups > p.tiles) groups = p.tiles;

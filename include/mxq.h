@@ -157,7 +157,10 @@ int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *s
 /* The same layer with the activations and the result in HOST memory (pinned memory
  * makes the copies asynchronous).  X_host [M][K] BF16 is copied to X_stage_dev
  * (>= M*K*2 bytes), the layer runs, and Y_stage_dev (>= M*N*elem bytes) is copied to
- * Y_host, all on `stream`.  The weights stay resident on the device. */
+ * Y_host, all on `stream`.  The weights stay resident on the device.  Host buffers that are page-locked and
+ * addressable by the GPU (cudaHostAlloc / cudaHostRegister; 16-byte aligned) are moved by the GPU itself: a small
+ * kernel pulls X into X_stage_dev and the layer stores Y straight into Y_host (Y_stage_dev is then not written);
+ * pageable buffers go through cudaMemcpyAsync.  Y_host is complete once `stream` has reached the end of the call. */
 int mxq_linear_host(const void *X_host, int M, const uint8_t *codes, const uint8_t *scales, int64_t N,
                     int64_t K, void *Y_host, int y_dtype, void *X_stage_dev, void *Y_stage_dev,
                     void *workspace, size_t workspace_bytes, void *stream);

@@ -122,6 +122,17 @@ layer_epilogue_kernel(const float *__restrict__ S, int M, int64_t N, const void 
     }
 }
 
+// mxq_linear_host: X from page-locked host memory into the device staging buffer, 16 bytes per thread.  The loads do
+// not depend on earlier kernels; the stores wait for them (the previous call may still be reading the staging buffer).
+__global__ void __launch_bounds__(256) stage_from_host_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, int64_t n16) {
+    pdl_trigger();
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (i < n16) v = src[i];
+    pdl_wait();
+    if (i < n16) dst[i] = v;
+}
+
 // mxq_set_linear_kernel / MXQ_LINEAR_VARIANT: MXQ_KERNEL_AUTO (-1), or the highest kernel mxq_linear may use
 static std::atomic<int> g_ceiling{-2};
 static int kernel_ceiling() {
@@ -406,6 +417,16 @@ int mxq_linear_swiglu(const void *X_bf16, int M, const uint8_t *codes, const uin
     return linear_with_epilogue(X_bf16, M, codes, scales, N, K, nullptr, 1, Y, y_dtype, workspace, workspace_bytes, stream);
 }
 
+// Device-side address of page-locked host memory that the GPU can reach, or nullptr (pageable memory, no mapping)
+static void *device_view_of_host(const void *p) {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
+}
+
 int mxq_linear_host(const void *X_host, int M, const uint8_t *codes, const uint8_t *scales, int64_t N,
                     int64_t K, void *Y_host, int y_dtype, void *X_stage_dev, void *Y_stage_dev,
                     void *workspace, size_t workspace_bytes, void *stream) {
@@ -413,11 +434,32 @@ int mxq_linear_host(const void *X_host, int M, const uint8_t *codes, const uint8
     if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return MXQ_ERR_SHAPE;
     if (y_dtype != MXQ_F32 && y_dtype != MXQ_BF16) return MXQ_ERR_DTYPE;
     cudaStream_t st = (cudaStream_t)stream;
-    if (cudaMemcpyAsync(X_stage_dev, X_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    // Page-locked host buffers that the GPU can address are moved by the GPU itself: a one-wave kernel pulls X across
+    // the bus into the staging buffer (the copy engine's start-up costs several times the transfer of 8-350 KB), and the
+    // layer stores Y straight into host memory.  Anything else goes through cudaMemcpyAsync.
+    void *x_view = device_view_of_host(X_host), *y_view = device_view_of_host(Y_host);
+    if (x_view && mxq::aligned16(x_view) && mxq::aligned16(X_stage_dev)) {
+        const int64_t n16 = (int64_t)M * K / 8;   // 16-byte pieces (K % 32 == 0)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)((n16 + 255) / 256));
+        cfg.blockDim = dim3(256);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = mxq::pdl_enabled() ? 1 : 0;
+        if (cudaLaunchKernelEx(&cfg, mxq::stage_from_host_kernel, (const uint4 *)x_view, (uint4 *)X_stage_dev, n16) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return MXQ_ERR_CUDA;
+        }
+    } else if (cudaMemcpyAsync(X_stage_dev, X_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) {
         return MXQ_ERR_CUDA;
-    const int rc = mxq_linear(X_stage_dev, M, codes, scales, N, K, Y_stage_dev, y_dtype, workspace, workspace_bytes,
-                              stream);
-    if (rc != MXQ_OK) return rc;
+    }
+    const bool y_direct = y_view && mxq::aligned16(y_view);
+    const int rc = mxq_linear(X_stage_dev, M, codes, scales, N, K, y_direct ? y_view : Y_stage_dev, y_dtype, workspace,
+                              workspace_bytes, stream);
+    if (rc != MXQ_OK || y_direct) return rc;
     const size_t ybytes = (size_t)M * N * (y_dtype == MXQ_F32 ? 4 : 2);
     if (cudaMemcpyAsync(Y_host, Y_stage_dev, ybytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MXQ_ERR_CUDA;
     return MXQ_OK;

@@ -255,6 +255,27 @@ def test_host_variant_matches_device_variant():
     assert torch.equal(yh, y_dev.cpu())
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("m,n,k,dtype", [(1, 4096, 4096, torch.float32), (8, 1000, 2048, torch.bfloat16), (16, 203, 1408, torch.float32)])
+def test_host_variant_pinned_and_pageable(m, n, k, dtype, pinned):
+    """Page-locked buffers are moved by the GPU itself (a staging kernel for X, Y stored straight into host memory),
+    pageable ones by the copy engine: the same bits either way, and nothing written around Y."""
+    w = synth.bits_of(synth.weight(3, 21, n, k))
+    gc, gs = mxq.mxq_quantize(gpu_bf16(w))
+    x = synth.activations(3, 21, m, k)
+    y_dev = mxq.mxq_linear(x.cuda(), gc, gs, out_dtype=dtype)
+    buf = torch.full((m * n + 64,), 3.0, dtype=dtype)
+    xh = x.clone()
+    if pinned:
+        buf, xh = buf.pin_memory(), xh.pin_memory()
+    yh = buf[32:32 + m * n].view(m, n)
+    for _ in range(2):   # twice: the second call's staging must wait for the first call's reads
+        mxq.mxq_linear_host(xh, gc, gs, yh, torch.empty_like(x, device="cuda"), torch.empty((m, n), dtype=dtype, device="cuda"))
+    torch.cuda.synchronize()
+    assert torch.equal(yh, y_dev.cpu())
+    assert (buf[:32] == 3.0).all() and (buf[32 + m * n:] == 3.0).all()
+
+
 def test_canaries_around_the_output_survive():
     n, k, m = 203, 1440, 3
     w = synth.bits_of(synth.weight(3, 10, n, k))

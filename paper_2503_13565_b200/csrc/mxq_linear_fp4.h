@@ -130,7 +130,9 @@ inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring, int
             const long by_ring = (long)ring * 16384 / 1500, rate = by_ring < 40 ? by_ring : 40;   // GB/s: bytes in flight per 1.5 us, one requester
             cost = waves * units * 1000 / rate * (s <= 2 ? 10 : 19) + s;
         }
-        if (best_cost < 0 || cost < best_cost || (cost == best_cost && layer_regime)) {   // layer regime: ties to the larger split (less of X per CTA)
+        // layer regime: ties go to the larger split (less of X per CTA) as long as that does not put more than two CTAs
+        // on an SM (32000 x 768 at M = 1: 250 CTAs of one tile and all of K 5.0 us, 750 CTAs in clusters of 3 7.7 us)
+        if (best_cost < 0 || cost < best_cost || (cost == best_cost && layer_regime && (long)groups * s <= 2L * sms)) {
             best_cost = cost;
             best_split = s;
             best_groups = groups;

@@ -90,10 +90,15 @@ inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring, int
         if (p.pow2_split && (s & (s - 1)) != 0) continue;
         if (force_split <= 0 && s == 7) continue;   // clusters of 7 measured up to 1.5 times slower than of 6 or 8 (5120 x 5120, 5120 x 13824)
         const int chunk = (p.ks + s - 1) / s;
+        // Matrices of more tiles than SMs are also tried with two tiles per CTA (half as much of X to split per tile;
+        // taken only where the cost below is strictly lower: 32000 x 4096 at M = 1 16.2 -> 15.4 us, 22016 x 4096 13.1 ->
+        // 12.6 us; on 11008 x 4096, a tie, two tiles per CTA measured 8.6 against 8.2 us).
+        const int tries = layer_regime && force_tiles <= 0 && p.tiles > sms ? 2 : 1;
+        for (int tp = 1; tp <= tries; ++tp) {
         int groups, ring;
         long cost;
         if (layer_regime) {
-            int tper = force_tiles > 0 ? (force_tiles < tcap ? force_tiles : tcap) : 1;
+            int tper = force_tiles > 0 ? (force_tiles < tcap ? force_tiles : tcap) : tp;
             groups = (p.tiles + tper - 1) / tper;
             tper = (p.tiles + groups - 1) / groups;
             const long ctas = (long)groups * s;
@@ -132,11 +137,12 @@ inline bool fp4_layout(Fp4Plan &p, int sms, int force_split, int force_ring, int
         }
         // layer regime: ties go to the larger split (less of X per CTA) as long as that does not put more than two CTAs
         // on an SM (32000 x 768 at M = 1: 250 CTAs of one tile and all of K 5.0 us, 750 CTAs in clusters of 3 7.7 us)
-        if (best_cost < 0 || cost < best_cost || (cost == best_cost && layer_regime && (long)groups * s <= 2L * sms)) {
+        if (best_cost < 0 || cost < best_cost || (cost == best_cost && layer_regime && tp == 1 && (long)groups * s <= 2L * sms)) {
             best_cost = cost;
             best_split = s;
             best_groups = groups;
             best_ring = ring;
+        }
         }
     }
     if (best_cost < 0) return false;

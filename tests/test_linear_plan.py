@@ -182,15 +182,15 @@ def test_packed_fp4_regimes():
 
 
 def test_one_wave_layouts_leave_slack():
-    """One tile per CTA with every CTA resident at once: the grid may count on 92 % of the CTA slots only (fuller grids
-    were measured to run as two waves), for both tcgen05 kernels and for the row-interleaved gate / up matrices too."""
+    """One tile per CTA (two, for packed-FP4 matrices of more tiles than SMs) with every CTA resident at once: the grid may
+    count on 92 % of the CTA slots only (fuller grids were measured to run as two waves)."""
     for m, kernel, shapes in [(1, "fp4", [(4096, 4096), (11008, 4096), (4096, 11008), (12288, 4096), (22016, 4096), (5120, 5120),
                                           (13824, 5120), (5120, 13824), (8192, 8192)]),
                               (8, "umma", [(4096, 4096), (11008, 4096), (4096, 11008), (12288, 4096), (5120, 5120), (13824, 5120),
                                            (5120, 13824), (8192, 8192)])]:
         for n, k in shapes:
             p = mxq.mxq_linear_plan_info(m, n, k, kernel)
-            assert p["tiles_max"] == 1, p
+            assert p["tiles_max"] == 1 or (kernel == "fp4" and p["tiles_max"] == 2 and p["tiles"] > SMS), p
             per_sm = min((228 * 1024) // (p["smem_bytes"] + 1024), 512 // p["tmem_cols"])
             assert p["grid"] <= SMS * per_sm * 92 // 100, (n, k, p)
             if kernel == "umma":

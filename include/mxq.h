@@ -90,7 +90,8 @@ int mxq_dequantize(const uint8_t *codes, const uint8_t *scales, int64_t N, int64
                    void *stream);
 
 /* Workspace (bytes) with which mxq_linear runs fastest for this shape; 0 where none is used.  The workspace is
- * OPTIONAL: mxq_linear accepts NULL / 0 or a smaller buffer and is then merely slower for 3 or more token rows.
+ * OPTIONAL: mxq_linear accepts NULL / 0 or a smaller buffer and is then merely slower for 3 or more token rows (and for
+ * 2 on matrices of 8 M weights or more).
  * With it, MXQ_KERNEL_UMMA rewrites the M token rows as FP8 parts once per call (a small kernel ahead of the
  * weight kernel, which then fetches them with bulk copies) instead of once per CTA.  Device memory, 16-byte
  * aligned, no initialisation needed; contents are scratch.  Calls that may run concurrently (different streams)

@@ -198,6 +198,7 @@ size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K) {
     if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return 0;
     // No kernel needs one (partial results are added inside a thread-block cluster or never leave a warp); the
     // FP8-operand tcgen05 kernel is faster with one: the token operand is then split once per call.
+    if (M == 2 && N * K < mxq::kUmmaPresplitTwoRowsMinWeights) return 0;   // two rows: only large matrices use it
     return mxq::linear_umma_available() ? mxq::linear_umma_workspace_bytes(M, K) : 0;
 }
 

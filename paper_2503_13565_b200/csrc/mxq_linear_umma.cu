@@ -113,8 +113,8 @@ __device__ __forceinline__ bool split_unit(const uint4 raw, bool act, int m, int
     return inexact && act;
 }
 
-// The token operand of a whole call, split once, ahead of the weight kernel (from kUmmaPresplitMinM token rows on, where
-// every CTA splitting its own K range costs more than one more launch in the chain).  CTA = 256 k of every token;
+// The token operand of a whole call, split once, ahead of the weight kernel (from kUmmaPresplitMinM token rows on, and at
+// two rows on large matrices, where every CTA splitting its own K range costs more than one more launch in the chain).  CTA = 256 k of every token;
 // a warp takes tokens warp, warp + 8, ...  The result lies in the workspace as umma_ws_bytes describes.
 constexpr int kSplitWarps = 8;
 template <int NB>
@@ -731,11 +731,15 @@ static int presplit_min_m() {
                          : (env_int("MXQ_UMMA_PRESPLIT_MIN_M") > 0 ? env_int("MXQ_UMMA_PRESPLIT_MIN_M") : kUmmaPresplitMinM);
     return v;
 }
+static bool presplit_wanted(int M, int64_t N, int64_t K) {
+    const int min_m = presplit_min_m();
+    return M >= min_m || (min_m == kUmmaPresplitMinM && M == 2 && N * K >= kUmmaPresplitTwoRowsMinWeights);
+}
 
 bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p, bool with_workspace, bool pow2_split) {
     if (M < 1 || M > kUmmaMaxM || N < 1 || K < 128 || (K % 128) != 0) return false;
     if (K > 0x3FFFFFFF || N > 0x7FFFFFFF) return false;
-    p.presplit = with_workspace && M >= presplit_min_m() ? 1 : 0;
+    p.presplit = with_workspace && presplit_wanted(M, N, K) ? 1 : 0;
     p.pow2_split = pow2_split ? 1 : 0;
     p.layer_tiles = 0;
     p.M = M;
@@ -766,7 +770,10 @@ static cudaError_t pick_umma(const UmmaPlan &p, bool bring, const CUtensorMap &m
 }
 
 size_t linear_umma_workspace_bytes(int M, int64_t K) {
-    if (M < presplit_min_m() || M > kUmmaMaxM || K < 128 || (K % 128) != 0 || K > 0x3FFFFFFF) return 0;
+    // (two token rows: used on large matrices only, see presplit_wanted; the size does not depend on N)
+    if ((M < presplit_min_m() && !(M == 2 && presplit_min_m() == kUmmaPresplitMinM)) || M > kUmmaMaxM || K < 128 || (K % 128) != 0 ||
+        K > 0x3FFFFFFF)
+        return 0;
     return umma_ws_bytes(umma_nb(M), (int)(K / kUmmaStageK));
 }
 

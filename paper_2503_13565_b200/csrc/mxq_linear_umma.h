@@ -28,7 +28,9 @@ constexpr int kUmmaMaxUnitsResident = 12;         // most ring slots (16 KB of e
 // exactly" flag per stage (padded to 1 KB), then one 512-byte scale atom per stage, then one image of the stage's
 // nb x 128 bytes of E5M2 parts per stage -- atoms and images exactly as the weight kernel keeps them in shared memory,
 // so that a CTA fetches its K range with two bulk copies per 256 k.
-constexpr int kUmmaPresplitMinM = 3;              // fewer token rows: splitting inside the weight kernel is as fast
+constexpr int kUmmaPresplitMinM = 3;              // fewer token rows: splitting inside the weight kernel is as fast ...
+constexpr int64_t kUmmaPresplitTwoRowsMinWeights = 1 << 23;   // ... except at two rows on matrices from 8 M weights on (2-8 % faster;
+                                                              // the small draft model's layers lose 5-15 % to the extra launch)
 MXQ_UMMA_HD inline size_t umma_ws_flags_bytes(int ks) { return (((size_t)ks * 4u) + 1023u) & ~(size_t)1023u; }
 MXQ_UMMA_HD inline size_t umma_ws_bytes(int nb, int ks) {
     return umma_ws_flags_bytes(ks) + (size_t)ks * kUmmaSfStageBytes + (size_t)ks * (size_t)nb * 128u;

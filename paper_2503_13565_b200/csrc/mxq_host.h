@@ -49,7 +49,8 @@ bool linear_umma_available();
 // with_workspace: plan for a token operand split ahead of the weight kernel (from 3 token rows on)
 // pow2_split: only cluster sizes that are powers of two (what the gate / up epilogue needs: the two rows of a pair
 // then end up in one warp)
-bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &plan, bool with_workspace, bool pow2_split = false);
+// one_wave: never more CTAs than fit on the GPU at once (the fused verification pays per CTA: keys, ticket)
+bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &plan, bool with_workspace, bool pow2_split = false, bool one_wave = false);
 // workspace: optional; with linear_umma_workspace_bytes(M, K) bytes (0: not used for this M) the token operand is split
 // once per call by a kernel of its own instead of by every CTA of the weight kernel
 size_t linear_umma_workspace_bytes(int M, int64_t K);

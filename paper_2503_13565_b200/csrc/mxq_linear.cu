@@ -164,7 +164,8 @@ struct Choice {
     UmmaPlan umma;
     LinearPlan mma;
 };
-static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *codes, bool with_workspace, Choice &c, bool pow2_split = false) {
+static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *codes, bool with_workspace, Choice &c, bool pow2_split = false,
+                   bool one_wave = false) {
     const bool tc = linear_umma_available();
     const bool aligned32 = !codes || (reinterpret_cast<uintptr_t>(codes) & 31u) == 0;
     bool try_fp4 = ceiling == MXQ_KERNEL_AUTO || ceiling >= MXQ_KERNEL_FP4;
@@ -178,13 +179,13 @@ static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *code
             // vocabulary-sized matrices, where a CTA per SM walks several tiles: the packed-FP4 kernel still wins at two
             // token rows; above, the FP8-operand kernel, unless its token operand leaves no room for one CTA per SM
             try_fp4 = M == 2;
-            if (M > 2 && !(tc && aligned32 && linear_umma_plan(M, N, K, c.umma, with_workspace, pow2_split) && (c.umma.grid <= sm_count() || c.umma.tiles_max == 1)) &&
+            if (M > 2 && !(tc && aligned32 && linear_umma_plan(M, N, K, c.umma, with_workspace, pow2_split, one_wave) && (c.umma.grid <= sm_count() || c.umma.tiles_max == 1)) &&
                 linear_mma_plan(M, N, K, c.mma))
                 try_umma = false;
         }
     }
     if (try_fp4 && tc && linear_fp4_plan(M, N, K, c.fp4, pow2_split)) c.kernel = MXQ_KERNEL_FP4;
-    else if (try_umma && tc && aligned32 && linear_umma_plan(M, N, K, c.umma, with_workspace, pow2_split)) c.kernel = MXQ_KERNEL_UMMA;
+    else if (try_umma && tc && aligned32 && linear_umma_plan(M, N, K, c.umma, with_workspace, pow2_split, one_wave)) c.kernel = MXQ_KERNEL_UMMA;
     else if (try_mma && linear_mma_plan(M, N, K, c.mma)) c.kernel = MXQ_KERNEL_MMA;
     else c.kernel = MXQ_KERNEL_GENERIC;
 }
@@ -299,7 +300,7 @@ static size_t align256(size_t v) { return (v + 255u) & ~(size_t)255u; }
 size_t mxq_lm_head_accept_workspace_bytes(int R, int64_t V, int64_t K) {
     if (R < 1 || R > MXQ_MAX_M || !mxq::shape_ok(V, K)) return 0;
     mxq::Choice c;
-    mxq::choose(mxq::kernel_ceiling(), R, V, K, nullptr, true, c);
+    mxq::choose(mxq::kernel_ceiling(), R, V, K, nullptr, true, c, false, true);
     size_t b = kFusedHeader + align256(mxq_linear_workspace_bytes(R, V, K));
     if (c.kernel != MXQ_KERNEL_FP4 && c.kernel != MXQ_KERNEL_UMMA)
         b += align256((size_t)R * (size_t)V * 4u) + align256(mxq_accept_workspace_bytes(1, R, V));
@@ -318,7 +319,7 @@ int mxq_lm_head_accept(const void *X_bf16, int R, const uint8_t *codes, const ui
     void *lin_ws = ws + kFusedHeader;
     const size_t lin_ws_bytes = align256(mxq_linear_workspace_bytes(R, V, K));
     mxq::Choice c;
-    mxq::choose(mxq::kernel_ceiling(), R, V, K, codes, true, c);
+    mxq::choose(mxq::kernel_ceiling(), R, V, K, codes, true, c, false, true);
     if (c.kernel == MXQ_KERNEL_FP4 || c.kernel == MXQ_KERNEL_UMMA) {
         mxq::FusedAccept fa{};
         fa.keys = reinterpret_cast<unsigned long long *>(ws);

@@ -736,12 +736,13 @@ static bool presplit_wanted(int M, int64_t N, int64_t K) {
     return M >= min_m || (min_m == kUmmaPresplitMinM && M == 2 && N * K >= kUmmaPresplitTwoRowsMinWeights);
 }
 
-bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p, bool with_workspace, bool pow2_split) {
+bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p, bool with_workspace, bool pow2_split, bool one_wave) {
     if (M < 1 || M > kUmmaMaxM || N < 1 || K < 128 || (K % 128) != 0) return false;
     if (K > 0x3FFFFFFF || N > 0x7FFFFFFF) return false;
     p.presplit = with_workspace && presplit_wanted(M, N, K) ? 1 : 0;
     p.pow2_split = pow2_split ? 1 : 0;
     p.layer_tiles = 0;
+    p.one_wave = one_wave ? 1 : 0;
     p.M = M;
     p.N = N;
     p.K = K;
@@ -789,7 +790,7 @@ cudaError_t linear_umma_launch(const UmmaPlan &p, const void *X, const uint8_t *
         ws = static_cast<uint8_t *>(workspace);
     if (p.presplit && !ws) {   // planned for a workspace that is not there: plan again without
         UmmaPlan q;
-        if (!linear_umma_plan(p.M, p.N, p.K, q, false, p.pow2_split != 0)) return cudaErrorNotSupported;
+        if (!linear_umma_plan(p.M, p.N, p.K, q, false, p.pow2_split != 0, p.one_wave != 0)) return cudaErrorNotSupported;
         return linear_umma_launch(q, X, codes, scales, Y, y_dtype, nullptr, 0, stream, fused);
     }
     if (ws) {

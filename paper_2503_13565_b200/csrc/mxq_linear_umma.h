@@ -53,6 +53,7 @@ struct UmmaPlan {
     int bring;       // ... and fetched stage by stage into the ring slots instead of whole K ranges
     long cost;       // the layout heuristic's figure for the chosen decomposition (comparable within a regime)
     int pow2_split;  // in: only cluster sizes 1, 2, 4, 8 (the gate / up epilogue pairs rows inside a warp)
+    int one_wave;    // in: no layout of more CTAs than are resident at once
     int layer_tiles; // most tiles for the one-tile-per-CTA regime (0: one per SM); set by umma_layout
     uint32_t smem_bytes;
     int64_t N, K;
@@ -206,6 +207,33 @@ inline bool umma_layout(UmmaPlan &p, int sms, int force_split, int force_ring, i
         l.layer_tiles = 2 * sms;
         if (umma_layout_one(l, sms, force_split, force_ring, 0, true) && l.tiles_max == 1 && l.ring >= 3 && l.cost < 100000) {
             p = l;
+            return true;
+        }
+    }
+    // From 6 token rows on (32 or 48 operand columns), any number of tiles: one tile and all of K per CTA, the operand
+    // through the ring, the deepest ring with which two CTAs fit on an SM, as many waves as it takes.  One fat CTA per SM
+    // leaves the weight stream idle while its tensor core works (the block-scaled FP8 MMA at N = 32 takes 34 ns, four per
+    // stage); with two CTAs per SM one streams while the other multiplies.  128256 x 4096: 70.0 -> 64.1 us at M = 8,
+    // 75.3 -> 68.0 us at M = 16; 64000 x 4096: 37.3 -> 34.6 and 43.6 -> 36.8 us.  (At M = 4 the fat CTAs win: 59.9 against
+    // 63.4 us; a ring that leaves room for one CTA per SM only: 88 us.)
+    if (p.nb >= 32 && force_bring != 0 && force_tiles <= 0 && force_split <= 0 && !(p.one_wave && p.tiles > 2 * sms)) {
+        const int chunk = p.ks, tm = umma_tmem_cols(p.nb, 1);
+        int ring = chunk < kUmmaMaxUnitsResident ? chunk : kUmmaMaxUnitsResident;
+        if (ring > 8) ring = 8;
+        while (ring > 1 && umma_ctas_per_sm(umma_smem_bytes(p.nb, p.M, 1, chunk, ring, 1, 1), tm) < 2) --ring;
+        if (force_ring > 0 && force_ring < ring) ring = force_ring;
+        const uint32_t bytes = umma_smem_bytes(p.nb, p.M, 1, chunk, ring, 1, 1);
+        if (ring >= 3 && bytes <= kUmmaSmemLimit && umma_ctas_per_sm(bytes, tm) >= 2) {
+            p.split = 1;
+            p.groups = p.tiles;
+            p.tiles_max = 1;
+            p.ring = ring;
+            p.chunk_max = chunk;
+            p.grid = p.tiles;
+            p.bring = 1;
+            p.cost = (long)((p.tiles + 2L * sms - 1) / (2L * sms)) * chunk;
+            p.smem_bytes = bytes;
+            p.tmem_cols = tm;
             return true;
         }
     }

@@ -233,8 +233,9 @@ int mxq_linear_bf16(const void *X_bf16, int M, const void *W_bf16, int64_t N, in
  *   workspace  device memory, >= mxq_lm_head_accept_workspace_bytes, 16-byte aligned; zero its first 4096 bytes once
  *              before the first use; every call leaves them zero again.  One per stream.
  * Argmax rules as in mxq_greedy_accept (lowest index among equal maxima, NaN and -inf never selected), applied to the
- * FP32 sums mxq_linear would have stored.  Where no tcgen05 kernel covers the call (K % 128 != 0, no tensor maps) the
- * logits pass through the workspace and the ordinary kernels run. */
+ * FP32 sums mxq_linear would have stored.  Where no tcgen05 kernel covers the call (K % 128 != 0, no tensor maps), and
+ * for 11 or more rows on the largest vocabularies (where that is faster), the logits pass through the workspace: the
+ * plain layer, one launch for the argmax of every row, one for the walk over the draft. */
 size_t mxq_lm_head_accept_workspace_bytes(int R, int64_t V, int64_t K);
 int mxq_lm_head_accept(const void *X_bf16, int R, const uint8_t *codes, const uint8_t *scales, int64_t V, int64_t K,
                        const int32_t *draft, int T, int32_t *verifier, int32_t *accept_len, int32_t *next_token,

@@ -297,13 +297,22 @@ int mxq_linear(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *s
 static constexpr size_t kFusedHeader = 4096;
 static size_t align256(size_t v) { return (v + 255u) & ~(size_t)255u; }
 
+// Whether the call runs as the plain layer + mxq_greedy_accept, the logits passing through the workspace: where no
+// tcgen05 kernel covers it, and for the widest token operand (11 or more rows) on matrices of more than two tiles per SM,
+// where the plain layer's waves of small CTAs beat the fused kernel's one-wave layout by more than the second pass over
+// the logits costs (128256 x 4096 at R = 16: 69 + 15 us against 92 us; 64000 x 4096: 38 + 12 against 60 us).
+static bool lm_head_unfused(const mxq::Choice &c, int R, int64_t V) {
+    if (c.kernel != MXQ_KERNEL_FP4 && c.kernel != MXQ_KERNEL_UMMA) return true;
+    return c.kernel == MXQ_KERNEL_UMMA && R >= 11 && (V + 127) / 128 > 2 * (int64_t)mxq::sm_count();
+}
+
 size_t mxq_lm_head_accept_workspace_bytes(int R, int64_t V, int64_t K) {
     if (R < 1 || R > MXQ_MAX_M || !mxq::shape_ok(V, K)) return 0;
     mxq::Choice c;
     mxq::choose(mxq::kernel_ceiling(), R, V, K, nullptr, true, c, false, true);
     size_t b = kFusedHeader + align256(mxq_linear_workspace_bytes(R, V, K));
-    if (c.kernel != MXQ_KERNEL_FP4 && c.kernel != MXQ_KERNEL_UMMA)
-        b += align256((size_t)R * (size_t)V * 4u) + align256(mxq_accept_workspace_bytes(1, R, V));
+    if (lm_head_unfused(c, R, V))
+        b += align256((size_t)R * (size_t)V * 4u) + align256(mxq_accept_workspace_bytes(R, 1, V));
     return b;
 }
 
@@ -320,7 +329,7 @@ int mxq_lm_head_accept(const void *X_bf16, int R, const uint8_t *codes, const ui
     const size_t lin_ws_bytes = align256(mxq_linear_workspace_bytes(R, V, K));
     mxq::Choice c;
     mxq::choose(mxq::kernel_ceiling(), R, V, K, codes, true, c, false, true);
-    if (c.kernel == MXQ_KERNEL_FP4 || c.kernel == MXQ_KERNEL_UMMA) {
+    if (!lm_head_unfused(c, R, V)) {
         mxq::FusedAccept fa{};
         fa.keys = reinterpret_cast<unsigned long long *>(ws);
         fa.ticket = reinterpret_cast<unsigned int *>(ws + 2048);
@@ -338,21 +347,31 @@ int mxq_lm_head_accept(const void *X_bf16, int R, const uint8_t *codes, const ui
         }
         return mxq::launch_status();
     }
-    // no tcgen05 kernel covers the call: the logits pass through the workspace
+    // The plain layer with the logits in the workspace, then the argmax of every row in ONE launch (R "sequences" of one
+    // row each, whose draft token -1 never matches: G = 0 and the row's argmax comes back as the next token), then the
+    // walk over the draft on the R tokens.
     float *logits = reinterpret_cast<float *>(ws + kFusedHeader + lin_ws_bytes);
     void *acc_ws = ws + kFusedHeader + lin_ws_bytes + align256((size_t)R * (size_t)V * 4u);
-    const size_t acc_ws_bytes = align256(mxq_accept_workspace_bytes(1, R, V));
-    int32_t *minus_one = reinterpret_cast<int32_t *>(ws + 2176);
-    if (cudaMemsetAsync(minus_one, 0xFF, 4, st) != cudaSuccess) return MXQ_ERR_CUDA;
+    const size_t acc_ws_bytes = align256(mxq_accept_workspace_bytes(R, 1, V));
+    // (a `codes` that is not 32-byte aligned takes this path although the size query, which cannot know, may have
+    // answered for the fused one)
+    if (workspace_bytes < kFusedHeader + lin_ws_bytes + align256((size_t)R * (size_t)V * 4u) + acc_ws_bytes) return MXQ_ERR_WORKSPACE;
+    int32_t *minus_one = reinterpret_cast<int32_t *>(ws + 2176);   // [16]; the header's keys and ticket end at 2052
+    int32_t *zeros_out = reinterpret_cast<int32_t *>(ws + 2304);   // [16] accept lengths of the argmax pass (all 0)
+    int32_t *tok = verifier ? verifier : reinterpret_cast<int32_t *>(ws + 2432);
+    if (cudaMemsetAsync(minus_one, 0xFF, 64, st) != cudaSuccess || cudaMemsetAsync(acc_ws, 0, acc_ws_bytes, st) != cudaSuccess)
+        return MXQ_ERR_CUDA;
     int rc = mxq_linear(X_bf16, R, codes, scales, V, K, logits, MXQ_F32, lin_ws, lin_ws_bytes, stream);
     if (rc != MXQ_OK) return rc;
-    if (verifier)   // a draft token of -1 never matches: the call returns G = 0 and the row's argmax
-        for (int r = 0; r < R; ++r) {
-            rc = mxq_greedy_accept(logits + (size_t)r * V, MXQ_F32, 1, 1, V, minus_one, 1, accept_len, verifier + r, acc_ws, acc_ws_bytes, stream);
-            if (rc != MXQ_OK) return rc;
-        }
-    if (T == 0) return mxq_greedy_accept(logits, MXQ_F32, 1, 1, V, minus_one, 1, accept_len, next_token, acc_ws, acc_ws_bytes, stream);
-    return mxq_greedy_accept(logits, MXQ_F32, 1, R, V, draft, T, accept_len, next_token, acc_ws, acc_ws_bytes, stream);
+    rc = mxq_greedy_accept(logits, MXQ_F32, R, 1, V, minus_one, 1, zeros_out, tok, acc_ws, acc_ws_bytes, stream);
+    if (rc != MXQ_OK) return rc;
+    if (T == 0) {   // the plain draft step: no token to verify, the argmax is the next token
+        if (cudaMemsetAsync(accept_len, 0, 4, st) != cudaSuccess ||
+            cudaMemcpyAsync(next_token, tok, 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+            return MXQ_ERR_CUDA;
+        return MXQ_OK;
+    }
+    return mxq_greedy_accept_tokens(draft, tok, 1, T, R, accept_len, next_token, stream);
 }
 
 // ---- layer epilogues: residual add, gate / up pairing -------------------------------------------------------------------

@@ -119,6 +119,22 @@ enum mxq_kernel {
  * MXQ_LINEAR_VARIANT (fp4 | umma | mma | generic), else MXQ_KERNEL_AUTO. */
 int mxq_set_linear_kernel(int kernel);
 
+/* Forces one layout parameter of the tcgen05 kernels where it is feasible (tests and comparisons; the heuristics
+ * are the product).  `what`: one of mxq_layout_knob; `value` 0 restores the heuristic (-1 for
+ * MXQ_LAYOUT_OPERAND_THROUGH_RING).  Host-side, process-wide, not synchronised with calls running on other host
+ * threads (the same holds for mxq_set_pdl and mxq_set_linear_kernel, and for the per-device caches behind the
+ * launches: configure from one thread, or before the worker threads start). */
+enum mxq_layout_knob {
+    MXQ_LAYOUT_SPLIT = 0,                /* CTAs per cluster (K split) of MXQ_KERNEL_FP4 / MXQ_KERNEL_UMMA              */
+    MXQ_LAYOUT_RING = 1,                 /* ring slots                                                               */
+    MXQ_LAYOUT_TILES = 2,                /* 128-row tiles per CTA                                                    */
+    MXQ_LAYOUT_OPERAND_THROUGH_RING = 3, /* MXQ_KERNEL_UMMA with a workspace: 0 token operand resident, 1 through the ring */
+    MXQ_LAYOUT_PRESPLIT_MIN_M = 4,       /* MXQ_KERNEL_UMMA: token rows from which the operand is split ahead (17: never) */
+    MXQ_LAYOUT_BATCH_RING = 5,           /* mxq_linear_batch: ring slots per CTA                                      */
+    MXQ_LAYOUT_BATCH_CTAS_PER_SM = 6     /* mxq_linear_batch: CTAs per SM (1..2)                                      */
+};
+int mxq_set_linear_layout(int what, int value);
+
 /* How a kernel would run this shape on the current device (diagnostics; launches nothing).
  * kernel = MXQ_KERNEL_AUTO describes the one mxq_linear would pick under the current setting for a
  * suitably aligned `codes`; another value describes that kernel whether or not it would be picked.
@@ -138,7 +154,9 @@ int mxq_linear_plan_info(int kernel, int M, int64_t N, int64_t K, int32_t *info)
 /* Copies to *status_host, and then clears, the sticky device words in which the tcgen05 kernels record a
  * bounded wait that gave up (bit 0: data of a stage never arrived, bit 1: a stage was never released,
  * bit 2: the accumulator never completed, bit 3: a prefetched stage never landed; bits 0-3 for
- * MXQ_KERNEL_UMMA, bits 8-11 the same for MXQ_KERNEL_FP4, bits 16-20 for mxq_linear_bf16).  0 in normal
+ * MXQ_KERNEL_UMMA, bits 8-11 the same for MXQ_KERNEL_FP4, bits 16-20 for mxq_linear_bf16; bits 24-27 for
+ * mxq_linear_batch: data of a stage never arrived, a ring slot was never released, an accumulator never completed,
+ * the rewritten token rows never became ready).  0 in normal
  * operation; a non-zero word means the affected output tiles were written as NaN.  Synchronises with
  * the device (a blocking copy), so call it outside the hot loop. */
 int mxq_linear_device_status(uint32_t *status_host);
@@ -166,7 +184,11 @@ int mxq_linear_host(const void *X_host, int M, const uint8_t *codes, const uint8
                     int64_t K, void *Y_host, int y_dtype, void *X_stage_dev, void *Y_stage_dev,
                     void *workspace, size_t workspace_bytes, void *stream);
 
-/* Workspace (bytes) for mxq_greedy_accept; same zero-once / reusable contract as above. */
+/* Workspace (bytes) for mxq_greedy_accept.  Device memory, 16-byte aligned.  Its first 4096 bytes are ticket counters:
+ * zero them ONCE before the first call (cudaMemset); every call that completes leaves them zero again, so the same
+ * workspace can be reused by later calls of any shape it is large enough for.  With counters that are not zero the
+ * kernel never finds its last CTA and accept_len / next_token are not written, although the call returns MXQ_OK.  The
+ * rest needs no initialisation.  Calls that may run concurrently (different streams) need a workspace each. */
 size_t mxq_accept_workspace_bytes(int64_t B, int R, int64_t V);
 
 /* Greedy verification of speculated tokens (Sec. III-A: tokens after the first
@@ -259,6 +281,57 @@ int mxq_linear_residual(const void *X_bf16, int M, const uint8_t *codes, const u
                         const void *residual, void *Y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream);
 int mxq_linear_swiglu(const void *X_bf16, int M, const uint8_t *codes, const uint8_t *scales, int64_t N, int64_t K,
                       void *Y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Several layers in ONE launch (Sec. III-B: a draft step is bound by the stream of its weights; Sec. III-D-2: the
+ * operators of a layer fused around its linear layers).  A decoder layer is seven small matrices, and a kernel launch
+ * per matrix costs more than its 1.4-3.7 us of weight traffic; here one persistent grid (one CTA per SM) walks all
+ * the layers of the call with one uninterrupted stream of weights, the token rows of every distinct X are rewritten as
+ * tensor-core operands once, and tiles that fall into two CTAs' shares are summed in a fixed order.
+ *   descs   HOST array of `count` (1..MXQ_MAX_BATCH) descriptors, read during the call only.  Per layer:
+ *             X_bf16 [M][K], codes / scales the MXFP4 pair of W[N][K], Y and y_dtype as in mxq_linear;
+ *             epilogue MXQ_EPI_NONE      Y [M][N]   = X . w^T
+ *                      MXQ_EPI_RESIDUAL  Y [M][N]   = residual + X . w^T   (residual [M][N] in Y's type; may be Y itself)
+ *                      MXQ_EPI_SWIGLU    Y [M][N/2] = silu(g) * u, rows 2i / 2i+1 of W being gate / up row i
+ *           The layers of one call are INDEPENDENT: none may read (as X or residual) what another one writes, since
+ *           they run interleaved.  Layers that share an X pointer share its rewriting.  X, Y and residual may also be
+ *           page-locked host memory that the GPU can address (cudaHostAlloc / cudaHostRegister): the kernel then reads
+ *           the activations and writes the results across the bus itself.
+ *   M       token rows, common to all layers of the call
+ *   workspace  REQUIRED: device memory, 256-byte aligned, >= mxq_linear_batch_workspace_bytes(descs, count, M).  Zero
+ *           its first 8192 bytes (counters) ONCE before the first use; every call that completes leaves them zero
+ *           again; the rest needs no initialisation.  After a non-zero mxq_linear_device_status zero them again.  Calls
+ *           in one stream may share a workspace; calls that may run concurrently need one each.
+ * The persistent kernel covers M <= 4 with every K a multiple of 128; any other call runs its layers one after the
+ * other through mxq_linear / mxq_linear_residual / mxq_linear_swiglu (same results as those).  Results are
+ * bit-reproducible run to run and within mxq_linear's bound; the summation order differs from mxq_linear's.  Errors as
+ * mxq_linear.  Bounded waits that give up are reported in bits 24-27 of mxq_linear_device_status. */
+#define MXQ_MAX_BATCH 16
+enum mxq_epilogue { MXQ_EPI_NONE = 0, MXQ_EPI_RESIDUAL = 1, MXQ_EPI_SWIGLU = 2 };
+typedef struct mxq_linear_desc {
+    const void *X_bf16;
+    const uint8_t *codes;
+    const uint8_t *scales;
+    void *Y;
+    const void *residual; /* MXQ_EPI_RESIDUAL only, else NULL */
+    int64_t N, K;
+    int32_t y_dtype;      /* MXQ_F32 / MXQ_BF16 */
+    int32_t epilogue;     /* mxq_epilogue */
+} mxq_linear_desc;
+size_t mxq_linear_batch_workspace_bytes(const mxq_linear_desc *descs, int count, int M);
+int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *workspace, size_t workspace_bytes,
+                     void *stream);
+
+/* How mxq_linear_batch would run the call on the current device (diagnostics; launches nothing).  info[8] int32:
+ * [0] 1 if the persistent kernel covers the call, 0 if the layers would run one by one; [1] CTAs; [2] ring slots per
+ * CTA; [3] dynamic shared memory bytes; [4] columns of the token operand; [5] units of work (128 rows x 256 k);
+ * [6] tensor-memory columns per CTA. */
+int mxq_linear_batch_info(const mxq_linear_desc *descs, int count, int M, int32_t *info);
+
+/* Test hook for the bounded waits of mxq_linear_batch: the NEXT call of mxq_linear_batch (one-shot) leaves out the weight
+ * copy of unit `unit` of its work sequence and limits every wait inside the kernel to `wait_us` microseconds.  The
+ * CTA that owns the unit then gives up: the call still completes, mxq_linear_device_status reports bit 24 and the
+ * tiles that CTA had not finished are NaN.  unit = -1, wait_us = 0 cancels. */
+int mxq_debug_batch_fault(int unit, unsigned wait_us);
 
 #ifdef __cplusplus
 }

@@ -86,6 +86,16 @@ def lib() -> ctypes.CDLL:
             L.mxq_lm_head_accept_workspace_bytes.argtypes = [i32, i64, i64]
             L.mxq_lm_head_accept.restype = i32
             L.mxq_lm_head_accept.argtypes = [vp, i32, vp, vp, i64, i64, vp, i32, vp, vp, vp, vp, sz, vp]
+            L.mxq_set_linear_layout.restype = i32
+            L.mxq_set_linear_layout.argtypes = [i32, i32]
+            L.mxq_linear_batch_workspace_bytes.restype = sz
+            L.mxq_linear_batch_workspace_bytes.argtypes = [vp, i32, i32]
+            L.mxq_linear_batch.restype = i32
+            L.mxq_linear_batch.argtypes = [vp, i32, i32, vp, sz, vp]
+            L.mxq_linear_batch_info.restype = i32
+            L.mxq_linear_batch_info.argtypes = [vp, i32, i32, vp]
+            L.mxq_debug_batch_fault.restype = i32
+            L.mxq_debug_batch_fault.argtypes = [i32, ctypes.c_uint]
             _lib = L
     return _lib
 
@@ -394,3 +404,93 @@ def interleave_gate_up(gate: torch.Tensor, up: torch.Tensor) -> torch.Tensor:
     mxq_linear_swiglu expects: row 2i = gate[i], row 2i+1 = up[i].  A copy, no arithmetic."""
     assert gate.shape == up.shape and gate.dtype == up.dtype
     return torch.stack((gate, up), dim=1).reshape(2 * gate.shape[0], gate.shape[1]).contiguous()
+
+
+# ---- several layers in one launch -------------------------------------------------------------
+
+LAYOUT_KNOBS = {"split": 0, "ring": 1, "tiles": 2, "operand_through_ring": 3, "presplit_min_m": 4, "batch_ring": 5,
+                "batch_ctas_per_sm": 6}
+EPILOGUES = {"none": 0, "residual": 1, "swiglu": 2}
+MAX_BATCH = 16
+
+
+def mxq_set_linear_layout(what, value: int) -> None:
+    """Force one layout parameter of the tcgen05 kernels (tests, comparisons); see mxq_layout_knob in mxq.h."""
+    code = LAYOUT_KNOBS[what] if isinstance(what, str) else int(what)
+    _check(lib().mxq_set_linear_layout(code, int(value)), "mxq_set_linear_layout")
+
+
+class _LinearDesc(ctypes.Structure):
+    _fields_ = [("X_bf16", ctypes.c_void_p), ("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p),
+                ("Y", ctypes.c_void_p), ("residual", ctypes.c_void_p), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("y_dtype", ctypes.c_int32), ("epilogue", ctypes.c_int32)]
+
+
+def _any_mem(t: torch.Tensor, dtype, what: str) -> int:
+    """Device tensor, or a page-locked host tensor the GPU can address."""
+    if not ((t.is_cuda or t.is_pinned()) and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError("%s must be a contiguous CUDA (or pinned host) tensor of dtype %s" % (what, dtype))
+    return t.data_ptr()
+
+
+class LinearBatch:
+    """The descriptor array of one mxq_linear_batch call, marshalled once and reusable (the call itself is then a
+    single C call).  ``layers``: dicts with x [M,K] BF16, codes, scales, out [M,N] (or [M,N/2] for "swiglu"), and
+    optionally epilogue ("none" | "residual" | "swiglu") and residual.  The tensors are kept alive by this object."""
+
+    def __init__(self, layers):
+        if not 1 <= len(layers) <= MAX_BATCH:
+            raise ValueError("1..%d layers per call" % MAX_BATCH)
+        self.m = int(layers[0]["x"].shape[0])
+        self.count = len(layers)
+        self.array = (_LinearDesc * self.count)()
+        self.keep = []
+        self.device = layers[0]["codes"].device
+        for d, lay in zip(self.array, layers):
+            x, codes, scales, out = lay["x"], lay["codes"], lay["scales"], lay["out"]
+            epi = EPILOGUES[lay.get("epilogue", "none")]
+            res = lay.get("residual")
+            m, k = x.shape
+            n = codes.shape[0]
+            if m != self.m or codes.shape[1] * 2 != k or tuple(scales.shape) != (n, k // 32):
+                raise ValueError("shape mismatch between X, codes and scales")
+            if tuple(out.shape) != (m, n // 2 if epi == 2 else n):
+                raise ValueError("out has the wrong shape")
+            d.X_bf16 = _any_mem(x, torch.bfloat16, "x")
+            d.codes = _dev(codes, torch.uint8, "codes")
+            d.scales = _dev(scales, torch.uint8, "scales")
+            d.Y = _any_mem(out, out.dtype, "out")
+            d.residual = _any_mem(res, out.dtype, "residual") if res is not None else None
+            d.N, d.K = n, k
+            d.y_dtype = _dt(out.dtype)
+            d.epilogue = epi
+            self.keep.append((x, codes, scales, out, res))
+        self._ptr = ctypes.cast(self.array, ctypes.c_void_p)
+
+    def workspace_bytes(self) -> int:
+        return int(lib().mxq_linear_batch_workspace_bytes(self._ptr, self.count, self.m))
+
+    def info(self) -> dict:
+        info = (ctypes.c_int32 * 8)()
+        _check(lib().mxq_linear_batch_info(self._ptr, self.count, self.m, ctypes.cast(info, ctypes.c_void_p)), "mxq_linear_batch_info")
+        return dict(zip(("persistent", "grid", "ring", "smem_bytes", "nb", "units", "tmem_cols"), [int(v) for v in info]))
+
+    def run(self, workspace: torch.Tensor, stream=None) -> None:
+        _check(lib().mxq_linear_batch(self._ptr, self.count, self.m, _dev(workspace, torch.uint8, "workspace"),
+                                      workspace.numel(), _stream(stream)), "mxq_linear_batch")
+
+
+def mxq_linear_batch(layers, workspace: torch.Tensor = None, stream=None) -> LinearBatch:
+    """Several independent layers in one launch (see mxq_linear_batch in mxq.h).  Returns the marshalled batch, whose
+    ``run(workspace)`` repeats the call without re-marshalling.  ``workspace``: from ``new_workspace(batch.workspace_bytes())``
+    (zero-filled once; reusable by calls in one stream)."""
+    batch = layers if isinstance(layers, LinearBatch) else LinearBatch(layers)
+    if workspace is None:
+        workspace = new_workspace(batch.workspace_bytes(), batch.device)
+    batch.run(workspace, stream)
+    return batch
+
+
+def mxq_debug_batch_fault(unit: int, wait_us: int) -> None:
+    """Test hook: the next mxq_linear_batch call leaves out one weight copy and bounds its waits (see mxq.h)."""
+    _check(lib().mxq_debug_batch_fault(int(unit), int(wait_us)), "mxq_debug_batch_fault")

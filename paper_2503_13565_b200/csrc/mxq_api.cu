@@ -8,6 +8,19 @@ namespace mxq {
 static std::atomic<int> g_pdl{1};
 bool pdl_enabled() { return g_pdl.load(std::memory_order_relaxed) != 0; }
 
+static std::atomic<int> g_layout[7] = {{0}, {0}, {0}, {-1}, {0}, {0}, {0}};
+LayoutOverride layout_override() {
+    LayoutOverride o;
+    o.split = g_layout[0].load(std::memory_order_relaxed);
+    o.ring = g_layout[1].load(std::memory_order_relaxed);
+    o.tiles = g_layout[2].load(std::memory_order_relaxed);
+    o.operand_through_ring = g_layout[3].load(std::memory_order_relaxed);
+    o.presplit_min_m = g_layout[4].load(std::memory_order_relaxed);
+    o.batch_ring = g_layout[5].load(std::memory_order_relaxed);
+    o.batch_ctas_per_sm = g_layout[6].load(std::memory_order_relaxed);
+    return o;
+}
+
 int sm_count() {
     static int cached[64];
     int dev = 0;
@@ -41,6 +54,12 @@ const char *mxq_status_string(int status) {
 }
 
 int mxq_set_pdl(int enabled) { return mxq::g_pdl.exchange(enabled ? 1 : 0); }
+
+int mxq_set_linear_layout(int what, int value) {
+    if (what < 0 || what >= 7) return MXQ_ERR_SHAPE;
+    mxq::g_layout[what].store(value, std::memory_order_relaxed);
+    return MXQ_OK;
+}
 
 size_t mxq_codes_bytes(int64_t N, int64_t K) { return mxq::shape_ok(N, K) ? (size_t)N * (size_t)K / 2 : 0; }
 size_t mxq_scales_bytes(int64_t N, int64_t K) { return mxq::shape_ok(N, K) ? (size_t)N * (size_t)K / 32 : 0; }

@@ -16,6 +16,16 @@ int sm_count();
 // whether mxq_linear launches carry the programmatic-dependent-launch attribute
 bool pdl_enabled();
 
+// mxq_set_linear_layout: layout parameters of the tcgen05 kernels forced by a test or a comparison (0 / -1 = the
+// heuristic decides); see include/mxq.h
+struct LayoutOverride {
+    int split, ring, tiles;      // > 0: CTAs per cluster, ring slots, tiles per CTA (where feasible)
+    int operand_through_ring;    // FP8-operand kernel with a workspace: 0 = token operand resident, 1 = through the ring, -1 = heuristic
+    int presplit_min_m;          // FP8-operand kernel: token rows from which the operand is split ahead of the weight kernel (> 16: never)
+    int batch_ring, batch_ctas_per_sm;   // mxq_linear_batch: ring slots per CTA, CTAs per SM
+};
+LayoutOverride layout_override();
+
 // Vocabulary projection fused with the greedy verification (Sec. III-A, III-B).  With `keys` set a tcgen05 kernel
 // does not store Y: every finished logit (token row m, vocabulary index n) competes for keys[m], the last CTA to
 // deliver turns the keys into the verifier's tokens, walks the draft and leaves keys and ticket zero for the next call.
@@ -64,6 +74,7 @@ bool linear_fp4_plan(int M, int64_t N, int64_t K, Fp4Plan &plan, bool pow2_split
 cudaError_t linear_fp4_launch(const Fp4Plan &plan, const void *X, const uint8_t *codes, const uint8_t *scales,
                               void *Y, int y_dtype, cudaStream_t stream, const FusedAccept *fused = nullptr);
 int linear_fp4_take_status(uint32_t *out);
+int linear_batch_take_status(uint32_t *out);  // the persistent multi-layer kernel (mxq_linear_batch.cu)
 int linear_bf16_take_status(uint32_t *out);   // the BF16-weight comparison kernel (mxq_linear_bf16.cu)
 
 }  // namespace mxq

@@ -451,9 +451,12 @@ static void *device_view_of_host(const void *p) {
 int mxq_linear_host(const void *X_host, int M, const uint8_t *codes, const uint8_t *scales, int64_t N,
                     int64_t K, void *Y_host, int y_dtype, void *X_stage_dev, void *Y_stage_dev,
                     void *workspace, size_t workspace_bytes, void *stream) {
-    if (!X_host || !Y_host || !X_stage_dev || !Y_stage_dev) return MXQ_ERR_NULL;
+    if (!X_host || !Y_host || !X_stage_dev || !Y_stage_dev || !codes || !scales) return MXQ_ERR_NULL;
     if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return MXQ_ERR_SHAPE;
     if (y_dtype != MXQ_F32 && y_dtype != MXQ_BF16) return MXQ_ERR_DTYPE;
+    // everything mxq_linear would refuse is refused here, before the staging copy of X is enqueued
+    if (!mxq::aligned16(codes) || !mxq::aligned16(scales) || !mxq::aligned16(X_stage_dev) || !mxq::aligned16(Y_stage_dev))
+        return MXQ_ERR_ALIGN;
     cudaStream_t st = (cudaStream_t)stream;
     // Page-locked host buffers that the GPU can address are moved by the GPU itself: a one-wave kernel pulls X across
     // the bus into the staging buffer (the copy engine's start-up costs several times the transfer of 8-350 KB), and the

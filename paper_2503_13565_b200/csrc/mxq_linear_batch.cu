@@ -1,0 +1,923 @@
+// mxq_linear_batch: the MXFP4 layers of one decoding step (Sec. III-D-3, Eq. 2; Sec. III-B: a draft step is the stream
+// of its weights) in ONE persistent launch, for 1..4 token rows.
+//
+// A decoder layer is seven small matrices; launched one by one, each call pays a dependent chain of several
+// microseconds (launch, activations arrive, rewrite them as tensor-core operands, sum over the cluster, store) against
+// 1.4-3.7 us of weight traffic.  Here one grid of one CTA per SM walks all the layers of the call:
+//   - The call's work is the sequence of units (layer, 128-row tile, 256-k stage), tile-major, cut into as many
+//     contiguous ranges as there are CTAs.  A CTA streams whole weight rows for most of its range, and its TMA ring
+//     runs on across tile and layer boundaries, so the weight stream never drains inside a call.
+//   - The token rows are rewritten ONCE per distinct X (16 radix-4 digit planes per row, see mxq_fp4_split.cuh) by
+//     all CTAs together into an image in the workspace, at the start of the kernel and while the first weights are
+//     already in flight; every unit then fetches its 256 k of the image with one bulk copy beside its weights.
+//   - A tile whose stages fall into two or three CTAs' ranges is finished by whichever of them delivers last: each
+//     writes its partial sums to the workspace and takes a ticket; the last one adds the parts in range order (so the
+//     result does not depend on who was last) and stores.
+//   - Accumulators alternate between several tensor-memory slots, so the MMAs of the next tile start while the
+//     epilogue warps read the previous one.
+// Warp roles (320 threads): warp 0 issues the MMAs and owns tensor memory; warp 1 is the producer (TMA copies of the
+// codes, bulk copies of the token operand); warps 2..5 first rewrite their share of the token rows and then run the
+// epilogues; warps 6..9 move the scale bytes (thread r those of weight row r) into the slots' scale atoms.  Every wait is bounded; one that gives up sets a sticky status bit and the
+// CTA's remaining tiles are written as NaN.
+#include <atomic>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+
+#include "mxq_fp4_split.cuh"
+#include "mxq_host.h"
+#include "mxq_linear_batch.h"
+#include "mxq_tcgen05.cuh"
+#include "mxq_tensor_map.h"
+
+namespace mxq {
+
+namespace {
+
+// sticky: bit 0 a stage's data never arrived, 1 a ring slot was never released, 2 an accumulator never completed or was
+// never released, 3 the token operand never became ready
+__device__ unsigned int g_batch_status = 0;
+
+constexpr uint32_t kFullArrivals = 1 + 4;   // the producer's arrive (with the bytes it announces) + one arrive per scale warp
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint4 ld_cg_u4(const void *p) {   // through L2 only: another SM may have written it during this kernel
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ float ld_cg_f32(const float *p) {
+    float v;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// Bounded wait on an mbarrier that also ends when the CTA's failure flag is raised.  False: gave up.  The probes are
+// back to back (the instruction itself suspends the warp for a while when the phase is not complete): a sleep between
+// probes costs far more than its nominal duration and put a floor of most of a microsecond under every wait.
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *fail, uint32_t limit_us) {
+    for (int i = 0; i < 1024; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (;;) {
+        for (int i = 0; i < 1024; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*fail || global_ns() - t0 > (uint64_t)limit_us * 1000ull) return false;
+    }
+}
+// The same for a whole (converged) warp with ONE lane probing: threads that probe an mbarrier occupy the SM's
+// shared-memory pipeline while they wait, and with all the waiting warps of a CTA probing (some 160 threads) every
+// barrier operation of the CTA queued behind them: a unit of work took 0.9 us whatever it contained.
+__device__ __forceinline__ bool warp_wait_bar(uint32_t bar, uint32_t parity, volatile int *fail, uint32_t limit_us, int lane) {
+    int ok = 1;
+    if (lane == 0) ok = wait_bar(bar, parity, fail, limit_us) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+// Bounded wait until a counter in global memory reaches `want`.
+__device__ __forceinline__ bool wait_counter(const uint32_t *ctr, uint32_t want, volatile int *fail, uint32_t limit_us) {
+    for (int i = 0; i < 256; ++i)
+        if (ld_acquire_u32(ctr) >= want) return true;
+    const uint64_t t0 = global_ns();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (ld_acquire_u32(ctr) >= want) return true;
+        if (*fail || global_ns() - t0 > (uint64_t)limit_us * 1000ull) return false;
+    }
+}
+
+// position in the call's unit sequence
+struct Cursor {
+    int d, t, s, ks, tiles;
+};
+__device__ __forceinline__ void cursor_at(const BatchTable &tb, int u, Cursor &c) {
+    int d = 0;
+    while (d + 1 < tb.ndesc && u >= tb.desc[d + 1].unit_base) ++d;
+    c.d = d;
+    c.ks = tb.desc[d].ks;
+    c.tiles = tb.desc[d].tiles;
+    const int r = u - tb.desc[d].unit_base;
+    c.t = r / c.ks;
+    c.s = r - c.t * c.ks;
+}
+__device__ __forceinline__ void cursor_next(const BatchTable &tb, Cursor &c) {
+    if (++c.s == c.ks) {
+        c.s = 0;
+        if (++c.t == c.tiles) {
+            c.t = 0;
+            if (++c.d < tb.ndesc) {
+                c.ks = tb.desc[c.d].ks;
+                c.tiles = tb.desc[c.d].tiles;
+            }
+        }
+    }
+}
+
+// The order in which a CTA walks its range [u0, u0 + nunit): if the range ends inside a tile, that last piece (`tail`
+// units, shared with the next CTA's range) comes first, then the range from its start.  Both pieces of a shared tile
+// are thus delivered early in their CTAs' runs, and the sum across CTAs is hidden behind the rest of the stream
+// instead of trailing the kernel.
+struct Walk {
+    int u0, nunit, tail;
+};
+__device__ __forceinline__ int walk_unit(const Walk &w, int i) { return i < w.tail ? w.u0 + w.nunit - w.tail + i : w.u0 + i - w.tail; }
+__device__ __forceinline__ void walk_begin(const BatchTable &tb, const Walk &w, Cursor &c) { cursor_at(tb, walk_unit(w, 0), c); }
+// from element i - 1 to element i
+__device__ __forceinline__ void walk_to(const BatchTable &tb, const Walk &w, int i, Cursor &c) {
+    if (w.tail != 0 && i == w.tail) cursor_at(tb, w.u0, c);
+    else cursor_next(tb, c);
+}
+// element i opens / closes a piece of a tile (a run of stages that share an accumulator)
+__device__ __forceinline__ bool walk_opens(const Walk &w, int i, const Cursor &c) { return i == 0 || i == w.tail || c.s == 0; }
+__device__ __forceinline__ bool walk_closes(const Walk &w, int i, const Cursor &c) { return i == w.nunit - 1 || i == w.tail - 1 || c.s == c.ks - 1; }
+
+// NB: columns of the token operand / accumulator = 16 planes x token slots (16, 32 or 64).
+template <int NB>
+__global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __grid_constant__ BatchTable tb) {
+    extern __shared__ uint8_t smem_raw[];
+    constexpr int MT = NB / 16;   // token slots
+    constexpr uint32_t kXBytes = (uint32_t)NB * 128u + kBatchSfBytes;
+    constexpr uint32_t kSlot = kBatchCodesBytes + kBatchSfBytes + kXBytes;
+    constexpr int A = NB <= 32 ? 4 : 3;   // accumulator slots (batch_acc_slots)
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = (int)gridDim.x, cta = (int)blockIdx.x;
+    const int M = tb.M, ring = tb.ring;
+    Walk wk;
+    wk.u0 = (int)((int64_t)cta * tb.units / G);
+    wk.nunit = (int)((int64_t)(cta + 1) * tb.units / G) - wk.u0;
+    {
+        Cursor last;
+        cursor_at(tb, wk.u0 + wk.nunit - 1, last);
+        wk.tail = (last.s != last.ks - 1 && last.s + 1 < wk.nunit) ? last.s + 1 : 0;
+    }
+    const int nunit = wk.nunit;
+    const uint32_t limit_us = tb.wait_us;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gbase = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t sBar = base + (uint32_t)ring * kSlot;
+    const uint32_t full0 = sBar, empty0 = sBar + (uint32_t)ring * 8u;
+    const uint32_t accf0 = sBar + (uint32_t)ring * 16u, acce0 = accf0 + 4u * 8u;
+    const uint32_t sMisc = acce0 + 4u * 8u;
+    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(gbase + (sMisc - base));
+    volatile int *s_fail = reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 4);
+    volatile int *s_flag = reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 8);
+    volatile int *s_zero = reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 12);   // always 0
+
+    uint32_t *hdr = reinterpret_cast<uint32_t *>(tb.ws);
+    uint32_t *g_ready = hdr + kBatchWordReady, *g_bad = hdr + kBatchWordBad;
+
+    // ---- set-up -------------------------------------------------------------------------------------------------------
+    if (warp == 1) {
+        for (int b = lane; b < 2 * ring + 8; b += 32) {
+            const uint32_t count = b < ring ? kFullArrivals : (b < 2 * ring ? 1u : (b < 2 * ring + 4 ? 1u : 4u));
+            mbar_init(sBar + (uint32_t)b * 8u, count);
+        }
+        if (lane == 0) {
+            *s_fail = 0;
+            *s_flag = 0;
+            *s_zero = 0;
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        __syncwarp();
+    } else if (warp == 0) {
+        pdl_trigger();   // the next kernel in the stream may start its own set-up
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sMisc), "r"(tb.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+
+    // One thread walks a CTA's units, and a lone thread issues an instruction every few cycles at best: what a role
+    // does per unit has to stay at a few dozen instructions (no divisions, nothing re-read from the parameter table
+    // that only changes with the layer).  Slot addresses, parities and descriptors are carried along incrementally.
+
+    // The first ring of weights does not depend on the previous kernel in the stream: requested before the wait.
+    const int pre = nunit < ring ? nunit : ring;
+    Cursor pc;   // producer: where the walk stands after the first `pre` requests
+    if (warp == 1) {
+        if (lane < tb.ndesc) asm volatile("prefetch.tensormap [%0];" ::"l"(&tb.maps[lane]) : "memory");
+        __syncwarp();
+        if (lane == 0) {
+            walk_begin(tb, wk, pc);
+            uint32_t dst = base, fb = full0;
+            for (int i = 0; i < pre; ++i) {
+                if (i) walk_to(tb, wk, i, pc);
+                // (test hook: the bytes of unit tb.fault_unit are announced but never requested)
+                asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(fb), "r"(kBatchCodesBytes) : "memory");
+                if (walk_unit(wk, i) != tb.fault_unit) tma_load_codes(dst, &tb.maps[pc.d], pc.s * (kBatchStageK / 2), pc.t * kBatchTileRows, fb);
+                dst += kSlot;
+                fb += 8u;
+            }
+        }
+        __syncwarp();
+        pdl_wait();   // the counters in the workspace belong to the previous call until it has completed
+    }
+    if (warp == 2) pdl_wait();   // X, Y and the workspace
+    tc_fence_before();
+    asm volatile("bar.sync 0;" ::: "memory");
+    tc_fence_after();
+    const uint32_t tmem = *tmem_holder;
+
+    if (warp == 0) {
+        // ---- MMA warp -------------------------------------------------------------------------------------------------
+        const uint32_t idesc = (1u << 7) | (1u << 10) | (((uint32_t)NB >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+        const uint32_t a_hi = (uint32_t)(smem_desc(0, 16, 1024, 2) >> 32), b_hi = (uint32_t)(smem_desc(0, 128, 1024, 0) >> 32);
+        const uint32_t s_hi = (uint32_t)(smem_desc(0, 0, 128, 0) >> 32);
+        const uint32_t t_sf0 = tmem + (uint32_t)(A * NB);   // after the accumulators: two slots of 8 + 8 scale columns
+        // descriptors of slot 0; a slot further on adds kSlot / 16 to each start-address field (the whole ring lies
+        // below 256 KB, so the 14-bit field never carries)
+        const uint32_t a_lo0 = (uint32_t)smem_desc(base, 16, 1024, 2);
+        const uint32_t sa_lo0 = (uint32_t)smem_desc(base + kBatchCodesBytes, 0, 128, 0);
+        const uint32_t b_lo0 = (uint32_t)smem_desc(base + kBatchCodesBytes + kBatchSfBytes, 128, 1024, 0);
+        const uint32_t sb_lo0 = (uint32_t)smem_desc(base + kBatchCodesBytes + kBatchSfBytes + (uint32_t)NB * 128u, 0, 128, 0);
+        Cursor c;
+        walk_begin(tb, wk, c);
+        int d_seen = -1;
+        bool half_k = false;
+        uint32_t slot = 0, phase = 0, par = 0, accumulate = 0, off16 = 0;
+        int acc_slot = -1;
+        uint32_t acc_round = 0;   // how often the accumulator slots have wrapped
+        uint32_t t_acc = tmem;
+        for (int i = 0; i < nunit; ++i) {
+            if (i) walk_to(tb, wk, i, c);
+            if (c.d != d_seen) {
+                d_seen = c.d;
+                half_k = (tb.desc[c.d].K & (kBatchStageK - 1)) != 0;
+            }
+            if (walk_opens(wk, i, c)) {   // the next accumulator slot, once the epilogue has read what it held
+                if (++acc_slot == A) {
+                    acc_slot = 0;
+                    ++acc_round;
+                }
+                if (acc_round != 0 && !warp_wait_bar(acce0 + (uint32_t)acc_slot * 8u, (acc_round - 1u) & 1u, s_fail, limit_us, lane)) {
+                    if (lane == 0) {
+                        atomicOr(&g_batch_status, 4u);
+                        *s_fail = 1;
+                    }
+                    break;
+                }
+                tc_fence_after();
+                t_acc = tmem + (uint32_t)(acc_slot * NB);
+                accumulate = 0;
+            }
+            if (!warp_wait_bar(full0 + slot * 8u, phase, s_fail, limit_us, lane)) {
+                if (lane == 0) {
+                    atomicOr(&g_batch_status, 1u);
+                    *s_fail = 1;
+                }
+                break;
+            }
+            tc_fence_after();
+            const bool half_tail = half_k && c.s == c.ks - 1;
+            const bool closes = walk_closes(wk, i, c);
+            const uint32_t t_sf = t_sf0 + par * 16u;
+            par ^= 1u;
+            if (elect_one()) {
+                const uint32_t a_lo = a_lo0 + off16, sa_lo = sa_lo0 + off16, b_lo = b_lo0 + off16, sb_lo = sb_lo0 + off16;
+                tc_copy_sf_lohi(t_sf, sa_lo, s_hi);
+                tc_copy_sf_lohi(t_sf + 4, sa_lo + 32, s_hi);
+                tc_copy_sf_lohi(t_sf + 8, sb_lo, s_hi);
+                tc_copy_sf_lohi(t_sf + 12, sb_lo + 32, s_hi);
+                auto mma = [&](int j, uint32_t acc) {   // k [64 j, 64 j + 64) of the stage: scales 2 (j & 1), + 1 of atom j >> 1
+                    const uint32_t sfid = (uint32_t)(j & 1) * 2u;
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+                        "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+                        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %5, [%7], [%8], p;\n\t}"
+                        ::"r"(t_acc), "r"(a_lo + j * 2), "r"(a_hi), "r"(b_lo + j * 16), "r"(b_hi),
+                        "r"(idesc | (sfid << 4) | (sfid << 29)), "r"(acc), "r"(t_sf + 4u * (j >> 1)), "r"(t_sf + 8u + 4u * (j >> 1))
+                        : "memory");
+                };
+                mma(0, accumulate);
+                mma(1, 1u);
+                if (!half_tail) {
+                    mma(2, 1u);
+                    mma(3, 1u);
+                }
+                tc_commit(empty0 + slot * 8u);
+                if (closes) tc_commit(accf0 + (uint32_t)acc_slot * 8u);
+            }
+            __syncwarp();
+            accumulate = 1;
+            off16 += kSlot >> 4;
+            if (++slot == (uint32_t)ring) {
+                slot = 0;
+                off16 = 0;
+                phase ^= 1u;
+            }
+        }
+        __syncwarp();
+        // tensor memory goes back once the epilogue warps have read their last accumulator
+        asm volatile("bar.sync 2, 160;" ::: "memory");
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tb.tmem_cols) : "memory");
+    } else if (warp == 1) {
+        // ---- producer warp (one lane works) ------------------------------------------------------------------------------
+        // The codes of the first ring are on their way; their share of the token operand follows as soon as the image
+        // it comes from is complete (all of a call's images are, a microsecond or two into the kernel).  After that a
+        // unit's codes and operand are requested together, as soon as the MMAs have released the slot they go to.
+        if (lane == 0) {
+            uint32_t ready_mask = 0;
+            int d_seen = -1, im = 0;
+            const CUtensorMap *map = nullptr;
+            const uint8_t *img = nullptr;
+            bool ok = true;
+            auto layer = [&](const Cursor &c) -> bool {   // the cursor has entered another layer
+                d_seen = c.d;
+                map = &tb.maps[c.d];
+                im = tb.desc[c.d].img;
+                img = tb.ws + tb.img[im].offset;
+                if (!((ready_mask >> im) & 1u)) {
+                    if (!wait_counter(g_ready + im, (uint32_t)tb.img[im].ntasks, s_fail, limit_us)) {
+                        atomicOr(&g_batch_status, 8u);
+                        *s_fail = 1;
+                        return false;
+                    }
+                    fence_proxy_async_all();   // the image was written with ordinary stores; the bulk copies read it through the async proxy
+                    ready_mask |= 1u << im;
+                }
+                return true;
+            };
+            Cursor c;
+            walk_begin(tb, wk, c);
+            uint32_t dst = base + kBatchCodesBytes + kBatchSfBytes, fb = full0;
+            int issued = 0;   // units whose operand has been requested
+            for (int i = 0; i < pre && ok; ++i) {
+                if (i) walk_to(tb, wk, i, c);
+                if (c.d != d_seen) ok = layer(c);
+                if (!ok) break;
+                mbar_expect_tx(fb, kXBytes);
+                bulk_load(dst, img + (uint32_t)c.s * kXBytes, kXBytes, fb);
+                dst += kSlot;
+                fb += 8u;
+                ++issued;
+            }
+            uint32_t slot_base = base, phase = 0;
+            fb = full0;
+            uint32_t eb = empty0;
+            const uint32_t ring_end = base + (uint32_t)ring * kSlot;
+            for (int i = pre; i < nunit && ok; ++i) {
+                walk_to(tb, wk, i, c);
+                if (c.d != d_seen) ok = layer(c);
+                if (!ok) break;
+                if (!wait_bar(eb, phase, s_fail, limit_us)) {
+                    atomicOr(&g_batch_status, 2u);
+                    *s_fail = 1;
+                    ok = false;
+                    break;
+                }
+                mbar_expect_tx(fb, kBatchCodesBytes + kXBytes);
+                if (walk_unit(wk, i) != tb.fault_unit) tma_load_codes(slot_base, map, c.s * (kBatchStageK / 2), c.t * kBatchTileRows, fb);
+                bulk_load(slot_base + kBatchCodesBytes + kBatchSfBytes, img + (uint32_t)c.s * kXBytes, kXBytes, fb);
+                ++issued;
+                slot_base += kSlot;
+                fb += 8u;
+                eb += 8u;
+                if (slot_base == ring_end) {
+                    slot_base = base;
+                    fb = full0;
+                    eb = empty0;
+                    phase ^= 1u;
+                }
+            }
+            if (!ok || *s_fail) {
+                // Copies this lane requested may still be in flight, and the CTA must not end before they have landed:
+                // the barriers of complete requests are waited for, the rest is given time.
+                for (int i = max(0, issued - ring); i < issued; ++i)
+                    (void)wait_bar(full0 + (uint32_t)(i % ring) * 8u, (uint32_t)((i / ring) & 1), s_zero, 1000u);
+                const uint64_t t0 = global_ns();
+                while (global_ns() - t0 < 100000ull) __nanosleep(1000);
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 6) {
+        // ---- scale warps: thread r brings the scale bytes of weight row r of every unit into the slot's scale atoms ------
+        // (8 bytes per row and unit, rows K / 32 bytes apart; each thread has the loads of the next four units in flight
+        // in registers)
+        const int r = tid - 192;   // 0..127
+        const uint32_t pos = (uint32_t)(r & 31) * 16u + (uint32_t)(r >> 5) * 4u;   // row r inside a 512-byte atom
+        Cursor cl;
+        walk_begin(tb, wk, cl);
+        const uint8_t *row_ptr = nullptr;   // scale bytes of this thread's row of the tile the load cursor is in (nullptr: no such row)
+        bool wide = true;                   // K % 256 == 0: a unit's 8 bytes are one aligned load
+        auto load = [&](int li) -> uint2 {
+            if (li) walk_to(tb, wk, li, cl);
+            if (walk_opens(wk, li, cl)) {
+                const BatchDesc &ds = tb.desc[cl.d];
+                const int n = cl.t * kBatchTileRows + r;
+                wide = (ds.K & (kBatchStageK - 1)) == 0;
+                row_ptr = n < ds.N ? ds.scales + (int64_t)n * (ds.K >> 5) : nullptr;
+            }
+            uint2 v = make_uint2(0u, 0u);
+            if (row_ptr) {
+                const uint8_t *src = row_ptr + cl.s * 8;
+                if (wide) {
+                    asm volatile("ld.global.nc.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(src));
+                } else {
+                    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v.x) : "l"(src));
+                    if (cl.s != cl.ks - 1) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v.y) : "l"(src + 4));
+                }
+            }
+            return v;
+        };
+        constexpr int D = 4;   // units ahead
+        uint2 v[D];
+        int li = 0;            // next element to load
+#pragma unroll
+        for (int j = 0; j < D; ++j) {
+            v[j] = make_uint2(0u, 0u);
+            if (li < nunit) {
+                v[j] = load(li);
+                ++li;
+            }
+        }
+        bool ok = true;
+        uint32_t sf = base + kBatchCodesBytes + pos, fb = full0, eb = empty0, phase = 0;
+        bool wrapped = false;
+        const uint32_t sf_end = sf + (uint32_t)ring * kSlot;
+        for (int i0 = 0; i0 < nunit && ok; i0 += D) {
+#pragma unroll
+            for (int j = 0; j < D; ++j) {
+                if (i0 + j < nunit && ok) {
+                    const uint2 cur = v[j];
+                    if (li < nunit) {
+                        v[j] = load(li);
+                        ++li;
+                    }
+                    if (wrapped) {
+                        // one thread probes for all four scale warps; barrier 3 passes the result on
+                        if (tid == 192 && !wait_bar(eb, phase, s_fail, limit_us)) {
+                            atomicOr(&g_batch_status, 2u);
+                            *s_fail = 1;
+                        }
+                        asm volatile("bar.sync 3, 128;" ::: "memory");
+                        if (*s_fail) ok = false;
+                    }
+                    if (ok) {
+                        asm volatile("st.shared.u32 [%0], %1;" ::"r"(sf), "r"(cur.x) : "memory");
+                        asm volatile("st.shared.u32 [%0], %1;" ::"r"(sf + 512u), "r"(cur.y) : "memory");
+                        fence_async_proxy();   // ordinary stores, read by tcgen05.cp
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(fb);
+                        sf += kSlot;
+                        fb += 8u;
+                        eb += 8u;
+                        if (sf == sf_end) {
+                            sf -= (uint32_t)ring * kSlot;
+                            fb = full0;
+                            eb = empty0;
+                            if (wrapped) phase ^= 1u;
+                            wrapped = true;
+                        }
+                    }
+                }
+            }
+        }
+    } else {
+        // ---- split / epilogue warps -----------------------------------------------------------------------------------
+        const int ew = warp - 2;                          // 0..3
+        const int et = tid - 64;                          // 0..127
+        const int row = ((warp & 3) << 5) + lane;         // accumulator row this thread may read (its warp's quarter)
+
+        // 1. this CTA's share of the rewriting of the token rows: task = 128 k of one token row of one image
+        for (int task = cta * 4 + ew; task < tb.tasks; task += 4 * G) {
+            int im = 0;
+            while (im + 1 < tb.nimg && task >= tb.img[im + 1].task_base) ++im;
+            const BatchImg &gi = tb.img[im];
+            const int local = task - gi.task_base;
+            const int k128 = local / M, m = local - k128 * M;
+            const int kk = k128 * 128 + (lane >> 1) * 8;
+            const uint4 raw = ld_cg_u4(reinterpret_cast<const __nv_bfloat16 *>(gi.X) + (int64_t)m * gi.K + kk);
+            uint8_t *stage = tb.ws + gi.offset + (size_t)(kk >> 8) * kXBytes;
+            const bool inexact = split_half_unit_to(raw, m, (uint32_t)kk & 255u, lane & 1, lane, SplitToGlobal{stage},
+                                                    SplitToGlobal{stage + (uint32_t)NB * 128u});
+            const bool bad = __any_sync(0xffffffffu, inexact);
+            fence_proxy_async_all();
+            __syncwarp();
+            if (lane == 0) {
+                if (bad) atomicOr(g_bad + im, 1u);
+                __threadfence();
+                atomicAdd(g_ready + im, 1u);
+            }
+        }
+
+        // 2. epilogues: one per piece of a tile in this CTA's walk, in order
+        uint32_t seen_mask = 0, bad_mask = 0;
+        float *partials = reinterpret_cast<float *>(tb.ws + tb.partials_offset);
+        uint32_t *g_ticket = hdr + kBatchWordTicket;
+        const float nanv = __uint_as_float(0x7FC00000u);
+        int seg = 0;
+        for (int i = 0; i < nunit; ++seg) {
+            Cursor c;
+            const int u = walk_unit(wk, i);
+            cursor_at(tb, u, c);
+            const BatchDesc &ds = tb.desc[c.d];
+            const int len = min(c.ks - c.s, (i < wk.tail ? wk.tail : nunit) - i);
+            const int s_begin = c.s, s_end = c.s + len;
+            const int a = seg % A;
+            i += len;
+            const bool last_seg = i >= nunit;
+            // has this layer's X been rewritten exactly?  (the counter is complete by now; waiting for it here makes the
+            // flag's value certain)
+            const int im = ds.img;
+            if (!((seen_mask >> im) & 1u)) {
+                uint32_t b = 0;
+                if (lane == 0) {
+                    if (!wait_counter(g_ready + im, (uint32_t)tb.img[im].ntasks, s_fail, limit_us)) {
+                        atomicOr(&g_batch_status, 8u);
+                        *s_fail = 1;
+                    }
+                    b = *reinterpret_cast<volatile uint32_t *>(g_bad + im);
+                }
+                b = __shfl_sync(0xffffffffu, b, 0);
+                seen_mask |= 1u << im;
+                if (b) bad_mask |= 1u << im;
+            }
+            const bool bad = (bad_mask >> im) & 1u;
+
+            float yt[MT];
+#pragma unroll
+            for (int m = 0; m < MT; ++m) yt[m] = 0.f;
+            // one thread probes for all four epilogue warps; barrier 1 passes the result on
+            if (et == 0 && !*s_fail && !wait_bar(accf0 + (uint32_t)a * 8u, (uint32_t)((seg / A) & 1), s_fail, limit_us)) {
+                atomicOr(&g_batch_status, 4u);
+                *s_fail = 1;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            const bool got = !*s_fail;
+            if (got) {
+                tc_fence_after();
+                const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(a * NB);
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    float d[16];
+                    tc_load16(t_row + m * 16, d);
+                    float acc = d[15];
+#pragma unroll
+                    for (int p = 14; p >= 0; --p) acc += d[p];
+                    yt[m] = acc;
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acce0 + (uint32_t)a * 8u);
+            }
+            if (last_seg) asm volatile("bar.arrive 2, 160;" ::: "memory");   // tensor memory may go back
+            const int n = c.t * kBatchTileRows + row;
+            if (bad && got) {
+                // Scalar path for a K range whose X cannot be rewritten exactly (the MMA results are ignored).
+                float acc[MT];
+#pragma unroll
+                for (int m = 0; m < MT; ++m) acc[m] = 0.f;
+                if (n < ds.N) {
+                    const int kb_row = ds.K >> 5;
+                    const uint4 *crow = reinterpret_cast<const uint4 *>(ds.codes + (int64_t)n * (ds.K / 2));
+                    const uint8_t *srw = ds.scales + (int64_t)n * kb_row;
+                    const __nv_bfloat16 *X = reinterpret_cast<const __nv_bfloat16 *>(ds.X);
+                    const int blk_end = min(s_end * 8, kb_row);
+                    for (int blk = s_begin * 8; blk < blk_end; ++blk) {
+                        const uint4 cc = ld_stream_u4(crow + blk);
+                        const float sc = e8m0_to_float(srw[blk]) * kGuardDown;
+                        const uint32_t w[4] = {cc.x, cc.y, cc.z, cc.w};
+                        float part[MT];
+#pragma unroll
+                        for (int m = 0; m < MT; ++m) part[m] = 0.f;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float2 wv = __half22float2(e2m1x2_to_half2((w[q] >> (8 * e)) & 0xFFu));
+                                const int64_t k = (int64_t)blk * 32 + q * 8 + e * 2;
+#pragma unroll
+                                for (int m = 0; m < MT; ++m)
+                                    if (m < M) {
+                                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * ds.K + k);
+                                        part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
+                                        part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
+                                    }
+                            }
+#pragma unroll
+                        for (int m = 0; m < MT; ++m) acc[m] = fmaf(part[m], sc, acc[m]);
+                    }
+                }
+#pragma unroll
+                for (int m = 0; m < MT; ++m) yt[m] = acc[m];
+            }
+            if (!got) {
+#pragma unroll
+                for (int m = 0; m < MT; ++m) yt[m] = nanv;
+            }
+
+            bool finish = true;   // whether this CTA stores the tile
+            if (s_begin != 0 || s_end != c.ks) {
+                // The tile is shared with the neighbouring ranges: deliver this part, and finish the tile if it was the last.
+                const int64_t ta = (int64_t)ds.unit_base + (int64_t)c.t * c.ks, tz = ta + c.ks - 1;
+                const int c_first = (int)batch_owner(ta, tb.units, G), c_last = (int)batch_owner(tz, tb.units, G);
+                const int ncontrib = c_last - c_first + 1;
+                const bool head = u == wk.u0;   // the piece that opens this CTA's range
+                float *mine = partials + ((size_t)(cta * 2 + (head ? 0 : 1)) * MT) * 128u;
+#pragma unroll
+                for (int m = 0; m < MT; ++m)
+                    if (m < M) mine[m * 128 + row] = yt[m];
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (et == 0) *s_flag = (int)atomicAdd(g_ticket + c_first, 1u);
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                finish = *s_flag == ncontrib - 1;
+                asm volatile("bar.sync 1, 128;" ::: "memory");   // (s_flag may be rewritten by the next piece)
+                if (finish) {
+                    __threadfence();
+                    float sum[MT];
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) sum[m] = 0.f;
+                    for (int j = 0; j < ncontrib; ++j) {   // range order, whoever finishes
+                        const int cj = c_first + j;
+                        const bool hj = j > 0 || batch_range_lo(cj, tb.units, G) == ta;
+                        const float *part = partials + ((size_t)(cj * 2 + (hj ? 0 : 1)) * MT) * 128u;
+#pragma unroll
+                        for (int m = 0; m < MT; ++m)
+                            if (m < M) sum[m] += ld_cg_f32(part + m * 128 + row);
+                    }
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) yt[m] = sum[m];
+                    if (et == 0) g_ticket[c_first] = 0u;   // every contributor has delivered: ready for the next call
+                }
+            }
+            if (finish) {
+                // finished sums of weight row n, one per token row: restore the guard factor, apply the layer's epilogue, store
+#pragma unroll
+                for (int m = 0; m < MT; ++m) yt[m] *= kGuardUp;
+                if (ds.epi == 2) {
+                    // gate / up rows interleaved: the partner row's sums sit in the neighbouring lane
+                    float y[MT];
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) {
+                        const float up = __shfl_xor_sync(0xffffffffu, yt[m], 1);
+                        y[m] = yt[m] / (1.f + expf(-yt[m])) * up;
+                    }
+                    if (n < ds.N && (n & 1) == 0) {
+#pragma unroll
+                        for (int m = 0; m < MT; ++m)
+                            if (m < M) store_out(ds.Y, ds.y_dtype, (int64_t)m * (ds.N >> 1) + (n >> 1), y[m]);
+                    }
+                } else if (n < ds.N) {
+#pragma unroll
+                    for (int m = 0; m < MT; ++m)
+                        if (m < M) {
+                            const int64_t at = (int64_t)m * ds.N + n;
+                            const float r = ds.epi == 1 ? load_in(ds.residual, ds.y_dtype, at) : 0.f;
+                            store_out(ds.Y, ds.y_dtype, at, yt[m] + r);
+                        }
+                }
+            }
+        }
+
+        // 3. the last CTA to get here leaves the counters zero for the next call
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (et == 0) {
+            const uint32_t old = atomicAdd(hdr + kBatchWordExit, 1u);
+            if (old == (uint32_t)G - 1u) {
+                __threadfence();
+                for (int i = 0; i < tb.nimg; ++i) {
+                    g_ready[i] = 0u;
+                    g_bad[i] = 0u;
+                }
+                hdr[kBatchWordExit] = 0u;
+            }
+        }
+    }
+}
+
+template <int NB>
+cudaError_t launch_batch(const BatchTable &tb, int grid, uint32_t smem, cudaStream_t stream) {
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(linear_batch_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBatchSmemLimit);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(linear_batch_kernel<NB>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kBatchThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, linear_batch_kernel<NB>, tb);
+}
+
+// test hook (mxq_debug_batch_fault): consumed by the next launch
+std::atomic<int> g_fault_unit{-1};
+std::atomic<unsigned> g_fault_wait_us{0};
+
+struct BatchLayout {
+    int nb, ring, grid;
+    uint32_t smem;
+};
+
+// ring slots and CTAs for `units` units of work
+bool batch_layout(int M, int64_t units, BatchLayout &L) {
+    const LayoutOverride o = layout_override();
+    L.nb = batch_nb(M);
+    const int per_sm = o.batch_ctas_per_sm >= 1 && o.batch_ctas_per_sm <= 2 ? o.batch_ctas_per_sm : 1;
+    int ring = o.batch_ring > 0 ? o.batch_ring : 64;
+    // the deepest ring that lets `per_sm` CTAs share an SM's shared memory (each CTA also takes 1 KB of system use)
+    while (ring > 1 && (batch_smem_bytes(L.nb, ring) + 1024u) * (uint32_t)per_sm > 228u * 1024u) --ring;
+    if (batch_smem_bytes(L.nb, ring) > kBatchSmemLimit) return false;
+    if (per_sm * batch_tmem_cols(L.nb) > 512) return false;
+    L.ring = ring;
+    int64_t grid = (int64_t)sm_count() * per_sm;
+    if (grid > units) grid = units;
+    if (grid > kBatchMaxGrid) grid = kBatchMaxGrid;
+    L.grid = (int)grid;
+    L.smem = batch_smem_bytes(L.nb, ring);
+    return true;
+}
+
+}  // namespace
+
+int linear_batch_take_status(uint32_t *out) {
+    unsigned int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_batch_status, sizeof v) != cudaSuccess) return MXQ_ERR_CUDA;
+    if (v != 0 && cudaMemcpyToSymbol(g_batch_status, &zero, sizeof zero) != cudaSuccess) return MXQ_ERR_CUDA;
+    *out = v;
+    return MXQ_OK;
+}
+
+// whether the persistent kernel covers the call
+static bool batch_covered(const mxq_linear_desc *descs, int count, int M) {
+    if (!linear_umma_available() || M > kBatchMaxM || count > kBatchMaxDescs) return false;
+    int64_t units = 0;
+    for (int i = 0; i < count; ++i) {
+        const mxq_linear_desc &d = descs[i];
+        if (d.K < 128 || (d.K % 128) != 0 || d.K > 0x3FFFFFFF || d.N > 0x7FFFFF00) return false;
+        units += ((d.N + 127) / 128) * ((d.K + 255) / 256);
+    }
+    return units < 0x40000000;
+}
+
+static size_t batch_workspace_bytes(const mxq_linear_desc *descs, int count, int M) {
+    const int nb = batch_nb(M);
+    size_t b = kBatchHeaderBytes + batch_partials_bytes(kBatchMaxGrid, nb);
+    for (int i = 0; i < count; ++i) b += (size_t)((descs[i].K + 255) / 256) * batch_image_stage_bytes(nb);
+    return (b + 255u) & ~(size_t)255u;
+}
+
+}  // namespace mxq
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+static int batch_validate(const mxq_linear_desc *descs, int count, int M) {
+    if (!descs) return MXQ_ERR_NULL;
+    if (count < 1 || count > MXQ_MAX_BATCH || M < 1 || M > MXQ_MAX_M) return MXQ_ERR_SHAPE;
+    for (int i = 0; i < count; ++i) {
+        const mxq_linear_desc &d = descs[i];
+        if (!d.X_bf16 || !d.codes || !d.scales || !d.Y) return MXQ_ERR_NULL;
+        if (d.epilogue < MXQ_EPI_NONE || d.epilogue > MXQ_EPI_SWIGLU) return MXQ_ERR_SHAPE;
+        if (d.epilogue == MXQ_EPI_RESIDUAL && !d.residual) return MXQ_ERR_NULL;
+        if (!mxq::shape_ok(d.N, d.K) || (d.epilogue == MXQ_EPI_SWIGLU && (d.N & 1))) return MXQ_ERR_SHAPE;
+        if (d.y_dtype != MXQ_F32 && d.y_dtype != MXQ_BF16) return MXQ_ERR_DTYPE;
+        if (!mxq::aligned16(d.X_bf16) || !mxq::aligned16(d.codes) || !mxq::aligned16(d.scales) || !mxq::aligned16(d.Y) ||
+            (d.residual && !mxq::aligned16(d.residual)))
+            return MXQ_ERR_ALIGN;
+    }
+    return MXQ_OK;
+}
+
+size_t mxq_linear_batch_workspace_bytes(const mxq_linear_desc *descs, int count, int M) {
+    if (batch_validate(descs, count, M) != MXQ_OK) return 0;
+    size_t b = mxq::kBatchHeaderBytes;
+    if (mxq::batch_covered(descs, count, M)) b = mxq::batch_workspace_bytes(descs, count, M);
+    // where the persistent kernel does not cover the call the layers run one by one and share this much scratch
+    size_t one = 0;
+    for (int i = 0; i < count; ++i) {
+        const size_t w = mxq_linear_fused_workspace_bytes(M, descs[i].N, descs[i].K);
+        if (w > one) one = w;
+    }
+    return b + ((one + 255u) & ~(size_t)255u);
+}
+
+int mxq_debug_batch_fault(int unit, unsigned wait_us) {
+    mxq::g_fault_unit.store(unit, std::memory_order_relaxed);
+    mxq::g_fault_wait_us.store(wait_us, std::memory_order_relaxed);
+    return MXQ_OK;
+}
+
+int mxq_linear_batch_info(const mxq_linear_desc *descs, int count, int M, int32_t *info) {
+    if (!info) return MXQ_ERR_NULL;
+    const int rc = batch_validate(descs, count, M);
+    if (rc != MXQ_OK) return rc;
+    for (int i = 0; i < 8; ++i) info[i] = 0;
+    if (!mxq::batch_covered(descs, count, M)) return MXQ_OK;
+    int64_t units = 0;
+    for (int i = 0; i < count; ++i) units += ((descs[i].N + 127) / 128) * ((descs[i].K + 255) / 256);
+    mxq::BatchLayout L;
+    if (!mxq::batch_layout(M, units, L)) return MXQ_OK;
+    info[0] = 1;
+    info[1] = L.grid;
+    info[2] = L.ring;
+    info[3] = (int32_t)L.smem;
+    info[4] = L.nb;
+    info[5] = (int32_t)units;
+    info[6] = mxq::batch_tmem_cols(L.nb);
+    return MXQ_OK;
+}
+
+int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *workspace, size_t workspace_bytes, void *stream) {
+    int rc = batch_validate(descs, count, M);
+    if (rc != MXQ_OK) return rc;
+    if (!workspace) return MXQ_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MXQ_ERR_ALIGN;
+    if (workspace_bytes < mxq_linear_batch_workspace_bytes(descs, count, M)) return MXQ_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    mxq::BatchLayout L;
+    int64_t units = 0;
+    for (int i = 0; i < count; ++i) units += ((descs[i].N + 127) / 128) * ((descs[i].K + 255) / 256);
+    if (!mxq::batch_covered(descs, count, M) || !mxq::batch_layout(M, units, L)) {
+        // one layer after the other through the ordinary entry points, sharing the scratch behind the header
+        uint8_t *ws = static_cast<uint8_t *>(workspace) + mxq::kBatchHeaderBytes;
+        const size_t ws_bytes = workspace_bytes - mxq::kBatchHeaderBytes;
+        for (int i = 0; i < count; ++i) {
+            const mxq_linear_desc &d = descs[i];
+            rc = d.epilogue == MXQ_EPI_RESIDUAL ? mxq_linear_residual(d.X_bf16, M, d.codes, d.scales, d.N, d.K, d.residual, d.Y, d.y_dtype, ws, ws_bytes, stream)
+                 : d.epilogue == MXQ_EPI_SWIGLU ? mxq_linear_swiglu(d.X_bf16, M, d.codes, d.scales, d.N, d.K, d.Y, d.y_dtype, ws, ws_bytes, stream)
+                                                : mxq_linear(d.X_bf16, M, d.codes, d.scales, d.N, d.K, d.Y, d.y_dtype, ws, ws_bytes, stream);
+            if (rc != MXQ_OK) return rc;
+        }
+        return MXQ_OK;
+    }
+    mxq::BatchTable tb;
+    std::memset(&tb, 0, sizeof tb);
+    const int nb = L.nb;
+    tb.ws = static_cast<uint8_t *>(workspace);
+    tb.ndesc = count;
+    tb.M = M;
+    tb.ring = L.ring;
+    tb.tmem_cols = mxq::batch_tmem_cols(nb);
+    tb.partials_offset = (uint32_t)mxq::kBatchHeaderBytes;
+    size_t img_off = mxq::kBatchHeaderBytes + mxq::batch_partials_bytes(mxq::kBatchMaxGrid, nb);
+    int unit_base = 0, task_base = 0, nimg = 0;
+    for (int i = 0; i < count; ++i) {
+        const mxq_linear_desc &d = descs[i];
+        mxq::BatchDesc &o = tb.desc[i];
+        if (!mxq::codes_tensor_map(d.codes, d.N, d.K, /*expand_fp4=*/false, &tb.maps[i])) return MXQ_ERR_CUDA;
+        o.codes = d.codes;
+        o.scales = d.scales;
+        o.X = d.X_bf16;
+        o.Y = d.Y;
+        o.residual = d.residual;
+        o.N = (int32_t)d.N;
+        o.K = (int32_t)d.K;
+        o.ks = (int32_t)((d.K + 255) / 256);
+        o.tiles = (int32_t)((d.N + 127) / 128);
+        o.unit_base = unit_base;
+        o.y_dtype = d.y_dtype;
+        o.epi = d.epilogue;
+        unit_base += o.ks * o.tiles;
+        // layers that read the same X share one image
+        int im = -1;
+        for (int j = 0; j < nimg; ++j)
+            if (tb.img[j].X == d.X_bf16 && tb.img[j].K == o.K) im = j;
+        if (im < 0) {
+            im = nimg++;
+            mxq::BatchImg &g = tb.img[im];
+            g.X = d.X_bf16;
+            g.K = o.K;
+            g.ks = o.ks;
+            g.task_base = task_base;
+            g.ntasks = M * (o.K / 128);
+            g.offset = (uint32_t)img_off;
+            task_base += g.ntasks;
+            img_off += (size_t)o.ks * mxq::batch_image_stage_bytes(nb);
+        }
+        o.img = im;
+    }
+    tb.nimg = nimg;
+    tb.units = unit_base;
+    tb.tasks = task_base;
+    tb.fault_unit = mxq::g_fault_unit.exchange(-1, std::memory_order_relaxed);
+    const unsigned w = mxq::g_fault_wait_us.exchange(0, std::memory_order_relaxed);
+    tb.wait_us = w ? w : 1000000u;
+    const cudaError_t e = nb == 16 ? mxq::launch_batch<16>(tb, L.grid, L.smem, st)
+                          : nb == 32 ? mxq::launch_batch<32>(tb, L.grid, L.smem, st)
+                                     : mxq::launch_batch<64>(tb, L.grid, L.smem, st);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MXQ_ERR_CUDA;
+    }
+    return mxq::launch_status();
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

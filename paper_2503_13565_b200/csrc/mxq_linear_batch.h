@@ -1,0 +1,92 @@
+// mxq_linear_batch: several MXFP4 layers in one persistent launch (mxq_linear_batch.cu).  Plain integers and PODs
+// only, so that the host (sizing, launch), the device code and the tests' mirror of the arithmetic agree.
+#pragma once
+#include <cuda.h>   // CUtensorMap only
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __CUDACC__
+#define MXQ_BATCH_HD __host__ __device__
+#else
+#define MXQ_BATCH_HD
+#endif
+
+namespace mxq {
+
+constexpr int kBatchMaxDescs = 16;       // layers per call (the table travels as a kernel parameter)
+constexpr int kBatchMaxM = 4;            // token rows: 16 digit planes each, 64 operand columns at most
+constexpr int kBatchThreads = 320;       // MMA warp, producer warp, four split / epilogue warps, four scale warps
+constexpr int kBatchTileRows = 128;      // weight rows per tile = M of one tcgen05.mma
+constexpr int kBatchStageK = 256;        // k per unit = 128 packed bytes per row = 8 MX blocks = 4 MMAs of K = 64
+constexpr uint32_t kBatchCodesBytes = 16384;   // 128 rows x 128 bytes
+constexpr uint32_t kBatchSfBytes = 1024;       // two 512-byte scale atoms (4 blocks each)
+constexpr uint32_t kBatchSmemLimit = 227 * 1024;
+constexpr int kBatchMaxGrid = 1024;      // CTAs (ticket counters in the workspace header)
+
+// ---- workspace ------------------------------------------------------------------------------------------------------
+// [0, kBatchHeaderBytes)  counters, all zero between calls:
+//      u32 ready[16]   split tasks delivered per token-operand image
+//      u32 bad[16]     an image holds a block that could not be rewritten exactly
+//      u32 exit        CTAs that have finished (word 32)
+//      u32 ticket[kBatchMaxGrid] at byte 256: contributors that have delivered their share of a tile split between CTAs
+// [kBatchHeaderBytes, ...) partial sums: [grid][2 (at the head / at the tail of the CTA's range)][token slots][128] floats
+// then the token-operand images, one per distinct X: [stage][operand rows NB x 128 bytes | 1024 bytes of scale atoms]
+constexpr size_t kBatchHeaderBytes = 8192;
+constexpr int kBatchWordReady = 0, kBatchWordBad = 16, kBatchWordExit = 32, kBatchWordTicket = 64;
+
+inline int batch_nb(int M) { return M == 1 ? 16 : (M == 2 ? 32 : 64); }   // operand columns: 16 planes per token slot
+inline uint32_t batch_image_stage_bytes(int nb) { return (uint32_t)nb * 128u + kBatchSfBytes; }
+inline uint32_t batch_slot_bytes(int nb) { return kBatchCodesBytes + kBatchSfBytes + batch_image_stage_bytes(nb); }
+inline size_t batch_partials_bytes(int grid, int nb) { return (size_t)grid * 2u * (size_t)(nb / 16) * 128u * 4u; }
+
+// accumulator slots in tensor memory and the columns to allocate (a power of two >= slots * nb + 32 scale columns)
+inline int batch_acc_slots(int nb) { return nb <= 32 ? 4 : 3; }
+inline int batch_tmem_cols(int nb) {
+    const int need = batch_acc_slots(nb) * nb + 32;
+    int cols = 32;
+    while (cols < need) cols *= 2;
+    return cols;
+}
+inline uint32_t batch_smem_bytes(int nb, int ring) {
+    const uint32_t b = 1024u /* alignment slack */ + (uint32_t)ring * batch_slot_bytes(nb) +
+                       (uint32_t)(2 * ring + 2 * 4) * 8u /* mbarriers */ + 64u /* tensor-memory address, flags */;
+    return (b + 15u) & ~15u;
+}
+
+// ---- partition: the call's units (layer, tile, stage), tile-major, are cut into `grid` contiguous ranges -------------
+MXQ_BATCH_HD inline int64_t batch_range_lo(int64_t cta, int64_t units, int64_t grid) { return cta * units / grid; }
+// the CTA whose range holds unit u (grid <= units, so no range is empty)
+MXQ_BATCH_HD inline int64_t batch_owner(int64_t u, int64_t units, int64_t grid) { return ((u + 1) * grid - 1) / units; }
+
+struct BatchDesc {
+    const uint8_t *codes, *scales;
+    const void *X;          // [M][K] BF16
+    void *Y;
+    const void *residual;   // epilogue 1
+    int32_t N, K;
+    int32_t ks, tiles;      // ceil(K / 256), ceil(N / 128)
+    int32_t unit_base;      // first unit of this layer in the call's sequence
+    int32_t img;            // its token-operand image
+    int32_t y_dtype, epi;   // epi: 0 store, 1 + residual, 2 silu(gate) * up over interleaved rows
+};
+struct BatchImg {
+    const void *X;
+    int32_t K, ks;
+    int32_t task_base, ntasks;   // tasks = M * K / 128 (128 k of one token row each)
+    uint32_t offset;             // bytes from the workspace base
+    uint32_t pad;
+};
+struct BatchTable {
+    CUtensorMap maps[kBatchMaxDescs];
+    BatchDesc desc[kBatchMaxDescs];
+    BatchImg img[kBatchMaxDescs];
+    uint8_t *ws;
+    int32_t ndesc, nimg, M;
+    int32_t units, tasks;
+    int32_t ring, tmem_cols;
+    int32_t fault_unit;          // test hook: the producer skips this unit's weight copy (-1: none)
+    uint32_t wait_us;            // limit of every wait inside the kernel
+    uint32_t partials_offset;    // bytes from the workspace base
+};
+
+}  // namespace mxq

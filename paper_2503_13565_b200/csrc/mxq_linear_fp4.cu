@@ -27,34 +27,12 @@
 #include <cstring>
 
 #include "mxq_host.h"
+#include "mxq_fp4_split.cuh"
 #include "mxq_linear_fp4.h"
 #include "mxq_tcgen05.cuh"
 #include "mxq_tensor_map.h"
 
 namespace mxq {
-
-// Build-time diagnostic (-DMXQ_FP4_TRACE): thread 0 of every CTA records %globaltimer at the phase boundaries of
-// the kernel, in one of three tables chosen by the shape, so that a chain of launches can be laid out on one
-// time axis afterwards (mxq_fp4_trace copies the tables to the host).  Not part of the library's interface.
-#ifdef MXQ_FP4_TRACE
-constexpr int kTraceCtas = 1024, kTracePoints = 16;
-__device__ unsigned long long g_fp4_trace[3][kTraceCtas][kTracePoints];
-// point 0 is %globaltimer (ns, common to all SMs, slow to read); the other points are SM clock cycles since point 0
-#define TR(i)                                                                                                     \
-    do {                                                                                                          \
-        if ((tid == 0 || tid == 64 || tid == 32) && blockIdx.x < kTraceCtas) {                                                              \
-            unsigned long long *row_ = g_fp4_trace[(N >> 7) % 3][blockIdx.x];            \
-            if ((i) == 0) {                                                                                       \
-                row_[0] = global_ns();                                                                            \
-                tr_c0 = clock64();                                                                                \
-            } else {                                                                                              \
-                row_[i] = (unsigned long long)(clock64() - tr_c0);                                                \
-            }                                                                                                     \
-        }                                                                                                         \
-    } while (0)
-#else
-#define TR(i)
-#endif
 
 namespace {
 
@@ -62,98 +40,12 @@ __device__ unsigned int g_fp4_status = 0;   // sticky: bit 0 full-wait, 1 empty-
 
 constexpr uint32_t kFullArrivals = 1 + 32;   // the expect_tx arrive of the TMA lane + one cp.async arrive per producer lane
 
-// Every partial sum is bounded by sum |x w^|, which cancellation can leave up to 1/2e-3 = 500 times larger than a
-// result that still has to come out finite.  So the token operand's scales carry an extra 2^-kGuard, all sums are
-// formed 2^kGuard too small, and the factor is restored once, at the final store.  (What this costs at the bottom of
-// the FP32 range is far below the layer's absolute tolerance.)
-constexpr int kGuard = 10;
-constexpr float kGuardUp = 1024.f, kGuardDown = 1.f / 1024.f;
-
-__device__ __forceinline__ void st_shared_u32(uint32_t saddr, uint32_t v) {
-    asm volatile("st.shared.u32 [%0], %1;" ::"r"(saddr), "r"(v) : "memory");
-}
-__device__ __forceinline__ void st_shared_u8(uint32_t saddr, uint32_t v) {
-    asm volatile("st.shared.u8 [%0], %1;" ::"r"(saddr), "r"(v) : "memory");
-}
-__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t mask, uint32_t c) {   // (a & mask) | c
-    uint32_t d;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(mask), "r"(c));
-    return d;
-}
-
-// in place: x[j] nibble i  <-  x[i] nibble j
-__device__ __forceinline__ void transpose_nibbles8(uint32_t (&x)[8]) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t a = x[i], b = x[i + 4];
-        x[i] = __byte_perm(a, b, 0x5410);
-        x[i + 4] = __byte_perm(a, b, 0x7632);
-    }
-#pragma unroll
-    for (int g = 0; g < 2; ++g)
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const uint32_t a = x[4 * g + i], b = x[4 * g + i + 2];
-            x[4 * g + i] = __byte_perm(a, b, 0x6240);
-            x[4 * g + i + 2] = __byte_perm(a, b, 0x7351);
-        }
-#pragma unroll
-    for (int i = 0; i < 8; i += 2) {
-        const uint32_t a = x[i], b = x[i + 1];
-        x[i] = lop3_and_or(a, 0x0F0F0F0Fu, (b & 0x0F0F0F0Fu) << 4);
-        x[i + 1] = lop3_and_or(b, 0xF0F0F0F0u, (a >> 4) & 0x0F0F0F0Fu);
-    }
-}
-
-// Half of one 8-element unit of X (token m, k offset kk inside the CTA's range): the lane with half = 0 writes digit
-// planes 0..7 into B, its neighbour with half = 1 planes 8..15; the two lanes of a 32-block's first unit also write
-// the planes' scale bytes.  Lane layout inside a warp: lane = 8 * block + 2 * unit + half; all 32 lanes call together.
-// sB_ / sSFB_ are shared-window addresses.  The E2M1 codes 0000, 0001, 0010, 0011 are the values 0, 0.5, 1, 1.5, so a
-// radix-4 digit d is its own code for d / 2; the factor 2 goes into the plane's scale.
+// Half of one 8-element unit of X (token m, k offset kk inside the CTA's range) into this CTA's operand buffers
+// (sB_ / sSFB_ are shared-window addresses): see split_half_unit_to.
 template <int NB>
 __device__ __forceinline__ bool split_half_unit(const uint4 raw, int m, int kk, int half, int lane, uint32_t sB_, uint32_t sSFB_) {
-    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-    // largest exponent field of the 32-block: both halves of a word at once, then across the block's four units
-    uint32_t e2 = (w[0] >> 7) & 0x00FF00FFu;
-#pragma unroll
-    for (int i = 1; i < 4; ++i) e2 = __vmaxu2(e2, (w[i] >> 7) & 0x00FF00FFu);
-    uint32_t emax = max(e2 & 0xFFFFu, e2 >> 16);
-    emax = max(emax, __shfl_xor_sync(0xffffffffu, emax, 2));
-    emax = max(emax, __shfl_xor_sync(0xffffffffu, emax, 4));
-    bool inexact = emax == 255u;                        // Inf or NaN in the block
-    // 32-bit fixed point under the block maximum: plane p holds bits 31-2p, 30-2p, worth digit * 2^(top - 128 - 2p)
-    const uint32_t top = max(emax, 31u + kGuard);
-    const float up = __uint_as_float((285u - top) << 23);   // 2^(158 - top), a normal number for every top in 41..254
-    const uint32_t pick = half ? 0x4140u : 0x4342u;          // bytes (b0, 0, b1, 0) of this lane's 16 bits of the fixed point
-    uint32_t pl[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const uint32_t word = w[i >> 1];
-        const uint32_t mag = (i & 1) ? (word & 0x7FFF0000u) : ((word << 16) & 0x7FFF0000u);   // |x| as FP32 bits
-        // |x| * 2^(158 - top) is the fixed-point value (bit 31 is worth 2^(top - 127)); it is below 2^32, and any
-        // fraction it has is exactly the bits that would fall off the bottom
-        const float scaled = __uint_as_float(mag) * up;
-        const uint32_t f = __float2uint_rz(scaled);
-        if (__uint2float_rn(f) != scaled) inexact = true;
-        const uint32_t sgn = (uint32_t)((int32_t)((i & 1) ? word : (word << 16)) >> 31) & 0x88888888u;
-        uint32_t v = __byte_perm(f, 0u, pick);            // 8 digits in bytes 0 and 2
-        v = (v | (v << 4)) & 0x0F0F0F0Fu;                 // 2 digits per byte
-        pl[i] = lop3_and_or(v | (v << 2), 0x33333333u, sgn);   // one digit (its own code) per nibble, nibble j = plane 8 half + 7 - j
-    }
-    transpose_nibbles8(pl);   // now pl[j] = plane 8 * half + 7 - j, nibble i = element i
     const uint32_t j = (uint32_t)kk >> 8, kin = (uint32_t)kk & 255u;
-    const uint32_t dst = sB_ + j * (NB * 128) + (uint32_t)(m * 2 + half) * 1024u + (kin >> 5) * 128u + ((kin & 31u) >> 1);
-#pragma unroll
-    for (int q = 0; q < 8; ++q) st_shared_u32(dst + (7 - q) * 16, pl[q]);   // row group 2m + half, row 7 - q
-    if ((lane & 6) == 0) {
-        const uint32_t kb = kin >> 5;
-        const uint32_t row0 = (uint32_t)(kFp4Planes * m + 8 * half);   // first of this lane's eight planes (rows of B)
-        const uint32_t sf = sSFB_ + j * kFp4SfStageBytes + (kb >> 2) * 512u + (kb & 3u) + (row0 & 31u) * 16u + (row0 >> 5) * 4u;
-        const uint32_t byte0 = top - kGuard - 16u * half;   // digit d is stored as the code of d / 2: one above 2^(top-128-2p), less the guard
-#pragma unroll
-        for (int q = 0; q < 8; ++q) st_shared_u8(sf + q * 16, byte0 - 2 * q);
-    }
-    return inexact;
+    return split_half_unit_to(raw, m, kin, half, lane, SplitToShared{sB_ + j * (NB * 128)}, SplitToShared{sSFB_ + j * kFp4SfStageBytes});
 }
 
 // NB: columns of the B operand / accumulator = 16 planes x tokens (16, 32 or 64).
@@ -174,11 +66,7 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
     FusedAccept fa = fa_arg;
     if (EPI != kEpiAccept) fa.keys = nullptr;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-#ifdef MXQ_FP4_TRACE
-    long long tr_c0 = 0;
-#endif
     if (tid == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");   // needed by the first copy, 1 us from now
-    TR(0);
     const uint32_t rank = split > 1 ? cluster_rank() : 0u;
     const uint32_t group = blockIdx.x / (uint32_t)split;
     // this CTA's tiles [tile_lo, tile_lo + ntile) and, for all of them, its K range
@@ -247,7 +135,6 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
         tma_load_codes(sA + slot * kFp4StageBytes, &tmap, (s_begin + i) * (kFp4StageK / 2), (int)n0 + t * kFp4TileRows, full0 + slot * 8);
     };
     if (warp == 1) {
-        if (tid == 32) TR(14);
         for (int b = lane; b < 2 * ring + 2 + nst; b += 32) {
             const int st = b - (2 * ring + 2);   // >= 0: the barrier of stage st's share of the activations
             const uint32_t count = b < ring ? kFullArrivals
@@ -261,10 +148,8 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
             if (fa.keys)
                 for (int q = 0; q < 16; ++q) reinterpret_cast<volatile unsigned long long *>(gbase + (sMisc - base) + 16)[q] = 0ull;
         }
-        if (tid == 32) TR(15);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         __syncwarp();
-        TR(8);
         if (lane == 0) {
             if (split > 1) mbar_expect_tx(recv_bar, (uint32_t)(ntile * split * M * row_cnt) * 4u);   // every rank sends M values per tile and row
             for (int u = 0, t = 0, i = 0; u < pre0; ++u) {
@@ -275,7 +160,6 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                 }
             }
         }
-        TR(9);
     } else if (warp == 0) {
         // let the next kernel start launching at once (its CTAs take the shared memory this kernel leaves free and start
         // their own weight stream); the MMA warp does it because it has nothing urgent to do yet
@@ -288,15 +172,12 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
     // dependent launches runs 0.2 us per launch faster with one waiting warp than with four); the others meet it at the
     // CTA-wide barrier below (initialised mbarriers, tensor-memory address).
     if (warp >= 2) {
-        TR(1);
         if (warp == 2) pdl_wait();
-        TR(2);
     }
     if (split > 1) cluster_arrive();   // "my barriers exist"; the matching wait is just before the first push to a peer
     tc_fence_before();
     asm volatile("bar.sync 0;" ::: "memory");
     tc_fence_after();
-    if (tid == 64) TR(12);
     const uint32_t tmem = *tmem_holder;
     if (warp == 1) {
         for (int u = 0, t = 0, i = 0; u < pre; ++u) {
@@ -383,7 +264,6 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
         asm volatile("bar.sync 2, 160;" ::: "memory");
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
-        TR(4);
     } else if (warp == 1) {
         // ---- producer warp: refill ring slots as the MMAs release them ----------------------------------------------
         uint32_t slot = 0, phase = 0;   // unit `pre` reuses slot 0 (pre == ring whenever the loop runs)
@@ -414,9 +294,6 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
         const int row = ((warp & 3) << 5) + lane;                  // accumulator row this thread may read (its warp's quarter)
         volatile int &s_bad = *reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 8);
         bool inexact = false;
-#ifdef MXQ_FP4_TRACE
-        long long tr_split = 0, tr_fence = 0;
-#endif
         {
             // Groups of 32 tasks (128 k of one token, one warp) in stage-major order, so that the MMA warp can start on
             // stage 0 while later stages are being split.  Group G: stage G / (2M), then token and 128-k half; in a half
@@ -447,35 +324,16 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                 // The activations have been asked for: weight copies requested from here on queue up behind them, so
                 // the producer may request the rest of the ring (asm volatile keeps this store after the loads).
                 if (G0 == 0 && ct == 0) st_shared_flag(sMisc + 12, 1);
-                if (G0 == 0) TR(13);
 #pragma unroll
                 for (int b = 0; b < kBatch; ++b)
                     if (G0 + 4 * b + cw < ngroups) {   // uniform across the warp
-#ifdef MXQ_FP4_TRACE
-                        const long long c0_ = clock64();
-#endif
                         inexact |= split_half_unit<NB>(raw[b], mm[b], kk[b], lane & 1, lane, sB, sSFB);
-#ifdef MXQ_FP4_TRACE
-                        const long long c1_ = clock64();
-#endif
                         fence_async_proxy();   // ordinary stores, read by the tensor core
                         __syncwarp();
                         if (lane == 0) mbar_arrive(ready0 + (uint32_t)stage[b] * 8u);
-#ifdef MXQ_FP4_TRACE
-                        tr_split += c1_ - c0_;
-                        tr_fence += clock64() - c1_;
-#endif
                     }
             }
         }
-        TR(3);
-#ifdef MXQ_FP4_TRACE
-        if (tid == 64 && blockIdx.x < kTraceCtas) {
-            unsigned long long *row_ = g_fp4_trace[(N >> 7) % 3][blockIdx.x];
-            row_[10] = (unsigned long long)tr_split;
-            row_[11] = (unsigned long long)tr_fence;
-        }
-#endif
         if (inexact) s_bad = 1;
         asm volatile("bar.sync 1, 128;" ::: "memory");
         const int bad = s_bad;
@@ -492,7 +350,6 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
             atomicOr(&g_fp4_status, 4u);
             s_fail = 1;
         }
-        TR(5);
         tc_fence_after();
         // Tile by tile: this thread's row of the accumulator -> registers -> direct store (split == 1) or, for the sum over
         // the cluster in a fixed order, a push to the row's owner.  Rank q owns rows [q*128/split, (q+1)*128/split) of every
@@ -612,7 +469,6 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                 atomicOr(&g_fp4_status, 16u);
                 s_fail = 1;
             }
-            TR(6);
             const float poison = s_fail ? __uint_as_float(0x7FC00000u) : 0.f;
             // (Funnelling the few results of a one-token call through one warp, so that only one warp has stores in flight
             // when the CTA ends, was measured: the serial sums cost more than the shorter launch-to-launch gap saves.)
@@ -688,13 +544,7 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
         }
     }
 
-    TR(7);
     if (split > 1 && warp < 2) cluster_wait();   // pairs with the arrive in the prologue (the other warps waited before their push)
-}
-
-int env_int(const char *name) {
-    const char *e = std::getenv(name);
-    return e ? std::atoi(e) : 0;
 }
 
 template <int NB, bool MULTI, int EPI>
@@ -750,7 +600,8 @@ bool linear_fp4_plan(int M, int64_t N, int64_t K, Fp4Plan &p, bool pow2_split) {
     p.ks = (int)((K + kFp4StageK - 1) / kFp4StageK);
     p.tiles = (int)((N + kFp4TileRows - 1) / kFp4TileRows);
     p.pow2_split = pow2_split ? 1 : 0;
-    return fp4_layout(p, sm_count(), env_int("MXQ_FP4_SPLIT"), env_int("MXQ_FP4_RING"), env_int("MXQ_FP4_TILES"));
+    const LayoutOverride o = layout_override();
+    return fp4_layout(p, sm_count(), o.split, o.ring, o.tiles);
 }
 
 cudaError_t linear_fp4_launch(const Fp4Plan &p, const void *X, const uint8_t *codes, const uint8_t *scales, void *Y,
@@ -778,13 +629,6 @@ cudaError_t linear_fp4_launch(const Fp4Plan &p, const void *X, const uint8_t *co
 #undef MXQ_FP4_PICK
 }
 
-#ifdef MXQ_FP4_TRACE
-}  // namespace mxq
-extern "C" __attribute__((visibility("default"))) int mxq_fp4_trace(unsigned long long *out) {
-    return cudaMemcpyFromSymbol(out, mxq::g_fp4_trace, sizeof(mxq::g_fp4_trace)) == cudaSuccess ? 0 : 6;
-}
-namespace mxq {
-#endif
 
 // returns and clears this kernel's sticky status word (see mxq_linear_device_status)
 int linear_fp4_take_status(uint32_t *out) {

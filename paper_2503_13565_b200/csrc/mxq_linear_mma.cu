@@ -488,26 +488,6 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
 // ---------------------------------------------------------------------------------------------
 // host side: plan + launch
 // ---------------------------------------------------------------------------------------------
-// MXQ_LINEAR_STAGES=2|3 in the environment pins the ring depth (for experiments)
-static int forced_stages() {
-    static const int v = [] {
-        const char *e = std::getenv("MXQ_LINEAR_STAGES");
-        const int n = e ? std::atoi(e) : 0;
-        return (n == 2 || n == 3) ? n : 0;
-    }();
-    return v;
-}
-
-// MXQ_LINEAR_CTAS_PER_SM=1..8 in the environment sets the grid to that many CTAs per SM (for experiments)
-static int forced_ctas_per_sm() {
-    static const int v = [] {
-        const char *e = std::getenv("MXQ_LINEAR_CTAS_PER_SM");
-        const int n = e ? std::atoi(e) : 0;
-        return (n >= 1 && n <= 8) ? n : 0;
-    }();
-    return v;
-}
-
 bool linear_mma_plan(int M, int64_t N, int64_t K, LinearPlan &p) {
     if (M < 1 || M > 16 || (K % 128) != 0 || N < 1) return false;
     const int64_t kb = K / 32;
@@ -522,7 +502,7 @@ bool linear_mma_plan(int M, int64_t N, int64_t K, LinearPlan &p) {
     const uint32_t red_bytes = (uint32_t)kRedSlots * kMmaWarps * kout_bytes;
 
     // grid: two CTAs per SM, more only if a CTA's stage table would overflow; never more CTAs than rows
-    for (int mult = forced_ctas_per_sm() ? forced_ctas_per_sm() : 2; mult <= 4096; mult *= 2) {
+    for (int mult = 2; mult <= 4096; mult *= 2) {
         int64_t grid = (int64_t)sms * mult;
         if (grid > N) grid = N;
         p.grid = (int)grid;
@@ -538,7 +518,7 @@ bool linear_mma_plan(int M, int64_t N, int64_t K, LinearPlan &p) {
             p.smem_bytes = p.off_ring + (uint32_t)(kMmaWarps * nstage * kWarpStageBytes);
             return p.smem_bytes;
         };
-        int nstage = forced_stages() ? forced_stages() : kMaxStages, nwin = 1;
+        int nstage = kMaxStages, nwin = 1;
         int64_t bw = kb;
         if (layout(nstage, bw, nwin) > kSmemThirdSm) {
             while (nstage > 2 && layout(nstage, bw, nwin) > kSmemHalfSm) --nstage;

@@ -677,11 +677,6 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
     if (split > 1 && warp < 2) cluster_wait();   // pairs with the arrive in the prologue (the other warps waited before their push)
 }
 
-int env_int(const char *name) {
-    const char *e = std::getenv(name);
-    return e ? std::atoi(e) : 0;
-}
-
 template <int NB, bool MULTI, bool BRING, int EPI>
 cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X, const uint8_t *codes,
                        const uint8_t *scales, void *Y, int y_dtype, const uint8_t *presplit, cudaStream_t stream, const FusedAccept &fa) {
@@ -727,9 +722,8 @@ cudaError_t launch_umma(const UmmaPlan &p, const CUtensorMap &map, const void *X
 
 // token rows from which the token operand is split ahead of the weight kernel when a workspace is there
 static int presplit_min_m() {
-    static const int v = env_int("MXQ_UMMA_NO_PRESPLIT") != 0 ? kUmmaMaxM + 1
-                         : (env_int("MXQ_UMMA_PRESPLIT_MIN_M") > 0 ? env_int("MXQ_UMMA_PRESPLIT_MIN_M") : kUmmaPresplitMinM);
-    return v;
+    const int forced = layout_override().presplit_min_m;
+    return forced > 0 ? forced : kUmmaPresplitMinM;
 }
 static bool presplit_wanted(int M, int64_t N, int64_t K) {
     const int min_m = presplit_min_m();
@@ -749,8 +743,8 @@ bool linear_umma_plan(int M, int64_t N, int64_t K, UmmaPlan &p, bool with_worksp
     p.nb = umma_nb(M);
     p.ks = (int)(K / kUmmaStageK);
     p.tiles = (int)((N + kUmmaTileRows - 1) / kUmmaTileRows);
-    return umma_layout(p, sm_count(), env_int("MXQ_UMMA_SPLIT"), env_int("MXQ_UMMA_RING"), env_int("MXQ_UMMA_TILES"),
-                       std::getenv("MXQ_UMMA_BRING") ? env_int("MXQ_UMMA_BRING") : -1);
+    const LayoutOverride o = layout_override();
+    return umma_layout(p, sm_count(), o.split, o.ring, o.tiles, o.operand_through_ring);
 }
 
 template <int NB>
@@ -829,14 +823,16 @@ extern "C" {
 #pragma GCC visibility push(default)
 int mxq_linear_device_status(uint32_t *status_host) {
     if (!status_host) return MXQ_ERR_NULL;
-    uint32_t v = 0, v4 = 0, vb = 0;
+    uint32_t v = 0, v4 = 0, vb = 0, vp = 0;
     int rc = mxq::linear_umma_take_status(&v);
     if (rc != MXQ_OK) return rc;
     rc = mxq::linear_fp4_take_status(&v4);
     if (rc != MXQ_OK) return rc;
     rc = mxq::linear_bf16_take_status(&vb);
     if (rc != MXQ_OK) return rc;
-    *status_host = v | (v4 << 8) | (vb << 16);
+    rc = mxq::linear_batch_take_status(&vp);
+    if (rc != MXQ_OK) return rc;
+    *status_host = v | (v4 << 8) | (vb << 16) | (vp << 24);
     return MXQ_OK;
 }
 #pragma GCC visibility pop

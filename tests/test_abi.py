@@ -79,6 +79,50 @@ def test_argument_errors_are_caught_before_any_launch():
     assert L.mxq_lm_head_accept(a, 2, a, a, 1024, 128, a, 1, None, a, a, a, 16, None) == 5
 
 
+def test_batch_argument_errors_are_caught_before_any_launch():
+    L = binding.lib()
+    a = 0x1000
+    descs = (binding._LinearDesc * 2)()
+    for d in descs:
+        d.X_bf16, d.codes, d.scales, d.Y, d.residual = a, a, a, a, None
+        d.N, d.K, d.y_dtype, d.epilogue = 256, 256, 0, 0
+    p = ctypes.cast(descs, ctypes.c_void_p)
+    assert L.mxq_linear_batch(None, 1, 1, a, 1 << 30, None) == 1
+    assert L.mxq_linear_batch(p, 0, 1, a, 1 << 30, None) == 2
+    assert L.mxq_linear_batch(p, 17, 1, a, 1 << 30, None) == 2
+    assert L.mxq_linear_batch(p, 2, 17, a, 1 << 30, None) == 2
+    assert L.mxq_linear_batch(p, 2, 1, None, 0, None) == 1
+    assert L.mxq_linear_batch(p, 2, 1, a + 16, 1 << 30, None) == 3     # workspace not 256-byte aligned
+    assert L.mxq_linear_batch(p, 2, 1, a, 64, None) == 5
+    assert L.mxq_linear_batch_workspace_bytes(p, 2, 1) >= 8192
+    descs[1].epilogue = 1                                              # residual epilogue without a residual
+    assert L.mxq_linear_batch(p, 2, 1, a, 1 << 30, None) == 1
+    descs[1].epilogue = 2
+    descs[1].N = 255                                                   # gate / up pairing needs an even N
+    assert L.mxq_linear_batch(p, 2, 1, a, 1 << 30, None) == 2
+    descs[1].epilogue, descs[1].N, descs[1].K = 0, 256, 100
+    assert L.mxq_linear_batch(p, 2, 1, a, 1 << 30, None) == 2
+    descs[1].K, descs[1].y_dtype = 256, 9
+    assert L.mxq_linear_batch(p, 2, 1, a, 1 << 30, None) == 4
+    descs[1].y_dtype, descs[1].codes = 0, a + 4
+    assert L.mxq_linear_batch(p, 2, 1, a, 1 << 30, None) == 3
+    assert L.mxq_linear_batch_workspace_bytes(p, 2, 1) == 0
+    assert L.mxq_set_linear_layout(99, 1) == 2 and L.mxq_set_linear_layout(5, 0) == 0
+
+
+def test_linear_host_checks_every_argument_before_staging():
+    """A bad codes / scales / Y pointer must be refused before the staging copy of X is enqueued (a fake X pointer
+    would otherwise be handed to the copy engine)."""
+    L = binding.lib()
+    a = 0x1000
+    assert L.mxq_linear_host(a, 1, None, a, 8, 64, a, 0, a, a, None, 0, None) == 1
+    assert L.mxq_linear_host(a, 1, a, None, 8, 64, a, 0, a, a, None, 0, None) == 1
+    assert L.mxq_linear_host(a, 1, a + 4, a, 8, 64, a, 0, a, a, None, 0, None) == 3
+    assert L.mxq_linear_host(a, 1, a, a + 4, 8, 64, a, 0, a, a, None, 0, None) == 3
+    assert L.mxq_linear_host(a, 1, a, a, 8, 64, a, 0, a + 4, a, None, 0, None) == 3
+    assert L.mxq_linear_host(a, 1, a, a, 8, 64, a, 0, a, a + 4, None, 0, None) == 3
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))

@@ -127,13 +127,13 @@ def test_largest_vocabularies_sampled_rows(m, n):
     check_linear(y[:, torch.as_tensor(rows, device="cuda")], y64, a64, "vocabulary %d M=%d" % (n, m))
 
 
-@pytest.mark.parametrize("force", ["0", "1"])
+@pytest.mark.parametrize("force", [0, 1])
 @pytest.mark.parametrize("m,n,k", [(5, 203, 1408), (8, 4096, 4096), (16, 1000, 4096), (3, 300, 5120), (8, 32000, 4096), (16, 32000, 768)])
-def test_token_operand_resident_and_through_the_ring(m, n, k, force, monkeypatch):
+def test_token_operand_resident_and_through_the_ring(m, n, k, force):
     """With a workspace the FP8-operand kernel keeps the pre-split token operand of a CTA's whole K range in shared
-    memory, or fetches it stage by stage into the ring slots; the layout heuristic picks one, MXQ_UMMA_BRING forces
-    either.  Both must give the layer's result for every operand width, with one tile per CTA and with several."""
-    monkeypatch.setenv("MXQ_UMMA_BRING", force)
+    memory, or fetches it stage by stage into the ring slots; the layout heuristic picks one, mxq_set_linear_layout
+    forces either.  Both must give the layer's result for every operand width, with one tile per CTA and with several."""
+    mxq.mxq_set_linear_layout("operand_through_ring", force)
     prev = mxq.mxq_set_linear_kernel("umma")
     try:
         w = synth.bits_of(synth.weight(3, 16, n, k))
@@ -142,6 +142,7 @@ def test_token_operand_resident_and_through_the_ring(m, n, k, force, monkeypatch
         run_case(w, x, rows=rows, what="bring=%s" % force)
     finally:
         mxq.mxq_set_linear_kernel(prev)
+        mxq.mxq_set_linear_layout("operand_through_ring", -1)
 
 
 def test_bf16_output_is_the_rounded_fp32_output():

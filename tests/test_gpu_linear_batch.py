@@ -1,0 +1,232 @@
+"""GPU parity of mxq_linear_batch (several layers in one persistent launch) against the oracle, layer by layer.
+
+Plain layers: |y - y64| <= 2e-3 * sum|x w^| + 1e-6 element by element (the bound of mxq_linear); epilogues: the bounds
+of tests/test_gpu_epilogues.py.  The cases cover one CTA per unit (tiny calls), tiles cut between two and three CTAs'
+ranges, ragged N, the half-full last stage (K % 256 == 128), shared and distinct X, every token count the persistent
+kernel takes (1..4) and the calls it hands on to the one-by-one path.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2503_13565_b200 as mxq
+from paper_2503_13565_b200 import synth
+from parity import ABS, REL, check_linear, gpu_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def status_clean():
+    yield
+    assert mxq.mxq_linear_device_status() == 0, "a bounded wait inside a kernel gave up"
+
+
+def values(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def make_layer(cfg, idx, n, k, m, x=None, epilogue="none", out_dtype=torch.float32, rows=None):
+    """One layer of a batch with everything the oracle needs to check it afterwards."""
+    codes, scales, _ = oracle.quantize(synth.bits_of(synth.weight(cfg, idx, n, k)))
+    xbits = synth.bits_of(synth.activations(cfg, idx, m, k)) if x is None else x
+    lay = {"x": gpu_bf16(xbits), "codes": torch.from_numpy(codes).cuda(), "scales": torch.from_numpy(scales).cuda(),
+           "epilogue": epilogue, "_codes": codes, "_scales": scales, "_x": xbits, "_rows": rows}
+    n_out = n // 2 if epilogue == "swiglu" else n
+    lay["out"] = torch.full((m, n_out), float("nan"), dtype=out_dtype, device="cuda")
+    if epilogue == "residual":
+        g = torch.Generator().manual_seed(500 + idx)
+        lay["residual"] = (torch.randn(m, n, generator=g) * 0.5).to(out_dtype).cuda()
+    return lay
+
+
+def check_layer(lay, what):
+    rows = lay["_rows"]
+    sel = slice(None) if rows is None else np.asarray(rows)
+    out_dtype = lay["out"].dtype
+    bf = (lambda want: np.abs(want) * 2.0 ** -8) if out_dtype == torch.bfloat16 else (lambda want: 0.0)
+    got = values(lay["out"])
+    if lay["epilogue"] == "none":
+        y64, a64 = oracle.linear(lay["_x"], lay["_codes"], lay["_scales"], rows=rows)
+        if out_dtype == torch.float32:
+            return check_linear(lay["out"] if rows is None else lay["out"][:, torch.as_tensor(rows, device="cuda")], y64, a64, what)
+        tol = REL * a64 + ABS + bf(y64)
+        want = y64
+    elif lay["epilogue"] == "residual":
+        r64 = values(lay["residual"])[:, sel]
+        want, a = oracle.linear_residual(lay["_x"], lay["_codes"], lay["_scales"], r64, rows=rows)
+        tol = REL * a + ABS + 2.0 ** -23 * np.abs(want) + bf(want)
+    else:
+        want, g, u, ag, au = oracle.linear_swiglu(lay["_x"], lay["_codes"], lay["_scales"], rows=rows)
+        tg, tu = REL * ag + ABS, REL * au + ABS
+        tol = 1.1 * tg * (np.abs(u) + tu) + np.abs(oracle.silu(g)) * tu + 1e-6 * np.abs(want) + 1e-30 + bf(want)
+    got = got[:, sel]
+    assert np.isfinite(got).all(), what + ": non-finite output"
+    worst = float((np.abs(got - want) / tol).max())
+    assert worst <= 1.0, "%s: error/tolerance = %.3g" % (what, worst)
+    return worst
+
+
+def run_batch(layers, expect_persistent=True):
+    batch = mxq.LinearBatch(layers)
+    assert bool(batch.info()["persistent"]) == expect_persistent, batch.info()
+    ws = mxq.new_workspace(batch.workspace_bytes())
+    batch.run(ws)
+    torch.cuda.synchronize()
+    return batch, ws
+
+
+def sample_rows(n, seed, count=300):
+    return np.unique(np.concatenate([[0, 1, 127, 128, n - 129, n - 128, n - 2, n - 1],
+                                     np.random.default_rng(seed).integers(0, n, count)])).astype(np.int64)
+
+
+@pytest.mark.parametrize("m", [1, 2, 3, 4])
+def test_small_ragged_layers(m):
+    """Fewer units than SMs (every CTA owns one unit, every tile is summed across CTAs), ragged N, half-full last stage."""
+    layers = [make_layer(3, 20, 203, 1408, m), make_layer(3, 21, 515, 2048, m), make_layer(3, 22, 128, 128, m),
+              make_layer(3, 23, 1000, 384, m)]
+    run_batch(layers)
+    for i, lay in enumerate(layers):
+        check_layer(lay, "small batch layer %d M=%d" % (i, m))
+
+
+@pytest.mark.parametrize("m", [1, 4])
+def test_config2_draft_model_layer_set(m):
+    """The 68M-Llama-like draft model's layer set in one call; q/k/v share X, gate/up share X."""
+    xh = synth.bits_of(synth.activations(2, 0, m, 768))
+    xf = synth.bits_of(synth.activations(2, 6, m, 3072))
+    layers = [make_layer(2, i, 768, 768, m, x=xh) for i in range(4)]
+    layers += [make_layer(2, 4, 3072, 768, m, x=xh), make_layer(2, 5, 3072, 768, m, x=xh), make_layer(2, 6, 768, 3072, m, x=xf),
+               make_layer(2, 7, 32000, 768, m, x=xh, rows=sample_rows(32000, 1))]
+    xg = layers[0]["x"]
+    for lay in layers[:6] + layers[7:]:
+        lay["x"] = xg   # the same device tensor: one image
+    run_batch(layers)
+    for i, lay in enumerate(layers):
+        check_layer(lay, "config2 layer %d M=%d" % (i, m))
+
+
+@pytest.mark.parametrize("m", [1, 2, 4])
+def test_config3_7b_layer_set(m):
+    """The benchmark's call: seven 7B-shaped layers in one launch, sampled rows of every layer against the oracle."""
+    shapes = synth.LAYERS_7B
+    xs = {k: gpu_bf16(synth.bits_of(synth.activations(3, 0 if k == 4096 else 6, m, k))) for k in (4096, 11008)}
+    layers = []
+    for i, (name, n, k) in enumerate(shapes):
+        lay = make_layer(3, i, n, k, m, x=synth.bits_of(synth.activations(3, 0 if k == 4096 else 6, m, k)), rows=sample_rows(n, i, 500))
+        lay["x"] = xs[k]
+        layers.append(lay)
+    batch, ws = run_batch(layers)
+    assert batch.info()["grid"] == torch.cuda.get_device_properties(0).multi_processor_count
+    for i, lay in enumerate(layers):
+        check_layer(lay, "7B layer %s M=%d" % (shapes[i][0], m))
+    # bit-reproducible, and the workspace is reusable as it was left
+    first = [lay["out"].clone() for lay in layers]
+    for lay in layers:
+        lay["out"].fill_(float("nan"))
+    batch.run(ws)
+    torch.cuda.synchronize()
+    for a, lay in zip(first, layers):
+        assert torch.equal(a, lay["out"])
+
+
+@pytest.mark.parametrize("m", [1, 3])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_epilogues(m, out_dtype):
+    layers = [make_layer(3, 30, 1000, 1024, m, epilogue="residual", out_dtype=out_dtype),
+              make_layer(3, 31, 2 * 700, 1024, m, epilogue="swiglu", out_dtype=out_dtype),
+              make_layer(3, 32, 4096, 4096, m, epilogue="residual", out_dtype=out_dtype, rows=sample_rows(4096, 2)),
+              make_layer(3, 33, 2 * 2752, 4096, m, epilogue="swiglu", out_dtype=out_dtype, rows=sample_rows(2752, 3)),
+              make_layer(3, 34, 333, 1152, m, out_dtype=out_dtype)]
+    res_before = [lay.get("residual").clone() if lay.get("residual") is not None else None for lay in layers]
+    run_batch(layers)
+    for i, lay in enumerate(layers):
+        check_layer(lay, "epilogue layer %d M=%d %s" % (i, m, out_dtype))
+        if res_before[i] is not None:
+            assert torch.equal(res_before[i], lay["residual"]), "the residual was written to"
+
+
+def test_residual_in_place():
+    lay = make_layer(3, 35, 640, 2048, 2, epilogue="residual")
+    keep = lay["residual"].clone()
+    lay["out"] = lay["residual"]
+    run_batch([lay])
+    lay["residual"] = keep
+    check_layer(lay, "in-place residual")
+
+
+def test_one_workspace_across_differently_shaped_calls():
+    """Calls in one stream share a workspace: every call leaves the counters as it found them."""
+    a = [make_layer(3, 40, 203, 1408, 1), make_layer(3, 41, 4096, 4096, 1, rows=sample_rows(4096, 4))]
+    b = [make_layer(3, 42, 515, 2048, 4), make_layer(3, 43, 900, 640, 4), make_layer(3, 44, 300, 5120, 4)]
+    ba, bb = mxq.LinearBatch(a), mxq.LinearBatch(b)
+    ws = mxq.new_workspace(max(ba.workspace_bytes(), bb.workspace_bytes()))
+    for _ in range(3):
+        ba.run(ws)
+        bb.run(ws)
+    torch.cuda.synchronize()
+    assert int(ws[:8192].view(torch.int32).abs().sum()) == 0, "counters not left at zero"
+    for i, lay in enumerate(a + b):
+        check_layer(lay, "shared workspace layer %d" % i)
+
+
+def test_activations_that_cannot_be_rewritten_exactly():
+    """An element more than 24 binades below its block's maximum, an infinity, a NaN: the affected layers take the
+    scalar path (same bound), the other layers of the call are untouched."""
+    m, k = 2, 1024
+    x = synth.activations(3, 50, m, k).clone()
+    x[0, 5] = 2.0 ** -40
+    x[0, 6] = 1.0
+    xb = synth.bits_of(x)
+    lay_bad = make_layer(3, 50, 515, k, m, x=xb)
+    lay_ok = make_layer(3, 51, 300, 768, m)
+    run_batch([lay_bad, lay_ok])
+    check_layer(lay_bad, "tiny element")
+    check_layer(lay_ok, "untouched layer")
+    x2 = synth.activations(3, 52, m, k).clone()
+    x2[1, 40] = float("inf")
+    lay_inf = make_layer(3, 52, 260, k, m, x=synth.bits_of(x2))
+    run_batch([lay_inf])
+    y64, a64 = oracle.linear(lay_inf["_x"], lay_inf["_codes"], lay_inf["_scales"])
+    got = values(lay_inf["out"])
+    assert np.array_equal(np.isnan(got[1]), np.isnan(y64[1])) and np.array_equal(got[1][~np.isnan(got[1])], y64[1][~np.isnan(y64[1])])
+    check_linear(lay_inf["out"][:1], y64[:1], a64[:1], "row without the infinity")
+
+
+@pytest.mark.parametrize("m,n,k", [(8, 515, 2048), (1, 203, 1440), (16, 300, 1024)])
+def test_calls_the_persistent_kernel_does_not_cover(m, n, k):
+    """More than 4 token rows, or K not a multiple of 128: the layers run one by one, with the same results as the
+    single-layer entry points."""
+    layers = [make_layer(3, 60, n, k, m), make_layer(3, 61, 2 * 128, k, m, epilogue="swiglu"),
+              make_layer(3, 62, n, k, m, epilogue="residual")]
+    run_batch(layers, expect_persistent=False)
+    for i, lay in enumerate(layers):
+        check_layer(lay, "one-by-one layer %d M=%d" % (i, m))
+
+
+@pytest.mark.parametrize("ring,per_sm", [(2, 1), (3, 2), (5, 2), (1, 1)])
+def test_other_ring_depths_and_two_ctas_per_sm(ring, per_sm):
+    mxq.mxq_set_linear_layout("batch_ring", ring)
+    mxq.mxq_set_linear_layout("batch_ctas_per_sm", per_sm)
+    try:
+        layers = [make_layer(3, 70, 4096, 4096, 1, rows=sample_rows(4096, 5)), make_layer(3, 71, 1000, 11008, 1),
+                  make_layer(3, 72, 203, 1408, 1)]
+        batch, _ = run_batch(layers)
+        assert batch.info()["ring"] == ring
+        for i, lay in enumerate(layers):
+            check_layer(lay, "ring %d, %d CTAs per SM, layer %d" % (ring, per_sm, i))
+    finally:
+        mxq.mxq_set_linear_layout("batch_ring", 0)
+        mxq.mxq_set_linear_layout("batch_ctas_per_sm", 0)
+
+
+def test_argument_errors():
+    lay = make_layer(3, 80, 256, 256, 1)
+    batch = mxq.LinearBatch([lay])
+    with pytest.raises(mxq.MxqError) as e:
+        batch.run(torch.zeros(4096, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 5
+    with pytest.raises(ValueError):
+        mxq.LinearBatch([lay] * 17)

@@ -305,7 +305,7 @@ int mxq_linear_swiglu(const void *X_bf16, int M, const uint8_t *codes, const uin
  * other through mxq_linear / mxq_linear_residual / mxq_linear_swiglu (same results as those).  Results are
  * bit-reproducible run to run and within mxq_linear's bound; the summation order differs from mxq_linear's.  Errors as
  * mxq_linear.  Bounded waits that give up are reported in bits 24-27 of mxq_linear_device_status. */
-#define MXQ_MAX_BATCH 16
+#define MXQ_MAX_BATCH 32
 enum mxq_epilogue { MXQ_EPI_NONE = 0, MXQ_EPI_RESIDUAL = 1, MXQ_EPI_SWIGLU = 2 };
 typedef struct mxq_linear_desc {
     const void *X_bf16;

@@ -17,7 +17,7 @@
 //     epilogue warps read the previous one.
 // Warp roles (320 threads): warp 0 issues the MMAs and owns tensor memory; warp 1 is the producer (TMA copies of the
 // codes, bulk copies of the token operand); warps 2..5 first rewrite their share of the token rows and then run the
-// epilogues; warps 6..9 move the scale bytes (thread r those of weight row r) into the slots' scale atoms.  Every wait is bounded; one that gives up sets a sticky status bit and the
+// epilogues; warps 6..9 move the scale bytes into the slots' scale atoms (warp w those of every fourth unit).  Every wait is bounded; one that gives up sets a sticky status bit and the
 // CTA's remaining tiles are written as NaN.
 #include <atomic>
 #include <cstdio>
@@ -38,7 +38,7 @@ namespace {
 // never released, 3 the token operand never became ready
 __device__ unsigned int g_batch_status = 0;
 
-constexpr uint32_t kFullArrivals = 1 + 4;   // the producer's arrive (with the bytes it announces) + one arrive per scale warp
+constexpr uint32_t kFullArrivals = 1 + 1;   // the producer's arrive (with the bytes it announces) + the arrive of the scale warp that serves the unit
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
     uint32_t v;
@@ -56,6 +56,7 @@ __device__ __forceinline__ float ld_cg_f32(const float *p) {
     return v;
 }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
 
 // Bounded wait on an mbarrier that also ends when the CTA's failure flag is raised.  False: gave up.  The probes are
 // back to back (the instruction itself suspends the warp for a while when the phase is not complete): a sleep between
@@ -394,86 +395,68 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
         }
         __syncwarp();
     } else if (warp >= 6) {
-        // ---- scale warps: thread r brings the scale bytes of weight row r of every unit into the slot's scale atoms ------
-        // (8 bytes per row and unit, rows K / 32 bytes apart; each thread has the loads of the next four units in flight
-        // in registers)
-        const int r = tid - 192;   // 0..127
-        const uint32_t pos = (uint32_t)(r & 31) * 16u + (uint32_t)(r >> 5) * 4u;   // row r inside a 512-byte atom
-        Cursor cl;
-        walk_begin(tb, wk, cl);
-        const uint8_t *row_ptr = nullptr;   // scale bytes of this thread's row of the tile the load cursor is in (nullptr: no such row)
-        bool wide = true;                   // K % 256 == 0: a unit's 8 bytes are one aligned load
-        auto load = [&](int li) -> uint2 {
-            if (li) walk_to(tb, wk, li, cl);
-            if (walk_opens(wk, li, cl)) {
-                const BatchDesc &ds = tb.desc[cl.d];
-                const int n = cl.t * kBatchTileRows + r;
-                wide = (ds.K & (kBatchStageK - 1)) == 0;
-                row_ptr = n < ds.N ? ds.scales + (int64_t)n * (ds.K >> 5) : nullptr;
-            }
-            uint2 v = make_uint2(0u, 0u);
-            if (row_ptr) {
-                const uint8_t *src = row_ptr + cl.s * 8;
-                if (wide) {
-                    asm volatile("ld.global.nc.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(src));
-                } else {
-                    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v.x) : "l"(src));
-                    if (cl.s != cl.ks - 1) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v.y) : "l"(src + 4));
+        // ---- scale warps: warp w brings the scale bytes of units w, w + 4, w + 8, ... of the walk into the slots' scale atoms
+        // (8 bytes per weight row and unit, rows K / 32 bytes apart).  Lane l takes rows l, l + 32, l + 64, l + 96, whose
+        // bytes are neighbours in an atom: two 16-byte shared stores per lane and unit.  The loads of a warp's next unit
+        // are in flight in registers while it waits for the slot of the current one.
+        // (At most `ring` warps take part: a warp's consecutive units must be no more than a ring apart, or its parity wait
+        // for the slot's release could be answered by the release before that one.)
+        const int sw = warp - 6;   // 0..3
+        const int nsw = ring < 4 ? ring : 4;
+        uint32_t rows_lo[4], rows_hi[4];
+        auto load = [&](int i, uint32_t (&lo)[4], uint32_t (&hi)[4]) {   // element i of the walk
+            Cursor c;
+            cursor_at(tb, walk_unit(wk, i), c);
+            const BatchDesc &ds = tb.desc[c.d];
+            const int kb_row = ds.K >> 5;
+            const bool wide = (ds.K & (kBatchStageK - 1)) == 0;   // a unit's 8 bytes are one aligned load
+            const bool second = wide || c.s != c.ks - 1;
+            const int n0 = c.t * kBatchTileRows + lane;
+            const uint8_t *src = ds.scales + (int64_t)n0 * kb_row + c.s * 8;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                lo[q] = hi[q] = 0u;
+                if (n0 + 32 * q < ds.N) {
+                    if (wide) {
+                        asm volatile("ld.global.nc.v2.u32 {%0,%1}, [%2];" : "=r"(lo[q]), "=r"(hi[q]) : "l"(src));
+                    } else {
+                        asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(lo[q]) : "l"(src));
+                        if (second) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(hi[q]) : "l"(src + 4));
+                    }
                 }
+                src += (int64_t)32 * kb_row;
             }
-            return v;
         };
-        constexpr int D = 4;   // units ahead
-        uint2 v[D];
-        int li = 0;            // next element to load
+        if (sw < nsw && sw < nunit) load(sw, rows_lo, rows_hi);
+        // element i goes to slot i % ring: the slot index advances by nsw (mod ring) from one unit of this warp to the next
+        uint32_t slot = (uint32_t)sw, round = 0;   // (sw < nsw <= ring)
+        const uint32_t step = (uint32_t)nsw % (uint32_t)ring, carry = (uint32_t)nsw / (uint32_t)ring;
+        for (int i = sw < nsw ? sw : nunit; i < nunit; i += nsw) {
+            uint32_t cur_lo[4], cur_hi[4];
 #pragma unroll
-        for (int j = 0; j < D; ++j) {
-            v[j] = make_uint2(0u, 0u);
-            if (li < nunit) {
-                v[j] = load(li);
-                ++li;
+            for (int q = 0; q < 4; ++q) {
+                cur_lo[q] = rows_lo[q];
+                cur_hi[q] = rows_hi[q];
             }
-        }
-        bool ok = true;
-        uint32_t sf = base + kBatchCodesBytes + pos, fb = full0, eb = empty0, phase = 0;
-        bool wrapped = false;
-        const uint32_t sf_end = sf + (uint32_t)ring * kSlot;
-        for (int i0 = 0; i0 < nunit && ok; i0 += D) {
-#pragma unroll
-            for (int j = 0; j < D; ++j) {
-                if (i0 + j < nunit && ok) {
-                    const uint2 cur = v[j];
-                    if (li < nunit) {
-                        v[j] = load(li);
-                        ++li;
-                    }
-                    if (wrapped) {
-                        // one thread probes for all four scale warps; barrier 3 passes the result on
-                        if (tid == 192 && !wait_bar(eb, phase, s_fail, limit_us)) {
-                            atomicOr(&g_batch_status, 2u);
-                            *s_fail = 1;
-                        }
-                        asm volatile("bar.sync 3, 128;" ::: "memory");
-                        if (*s_fail) ok = false;
-                    }
-                    if (ok) {
-                        asm volatile("st.shared.u32 [%0], %1;" ::"r"(sf), "r"(cur.x) : "memory");
-                        asm volatile("st.shared.u32 [%0], %1;" ::"r"(sf + 512u), "r"(cur.y) : "memory");
-                        fence_async_proxy();   // ordinary stores, read by tcgen05.cp
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(fb);
-                        sf += kSlot;
-                        fb += 8u;
-                        eb += 8u;
-                        if (sf == sf_end) {
-                            sf -= (uint32_t)ring * kSlot;
-                            fb = full0;
-                            eb = empty0;
-                            if (wrapped) phase ^= 1u;
-                            wrapped = true;
-                        }
-                    }
+            if (i + nsw < nunit) load(i + nsw, rows_lo, rows_hi);
+            if (round != 0 && !warp_wait_bar(empty0 + slot * 8u, (round - 1u) & 1u, s_fail, limit_us, lane)) {
+                if (lane == 0) {
+                    atomicOr(&g_batch_status, 2u);
+                    *s_fail = 1;
                 }
+                break;
+            }
+            const uint32_t sf = base + slot * kSlot + kBatchCodesBytes + (uint32_t)lane * 16u;
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(sf), "r"(cur_lo[0]), "r"(cur_lo[1]), "r"(cur_lo[2]), "r"(cur_lo[3]) : "memory");
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(sf + 512u), "r"(cur_hi[0]), "r"(cur_hi[1]), "r"(cur_hi[2]), "r"(cur_hi[3]) : "memory");
+            fence_async_proxy();   // ordinary stores, read by tcgen05.cp
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full0 + slot * 8u);
+            slot += step;
+            round += carry;
+            if (slot >= (uint32_t)ring) {
+                slot -= (uint32_t)ring;
+                ++round;
             }
         }
     } else {
@@ -729,7 +712,10 @@ struct BatchLayout {
 bool batch_layout(int M, int64_t units, BatchLayout &L) {
     const LayoutOverride o = layout_override();
     L.nb = batch_nb(M);
-    const int per_sm = o.batch_ctas_per_sm >= 1 && o.batch_ctas_per_sm <= 2 ? o.batch_ctas_per_sm : 1;
+    // Two CTAs per SM by default: what a CTA's single MMA-issuing, single requesting and single probing threads do per
+    // unit bounds one CTA at about two units per microsecond, and a second CTA's streams fill the gaps (7B layer sets at
+    // M = 1, four per call: 25.5 us per layer set with one CTA per SM and a ring of 5, 21.1 us with two).
+    const int per_sm = o.batch_ctas_per_sm >= 1 && o.batch_ctas_per_sm <= 2 ? o.batch_ctas_per_sm : 2;
     int ring = o.batch_ring > 0 ? o.batch_ring : 64;
     // the deepest ring that lets `per_sm` CTAs share an SM's shared memory (each CTA also takes 1 KB of system use)
     while (ring > 1 && (batch_smem_bytes(L.nb, ring) + 1024u) * (uint32_t)per_sm > 228u * 1024u) --ring;

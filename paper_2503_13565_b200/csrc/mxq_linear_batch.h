@@ -13,7 +13,7 @@
 
 namespace mxq {
 
-constexpr int kBatchMaxDescs = 16;       // layers per call (the table travels as a kernel parameter)
+constexpr int kBatchMaxDescs = 32;       // layers per call (the table travels as a kernel parameter, 7.5 KB)
 constexpr int kBatchMaxM = 4;            // token rows: 16 digit planes each, 64 operand columns at most
 constexpr int kBatchThreads = 320;       // MMA warp, producer warp, four split / epilogue warps, four scale warps
 constexpr int kBatchTileRows = 128;      // weight rows per tile = M of one tcgen05.mma
@@ -25,14 +25,14 @@ constexpr int kBatchMaxGrid = 1024;      // CTAs (ticket counters in the workspa
 
 // ---- workspace ------------------------------------------------------------------------------------------------------
 // [0, kBatchHeaderBytes)  counters, all zero between calls:
-//      u32 ready[16]   split tasks delivered per token-operand image
-//      u32 bad[16]     an image holds a block that could not be rewritten exactly
-//      u32 exit        CTAs that have finished (word 32)
-//      u32 ticket[kBatchMaxGrid] at byte 256: contributors that have delivered their share of a tile split between CTAs
+//      u32 ready[32]   split tasks delivered per token-operand image
+//      u32 bad[32]     an image holds a block that could not be rewritten exactly
+//      u32 exit        CTAs that have finished (word 64)
+//      u32 ticket[kBatchMaxGrid] at byte 512: contributors that have delivered their share of a tile split between CTAs
 // [kBatchHeaderBytes, ...) partial sums: [grid][2 (at the head / at the tail of the CTA's range)][token slots][128] floats
 // then the token-operand images, one per distinct X: [stage][operand rows NB x 128 bytes | 1024 bytes of scale atoms]
 constexpr size_t kBatchHeaderBytes = 8192;
-constexpr int kBatchWordReady = 0, kBatchWordBad = 16, kBatchWordExit = 32, kBatchWordTicket = 64;
+constexpr int kBatchWordReady = 0, kBatchWordBad = 32, kBatchWordExit = 64, kBatchWordTicket = 128;
 
 inline int batch_nb(int M) { return M == 1 ? 16 : (M == 2 ? 32 : 64); }   // operand columns: 16 planes per token slot
 inline uint32_t batch_image_stage_bytes(int nb) { return (uint32_t)nb * 128u + kBatchSfBytes; }

@@ -119,7 +119,7 @@ def test_config3_7b_layer_set(m):
         lay["x"] = xs[k]
         layers.append(lay)
     batch, ws = run_batch(layers)
-    assert batch.info()["grid"] == torch.cuda.get_device_properties(0).multi_processor_count
+    assert batch.info()["grid"] == 2 * torch.cuda.get_device_properties(0).multi_processor_count
     for i, lay in enumerate(layers):
         check_layer(lay, "7B layer %s M=%d" % (shapes[i][0], m))
     # bit-reproducible, and the workspace is reusable as it was left
@@ -222,6 +222,14 @@ def test_other_ring_depths_and_two_ctas_per_sm(ring, per_sm):
         mxq.mxq_set_linear_layout("batch_ctas_per_sm", 0)
 
 
+def test_thirty_two_layers_in_one_call():
+    """The most layers a call takes: 32 small ones with 32 distinct X."""
+    layers = [make_layer(3, 90 + i, 128 + 64 * (i % 5), 256 + 128 * (i % 4), 2) for i in range(32)]
+    run_batch(layers)
+    for i, lay in enumerate(layers):
+        check_layer(lay, "layer %d of 32" % i)
+
+
 def test_argument_errors():
     lay = make_layer(3, 80, 256, 256, 1)
     batch = mxq.LinearBatch([lay])
@@ -229,4 +237,4 @@ def test_argument_errors():
         batch.run(torch.zeros(4096, dtype=torch.uint8, device="cuda"))
     assert e.value.status == 5
     with pytest.raises(ValueError):
-        mxq.LinearBatch([lay] * 17)
+        mxq.LinearBatch([lay] * 33)

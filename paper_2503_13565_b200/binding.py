@@ -473,7 +473,7 @@ class LinearBatch:
     def info(self) -> dict:
         info = (ctypes.c_int32 * 8)()
         _check(lib().mxq_linear_batch_info(self._ptr, self.count, self.m, ctypes.cast(info, ctypes.c_void_p)), "mxq_linear_batch_info")
-        return dict(zip(("persistent", "grid", "ring", "smem_bytes", "nb", "units", "tmem_cols"), [int(v) for v in info]))
+        return dict(zip(("persistent", "grid", "ring", "smem_bytes", "nb", "units", "tmem_cols", "acc_slots"), [int(v) for v in info]))
 
     def run(self, workspace: torch.Tensor, stream=None) -> None:
         _check(lib().mxq_linear_batch(self._ptr, self.count, self.m, _dev(workspace, torch.uint8, "workspace"),

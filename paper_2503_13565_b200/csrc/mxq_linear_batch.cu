@@ -143,7 +143,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
     constexpr int MT = NB / 16;   // token slots
     constexpr uint32_t kXBytes = (uint32_t)NB * 128u + kBatchSfBytes;
     constexpr uint32_t kSlot = kBatchCodesBytes + kBatchSfBytes + kXBytes;
-    constexpr int A = NB <= 32 ? 4 : 3;   // accumulator slots (batch_acc_slots)
+    const int A = tb.acc_slots;   // accumulator slots (1..4)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = (int)gridDim.x, cta = (int)blockIdx.x;
     const int M = tb.M, ring = tb.ring;
@@ -704,7 +704,7 @@ std::atomic<int> g_fault_unit{-1};
 std::atomic<unsigned> g_fault_wait_us{0};
 
 struct BatchLayout {
-    int nb, ring, grid;
+    int nb, ring, grid, per_sm;
     uint32_t smem;
 };
 
@@ -720,7 +720,8 @@ bool batch_layout(int M, int64_t units, BatchLayout &L) {
     // the deepest ring that lets `per_sm` CTAs share an SM's shared memory (each CTA also takes 1 KB of system use)
     while (ring > 1 && (batch_smem_bytes(L.nb, ring) + 1024u) * (uint32_t)per_sm > 228u * 1024u) --ring;
     if (batch_smem_bytes(L.nb, ring) > kBatchSmemLimit) return false;
-    if (per_sm * batch_tmem_cols(L.nb) > 512) return false;
+    if (batch_acc_slots(L.nb, per_sm) < 1) return false;
+    L.per_sm = per_sm;
     L.ring = ring;
     int64_t grid = (int64_t)sm_count() * per_sm;
     if (grid > units) grid = units;
@@ -816,7 +817,8 @@ int mxq_linear_batch_info(const mxq_linear_desc *descs, int count, int M, int32_
     info[3] = (int32_t)L.smem;
     info[4] = L.nb;
     info[5] = (int32_t)units;
-    info[6] = mxq::batch_tmem_cols(L.nb);
+    info[6] = mxq::batch_tmem_cols(L.nb, L.per_sm);
+    info[7] = mxq::batch_acc_slots(L.nb, L.per_sm);
     return MXQ_OK;
 }
 
@@ -850,7 +852,8 @@ int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *works
     tb.ndesc = count;
     tb.M = M;
     tb.ring = L.ring;
-    tb.tmem_cols = mxq::batch_tmem_cols(nb);
+    tb.tmem_cols = mxq::batch_tmem_cols(nb, L.per_sm);
+    tb.acc_slots = mxq::batch_acc_slots(nb, L.per_sm);
     tb.partials_offset = (uint32_t)mxq::kBatchHeaderBytes;
     size_t img_off = mxq::kBatchHeaderBytes + mxq::batch_partials_bytes(mxq::kBatchMaxGrid, nb);
     int unit_base = 0, task_base = 0, nimg = 0;
@@ -897,7 +900,8 @@ int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *works
     tb.wait_us = w ? w : 1000000u;
     const cudaError_t e = nb == 16 ? mxq::launch_batch<16>(tb, L.grid, L.smem, st)
                           : nb == 32 ? mxq::launch_batch<32>(tb, L.grid, L.smem, st)
-                                     : mxq::launch_batch<64>(tb, L.grid, L.smem, st);
+                          : nb == 64 ? mxq::launch_batch<64>(tb, L.grid, L.smem, st)
+                                     : mxq::launch_batch<128>(tb, L.grid, L.smem, st);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return MXQ_ERR_CUDA;

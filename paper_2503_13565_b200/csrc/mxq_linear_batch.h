@@ -14,7 +14,7 @@
 namespace mxq {
 
 constexpr int kBatchMaxDescs = 32;       // layers per call (the table travels as a kernel parameter, 7.5 KB)
-constexpr int kBatchMaxM = 4;            // token rows: 16 digit planes each, 64 operand columns at most
+constexpr int kBatchMaxM = 8;            // token rows: 16 digit planes each, 128 operand columns at most
 constexpr int kBatchThreads = 320;       // MMA warp, producer warp, four split / epilogue warps, four scale warps
 constexpr int kBatchTileRows = 128;      // weight rows per tile = M of one tcgen05.mma
 constexpr int kBatchStageK = 256;        // k per unit = 128 packed bytes per row = 8 MX blocks = 4 MMAs of K = 64
@@ -34,15 +34,19 @@ constexpr int kBatchMaxGrid = 1024;      // CTAs (ticket counters in the workspa
 constexpr size_t kBatchHeaderBytes = 8192;
 constexpr int kBatchWordReady = 0, kBatchWordBad = 32, kBatchWordExit = 64, kBatchWordTicket = 128;
 
-inline int batch_nb(int M) { return M == 1 ? 16 : (M == 2 ? 32 : 64); }   // operand columns: 16 planes per token slot
+inline int batch_nb(int M) { return M == 1 ? 16 : (M == 2 ? 32 : (M <= 4 ? 64 : 128)); }   // operand columns: 16 planes per token slot
 inline uint32_t batch_image_stage_bytes(int nb) { return (uint32_t)nb * 128u + kBatchSfBytes; }
 inline uint32_t batch_slot_bytes(int nb) { return kBatchCodesBytes + kBatchSfBytes + batch_image_stage_bytes(nb); }
 inline size_t batch_partials_bytes(int grid, int nb) { return (size_t)grid * 2u * (size_t)(nb / 16) * 128u * 4u; }
 
-// accumulator slots in tensor memory and the columns to allocate (a power of two >= slots * nb + 32 scale columns)
-inline int batch_acc_slots(int nb) { return nb <= 32 ? 4 : 3; }
-inline int batch_tmem_cols(int nb) {
-    const int need = batch_acc_slots(nb) * nb + 32;
+// accumulator slots in tensor memory (at most 4; the SM's 512 columns are shared by the CTAs on it, and 32 columns go
+// to the scale factors) and the columns to allocate (a power of two >= slots * nb + 32)
+inline int batch_acc_slots(int nb, int ctas_per_sm) {
+    const int a = (512 / ctas_per_sm - 32) / nb;
+    return a < 1 ? 0 : (a > 4 ? 4 : a);
+}
+inline int batch_tmem_cols(int nb, int ctas_per_sm) {
+    const int need = batch_acc_slots(nb, ctas_per_sm) * nb + 32;
     int cols = 32;
     while (cols < need) cols *= 2;
     return cols;
@@ -83,7 +87,7 @@ struct BatchTable {
     uint8_t *ws;
     int32_t ndesc, nimg, M;
     int32_t units, tasks;
-    int32_t ring, tmem_cols;
+    int32_t ring, tmem_cols, acc_slots;
     int32_t fault_unit;          // test hook: the producer skips this unit's weight copy (-1: none)
     uint32_t wait_us;            // limit of every wait inside the kernel
     uint32_t partials_offset;    // bytes from the workspace base

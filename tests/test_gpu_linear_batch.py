@@ -3,7 +3,7 @@
 Plain layers: |y - y64| <= 2e-3 * sum|x w^| + 1e-6 element by element (the bound of mxq_linear); epilogues: the bounds
 of tests/test_gpu_epilogues.py.  The cases cover one CTA per unit (tiny calls), tiles cut between two and three CTAs'
 ranges, ragged N, the half-full last stage (K % 256 == 128), shared and distinct X, every token count the persistent
-kernel takes (1..4) and the calls it hands on to the one-by-one path.
+kernel takes (1..8) and the calls it hands on to the one-by-one path.
 """
 import numpy as np
 import pytest
@@ -82,7 +82,7 @@ def sample_rows(n, seed, count=300):
                                      np.random.default_rng(seed).integers(0, n, count)])).astype(np.int64)
 
 
-@pytest.mark.parametrize("m", [1, 2, 3, 4])
+@pytest.mark.parametrize("m", [1, 2, 3, 4, 5, 7, 8])
 def test_small_ragged_layers(m):
     """Fewer units than SMs (every CTA owns one unit, every tile is summed across CTAs), ragged N, half-full last stage."""
     layers = [make_layer(3, 20, 203, 1408, m), make_layer(3, 21, 515, 2048, m), make_layer(3, 22, 128, 128, m),
@@ -108,7 +108,7 @@ def test_config2_draft_model_layer_set(m):
         check_layer(lay, "config2 layer %d M=%d" % (i, m))
 
 
-@pytest.mark.parametrize("m", [1, 2, 4])
+@pytest.mark.parametrize("m", [1, 2, 4, 8])
 def test_config3_7b_layer_set(m):
     """The benchmark's call: seven 7B-shaped layers in one launch, sampled rows of every layer against the oracle."""
     shapes = synth.LAYERS_7B
@@ -132,7 +132,7 @@ def test_config3_7b_layer_set(m):
         assert torch.equal(a, lay["out"])
 
 
-@pytest.mark.parametrize("m", [1, 3])
+@pytest.mark.parametrize("m", [1, 3, 6])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_epilogues(m, out_dtype):
     layers = [make_layer(3, 30, 1000, 1024, m, epilogue="residual", out_dtype=out_dtype),
@@ -195,9 +195,9 @@ def test_activations_that_cannot_be_rewritten_exactly():
     check_linear(lay_inf["out"][:1], y64[:1], a64[:1], "row without the infinity")
 
 
-@pytest.mark.parametrize("m,n,k", [(8, 515, 2048), (1, 203, 1440), (16, 300, 1024)])
+@pytest.mark.parametrize("m,n,k", [(9, 515, 2048), (1, 203, 1440), (16, 300, 1024)])
 def test_calls_the_persistent_kernel_does_not_cover(m, n, k):
-    """More than 4 token rows, or K not a multiple of 128: the layers run one by one, with the same results as the
+    """More than 8 token rows, or K not a multiple of 128: the layers run one by one, with the same results as the
     single-layer entry points."""
     layers = [make_layer(3, 60, n, k, m), make_layer(3, 61, 2 * 128, k, m, epilogue="swiglu"),
               make_layer(3, 62, n, k, m, epilogue="residual")]

@@ -3,9 +3,11 @@
 
 Workload (BASELINE.json config "7B-Llama-shaped decode layer set", M=1): one *step* is one
 draft-token pass over the linear projections of ``--layers`` (default 32) distinct 7B decoder
-layers -- q/k/v/o 4096x4096, gate/up 11008x4096, down 4096x11008 -- i.e. 7 mxq_linear calls per
-layer set, 224 per step, streaming 3.44 GB of MXFP4 weights (far larger than the 126 MB L2, so
-every step reads HBM).  Weights are synthetic (Student-t, seeded), direct-cast on the device by
+layers -- q/k/v/o 4096x4096, gate/up 11008x4096, down 4096x11008 -- i.e. 224 independent layer
+problems per step, streaming 3.44 GB of MXFP4 weights (far larger than the 126 MB L2, so every
+step reads HBM).  They run through mxq_linear_batch, ``--layers-per-call`` (default 4) layer
+sets = 28 layers per launch; the same step as one launch per layer set and as 224 separate
+mxq_linear calls is timed beside it (``extra.routes``).  Weights are synthetic (Student-t, seeded), direct-cast on the device by
 mxq_quantize before timing; the offline cast and the greedy-accept step are timed separately and
 reported under "extra".
 
@@ -36,8 +38,11 @@ UNIT = "GB/s"
 HBM_DATASHEET_GBS = 8000.0
 
 
-# DRAM bytes (read + write) over algorithmic bytes of one mxq_linear launch, from the committed profiler summary of the
-# 11008x4096 M=1 launch (profiles/mxq_linear_fp4_m1_11008x4096_full.md): 24.034816 MB / 23.957504 MB
+# DRAM bytes (read + write) over algorithmic bytes of one launch, from the committed profiler summaries:
+#   mxq_linear_batch, four 7B layer sets at M=1 (profiles/mxq_linear_batch_m1_4x7B_layer_sets_full.md):
+#     433.47 MB read + 5.92 MB written against 431.01 MB algorithmic
+#   one mxq_linear call, 11008x4096 at M=1 (profiles/mxq_linear_fp4_m1_11008x4096_full.md): 24.034816 MB / 23.957504 MB
+DRAM_OVER_ALGORITHMIC_BATCH = (433.469184 + 5.915264) / 431.011840
 DRAM_OVER_ALGORITHMIC = 24.034816 / 23.957504
 
 
@@ -137,15 +142,25 @@ def build_layers(mxq, n_layers: int, shapes, device):
 class LinearPass:
     """One pass over a list of quantised matrices at M token rows, replayed from a CUDA graph."""
 
-    def __init__(self, mxq, mats, m: int, device, seed: int, use_graph: bool = True):
+    def __init__(self, mxq, mats, m: int, device, seed: int, use_graph: bool = True, per_call: int = 0):
+        """per_call = 0: one mxq_linear call per matrix; > 0: mxq_linear_batch, that many matrices per call."""
         self.mxq, self.mats, self.m = mxq, mats, m
         ks = sorted({k for _, _, k, _, _ in mats})
         self.x = {k: synth.normal_bf16((m, k), 1.0, seed + k, device) for k in ks}
         self.y = [torch.empty((m, n), dtype=torch.float32, device=device) for _, n, _, _, _ in mats]
-        ws_bytes = max([mxq.mxq_linear_workspace_bytes(m, n, k) for _, n, k, _, _ in mats] + [16])
-        self.ws = mxq.new_workspace(ws_bytes, device)
         self.bytes = sum(algorithmic_bytes(m, n, k) for _, n, k, _, _ in mats)
-        self.launches = len(mats)
+        self.batches = None
+        if per_call > 0:
+            self.batches = [mxq.LinearBatch([dict(x=self.x[k], codes=c, scales=s, out=y)
+                                             for (_, n, k, c, s), y in zip(mats[i:i + per_call], self.y[i:i + per_call])])
+                            for i in range(0, len(mats), per_call)]
+            self.ws = mxq.new_workspace(max(b.workspace_bytes() for b in self.batches), device)
+            self.launches = len(self.batches)
+            self.info = self.batches[0].info()
+        else:
+            ws_bytes = max([mxq.mxq_linear_workspace_bytes(m, n, k) for _, n, k, _, _ in mats] + [16])
+            self.ws = mxq.new_workspace(ws_bytes, device)
+            self.launches = len(mats)
         self.graph = None
         self.stream = torch.cuda.Stream(device=device)
         self.stream.wait_stream(torch.cuda.current_stream(device))   # the inputs were produced on the current stream
@@ -159,6 +174,10 @@ class LinearPass:
                 self.graph = g
 
     def enqueue(self):
+        if self.batches is not None:
+            for b in self.batches:
+                b.run(self.ws)
+            return
         for (_, n, k, codes, scales), y in zip(self.mats, self.y):
             self.mxq.mxq_linear(self.x[k], codes, scales, out=y, workspace=self.ws)
 
@@ -208,6 +227,47 @@ def time_e2e(mxq, mats, m: int, steps: int, warmup: int, device):
     def one():
         for (_, n, k, codes, scales), yh_i, ys_i in zip(mats, yh, ys):
             mxq.mxq_linear_host(xh[k], codes, scales, yh_i, xs[k], ys_i, workspace=ws, stream=stream)
+
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            one()
+        stream.synchronize()
+        replicas.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        e0.record(stream)
+        for _ in range(steps):
+            one()
+        e1.record(stream)
+        stream.synchronize()
+        wall = time.perf_counter() - t0
+        replicas.barrier()
+    return max(e0.elapsed_time(e1) * 1e-3, 0.0), wall, h2d, d2h
+
+
+def time_e2e_batch(mxq, mats, m: int, per_call: int, steps: int, warmup: int, device):
+    """The same pass through mxq_linear_batch with the activations and the results in pinned HOST memory: the kernel
+    reads every layer's X across the bus itself and stores Y straight into host memory, inside the timed region.
+    Every layer of a call has a host buffer of its own (the library shares the rewriting of X only between layers
+    that pass the same pointer), so each layer's activations cross the bus, as with one call per layer."""
+    xh = [synth.normal_bf16((m, k), 1.0, 77 + i).pin_memory() for i, (_, _, k, _, _) in enumerate(mats[:per_call])]
+    yh = [torch.empty((m, n), dtype=torch.float32).pin_memory() for _, n, _, _, _ in mats]
+    batches = []
+    for i in range(0, len(mats), per_call):
+        lays = []
+        for j, ((_, n, k, c, s_), y) in enumerate(zip(mats[i:i + per_call], yh[i:i + per_call])):
+            assert xh[j].shape[1] == k   # every call holds the same sequence of shapes
+            lays.append(dict(x=xh[j], codes=c, scales=s_, out=y))
+        batches.append(mxq.LinearBatch(lays))
+    ws = mxq.new_workspace(max(b.workspace_bytes() for b in batches), device)
+    stream = torch.cuda.Stream(device=device)
+    stream.wait_stream(torch.cuda.current_stream(device))
+    h2d = sum(2 * m * k for _, _, k, _, _ in mats)
+    d2h = sum(4 * m * n for _, n, _, _, _ in mats)
+
+    def one():
+        for b in batches:
+            b.run(ws, stream)
 
     with torch.cuda.stream(stream):
         for _ in range(warmup):
@@ -324,7 +384,10 @@ def run_ours(args):
     m = args.m
     monitor = ClockMonitor(local_rank)
 
-    main = LinearPass(mxq, mats, m, device, seed=31, use_graph=not args.no_graph)
+    per_call = len(shapes) * max(1, min(args.layers_per_call, args.layers))   # layers (matrices) per mxq_linear_batch call
+    if args.route == "separate" or m > 8:
+        per_call = 0
+    main = LinearPass(mxq, mats, m, device, seed=31, use_graph=not args.no_graph, per_call=per_call)
     secs = main.time(args.steps, args.warmup, monitor)
     secs_max = replicas.max_over_ranks(secs, device)
     bytes_step = main.bytes
@@ -333,21 +396,59 @@ def run_ours(args):
     per_launch_s = secs / (args.steps * main.launches)
     achieved = bytes_step / main.launches / per_launch_s / 1e9
     peaks, peak_kind = measured_peaks()
+    route_text = ("mxq_linear_batch, %d layer set(s) = %d layers per launch" % (per_call // len(shapes), per_call)) if per_call \
+        else "one mxq_linear call per layer"
 
     # end to end with host buffers
     e2e_steps = max(3, min(args.steps, 50))
-    e2e_dev, e2e_wall, h2d, d2h = time_e2e(mxq, mats, m, e2e_steps, 3, device)
+    if per_call:
+        e2e_dev, e2e_wall, h2d, d2h = time_e2e_batch(mxq, mats, m, per_call, e2e_steps, 3, device)
+    else:
+        e2e_dev, e2e_wall, h2d, d2h = time_e2e(mxq, mats, m, e2e_steps, 3, device)
     e2e_secs = replicas.max_over_ranks(max(e2e_dev, e2e_wall), device)
     e2e_value = replicas.sum_over_ranks(bytes_step * e2e_steps, device) / e2e_secs / 1e9
 
     extra = {}
     if rank == 0 and not args.quick:
-        # the verify-side pass (M=8) over the same layers
-        p8 = LinearPass(mxq, mats, 8, device, seed=32, use_graph=not args.no_graph)
-        s8 = p8.time(max(3, args.steps // 2), 3)
-        extra["m8"] = {"gbs": p8.bytes * max(3, args.steps // 2) / s8 / 1e9,
-                       "us_per_layer_set": s8 / max(3, args.steps // 2) / args.layers * 1e6}
+        # the same step through the other routes: one launch per layer set, and one mxq_linear call per layer
+        routes = {}
+        n7 = len(shapes)
+        st_r = max(3, min(args.steps, 40))
+        for name, pc in (("batch_%d_layer_sets_per_call" % max(1, min(args.layers_per_call, args.layers)), per_call),
+                         ("batch_1_layer_set_per_call", n7), ("separate_calls", 0)):
+            if pc == per_call:
+                routes[name] = {"us_per_layer_set": ms_per_step * 1e3 / args.layers, "gbs": value, "launches_per_step": main.launches,
+                                "frac_of_peak": value / peaks["hbm_gbs"], "headline": True}
+                continue
+            if m > 8 and pc:
+                continue
+            pr = LinearPass(mxq, mats, m, device, seed=31, use_graph=not args.no_graph, per_call=pc)
+            sr = pr.time(st_r, 3)
+            routes[name] = {"us_per_layer_set": sr / st_r / args.layers * 1e6, "gbs": pr.bytes * st_r / sr / 1e9,
+                            "launches_per_step": pr.launches, "frac_of_peak": pr.bytes * st_r / sr / 1e9 / peaks["hbm_gbs"]}
+            del pr
+        extra["routes"] = routes
+        # the verify-side pass (M=8) over the same layers, through the same route and as separate calls
+        st8 = max(3, args.steps // 2)
+        p8 = LinearPass(mxq, mats, 8, device, seed=32, use_graph=not args.no_graph, per_call=per_call)
+        s8 = p8.time(st8, 3)
+        extra["m8"] = {"gbs": p8.bytes * st8 / s8 / 1e9, "us_per_layer_set": s8 / st8 / args.layers * 1e6,
+                       "route": "batch" if per_call else "separate", "launches_per_step": p8.launches}
         del p8
+        p8 = LinearPass(mxq, mats, 8, device, seed=32, use_graph=not args.no_graph)
+        s8 = p8.time(st8, 3)
+        extra["m8"]["separate_calls_us_per_layer_set"] = s8 / st8 / args.layers * 1e6
+        del p8
+        # and the token counts between (verifying 1..7 speculated tokens)
+        mrows = {}
+        for mm in (2, 3, 4, 5, 6):
+            if not per_call:
+                break
+            pm = LinearPass(mxq, mats, mm, device, seed=35, use_graph=not args.no_graph, per_call=per_call)
+            sm_ = pm.time(5, 3)
+            mrows["m%d" % mm] = {"us_per_layer_set": sm_ / 5 / args.layers * 1e6, "gbs": pm.bytes * 5 / sm_ / 1e9}
+            del pm
+        extra["m8"]["other_token_counts"] = mrows
         # per-shape, one matrix at a time, rotating over the layers (each pass > L2)
         per_shape = {}
         for name, n, k in [("4096x4096", 4096, 4096), ("11008x4096", 11008, 4096), ("4096x11008", 4096, 11008)]:
@@ -623,8 +724,9 @@ def run_ours(args):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": "7B decode layer set (q,k,v,o 4096x4096; gate,up 11008x4096; down 4096x11008), "
-                               "M=%d, %d distinct layers per step" % (m, args.layers),
-                   "M": m, "layers": args.layers, "calls_per_step": main.launches, "bytes_per_step": bytes_step,
+                               "M=%d, %d distinct layer sets (%d independent layers) per step, run as: %s"
+                               % (m, args.layers, len(mats), route_text),
+                   "M": m, "layers": args.layers, "route": route_text, "calls_per_step": main.launches, "bytes_per_step": bytes_step,
                    "y_dtype": "f32", "l2": "inputs larger than L2 (%.2f GB of weights per step)" % (bytes_step / 1e9),
                    "cuda_graph": not args.no_graph, "multi_gpu": "replicas only"},
         "us_per_layer_set": ms_per_step * 1e3 / args.layers,
@@ -634,11 +736,14 @@ def run_ours(args):
                 "steps": e2e_steps},
         "gpu_launches": main.launches * args.steps,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "traffic": DRAM_OVER_ALGORITHMIC * bytes_step / main.launches,
-                     "traffic_kind": "dram read+write bytes of one profiler capture of the 11008x4096 launch "
-                                     "(24.03 MB against 23.96 MB algorithmic), scaled to the average launch",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": (DRAM_OVER_ALGORITHMIC_BATCH if per_call else DRAM_OVER_ALGORITHMIC) * bytes_step / main.launches,
+                     "traffic_kind": ("dram read+write bytes of a profiler capture of one mxq_linear_batch launch of four 7B layer sets "
+                                      "(439.4 MB against 431.0 MB algorithmic), scaled to this launch's bytes") if per_call else
+                                     ("dram read+write bytes of one profiler capture of the 11008x4096 launch "
+                                      "(24.03 MB against 23.96 MB algorithmic), scaled to the average launch"),
                      "peak_kind": "of " + peak_kind,
-                     "kernel": "mxq_linear M=%d" % m, "bytes_per_launch": bytes_step / main.launches},
+                     "kernel": ("linear_batch_kernel" if per_call else "linear_fp4_kernel") + " M=%d" % m,
+                     "bytes_per_launch": bytes_step / main.launches},
         "cpu_baseline": cpu,
         "extra": extra,
     }
@@ -661,6 +766,8 @@ def run_case(args):
     case = args.case.lower()
     if case.split(":")[0] in ("quantize", "accept", "bf16", "swiglu", "residual"):
         return run_case_other(mxq, case, args.steps, device)
+    if case.split(":")[0] == "batch":
+        return run_case_batch(mxq, case, args.steps, device)
     n, k, m = (int(v) for v in case.split("x"))
     nbytes = algorithmic_bytes(m, n, k)
     copies = max(2, min(8, int(200e6 // nbytes) + 1))
@@ -682,6 +789,44 @@ def run_case(args):
     us = e0.elapsed_time(e1) * 1e3 / args.steps
     print(json.dumps({"case": args.case, "kernel": mxq.mxq_linear_plan_info(m, n, k)["kernel"], "launches": args.steps,
                       "us_per_call": us, "gbs": nbytes / us / 1e3, "bytes_per_call": nbytes,
+                      "device_status": mxq.mxq_linear_device_status()}))
+
+
+def run_case_batch(mxq, case: str, steps: int, device):
+    """--case batch:LxM : mxq_linear_batch calls of L 7B layer sets (7 L layers per launch) at M token rows, launched
+    `steps` times over distinct weights (together larger than L2): the small case profiler captures of the persistent
+    kernel run on."""
+    lsets, m = (int(v) for v in case.split(":")[1].split("x"))
+    copies = max(2, 300 // (108 * lsets) + 1)
+    gen = torch.Generator(device=device).manual_seed(7)
+    x = {k: synth.normal_bf16((m, k), 1.0, 3 + k, device) for k in (4096, 11008)}
+    batches, nbytes = [], 0
+    for _ in range(copies):
+        lays = []
+        for _ in range(lsets):
+            for _, n, k in synth.LAYERS_7B:
+                lays.append(dict(x=x[k], codes=torch.randint(0, 256, (n, k // 2), dtype=torch.uint8, device=device, generator=gen),
+                                 scales=torch.randint(110, 126, (n, k // 32), dtype=torch.uint8, device=device, generator=gen),
+                                 out=torch.empty((m, n), dtype=torch.float32, device=device)))
+        batches.append(mxq.LinearBatch(lays))
+        nbytes = sum(algorithmic_bytes(m, d["codes"].shape[0], d["x"].shape[1]) for d in lays)
+    ws = mxq.new_workspace(batches[0].workspace_bytes(), device)
+    batches[0].run(ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        batches[i % copies].run(ws)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / steps
+
+    def all_copies():
+        for b in batches:
+            b.run(ws)
+    graph_us = time_graph(all_copies, 10) / copies * 1e6
+    print(json.dumps({"case": case, "launches": steps, "us_per_call_from_python": us, "us_per_call": graph_us,
+                      "gbs": nbytes / graph_us / 1e3, "bytes_per_call": nbytes, "layout": batches[0].info(),
                       "device_status": mxq.mxq_linear_device_status()}))
 
 
@@ -828,6 +973,9 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--layers", type=int, default=32, help="distinct 7B layer sets per step")
     ap.add_argument("--m", type=int, default=1, help="token rows (1 = draft step)")
+    ap.add_argument("--route", choices=["batch", "separate"], default="batch",
+                    help="batch: mxq_linear_batch, --layers-per-call layer sets per launch; separate: one mxq_linear call per layer")
+    ap.add_argument("--layers-per-call", type=int, default=4, help="layer sets (7 layers each) per mxq_linear_batch call, 1..4")
     ap.add_argument("--no-graph", action="store_true", help="launch from Python instead of replaying a CUDA graph")
     ap.add_argument("--quick", action="store_true", help="skip the extra measurements")
     ap.add_argument("--no-cpu-baseline", action="store_true")

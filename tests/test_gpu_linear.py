@@ -287,3 +287,44 @@ def test_canaries_around_the_output_survive():
     mxq.mxq_linear(x, gc, gs, out=out)
     torch.cuda.synchronize()
     assert (buf[:32] == 12345.0).all() and (buf[32 + m * n:] == 12345.0).all()
+
+
+# ---- the launch plans bench.py times on the 13B layer shapes, the paper's 8192 x 8192 and the fused q/k/v matrix -------
+
+import functools
+
+
+@functools.lru_cache(maxsize=2)
+def _big_case(idx, n, k):
+    """Weights of one full-size matrix, cast by the oracle once and shared by the token counts (and kernel settings)."""
+    w = synth.bits_of(synth.weight(5 if k in (5120, 13824) else 3, idx, n, k))
+    codes, scales, _ = oracle.quantize(w)
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, n - 129, n - 128, n - 1],
+                                     np.random.default_rng(idx).integers(0, n, 160)])).astype(np.int64)
+    return codes, scales, rows, torch.from_numpy(codes).cuda(), torch.from_numpy(scales).cuda()
+
+
+def _run_big(idx, n, k, m):
+    codes, scales, rows, gc, gs = _big_case(idx, n, k)
+    x = synth.bits_of(synth.activations(5, idx, m, k))
+    y64, a64 = oracle.linear(x, codes, scales, rows=rows)
+    ws = mxq.new_workspace(mxq.mxq_linear_workspace_bytes(m, n, k))
+    y = mxq.mxq_linear(gpu_bf16(x), gc, gs, workspace=ws)
+    torch.cuda.synchronize()
+    check_linear(y[:, torch.as_tensor(rows, device="cuda")], y64, a64, "%dx%d M=%d" % (n, k, m))
+
+
+@pytest.mark.parametrize("m", list(range(1, 17)))
+@pytest.mark.parametrize("idx,n,k", [(0, 5120, 5120), (4, 13824, 5120), (6, 5120, 13824)])
+def test_config5_13b_layer_shapes_every_token_count(idx, n, k, m):
+    """Config 5: the three 13B layer shapes at every M in 1..16, in the launch plans the benchmark's curves time
+    (e.g. 13824 x 5120 as 540 CTAs on 592 slots); sampled rows spread over the first, the last and random tiles."""
+    _run_big(idx, n, k, m)
+
+
+@pytest.mark.parametrize("m", [1, 8])
+@pytest.mark.parametrize("idx,n,k", [(20, 8192, 8192), (21, 12288, 4096), (22, 22016, 4096)])
+def test_micro_benchmark_and_fused_projection_shapes(idx, n, k, m):
+    """8192 x 8192 (the paper's micro-benchmark shape) and the fused q/k/v (12288 x 4096) and gate/up (22016 x 4096)
+    matrices of the four-call layer, as bench.py times them."""
+    _run_big(idx, n, k, m)

@@ -132,6 +132,22 @@ def test_config3_7b_layer_set(m):
         assert torch.equal(a, lay["out"])
 
 
+@pytest.mark.parametrize("m", [1, 8])
+def test_config5_13b_layer_set(m):
+    """The seven 13B-shaped layers (hidden 5120, FFN 13824) in one call, sampled rows of every layer."""
+    shapes = [(5120, 5120)] * 4 + [(13824, 5120)] * 2 + [(5120, 13824)]
+    xs = {k: synth.bits_of(synth.activations(5, k, m, k)) for k in (5120, 13824)}
+    gx = {k: gpu_bf16(v) for k, v in xs.items()}
+    layers = []
+    for i, (n, k) in enumerate(shapes):
+        lay = make_layer(5, i, n, k, m, x=xs[k], rows=sample_rows(n, 50 + i, 200))
+        lay["x"] = gx[k]
+        layers.append(lay)
+    run_batch(layers)
+    for i, lay in enumerate(layers):
+        check_layer(lay, "13B layer %d M=%d" % (i, m))
+
+
 @pytest.mark.parametrize("m", [1, 3, 6])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_epilogues(m, out_dtype):
@@ -228,6 +244,42 @@ def test_thirty_two_layers_in_one_call():
     run_batch(layers)
     for i, lay in enumerate(layers):
         check_layer(lay, "layer %d of 32" % i)
+
+
+def test_a_bounded_wait_that_expires_is_reported_and_contained():
+    """Test hook: the weight copy of one unit of the call is left out, so the MMA warp of the CTA that owns it waits for
+    bytes that never arrive.  Its wait is bounded (20 ms here): the call must still complete, mxq_linear_device_status must
+    report the expired wait (bit 24), the tiles that CTA had not finished (and the tiles it shares with its neighbours)
+    must be NaN, and every other output must be within the bound.  Afterwards the library works as before."""
+    m = 1
+    layers = [make_layer(3, 100, 4096, 4096, m, rows=None), make_layer(3, 101, 1000, 2048, m)]
+    batch = mxq.LinearBatch(layers)
+    info = batch.info()
+    assert info["persistent"] == 1
+    ws = mxq.new_workspace(batch.workspace_bytes())
+    unit = info["units"] // 3            # somewhere inside the first layer
+    mxq.mxq_debug_batch_fault(unit, 20000)
+    batch.run(ws)
+    torch.cuda.synchronize()             # returns: nothing hangs
+    status = mxq.mxq_linear_device_status()
+    assert status & (1 << 24), "the expired wait was not reported (status %#x)" % status
+    y64, a64 = oracle.linear(layers[0]["_x"], layers[0]["_codes"], layers[0]["_scales"])
+    got = values(layers[0]["out"])
+    bad = np.isnan(got)
+    ks, tile_of_unit = 4096 // 256, unit // (4096 // 256)
+    assert bad[0, tile_of_unit * 128:(tile_of_unit + 1) * 128].all(), "the tile whose data never arrived must be NaN"
+    per_cta = -(-info["units"] // info["grid"])
+    assert bad.sum() <= 128 * (per_cta // ks + 3), "more than one CTA's tiles were lost: %d outputs" % bad.sum()
+    ok = ~bad
+    assert (np.abs(got - y64)[ok] <= (REL * a64 + ABS)[ok]).all()
+    check_layer(layers[1], "the layer after the lost tiles") if not np.isnan(values(layers[1]["out"])).any() else None
+    # a fresh workspace (the counters of the failed call are not to be trusted) and the same call again: all good
+    ws2 = mxq.new_workspace(batch.workspace_bytes())
+    batch.run(ws2)
+    torch.cuda.synchronize()
+    assert mxq.mxq_linear_device_status() == 0
+    for i, lay in enumerate(layers):
+        check_layer(lay, "after the fault, layer %d" % i)
 
 
 def test_argument_errors():

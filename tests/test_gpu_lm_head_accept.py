@@ -92,6 +92,14 @@ def test_full_vocabulary_sizes(r, t, v):
         assert int(g[0]) == 0 and int(nxt[0]) == int(tok[0])
 
 
+@pytest.mark.parametrize("r,t,v", [(1, 0, 32000), (9, 8, 32000), (16, 15, 32000), (1, 0, 128256), (12, 11, 128256)])
+def test_full_vocabulary_sizes_against_the_oracle(r, t, v):
+    """The same launch configurations (at 12 rows on 128256 x 4096 the call runs unfused: plain layer, argmax of every
+    row, walk over the draft) against the ORACLE's FP64 logits: every token the kernel picks must lie within the layer's
+    tolerance of the row's FP64 maximum, and the accept length / next token must follow from those tokens exactly."""
+    run(r, v, 4096, t, seed=40 + r, accept_upto=t // 2)
+
+
 def test_workspace_is_left_reusable_and_ties_go_to_the_lowest_index():
     v, k, r = 384, 256, 3
     # identical weight rows: every logit of a row of X is the same number -> token 0 everywhere

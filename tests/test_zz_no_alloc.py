@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2503_13565_b200 as mxq
 from paper_2503_13565_b200 import binding, synth
 
@@ -29,6 +30,11 @@ def test_static_variant_matches_the_workspace_variant_on_two_calls_in_a_row():
         torch.cuda.synchronize()
         assert torch.equal(got_len, want_len) and torch.equal(got_next, want_next)   # integers: no tolerance
         assert np.array_equal(got_len.cpu().numpy(), p.cpu().numpy())               # and they are the planted answer
+        # and both outputs are what the oracle computes from the same logits (BF16 logits go over as bit patterns)
+        lg = logits.cpu()
+        lg_np = lg.numpy() if dtype == torch.float32 else synth.bits_of(lg)
+        o_len, o_next = oracle.greedy_accept(lg_np, draft.cpu().numpy())
+        assert np.array_equal(got_len.cpu().numpy(), o_len) and np.array_equal(got_next.cpu().numpy(), o_next)
     # same shape again right away: the array holds the previous call's partial results and must not mind
     logits, draft, _, p = synth.accept_trials(250, 16, 17, 32000, seed=903, device="cuda")
     want_len, want_next = mxq.mxq_greedy_accept(logits, draft)

@@ -706,8 +706,27 @@ def run_ours(args):
             for w_ in ws_:
                 mxq.mxq_quantize(w_, codes, scales)
         tq = time_graph(q, 10) / 4
-        extra["quantize"] = {"gbs": 11008 * 4096 * 2.53125 / tq / 1e9, "us_per_call": tq * 1e6, "shape": "11008x4096"}
+        extra["quantize"] = {"gbs": 11008 * 4096 * 2.53125 / tq / 1e9, "us_per_call": tq * 1e6, "shape": "11008x4096",
+                             "frac_of_peak": 11008 * 4096 * 2.53125 / tq / 1e9 / peaks["hbm_gbs"]}
         del w, ws_
+        # config 5: the direct cast of all 40 layers of a 13B-shaped model (12.69 G weights, 25.4 GB of BF16 in, 6.7 GB
+        # out), every matrix resident, one replayed graph of the 280 casts
+        try:
+            shapes13 = [(n_, k_) for _, n_, k_ in synth.LAYERS_13B]
+            w13 = [synth.weight(5, 100 + li * len(shapes13) + j, n_, k_, device=device) for li in range(40) for j, (n_, k_) in enumerate(shapes13)]
+            c13 = [torch.empty((w_.shape[0], w_.shape[1] // 2), dtype=torch.uint8, device=device) for w_ in w13]
+            s13 = [torch.empty((w_.shape[0], w_.shape[1] // 32), dtype=torch.uint8, device=device) for w_ in w13]
+
+            def q13():
+                for w_, c_, s_ in zip(w13, c13, s13):
+                    mxq.mxq_quantize(w_, c_, s_)
+            t13 = time_graph(q13, 3)
+            weights13 = sum(w_.numel() for w_ in w13)
+            extra["quantize_13b"] = {"ms_per_sweep": t13 * 1e3, "weights": weights13, "gbs": weights13 * 2.53125 / t13 / 1e9,
+                                     "frac_of_peak": weights13 * 2.53125 / t13 / 1e9 / peaks["hbm_gbs"], "matrices": len(w13)}
+            del w13, c13, s13
+        except torch.OutOfMemoryError as e:   # (a GPU with less memory than the 32 GB this leg holds)
+            extra["quantize_13b"] = {"skipped": str(e)[:80]}
         # greedy accept: 250 sequences x 17 rows x 32000 logits (FP32), one call
         lg, draft, _, _ = synth.accept_trials(250, 16, 17, 32000, seed=1, device=device)
         ws2 = mxq.new_workspace(mxq.mxq_accept_workspace_bytes(250, 17, 32000), device)

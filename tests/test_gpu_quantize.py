@@ -120,3 +120,31 @@ def test_quantize_then_dequantize_matches_oracle_values():
     got = mxq.mxq_dequantize(gc, gs).float().cpu().numpy().astype(np.float64)
     oc, os_, _ = oracle.quantize(bits)
     assert np.array_equal(got, oracle.dequantize(oc, os_))
+
+
+def test_config5_direct_cast_of_all_forty_13b_layers():
+    """Config 5 at scale: the 40 x 7 weight matrices of a 13B-shaped model (12.69 G weights: q, k, v, o 5120 x 5120;
+    gate, up 13824 x 5120; down 5120 x 13824), Student-t with zeroed blocks, blocks pushed into the BF16 subnormals
+    and the hand blocks planted, drawn on the GPU from per-matrix seeds.  Every matrix is cast by mxq_quantize and by
+    the oracle from the same bits; codes, scales and the non-finite counter must agree byte for byte, layer by layer.
+    (One block per layer is overwritten with an Inf and a NaN here, so that the counter is exercised at scale too.)"""
+    shapes = [(n, k) for _, n, k in synth.LAYERS_13B]
+    total = 0
+    for layer in range(40):
+        for j, (n, k) in enumerate(shapes):
+            w = synth.weight(5, 100 + layer * len(shapes) + j, n, k, device="cuda")
+            if j == layer % len(shapes):
+                blk = w.view(-1, 32)
+                blk[(layer * 7919 + 13) % blk.shape[0], 3] = float("inf")
+                blk[(layer * 104729 + 5) % blk.shape[0], 31] = float("nan")
+            cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+            gc, gs = mxq.mxq_quantize(w, nonfinite_blocks=cnt)
+            bits = synth.bits_of(w)
+            oc, os_, obad = oracle.quantize(bits)
+            torch.cuda.synchronize()
+            assert np.array_equal(os_, to_np_u8(gs)), "scales differ in layer %d matrix %d" % (layer, j)
+            assert np.array_equal(oc, to_np_u8(gc)), "codes differ in layer %d matrix %d" % (layer, j)
+            assert obad == int(cnt.item()), "non-finite counter differs in layer %d matrix %d" % (layer, j)
+            total += n * k
+            del w, gc, gs, bits, oc, os_
+    assert total == 40 * 317194240

@@ -65,3 +65,52 @@ def test_on_step_sees_every_pass():
     seen = []
     specdec.simulate(2, [3], lambda lvl, k: 1, tokens=10, on_step=lambda lvl, rows: seen.append((lvl, rows)))
     assert seen[:4] == [(1, 1), (1, 1), (1, 1), (0, 4)] and len(seen) == 5 * 4
+
+
+class _TableModel:
+    """A deterministic stand-in: the next token is a fixed function of (token, position); `wrong_every` makes the model
+    disagree with the reference function at some positions, as a draft would."""
+
+    def __init__(self, v, salt, wrong_every=0):
+        self.v, self.salt, self.wrong_every = v, salt, wrong_every
+        self.passes = 0
+
+    def choice(self, tok, pos):
+        t = (tok * 31 + pos * 17 + 7) % self.v
+        if self.wrong_every and (tok + pos + self.salt) % self.wrong_every == 0:
+            t = (t + 1) % self.v
+        return t
+
+    def next(self, cur, pos):
+        self.passes += 1
+        return self.choice(cur, pos)
+
+    def verify(self, cur, pos, proposals):
+        self.passes += 1
+        rows = [cur] + list(proposals)
+        mine = [self.choice(t, pos + j) for j, t in enumerate(rows)]
+        g = 0
+        while g < len(proposals) and proposals[g] == mine[g]:
+            g += 1
+        return g, mine[g]
+
+
+@pytest.mark.parametrize("levels,n", [(1, []), (2, [4]), (2, [1]), (3, [4, 3]), (3, [8, 2])])
+def test_decode_reproduces_the_targets_own_greedy_decoding(levels, n):
+    target = _TableModel(97, 0)
+    models = [target] + [_TableModel(97, 3 + i, wrong_every=3 + 2 * i) for i in range(levels - 1)]
+    out, tally = specdec.decode(models, n, first_token=5, tokens=300)
+    want, cur = [], 5
+    for pos in range(len(out)):
+        cur = target.choice(cur, pos)
+        want.append(cur)
+    assert out == want and len(out) >= 300
+    assert tally.steps == [m.passes for m in models]
+    for i in range(levels - 1):
+        assert tally.proposed[i] == tally.steps[i] * n[i] and 0 < tally.accepted[i] < tally.proposed[i]
+    if levels == 2:   # Eq. 1 at the observed acceptance, with a draft step S times cheaper than a target step
+        s = 4.0
+        alpha = tally.accepted[0] / tally.proposed[0]
+        produced = tally.accepted[0] + tally.steps[0]
+        assert produced == len(out)
+        assert produced / tally.time([1.0, 1.0 / s]) == pytest.approx(specdec.eq1_speedup(alpha, n[0], s), rel=1e-12)

@@ -156,7 +156,7 @@ int mxq_linear_plan_info(int kernel, int M, int64_t N, int64_t K, int32_t *info)
  * bit 2: the accumulator never completed, bit 3: a prefetched stage never landed; bits 0-3 for
  * MXQ_KERNEL_UMMA, bits 8-11 the same for MXQ_KERNEL_FP4, bits 16-20 for mxq_linear_bf16; bits 24-27 for
  * mxq_linear_batch: data of a stage never arrived, a ring slot was never released, an accumulator never completed,
- * the rewritten token rows never became ready).  0 in normal
+ * the rewritten token rows never became ready; bit 28 for MXQ_KERNEL_MMA: the wait for a reduction slot).  0 in normal
  * operation; a non-zero word means the affected output tiles were written as NaN.  Synchronises with
  * the device (a blocking copy), so call it outside the hot loop. */
 int mxq_linear_device_status(uint32_t *status_host);

@@ -74,6 +74,7 @@ bool linear_fp4_plan(int M, int64_t N, int64_t K, Fp4Plan &plan, bool pow2_split
 cudaError_t linear_fp4_launch(const Fp4Plan &plan, const void *X, const uint8_t *codes, const uint8_t *scales,
                               void *Y, int y_dtype, cudaStream_t stream, const FusedAccept *fused = nullptr);
 int linear_fp4_take_status(uint32_t *out);
+int linear_mma_take_status(uint32_t *out);    // the mma.sync kernel (mxq_linear_mma.cu)
 int linear_batch_take_status(uint32_t *out);  // the persistent multi-layer kernel (mxq_linear_batch.cu)
 int linear_bf16_take_status(uint32_t *out);   // the BF16-weight comparison kernel (mxq_linear_bf16.cu)
 

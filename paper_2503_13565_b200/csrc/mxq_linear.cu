@@ -308,12 +308,18 @@ static bool lm_head_unfused(const mxq::Choice &c, int R, int64_t V) {
 
 size_t mxq_lm_head_accept_workspace_bytes(int R, int64_t V, int64_t K) {
     if (R < 1 || R > MXQ_MAX_M || !mxq::shape_ok(V, K)) return 0;
-    mxq::Choice c;
-    mxq::choose(mxq::kernel_ceiling(), R, V, K, nullptr, true, c, false, true);
-    size_t b = kFusedHeader + align256(mxq_linear_workspace_bytes(R, V, K));
-    if (lm_head_unfused(c, R, V))
-        b += align256((size_t)R * (size_t)V * 4u) + align256(mxq_accept_workspace_bytes(R, 1, V));
-    return b;
+    // The query does not know `codes`: a base that is 16-byte but not 32-byte aligned rules out the FP8-operand kernel
+    // and may send the call down the unfused path, which needs room for the logits.  The answer covers both.
+    size_t need = 0;
+    for (int variant = 0; variant < 2; ++variant) {
+        mxq::Choice c;
+        mxq::choose(mxq::kernel_ceiling(), R, V, K, variant ? reinterpret_cast<const uint8_t *>(uintptr_t(16)) : nullptr, true, c, false, true);
+        size_t b = kFusedHeader + align256(mxq_linear_workspace_bytes(R, V, K));
+        if (lm_head_unfused(c, R, V))
+            b += align256((size_t)R * (size_t)V * 4u) + align256(mxq_accept_workspace_bytes(R, 1, V));
+        if (b > need) need = b;
+    }
+    return need;
 }
 
 int mxq_lm_head_accept(const void *X_bf16, int R, const uint8_t *codes, const uint8_t *scales, int64_t V, int64_t K,
@@ -353,8 +359,6 @@ int mxq_lm_head_accept(const void *X_bf16, int R, const uint8_t *codes, const ui
     float *logits = reinterpret_cast<float *>(ws + kFusedHeader + lin_ws_bytes);
     void *acc_ws = ws + kFusedHeader + lin_ws_bytes + align256((size_t)R * (size_t)V * 4u);
     const size_t acc_ws_bytes = align256(mxq_accept_workspace_bytes(R, 1, V));
-    // (a `codes` that is not 32-byte aligned takes this path although the size query, which cannot know, may have
-    // answered for the fused one)
     if (workspace_bytes < kFusedHeader + lin_ws_bytes + align256((size_t)R * (size_t)V * 4u) + acc_ws_bytes) return MXQ_ERR_WORKSPACE;
     int32_t *minus_one = reinterpret_cast<int32_t *>(ws + 2176);   // [16]; the header's keys and ticket end at 2052
     int32_t *zeros_out = reinterpret_cast<int32_t *>(ws + 2304);   // [16] accept lengths of the argmax pass (all 0)

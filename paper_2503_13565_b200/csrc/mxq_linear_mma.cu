@@ -40,6 +40,8 @@ namespace mxq {
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
 // ---------------------------------------------------------------------------------------------
+__device__ unsigned int g_mma_status = 0;   // sticky: bit 0 the wait for a reduction slot gave up
+
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
@@ -387,20 +389,26 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
         // order and finishes the pair.  No CTA-wide barrier: the other warps move on to the next tile.
         const int tile_now = e.w & 0xFFFFF, w_now = e.w >> 20;
         const int rslot = seg_index % kRedSlots;
-        {   // the slot's previous pair (kRedSlots pairs ago) must have been summed.  The wait is bounded;
-            // if it ever gave up the result would be wrong, which the parity tests would show.
+        float poison = 0.f;
+        {   // the slot's previous pair (kRedSlots pairs ago) must have been summed.  The wait is bounded; if it
+            // gives up, a sticky status bit is set (mxq_linear_device_status, bit 28) and this warp's share of the
+            // tile goes out as NaN, so that the tile cannot pass for a result
             const int need = seg_index / kRedSlots;
             int spins = 0;
             while (*reinterpret_cast<volatile int *>(&s_gen[rslot]) < need && ++spins < (1 << 22)) __nanosleep(40);
+            if (spins >= (1 << 22)) {
+                poison = __uint_as_float(0x7FC00000u);
+                if (lane == 0) atomicOr(&g_mma_status, 1u);
+            }
         }
         float *mine = s_red + (rslot * kMmaWarps + warp) * kOut;
         if (exact_ok) {
 #pragma unroll
             for (int n = 0; n < NT8; ++n) {
-                mine[(8 * n + 2 * t) * kTileRows + g] = acc[n][0];
-                mine[(8 * n + 2 * t + 1) * kTileRows + g] = acc[n][1];
-                mine[(8 * n + 2 * t) * kTileRows + g + 8] = acc[n][2];
-                mine[(8 * n + 2 * t + 1) * kTileRows + g + 8] = acc[n][3];
+                mine[(8 * n + 2 * t) * kTileRows + g] = acc[n][0] + poison;
+                mine[(8 * n + 2 * t + 1) * kTileRows + g] = acc[n][1] + poison;
+                mine[(8 * n + 2 * t) * kTileRows + g + 8] = acc[n][2] + poison;
+                mine[(8 * n + 2 * t + 1) * kTileRows + g + 8] = acc[n][3] + poison;
                 acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
             }
         } else {
@@ -409,7 +417,7 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
             // tile is zero everywhere else, so the common sum below still applies
             const int bwid = (w_now == p.nwin - 1) ? p.bw_last : p.bw;
             const int64_t j0 = (int64_t)w_now * p.bw;
-            for (int i = lane; i < kOut; i += 32) mine[i] = 0.f;
+            for (int i = lane; i < kOut; i += 32) mine[i] = poison;
             __syncwarp();
             for (int half = 0; half < 2; ++half) {
                 const int64_t row = r0 + (int64_t)tile_now * kTileRows + warp + 8 * half;
@@ -573,6 +581,15 @@ cudaError_t linear_mma_launch(const LinearPlan &p, const void *X, const uint8_t 
     if (p.nt8 == 1) return p.nstage == 3 ? MXQ_LAUNCH(1, 3) : MXQ_LAUNCH(1, 2);
     return p.nstage == 3 ? MXQ_LAUNCH(2, 3) : MXQ_LAUNCH(2, 2);
 #undef MXQ_LAUNCH
+}
+
+// returns and clears this kernel's sticky status word (see mxq_linear_device_status)
+int linear_mma_take_status(uint32_t *out) {
+    unsigned int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_mma_status, sizeof v) != cudaSuccess) return MXQ_ERR_CUDA;
+    if (v != 0 && cudaMemcpyToSymbol(g_mma_status, &zero, sizeof zero) != cudaSuccess) return MXQ_ERR_CUDA;
+    *out = v;
+    return MXQ_OK;
 }
 
 }  // namespace mxq

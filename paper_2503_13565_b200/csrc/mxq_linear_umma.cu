@@ -823,7 +823,7 @@ extern "C" {
 #pragma GCC visibility push(default)
 int mxq_linear_device_status(uint32_t *status_host) {
     if (!status_host) return MXQ_ERR_NULL;
-    uint32_t v = 0, v4 = 0, vb = 0, vp = 0;
+    uint32_t v = 0, v4 = 0, vb = 0, vp = 0, vm = 0;
     int rc = mxq::linear_umma_take_status(&v);
     if (rc != MXQ_OK) return rc;
     rc = mxq::linear_fp4_take_status(&v4);
@@ -832,7 +832,9 @@ int mxq_linear_device_status(uint32_t *status_host) {
     if (rc != MXQ_OK) return rc;
     rc = mxq::linear_batch_take_status(&vp);
     if (rc != MXQ_OK) return rc;
-    *status_host = v | (v4 << 8) | (vb << 16) | (vp << 24);
+    rc = mxq::linear_mma_take_status(&vm);
+    if (rc != MXQ_OK) return rc;
+    *status_host = v | (v4 << 8) | (vb << 16) | (vp << 24) | (vm << 28);
     return MXQ_OK;
 }
 #pragma GCC visibility pop

@@ -118,3 +118,30 @@ def test_accept_tokens_variant():
         og, on = oracle.greedy_accept_tokens(draft.numpy(), ver.numpy())
         gg, nn = mxq.mxq_greedy_accept_tokens(draft.cuda(), ver.cuda())
         assert np.array_equal(gg.cpu().numpy(), og) and np.array_equal(nn.cpu().numpy(), on)
+
+
+def test_one_workspace_across_differently_shaped_calls_through_the_c_abi():
+    """The contract of mxq_accept_workspace_bytes: zero the first 4096 bytes once, then every call that completes leaves
+    them zero, so one workspace serves later calls of other shapes.  Raw C calls (no helper re-zeroes anything)."""
+    import ctypes
+
+    from paper_2503_13565_b200 import binding
+    L = binding.lib()
+    shapes = [(40, 16, 17, 32000, torch.float32), (3, 8, 9, 128256, torch.bfloat16), (250, 4, 4, 5000, torch.float32),
+              (40, 16, 17, 32000, torch.float32)]
+    need = max(mxq.mxq_accept_workspace_bytes(b, r, v) for b, t, r, v, _ in shapes)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda").fill_(0xAB)   # scratch part deliberately dirty
+    ws[:4096].zero_()                                                      # the one-time initialisation
+    st = torch.cuda.current_stream().cuda_stream
+    for i, (b, t, r, v, dtype) in enumerate(shapes):
+        logits, draft, _, p = synth.accept_trials(b, t, r, v, seed=300 + i, dtype=dtype, device="cuda")
+        g = torch.full((b,), -9, dtype=torch.int32, device="cuda")
+        nxt = torch.full((b,), -9, dtype=torch.int32, device="cuda")
+        rc = L.mxq_greedy_accept(logits.data_ptr(), 0 if dtype == torch.float32 else 1, b, r, v, draft.data_ptr(), t,
+                                 g.data_ptr(), nxt.data_ptr(), ws.data_ptr(), ws.numel(), ctypes.c_void_p(st))
+        assert rc == 0
+        torch.cuda.synchronize()
+        lg = logits.cpu()
+        og, on = oracle.greedy_accept(lg.numpy() if dtype == torch.float32 else synth.bits_of(lg), draft.cpu().numpy())
+        assert np.array_equal(g.cpu().numpy(), og) and np.array_equal(nxt.cpu().numpy(), on)
+        assert int(ws[:4096].to(torch.int64).sum()) == 0, "the counters were not left at zero"

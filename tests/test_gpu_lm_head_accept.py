@@ -114,6 +114,28 @@ def test_workspace_is_left_reusable_and_ties_go_to_the_lowest_index():
     assert int(ws[:2176].to(torch.int64).sum()) == 0   # keys and ticket are zero again
 
 
+@pytest.mark.parametrize("r,t", [(1, 0), (4, 3), (9, 8)])
+def test_codes_that_are_only_16_byte_aligned(r, t):
+    """`codes` 16 bytes into an allocation: the FP8-operand kernel (32-byte aligned bases only) is ruled out, and a
+    workspace of the size the query names must still be enough whichever path the call then takes."""
+    v, k = 3000, 1024
+    w = synth.bits_of(synth.weight(4, 9, v, k))
+    x = synth.bits_of(synth.activations(4, 9, r, k))
+    codes, scales, _ = oracle.quantize(w)
+    y64, tok, allowed = oracle_tokens(x, codes, scales)
+    raw = torch.empty(codes.size + 64, dtype=torch.uint8, device="cuda")
+    off = 16 if raw.data_ptr() % 32 == 0 else 32 - raw.data_ptr() % 32 + 16   # 16 mod 32
+    gc = raw[off:off + codes.size].view(v, k // 2)
+    gc.copy_(torch.from_numpy(codes))
+    assert gc.data_ptr() % 32 == 16
+    ws = mxq.new_workspace(mxq.mxq_lm_head_accept_workspace_bytes(r, v, k))
+    draft = torch.from_numpy(tok[:t].astype(np.int32)).cuda() if t else None
+    ver, g, nxt = mxq.mxq_lm_head_accept(gpu_bf16(x), gc, torch.from_numpy(scales).cuda(), draft, workspace=ws)
+    torch.cuda.synchronize()
+    for row in range(r):
+        assert int(ver[row]) in allowed[row]
+
+
 def test_nan_and_minus_inf_are_never_selected():
     v, k = 256, 128
     codes = np.zeros((v, k // 2), np.uint8)

@@ -592,17 +592,28 @@ def run_ours(args):
             mxq.mxq_linear_bf16(xs_[(r_, 4096)], th, out=lg_[r_][0])
             mxq.mxq_greedy_accept(lg_[r_], dr_[:, :max(r_ - 1, 1)], workspace=wsa_)
 
-        def draft_step():
+        def draft_step_separate():   # one mxq_linear call per layer
             for lay in dq:
                 for (c_, s_) in lay:
                     mxq.mxq_linear(xs_[(1, c_.shape[1] * 2)], c_, s_, out=yo_[(1, c_.shape[0])], workspace=self_ws)
+            mxq.mxq_lm_head_accept(xs_[(1, 4096)], dh[0], dh[1], None, workspace=wsf_)
+
+        # the draft's 28 layers in one mxq_linear_batch launch (here, as in the timed step above, the layers' inputs are
+        # fixed buffers: a real decoder's layers depend on one another, which bounds what a call may hold)
+        d_batch = mxq.LinearBatch([dict(x=xs_[(1, c_.shape[1] * 2)], codes=c_, scales=s_,
+                                        out=torch.empty((1, c_.shape[0]), dtype=torch.float32, device=device)) for lay in dq for (c_, s_) in lay])
+        d_ws = mxq.new_workspace(d_batch.workspace_bytes(), device)
+
+        def draft_step():
+            d_batch.run(d_ws)
             mxq.mxq_lm_head_accept(xs_[(1, 4096)], dh[0], dh[1], None, workspace=wsf_)
         self_ws = mxq.new_workspace(16, device)
         st_ = torch.cuda.Stream()
         st_.wait_stream(torch.cuda.current_stream())
         graphs = {}
         with torch.cuda.stream(st_):
-            for name_, fn_ in (("t1", lambda: target_step(1)), ("tv", lambda: target_step(n_draft + 1)), ("d", draft_step)):
+            for name_, fn_ in (("t1", lambda: target_step(1)), ("tv", lambda: target_step(n_draft + 1)), ("d", draft_step),
+                               ("ds", draft_step_separate)):
                 fn_()
                 st_.synchronize()
                 g_ = torch.cuda.CUDAGraph()
@@ -624,8 +635,10 @@ def run_ours(args):
             t_t1 = timed(graphs["t1"].replay, 20)
             t_tv = timed(graphs["tv"].replay, 20)
             t_d = timed(graphs["d"].replay, 20)
+            t_ds = timed(graphs["ds"].replay, 20)
             sd = {"layers": nl_, "draft_tokens_per_round": n_draft, "target_step_us": t_t1 * 1e6, "target_verify_us": t_tv * 1e6,
-                  "draft_step_us": t_d * 1e6, "S": t_t1 / t_d, "runs": {}}
+                  "draft_step_us": t_d * 1e6, "S": t_t1 / t_d, "draft_route": "mxq_linear_batch (28 layers in one launch) + mxq_lm_head_accept",
+                  "draft_step_one_call_per_layer_us": t_ds * 1e6, "S_one_call_per_layer": t_t1 / t_ds, "runs": {}}
             for p_ in (0.7, 0.9):
                 rng_ = _random.Random(1)
                 steps_ = []
@@ -658,16 +671,19 @@ def run_ours(args):
             wsfv = mxq.new_workspace(mxq.mxq_lm_head_accept_workspace_bytes(rv, 32000, 4096), device)
             drv = torch.zeros(n_tiny, dtype=torch.int32, device=device)
 
+            t_batch = mxq.LinearBatch([dict(x=xt_[c_.shape[1] * 2], codes=c_, scales=s_,
+                                            out=torch.empty((1, c_.shape[0]), dtype=torch.float32, device=device)) for lay in tq for (c_, s_) in lay])
+            t_ws = mxq.new_workspace(t_batch.workspace_bytes(), device)
+            v_batch = mxq.LinearBatch([dict(x=xv_[c_.shape[1] * 2], codes=c_, scales=s_,
+                                            out=torch.empty((rv, c_.shape[0]), dtype=torch.float32, device=device)) for lay in dq for (c_, s_) in lay])
+            v_ws = mxq.new_workspace(v_batch.workspace_bytes(), device)
+
             def tiny_step():
-                for lay in tq:
-                    for (c_, s_) in lay:
-                        mxq.mxq_linear(xt_[c_.shape[1] * 2], c_, s_, out=yt_[c_.shape[0]], workspace=self_ws)
+                t_batch.run(t_ws)
                 mxq.mxq_lm_head_accept(xt_[768], tqh[0], tqh[1], None, workspace=wsf_t)
 
             def draft_verify():   # the MXFP4 model checks the tiny draft's n_tiny tokens in one pass of n_tiny + 1 rows
-                for lay in dq:
-                    for (c_, s_) in lay:
-                        mxq.mxq_linear(xv_[c_.shape[1] * 2], c_, s_, out=yv_[c_.shape[0]], workspace=wsv)
+                v_batch.run(v_ws)
                 mxq.mxq_lm_head_accept(xv_[4096], dh[0], dh[1], drv, workspace=wsfv)
             for name_, fn_ in (("y", tiny_step), ("dv", draft_verify)):
                 fn_()

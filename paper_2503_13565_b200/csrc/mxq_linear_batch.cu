@@ -465,8 +465,14 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
         const int et = tid - 64;                          // 0..127
         const int row = ((warp & 3) << 5) + lane;         // accumulator row this thread may read (its warp's quarter)
 
-        // 1. this CTA's share of the rewriting of the token rows: task = 128 k of one token row of one image
-        for (int task = cta * 4 + ew; task < tb.tasks; task += 4 * G) {
+        // 1. the rewriting of the token rows: task = 128 k of one token row of one image.  Tasks are handed out by a counter
+        //    in the workspace, not by CTA index: every consumer waits for whole images, so a CTA that starts late (CTAs
+        //    start over several microseconds as the previous kernel's leave) must not be holding tasks.
+        for (;;) {
+            int task = 0;
+            if (lane == 0) task = (int)atomicAdd(hdr + kBatchWordTask, 1u);
+            task = __shfl_sync(0xffffffffu, task, 0);
+            if (task >= tb.tasks) break;
             int im = 0;
             while (im + 1 < tb.nimg && task >= tb.img[im + 1].task_base) ++im;
             const BatchImg &gi = tb.img[im];
@@ -478,12 +484,10 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
             const bool inexact = split_half_unit_to(raw, m, (uint32_t)kk & 255u, lane & 1, lane, SplitToGlobal{stage},
                                                     SplitToGlobal{stage + (uint32_t)NB * 128u});
             const bool bad = __any_sync(0xffffffffu, inexact);
-            fence_proxy_async_all();
-            __syncwarp();
+            __syncwarp();   // (orders the lanes' stores before lane 0's release; the readers order them against their bulk copies)
             if (lane == 0) {
                 if (bad) atomicOr(g_bad + im, 1u);
-                __threadfence();
-                atomicAdd(g_ready + im, 1u);
+                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(g_ready + im) : "memory");
             }
         }
 
@@ -668,6 +672,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                     g_ready[i] = 0u;
                     g_bad[i] = 0u;
                 }
+                hdr[kBatchWordTask] = 0u;
                 hdr[kBatchWordExit] = 0u;
             }
         }

@@ -28,11 +28,12 @@ constexpr int kBatchMaxGrid = 1024;      // CTAs (ticket counters in the workspa
 //      u32 ready[32]   split tasks delivered per token-operand image
 //      u32 bad[32]     an image holds a block that could not be rewritten exactly
 //      u32 exit        CTAs that have finished (word 64)
+//      u32 task        rewriting tasks handed out (word 65)
 //      u32 ticket[kBatchMaxGrid] at byte 512: contributors that have delivered their share of a tile split between CTAs
 // [kBatchHeaderBytes, ...) partial sums: [grid][2 (at the head / at the tail of the CTA's range)][token slots][128] floats
 // then the token-operand images, one per distinct X: [stage][operand rows NB x 128 bytes | 1024 bytes of scale atoms]
 constexpr size_t kBatchHeaderBytes = 8192;
-constexpr int kBatchWordReady = 0, kBatchWordBad = 32, kBatchWordExit = 64, kBatchWordTicket = 128;
+constexpr int kBatchWordReady = 0, kBatchWordBad = 32, kBatchWordExit = 64, kBatchWordTask = 65, kBatchWordTicket = 128;
 
 inline int batch_nb(int M) { return M == 1 ? 16 : (M == 2 ? 32 : (M <= 4 ? 64 : 128)); }   // operand columns: 16 planes per token slot
 inline uint32_t batch_image_stage_bytes(int nb) { return (uint32_t)nb * 128u + kBatchSfBytes; }

@@ -565,6 +565,21 @@ def run_ours(args):
             tf_ = time_graph(fused_pass, 10) / nlay
             wbytes = sum(n_ * k_ * 17 // 32 for n_, k_ in [(12288, 4096), (4096, 4096), (22016, 4096), (4096, 11008)])
             fl["m%d" % mm] = {"us_per_layer": tf_ * 1e6, "gbs": wbytes / tf_ / 1e9, "calls": 4, "weight_bytes": wbytes}
+            # the same layer, dependences included, as ONE mxq_linear_batch call of three groups:
+            # {q/k/v, o + residual} | {gate/up with SiLU(gate) * up} | {down + residual}
+            one = [mxq.LinearBatch([dict(x=h0, codes=wqkv[0], scales=wqkv[1], out=qkv),
+                                    dict(x=att, codes=wo[0], scales=wo[1], out=h1, epilogue="residual", residual=h0),
+                                    dict(x=h1, codes=wgu[0], scales=wgu[1], out=act, epilogue="swiglu", depends=True),
+                                    dict(x=act, codes=wd[0], scales=wd[1], out=h2, epilogue="residual", residual=h1, depends=True)])
+                   for (wqkv, wo, wgu, wd) in lay4]
+            ws1 = mxq.new_workspace(one[0].workspace_bytes(), device)
+
+            def one_call_pass():
+                for b_ in one:
+                    b_.run(ws1)
+            t1_ = time_graph(one_call_pass, 10) / nlay
+            fl["m%d" % mm]["one_call_three_groups_us_per_layer"] = t1_ * 1e6
+            fl["m%d" % mm]["one_call_three_groups_gbs"] = wbytes / t1_ / 1e9
         fl["status"] = mxq.mxq_linear_device_status()
         extra["fused_layer"] = fl
         del lay4

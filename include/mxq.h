@@ -292,13 +292,16 @@ int mxq_linear_swiglu(const void *X_bf16, int M, const uint8_t *codes, const uin
  *             epilogue MXQ_EPI_NONE      Y [M][N]   = X . w^T
  *                      MXQ_EPI_RESIDUAL  Y [M][N]   = residual + X . w^T   (residual [M][N] in Y's type; may be Y itself)
  *                      MXQ_EPI_SWIGLU    Y [M][N/2] = silu(g) * u, rows 2i / 2i+1 of W being gate / up row i
- *           The layers of one call are INDEPENDENT: none may read (as X or residual) what another one writes, since
- *           they run interleaved.  Layers that share an X pointer share its rewriting.  X, Y and residual may also be
+ *           Layers run interleaved, so by default none may read (as X or residual) what another layer of the call
+ *           writes.  A layer with flags = MXQ_BATCH_DEPENDS opens a new GROUP (at most MXQ_MAX_BATCH_GROUPS per call):
+ *           it and the layers after it start only when every layer before it in the array has been stored, and may
+ *           read those outputs (a BF16 Y as the next X, e.g. gate/up with MXQ_EPI_SWIGLU followed by down); the weight
+ *           stream runs on across the group boundary.  Within a group, layers that share an X pointer share its rewriting.  X, Y and residual may also be
  *           page-locked host memory that the GPU can address (cudaHostAlloc / cudaHostRegister): the kernel then reads
  *           the activations and writes the results across the bus itself.
  *   M       token rows, common to all layers of the call
  *   workspace  REQUIRED: device memory, 256-byte aligned, >= mxq_linear_batch_workspace_bytes(descs, count, M).  Zero
- *           its first 8192 bytes (counters) ONCE before the first use; every call that completes leaves them zero
+ *           its first 16384 bytes (counters) ONCE before the first use; every call that completes leaves them zero
  *           again; the rest needs no initialisation.  After a non-zero mxq_linear_device_status zero them again.  Calls
  *           in one stream may share a workspace; calls that may run concurrently need one each.
  * The persistent kernel covers M <= 4 with every K a multiple of 128; any other call runs its layers one after the
@@ -306,6 +309,8 @@ int mxq_linear_swiglu(const void *X_bf16, int M, const uint8_t *codes, const uin
  * bit-reproducible run to run and within mxq_linear's bound; the summation order differs from mxq_linear's.  Errors as
  * mxq_linear.  Bounded waits that give up are reported in bits 24-27 of mxq_linear_device_status. */
 #define MXQ_MAX_BATCH 32
+#define MXQ_MAX_BATCH_GROUPS 8
+#define MXQ_BATCH_DEPENDS 1 /* this layer and the ones after it may read what the layers before it in the array wrote */
 enum mxq_epilogue { MXQ_EPI_NONE = 0, MXQ_EPI_RESIDUAL = 1, MXQ_EPI_SWIGLU = 2 };
 typedef struct mxq_linear_desc {
     const void *X_bf16;
@@ -316,6 +321,8 @@ typedef struct mxq_linear_desc {
     int64_t N, K;
     int32_t y_dtype;      /* MXQ_F32 / MXQ_BF16 */
     int32_t epilogue;     /* mxq_epilogue */
+    int32_t flags;        /* 0, or MXQ_BATCH_DEPENDS */
+    int32_t reserved;     /* 0 */
 } mxq_linear_desc;
 size_t mxq_linear_batch_workspace_bytes(const mxq_linear_desc *descs, int count, int M);
 int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *workspace, size_t workspace_bytes,

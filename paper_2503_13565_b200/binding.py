@@ -423,7 +423,7 @@ def mxq_set_linear_layout(what, value: int) -> None:
 class _LinearDesc(ctypes.Structure):
     _fields_ = [("X_bf16", ctypes.c_void_p), ("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p),
                 ("Y", ctypes.c_void_p), ("residual", ctypes.c_void_p), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
-                ("y_dtype", ctypes.c_int32), ("epilogue", ctypes.c_int32)]
+                ("y_dtype", ctypes.c_int32), ("epilogue", ctypes.c_int32), ("flags", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 def _any_mem(t: torch.Tensor, dtype, what: str) -> int:
@@ -436,7 +436,8 @@ def _any_mem(t: torch.Tensor, dtype, what: str) -> int:
 class LinearBatch:
     """The descriptor array of one mxq_linear_batch call, marshalled once and reusable (the call itself is then a
     single C call).  ``layers``: dicts with x [M,K] BF16, codes, scales, out [M,N] (or [M,N/2] for "swiglu"), and
-    optionally epilogue ("none" | "residual" | "swiglu") and residual.  The tensors are kept alive by this object."""
+    optionally epilogue ("none" | "residual" | "swiglu"), residual, and depends=True for a layer that (with the ones after
+    it) reads what the layers before it write.  The tensors are kept alive by this object."""
 
     def __init__(self, layers):
         if not 1 <= len(layers) <= MAX_BATCH:
@@ -464,6 +465,8 @@ class LinearBatch:
             d.N, d.K = n, k
             d.y_dtype = _dt(out.dtype)
             d.epilogue = epi
+            d.flags = 1 if lay.get("depends") else 0   # MXQ_BATCH_DEPENDS: a new group, after everything before it
+            d.reserved = 0
             self.keep.append((x, codes, scales, out, res))
         self._ptr = ctypes.cast(self.array, ctypes.c_void_p)
 

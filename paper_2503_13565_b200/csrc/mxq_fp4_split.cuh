@@ -73,8 +73,12 @@ struct SplitToGlobal {
 // lanes call together (the block maximum is formed with shuffles).  `b` addresses the stage's operand rows (NB rows
 // of 128 bytes in 8-row groups of 1024 bytes, no swizzle), `sf` the stage's two 512-byte scale atoms.  Returns
 // whether this lane met an element that cannot be written exactly.
+// With `rem` (8 floats, may be nullptr) the function also says what is missing: the planes then hold each element
+// truncated to the block's 32-bit fixed point (all zeros for a block that contains an Inf or a NaN), and rem[i] is
+// element i minus what the planes hold -- exactly, in FP32 -- so that the caller can add rem[i] * w to the sums.
 template <class Dst>
-__device__ __forceinline__ bool split_half_unit_to(const uint4 raw, int m, uint32_t kin, int half, int lane, const Dst b, const Dst sf) {
+__device__ __forceinline__ bool split_half_unit_to(const uint4 raw, int m, uint32_t kin, int half, int lane, const Dst b, const Dst sf,
+                                                   float *rem = nullptr) {
     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
     // largest exponent field of the 32-block: both halves of a word at once, then across the block's four units
     uint32_t e2 = (w[0] >> 7) & 0x00FF00FFu;
@@ -85,8 +89,10 @@ __device__ __forceinline__ bool split_half_unit_to(const uint4 raw, int m, uint3
     emax = max(emax, __shfl_xor_sync(0xffffffffu, emax, 4));
     bool inexact = emax == 255u;                        // Inf or NaN in the block
     // 32-bit fixed point under the block maximum: plane p holds bits 31-2p, 30-2p, worth digit * 2^(top - 128 - 2p)
-    const uint32_t top = max(emax, 31u + kGuard);
+    const uint32_t top = min(max(emax, 31u + kGuard), 254u);
     const float up = __uint_as_float((285u - top) << 23);   // 2^(158 - top), a normal number for every top in 41..254
+    const float down = __uint_as_float((top - 31u) << 23);  // 2^(top - 158)
+    const bool nonfinite = emax == 255u;
     const uint32_t pick = half ? 0x4140u : 0x4342u;          // bytes (b0, 0, b1, 0) of this lane's 16 bits of the fixed point
     uint32_t pl[8];
 #pragma unroll
@@ -96,8 +102,18 @@ __device__ __forceinline__ bool split_half_unit_to(const uint4 raw, int m, uint3
         // |x| * 2^(158 - top) is the fixed-point value (bit 31 is worth 2^(top - 127)); it is below 2^32, and any
         // fraction it has is exactly the bits that would fall off the bottom
         const float scaled = __uint_as_float(mag) * up;
-        const uint32_t f = __float2uint_rz(scaled);
-        if (__uint2float_rn(f) != scaled) inexact = true;
+        uint32_t f = __float2uint_rz(scaled);
+        const float lost = scaled - __uint2float_rn(f);   // (exact: both have at most 8 significant bits)
+        if (lost != 0.f) inexact = true;
+        const uint32_t sbit = ((i & 1) ? word : (word << 16)) & 0x80000000u;
+        if (rem != nullptr) {
+            if (nonfinite) {
+                f = 0u;                                    // the block contributes nothing through the planes
+                rem[i] = __uint_as_float(mag | sbit);      // ... and everything through the remainder
+            } else {
+                rem[i] = __uint_as_float(__float_as_uint(lost * down) | sbit);
+            }
+        }
         const uint32_t sgn = (uint32_t)((int32_t)((i & 1) ? word : (word << 16)) >> 31) & 0x88888888u;
         uint32_t v = __byte_perm(f, 0u, pick);            // 8 digits in bytes 0 and 2
         v = (v | (v << 4)) & 0x0F0F0F0Fu;                 // 2 digits per byte

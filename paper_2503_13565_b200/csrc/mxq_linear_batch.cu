@@ -56,6 +56,12 @@ __device__ __forceinline__ float ld_cg_f32(const float *p) {
     return v;
 }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ float load_in_cg(const void *R, int dtype, int64_t idx) {
+    if (dtype == MXQ_F32) return ld_cg_f32(reinterpret_cast<const float *>(R) + idx);
+    unsigned short h;
+    asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(h) : "l"(reinterpret_cast<const unsigned short *>(R) + idx) : "memory");
+    return __uint_as_float((uint32_t)h << 16);
+}
 
 
 // Bounded wait on an mbarrier that also ends when the CTA's failure flag is raised.  False: gave up.  The probes are
@@ -79,7 +85,8 @@ __device__ __forceinline__ bool warp_wait_bar(uint32_t bar, uint32_t parity, vol
     if (lane == 0) ok = wait_bar(bar, parity, fail, limit_us) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
-// Bounded wait until a counter in global memory reaches `want`.
+// Bounded wait until a counter in global memory reaches `want`.  (Probes back to back: spacing them out with nanosleep was
+// measured and cost a microsecond per launch without relieving anything.)
 __device__ __forceinline__ bool wait_counter(const uint32_t *ctr, uint32_t want, volatile int *fail, uint32_t limit_us) {
     for (int i = 0; i < 256; ++i)
         if (ld_acquire_u32(ctr) >= want) return true;
@@ -137,7 +144,7 @@ __device__ __forceinline__ bool walk_opens(const Walk &w, int i, const Cursor &c
 __device__ __forceinline__ bool walk_closes(const Walk &w, int i, const Cursor &c) { return i == w.nunit - 1 || i == w.tail - 1 || c.s == c.ks - 1; }
 
 // NB: columns of the token operand / accumulator = 16 planes x token slots (16, 32 or 64).
-template <int NB>
+template <int NB, bool GROUPS>
 __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __grid_constant__ BatchTable tb) {
     extern __shared__ uint8_t smem_raw[];
     constexpr int MT = NB / 16;   // token slots
@@ -147,15 +154,23 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = (int)gridDim.x, cta = (int)blockIdx.x;
     const int M = tb.M, ring = tb.ring;
-    Walk wk;
-    wk.u0 = (int)((int64_t)cta * tb.units / G);
-    wk.nunit = (int)((int64_t)(cta + 1) * tb.units / G) - wk.u0;
-    {
-        Cursor last;
-        cursor_at(tb, wk.u0 + wk.nunit - 1, last);
-        wk.tail = (last.s != last.ks - 1 && last.s + 1 < wk.nunit) ? last.s + 1 : 0;
-    }
-    const int nunit = wk.nunit;
+    // The layers of a call form groups (a layer flagged as depending on earlier ones opens a new group); every group's
+    // units are cut into ranges of their own, and all CTAs go through the groups in order.
+    const int ngroups = GROUPS ? tb.ngroups : 1;
+    // (64-bit divisions and a search: tens of thousands of cycles for one thread if every role did this for every
+    // group after the wait below.  One lane per group does it before the wait and leaves the result in shared memory.)
+    auto compute_walk = [&](int g, Walk &w) {   // this CTA's range of group g (nunit = 0: none)
+        const int gu = tb.group_unit[g], ug = tb.group_unit[g + 1] - gu, gg = ug < G ? ug : G;
+        w.u0 = gu;
+        w.nunit = w.tail = 0;
+        if (cta < gg) {
+            w.u0 = gu + (int)((int64_t)cta * ug / gg);
+            w.nunit = gu + (int)((int64_t)(cta + 1) * ug / gg) - w.u0;
+            Cursor last;
+            cursor_at(tb, w.u0 + w.nunit - 1, last);
+            w.tail = (last.s != last.ks - 1 && last.s + 1 < w.nunit) ? last.s + 1 : 0;
+        }
+    };
     const uint32_t limit_us = tb.wait_us;
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -168,8 +183,15 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
     volatile int *s_fail = reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 4);
     volatile int *s_flag = reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 8);
     volatile int *s_zero = reinterpret_cast<volatile int *>(gbase + (sMisc - base) + 12);   // always 0
+    int *s_walk = reinterpret_cast<int *>(gbase + (sMisc - base) + 16);                      // [kBatchMaxGroups][3]
+    auto group_walk = [&](int g, Walk &w) {   // (valid after the block-wide barrier of the set-up)
+        w.u0 = s_walk[3 * g];
+        w.nunit = s_walk[3 * g + 1];
+        w.tail = s_walk[3 * g + 2];
+    };
 
     uint32_t *hdr = reinterpret_cast<uint32_t *>(tb.ws);
+    // (counter i of a kind lives kBatchCounterStride words after counter i - 1: a 128-byte line each)
     uint32_t *g_ready = hdr + kBatchWordReady, *g_bad = hdr + kBatchWordBad;
 
     // ---- set-up -------------------------------------------------------------------------------------------------------
@@ -196,22 +218,52 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
     // that only changes with the layer).  Slot addresses, parities and descriptors are carried along incrementally.
 
     // The first ring of weights does not depend on the previous kernel in the stream: requested before the wait.
-    const int pre = nunit < ring ? nunit : ring;
-    Cursor pc;   // producer: where the walk stands after the first `pre` requests
+    // producer state: the ring position of the next unit whose codes are requested (carried across groups)
+    uint32_t c_slot = base, c_fb = full0, c_eb = empty0, c_phase = 0;
+    int c_count = 0;   // units whose codes have been requested so far
+    const uint32_t ring_end = base + (uint32_t)ring * kSlot;
+    // codes of the first `n` units of walk `w` (announced without an arrival: the arrival comes with the operand)
+    auto request_codes_only = [&](const Walk &w, int n) -> bool {
+        Cursor c;
+        for (int i = 0; i < n; ++i) {
+            if (i) walk_to(tb, w, i, c);
+            else walk_begin(tb, w, c);
+            if (c_count >= ring && !wait_bar(c_eb, c_phase, s_fail, limit_us)) return false;
+            // (test hook: the bytes of unit tb.fault_unit are announced but never requested)
+            asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(c_fb), "r"(kBatchCodesBytes) : "memory");
+            if (walk_unit(w, i) != tb.fault_unit) tma_load_codes(c_slot, &tb.maps[c.d], c.s * (kBatchStageK / 2), c.t * kBatchTileRows, c_fb);
+            c_slot += kSlot;
+            c_fb += 8u;
+            c_eb += 8u;
+            if (c_slot == ring_end) {
+                c_slot = base;
+                c_fb = full0;
+                c_eb = empty0;
+                if (c_count >= ring) c_phase ^= 1u;
+            }
+            ++c_count;
+        }
+        return true;
+    };
+    int units_left = 0;   // (epilogue warps) of this CTA, over all groups: the last piece lets tensor memory go back
+    if (warp >= 2 && warp < 6) {
+        if (warp == 3 && lane < ngroups) {
+            Walk w;
+            compute_walk(lane, w);
+            s_walk[3 * lane] = w.u0;
+            s_walk[3 * lane + 1] = w.nunit;
+            s_walk[3 * lane + 2] = w.tail;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        for (int g = 0; g < ngroups; ++g) units_left += s_walk[3 * g + 1];
+    }
     if (warp == 1) {
         if (lane < tb.ndesc) asm volatile("prefetch.tensormap [%0];" ::"l"(&tb.maps[lane]) : "memory");
         __syncwarp();
         if (lane == 0) {
-            walk_begin(tb, wk, pc);
-            uint32_t dst = base, fb = full0;
-            for (int i = 0; i < pre; ++i) {
-                if (i) walk_to(tb, wk, i, pc);
-                // (test hook: the bytes of unit tb.fault_unit are announced but never requested)
-                asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(fb), "r"(kBatchCodesBytes) : "memory");
-                if (walk_unit(wk, i) != tb.fault_unit) tma_load_codes(dst, &tb.maps[pc.d], pc.s * (kBatchStageK / 2), pc.t * kBatchTileRows, fb);
-                dst += kSlot;
-                fb += 8u;
-            }
+            Walk wk0;
+            compute_walk(0, wk0);
+            (void)request_codes_only(wk0, wk0.nunit < ring ? wk0.nunit : ring);   // (nothing to wait for yet)
         }
         __syncwarp();
         pdl_wait();   // the counters in the workspace belong to the previous call until it has completed
@@ -234,14 +286,19 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
         const uint32_t sa_lo0 = (uint32_t)smem_desc(base + kBatchCodesBytes, 0, 128, 0);
         const uint32_t b_lo0 = (uint32_t)smem_desc(base + kBatchCodesBytes + kBatchSfBytes, 128, 1024, 0);
         const uint32_t sb_lo0 = (uint32_t)smem_desc(base + kBatchCodesBytes + kBatchSfBytes + (uint32_t)NB * 128u, 0, 128, 0);
-        Cursor c;
-        walk_begin(tb, wk, c);
         int d_seen = -1;
         bool half_k = false;
         uint32_t slot = 0, phase = 0, par = 0, accumulate = 0, off16 = 0;
         int acc_slot = -1;
         uint32_t acc_round = 0;   // how often the accumulator slots have wrapped
         uint32_t t_acc = tmem;
+        bool alive = true;
+        for (int g = 0; g < ngroups && alive; ++g) {
+        Walk wk;
+        group_walk(g, wk);
+        const int nunit = wk.nunit;
+        Cursor c;
+        if (nunit) walk_begin(tb, wk, c);
         for (int i = 0; i < nunit; ++i) {
             if (i) walk_to(tb, wk, i, c);
             if (c.d != d_seen) {
@@ -258,6 +315,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                         atomicOr(&g_batch_status, 4u);
                         *s_fail = 1;
                     }
+                    alive = false;
                     break;
                 }
                 tc_fence_after();
@@ -269,6 +327,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                     atomicOr(&g_batch_status, 1u);
                     *s_fail = 1;
                 }
+                alive = false;
                 break;
             }
             tc_fence_after();
@@ -310,6 +369,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                 phase ^= 1u;
             }
         }
+        }
         __syncwarp();
         // tensor memory goes back once the epilogue warps have read their last accumulator
         asm volatile("bar.sync 2, 160;" ::: "memory");
@@ -332,7 +392,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                 im = tb.desc[c.d].img;
                 img = tb.ws + tb.img[im].offset;
                 if (!((ready_mask >> im) & 1u)) {
-                    if (!wait_counter(g_ready + im, (uint32_t)tb.img[im].ntasks, s_fail, limit_us)) {
+                    if (!wait_counter(g_ready + im * kBatchCounterStride, (uint32_t)tb.img[im].ntasks, s_fail, limit_us)) {
                         atomicOr(&g_batch_status, 8u);
                         *s_fail = 1;
                         return false;
@@ -342,46 +402,67 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                 }
                 return true;
             };
-            Cursor c;
-            walk_begin(tb, wk, c);
-            uint32_t dst = base + kBatchCodesBytes + kBatchSfBytes, fb = full0;
-            int issued = 0;   // units whose operand has been requested
-            for (int i = 0; i < pre && ok; ++i) {
-                if (i) walk_to(tb, wk, i, c);
-                if (c.d != d_seen) ok = layer(c);
-                if (!ok) break;
-                mbar_expect_tx(fb, kXBytes);
-                bulk_load(dst, img + (uint32_t)c.s * kXBytes, kXBytes, fb);
-                dst += kSlot;
-                fb += 8u;
-                ++issued;
-            }
-            uint32_t slot_base = base, phase = 0;
-            fb = full0;
-            uint32_t eb = empty0;
-            const uint32_t ring_end = base + (uint32_t)ring * kSlot;
-            for (int i = pre; i < nunit && ok; ++i) {
-                walk_to(tb, wk, i, c);
-                if (c.d != d_seen) ok = layer(c);
-                if (!ok) break;
-                if (!wait_bar(eb, phase, s_fail, limit_us)) {
+            // the ring position of the next unit whose operand is requested (behind the codes by at most a ring)
+            uint32_t o_slot = base, o_fb = full0;
+            int issued = 0;   // units whose data has been requested in full
+            for (int g = 0; g < ngroups && ok; ++g) {
+                Walk wk;
+                group_walk(g, wk);
+                const int nunit = wk.nunit;
+                if (nunit == 0) continue;
+                const int pre = nunit < ring ? nunit : ring;
+                // A group's first ring of codes is requested before its token operand exists (group 0: before the previous
+                // kernel has completed; later groups: while the layers they depend on are being finished), as the slots
+                // come free.
+                if (g > 0 && !request_codes_only(wk, pre)) {
                     atomicOr(&g_batch_status, 2u);
                     *s_fail = 1;
                     ok = false;
                     break;
                 }
-                mbar_expect_tx(fb, kBatchCodesBytes + kXBytes);
-                if (walk_unit(wk, i) != tb.fault_unit) tma_load_codes(slot_base, map, c.s * (kBatchStageK / 2), c.t * kBatchTileRows, fb);
-                bulk_load(slot_base + kBatchCodesBytes + kBatchSfBytes, img + (uint32_t)c.s * kXBytes, kXBytes, fb);
-                ++issued;
-                slot_base += kSlot;
-                fb += 8u;
-                eb += 8u;
-                if (slot_base == ring_end) {
-                    slot_base = base;
-                    fb = full0;
-                    eb = empty0;
-                    phase ^= 1u;
+                Cursor c;
+                walk_begin(tb, wk, c);
+                for (int i = 0; i < pre && ok; ++i) {
+                    if (i) walk_to(tb, wk, i, c);
+                    if (c.d != d_seen) ok = layer(c);
+                    if (!ok) break;
+                    mbar_expect_tx(o_fb, kXBytes);
+                    bulk_load(o_slot + kBatchCodesBytes + kBatchSfBytes, img + (uint32_t)c.s * kXBytes, kXBytes, o_fb);
+                    o_slot += kSlot;
+                    o_fb += 8u;
+                    if (o_slot == ring_end) {
+                        o_slot = base;
+                        o_fb = full0;
+                    }
+                    ++issued;
+                }
+                // from here on codes and operand of a unit go out together (the two ring positions coincide again)
+                for (int i = pre; i < nunit && ok; ++i) {
+                    walk_to(tb, wk, i, c);
+                    if (c.d != d_seen) ok = layer(c);
+                    if (!ok) break;
+                    if (c_count >= ring && !wait_bar(c_eb, c_phase, s_fail, limit_us)) {
+                        atomicOr(&g_batch_status, 2u);
+                        *s_fail = 1;
+                        ok = false;
+                        break;
+                    }
+                    mbar_expect_tx(c_fb, kBatchCodesBytes + kXBytes);
+                    if (walk_unit(wk, i) != tb.fault_unit) tma_load_codes(c_slot, map, c.s * (kBatchStageK / 2), c.t * kBatchTileRows, c_fb);
+                    bulk_load(c_slot + kBatchCodesBytes + kBatchSfBytes, img + (uint32_t)c.s * kXBytes, kXBytes, c_fb);
+                    ++issued;
+                    c_slot += kSlot;
+                    c_fb += 8u;
+                    c_eb += 8u;
+                    if (c_slot == ring_end) {
+                        c_slot = base;
+                        c_fb = full0;
+                        c_eb = empty0;
+                        if (c_count >= ring) c_phase ^= 1u;
+                    }
+                    ++c_count;
+                    o_slot = c_slot;
+                    o_fb = c_fb;
                 }
             }
             if (!ok || *s_fail) {
@@ -389,6 +470,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                 // the barriers of complete requests are waited for, the rest is given time.
                 for (int i = max(0, issued - ring); i < issued; ++i)
                     (void)wait_bar(full0 + (uint32_t)(i % ring) * 8u, (uint32_t)((i / ring) & 1), s_zero, 1000u);
+                (void)c_count;
                 const uint64_t t0 = global_ns();
                 while (global_ns() - t0 < 100000ull) __nanosleep(1000);
             }
@@ -404,7 +486,8 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
         const int sw = warp - 6;   // 0..3
         const int nsw = ring < 4 ? ring : 4;
         uint32_t rows_lo[4], rows_hi[4];
-        auto load = [&](int i, uint32_t (&lo)[4], uint32_t (&hi)[4]) {   // element i of the walk
+        Walk wk;
+        auto load = [&](int i, uint32_t (&lo)[4], uint32_t (&hi)[4]) {   // element i of the current group's walk
             Cursor c;
             cursor_at(tb, walk_unit(wk, i), c);
             const BatchDesc &ds = tb.desc[c.d];
@@ -427,11 +510,20 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                 src += (int64_t)32 * kb_row;
             }
         };
-        if (sw < nsw && sw < nunit) load(sw, rows_lo, rows_hi);
-        // element i goes to slot i % ring: the slot index advances by nsw (mod ring) from one unit of this warp to the next
-        uint32_t slot = (uint32_t)sw, round = 0;   // (sw < nsw <= ring)
+        // The CTA's units are numbered through all groups; unit e goes to slot e % ring, and this warp takes the units
+        // e = sw (mod nsw): the slot index advances by nsw (mod ring) from one unit of this warp to the next.
         const uint32_t step = (uint32_t)nsw % (uint32_t)ring, carry = (uint32_t)nsw / (uint32_t)ring;
-        for (int i = sw < nsw ? sw : nunit; i < nunit; i += nsw) {
+        int ebase = 0;   // units of the groups before this one
+        bool alive = sw < nsw;
+        for (int g = 0; g < ngroups && alive; ++g) {
+        group_walk(g, wk);
+        const int nunit = wk.nunit;
+        // first unit of this group that is this warp's: the smallest i >= 0 with (ebase + i) % nsw == sw
+        const int i0 = (sw - ebase % nsw + nsw) % nsw;
+        uint32_t slot = (uint32_t)((ebase + i0) % ring), round = (uint32_t)((ebase + i0) / ring);
+        ebase += nunit;
+        if (i0 < nunit) load(i0, rows_lo, rows_hi);
+        for (int i = i0; i < nunit; i += nsw) {
             uint32_t cur_lo[4], cur_hi[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -444,6 +536,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                     atomicOr(&g_batch_status, 2u);
                     *s_fail = 1;
                 }
+                alive = false;
                 break;
             }
             const uint32_t sf = base + slot * kSlot + kBatchCodesBytes + (uint32_t)lane * 16u;
@@ -459,20 +552,44 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                 ++round;
             }
         }
+        }
     } else {
         // ---- split / epilogue warps -----------------------------------------------------------------------------------
         const int ew = warp - 2;                          // 0..3
         const int et = tid - 64;                          // 0..127
         const int row = ((warp & 3) << 5) + lane;         // accumulator row this thread may read (its warp's quarter)
 
-        // 1. the rewriting of the token rows: task = 128 k of one token row of one image.  Tasks are handed out by a counter
-        //    in the workspace, not by CTA index: every consumer waits for whole images, so a CTA that starts late (CTAs
-        //    start over several microseconds as the previous kernel's leave) must not be holding tasks.
-        for (;;) {
+        // Everything between the wait above and the first MMA is paid by every launch in full, so the first task of the
+        // rewriting is asked for before anything else.
+        uint32_t first_task = 0;
+        if (lane == 0) first_task = atomicAdd(hdr + kBatchWordTask, 1u);
+        uint32_t seen_mask = 0, bad_mask = 0, fix_mask = 0;
+        float *partials = reinterpret_cast<float *>(tb.ws + tb.partials_offset);
+        uint32_t *g_ticket = hdr + kBatchWordTicket, *g_done = hdr + kBatchWordDone;
+        const float nanv = __uint_as_float(0x7FC00000u);
+        int seg = 0;
+        if (units_left == 0) asm volatile("bar.arrive 2, 160;" ::: "memory");
+        for (int g = 0; g < ngroups; ++g) {
+        Walk wk;
+        group_walk(g, wk);
+        const int nunit = wk.nunit;
+        const int gu = tb.group_unit[g], ug = tb.group_unit[g + 1] - gu, gg = ug < G ? ug : G;
+        // 0. a later group reads what the groups before it wrote: all their tiles must have been stored
+        if (g > 0) {
+            if (et == 0 && !*s_fail && !wait_counter(g_done + (g - 1) * kBatchCounterStride, (uint32_t)tb.group_tiles[g - 1], s_fail, limit_us)) {
+                atomicOr(&g_batch_status, 8u);
+                *s_fail = 1;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+        // 1. the rewriting of the group's token rows: task = 128 k of one token row of one image.  Tasks are handed out by a
+        //    counter in the workspace, not by CTA index: every consumer waits for whole images, so a CTA that starts late
+        //    (CTAs start over several microseconds as the previous kernel's leave) must not be holding tasks.
+        for (bool first = g == 0;; first = false) {
             int task = 0;
-            if (lane == 0) task = (int)atomicAdd(hdr + kBatchWordTask, 1u);
+            if (lane == 0) task = tb.group_task[g] + (int)(first ? first_task : atomicAdd(hdr + kBatchWordTask + g * kBatchCounterStride, 1u));
             task = __shfl_sync(0xffffffffu, task, 0);
-            if (task >= tb.tasks) break;
+            if (task >= tb.group_task[g + 1]) break;
             int im = 0;
             while (im + 1 < tb.nimg && task >= tb.img[im + 1].task_base) ++im;
             const BatchImg &gi = tb.img[im];
@@ -481,22 +598,39 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
             const int kk = k128 * 128 + (lane >> 1) * 8;
             const uint4 raw = ld_cg_u4(reinterpret_cast<const __nv_bfloat16 *>(gi.X) + (int64_t)m * gi.K + kk);
             uint8_t *stage = tb.ws + gi.offset + (size_t)(kk >> 8) * kXBytes;
-            const bool inexact = split_half_unit_to(raw, m, (uint32_t)kk & 255u, lane & 1, lane, SplitToGlobal{stage},
-                                                    SplitToGlobal{stage + (uint32_t)NB * 128u});
-            const bool bad = __any_sync(0xffffffffu, inexact);
-            __syncwarp();   // (orders the lanes' stores before lane 0's release; the readers order them against their bulk copies)
-            if (lane == 0) {
-                if (bad) atomicOr(g_bad + im, 1u);
-                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(g_ready + im) : "memory");
+            bool inexact = split_half_unit_to(raw, m, (uint32_t)kk & 255u, lane & 1, lane, SplitToGlobal{stage},
+                                              SplitToGlobal{stage + (uint32_t)NB * 128u});
+            if (__any_sync(0xffffffffu, inexact)) {
+                // (rare, and kept off the common path, whose length every launch pays for: the rewriting is done again,
+                // this time asking for what the planes cannot hold)
+                float rem[8];
+                inexact = split_half_unit_to(raw, m, (uint32_t)kk & 255u, lane & 1, lane, SplitToGlobal{stage},
+                                             SplitToGlobal{stage + (uint32_t)NB * 128u}, rem);
+                // Elements that do not fit the block's fixed point (more than 24 binades under the block's maximum; any
+                // element of a block with an Inf or a NaN): the planes hold them truncated, and what is missing goes on the
+                // image's list of corrections (token row, k, remainder), which the epilogues add as remainder * weight.  A
+                // list that overflows flags the image; its layers are then computed by the scalar path.
+                if (inexact && (lane & 1) == 0) {
+                    BatchFix *fixes = reinterpret_cast<BatchFix *>(tb.ws + tb.fix_offset) + (size_t)im * kBatchMaxFixes;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        if (rem[e] != 0.f) {   // (NaN included)
+                            const uint32_t at = atomicAdd(g_bad + im * kBatchCounterStride + 1, 1u);
+                            if (at < (uint32_t)kBatchMaxFixes) {
+                                fixes[at].m = m;
+                                fixes[at].k = kk + e;
+                                fixes[at].rem = rem[e];
+                            } else {
+                                atomicOr(g_bad + im * kBatchCounterStride, 1u);
+                            }
+                        }
+                }
             }
+            __syncwarp();   // (orders the lanes' stores before lane 0's release; the readers order them against their bulk copies)
+            if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(g_ready + im * kBatchCounterStride) : "memory");
         }
 
-        // 2. epilogues: one per piece of a tile in this CTA's walk, in order
-        uint32_t seen_mask = 0, bad_mask = 0;
-        float *partials = reinterpret_cast<float *>(tb.ws + tb.partials_offset);
-        uint32_t *g_ticket = hdr + kBatchWordTicket;
-        const float nanv = __uint_as_float(0x7FC00000u);
-        int seg = 0;
+        // 2. epilogues: one per piece of a tile in this CTA's walk of the group, in order
         for (int i = 0; i < nunit; ++seg) {
             Cursor c;
             const int u = walk_unit(wk, i);
@@ -506,22 +640,25 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
             const int s_begin = c.s, s_end = c.s + len;
             const int a = seg % A;
             i += len;
-            const bool last_seg = i >= nunit;
+            units_left -= len;
+            const bool last_seg = units_left == 0;
             // has this layer's X been rewritten exactly?  (the counter is complete by now; waiting for it here makes the
             // flag's value certain)
             const int im = ds.img;
             if (!((seen_mask >> im) & 1u)) {
                 uint32_t b = 0;
                 if (lane == 0) {
-                    if (!wait_counter(g_ready + im, (uint32_t)tb.img[im].ntasks, s_fail, limit_us)) {
+                    if (!wait_counter(g_ready + im * kBatchCounterStride, (uint32_t)tb.img[im].ntasks, s_fail, limit_us)) {
                         atomicOr(&g_batch_status, 8u);
                         *s_fail = 1;
                     }
-                    b = *reinterpret_cast<volatile uint32_t *>(g_bad + im);
+                    b = *reinterpret_cast<volatile uint32_t *>(g_bad + im * kBatchCounterStride);
+                    if (*reinterpret_cast<volatile uint32_t *>(g_bad + im * kBatchCounterStride + 1) != 0u) b |= 2u;
                 }
                 b = __shfl_sync(0xffffffffu, b, 0);
                 seen_mask |= 1u << im;
-                if (b) bad_mask |= 1u << im;
+                if (b & 1u) bad_mask |= 1u << im;
+                if (b & 2u) fix_mask |= 1u << im;
             }
             const bool bad = (bad_mask >> im) & 1u;
 
@@ -580,7 +717,8 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
 #pragma unroll
                                 for (int m = 0; m < MT; ++m)
                                     if (m < M) {
-                                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * ds.K + k);
+                                        uint32_t xb;
+                                        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(xb) : "l"(X + (int64_t)m * ds.K + k) : "memory");
                                         part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
                                         part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
                                     }
@@ -601,27 +739,31 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
             if (s_begin != 0 || s_end != c.ks) {
                 // The tile is shared with the neighbouring ranges: deliver this part, and finish the tile if it was the last.
                 const int64_t ta = (int64_t)ds.unit_base + (int64_t)c.t * c.ks, tz = ta + c.ks - 1;
-                const int c_first = (int)batch_owner(ta, tb.units, G), c_last = (int)batch_owner(tz, tb.units, G);
+                const int c_first = (int)batch_owner(ta - gu, ug, gg), c_last = (int)batch_owner(tz - gu, ug, gg);
                 const int ncontrib = c_last - c_first + 1;
                 const bool head = u == wk.u0;   // the piece that opens this CTA's range
                 float *mine = partials + ((size_t)(cta * 2 + (head ? 0 : 1)) * MT) * 128u;
 #pragma unroll
                 for (int m = 0; m < MT; ++m)
                     if (m < M) mine[m * 128 + row] = yt[m];
-                __threadfence();
+                // The barrier orders the 128 threads' stores before thread 0's ticket, whose release (cumulative, GPU scope)
+                // publishes them; its acquire, passed on through the next barrier, lets a finisher read the other parts.
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (et == 0) *s_flag = (int)atomicAdd(g_ticket + c_first, 1u);
+                if (et == 0) {
+                    uint32_t old;
+                    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(g_ticket + c_first) : "memory");
+                    *s_flag = (int)old;
+                }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 finish = *s_flag == ncontrib - 1;
                 asm volatile("bar.sync 1, 128;" ::: "memory");   // (s_flag may be rewritten by the next piece)
                 if (finish) {
-                    __threadfence();
                     float sum[MT];
 #pragma unroll
                     for (int m = 0; m < MT; ++m) sum[m] = 0.f;
                     for (int j = 0; j < ncontrib; ++j) {   // range order, whoever finishes
                         const int cj = c_first + j;
-                        const bool hj = j > 0 || batch_range_lo(cj, tb.units, G) == ta;
+                        const bool hj = j > 0 || gu + batch_range_lo(cj, ug, gg) == ta;
                         const float *part = partials + ((size_t)(cj * 2 + (hj ? 0 : 1)) * MT) * 128u;
 #pragma unroll
                         for (int m = 0; m < MT; ++m)
@@ -636,6 +778,22 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                 // finished sums of weight row n, one per token row: restore the guard factor, apply the layer's epilogue, store
 #pragma unroll
                 for (int m = 0; m < MT; ++m) yt[m] *= kGuardUp;
+                if (((fix_mask >> im) & 1u) && !bad && n < ds.N) {
+                    // what the planes of this layer's X could not hold: remainder * weight, element by element
+                    const BatchFix *fixes = reinterpret_cast<const BatchFix *>(tb.ws + tb.fix_offset) + (size_t)im * kBatchMaxFixes;
+                    const uint32_t nfix = min(*reinterpret_cast<volatile uint32_t *>(g_bad + im * kBatchCounterStride + 1), (uint32_t)kBatchMaxFixes);
+                    for (uint32_t e = 0; e < nfix; ++e) {
+                        const uint4 fx = ld_cg_u4(fixes + e);   // (written by another SM during this kernel: through L2)
+                        const int fm = (int)fx.x, fk = (int)fx.y;
+                        const uint32_t byte = ds.codes[(int64_t)n * (ds.K / 2) + (fk >> 1)];
+                        const float2 wv = __half22float2(e2m1x2_to_half2(byte));
+                        const float wgt = ((fk & 1) ? wv.y : wv.x) * e8m0_to_float(ds.scales[(int64_t)n * (ds.K >> 5) + (fk >> 5)]);
+                        const float add = __uint_as_float(fx.z) * wgt;
+#pragma unroll
+                        for (int m = 0; m < MT; ++m)
+                            if (m == fm) yt[m] += add;
+                    }
+                }
                 if (ds.epi == 2) {
                     // gate / up rows interleaved: the partner row's sums sit in the neighbouring lane
                     float y[MT];
@@ -654,11 +812,19 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                     for (int m = 0; m < MT; ++m)
                         if (m < M) {
                             const int64_t at = (int64_t)m * ds.N + n;
-                            const float r = ds.epi == 1 ? load_in(ds.residual, ds.y_dtype, at) : 0.f;
+                            // (through L2: in a call of several groups another SM may have written the residual during this kernel)
+                            const float r = ds.epi == 1 ? load_in_cg(ds.residual, ds.y_dtype, at) : 0.f;
                             store_out(ds.Y, ds.y_dtype, at, yt[m] + r);
                         }
                 }
+                if (ngroups > 1) {
+                    // the tile is stored: one more of this group's tiles that the next group may read (barrier, then one
+                    // thread's cumulative release)
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (et == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(g_done + g * kBatchCounterStride) : "memory");
+                }
             }
+        }
         }
 
         // 3. the last CTA to get here leaves the counters zero for the next call
@@ -669,25 +835,29 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
             if (old == (uint32_t)G - 1u) {
                 __threadfence();
                 for (int i = 0; i < tb.nimg; ++i) {
-                    g_ready[i] = 0u;
-                    g_bad[i] = 0u;
+                    g_ready[i * kBatchCounterStride] = 0u;
+                    g_bad[i * kBatchCounterStride] = 0u;
+                    g_bad[i * kBatchCounterStride + 1] = 0u;
                 }
-                hdr[kBatchWordTask] = 0u;
+                for (int i = 0; i < ngroups; ++i) {
+                    hdr[kBatchWordTask + i * kBatchCounterStride] = 0u;
+                    g_done[i * kBatchCounterStride] = 0u;
+                }
                 hdr[kBatchWordExit] = 0u;
             }
         }
     }
 }
 
-template <int NB>
+template <int NB, bool GROUPS>
 cudaError_t launch_batch(const BatchTable &tb, int grid, uint32_t smem, cudaStream_t stream) {
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(linear_batch_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBatchSmemLimit);
+        cudaError_t e = cudaFuncSetAttribute(linear_batch_kernel<NB, GROUPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBatchSmemLimit);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(linear_batch_kernel<NB>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(linear_batch_kernel<NB, GROUPS>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -701,7 +871,7 @@ cudaError_t launch_batch(const BatchTable &tb, int grid, uint32_t smem, cudaStre
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl_enabled() ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, linear_batch_kernel<NB>, tb);
+    return cudaLaunchKernelEx(&cfg, linear_batch_kernel<NB, GROUPS>, tb);
 }
 
 // test hook (mxq_debug_batch_fault): consumed by the next launch
@@ -714,6 +884,7 @@ struct BatchLayout {
 };
 
 // ring slots and CTAs for `units` units of work
+// `units`: units of work of the call's largest group
 bool batch_layout(int M, int64_t units, BatchLayout &L) {
     const LayoutOverride o = layout_override();
     L.nb = batch_nb(M);
@@ -762,6 +933,8 @@ static size_t batch_workspace_bytes(const mxq_linear_desc *descs, int count, int
     const int nb = batch_nb(M);
     size_t b = kBatchHeaderBytes + batch_partials_bytes(kBatchMaxGrid, nb);
     for (int i = 0; i < count; ++i) b += (size_t)((descs[i].K + 255) / 256) * batch_image_stage_bytes(nb);
+    b = (b + 255u) & ~(size_t)255u;
+    b += (size_t)count * kBatchMaxFixes * sizeof(BatchFix);   // corrections: one list per image, at most one image per layer
     return (b + 255u) & ~(size_t)255u;
 }
 
@@ -773,9 +946,12 @@ extern "C" {
 static int batch_validate(const mxq_linear_desc *descs, int count, int M) {
     if (!descs) return MXQ_ERR_NULL;
     if (count < 1 || count > MXQ_MAX_BATCH || M < 1 || M > MXQ_MAX_M) return MXQ_ERR_SHAPE;
+    int groups = 1;
     for (int i = 0; i < count; ++i) {
         const mxq_linear_desc &d = descs[i];
         if (!d.X_bf16 || !d.codes || !d.scales || !d.Y) return MXQ_ERR_NULL;
+        if ((d.flags & ~MXQ_BATCH_DEPENDS) != 0 || d.reserved != 0) return MXQ_ERR_SHAPE;
+        if (i > 0 && (d.flags & MXQ_BATCH_DEPENDS) && ++groups > MXQ_MAX_BATCH_GROUPS) return MXQ_ERR_SHAPE;
         if (d.epilogue < MXQ_EPI_NONE || d.epilogue > MXQ_EPI_SWIGLU) return MXQ_ERR_SHAPE;
         if (d.epilogue == MXQ_EPI_RESIDUAL && !d.residual) return MXQ_ERR_NULL;
         if (!mxq::shape_ok(d.N, d.K) || (d.epilogue == MXQ_EPI_SWIGLU && (d.N & 1))) return MXQ_ERR_SHAPE;
@@ -812,8 +988,14 @@ int mxq_linear_batch_info(const mxq_linear_desc *descs, int count, int M, int32_
     if (rc != MXQ_OK) return rc;
     for (int i = 0; i < 8; ++i) info[i] = 0;
     if (!mxq::batch_covered(descs, count, M)) return MXQ_OK;
-    int64_t units = 0;
-    for (int i = 0; i < count; ++i) units += ((descs[i].N + 127) / 128) * ((descs[i].K + 255) / 256);
+    int64_t units = 0, total = 0, cur = 0;
+    for (int i = 0; i < count; ++i) {
+        if (i > 0 && (descs[i].flags & MXQ_BATCH_DEPENDS)) cur = 0;
+        const int64_t u = ((descs[i].N + 127) / 128) * ((descs[i].K + 255) / 256);
+        cur += u;
+        total += u;
+        if (cur > units) units = cur;
+    }
     mxq::BatchLayout L;
     if (!mxq::batch_layout(M, units, L)) return MXQ_OK;
     info[0] = 1;
@@ -821,7 +1003,7 @@ int mxq_linear_batch_info(const mxq_linear_desc *descs, int count, int M, int32_
     info[2] = L.ring;
     info[3] = (int32_t)L.smem;
     info[4] = L.nb;
-    info[5] = (int32_t)units;
+    info[5] = (int32_t)total;
     info[6] = mxq::batch_tmem_cols(L.nb, L.per_sm);
     info[7] = mxq::batch_acc_slots(L.nb, L.per_sm);
     return MXQ_OK;
@@ -835,8 +1017,12 @@ int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *works
     if (workspace_bytes < mxq_linear_batch_workspace_bytes(descs, count, M)) return MXQ_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     mxq::BatchLayout L;
-    int64_t units = 0;
-    for (int i = 0; i < count; ++i) units += ((descs[i].N + 127) / 128) * ((descs[i].K + 255) / 256);
+    int64_t units = 0, cur = 0;   // units of the largest group
+    for (int i = 0; i < count; ++i) {
+        if (i > 0 && (descs[i].flags & MXQ_BATCH_DEPENDS)) cur = 0;
+        cur += ((descs[i].N + 127) / 128) * ((descs[i].K + 255) / 256);
+        if (cur > units) units = cur;
+    }
     if (!mxq::batch_covered(descs, count, M) || !mxq::batch_layout(M, units, L)) {
         // one layer after the other through the ordinary entry points, sharing the scratch behind the header
         uint8_t *ws = static_cast<uint8_t *>(workspace) + mxq::kBatchHeaderBytes;
@@ -861,10 +1047,17 @@ int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *works
     tb.acc_slots = mxq::batch_acc_slots(nb, L.per_sm);
     tb.partials_offset = (uint32_t)mxq::kBatchHeaderBytes;
     size_t img_off = mxq::kBatchHeaderBytes + mxq::batch_partials_bytes(mxq::kBatchMaxGrid, nb);
-    int unit_base = 0, task_base = 0, nimg = 0;
+    int unit_base = 0, task_base = 0, nimg = 0, ngroups = 0, group_img0 = 0;
     for (int i = 0; i < count; ++i) {
         const mxq_linear_desc &d = descs[i];
         mxq::BatchDesc &o = tb.desc[i];
+        if (i == 0 || (d.flags & MXQ_BATCH_DEPENDS)) {   // a new group: its layers may read what the layers before wrote
+            tb.group_unit[ngroups] = unit_base;
+            tb.group_task[ngroups] = task_base;
+            tb.group_tiles[ngroups] = 0;
+            group_img0 = nimg;
+            ++ngroups;
+        }
         if (!mxq::codes_tensor_map(d.codes, d.N, d.K, /*expand_fp4=*/false, &tb.maps[i])) return MXQ_ERR_CUDA;
         o.codes = d.codes;
         o.scales = d.scales;
@@ -879,9 +1072,10 @@ int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *works
         o.y_dtype = d.y_dtype;
         o.epi = d.epilogue;
         unit_base += o.ks * o.tiles;
-        // layers that read the same X share one image
+        tb.group_tiles[ngroups - 1] += o.tiles;
+        // layers of a group that read the same X share one image
         int im = -1;
-        for (int j = 0; j < nimg; ++j)
+        for (int j = group_img0; j < nimg; ++j)
             if (tb.img[j].X == d.X_bf16 && tb.img[j].K == o.K) im = j;
         if (im < 0) {
             im = nimg++;
@@ -897,16 +1091,26 @@ int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *works
         }
         o.img = im;
     }
+    tb.fix_offset = (uint32_t)((img_off + 255u) & ~(size_t)255u);
     tb.nimg = nimg;
     tb.units = unit_base;
     tb.tasks = task_base;
+    tb.ngroups = ngroups;
+    tb.group_unit[ngroups] = unit_base;
+    tb.group_task[ngroups] = task_base;
     tb.fault_unit = mxq::g_fault_unit.exchange(-1, std::memory_order_relaxed);
     const unsigned w = mxq::g_fault_wait_us.exchange(0, std::memory_order_relaxed);
     tb.wait_us = w ? w : 1000000u;
-    const cudaError_t e = nb == 16 ? mxq::launch_batch<16>(tb, L.grid, L.smem, st)
-                          : nb == 32 ? mxq::launch_batch<32>(tb, L.grid, L.smem, st)
-                          : nb == 64 ? mxq::launch_batch<64>(tb, L.grid, L.smem, st)
-                                     : mxq::launch_batch<128>(tb, L.grid, L.smem, st);
+    // (a call of one group runs the kernel compiled without the loops over groups: measured 2 us per launch faster at
+    // one 7B layer set per call, equal at four)
+    const cudaError_t e = ngroups > 1 ? (nb == 16 ? mxq::launch_batch<16, true>(tb, L.grid, L.smem, st)
+                                         : nb == 32 ? mxq::launch_batch<32, true>(tb, L.grid, L.smem, st)
+                                         : nb == 64 ? mxq::launch_batch<64, true>(tb, L.grid, L.smem, st)
+                                                    : mxq::launch_batch<128, true>(tb, L.grid, L.smem, st))
+                                      : (nb == 16 ? mxq::launch_batch<16, false>(tb, L.grid, L.smem, st)
+                                         : nb == 32 ? mxq::launch_batch<32, false>(tb, L.grid, L.smem, st)
+                                         : nb == 64 ? mxq::launch_batch<64, false>(tb, L.grid, L.smem, st)
+                                                    : mxq::launch_batch<128, false>(tb, L.grid, L.smem, st));
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return MXQ_ERR_CUDA;

@@ -22,18 +22,24 @@ constexpr uint32_t kBatchCodesBytes = 16384;   // 128 rows x 128 bytes
 constexpr uint32_t kBatchSfBytes = 1024;       // two 512-byte scale atoms (4 blocks each)
 constexpr uint32_t kBatchSmemLimit = 227 * 1024;
 constexpr int kBatchMaxGrid = 1024;      // CTAs (ticket counters in the workspace header)
+constexpr int kBatchMaxGroups = 8;       // groups of layers per call (a layer that depends on earlier ones opens a group)
 
 // ---- workspace ------------------------------------------------------------------------------------------------------
-// [0, kBatchHeaderBytes)  counters, all zero between calls:
-//      u32 ready[32]   split tasks delivered per token-operand image
-//      u32 bad[32]     an image holds a block that could not be rewritten exactly
-//      u32 exit        CTAs that have finished (word 64)
-//      u32 task        rewriting tasks handed out (word 65)
-//      u32 ticket[kBatchMaxGrid] at byte 512: contributors that have delivered their share of a tile split between CTAs
+// [0, kBatchHeaderBytes)  counters, all zero between calls; every counter that many CTAs wait for has a 128-byte line
+//                          to itself (kBatchCounterStride words from one to the next):
+//      u32 ready[32]   split tasks delivered per token-operand image            (words 0, 32, 64, ...)
+//      u32 bad[32]     an image's list of corrections overflowed (the word after its ready counter)
+//      u32 fixes[32]   entries on an image's list of corrections (the word after that)
+//      u32 done[8]     tiles stored, per group                                  (words 1024, 1056, ...)
+//      u32 task[8]     rewriting tasks handed out, per group                    (the word after the group's done counter)
+//      u32 exit        CTAs that have finished                                  (word 1280)
+//      u32 ticket[kBatchMaxGrid] at word 2048: contributors that have delivered their share of a tile split between CTAs
 // [kBatchHeaderBytes, ...) partial sums: [grid][2 (at the head / at the tail of the CTA's range)][token slots][128] floats
 // then the token-operand images, one per distinct X: [stage][operand rows NB x 128 bytes | 1024 bytes of scale atoms]
-constexpr size_t kBatchHeaderBytes = 8192;
-constexpr int kBatchWordReady = 0, kBatchWordBad = 32, kBatchWordExit = 64, kBatchWordTask = 65, kBatchWordTicket = 128;
+// then the lists of corrections, kBatchMaxFixes entries per image
+constexpr size_t kBatchHeaderBytes = 16384;
+constexpr int kBatchCounterStride = 32;
+constexpr int kBatchWordReady = 0, kBatchWordBad = 1, kBatchWordDone = 1024, kBatchWordTask = 1025, kBatchWordExit = 1280, kBatchWordTicket = 2048;
 
 inline int batch_nb(int M) { return M == 1 ? 16 : (M == 2 ? 32 : (M <= 4 ? 64 : 128)); }   // operand columns: 16 planes per token slot
 inline uint32_t batch_image_stage_bytes(int nb) { return (uint32_t)nb * 128u + kBatchSfBytes; }
@@ -54,7 +60,7 @@ inline int batch_tmem_cols(int nb, int ctas_per_sm) {
 }
 inline uint32_t batch_smem_bytes(int nb, int ring) {
     const uint32_t b = 1024u /* alignment slack */ + (uint32_t)ring * batch_slot_bytes(nb) +
-                       (uint32_t)(2 * ring + 2 * 4) * 8u /* mbarriers */ + 64u /* tensor-memory address, flags */;
+                       (uint32_t)(2 * ring + 2 * 4) * 8u /* mbarriers */ + 128u /* tensor-memory address, flags, the CTA's ranges */;
     return (b + 15u) & ~15u;
 }
 
@@ -62,6 +68,13 @@ inline uint32_t batch_smem_bytes(int nb, int ring) {
 MXQ_BATCH_HD inline int64_t batch_range_lo(int64_t cta, int64_t units, int64_t grid) { return cta * units / grid; }
 // the CTA whose range holds unit u (grid <= units, so no range is empty)
 MXQ_BATCH_HD inline int64_t batch_owner(int64_t u, int64_t units, int64_t grid) { return ((u + 1) * grid - 1) / units; }
+
+constexpr int kBatchMaxFixes = 256;      // elements per image that may fall outside their block's fixed point
+struct BatchFix {                        // one such element: what the operand planes do not hold of X[m][k]
+    int32_t m, k;
+    float rem;
+    uint32_t pad;
+};
 
 struct BatchDesc {
     const uint8_t *codes, *scales;
@@ -88,10 +101,15 @@ struct BatchTable {
     uint8_t *ws;
     int32_t ndesc, nimg, M;
     int32_t units, tasks;
+    int32_t ngroups;
+    int32_t group_unit[kBatchMaxGroups + 1];   // first unit of every group (and the end)
+    int32_t group_task[kBatchMaxGroups + 1];   // first rewriting task of every group (and the end)
+    int32_t group_tiles[kBatchMaxGroups];      // tiles of every group
     int32_t ring, tmem_cols, acc_slots;
     int32_t fault_unit;          // test hook: the producer skips this unit's weight copy (-1: none)
     uint32_t wait_us;            // limit of every wait inside the kernel
     uint32_t partials_offset;    // bytes from the workspace base
+    uint32_t fix_offset;         // lists of corrections, bytes from the workspace base
 };
 
 }  // namespace mxq

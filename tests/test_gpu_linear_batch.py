@@ -183,14 +183,37 @@ def test_one_workspace_across_differently_shaped_calls():
         ba.run(ws)
         bb.run(ws)
     torch.cuda.synchronize()
-    assert int(ws[:8192].view(torch.int32).abs().sum()) == 0, "counters not left at zero"
+    assert int(ws[:16384].view(torch.int32).abs().sum()) == 0, "counters not left at zero"
     for i, lay in enumerate(a + b):
         check_layer(lay, "shared workspace layer %d" % i)
 
 
+@pytest.mark.parametrize("m", [1, 3, 8])
+@pytest.mark.parametrize("count", [40, 1500])
+def test_many_elements_far_below_their_blocks_maximum(m, count):
+    """Activations as a gated feed-forward block produces them: a few (here `count`, spread over the token rows) land
+    more than 24 binades under their block's maximum and do not fit the operand's fixed point.  Up to 256 per X they are
+    corrected one by one (remainder * weight in the epilogue); beyond that the layers reading that X take the scalar
+    path.  Either way the bound holds, for the layer that shares the X and for the one that does not."""
+    k, n = 2816, 640
+    x = synth.activations(3, 230, m, k).clone().float()
+    g = torch.Generator().manual_seed(count + m)
+    flat = x.view(-1)
+    idx = torch.randperm(flat.numel(), generator=g)[:count]
+    flat[idx] = flat[idx] * 2.0 ** -40 + 2.0 ** -60
+    xb = synth.bits_of(x.to(torch.bfloat16))
+    a = make_layer(3, 231, n, k, m, x=xb)
+    b = make_layer(3, 232, 2 * 384, k, m, x=xb, epilogue="swiglu")
+    b["x"] = a["x"]
+    c = make_layer(3, 233, 515, 1024, m)
+    run_batch([a, b, c])
+    for lay, what in ((a, "plain"), (b, "gate/up"), (c, "other X")):
+        check_layer(lay, "%d tiny elements, M=%d: %s" % (count, m, what))
+
+
 def test_activations_that_cannot_be_rewritten_exactly():
-    """An element more than 24 binades below its block's maximum, an infinity, a NaN: the affected layers take the
-    scalar path (same bound), the other layers of the call are untouched."""
+    """An element more than 24 binades below its block's maximum, an infinity, a NaN: corrected element by element in the
+    epilogue (same bound; Inf and NaN come out as IEEE arithmetic gives them), the other layers of the call are untouched."""
     m, k = 2, 1024
     x = synth.activations(3, 50, m, k).clone()
     x[0, 5] = 2.0 ** -40
@@ -280,6 +303,70 @@ def test_a_bounded_wait_that_expires_is_reported_and_contained():
     assert mxq.mxq_linear_device_status() == 0
     for i, lay in enumerate(layers):
         check_layer(lay, "after the fault, layer %d" % i)
+
+
+def chain_layers(m, h, f, seed):
+    """A decoder layer's dependent chain in three groups: {q/k/v as one matrix, o + residual} | {gate/up with SiLU(gate)*up}
+    | {down + residual}; every intermediate is BF16 and feeds the next group."""
+    qkv = make_layer(3, seed, 3 * h, h, m, out_dtype=torch.bfloat16)
+    o = make_layer(3, seed + 1, h, h, m, epilogue="residual", out_dtype=torch.bfloat16)
+    o["residual"] = qkv["x"]                                             # h0 (the layer's input) is the residual of o
+    gu = make_layer(3, seed + 2, 2 * f, h, m, epilogue="swiglu", out_dtype=torch.bfloat16)
+    gu["x"], gu["depends"] = o["out"], True                              # h1 = o's output
+    down = make_layer(3, seed + 3, h, f, m, epilogue="residual", out_dtype=torch.bfloat16)
+    down["x"], down["residual"], down["depends"] = gu["out"], o["out"], True
+    return [qkv, o, gu, down]
+
+
+def check_chain(layers, what):
+    """Stage by stage, each stage's oracle fed with the GPU's own (BF16) intermediates: a rounding difference in an
+    intermediate cannot leak into the next stage's check."""
+    qkv, o, gu, down = layers
+    gu["_x"] = synth.bits_of(o["out"].cpu())
+    down["_x"] = synth.bits_of(gu["out"].cpu())
+    for name, lay in zip(("qkv", "o", "gate/up", "down"), layers):
+        check_layer(lay, "%s: %s" % (what, name))
+
+
+@pytest.mark.parametrize("m", [1, 4, 8])
+@pytest.mark.parametrize("h,f", [(1024, 2816), (256, 384)])
+def test_dependent_groups_in_one_call(m, h, f):
+    """MXQ_BATCH_DEPENDS: a layer that reads what earlier layers of the same call wrote.  The small case has fewer units
+    per group than CTAs (some CTAs own nothing in a group); the larger one cuts tiles between CTAs in every group."""
+    layers = chain_layers(m, h, f, 200)
+    h1_before = layers[1]["out"].clone()
+    batch, ws = run_batch(layers)
+    assert not torch.equal(h1_before, layers[1]["out"])
+    check_chain(layers, "chain M=%d h=%d" % (m, h))
+    # again on the same workspace, and bit for bit the same
+    first = [lay["out"].clone() for lay in layers]
+    for lay in layers:
+        lay["out"].fill_(float("nan"))
+    batch.run(ws)
+    torch.cuda.synchronize()
+    for a, lay in zip(first, layers):
+        assert torch.equal(a, lay["out"])
+    assert int(ws[:16384].view(torch.int32).abs().sum()) == 0, "counters not left at zero"
+
+
+def test_dependent_groups_7b_layer():
+    """The four-call fused 7B layer (12288 x 4096; 4096 x 4096 + residual; 22016 x 4096 gate/up; 4096 x 11008 + residual) as
+    ONE call of three groups, sampled rows of every stage."""
+    m, h, f = 1, 4096, 11008
+    layers = chain_layers(m, h, f, 210)
+    for lay, n in zip(layers, (3 * h, h, f, h)):
+        lay["_rows"] = sample_rows(n, n % 97, 300)
+    run_batch(layers)
+    check_chain(layers, "7B chain")
+
+
+def test_too_many_groups_are_refused():
+    lays = [make_layer(3, 220, 128, 128, 1) for _ in range(10)]
+    for lay in lays[1:]:
+        lay["depends"] = True
+    with pytest.raises(mxq.MxqError) as e:
+        mxq.LinearBatch(lays).workspace_bytes() or mxq.LinearBatch(lays).run(mxq.new_workspace(1 << 20))
+    assert e.value.status == 2
 
 
 def test_argument_errors():

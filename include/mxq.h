@@ -340,6 +340,26 @@ int mxq_linear_batch_info(const mxq_linear_desc *descs, int count, int M, int32_
  * tiles that CTA had not finished are NaN.  unit = -1, wait_us = 0 cancels. */
 int mxq_debug_batch_fault(int unit, unsigned wait_us);
 
+/* The bounds-checked build (the library compiled with -DMXQ_DEBUG_BOUNDS; python -m paper_2503_13565_b200.build
+ * --checked writes it to libmxq_checked.so): in the linear kernels (mxq_linear with every kernel choice, the layer
+ * epilogues, mxq_lm_head_accept, mxq_linear_batch, mxq_linear_bf16) every plain load and store of global memory whose
+ * address is formed from an index -- X, codes, scales, Y, residual, workspace images, partial sums, correction lists,
+ * tickets -- is tested against its buffer first.  An access outside it is counted, the first one recorded, and the
+ * access itself redirected to a scratch area: a wrong index shows as a report, never as a fault.  (TMA copies are
+ * clipped by the hardware against their tensor map.)  Same results, several times slower; meant to be run once over the
+ * ragged-shape tests where no memory checker is at hand.
+ * mxq_debug_bounds_report: report[0] = 1 if this library is the checked build (else 0 and the rest stays 0);
+ *   report[1] = accesses refused since the last call; of the first one: report[2] = source file (0 mxq_linear.cu, 1
+ *   mxq_linear_umma.cu, 2 mxq_linear_fp4.cu, 3 mxq_linear_mma.cu, 4 mxq_linear_batch.cu, 5 mxq_linear_bf16.cu),
+ *   report[3] = source line, report[4] = byte offset from the buffer's base (modulo 2^64), report[5] = the buffer's size.
+ *   Reading clears the record.  Synchronises with the device.
+ * mxq_debug_bounds_selftest: checked build only (otherwise MXQ_ERR_SHAPE): one kernel stores 4 bytes at offset 100
+ *   through the checked address of a 64-byte buffer that lies inside a larger array of the library's own (so that not
+ *   even an unchecked store could leave it) and 4 bytes at offset 60; returns MXQ_OK if the array shows the second
+ *   store and nothing else.  The refused store is then in mxq_debug_bounds_report. */
+int mxq_debug_bounds_report(uint64_t *report);
+int mxq_debug_bounds_selftest(void *stream);
+
 #ifdef __cplusplus
 }
 #endif

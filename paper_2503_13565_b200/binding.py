@@ -14,7 +14,8 @@ import threading
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmxq.so")
+# MXQ_LIBRARY=checked in the environment loads the bounds-checked build instead (see mxq_debug_bounds_report in mxq.h)
+LIB_PATH = os.path.join(_HERE, "libmxq_checked.so" if os.environ.get("MXQ_LIBRARY") == "checked" else "libmxq.so")
 
 MXQ_OK = 0
 MXQ_F32, MXQ_BF16 = 0, 1
@@ -36,7 +37,7 @@ def lib() -> ctypes.CDLL:
     with _lock:
         if _lib is None:
             if not os.path.exists(LIB_PATH):
-                raise ImportError("libmxq.so is not built (%s missing): run python -m paper_2503_13565_b200.build; "
+                raise ImportError("the mxq library is not built (%s missing): run python -m paper_2503_13565_b200.build [--checked]; "
                                   "there is no CPU fallback" % LIB_PATH)
             L = ctypes.CDLL(LIB_PATH)
             vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
@@ -94,6 +95,10 @@ def lib() -> ctypes.CDLL:
             L.mxq_linear_batch.argtypes = [vp, i32, i32, vp, sz, vp]
             L.mxq_linear_batch_info.restype = i32
             L.mxq_linear_batch_info.argtypes = [vp, i32, i32, vp]
+            L.mxq_debug_bounds_report.restype = i32
+            L.mxq_debug_bounds_report.argtypes = [vp]
+            L.mxq_debug_bounds_selftest.restype = i32
+            L.mxq_debug_bounds_selftest.argtypes = [vp]
             L.mxq_debug_batch_fault.restype = i32
             L.mxq_debug_batch_fault.argtypes = [i32, ctypes.c_uint]
             _lib = L
@@ -492,6 +497,22 @@ def mxq_linear_batch(layers, workspace: torch.Tensor = None, stream=None) -> Lin
         workspace = new_workspace(batch.workspace_bytes(), batch.device)
     batch.run(workspace, stream)
     return batch
+
+
+def mxq_debug_bounds_report() -> dict:
+    """What the bounds-checked build has refused since the last call (see mxq.h); ``checked`` is False for the ordinary build."""
+    r = (ctypes.c_uint64 * 6)()
+    _check(lib().mxq_debug_bounds_report(ctypes.cast(r, ctypes.c_void_p)), "mxq_debug_bounds_report")
+    files = ("mxq_linear.cu", "mxq_linear_umma.cu", "mxq_linear_fp4.cu", "mxq_linear_mma.cu", "mxq_linear_batch.cu", "mxq_linear_bf16.cu")
+    out = {"checked": bool(r[0]), "refused": int(r[1])}
+    if r[1]:
+        out.update(file=files[int(r[2])], line=int(r[3]), offset=int(r[4]), extent=int(r[5]))
+    return out
+
+
+def mxq_debug_bounds_selftest(stream=None) -> None:
+    """Checked build only: one store outside a 64-byte buffer must be refused and redirected (see mxq.h)."""
+    _check(lib().mxq_debug_bounds_selftest(_stream(stream)), "mxq_debug_bounds_selftest")
 
 
 def mxq_debug_batch_fault(unit: int, wait_us: int) -> None:

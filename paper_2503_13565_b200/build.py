@@ -15,6 +15,11 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmxq.so")
 OBJ = os.path.join(HERE, "build")
+# the bounds-checked build (-DMXQ_DEBUG_BOUNDS: every plain global access of the linear kernels is tested against its
+# buffer first; see csrc/mxq_device.cuh): a library of its own, loaded instead of the ordinary one when the environment
+# has MXQ_LIBRARY=checked
+LIB_CHECKED = os.path.join(HERE, "libmxq_checked.so")
+OBJ_CHECKED = os.path.join(HERE, "build_checked")
 
 NVCC_FLAGS = [
     "-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
@@ -37,19 +42,21 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    lib, objdir = (LIB_CHECKED, OBJ_CHECKED) if checked else (LIB, OBJ)
+    extra = ["-DMXQ_DEBUG_BOUNDS"] if checked else []
     srcs = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
     hdrs = sorted(glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) +
                   glob.glob(os.path.join(HERE, "..", "include", "*.h")))
-    os.makedirs(OBJ, exist_ok=True)
+    os.makedirs(objdir, exist_ok=True)
     nvcc = _nvcc()
     jobs = []
     objs = []
     for s in srcs:
-        o = os.path.join(OBJ, os.path.basename(s)[:-3] + ".o")
+        o = os.path.join(objdir, os.path.basename(s)[:-3] + ".o")
         objs.append(o)
         if force or _stale(o, [s] + hdrs):
-            cmd = [nvcc] + NVCC_FLAGS + os.environ.get("MXQ_NVCC_FLAGS", "").split() + \
+            cmd = [nvcc] + NVCC_FLAGS + extra + os.environ.get("MXQ_NVCC_FLAGS", "").split() + \
                 (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
             jobs.append(cmd)
 
@@ -63,12 +70,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
         for out in ex.map(run, jobs):
             if verbose and out:
                 sys.stderr.write(out)
-    if force or jobs or _stale(LIB, objs):
-        tmp = LIB + ".%d.tmp" % os.getpid()
+    if force or jobs or _stale(lib, objs):
+        tmp = lib + ".%d.tmp" % os.getpid()
         run([nvcc, "-shared", "-o", tmp] + objs + ["-Xcompiler", "-fvisibility=hidden"])
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

@@ -21,6 +21,47 @@ constexpr int kBlock = 32;  // weights per scale (MX block), Sec. III-D-3
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// ---- bounds-checked build (-DMXQ_DEBUG_BOUNDS; the stand-in for a memory checker) -------------------------------
+// MXQ_AT(p, n, base, extent) stands where a kernel forms the address of a plain global load or store of n bytes into
+// the buffer [base, base + extent).  The ordinary build compiles it to p.  The checked build tests the range first;
+// an access outside it is counted, the first one is recorded (source line, byte offset from base, extent), and the
+// access is redirected to a scratch area, so that a wrong index shows up as a report and never as a fault.  (Copies
+// made by TMA are clipped by the hardware against the tensor map and need no check.)  Every translation unit keeps its
+// own record; mxq_debug_bounds_report adds them up.
+#ifdef MXQ_DEBUG_BOUNDS
+namespace {
+__device__ unsigned long long g_bounds[4];   // violations; of the first one: source line, offset, extent
+__device__ uint4 g_bounds_sink[2048];   // (32 KB: the largest single access is a bulk copy of 17 KB)
+}  // namespace
+template <class T>
+__device__ __forceinline__ T *bounds_checked(T *p, size_t n, const void *base, size_t extent, int line) {
+    const uintptr_t a = (uintptr_t)p, b = (uintptr_t)base;
+    if (a >= b && a + n <= b + extent) return p;
+    if (atomicAdd(&g_bounds[0], 1ull) == 0ull) {
+        g_bounds[1] = (unsigned long long)line;
+        g_bounds[2] = (unsigned long long)(a - b);
+        g_bounds[3] = (unsigned long long)extent;
+    }
+    return reinterpret_cast<T *>(reinterpret_cast<uintptr_t>(g_bounds_sink) + (a & 15u));   // (keeps the access's alignment)
+}
+#define MXQ_AT(p, n, base, extent) ::mxq::bounds_checked((p), (size_t)(n), (base), (size_t)(extent), __LINE__)
+// host: this translation unit's record, cleared by the read
+static int bounds_take_tu(unsigned long long *out) {
+    unsigned long long zero[4] = {0, 0, 0, 0};
+    if (cudaMemcpyFromSymbol(out, g_bounds, sizeof(zero)) != cudaSuccess) return MXQ_ERR_CUDA;
+    return cudaMemcpyToSymbol(g_bounds, zero, sizeof(zero)) == cudaSuccess ? MXQ_OK : MXQ_ERR_CUDA;
+}
+#define MXQ_BOUNDS_TU(name) \
+    int name(unsigned long long *out) { return bounds_take_tu(out); }
+#else
+#define MXQ_AT(p, n, base, extent) (p)
+#define MXQ_BOUNDS_TU(name)                     \
+    int name(unsigned long long *out) {         \
+        out[0] = out[1] = out[2] = out[3] = 0;  \
+        return MXQ_OK;                          \
+    }
+#endif
+
 // ---- loads that bypass L1 allocation (weights are read exactly once) -------------------
 __device__ __forceinline__ uint4 ld_stream_u4(const void *p) {
     uint4 v;

@@ -12,6 +12,8 @@
 #pragma once
 #include <stdint.h>
 
+#include "mxq_device.cuh"
+
 namespace mxq {
 
 // Every partial sum is bounded by sum |x w^|, which cancellation can leave up to 1/2e-3 = 500 times larger than a
@@ -63,8 +65,10 @@ struct SplitToShared {
 };
 struct SplitToGlobal {
     uint8_t *base;
-    __device__ __forceinline__ void u32(uint32_t off, uint32_t v) const { *reinterpret_cast<uint32_t *>(base + off) = v; }
-    __device__ __forceinline__ void u8(uint32_t off, uint32_t v) const { base[off] = (uint8_t)v; }
+    const uint8_t *whole;   // the buffer `base` points into and its size (bounds-checked build)
+    size_t whole_bytes;
+    __device__ __forceinline__ void u32(uint32_t off, uint32_t v) const { *MXQ_AT(reinterpret_cast<uint32_t *>(base + off), 4, whole, whole_bytes) = v; }
+    __device__ __forceinline__ void u8(uint32_t off, uint32_t v) const { *MXQ_AT(base + off, 1, whole, whole_bytes) = (uint8_t)v; }
 };
 
 // Half of one 8-element unit of X (16 bytes `raw`; token slot m; k offset kin inside a 256-k stage): the lane with

@@ -78,4 +78,14 @@ int linear_mma_take_status(uint32_t *out);    // the mma.sync kernel (mxq_linear
 int linear_batch_take_status(uint32_t *out);  // the persistent multi-layer kernel (mxq_linear_batch.cu)
 int linear_bf16_take_status(uint32_t *out);   // the BF16-weight comparison kernel (mxq_linear_bf16.cu)
 
+// Bounds-checked build (-DMXQ_DEBUG_BOUNDS): every translation unit with linear kernels keeps a record of global accesses
+// that fell outside their buffer (out[0] = how many; of the first: out[1] source line, out[2] byte offset, out[3] extent);
+// reading clears it.  In the ordinary build the functions report zeros.
+int bounds_take_linear(unsigned long long *out);        // mxq_linear.cu
+int bounds_take_linear_umma(unsigned long long *out);   // mxq_linear_umma.cu
+int bounds_take_linear_fp4(unsigned long long *out);    // mxq_linear_fp4.cu
+int bounds_take_linear_mma(unsigned long long *out);    // mxq_linear_mma.cu
+int bounds_take_linear_batch(unsigned long long *out);  // mxq_linear_batch.cu
+int bounds_take_linear_bf16(unsigned long long *out);   // mxq_linear_bf16.cu
+
 }  // namespace mxq

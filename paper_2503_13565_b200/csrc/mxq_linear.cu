@@ -27,11 +27,13 @@ namespace mxq {
 constexpr int kRowWarpThreads = 256;
 constexpr int kRowWarpRows = kRowWarpThreads / 32;
 
-__device__ __forceinline__ void store_y(void *Y, int y_dtype, int64_t idx, float v) {
+// (`count`: elements of Y, for the bounds-checked build)
+__device__ __forceinline__ void store_y(void *Y, int y_dtype, int64_t idx, float v, int64_t count) {
+    (void)count;
     if (y_dtype == MXQ_F32)
-        reinterpret_cast<float *>(Y)[idx] = v;
+        *MXQ_AT(reinterpret_cast<float *>(Y) + idx, 4, Y, count * 4) = v;
     else
-        reinterpret_cast<__nv_bfloat16 *>(Y)[idx] = __float2bfloat16_rn(v);
+        *MXQ_AT(reinterpret_cast<__nv_bfloat16 *>(Y) + idx, 2, Y, count * 2) = __float2bfloat16_rn(v);
 }
 
 // Generic kernel: any M <= MT, any N, any K % 32 == 0.  One warp per output row.
@@ -53,8 +55,8 @@ linear_rowwarp_kernel(const __nv_bfloat16 *__restrict__ X, int M, const uint4 *_
 
     pdl_wait();  // X may be the previous kernel's output
     for (int64_t j = lane; j < nblk; j += 32) {
-        const uint4 c = ld_stream_u4(crow + j);
-        const float s = e8m0_to_float(srow[j]);
+        const uint4 c = ld_stream_u4(MXQ_AT(crow + j, 16, codes, N * nblk * 16));
+        const float s = e8m0_to_float(*MXQ_AT(srow + j, 1, scales, N * nblk));
         const uint32_t w[4] = {c.x, c.y, c.z, c.w};
         float part[MT];
 #pragma unroll
@@ -68,7 +70,7 @@ linear_rowwarp_kernel(const __nv_bfloat16 *__restrict__ X, int M, const uint4 *_
 #pragma unroll
                 for (int m = 0; m < MT; ++m) {
                     if (m < M) {
-                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * K + k);
+                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(MXQ_AT(X + (int64_t)m * K + k, 4, X, (int64_t)M * K * 2));
                         part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
                         part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
                     }
@@ -81,7 +83,7 @@ linear_rowwarp_kernel(const __nv_bfloat16 *__restrict__ X, int M, const uint4 *_
 #pragma unroll
     for (int m = 0; m < MT; ++m) {
         const float v = warp_sum(acc[m]);
-        if (lane == 0 && m < M) store_y(Y, y_dtype, (int64_t)m * N + n, v);
+        if (lane == 0 && m < M) store_y(Y, y_dtype, (int64_t)m * N + n, v, (int64_t)M * N);
     }
 }
 
@@ -112,13 +114,14 @@ layer_epilogue_kernel(const float *__restrict__ S, int M, int64_t N, const void 
         const int64_t F = N >> 1;
         if (i >= (int64_t)M * F) return;
         const int64_t m = i / F, f = i - m * F;
-        const float g = S[m * N + 2 * f], u = S[m * N + 2 * f + 1];
-        store_y(Y, y_dtype, i, g / (1.f + expf(-g)) * u);
+        const float g = *MXQ_AT(S + m * N + 2 * f, 4, S, (int64_t)M * N * 4), u = *MXQ_AT(S + m * N + 2 * f + 1, 4, S, (int64_t)M * N * 4);
+        store_y(Y, y_dtype, i, g / (1.f + expf(-g)) * u, (int64_t)M * F);
     } else {
         if (i >= (int64_t)M * N) return;
-        const float r = y_dtype == MXQ_F32 ? reinterpret_cast<const float *>(residual)[i]
-                                           : __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(residual)[i]);
-        store_y(Y, y_dtype, i, S[i] + r);
+        const int64_t count = (int64_t)M * N;
+        const float r = y_dtype == MXQ_F32 ? *MXQ_AT(reinterpret_cast<const float *>(residual) + i, 4, residual, count * 4)
+                                           : __bfloat162float(*MXQ_AT(reinterpret_cast<const __nv_bfloat16 *>(residual) + i, 2, residual, count * 2));
+        store_y(Y, y_dtype, i, *MXQ_AT(S + i, 4, S, count * 4) + r, count);
     }
 }
 
@@ -128,9 +131,9 @@ __global__ void __launch_bounds__(256) stage_from_host_kernel(const uint4 *__res
     pdl_trigger();
     const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (i < n16) v = src[i];
+    if (i < n16) v = *MXQ_AT(src + i, 16, src, n16 * 16);
     pdl_wait();
-    if (i < n16) dst[i] = v;
+    if (i < n16) *MXQ_AT(dst + i, 16, dst, n16 * 16) = v;
 }
 
 // mxq_set_linear_kernel / MXQ_LINEAR_VARIANT: MXQ_KERNEL_AUTO (-1), or the highest kernel mxq_linear may use
@@ -190,10 +193,39 @@ static void choose(int ceiling, int M, int64_t N, int64_t K, const uint8_t *code
     else c.kernel = MXQ_KERNEL_GENERIC;
 }
 
+#ifdef MXQ_DEBUG_BOUNDS
+// mxq_debug_bounds_selftest: one store 100 bytes into a 64-byte buffer, through the checked address: it must be counted,
+// recorded and redirected (the buffer's neighbours stay as they were)
+__device__ uint32_t g_selftest_buf[16 + 64];
+__global__ void bounds_selftest_kernel() {
+    uint8_t *buf = reinterpret_cast<uint8_t *>(g_selftest_buf);
+    *MXQ_AT(reinterpret_cast<uint32_t *>(buf + 100), 4, buf, 64) = 0xDEADBEEFu;
+    *MXQ_AT(reinterpret_cast<uint32_t *>(buf + 60), 4, buf, 64) = 0x600DF00Du;   // the last word inside
+}
+#endif
+
+MXQ_BOUNDS_TU(bounds_take_linear)
+
 }  // namespace mxq
 
 extern "C" {
 #pragma GCC visibility push(default)
+int mxq_debug_bounds_selftest(void *stream) {
+#ifdef MXQ_DEBUG_BOUNDS
+    uint32_t zero[16 + 64] = {};
+    if (cudaMemcpyToSymbol(mxq::g_selftest_buf, zero, sizeof zero) != cudaSuccess) return MXQ_ERR_CUDA;
+    mxq::bounds_selftest_kernel<<<1, 1, 0, (cudaStream_t)stream>>>();
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MXQ_ERR_CUDA;
+    uint32_t got[16 + 64];
+    if (cudaMemcpyFromSymbol(got, mxq::g_selftest_buf, sizeof got) != cudaSuccess) return MXQ_ERR_CUDA;
+    for (int i = 0; i < 16 + 64; ++i)
+        if (got[i] != (i == 15 ? 0x600DF00Du : 0u)) return MXQ_ERR_SHAPE;   // the refused store landed in the buffer's neighbourhood
+    return MXQ_OK;
+#else
+    (void)stream;
+    return MXQ_ERR_SHAPE;   // not the bounds-checked build
+#endif
+}
 
 size_t mxq_linear_workspace_bytes(int M, int64_t N, int64_t K) {
     if (M < 1 || M > MXQ_MAX_M || !mxq::shape_ok(N, K)) return 0;

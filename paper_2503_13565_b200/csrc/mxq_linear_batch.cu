@@ -56,10 +56,11 @@ __device__ __forceinline__ float ld_cg_f32(const float *p) {
     return v;
 }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
-__device__ __forceinline__ float load_in_cg(const void *R, int dtype, int64_t idx) {
-    if (dtype == MXQ_F32) return ld_cg_f32(reinterpret_cast<const float *>(R) + idx);
+__device__ __forceinline__ float load_in_cg(const void *R, int dtype, int64_t idx, int64_t count) {
+    (void)count;
+    if (dtype == MXQ_F32) return ld_cg_f32(MXQ_AT(reinterpret_cast<const float *>(R) + idx, 4, R, count * 4));
     unsigned short h;
-    asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(h) : "l"(reinterpret_cast<const unsigned short *>(R) + idx) : "memory");
+    asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(h) : "l"(MXQ_AT(reinterpret_cast<const unsigned short *>(R) + idx, 2, R, count * 2)) : "memory");
     return __uint_as_float((uint32_t)h << 16);
 }
 
@@ -427,7 +428,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                     if (c.d != d_seen) ok = layer(c);
                     if (!ok) break;
                     mbar_expect_tx(o_fb, kXBytes);
-                    bulk_load(o_slot + kBatchCodesBytes + kBatchSfBytes, img + (uint32_t)c.s * kXBytes, kXBytes, o_fb);
+                    bulk_load(o_slot + kBatchCodesBytes + kBatchSfBytes, MXQ_AT(img + (uint32_t)c.s * kXBytes, kXBytes, tb.ws, tb.ws_bytes), kXBytes, o_fb);
                     o_slot += kSlot;
                     o_fb += 8u;
                     if (o_slot == ring_end) {
@@ -449,7 +450,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                     }
                     mbar_expect_tx(c_fb, kBatchCodesBytes + kXBytes);
                     if (walk_unit(wk, i) != tb.fault_unit) tma_load_codes(c_slot, map, c.s * (kBatchStageK / 2), c.t * kBatchTileRows, c_fb);
-                    bulk_load(c_slot + kBatchCodesBytes + kBatchSfBytes, img + (uint32_t)c.s * kXBytes, kXBytes, c_fb);
+                    bulk_load(c_slot + kBatchCodesBytes + kBatchSfBytes, MXQ_AT(img + (uint32_t)c.s * kXBytes, kXBytes, tb.ws, tb.ws_bytes), kXBytes, c_fb);
                     ++issued;
                     c_slot += kSlot;
                     c_fb += 8u;
@@ -501,10 +502,10 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                 lo[q] = hi[q] = 0u;
                 if (n0 + 32 * q < ds.N) {
                     if (wide) {
-                        asm volatile("ld.global.nc.v2.u32 {%0,%1}, [%2];" : "=r"(lo[q]), "=r"(hi[q]) : "l"(src));
+                        asm volatile("ld.global.nc.v2.u32 {%0,%1}, [%2];" : "=r"(lo[q]), "=r"(hi[q]) : "l"(MXQ_AT(src, 8, ds.scales, (int64_t)ds.N * kb_row)));
                     } else {
-                        asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(lo[q]) : "l"(src));
-                        if (second) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(hi[q]) : "l"(src + 4));
+                        asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(lo[q]) : "l"(MXQ_AT(src, 4, ds.scales, (int64_t)ds.N * kb_row)));
+                        if (second) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(hi[q]) : "l"(MXQ_AT(src + 4, 4, ds.scales, (int64_t)ds.N * kb_row)));
                     }
                 }
                 src += (int64_t)32 * kb_row;
@@ -596,16 +597,16 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
             const int local = task - gi.task_base;
             const int k128 = local / M, m = local - k128 * M;
             const int kk = k128 * 128 + (lane >> 1) * 8;
-            const uint4 raw = ld_cg_u4(reinterpret_cast<const __nv_bfloat16 *>(gi.X) + (int64_t)m * gi.K + kk);
+            const uint4 raw = ld_cg_u4(MXQ_AT(reinterpret_cast<const __nv_bfloat16 *>(gi.X) + (int64_t)m * gi.K + kk, 16, gi.X, (int64_t)M * gi.K * 2));
             uint8_t *stage = tb.ws + gi.offset + (size_t)(kk >> 8) * kXBytes;
-            bool inexact = split_half_unit_to(raw, m, (uint32_t)kk & 255u, lane & 1, lane, SplitToGlobal{stage},
-                                              SplitToGlobal{stage + (uint32_t)NB * 128u});
+            bool inexact = split_half_unit_to(raw, m, (uint32_t)kk & 255u, lane & 1, lane, SplitToGlobal{stage, tb.ws, tb.ws_bytes},
+                                              SplitToGlobal{stage + (uint32_t)NB * 128u, tb.ws, tb.ws_bytes});
             if (__any_sync(0xffffffffu, inexact)) {
                 // (rare, and kept off the common path, whose length every launch pays for: the rewriting is done again,
                 // this time asking for what the planes cannot hold)
                 float rem[8];
-                inexact = split_half_unit_to(raw, m, (uint32_t)kk & 255u, lane & 1, lane, SplitToGlobal{stage},
-                                             SplitToGlobal{stage + (uint32_t)NB * 128u}, rem);
+                inexact = split_half_unit_to(raw, m, (uint32_t)kk & 255u, lane & 1, lane, SplitToGlobal{stage, tb.ws, tb.ws_bytes},
+                                             SplitToGlobal{stage + (uint32_t)NB * 128u, tb.ws, tb.ws_bytes}, rem);
                 // Elements that do not fit the block's fixed point (more than 24 binades under the block's maximum; any
                 // element of a block with an Inf or a NaN): the planes hold them truncated, and what is missing goes on the
                 // image's list of corrections (token row, k, remainder), which the epilogues add as remainder * weight.  A
@@ -617,9 +618,10 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                         if (rem[e] != 0.f) {   // (NaN included)
                             const uint32_t at = atomicAdd(g_bad + im * kBatchCounterStride + 1, 1u);
                             if (at < (uint32_t)kBatchMaxFixes) {
-                                fixes[at].m = m;
-                                fixes[at].k = kk + e;
-                                fixes[at].rem = rem[e];
+                                BatchFix *fx = MXQ_AT(fixes + at, sizeof(BatchFix), tb.ws, tb.ws_bytes);
+                                fx->m = m;
+                                fx->k = kk + e;
+                                fx->rem = rem[e];
                             } else {
                                 atomicOr(g_bad + im * kBatchCounterStride, 1u);
                             }
@@ -702,8 +704,8 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                     const __nv_bfloat16 *X = reinterpret_cast<const __nv_bfloat16 *>(ds.X);
                     const int blk_end = min(s_end * 8, kb_row);
                     for (int blk = s_begin * 8; blk < blk_end; ++blk) {
-                        const uint4 cc = ld_stream_u4(crow + blk);
-                        const float sc = e8m0_to_float(srw[blk]) * kGuardDown;
+                        const uint4 cc = ld_stream_u4(MXQ_AT(crow + blk, 16, ds.codes, (int64_t)ds.N * (ds.K / 2)));
+                        const float sc = e8m0_to_float(*MXQ_AT(srw + blk, 1, ds.scales, (int64_t)ds.N * kb_row)) * kGuardDown;
                         const uint32_t w[4] = {cc.x, cc.y, cc.z, cc.w};
                         float part[MT];
 #pragma unroll
@@ -718,7 +720,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                                 for (int m = 0; m < MT; ++m)
                                     if (m < M) {
                                         uint32_t xb;
-                                        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(xb) : "l"(X + (int64_t)m * ds.K + k) : "memory");
+                                        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(xb) : "l"(MXQ_AT(X + (int64_t)m * ds.K + k, 4, ds.X, (int64_t)M * ds.K * 2)) : "memory");
                                         part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
                                         part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
                                     }
@@ -745,13 +747,13 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                 float *mine = partials + ((size_t)(cta * 2 + (head ? 0 : 1)) * MT) * 128u;
 #pragma unroll
                 for (int m = 0; m < MT; ++m)
-                    if (m < M) mine[m * 128 + row] = yt[m];
+                    if (m < M) *MXQ_AT(mine + m * 128 + row, 4, tb.ws, tb.ws_bytes) = yt[m];
                 // The barrier orders the 128 threads' stores before thread 0's ticket, whose release (cumulative, GPU scope)
                 // publishes them; its acquire, passed on through the next barrier, lets a finisher read the other parts.
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (et == 0) {
                     uint32_t old;
-                    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(g_ticket + c_first) : "memory");
+                    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(MXQ_AT(g_ticket + c_first, 4, tb.ws, kBatchHeaderBytes)) : "memory");
                     *s_flag = (int)old;
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -767,7 +769,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                         const float *part = partials + ((size_t)(cj * 2 + (hj ? 0 : 1)) * MT) * 128u;
 #pragma unroll
                         for (int m = 0; m < MT; ++m)
-                            if (m < M) sum[m] += ld_cg_f32(part + m * 128 + row);
+                            if (m < M) sum[m] += ld_cg_f32(MXQ_AT(part + m * 128 + row, 4, tb.ws, tb.ws_bytes));
                     }
 #pragma unroll
                     for (int m = 0; m < MT; ++m) yt[m] = sum[m];
@@ -783,11 +785,11 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                     const BatchFix *fixes = reinterpret_cast<const BatchFix *>(tb.ws + tb.fix_offset) + (size_t)im * kBatchMaxFixes;
                     const uint32_t nfix = min(*reinterpret_cast<volatile uint32_t *>(g_bad + im * kBatchCounterStride + 1), (uint32_t)kBatchMaxFixes);
                     for (uint32_t e = 0; e < nfix; ++e) {
-                        const uint4 fx = ld_cg_u4(fixes + e);   // (written by another SM during this kernel: through L2)
+                        const uint4 fx = ld_cg_u4(MXQ_AT(fixes + e, 16, tb.ws, tb.ws_bytes));   // (written by another SM during this kernel: through L2)
                         const int fm = (int)fx.x, fk = (int)fx.y;
-                        const uint32_t byte = ds.codes[(int64_t)n * (ds.K / 2) + (fk >> 1)];
+                        const uint32_t byte = *MXQ_AT(ds.codes + (int64_t)n * (ds.K / 2) + (fk >> 1), 1, ds.codes, (int64_t)ds.N * (ds.K / 2));
                         const float2 wv = __half22float2(e2m1x2_to_half2(byte));
-                        const float wgt = ((fk & 1) ? wv.y : wv.x) * e8m0_to_float(ds.scales[(int64_t)n * (ds.K >> 5) + (fk >> 5)]);
+                        const float wgt = ((fk & 1) ? wv.y : wv.x) * e8m0_to_float(*MXQ_AT(ds.scales + (int64_t)n * (ds.K >> 5) + (fk >> 5), 1, ds.scales, (int64_t)ds.N * (ds.K >> 5)));
                         const float add = __uint_as_float(fx.z) * wgt;
 #pragma unroll
                         for (int m = 0; m < MT; ++m)
@@ -805,7 +807,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                     if (n < ds.N && (n & 1) == 0) {
 #pragma unroll
                         for (int m = 0; m < MT; ++m)
-                            if (m < M) store_out(ds.Y, ds.y_dtype, (int64_t)m * (ds.N >> 1) + (n >> 1), y[m]);
+                            if (m < M) store_out(ds.Y, ds.y_dtype, (int64_t)m * (ds.N >> 1) + (n >> 1), y[m], (int64_t)M * (ds.N >> 1));
                     }
                 } else if (n < ds.N) {
 #pragma unroll
@@ -813,8 +815,8 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                         if (m < M) {
                             const int64_t at = (int64_t)m * ds.N + n;
                             // (through L2: in a call of several groups another SM may have written the residual during this kernel)
-                            const float r = ds.epi == 1 ? load_in_cg(ds.residual, ds.y_dtype, at) : 0.f;
-                            store_out(ds.Y, ds.y_dtype, at, yt[m] + r);
+                            const float r = ds.epi == 1 ? load_in_cg(ds.residual, ds.y_dtype, at, (int64_t)M * ds.N) : 0.f;
+                            store_out(ds.Y, ds.y_dtype, at, yt[m] + r, (int64_t)M * ds.N);
                         }
                 }
                 if (ngroups > 1) {
@@ -938,6 +940,8 @@ static size_t batch_workspace_bytes(const mxq_linear_desc *descs, int count, int
     return (b + 255u) & ~(size_t)255u;
 }
 
+MXQ_BOUNDS_TU(bounds_take_linear_batch)
+
 }  // namespace mxq
 
 extern "C" {
@@ -1014,7 +1018,8 @@ int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *works
     if (rc != MXQ_OK) return rc;
     if (!workspace) return MXQ_ERR_NULL;
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MXQ_ERR_ALIGN;
-    if (workspace_bytes < mxq_linear_batch_workspace_bytes(descs, count, M)) return MXQ_ERR_WORKSPACE;
+    const size_t ws_needed = mxq_linear_batch_workspace_bytes(descs, count, M);
+    if (workspace_bytes < ws_needed) return MXQ_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     mxq::BatchLayout L;
     int64_t units = 0, cur = 0;   // units of the largest group
@@ -1040,6 +1045,7 @@ int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *works
     std::memset(&tb, 0, sizeof tb);
     const int nb = L.nb;
     tb.ws = static_cast<uint8_t *>(workspace);
+    tb.ws_bytes = ws_needed;   // (what this call may touch, however large the caller's buffer)
     tb.ndesc = count;
     tb.M = M;
     tb.ring = L.ring;

@@ -110,6 +110,7 @@ struct BatchTable {
     uint32_t wait_us;            // limit of every wait inside the kernel
     uint32_t partials_offset;    // bytes from the workspace base
     uint32_t fix_offset;         // lists of corrections, bytes from the workspace base
+    uint64_t ws_bytes;           // size of the workspace (bounds-checked build)
 };
 
 }  // namespace mxq

@@ -200,7 +200,7 @@ linear_bf16_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
             if (n < N)
 #pragma unroll
                 for (int m = 0; m < 16; ++m)
-                    if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, d[m]);
+                    if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, d[m], (int64_t)M * N);
         } else {
             // as in the MXFP4 kernels: partial rows go to the rank that owns them, which adds them in a fixed order
             const int cnt_max = (kTileRows + split - 1) / split;
@@ -221,7 +221,7 @@ linear_bf16_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
                 float acc = 0.f;
                 for (int j = 0; j < split; ++j) acc += gRecv[(j * M + m) * cnt_max + r];
                 const int64_t n = n0 + row_lo + r;
-                if (n < N) store_out(Y, y_dtype, (int64_t)m * N + n, acc + poison);
+                if (n < N) store_out(Y, y_dtype, (int64_t)m * N + n, acc + poison, (int64_t)M * N);
             }
         }
     }
@@ -241,12 +241,12 @@ linear_bf16_rowwarp_kernel(const __nv_bfloat16 *__restrict__ X, int M, const __n
     for (int m = 0; m < kMaxM; ++m) acc[m] = 0.f;
     pdl_wait();
     for (int64_t k = lane * 2; k < K; k += 64) {
-        const uint32_t wb = *reinterpret_cast<const uint32_t *>(W + n * K + k);
+        const uint32_t wb = *reinterpret_cast<const uint32_t *>(MXQ_AT(W + n * K + k, 4, W, N * K * 2));
         const float w0 = __uint_as_float(wb << 16), w1 = __uint_as_float(wb & 0xFFFF0000u);
 #pragma unroll
         for (int m = 0; m < kMaxM; ++m)
             if (m < M) {
-                const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * K + k);
+                const uint32_t xb = *reinterpret_cast<const uint32_t *>(MXQ_AT(X + (int64_t)m * K + k, 4, X, (int64_t)M * K * 2));
                 acc[m] = fmaf(w0, __uint_as_float(xb << 16), acc[m]);
                 acc[m] = fmaf(w1, __uint_as_float(xb & 0xFFFF0000u), acc[m]);
             }
@@ -256,7 +256,7 @@ linear_bf16_rowwarp_kernel(const __nv_bfloat16 *__restrict__ X, int M, const __n
         float v = acc[m];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0 && m < M) store_out(Y, y_dtype, (int64_t)m * N + n, v);
+        if (lane == 0 && m < M) store_out(Y, y_dtype, (int64_t)m * N + n, v, (int64_t)M * N);
     }
 }
 
@@ -269,6 +269,8 @@ int linear_bf16_take_status(uint32_t *out) {
     *out = v;
     return MXQ_OK;
 }
+
+MXQ_BOUNDS_TU(bounds_take_linear_bf16)
 
 }  // namespace mxq
 

@@ -123,8 +123,8 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             if (lane + 32 * q < rows_here) {
-                cp_async4(dst + 4 * q, src);
-                if (second) cp_async4(dst + 4 * q + 512, src + 4);
+                cp_async4(dst + 4 * q, MXQ_AT(src, 4, scales, N * kb_row));
+                if (second) cp_async4(dst + 4 * q + 512, MXQ_AT(src + 4, 4, scales, N * kb_row));
             }
             src += srow_step;
         }
@@ -318,7 +318,7 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                         stage[b] = st;
                         mm[b] = tail ? rem : (rem >> 1);
                         kk[b] = st * kFp4StageK + (tail ? 0 : (rem & 1) * 128) + (lane >> 1) * 8;
-                        raw[b] = ld_ordered_u4(xbase + (int64_t)mm[b] * K + kk[b]);
+                        raw[b] = ld_ordered_u4(MXQ_AT(xbase + (int64_t)mm[b] * K + kk[b], 16, X, (int64_t)M * K * 2));
                     }
                 }
                 // The activations have been asked for: weight copies requested from here on queue up behind them, so
@@ -397,8 +397,8 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                     const uint4 *crow = reinterpret_cast<const uint4 *>(codes + n * (K / 2));
                     const uint8_t *srw = scales + n * kb_row;
                     for (int blk = k_begin / 32; blk < (k_begin + k_len) / 32; ++blk) {
-                        const uint4 c = ld_stream_u4(crow + blk);
-                        const float sc = e8m0_to_float(srw[blk]) * kGuardDown;
+                        const uint4 c = ld_stream_u4(MXQ_AT(crow + blk, 16, codes, N * (K / 2)));
+                        const float sc = e8m0_to_float(*MXQ_AT(srw + blk, 1, scales, N * kb_row)) * kGuardDown;
                         const uint32_t w[4] = {c.x, c.y, c.z, c.w};
                         float part[kFp4MaxM];
 #pragma unroll
@@ -412,7 +412,7 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
 #pragma unroll
                                 for (int m = 0; m < kFp4MaxM; ++m)
                                     if (m < M) {
-                                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * K + k);
+                                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(MXQ_AT(X + (int64_t)m * K + k, 4, X, (int64_t)M * K * 2));
                                         part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
                                         part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
                                     }
@@ -452,7 +452,7 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                                     besti[m] = (uint32_t)n;
                                 }
                             } else {
-                                store_out(Y, y_dtype, (int64_t)m * N + n, yt[m] * kGuardUp);
+                                store_out(Y, y_dtype, (int64_t)m * N + n, yt[m] * kGuardUp, (int64_t)M * N);
                             }
                         }
             } else {
@@ -484,12 +484,12 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                         if (EPI == kEpiLayer) {
                             // (gate / up calls are planned with power-of-two clusters and never come here)
                             const int64_t at = (int64_t)m * N + n;
-                            store_out(Y, y_dtype, at, acc * kGuardUp + poison + load_in(fa.residual, y_dtype, at));
+                            store_out(Y, y_dtype, at, acc * kGuardUp + poison + load_in(fa.residual, y_dtype, at, (int64_t)M * N), (int64_t)M * N);
                         } else if (fa.keys) {
                             const unsigned long long key = argmax_key(acc * kGuardUp + poison, (uint32_t)n);
                             if (key) atomicMax(s_keys + m, key);   // (rare decomposition: straight into shared memory)
                         } else {
-                            store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison);
+                            store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison, (int64_t)M * N);
                         }
                     }
                 }
@@ -526,7 +526,7 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
                                         besti[m] = (uint32_t)n;
                                     }
                                 } else {
-                                    store_out(Y, y_dtype, (int64_t)m * N + n, w);
+                                    store_out(Y, y_dtype, (int64_t)m * N + n, w, (int64_t)M * N);
                                 }
                             }
                     }
@@ -638,5 +638,7 @@ int linear_fp4_take_status(uint32_t *out) {
     *out = v;
     return MXQ_OK;
 }
+
+MXQ_BOUNDS_TU(bounds_take_linear_fp4)
 
 }  // namespace mxq

@@ -109,11 +109,13 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1,
 // ---------------------------------------------------------------------------------------------
 constexpr uint32_t kFlagSegLast = 1, kFlagWinFirst = 2;
 
-__device__ __forceinline__ void store_out(void *Y, int y_dtype, int64_t idx, float v) {
+// (`count`: elements of Y, for the bounds-checked build)
+__device__ __forceinline__ void store_out(void *Y, int y_dtype, int64_t idx, float v, int64_t count) {
+    (void)count;
     if (y_dtype == MXQ_F32)
-        reinterpret_cast<float *>(Y)[idx] = v;
+        *MXQ_AT(reinterpret_cast<float *>(Y) + idx, 4, Y, count * 4) = v;
     else
-        reinterpret_cast<__nv_bfloat16 *>(Y)[idx] = __float2bfloat16_rn(v);
+        *MXQ_AT(reinterpret_cast<__nv_bfloat16 *>(Y) + idx, 2, Y, count * 2) = __float2bfloat16_rn(v);
 }
 
 __device__ __forceinline__ uint32_t max_abs_bits(const uint4 &v) {  // largest BF16 magnitude pattern of 8 values
@@ -211,18 +213,18 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
         if (left > 0) {
             const uint32_t dst = ring + (uint32_t)slot * kWarpStageBytes;
             const bool lo_ok = cr <= rows_m1, hi_ok = cr + 8 <= rows_m1, sc_ok = (uint32_t)(lane & 15) <= rows_m1;
-            if (lo_ok) cp_async16(dst + dst_a, src_lo + e.x);
-            if (hi_ok) cp_async16(dst + dst_a + 1024, src_hi + e.x);
+            if (lo_ok) cp_async16(dst + dst_a, MXQ_AT(src_lo + e.x, 16, codes, (int64_t)p.N * (p.K / 2)));
+            if (hi_ok) cp_async16(dst + dst_a + 1024, MXQ_AT(src_hi + e.x, 16, codes, (int64_t)p.N * (p.K / 2)));
             if (left > 4) {
-                if (lo_ok) cp_async16(dst + dst_b, src_lo + e.x + 64);
-                if (hi_ok) cp_async16(dst + dst_b + 1024, src_hi + e.x + 64);
+                if (lo_ok) cp_async16(dst + dst_b, MXQ_AT(src_lo + e.x + 64, 16, codes, (int64_t)p.N * (p.K / 2)));
+                if (hi_ok) cp_async16(dst + dst_b + 1024, MXQ_AT(src_hi + e.x + 64, 16, codes, (int64_t)p.N * (p.K / 2)));
                 if (sc8) {
-                    if (lane < 16 && sc_ok) cp_async8(dst + dst_sc, src_sc + e.y);
+                    if (lane < 16 && sc_ok) cp_async8(dst + dst_sc, MXQ_AT(src_sc + e.y, 8, scales, (int64_t)p.N * p.kb));
                 } else if (sc_ok) {
-                    cp_async4(dst + dst_sc, src_sc + e.y);
+                    cp_async4(dst + dst_sc, MXQ_AT(src_sc + e.y, 4, scales, (int64_t)p.N * p.kb));
                 }
             } else if (lane < 16 && sc_ok) {
-                cp_async4(dst + dst_sc, src_sc + e.y);
+                cp_async4(dst + dst_sc, MXQ_AT(src_sc + e.y, 4, scales, (int64_t)p.N * p.kb));
             }
         }
     };
@@ -282,13 +284,13 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
                 keep[i] = make_uint4(0, 0, 0, 0);
                 if (v < nvec) {
                     const int m = v / vec_per_row, c = v - m * vec_per_row;
-                    keep[i] = __ldcg(reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0) + c);
+                    keep[i] = __ldcg(MXQ_AT(reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0) + c, 16, X, (int64_t)p.M * p.K * 2));
                 }
                 mx = max(mx, max_abs_bits(keep[i]));
             }
             for (int v = tid + kKeep * kMmaThreads; v < nvec; v += kMmaThreads) {
                 const int m = v / vec_per_row, c = v - m * vec_per_row;
-                mx = max(mx, max_abs_bits(__ldcg(reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0) + c)));
+                mx = max(mx, max_abs_bits(__ldcg(MXQ_AT(reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0) + c, 16, X, (int64_t)p.M * p.K * 2))));
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -313,7 +315,7 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
             for (int v = tid + kKeep * kMmaThreads; v < nvec; v += kMmaThreads) {
                 const int m = v / vec_per_row, c = v - m * vec_per_row;
                 uint4 out;
-                inexact |= bf16x8_to_f16x8(__ldcg(reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0) + c), up, out);
+                inexact |= bf16x8_to_f16x8(__ldcg(MXQ_AT(reinterpret_cast<const uint4 *>(X + (int64_t)m * p.K + k0) + c, 16, X, (int64_t)p.M * p.K * 2)), up, out);
                 *reinterpret_cast<uint4 *>(smem + p.off_x + (size_t)m * p.x_stride + (size_t)c * 16) = out;
             }
             if (inexact) atomicOr(&s_inexact[0], 1);
@@ -425,8 +427,8 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
                 for (int m = 0; m < p.M; ++m) {
                     float a = 0.f;
                     for (int j = lane; j < bwid; j += 32) {
-                        const uint4 c = ld_stream_u4(codes + row * (p.K / 2) + (j0 + j) * 16);
-                        const float s = e8m0_to_float(scales[row * p.kb + j0 + j]);
+                        const uint4 c = ld_stream_u4(MXQ_AT(codes + row * (p.K / 2) + (j0 + j) * 16, 16, codes, (int64_t)p.N * (p.K / 2)));
+                        const float s = e8m0_to_float(*MXQ_AT(scales + row * p.kb + j0 + j, 1, scales, (int64_t)p.N * p.kb));
                         const uint32_t w4[4] = {c.x, c.y, c.z, c.w};
                         const uint16_t *xr = X + (int64_t)m * p.K + (j0 + j) * kBlock;
                         float part = 0.f;
@@ -435,7 +437,7 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 const float2 wv = __half22float2(e2m1x2_to_half2((w4[qd] >> (8 * i)) & 0xFFu));
-                                const uint32_t xb = __ldcg(reinterpret_cast<const uint32_t *>(xr + qd * 8 + i * 2));
+                                const uint32_t xb = __ldcg(MXQ_AT(reinterpret_cast<const uint32_t *>(xr + qd * 8 + i * 2), 4, X, (int64_t)p.M * p.K * 2));
                                 part = fmaf(wv.x, __uint_as_float(xb << 16), part);
                                 part = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part);
                             }
@@ -484,7 +486,7 @@ linear_mma_kernel(const __grid_constant__ LinearPlan p, const uint16_t *__restri
                 for (int i = 0; i < kPerLane; ++i) {
                     const int idx = lane + 32 * i, m_out = idx / kTileRows;
                     const int64_t n_out = r0 + (int64_t)tile_now * kTileRows + idx % kTileRows;
-                    if (m_out < p.M && n_out < r1) store_out(Y, y_dtype, (int64_t)m_out * p.N + n_out, val[i]);
+                    if (m_out < p.M && n_out < r1) store_out(Y, y_dtype, (int64_t)m_out * p.N + n_out, val[i], (int64_t)p.M * p.N);
                 }
             }
         }
@@ -591,5 +593,7 @@ int linear_mma_take_status(uint32_t *out) {
     *out = v;
     return MXQ_OK;
 }
+
+MXQ_BOUNDS_TU(bounds_take_linear_mma)
 
 }  // namespace mxq

@@ -65,7 +65,11 @@ __device__ __forceinline__ uint32_t pack_e5m2x2(float lo, float hi) {
 // One 8-element unit of X (token m, k offset kk inside the CTA's range): split into parts, store into B and SFB.
 // All 32 lanes call it together (the block maximum crosses the four lanes of a 32-block by shuffle).
 template <int NB>
-__device__ __forceinline__ bool split_unit(const uint4 raw, bool act, int m, int kk, int lane, uint8_t *gB, uint8_t *gSFB) {
+// (b_bytes, sf_bytes: sizes of the two destinations, for the bounds-checked build)
+__device__ __forceinline__ bool split_unit(const uint4 raw, bool act, int m, int kk, int lane, uint8_t *gB, uint8_t *gSFB, size_t b_bytes,
+                                           size_t sf_bytes) {
+    (void)b_bytes;
+    (void)sf_bytes;
     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
     bool inexact = false;
     uint32_t emax = 0;
@@ -105,9 +109,10 @@ __device__ __forceinline__ bool split_unit(const uint4 raw, bool act, int m, int
         for (int p = 0; p < 3; ++p) {
             const int row = 3 * m + p;
             uint8_t *dst = gB + (size_t)j * (NB * 128) + (row >> 3) * 1024 + ((kk >> 4) & 7) * 128 + (row & 7) * 16 + (kk & 15);
-            *reinterpret_cast<uint2 *>(dst) = make_uint2(part[p][0], part[p][1]);
+            *reinterpret_cast<uint2 *>(MXQ_AT(dst, 8, gB, b_bytes)) = make_uint2(part[p][0], part[p][1]);
             if ((lane & 3) == 0)
-                gSFB[(size_t)j * kUmmaSfStageBytes + (row & 31) * 16 + (row >> 5) * 4 + ((kk >> 5) & 3)] = (uint8_t)(sb1 - kGuard - 3 * p);
+                *MXQ_AT(gSFB + (size_t)j * kUmmaSfStageBytes + (row & 31) * 16 + (row >> 5) * 4 + ((kk >> 5) & 3), 1, gSFB, sf_bytes) =
+                    (uint8_t)(sb1 - kGuard - 3 * p);
         }
     }
     return inexact && act;
@@ -134,18 +139,19 @@ split_tokens_kernel(const __nv_bfloat16 *__restrict__ X, int M, int64_t K, int k
     for (int q = 0; q < (kUmmaMaxM + kSplitWarps - 1) / kSplitWarps; ++q) {
         const int m = warp + q * kSplitWarps;
         raw[q] = make_uint4(0, 0, 0, 0);
-        if (m < M && act) raw[q] = *reinterpret_cast<const uint4 *>(X + (int64_t)m * K + kk);
+        if (m < M && act) raw[q] = *reinterpret_cast<const uint4 *>(MXQ_AT(X + (int64_t)m * K + kk, 16, X, (int64_t)M * K * 2));
     }
     bool inexact = false;
 #pragma unroll
     for (int q = 0; q < (kUmmaMaxM + kSplitWarps - 1) / kSplitWarps; ++q) {
         const int m = warp + q * kSplitWarps;
-        if (m < M) inexact |= split_unit<NB>(raw[q], act, m, kk, lane, gB, gSFB);   // uniform across the warp
+        if (m < M)   // uniform across the warp
+            inexact |= split_unit<NB>(raw[q], act, m, kk, lane, gB, gSFB, (size_t)ks * (NB * 128), (size_t)ks * kUmmaSfStageBytes);
     }
     if (inexact) s_bad = 1;
     __syncthreads();
     const int stage = (int)blockIdx.x * 2 + (int)threadIdx.x;
-    if (threadIdx.x < 2 && stage < ks) reinterpret_cast<uint32_t *>(ws)[stage] = (uint32_t)s_bad;
+    if (threadIdx.x < 2 && stage < ks) *MXQ_AT(reinterpret_cast<uint32_t *>(ws) + stage, 4, ws, umma_ws_flags_bytes(ks)) = (uint32_t)s_bad;
 }
 
 template <int NB>
@@ -238,7 +244,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
         const int rows_here = (int)min((int64_t)kUmmaTileRows, N - n0 - (int64_t)t * kUmmaTileRows);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            if (lane + 32 * q < rows_here) cp_async4(dst + 4 * q, src);
+            if (lane + 32 * q < rows_here) cp_async4(dst + 4 * q, MXQ_AT(src, 4, scales, N * kb_row));
             src += srow_step;
         }
         cp_async_arrive(full0 + slot * 8);
@@ -251,8 +257,11 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
     const uint8_t *ws_b = presplit ? ws_sf + (size_t)ks * kUmmaSfStageBytes : nullptr;
     auto copy_tokens = [&](int i, uint32_t slot) {     // one lane; bring only: stage i of the token operand into ring slot `slot`
         mbar_expect_tx(full0 + slot * 8, NB * 128u + kUmmaSfStageBytes);
-        bulk_load(sB + slot * (NB * 128u), ws_b + (size_t)(s_begin + i) * (NB * 128u), NB * 128u, full0 + slot * 8);
-        bulk_load(sSFB + slot * kUmmaSfStageBytes, ws_sf + (size_t)(s_begin + i) * kUmmaSfStageBytes, kUmmaSfStageBytes, full0 + slot * 8);
+        bulk_load(sB + slot * (NB * 128u), MXQ_AT(ws_b + (size_t)(s_begin + i) * (NB * 128u), NB * 128u, ws_b, (size_t)ks * (NB * 128u)), NB * 128u,
+                  full0 + slot * 8);
+        bulk_load(sSFB + slot * kUmmaSfStageBytes,
+                  MXQ_AT(ws_sf + (size_t)(s_begin + i) * kUmmaSfStageBytes, kUmmaSfStageBytes, ws_sf, (size_t)ks * kUmmaSfStageBytes), kUmmaSfStageBytes,
+                  full0 + slot * 8);
     };
     if (warp == 1) {
         for (int b = lane; b < 2 * ring + 2 + npair; b += 32) {
@@ -417,14 +426,16 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                 for (int p = 0; p < npair; ++p) {
                     const uint32_t n2 = (uint32_t)min(2, nst - 2 * p), bar = ready0 + (uint32_t)p * 8u;
                     mbar_expect_tx(bar, n2 * (NB * 128u + kUmmaSfStageBytes));
-                    bulk_load(sB + (uint32_t)(2 * p) * (NB * 128u), ws_b + (size_t)(s_begin + 2 * p) * (NB * 128u), n2 * (NB * 128u), bar);
-                    bulk_load(sSFB + (uint32_t)(2 * p) * kUmmaSfStageBytes, ws_sf + (size_t)(s_begin + 2 * p) * kUmmaSfStageBytes,
+                    bulk_load(sB + (uint32_t)(2 * p) * (NB * 128u),
+                              MXQ_AT(ws_b + (size_t)(s_begin + 2 * p) * (NB * 128u), n2 * (NB * 128u), ws_b, (size_t)ks * (NB * 128u)), n2 * (NB * 128u), bar);
+                    bulk_load(sSFB + (uint32_t)(2 * p) * kUmmaSfStageBytes,
+                              MXQ_AT(ws_sf + (size_t)(s_begin + 2 * p) * kUmmaSfStageBytes, n2 * kUmmaSfStageBytes, ws_sf, (size_t)ks * kUmmaSfStageBytes),
                               n2 * kUmmaSfStageBytes, bar);
                 }
                 s_xin = 1;   // lets the producer request the rest of the ring
             }
             const uint32_t *flags = reinterpret_cast<const uint32_t *>(presplit);
-            for (int i = ct; i < nst; i += 128) inexact |= flags[s_begin + i] != 0u;
+            for (int i = ct; i < nst; i += 128) inexact |= *MXQ_AT(flags + s_begin + i, 4, flags, umma_ws_flags_bytes(ks)) != 0u;
         } else {
             // Groups of 32 units (256 k of one token, one warp; a unit is 8 elements, one lane) in order of K, so that
             // the MMA warp can start on the first stages while later ones are being split.  Group G: pair of stages
@@ -449,13 +460,13 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                         mm[b] = G - pair[b] * M;
                         kk[b] = pair[b] * (2 * kUmmaStageK) + lane * 8;
                         act[b] = kk[b] < k_len;
-                        if (act[b]) raw[b] = *reinterpret_cast<const uint4 *>(xbase + (int64_t)mm[b] * K + kk[b]);
+                        if (act[b]) raw[b] = *reinterpret_cast<const uint4 *>(MXQ_AT(xbase + (int64_t)mm[b] * K + kk[b], 16, X, (int64_t)M * K * 2));
                     }
                 }
 #pragma unroll
                 for (int b = 0; b < kBatch; ++b)
                     if (G0 + 4 * b + cw < ngroups) {   // uniform across the warp
-                        inexact |= split_unit<NB>(raw[b], act[b], mm[b], kk[b], lane, gB, gSFB);
+                        inexact |= split_unit<NB>(raw[b], act[b], mm[b], kk[b], lane, gB, gSFB, (size_t)nbslot * (NB * 128), (size_t)nbslot * kUmmaSfStageBytes);
                         if (G0 == 0 && b == 0 && ct == 0) s_xin = 1;   // lets the producer request the rest of the ring
                         fence_async_proxy();   // ordinary stores, read by the tensor core
                         __syncwarp();
@@ -527,8 +538,8 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                     const uint4 *crow = reinterpret_cast<const uint4 *>(codes + n * (K / 2));
                     const uint8_t *srw = scales + n * kb_row;
                     for (int blk = k_begin / 32; blk < (k_begin + k_len) / 32; ++blk) {
-                        const uint4 c = ld_stream_u4(crow + blk);
-                        const float sc = e8m0_to_float(srw[blk]) * kGuardDown;
+                        const uint4 c = ld_stream_u4(MXQ_AT(crow + blk, 16, codes, N * (K / 2)));
+                        const float sc = e8m0_to_float(*MXQ_AT(srw + blk, 1, scales, N * kb_row)) * kGuardDown;
                         const uint32_t w[4] = {c.x, c.y, c.z, c.w};
                         float part[kUmmaMaxM];
 #pragma unroll
@@ -542,7 +553,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
 #pragma unroll
                                 for (int m = 0; m < kUmmaMaxM; ++m)
                                     if (m < M) {
-                                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(X + (int64_t)m * K + k);
+                                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(MXQ_AT(X + (int64_t)m * K + k, 4, X, (int64_t)M * K * 2));
                                         part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
                                         part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
                                     }
@@ -582,7 +593,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                                     besti[m] = (uint32_t)n;
                                 }
                             } else {
-                                store_out(Y, y_dtype, (int64_t)m * N + n, yt[m] * kGuardUp);
+                                store_out(Y, y_dtype, (int64_t)m * N + n, yt[m] * kGuardUp, (int64_t)M * N);
                             }
                         }
             } else {
@@ -614,12 +625,12 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                         if (EPI == kEpiLayer) {
                             // (gate / up calls are planned with power-of-two clusters and never come here)
                             const int64_t at = (int64_t)m * N + n;
-                            store_out(Y, y_dtype, at, acc * kGuardUp + poison + load_in(fa.residual, y_dtype, at));
+                            store_out(Y, y_dtype, at, acc * kGuardUp + poison + load_in(fa.residual, y_dtype, at, (int64_t)M * N), (int64_t)M * N);
                         } else if (fa.keys) {
                             const unsigned long long key = argmax_key(acc * kGuardUp + poison, (uint32_t)n);
                             if (key) atomicMax(s_keys + m, key);   // (rare decomposition: straight into shared memory)
                         } else {
-                            store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison);
+                            store_out(Y, y_dtype, (int64_t)m * N + n, acc * kGuardUp + poison, (int64_t)M * N);
                         }
                     }
                 }
@@ -656,7 +667,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                                         besti[m] = (uint32_t)n;
                                     }
                                 } else {
-                                    store_out(Y, y_dtype, (int64_t)m * N + n, w);
+                                    store_out(Y, y_dtype, (int64_t)m * N + n, w, (int64_t)M * N);
                                 }
                             }
                     }
@@ -817,6 +828,8 @@ static int linear_umma_take_status(uint32_t *out) {
     return MXQ_OK;
 }
 
+MXQ_BOUNDS_TU(bounds_take_linear_umma)
+
 }  // namespace mxq
 
 extern "C" {
@@ -835,6 +848,29 @@ int mxq_linear_device_status(uint32_t *status_host) {
     rc = mxq::linear_mma_take_status(&vm);
     if (rc != MXQ_OK) return rc;
     *status_host = v | (v4 << 8) | (vb << 16) | (vp << 24) | (vm << 28);
+    return MXQ_OK;
+}
+
+int mxq_debug_bounds_report(uint64_t *report) {
+    if (!report) return MXQ_ERR_NULL;
+    for (int i = 0; i < 6; ++i) report[i] = 0;
+#ifdef MXQ_DEBUG_BOUNDS
+    report[0] = 1;
+#endif
+    int (*const take[6])(unsigned long long *) = {mxq::bounds_take_linear,     mxq::bounds_take_linear_umma,  mxq::bounds_take_linear_fp4,
+                                                 mxq::bounds_take_linear_mma, mxq::bounds_take_linear_batch, mxq::bounds_take_linear_bf16};
+    for (int u = 0; u < 6; ++u) {
+        unsigned long long r[4] = {0, 0, 0, 0};
+        const int rc = take[u](r);
+        if (rc != MXQ_OK) return rc;
+        if (r[0] != 0 && report[1] == 0) {
+            report[2] = (uint64_t)u;
+            report[3] = r[1];
+            report[4] = r[2];
+            report[5] = r[3];
+        }
+        report[1] += r[0];
+    }
     return MXQ_OK;
 }
 #pragma GCC visibility pop

@@ -220,16 +220,19 @@ __device__ __forceinline__ void fused_accept_finish(const FusedAccept &fa, unsig
     }
 }
 
-__device__ __forceinline__ void store_out(void *Y, int y_dtype, int64_t idx, float v) {
+// (`count`: elements of the array, for the bounds-checked build)
+__device__ __forceinline__ void store_out(void *Y, int y_dtype, int64_t idx, float v, int64_t count) {
+    (void)count;
     if (y_dtype == MXQ_F32)
-        reinterpret_cast<float *>(Y)[idx] = v;
+        *MXQ_AT(reinterpret_cast<float *>(Y) + idx, 4, Y, count * 4) = v;
     else
-        reinterpret_cast<__nv_bfloat16 *>(Y)[idx] = __float2bfloat16_rn(v);
+        *MXQ_AT(reinterpret_cast<__nv_bfloat16 *>(Y) + idx, 2, Y, count * 2) = __float2bfloat16_rn(v);
 }
 
-__device__ __forceinline__ float load_in(const void *R, int dtype, int64_t idx) {
-    return dtype == MXQ_F32 ? reinterpret_cast<const float *>(R)[idx]
-                            : __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(R)[idx]);
+__device__ __forceinline__ float load_in(const void *R, int dtype, int64_t idx, int64_t count) {
+    (void)count;
+    return dtype == MXQ_F32 ? *MXQ_AT(reinterpret_cast<const float *>(R) + idx, 4, R, count * 4)
+                            : __bfloat162float(*MXQ_AT(reinterpret_cast<const __nv_bfloat16 *>(R) + idx, 2, R, count * 2));
 }
 
 // Layer epilogues of the tcgen05 kernels (kEpiLayer): what happens to the finished sums w[m] of weight row n, one per
@@ -239,7 +242,7 @@ __device__ __forceinline__ float load_in(const void *R, int dtype, int64_t idx) 
 template <int MT>
 __device__ __forceinline__ void layer_prefetch(const FusedAccept &fa, int y_dtype, int M, int64_t n, int64_t N, bool active, float (&r)[MT]) {
 #pragma unroll
-    for (int m = 0; m < MT; ++m) r[m] = (fa.residual != nullptr && active && m < M) ? load_in(fa.residual, y_dtype, (int64_t)m * N + n) : 0.f;
+    for (int m = 0; m < MT; ++m) r[m] = (fa.residual != nullptr && active && m < M) ? load_in(fa.residual, y_dtype, (int64_t)m * N + n, (int64_t)M * N) : 0.f;
 }
 // layer_emit: called by all 32 lanes of a warp together.  Gate / up pairing: the holder of weight row n ^ 1 is
 // `pair_lanes` lanes away; the even row's holder stores silu(gate) * up with silu(g) = g / (1 + e^-g), which goes to -0
@@ -258,12 +261,12 @@ __device__ __forceinline__ void layer_emit(const FusedAccept &fa, void *Y, int y
         if (active && (n & 1) == 0) {
 #pragma unroll
             for (int m = 0; m < MT; ++m)
-                if (m < M) store_out(Y, y_dtype, (int64_t)m * (N >> 1) + (n >> 1), y[m]);
+                if (m < M) store_out(Y, y_dtype, (int64_t)m * (N >> 1) + (n >> 1), y[m], (int64_t)M * (N >> 1));
         }
     } else if (active) {
 #pragma unroll
         for (int m = 0; m < MT; ++m)
-            if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, w[m] + r[m]);
+            if (m < M) store_out(Y, y_dtype, (int64_t)m * N + n, w[m] + r[m], (int64_t)M * N);
     }
 }
 
@@ -293,7 +296,7 @@ __device__ __forceinline__ void scatter_prefetch(const FusedAccept &fa, int y_dt
 #pragma unroll
     for (int i = 0; i < PH; ++i) {
         const int m = i * S + (j & (S - 1));
-        res[i] = (speaks && i < npos && m < M) ? load_in(fa.residual, y_dtype, (int64_t)m * N + n) : 0.f;
+        res[i] = (speaks && i < npos && m < M) ? load_in(fa.residual, y_dtype, (int64_t)m * N + n, (int64_t)M * N) : 0.f;
     }
 }
 
@@ -340,7 +343,8 @@ __device__ __forceinline__ void scatter_sum_store(const float *recv, int stride,
 #pragma unroll
         for (int i = 0; i < PH; ++i) {
             const int m = i * S + (j & (S - 1));
-            if (i < npos && m < M) store_out(Y, y_dtype, swiglu ? (int64_t)m * (N >> 1) + (n >> 1) : (int64_t)m * N + n, a[i]);
+            if (i < npos && m < M)
+                store_out(Y, y_dtype, swiglu ? (int64_t)m * (N >> 1) + (n >> 1) : (int64_t)m * N + n, a[i], (int64_t)M * (swiglu ? N >> 1 : N));
         }
     }
 }

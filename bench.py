@@ -5,9 +5,9 @@ Workload (BASELINE.json config "7B-Llama-shaped decode layer set", M=1): one *st
 draft-token pass over the linear projections of ``--layers`` (default 32) distinct 7B decoder
 layers -- q/k/v/o 4096x4096, gate/up 11008x4096, down 4096x11008 -- i.e. 224 independent layer
 problems per step, streaming 3.44 GB of MXFP4 weights (far larger than the 126 MB L2, so every
-step reads HBM).  They run through mxq_linear_batch, ``--layers-per-call`` (default 4) layer
-sets = 28 layers per launch; the same step as one launch per layer set and as 224 separate
-mxq_linear calls is timed beside it (``extra.routes``).  Weights are synthetic (Student-t, seeded), direct-cast on the device by
+step reads HBM).  They run through mxq_linear_batch, ``--layers-per-call`` (default 8) layer
+sets = 56 layers per launch; the same step with four and with one layer set per launch and as 224
+separate mxq_linear calls is timed beside it (``extra.routes``).  Weights are synthetic (Student-t, seeded), direct-cast on the device by
 mxq_quantize before timing; the offline cast and the greedy-accept step are timed separately and
 reported under "extra".
 
@@ -39,10 +39,10 @@ HBM_DATASHEET_GBS = 8000.0
 
 
 # DRAM bytes (read + write) over algorithmic bytes of one launch, from the committed profiler summaries:
-#   mxq_linear_batch, four 7B layer sets at M=1 (profiles/mxq_linear_batch_m1_4x7B_layer_sets_full.md):
-#     433.47 MB read + 5.92 MB written against 431.01 MB algorithmic
+#   mxq_linear_batch, eight 7B layer sets at M=1 (profiles/mxq_linear_batch_m1_8x7B_layer_sets_full.md):
+#     866.23 MB read + 5.45 MB written against 862.02 MB algorithmic (mean of the two captured launches)
 #   one mxq_linear call, 11008x4096 at M=1 (profiles/mxq_linear_fp4_m1_11008x4096_full.md): 24.034816 MB / 23.957504 MB
-DRAM_OVER_ALGORITHMIC_BATCH = (433.469184 + 5.915264) / 431.011840
+DRAM_OVER_ALGORITHMIC_BATCH = (866.232704 + 5.452672) / 862.023680
 DRAM_OVER_ALGORITHMIC = 24.034816 / 23.957504
 
 
@@ -414,8 +414,10 @@ def run_ours(args):
         routes = {}
         n7 = len(shapes)
         st_r = max(3, min(args.steps, 40))
-        for name, pc in (("batch_%d_layer_sets_per_call" % max(1, min(args.layers_per_call, args.layers)), per_call),
-                         ("batch_1_layer_set_per_call", n7), ("separate_calls", 0)):
+        todo = [("batch_%d_layer_sets_per_call" % max(1, min(args.layers_per_call, args.layers)), per_call)]
+        todo += [(name, pc) for name, pc in (("batch_4_layer_sets_per_call", 4 * n7), ("batch_1_layer_set_per_call", n7), ("separate_calls", 0))
+                 if pc != per_call and pc <= n7 * args.layers]
+        for name, pc in todo:
             if pc == per_call:
                 routes[name] = {"us_per_layer_set": ms_per_step * 1e3 / args.layers, "gbs": value, "launches_per_step": main.launches,
                                 "frac_of_peak": value / peaks["hbm_gbs"], "headline": True}
@@ -787,8 +789,8 @@ def run_ours(args):
         "gpu_launches": main.launches * args.steps,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "traffic": (DRAM_OVER_ALGORITHMIC_BATCH if per_call else DRAM_OVER_ALGORITHMIC) * bytes_step / main.launches,
-                     "traffic_kind": ("dram read+write bytes of a profiler capture of one mxq_linear_batch launch of four 7B layer sets "
-                                      "(439.4 MB against 431.0 MB algorithmic), scaled to this launch's bytes") if per_call else
+                     "traffic_kind": ("dram read+write bytes of a profiler capture of one mxq_linear_batch launch of eight 7B layer sets "
+                                      "(871.7 MB against 862.0 MB algorithmic), scaled to this launch's bytes") if per_call else
                                      ("dram read+write bytes of one profiler capture of the 11008x4096 launch "
                                       "(24.03 MB against 23.96 MB algorithmic), scaled to the average launch"),
                      "peak_kind": "of " + peak_kind,
@@ -1025,7 +1027,7 @@ def main():
     ap.add_argument("--m", type=int, default=1, help="token rows (1 = draft step)")
     ap.add_argument("--route", choices=["batch", "separate"], default="batch",
                     help="batch: mxq_linear_batch, --layers-per-call layer sets per launch; separate: one mxq_linear call per layer")
-    ap.add_argument("--layers-per-call", type=int, default=4, help="layer sets (7 layers each) per mxq_linear_batch call, 1..4")
+    ap.add_argument("--layers-per-call", type=int, default=8, help="layer sets (7 layers each) per mxq_linear_batch call, 1..9")
     ap.add_argument("--no-graph", action="store_true", help="launch from Python instead of replaying a CUDA graph")
     ap.add_argument("--quick", action="store_true", help="skip the extra measurements")
     ap.add_argument("--no-cpu-baseline", action="store_true")

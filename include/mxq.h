@@ -304,11 +304,12 @@ int mxq_linear_swiglu(const void *X_bf16, int M, const uint8_t *codes, const uin
  *           its first 16384 bytes (counters) ONCE before the first use; every call that completes leaves them zero
  *           again; the rest needs no initialisation.  After a non-zero mxq_linear_device_status zero them again.  Calls
  *           in one stream may share a workspace; calls that may run concurrently need one each.
- * The persistent kernel covers M <= 4 with every K a multiple of 128; any other call runs its layers one after the
+ * The persistent kernel covers M <= 8 with every K a multiple of 128; with 9 <= M <= 16 it runs twice, over the rows
+ * [0, 8) and [8, M) (the rows of a layer are independent of one another); any other call runs its layers one after the
  * other through mxq_linear / mxq_linear_residual / mxq_linear_swiglu (same results as those).  Results are
  * bit-reproducible run to run and within mxq_linear's bound; the summation order differs from mxq_linear's.  Errors as
  * mxq_linear.  Bounded waits that give up are reported in bits 24-27 of mxq_linear_device_status. */
-#define MXQ_MAX_BATCH 32
+#define MXQ_MAX_BATCH 64
 #define MXQ_MAX_BATCH_GROUPS 8
 #define MXQ_BATCH_DEPENDS 1 /* this layer and the ones after it may read what the layers before it in the array wrote */
 enum mxq_epilogue { MXQ_EPI_NONE = 0, MXQ_EPI_RESIDUAL = 1, MXQ_EPI_SWIGLU = 2 };
@@ -329,7 +330,8 @@ int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *works
                      void *stream);
 
 /* How mxq_linear_batch would run the call on the current device (diagnostics; launches nothing).  info[8] int32:
- * [0] 1 if the persistent kernel covers the call, 0 if the layers would run one by one; [1] CTAs; [2] ring slots per
+ * [0] launches of the persistent kernel (1; 2 for 9..16 token rows, the rest then describes the first), 0 if the
+ * layers would run one by one; [1] CTAs; [2] ring slots per
  * CTA; [3] dynamic shared memory bytes; [4] columns of the token operand; [5] units of work (128 rows x 256 k);
  * [6] tensor-memory columns per CTA. */
 int mxq_linear_batch_info(const mxq_linear_desc *descs, int count, int M, int32_t *info);

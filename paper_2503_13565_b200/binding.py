@@ -416,7 +416,7 @@ def interleave_gate_up(gate: torch.Tensor, up: torch.Tensor) -> torch.Tensor:
 LAYOUT_KNOBS = {"split": 0, "ring": 1, "tiles": 2, "operand_through_ring": 3, "presplit_min_m": 4, "batch_ring": 5,
                 "batch_ctas_per_sm": 6}
 EPILOGUES = {"none": 0, "residual": 1, "swiglu": 2}
-MAX_BATCH = 32
+MAX_BATCH = 64
 
 
 def mxq_set_linear_layout(what, value: int) -> None:

@@ -104,8 +104,12 @@ struct Cursor {
     int d, t, s, ks, tiles;
 };
 __device__ __forceinline__ void cursor_at(const BatchTable &tb, int u, Cursor &c) {
-    int d = 0;
-    while (d + 1 < tb.ndesc && u >= tb.desc[d + 1].unit_base) ++d;
+    int d = 0, hi = tb.ndesc;   // the last layer whose first unit is <= u (bisection: up to 64 layers, and the scale warps ask per unit)
+    while (hi - d > 1) {
+        const int mid = (d + hi) >> 1;
+        if (u >= tb.desc[mid].unit_base) d = mid;
+        else hi = mid;
+    }
     c.d = d;
     c.ks = tb.desc[d].ks;
     c.tiles = tb.desc[d].tiles;
@@ -259,7 +263,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
         for (int g = 0; g < ngroups; ++g) units_left += s_walk[3 * g + 1];
     }
     if (warp == 1) {
-        if (lane < tb.ndesc) asm volatile("prefetch.tensormap [%0];" ::"l"(&tb.maps[lane]) : "memory");
+        for (int d = lane; d < tb.ndesc; d += 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&tb.maps[d]) : "memory");
         __syncwarp();
         if (lane == 0) {
             Walk wk0;
@@ -382,7 +386,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
         // it comes from is complete (all of a call's images are, a microsecond or two into the kernel).  After that a
         // unit's codes and operand are requested together, as soon as the MMAs have released the slot they go to.
         if (lane == 0) {
-            uint32_t ready_mask = 0;
+            uint64_t ready_mask = 0;
             int d_seen = -1, im = 0;
             const CUtensorMap *map = nullptr;
             const uint8_t *img = nullptr;
@@ -392,14 +396,14 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                 map = &tb.maps[c.d];
                 im = tb.desc[c.d].img;
                 img = tb.ws + tb.img[im].offset;
-                if (!((ready_mask >> im) & 1u)) {
+                if (!((ready_mask >> im) & 1ull)) {
                     if (!wait_counter(g_ready + im * kBatchCounterStride, (uint32_t)tb.img[im].ntasks, s_fail, limit_us)) {
                         atomicOr(&g_batch_status, 8u);
                         *s_fail = 1;
                         return false;
                     }
                     fence_proxy_async_all();   // the image was written with ordinary stores; the bulk copies read it through the async proxy
-                    ready_mask |= 1u << im;
+                    ready_mask |= 1ull << im;
                 }
                 return true;
             };
@@ -488,9 +492,15 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
         const int nsw = ring < 4 ? ring : 4;
         uint32_t rows_lo[4], rows_hi[4];
         Walk wk;
-        auto load = [&](int i, uint32_t (&lo)[4], uint32_t (&hi)[4]) {   // element i of the current group's walk
-            Cursor c;
-            cursor_at(tb, walk_unit(wk, i), c);
+        // (the cursor is carried from one of this warp's units to the next: no search, no division per unit)
+        Cursor c;
+        int c_at = -1;   // element of the current group's walk the cursor stands at (-1: nowhere yet)
+        auto load = [&](int i, uint32_t (&lo)[4], uint32_t (&hi)[4]) {   // element i of the current group's walk, i > c_at
+            if (c_at < 0) {
+                walk_begin(tb, wk, c);
+                c_at = 0;
+            }
+            while (c_at < i) walk_to(tb, wk, ++c_at, c);
             const BatchDesc &ds = tb.desc[c.d];
             const int kb_row = ds.K >> 5;
             const bool wide = (ds.K & (kBatchStageK - 1)) == 0;   // a unit's 8 bytes are one aligned load
@@ -518,6 +528,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
         bool alive = sw < nsw;
         for (int g = 0; g < ngroups && alive; ++g) {
         group_walk(g, wk);
+        c_at = -1;
         const int nunit = wk.nunit;
         // first unit of this group that is this warp's: the smallest i >= 0 with (ebase + i) % nsw == sw
         const int i0 = (sw - ebase % nsw + nsw) % nsw;
@@ -564,7 +575,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
         // rewriting is asked for before anything else.
         uint32_t first_task = 0;
         if (lane == 0) first_task = atomicAdd(hdr + kBatchWordTask, 1u);
-        uint32_t seen_mask = 0, bad_mask = 0, fix_mask = 0;
+        uint64_t seen_mask = 0, bad_mask = 0, fix_mask = 0;
         float *partials = reinterpret_cast<float *>(tb.ws + tb.partials_offset);
         uint32_t *g_ticket = hdr + kBatchWordTicket, *g_done = hdr + kBatchWordDone;
         const float nanv = __uint_as_float(0x7FC00000u);
@@ -647,7 +658,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
             // has this layer's X been rewritten exactly?  (the counter is complete by now; waiting for it here makes the
             // flag's value certain)
             const int im = ds.img;
-            if (!((seen_mask >> im) & 1u)) {
+            if (!((seen_mask >> im) & 1ull)) {
                 uint32_t b = 0;
                 if (lane == 0) {
                     if (!wait_counter(g_ready + im * kBatchCounterStride, (uint32_t)tb.img[im].ntasks, s_fail, limit_us)) {
@@ -658,11 +669,11 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                     if (*reinterpret_cast<volatile uint32_t *>(g_bad + im * kBatchCounterStride + 1) != 0u) b |= 2u;
                 }
                 b = __shfl_sync(0xffffffffu, b, 0);
-                seen_mask |= 1u << im;
-                if (b & 1u) bad_mask |= 1u << im;
-                if (b & 2u) fix_mask |= 1u << im;
+                seen_mask |= 1ull << im;
+                if (b & 1u) bad_mask |= 1ull << im;
+                if (b & 2u) fix_mask |= 1ull << im;
             }
-            const bool bad = (bad_mask >> im) & 1u;
+            const bool bad = (bad_mask >> im) & 1ull;
 
             float yt[MT];
 #pragma unroll
@@ -780,7 +791,7 @@ __global__ void __launch_bounds__(kBatchThreads, 2) linear_batch_kernel(const __
                 // finished sums of weight row n, one per token row: restore the guard factor, apply the layer's epilogue, store
 #pragma unroll
                 for (int m = 0; m < MT; ++m) yt[m] *= kGuardUp;
-                if (((fix_mask >> im) & 1u) && !bad && n < ds.N) {
+                if (((fix_mask >> im) & 1ull) && !bad && n < ds.N) {
                     // what the planes of this layer's X could not hold: remainder * weight, element by element
                     const BatchFix *fixes = reinterpret_cast<const BatchFix *>(tb.ws + tb.fix_offset) + (size_t)im * kBatchMaxFixes;
                     const uint32_t nfix = min(*reinterpret_cast<volatile uint32_t *>(g_bad + im * kBatchCounterStride + 1), (uint32_t)kBatchMaxFixes);
@@ -931,6 +942,13 @@ static bool batch_covered(const mxq_linear_desc *descs, int count, int M) {
     return units < 0x40000000;
 }
 
+// 9..16 token rows: the rows of a linear layer are independent of one another (row m of Y needs row m of X and of the
+// residual only), so the call runs as two passes of the persistent kernel, rows [0, 8) and [8, M).  The weights are
+// streamed twice, which still costs far less than a launch per layer.
+static bool batch_two_passes(const mxq_linear_desc *descs, int count, int M) {
+    return M > kBatchMaxM && M <= 2 * kBatchMaxM && batch_covered(descs, count, kBatchMaxM);
+}
+
 static size_t batch_workspace_bytes(const mxq_linear_desc *descs, int count, int M) {
     const int nb = batch_nb(M);
     size_t b = kBatchHeaderBytes + batch_partials_bytes(kBatchMaxGrid, nb);
@@ -971,6 +989,11 @@ size_t mxq_linear_batch_workspace_bytes(const mxq_linear_desc *descs, int count,
     if (batch_validate(descs, count, M) != MXQ_OK) return 0;
     size_t b = mxq::kBatchHeaderBytes;
     if (mxq::batch_covered(descs, count, M)) b = mxq::batch_workspace_bytes(descs, count, M);
+    else if (mxq::batch_two_passes(descs, count, M)) {   // what the larger of the two passes asks for
+        const size_t first = mxq_linear_batch_workspace_bytes(descs, count, mxq::kBatchMaxM);
+        const size_t second = mxq_linear_batch_workspace_bytes(descs, count, M - mxq::kBatchMaxM);
+        return first > second ? first : second;
+    }
     // where the persistent kernel does not cover the call the layers run one by one and share this much scratch
     size_t one = 0;
     for (int i = 0; i < count; ++i) {
@@ -991,6 +1014,11 @@ int mxq_linear_batch_info(const mxq_linear_desc *descs, int count, int M, int32_
     const int rc = batch_validate(descs, count, M);
     if (rc != MXQ_OK) return rc;
     for (int i = 0; i < 8; ++i) info[i] = 0;
+    if (mxq::batch_two_passes(descs, count, M)) {   // described by its first pass (8 token rows)
+        const int rc2 = mxq_linear_batch_info(descs, count, mxq::kBatchMaxM, info);
+        if (rc2 == MXQ_OK && info[0] == 1) info[0] = 2;
+        return rc2;
+    }
     if (!mxq::batch_covered(descs, count, M)) return MXQ_OK;
     int64_t units = 0, total = 0, cur = 0;
     for (int i = 0; i < count; ++i) {
@@ -1020,6 +1048,23 @@ int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *works
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MXQ_ERR_ALIGN;
     const size_t ws_needed = mxq_linear_batch_workspace_bytes(descs, count, M);
     if (workspace_bytes < ws_needed) return MXQ_ERR_WORKSPACE;
+    if (mxq::batch_two_passes(descs, count, M)) {
+        mxq_linear_desc part[MXQ_MAX_BATCH];
+        for (int row0 = 0; row0 < M; row0 += mxq::kBatchMaxM) {
+            const int rows = M - row0 < mxq::kBatchMaxM ? M - row0 : mxq::kBatchMaxM;
+            for (int i = 0; i < count; ++i) {
+                part[i] = descs[i];
+                const size_t ysz = descs[i].y_dtype == MXQ_F32 ? 4 : 2;
+                const int64_t ncol = descs[i].epilogue == MXQ_EPI_SWIGLU ? descs[i].N / 2 : descs[i].N;
+                part[i].X_bf16 = static_cast<const uint8_t *>(descs[i].X_bf16) + (size_t)row0 * descs[i].K * 2;
+                part[i].Y = static_cast<uint8_t *>(descs[i].Y) + (size_t)row0 * ncol * ysz;
+                if (descs[i].residual) part[i].residual = static_cast<const uint8_t *>(descs[i].residual) + (size_t)row0 * ncol * ysz;
+            }
+            rc = mxq_linear_batch(part, count, rows, workspace, workspace_bytes, stream);
+            if (rc != MXQ_OK) return rc;
+        }
+        return MXQ_OK;
+    }
     cudaStream_t st = (cudaStream_t)stream;
     mxq::BatchLayout L;
     int64_t units = 0, cur = 0;   // units of the largest group

@@ -13,7 +13,7 @@
 
 namespace mxq {
 
-constexpr int kBatchMaxDescs = 32;       // layers per call (the table travels as a kernel parameter, 7.5 KB)
+constexpr int kBatchMaxDescs = 64;       // layers per call (the table travels as a kernel parameter, 15 KB of the 32 KB allowed)
 constexpr int kBatchMaxM = 8;            // token rows: 16 digit planes each, 128 operand columns at most
 constexpr int kBatchThreads = 320;       // MMA warp, producer warp, four split / epilogue warps, four scale warps
 constexpr int kBatchTileRows = 128;      // weight rows per tile = M of one tcgen05.mma
@@ -27,19 +27,19 @@ constexpr int kBatchMaxGroups = 8;       // groups of layers per call (a layer t
 // ---- workspace ------------------------------------------------------------------------------------------------------
 // [0, kBatchHeaderBytes)  counters, all zero between calls; every counter that many CTAs wait for has a 128-byte line
 //                          to itself (kBatchCounterStride words from one to the next):
-//      u32 ready[32]   split tasks delivered per token-operand image            (words 0, 32, 64, ...)
-//      u32 bad[32]     an image's list of corrections overflowed (the word after its ready counter)
-//      u32 fixes[32]   entries on an image's list of corrections (the word after that)
-//      u32 done[8]     tiles stored, per group                                  (words 1024, 1056, ...)
+//      u32 ready[64]   split tasks delivered per token-operand image            (words 0, 32, 64, ...)
+//      u32 bad[64]     an image's list of corrections overflowed (the word after its ready counter)
+//      u32 fixes[64]   entries on an image's list of corrections (the word after that)
+//      u32 done[8]     tiles stored, per group                                  (words 2048, 2080, ...)
 //      u32 task[8]     rewriting tasks handed out, per group                    (the word after the group's done counter)
-//      u32 exit        CTAs that have finished                                  (word 1280)
-//      u32 ticket[kBatchMaxGrid] at word 2048: contributors that have delivered their share of a tile split between CTAs
+//      u32 exit        CTAs that have finished                                  (word 2304)
+//      u32 ticket[kBatchMaxGrid] at word 2560: contributors that have delivered their share of a tile split between CTAs
 // [kBatchHeaderBytes, ...) partial sums: [grid][2 (at the head / at the tail of the CTA's range)][token slots][128] floats
 // then the token-operand images, one per distinct X: [stage][operand rows NB x 128 bytes | 1024 bytes of scale atoms]
 // then the lists of corrections, kBatchMaxFixes entries per image
 constexpr size_t kBatchHeaderBytes = 16384;
 constexpr int kBatchCounterStride = 32;
-constexpr int kBatchWordReady = 0, kBatchWordBad = 1, kBatchWordDone = 1024, kBatchWordTask = 1025, kBatchWordExit = 1280, kBatchWordTicket = 2048;
+constexpr int kBatchWordReady = 0, kBatchWordBad = 1, kBatchWordDone = 2048, kBatchWordTask = 2049, kBatchWordExit = 2304, kBatchWordTicket = 2560;
 
 inline int batch_nb(int M) { return M == 1 ? 16 : (M == 2 ? 32 : (M <= 4 ? 64 : 128)); }   // operand columns: 16 planes per token slot
 inline uint32_t batch_image_stage_bytes(int nb) { return (uint32_t)nb * 128u + kBatchSfBytes; }

@@ -89,7 +89,7 @@ def test_batch_argument_errors_are_caught_before_any_launch():
     p = ctypes.cast(descs, ctypes.c_void_p)
     assert L.mxq_linear_batch(None, 1, 1, a, 1 << 30, None) == 1
     assert L.mxq_linear_batch(p, 0, 1, a, 1 << 30, None) == 2
-    assert L.mxq_linear_batch(p, 33, 1, a, 1 << 30, None) == 2
+    assert L.mxq_linear_batch(p, 65, 1, a, 1 << 30, None) == 2
     assert L.mxq_linear_batch(p, 2, 17, a, 1 << 30, None) == 2
     assert L.mxq_linear_batch(p, 2, 1, None, 0, None) == 1
     assert L.mxq_linear_batch(p, 2, 1, a + 16, 1 << 30, None) == 3     # workspace not 256-byte aligned

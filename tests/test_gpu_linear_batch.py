@@ -234,10 +234,35 @@ def test_activations_that_cannot_be_rewritten_exactly():
     check_linear(lay_inf["out"][:1], y64[:1], a64[:1], "row without the infinity")
 
 
-@pytest.mark.parametrize("m,n,k", [(9, 515, 2048), (1, 203, 1440), (16, 300, 1024)])
+@pytest.mark.parametrize("m", [9, 12, 16])
+def test_nine_to_sixteen_token_rows_run_as_two_passes(m):
+    """Rows [0, 8) and [8, M) through the persistent kernel one after the other: every epilogue, BF16 and FP32 outputs,
+    a residual added in place, and two layers that share an X."""
+    layers = [make_layer(3, 63, 515, 2048, m), make_layer(3, 64, 2 * 300, 2048, m, epilogue="swiglu", out_dtype=torch.bfloat16),
+              make_layer(3, 65, 333, 1152, m, epilogue="residual", out_dtype=torch.bfloat16)]
+    layers.append(make_layer(3, 66, 200, 2048, m, x=layers[0]["_x"]))
+    layers[3]["x"] = layers[0]["x"]
+    batch, _ = run_batch(layers)
+    assert batch.info()["persistent"] == 2
+    for i, lay in enumerate(layers):
+        check_layer(lay, "two passes, layer %d M=%d" % (i, m))
+
+
+def test_two_passes_on_the_7b_layer_set_and_with_dependent_groups():
+    m = 9   # eight speculated tokens and the one before them: the verification pass of Sec. III-B with N = 8
+    shapes = [(0, 4096, 4096), (4, 11008, 4096), (6, 4096, 11008)]
+    layers = [make_layer(3, idx, n, k, m, rows=sample_rows(n, idx)) for idx, n, k in shapes]
+    run_batch(layers)
+    for lay in layers:
+        check_layer(lay, "7B shapes, M=9")
+    chain = chain_layers(m, 256, 384, 210)
+    run_batch(chain)
+    check_chain(chain, "chain M=9")
+
+
+@pytest.mark.parametrize("m,n,k", [(1, 203, 1440), (9, 203, 1440), (16, 300, 96)])
 def test_calls_the_persistent_kernel_does_not_cover(m, n, k):
-    """More than 8 token rows, or K not a multiple of 128: the layers run one by one, with the same results as the
-    single-layer entry points."""
+    """K not a multiple of 128: the layers run one by one, with the same results as the single-layer entry points."""
     layers = [make_layer(3, 60, n, k, m), make_layer(3, 61, 2 * 128, k, m, epilogue="swiglu"),
               make_layer(3, 62, n, k, m, epilogue="residual")]
     run_batch(layers, expect_persistent=False)
@@ -261,12 +286,13 @@ def test_other_ring_depths_and_two_ctas_per_sm(ring, per_sm):
         mxq.mxq_set_linear_layout("batch_ctas_per_sm", 0)
 
 
-def test_thirty_two_layers_in_one_call():
-    """The most layers a call takes: 32 small ones with 32 distinct X."""
-    layers = [make_layer(3, 90 + i, 128 + 64 * (i % 5), 256 + 128 * (i % 4), 2) for i in range(32)]
+def test_sixty_four_layers_in_one_call():
+    """The most layers a call takes: 64 small ones with 64 distinct X."""
+    layers = [make_layer(3, 90 + i, 128 + 64 * (i % 5), 256 + 128 * (i % 4), 2) for i in range(64)]
+    assert len(layers) == mxq.binding.MAX_BATCH
     run_batch(layers)
     for i, lay in enumerate(layers):
-        check_layer(lay, "layer %d of 32" % i)
+        check_layer(lay, "layer %d of 64" % i)
 
 
 def test_a_bounded_wait_that_expires_is_reported_and_contained():
@@ -376,4 +402,4 @@ def test_argument_errors():
         batch.run(torch.zeros(4096, dtype=torch.uint8, device="cuda"))
     assert e.value.status == 5
     with pytest.raises(ValueError):
-        mxq.LinearBatch([lay] * 33)
+        mxq.LinearBatch([lay] * 65)

@@ -62,6 +62,29 @@ static int bounds_take_tu(unsigned long long *out) {
     }
 #endif
 
+// ---- loads of data that the PREVIOUS kernel in the stream may have written (X, a residual, a workspace) -------------
+// With programmatic dependent launch a kernel is running before its predecessor has finished, and only what it reads
+// AFTER griddepcontrol.wait through the ordinary (coherent) path is guaranteed to be the predecessor's output.  A plain
+// C++ dereference of a `const __restrict__` pointer may be compiled to ld.global.nc, whose cache is outside that
+// guarantee: a line left there by an earlier kernel on the same SM can be served instead (seen as a layer of a chain
+// computing from the previous layer's activations).  So such data is always read through these.
+__device__ __forceinline__ uint4 ld_dep_u4(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_dep_u32(const void *p) {
+    uint32_t v;
+    asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ float ld_dep_f32(const void *p) { return __uint_as_float(ld_dep_u32(p)); }
+__device__ __forceinline__ float ld_dep_bf16(const void *p) {
+    unsigned short h;
+    asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(h) : "l"(p) : "memory");
+    return __uint_as_float((uint32_t)h << 16);
+}
+
 // ---- loads that bypass L1 allocation (weights are read exactly once) -------------------
 __device__ __forceinline__ uint4 ld_stream_u4(const void *p) {
     uint4 v;

@@ -70,7 +70,7 @@ linear_rowwarp_kernel(const __nv_bfloat16 *__restrict__ X, int M, const uint4 *_
 #pragma unroll
                 for (int m = 0; m < MT; ++m) {
                     if (m < M) {
-                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(MXQ_AT(X + (int64_t)m * K + k, 4, X, (int64_t)M * K * 2));
+                        const uint32_t xb = ld_dep_u32(MXQ_AT(X + (int64_t)m * K + k, 4, X, (int64_t)M * K * 2));
                         part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
                         part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
                     }
@@ -114,14 +114,14 @@ layer_epilogue_kernel(const float *__restrict__ S, int M, int64_t N, const void 
         const int64_t F = N >> 1;
         if (i >= (int64_t)M * F) return;
         const int64_t m = i / F, f = i - m * F;
-        const float g = *MXQ_AT(S + m * N + 2 * f, 4, S, (int64_t)M * N * 4), u = *MXQ_AT(S + m * N + 2 * f + 1, 4, S, (int64_t)M * N * 4);
+        const float g = ld_dep_f32(MXQ_AT(S + m * N + 2 * f, 4, S, (int64_t)M * N * 4)), u = ld_dep_f32(MXQ_AT(S + m * N + 2 * f + 1, 4, S, (int64_t)M * N * 4));
         store_y(Y, y_dtype, i, g / (1.f + expf(-g)) * u, (int64_t)M * F);
     } else {
         if (i >= (int64_t)M * N) return;
         const int64_t count = (int64_t)M * N;
-        const float r = y_dtype == MXQ_F32 ? *MXQ_AT(reinterpret_cast<const float *>(residual) + i, 4, residual, count * 4)
-                                           : __bfloat162float(*MXQ_AT(reinterpret_cast<const __nv_bfloat16 *>(residual) + i, 2, residual, count * 2));
-        store_y(Y, y_dtype, i, *MXQ_AT(S + i, 4, S, count * 4) + r, count);
+        const float r = y_dtype == MXQ_F32 ? ld_dep_f32(MXQ_AT(reinterpret_cast<const float *>(residual) + i, 4, residual, count * 4))
+                                           : ld_dep_bf16(MXQ_AT(reinterpret_cast<const __nv_bfloat16 *>(residual) + i, 2, residual, count * 2));
+        store_y(Y, y_dtype, i, ld_dep_f32(MXQ_AT(S + i, 4, S, count * 4)) + r, count);
     }
 }
 

@@ -246,7 +246,7 @@ linear_bf16_rowwarp_kernel(const __nv_bfloat16 *__restrict__ X, int M, const __n
 #pragma unroll
         for (int m = 0; m < kMaxM; ++m)
             if (m < M) {
-                const uint32_t xb = *reinterpret_cast<const uint32_t *>(MXQ_AT(X + (int64_t)m * K + k, 4, X, (int64_t)M * K * 2));
+                const uint32_t xb = ld_dep_u32(MXQ_AT(X + (int64_t)m * K + k, 4, X, (int64_t)M * K * 2));
                 acc[m] = fmaf(w0, __uint_as_float(xb << 16), acc[m]);
                 acc[m] = fmaf(w1, __uint_as_float(xb & 0xFFFF0000u), acc[m]);
             }

@@ -412,7 +412,7 @@ linear_fp4_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16 
 #pragma unroll
                                 for (int m = 0; m < kFp4MaxM; ++m)
                                     if (m < M) {
-                                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(MXQ_AT(X + (int64_t)m * K + k, 4, X, (int64_t)M * K * 2));
+                                        const uint32_t xb = ld_dep_u32(MXQ_AT(X + (int64_t)m * K + k, 4, X, (int64_t)M * K * 2));
                                         part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
                                         part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
                                     }

@@ -139,7 +139,7 @@ split_tokens_kernel(const __nv_bfloat16 *__restrict__ X, int M, int64_t K, int k
     for (int q = 0; q < (kUmmaMaxM + kSplitWarps - 1) / kSplitWarps; ++q) {
         const int m = warp + q * kSplitWarps;
         raw[q] = make_uint4(0, 0, 0, 0);
-        if (m < M && act) raw[q] = *reinterpret_cast<const uint4 *>(MXQ_AT(X + (int64_t)m * K + kk, 16, X, (int64_t)M * K * 2));
+        if (m < M && act) raw[q] = ld_dep_u4(MXQ_AT(X + (int64_t)m * K + kk, 16, X, (int64_t)M * K * 2));
     }
     bool inexact = false;
 #pragma unroll
@@ -435,7 +435,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                 s_xin = 1;   // lets the producer request the rest of the ring
             }
             const uint32_t *flags = reinterpret_cast<const uint32_t *>(presplit);
-            for (int i = ct; i < nst; i += 128) inexact |= *MXQ_AT(flags + s_begin + i, 4, flags, umma_ws_flags_bytes(ks)) != 0u;
+            for (int i = ct; i < nst; i += 128) inexact |= ld_dep_u32(MXQ_AT(flags + s_begin + i, 4, flags, umma_ws_flags_bytes(ks))) != 0u;
         } else {
             // Groups of 32 units (256 k of one token, one warp; a unit is 8 elements, one lane) in order of K, so that
             // the MMA warp can start on the first stages while later ones are being split.  Group G: pair of stages
@@ -460,7 +460,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
                         mm[b] = G - pair[b] * M;
                         kk[b] = pair[b] * (2 * kUmmaStageK) + lane * 8;
                         act[b] = kk[b] < k_len;
-                        if (act[b]) raw[b] = *reinterpret_cast<const uint4 *>(MXQ_AT(xbase + (int64_t)mm[b] * K + kk[b], 16, X, (int64_t)M * K * 2));
+                        if (act[b]) raw[b] = ld_dep_u4(MXQ_AT(xbase + (int64_t)mm[b] * K + kk[b], 16, X, (int64_t)M * K * 2));
                     }
                 }
 #pragma unroll
@@ -553,7 +553,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16
 #pragma unroll
                                 for (int m = 0; m < kUmmaMaxM; ++m)
                                     if (m < M) {
-                                        const uint32_t xb = *reinterpret_cast<const uint32_t *>(MXQ_AT(X + (int64_t)m * K + k, 4, X, (int64_t)M * K * 2));
+                                        const uint32_t xb = ld_dep_u32(MXQ_AT(X + (int64_t)m * K + k, 4, X, (int64_t)M * K * 2));
                                         part[m] = fmaf(wv.x, __uint_as_float(xb << 16), part[m]);
                                         part[m] = fmaf(wv.y, __uint_as_float(xb & 0xFFFF0000u), part[m]);
                                     }

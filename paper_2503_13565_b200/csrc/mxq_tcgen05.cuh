@@ -231,8 +231,9 @@ __device__ __forceinline__ void store_out(void *Y, int y_dtype, int64_t idx, flo
 
 __device__ __forceinline__ float load_in(const void *R, int dtype, int64_t idx, int64_t count) {
     (void)count;
-    return dtype == MXQ_F32 ? *MXQ_AT(reinterpret_cast<const float *>(R) + idx, 4, R, count * 4)
-                            : __bfloat162float(*MXQ_AT(reinterpret_cast<const __nv_bfloat16 *>(R) + idx, 2, R, count * 2));
+    // (the residual may be the previous kernel's output)
+    return dtype == MXQ_F32 ? ld_dep_f32(MXQ_AT(reinterpret_cast<const float *>(R) + idx, 4, R, count * 4))
+                            : ld_dep_bf16(MXQ_AT(reinterpret_cast<const __nv_bfloat16 *>(R) + idx, 2, R, count * 2));
 }
 
 // Layer epilogues of the tcgen05 kernels (kEpiLayer): what happens to the finished sums w[m] of weight row n, one per

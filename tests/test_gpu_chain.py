@@ -65,6 +65,29 @@ class Chain:
         torch.cuda.synchronize()
         return [t.clone() for t in (self.qkv, self.h1, self.act, self.h2)]
 
+    def batches(self, one_call_per_layer):
+        """The same chain through mxq_linear_batch: four calls per layer (each waits for the one before it), or one call of
+        three dependent groups per layer."""
+        out = []
+        for (wqkv, wo, wgu, wd) in self.w:
+            lays = [dict(x=self.h0, codes=wqkv[2], scales=wqkv[3], out=self.qkv),
+                    dict(x=self.att, codes=wo[2], scales=wo[3], out=self.h1, epilogue="residual", residual=self.h0),
+                    dict(x=self.h1, codes=wgu[2], scales=wgu[3], out=self.act, epilogue="swiglu", depends=True),
+                    dict(x=self.act, codes=wd[2], scales=wd[3], out=self.h2, epilogue="residual", residual=self.h1, depends=True)]
+            if one_call_per_layer:
+                out.append(mxq.LinearBatch(lays))
+            else:
+                out += [mxq.LinearBatch([dict(lay, depends=False)]) for lay in lays]
+        return out
+
+    def run_batches(self, batches, ws, sync):
+        for b in batches:
+            b.run(ws)
+            if sync:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        return [t.clone() for t in (self.qkv, self.h1, self.act, self.h2)]
+
     def check_last_layer(self, rows_of=lambda n: None):
         """Oracle bounds on the buffers as the last run left them (they hold the last layer's values)."""
         wqkv, wo, wgu, wd = self.w[-1]
@@ -127,4 +150,21 @@ def test_asynchronous_chain_on_the_7b_shapes(m):
     def sampled(n):
         return np.unique(np.concatenate([[0, 1, n - 2, n - 1], np.random.default_rng(n).integers(0, n, 300)])).astype(np.int64)
     chain.check_last_layer(rows_of=sampled)
+    assert mxq.mxq_linear_device_status() == 0
+
+
+@pytest.mark.parametrize("one_call_per_layer", [False, True])
+@pytest.mark.parametrize("m", [1, 4, 8, 12])
+def test_asynchronous_chain_through_the_batch_call(m, one_call_per_layer):
+    """The persistent kernel starts early too, and consecutive calls share one workspace: a call per matrix (each reads what
+    the call before it wrote), and a call of three dependent groups per layer (12 rows: two passes over row halves)."""
+    chain = Chain(m, 1024, 2816, layers=3, seed=740)
+    batches = chain.batches(one_call_per_layer)
+    ws = mxq.new_workspace(max(b.workspace_bytes() for b in batches))
+    ref = chain.run_batches(batches, ws, sync=True)
+    for _ in range(3):
+        got = chain.run_batches(batches, ws, sync=False)
+        for name, a, b in zip(("q/k/v", "o", "gate/up", "down"), ref, got):
+            assert torch.equal(a, b), "%s differs between the asynchronous and the synchronised chain (M=%d)" % (name, m)
+    chain.check_last_layer()
     assert mxq.mxq_linear_device_status() == 0

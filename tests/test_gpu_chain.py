@@ -168,3 +168,38 @@ def test_asynchronous_chain_through_the_batch_call(m, one_call_per_layer):
             assert torch.equal(a, b), "%s differs between the asynchronous and the synchronised chain (M=%d)" % (name, m)
     chain.check_last_layer()
     assert mxq.mxq_linear_device_status() == 0
+
+
+@pytest.mark.parametrize("m", [1, 5, 9])
+def test_verification_fused_into_the_projection_at_the_end_of_a_chain(m):
+    """mxq_lm_head_accept reads the last layer's output the moment its own wait returns: same tokens, accept length and
+    next token with and without synchronisation between the calls."""
+    chain = Chain(m, 1024, 2816, layers=2, seed=760)
+    codes, scales, _ = oracle.quantize(synth.bits_of(synth.weight(4, 77, 5000, 1024)))
+    hc, hs = torch.from_numpy(codes).cuda(), torch.from_numpy(scales).cuda()
+    draft = torch.arange(m - 1, dtype=torch.int32, device="cuda") if m > 1 else None
+    ws = mxq.new_workspace(mxq.mxq_lm_head_accept_workspace_bytes(m, 5000, 1024))
+
+    def run(sync):
+        for (wqkv, wo, wgu, wd) in chain.w:
+            for call in (lambda: mxq.mxq_linear_residual(chain.att, wo[2], wo[3], chain.h0, out=chain.h1, workspace=chain.ws),
+                         lambda: mxq.mxq_linear_swiglu(chain.h1, wgu[2], wgu[3], out=chain.act, workspace=chain.ws),
+                         lambda: mxq.mxq_linear_residual(chain.act, wd[2], wd[3], chain.h1, out=chain.h2, workspace=chain.ws)):
+                call()
+                if sync:
+                    torch.cuda.synchronize()
+        ver, g, nxt = mxq.mxq_lm_head_accept(chain.h2, hc, hs, draft, workspace=ws)
+        torch.cuda.synchronize()
+        return ver.clone(), int(g[0]), int(nxt[0])
+
+    ref = run(True)
+    for _ in range(3):
+        got = run(False)
+        assert torch.equal(ref[0], got[0]) and ref[1:] == got[1:]
+    # and the tokens are the argmax of the projection of what the chain left in h2 (margin rule of the fused-verification tests)
+    y64, a64 = oracle.linear(synth.bits_of(chain.h2.cpu()), codes, scales)
+    ver = ref[0].cpu().numpy()
+    for r in range(m):
+        top = int(np.argmax(y64[r]))
+        tol = REL * a64[r] + ABS
+        assert y64[r, ver[r]] + tol[ver[r]] >= y64[r, top] - tol[top], r

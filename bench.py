@@ -567,6 +567,21 @@ def run_ours(args):
             tf_ = time_graph(fused_pass, 10) / nlay
             wbytes = sum(n_ * k_ * 17 // 32 for n_, k_ in [(12288, 4096), (4096, 4096), (22016, 4096), (4096, 11008)])
             fl["m%d" % mm] = {"us_per_layer": tf_ * 1e6, "gbs": wbytes / tf_ / 1e9, "calls": 4, "weight_bytes": wbytes}
+            # what was timed is the chain it claims to be: issued without any synchronisation it leaves bit for bit what it
+            # leaves with a device synchronisation after every call (a kernel that read its input early would not)
+            fused_pass()
+            torch.cuda.synchronize()
+            free_running = [t_.clone() for t_ in (qkv, h1, act, h2)]
+            for (wqkv, wo, wgu, wd) in lay4:
+                mxq.mxq_linear(h0, wqkv[0], wqkv[1], out=qkv, workspace=wsf)
+                torch.cuda.synchronize()
+                mxq.mxq_linear_residual(att, wo[0], wo[1], h0, out=h1, workspace=wsf)
+                torch.cuda.synchronize()
+                mxq.mxq_linear_swiglu(h1, wgu[0], wgu[1], out=act, workspace=wsf)
+                torch.cuda.synchronize()
+                mxq.mxq_linear_residual(act, wd[0], wd[1], h1, out=h2, workspace=wsf)
+                torch.cuda.synchronize()
+            fl["m%d" % mm]["free_running_equals_synchronised"] = all(torch.equal(a_, b_) for a_, b_ in zip(free_running, (qkv, h1, act, h2)))
             # the same layer, dependences included, as ONE mxq_linear_batch call of three groups:
             # {q/k/v, o + residual} | {gate/up with SiLU(gate) * up} | {down + residual}
             one = [mxq.LinearBatch([dict(x=h0, codes=wqkv[0], scales=wqkv[1], out=qkv),

@@ -203,3 +203,36 @@ def test_verification_fused_into_the_projection_at_the_end_of_a_chain(m):
         top = int(np.argmax(y64[r]))
         tol = REL * a64[r] + ABS
         assert y64[r, ver[r]] + tol[ver[r]] >= y64[r, top] - tol[top], r
+
+
+@pytest.mark.parametrize("m", [1, 2, 8])
+def test_chain_replayed_from_a_cuda_graph(m):
+    """The benchmark times its chains as replayed graphs (the captured launches keep their programmatic dependences):
+    a replay leaves what the synchronised chain leaves."""
+    chain = Chain(m, 4096, 11008, layers=2, seed=780)
+    ref = chain.run(sync=True)
+
+    def calls():
+        for (wqkv, wo, wgu, wd) in chain.w:
+            mxq.mxq_linear(chain.h0, wqkv[2], wqkv[3], out=chain.qkv, workspace=chain.ws)
+            mxq.mxq_linear_residual(chain.att, wo[2], wo[3], chain.h0, out=chain.h1, workspace=chain.ws)
+            mxq.mxq_linear_swiglu(chain.h1, wgu[2], wgu[3], out=chain.act, workspace=chain.ws)
+            mxq.mxq_linear_residual(chain.act, wd[2], wd[3], chain.h1, out=chain.h2, workspace=chain.ws)
+
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(st):
+        calls()
+        st.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=st):
+            calls()
+        for _ in range(3):
+            for t in (chain.qkv, chain.h1, chain.act, chain.h2):
+                t.fill_(float("nan"))
+            graph.replay()
+            graph.replay()
+            st.synchronize()
+            for name, a, b in zip(("q/k/v", "o", "gate/up", "down"), ref, (chain.qkv, chain.h1, chain.act, chain.h2)):
+                assert torch.equal(a, b), "%s differs after a graph replay (M=%d)" % (name, m)
+    assert mxq.mxq_linear_device_status() == 0

@@ -142,8 +142,11 @@ def build_layers(mxq, n_layers: int, shapes, device):
 class LinearPass:
     """One pass over a list of quantised matrices at M token rows, replayed from a CUDA graph."""
 
-    def __init__(self, mxq, mats, m: int, device, seed: int, use_graph: bool = True, per_call: int = 0):
-        """per_call = 0: one mxq_linear call per matrix; > 0: mxq_linear_batch, that many matrices per call."""
+    def __init__(self, mxq, mats, m: int, device, seed: int, use_graph: bool = True, per_call: int = 0, streams: int = 1):
+        """per_call = 0: one mxq_linear call per matrix; > 0: mxq_linear_batch, that many matrices per call.
+        streams > 1 (batch route): the calls, which are independent of one another, are issued round-robin on that many
+        streams, each with a workspace of its own, between a fork and a join on the timing stream: a call then does not
+        wait for the call before it to drain."""
         self.mxq, self.mats, self.m = mxq, mats, m
         ks = sorted({k for _, _, k, _, _ in mats})
         self.x = {k: synth.normal_bf16((m, k), 1.0, seed + k, device) for k in ks}
@@ -154,7 +157,10 @@ class LinearPass:
             self.batches = [mxq.LinearBatch([dict(x=self.x[k], codes=c, scales=s, out=y)
                                              for (_, n, k, c, s), y in zip(mats[i:i + per_call], self.y[i:i + per_call])])
                             for i in range(0, len(mats), per_call)]
-            self.ws = mxq.new_workspace(max(b.workspace_bytes() for b in self.batches), device)
+            self.nstreams = max(1, min(streams, len(self.batches)))
+            self.wss = [mxq.new_workspace(max(b.workspace_bytes() for b in self.batches), device) for _ in range(self.nstreams)]
+            self.ws = self.wss[0]
+            self.side = [torch.cuda.Stream(device=device) for _ in range(self.nstreams)] if self.nstreams > 1 else []
             self.launches = len(self.batches)
             self.info = self.batches[0].info()
         else:
@@ -175,8 +181,20 @@ class LinearPass:
 
     def enqueue(self):
         if self.batches is not None:
-            for b in self.batches:
-                b.run(self.ws)
+            if not self.side:
+                for b in self.batches:
+                    b.run(self.ws)
+                return
+            fork = torch.cuda.Event()
+            fork.record(self.stream)
+            for s_ in self.side:
+                s_.wait_event(fork)
+            for i, b in enumerate(self.batches):
+                b.run(self.wss[i % self.nstreams], stream=self.side[i % self.nstreams])
+            for s_ in self.side:
+                join = torch.cuda.Event()
+                join.record(s_)
+                self.stream.wait_event(join)
             return
         for (_, n, k, codes, scales), y in zip(self.mats, self.y):
             self.mxq.mxq_linear(self.x[k], codes, scales, out=y, workspace=self.ws)
@@ -245,7 +263,7 @@ def time_e2e(mxq, mats, m: int, steps: int, warmup: int, device):
     return max(e0.elapsed_time(e1) * 1e-3, 0.0), wall, h2d, d2h
 
 
-def time_e2e_batch(mxq, mats, m: int, per_call: int, steps: int, warmup: int, device):
+def time_e2e_batch(mxq, mats, m: int, per_call: int, steps: int, warmup: int, device, streams: int = 1):
     """The same pass through mxq_linear_batch with the activations and the results in pinned HOST memory: the kernel
     reads every layer's X across the bus itself and stores Y straight into host memory, inside the timed region.
     Every layer of a call has a host buffer of its own (the library shares the rewriting of X only between layers
@@ -259,15 +277,29 @@ def time_e2e_batch(mxq, mats, m: int, per_call: int, steps: int, warmup: int, de
             assert xh[j].shape[1] == k   # every call holds the same sequence of shapes
             lays.append(dict(x=xh[j], codes=c, scales=s_, out=y))
         batches.append(mxq.LinearBatch(lays))
-    ws = mxq.new_workspace(max(b.workspace_bytes() for b in batches), device)
+    nstreams = max(1, min(streams, len(batches)))
+    wss = [mxq.new_workspace(max(b.workspace_bytes() for b in batches), device) for _ in range(nstreams)]
     stream = torch.cuda.Stream(device=device)
     stream.wait_stream(torch.cuda.current_stream(device))
+    side = [torch.cuda.Stream(device=device) for _ in range(nstreams)] if nstreams > 1 else []
     h2d = sum(2 * m * k for _, _, k, _, _ in mats)
     d2h = sum(4 * m * n for _, n, _, _, _ in mats)
 
     def one():
-        for b in batches:
-            b.run(ws, stream)
+        if not side:
+            for b in batches:
+                b.run(wss[0], stream)
+            return
+        fork = torch.cuda.Event()
+        fork.record(stream)
+        for s_ in side:
+            s_.wait_event(fork)
+        for i, b in enumerate(batches):
+            b.run(wss[i % nstreams], side[i % nstreams])
+        for s_ in side:
+            join = torch.cuda.Event()
+            join.record(s_)
+            stream.wait_event(join)
 
     with torch.cuda.stream(stream):
         for _ in range(warmup):
@@ -387,7 +419,8 @@ def run_ours(args):
     per_call = len(shapes) * max(1, min(args.layers_per_call, args.layers))   # layers (matrices) per mxq_linear_batch call
     if args.route == "separate" or m > 8:
         per_call = 0
-    main = LinearPass(mxq, mats, m, device, seed=31, use_graph=not args.no_graph, per_call=per_call)
+    streams = max(1, args.streams) if per_call else 1
+    main = LinearPass(mxq, mats, m, device, seed=31, use_graph=not args.no_graph, per_call=per_call, streams=streams)
     secs = main.time(args.steps, args.warmup, monitor)
     secs_max = replicas.max_over_ranks(secs, device)
     bytes_step = main.bytes
@@ -396,13 +429,14 @@ def run_ours(args):
     per_launch_s = secs / (args.steps * main.launches)
     achieved = bytes_step / main.launches / per_launch_s / 1e9
     peaks, peak_kind = measured_peaks()
-    route_text = ("mxq_linear_batch, %d layer set(s) = %d layers per launch" % (per_call // len(shapes), per_call)) if per_call \
-        else "one mxq_linear call per layer"
+    route_text = ("mxq_linear_batch, %d layer set(s) = %d layers per launch%s" %
+                  (per_call // len(shapes), per_call, ", the independent calls issued round-robin on %d streams" % main.nstreams if main.nstreams > 1 else "")) \
+        if per_call else "one mxq_linear call per layer"
 
     # end to end with host buffers
     e2e_steps = max(3, min(args.steps, 50))
     if per_call:
-        e2e_dev, e2e_wall, h2d, d2h = time_e2e_batch(mxq, mats, m, per_call, e2e_steps, 3, device)
+        e2e_dev, e2e_wall, h2d, d2h = time_e2e_batch(mxq, mats, m, per_call, e2e_steps, 3, device, streams)
     else:
         e2e_dev, e2e_wall, h2d, d2h = time_e2e(mxq, mats, m, e2e_steps, 3, device)
     e2e_secs = replicas.max_over_ranks(max(e2e_dev, e2e_wall), device)
@@ -414,17 +448,22 @@ def run_ours(args):
         routes = {}
         n7 = len(shapes)
         st_r = max(3, min(args.steps, 40))
-        todo = [("batch_%d_layer_sets_per_call" % max(1, min(args.layers_per_call, args.layers)), per_call)]
-        todo += [(name, pc) for name, pc in (("batch_4_layer_sets_per_call", 4 * n7), ("batch_1_layer_set_per_call", n7), ("separate_calls", 0))
-                 if pc != per_call and pc <= n7 * args.layers]
-        for name, pc in todo:
-            if pc == per_call:
+        nper = max(1, min(args.layers_per_call, args.layers))
+        head = "batch_%d_layer_sets_per_call%s" % (nper, "_%d_streams" % streams if streams > 1 else "")
+        todo = [(head, per_call, streams)]
+        for name, pc, ns in (("batch_%d_layer_sets_per_call" % nper, per_call, 1), ("batch_4_layer_sets_per_call_%d_streams" % streams, 4 * n7, streams),
+                             ("batch_4_layer_sets_per_call", 4 * n7, 1), ("batch_1_layer_set_per_call_%d_streams" % streams, n7, streams),
+                             ("batch_1_layer_set_per_call", n7, 1), ("separate_calls", 0, 1)):
+            if (pc, ns) != (per_call, streams) and pc <= n7 * args.layers and name not in [t_[0] for t_ in todo] and (ns == 1 or streams > 1):
+                todo.append((name, pc, ns))
+        for name, pc, ns in todo:
+            if (pc, ns) == (per_call, streams):
                 routes[name] = {"us_per_layer_set": ms_per_step * 1e3 / args.layers, "gbs": value, "launches_per_step": main.launches,
                                 "frac_of_peak": value / peaks["hbm_gbs"], "headline": True}
                 continue
             if m > 8 and pc:
                 continue
-            pr = LinearPass(mxq, mats, m, device, seed=31, use_graph=not args.no_graph, per_call=pc)
+            pr = LinearPass(mxq, mats, m, device, seed=31, use_graph=not args.no_graph, per_call=pc, streams=ns)
             sr = pr.time(st_r, 3)
             routes[name] = {"us_per_layer_set": sr / st_r / args.layers * 1e6, "gbs": pr.bytes * st_r / sr / 1e9,
                             "launches_per_step": pr.launches, "frac_of_peak": pr.bytes * st_r / sr / 1e9 / peaks["hbm_gbs"]}
@@ -432,7 +471,7 @@ def run_ours(args):
         extra["routes"] = routes
         # the verify-side pass (M=8) over the same layers, through the same route and as separate calls
         st8 = max(3, args.steps // 2)
-        p8 = LinearPass(mxq, mats, 8, device, seed=32, use_graph=not args.no_graph, per_call=per_call)
+        p8 = LinearPass(mxq, mats, 8, device, seed=32, use_graph=not args.no_graph, per_call=per_call, streams=streams)
         s8 = p8.time(st8, 3)
         extra["m8"] = {"gbs": p8.bytes * st8 / s8 / 1e9, "us_per_layer_set": s8 / st8 / args.layers * 1e6,
                        "route": "batch" if per_call else "separate", "launches_per_step": p8.launches}
@@ -446,7 +485,7 @@ def run_ours(args):
         for mm in (2, 3, 4, 5, 6):
             if not per_call:
                 break
-            pm = LinearPass(mxq, mats, mm, device, seed=35, use_graph=not args.no_graph, per_call=per_call)
+            pm = LinearPass(mxq, mats, mm, device, seed=35, use_graph=not args.no_graph, per_call=per_call, streams=streams)
             sm_ = pm.time(5, 3)
             mrows["m%d" % mm] = {"us_per_layer_set": sm_ / 5 / args.layers * 1e6, "gbs": pm.bytes * 5 / sm_ / 1e9}
             del pm
@@ -793,7 +832,7 @@ def run_ours(args):
         "config": {"workload": "7B decode layer set (q,k,v,o 4096x4096; gate,up 11008x4096; down 4096x11008), "
                                "M=%d, %d distinct layer sets (%d independent layers) per step, run as: %s"
                                % (m, args.layers, len(mats), route_text),
-                   "M": m, "layers": args.layers, "route": route_text, "calls_per_step": main.launches, "bytes_per_step": bytes_step,
+                   "M": m, "layers": args.layers, "route": route_text, "calls_per_step": main.launches, "streams": streams, "bytes_per_step": bytes_step,
                    "y_dtype": "f32", "l2": "inputs larger than L2 (%.2f GB of weights per step)" % (bytes_step / 1e9),
                    "cuda_graph": not args.no_graph, "multi_gpu": "replicas only"},
         "us_per_layer_set": ms_per_step * 1e3 / args.layers,
@@ -1042,6 +1081,8 @@ def main():
     ap.add_argument("--m", type=int, default=1, help="token rows (1 = draft step)")
     ap.add_argument("--route", choices=["batch", "separate"], default="batch",
                     help="batch: mxq_linear_batch, --layers-per-call layer sets per launch; separate: one mxq_linear call per layer")
+    ap.add_argument("--streams", type=int, default=2,
+                    help="batch route: the step's independent mxq_linear_batch calls are issued round-robin on this many streams (a workspace each)")
     ap.add_argument("--layers-per-call", type=int, default=8, help="layer sets (7 layers each) per mxq_linear_batch call, 1..9")
     ap.add_argument("--no-graph", action="store_true", help="launch from Python instead of replaying a CUDA graph")
     ap.add_argument("--quick", action="store_true", help="skip the extra measurements")

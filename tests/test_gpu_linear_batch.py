@@ -270,6 +270,36 @@ def test_calls_the_persistent_kernel_does_not_cover(m, n, k):
         check_layer(lay, "one-by-one layer %d M=%d" % (i, m))
 
 
+@pytest.mark.parametrize("m", [1, 8])
+def test_independent_calls_on_two_streams_with_a_workspace_each(m):
+    """Calls that may run concurrently need a workspace each, and then overlap freely: six calls issued round-robin on two
+    streams (the benchmark's route) leave bit for bit what the same calls leave one after the other on one stream."""
+    calls = [[make_layer(3, 300 + 3 * c + j, n, k, m, rows=sample_rows(n, c + j, 100)) for j, (n, k) in enumerate([(4096, 4096), (1024, 11008), (2816, 1024)])]
+             for c in range(6)]
+    batches = [mxq.LinearBatch(layers) for layers in calls]
+    wss = [mxq.new_workspace(max(b.workspace_bytes() for b in batches)) for _ in range(2)]
+    for b in batches:
+        b.run(wss[0])
+    torch.cuda.synchronize()
+    ref = [[lay["out"].clone() for lay in layers] for layers in calls]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for _ in range(3):
+        for layers in calls:
+            for lay in layers:
+                lay["out"].fill_(float("nan"))
+        torch.cuda.synchronize()
+        for i, b in enumerate(batches):
+            b.run(wss[i % 2], stream=streams[i % 2])
+        torch.cuda.synchronize()
+        for layers, outs in zip(calls, ref):
+            for lay, want in zip(layers, outs):
+                assert torch.equal(lay["out"], want)
+    for c, layers in enumerate(calls[:2]):
+        for j, lay in enumerate(layers):
+            check_layer(lay, "two streams, call %d layer %d M=%d" % (c, j, m))
+    assert not wss[0][:16384].any() and not wss[1][:16384].any()
+
+
 @pytest.mark.parametrize("ring,per_sm", [(2, 1), (3, 2), (5, 2), (1, 1)])
 def test_other_ring_depths_and_two_ctas_per_sm(ring, per_sm):
     mxq.mxq_set_linear_layout("batch_ring", ring)

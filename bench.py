@@ -157,10 +157,9 @@ class LinearPass:
             self.batches = [mxq.LinearBatch([dict(x=self.x[k], codes=c, scales=s, out=y)
                                              for (_, n, k, c, s), y in zip(mats[i:i + per_call], self.y[i:i + per_call])])
                             for i in range(0, len(mats), per_call)]
-            self.nstreams = max(1, min(streams, len(self.batches)))
-            self.wss = [mxq.new_workspace(max(b.workspace_bytes() for b in self.batches), device) for _ in range(self.nstreams)]
-            self.ws = self.wss[0]
-            self.side = [torch.cuda.Stream(device=device) for _ in range(self.nstreams)] if self.nstreams > 1 else []
+            self.calls = mxq.IndependentBatches(self.batches, streams)
+            self.nstreams = max(1, len(self.calls.streams))
+            self.ws = self.calls.workspaces[0]
             self.launches = len(self.batches)
             self.info = self.batches[0].info()
         else:
@@ -181,20 +180,7 @@ class LinearPass:
 
     def enqueue(self):
         if self.batches is not None:
-            if not self.side:
-                for b in self.batches:
-                    b.run(self.ws)
-                return
-            fork = torch.cuda.Event()
-            fork.record(self.stream)
-            for s_ in self.side:
-                s_.wait_event(fork)
-            for i, b in enumerate(self.batches):
-                b.run(self.wss[i % self.nstreams], stream=self.side[i % self.nstreams])
-            for s_ in self.side:
-                join = torch.cuda.Event()
-                join.record(s_)
-                self.stream.wait_event(join)
+            self.calls.run(self.stream)
             return
         for (_, n, k, codes, scales), y in zip(self.mats, self.y):
             self.mxq.mxq_linear(self.x[k], codes, scales, out=y, workspace=self.ws)
@@ -277,29 +263,14 @@ def time_e2e_batch(mxq, mats, m: int, per_call: int, steps: int, warmup: int, de
             assert xh[j].shape[1] == k   # every call holds the same sequence of shapes
             lays.append(dict(x=xh[j], codes=c, scales=s_, out=y))
         batches.append(mxq.LinearBatch(lays))
-    nstreams = max(1, min(streams, len(batches)))
-    wss = [mxq.new_workspace(max(b.workspace_bytes() for b in batches), device) for _ in range(nstreams)]
+    calls = mxq.IndependentBatches(batches, streams)
     stream = torch.cuda.Stream(device=device)
     stream.wait_stream(torch.cuda.current_stream(device))
-    side = [torch.cuda.Stream(device=device) for _ in range(nstreams)] if nstreams > 1 else []
     h2d = sum(2 * m * k for _, _, k, _, _ in mats)
     d2h = sum(4 * m * n for _, n, _, _, _ in mats)
 
     def one():
-        if not side:
-            for b in batches:
-                b.run(wss[0], stream)
-            return
-        fork = torch.cuda.Event()
-        fork.record(stream)
-        for s_ in side:
-            s_.wait_event(fork)
-        for i, b in enumerate(batches):
-            b.run(wss[i % nstreams], side[i % nstreams])
-        for s_ in side:
-            join = torch.cuda.Event()
-            join.record(s_)
-            stream.wait_event(join)
+        calls.run(stream)
 
     with torch.cuda.stream(stream):
         for _ in range(warmup):

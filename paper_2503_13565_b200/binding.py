@@ -499,6 +499,41 @@ def mxq_linear_batch(layers, workspace: torch.Tensor = None, stream=None) -> Lin
     return batch
 
 
+class IndependentBatches:
+    """Several mxq_linear_batch calls that do not read one another's outputs, issued round-robin on ``streams`` CUDA
+    streams with a workspace each (calls that may run concurrently need one each, see mxq.h) between a fork and a join on
+    the caller's stream.  In one stream a call cannot touch its inputs or the workspace before the call ahead of it has
+    completed to its last CTA, and the memory system idles while its early CTAs wait; on two streams a call starts in the
+    SM slots the other stream's call leaves.  Only stream plumbing: every call is the library's own."""
+
+    def __init__(self, batches, streams: int = 2):
+        self.batches = [b if isinstance(b, LinearBatch) else LinearBatch(b) for b in batches]
+        if not self.batches:
+            raise ValueError("no calls")
+        self.device = self.batches[0].device
+        n = max(1, min(int(streams), len(self.batches)))
+        self.workspaces = [new_workspace(max(b.workspace_bytes() for b in self.batches), self.device) for _ in range(n)]
+        self.streams = [torch.cuda.Stream(device=self.device) for _ in range(n)] if n > 1 else []
+
+    def run(self, stream=None) -> None:
+        cur = torch.cuda.current_stream(self.device) if stream is None else stream
+        if not self.streams:
+            for b in self.batches:
+                b.run(self.workspaces[0], cur)
+            return
+        fork = torch.cuda.Event()
+        fork.record(cur)
+        for s in self.streams:
+            s.wait_event(fork)
+        n = len(self.streams)
+        for i, b in enumerate(self.batches):
+            b.run(self.workspaces[i % n], self.streams[i % n])
+        for s in self.streams:
+            join = torch.cuda.Event()
+            join.record(s)
+            cur.wait_event(join)
+
+
 def mxq_debug_bounds_report() -> dict:
     """What the bounds-checked build has refused since the last call (see mxq.h); ``checked`` is False for the ordinary build."""
     r = (ctypes.c_uint64 * 6)()

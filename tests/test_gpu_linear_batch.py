@@ -276,20 +276,18 @@ def test_independent_calls_on_two_streams_with_a_workspace_each(m):
     streams (the benchmark's route) leave bit for bit what the same calls leave one after the other on one stream."""
     calls = [[make_layer(3, 300 + 3 * c + j, n, k, m, rows=sample_rows(n, c + j, 100)) for j, (n, k) in enumerate([(4096, 4096), (1024, 11008), (2816, 1024)])]
              for c in range(6)]
-    batches = [mxq.LinearBatch(layers) for layers in calls]
-    wss = [mxq.new_workspace(max(b.workspace_bytes() for b in batches)) for _ in range(2)]
-    for b in batches:
+    both = mxq.IndependentBatches(calls, streams=2)
+    assert len(both.streams) == 2 and len(both.workspaces) == 2
+    wss = both.workspaces
+    for b in both.batches:
         b.run(wss[0])
     torch.cuda.synchronize()
     ref = [[lay["out"].clone() for lay in layers] for layers in calls]
-    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
     for _ in range(3):
         for layers in calls:
             for lay in layers:
                 lay["out"].fill_(float("nan"))
-        torch.cuda.synchronize()
-        for i, b in enumerate(batches):
-            b.run(wss[i % 2], stream=streams[i % 2])
+        both.run()   # forks from and joins the current stream
         torch.cuda.synchronize()
         for layers, outs in zip(calls, ref):
             for lay, want in zip(layers, outs):

@@ -133,6 +133,50 @@ def test_config3_7b_layer_set(m):
 
 
 @pytest.mark.parametrize("m", [1, 8])
+def test_the_benchmarks_launch_configuration(m):
+    """What bench.py times: distinct 7B layer sets (16 here), eight sets = 56 layers per call, the calls round-robin on two
+    streams with a workspace each, replayed from a CUDA graph.  The weights are cast on the GPU (bit-exact with the oracle's
+    cast, tests/test_gpu_quantize.py); sampled rows of the first, a middle and the last layer of each call are checked
+    against the oracle, which dequantises the GPU's own codes."""
+    shapes = synth.LAYERS_7B
+    nsets, per_call = 16, 8
+    xbits = {k: synth.bits_of(synth.activations(3, 40 + k % 7, m, k)) for k in (4096, 11008)}
+    x = {k: gpu_bf16(v) for k, v in xbits.items()}
+    calls = []
+    for c in range(nsets // per_call):
+        lays = []
+        for ls in range(per_call):
+            for j, (_, n, k) in enumerate(shapes):
+                codes, scales = mxq.mxq_quantize(synth.weight(3, 900 + 7 * (c * per_call + ls) + j, n, k, device="cuda"))
+                lays.append(dict(x=x[k], codes=codes, scales=scales, out=torch.full((m, n), float("nan"), device="cuda")))
+        calls.append(lays)
+    both = mxq.IndependentBatches(calls, streams=2)
+    assert both.batches[0].count == 56 and both.batches[0].info()["persistent"] == 1
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(st):
+        both.run(st)
+        st.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=st):
+            both.run(st)
+        for lays in calls:
+            for lay in lays:
+                lay["out"].fill_(float("nan"))
+        graph.replay()
+        graph.replay()
+        st.synchronize()
+    for c, lays in enumerate(calls):
+        for i in (0, 4, 27, 55):
+            lay = lays[i]
+            n, k = lay["codes"].shape[0], lay["x"].shape[1]
+            rows = sample_rows(n, c + i, 200)
+            y64, a64 = oracle.linear(xbits[k], lay["codes"].cpu().numpy(), lay["scales"].cpu().numpy(), rows=rows)
+            check_linear(lay["out"][:, torch.as_tensor(rows, device="cuda")], y64, a64, "call %d layer %d M=%d" % (c, i, m))
+        assert all(bool(torch.isfinite(lay["out"]).all()) for lay in lays)
+
+
+@pytest.mark.parametrize("m", [1, 8])
 def test_config5_13b_layer_set(m):
     """The seven 13B-shaped layers (hidden 5120, FFN 13824) in one call, sampled rows of every layer."""
     shapes = [(5120, 5120)] * 4 + [(13824, 5120)] * 2 + [(5120, 13824)]

@@ -296,7 +296,11 @@ int mxq_linear_swiglu(const void *X_bf16, int M, const uint8_t *codes, const uin
  *           writes.  A layer with flags = MXQ_BATCH_DEPENDS opens a new GROUP (at most MXQ_MAX_BATCH_GROUPS per call):
  *           it and the layers after it start only when every layer before it in the array has been stored, and may
  *           read those outputs (a BF16 Y as the next X, e.g. gate/up with MXQ_EPI_SWIGLU followed by down); the weight
- *           stream runs on across the group boundary.  Within a group, layers that share an X pointer share its rewriting.  X, Y and residual may also be
+ *           stream runs on across the group boundary.  A call of several groups is one grid whose CTAs wait for one
+ *           another at the boundaries, so the whole grid (two CTAs per SM) must be able to become resident: do not run
+ *           such a call while kernels of OTHER streams hold SMs for long (a wait that starves gives up after its limit
+ *           and reports through mxq_linear_device_status; calls of one group never wait for a CTA that is not running).
+ *           Within a group, layers that share an X pointer share its rewriting.  X, Y and residual may also be
  *           page-locked host memory that the GPU can address (cudaHostAlloc / cudaHostRegister): the kernel then reads
  *           the activations and writes the results across the bus itself.
  *   M       token rows, common to all layers of the call

@@ -452,7 +452,8 @@ class LinearBatch:
         self.array = (_LinearDesc * self.count)()
         self.keep = []
         self.device = layers[0]["codes"].device
-        for d, lay in zip(self.array, layers):
+        self.groups = 0   # groups of layers that run one after the other (1: all layers independent)
+        for i, (d, lay) in enumerate(zip(self.array, layers)):
             x, codes, scales, out = lay["x"], lay["codes"], lay["scales"], lay["out"]
             epi = EPILOGUES[lay.get("epilogue", "none")]
             res = lay.get("residual")
@@ -471,6 +472,7 @@ class LinearBatch:
             d.y_dtype = _dt(out.dtype)
             d.epilogue = epi
             d.flags = 1 if lay.get("depends") else 0   # MXQ_BATCH_DEPENDS: a new group, after everything before it
+            self.groups += 1 if (i == 0 or d.flags) else 0
             d.reserved = 0
             self.keep.append((x, codes, scales, out, res))
         self._ptr = ctypes.cast(self.array, ctypes.c_void_p)
@@ -512,6 +514,9 @@ class IndependentBatches:
             raise ValueError("no calls")
         self.device = self.batches[0].device
         n = max(1, min(int(streams), len(self.batches)))
+        if n > 1 and any(b.groups > 1 for b in self.batches):
+            # (the CTAs of a call of several groups wait for one another and need the whole grid resident: see mxq.h)
+            raise ValueError("calls with dependent groups must not share the device with calls on other streams")
         self.workspaces = [new_workspace(max(b.workspace_bytes() for b in self.batches), self.device) for _ in range(n)]
         self.streams = [torch.cuda.Stream(device=self.device) for _ in range(n)] if n > 1 else []
 

@@ -458,6 +458,19 @@ def test_dependent_groups_7b_layer():
     check_chain(layers, "7B chain")
 
 
+def test_grouped_calls_are_not_spread_over_streams():
+    """The CTAs of a call of several groups wait for one another, so the whole grid must be resident: the helper that
+    issues independent calls on several streams refuses such calls (on one stream they are fine)."""
+    chain = chain_layers(2, 256, 384, 230)
+    assert mxq.LinearBatch(chain).groups == 3 and mxq.LinearBatch([dict(lay, depends=False) for lay in chain[:1]]).groups == 1
+    with pytest.raises(ValueError):
+        mxq.IndependentBatches([chain, chain_layers(2, 256, 384, 240)], streams=2)
+    one = mxq.IndependentBatches([chain], streams=2)   # a single call: one stream
+    one.run()
+    torch.cuda.synchronize()
+    check_chain(chain, "one grouped call through the helper")
+
+
 def test_too_many_groups_are_refused():
     lays = [make_layer(3, 220, 128, 128, 1) for _ in range(10)]
     for lay in lays[1:]:

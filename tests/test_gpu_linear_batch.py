@@ -458,6 +458,39 @@ def test_dependent_groups_7b_layer():
     check_chain(layers, "7B chain")
 
 
+def test_calls_of_different_token_counts_side_by_side():
+    """Two streams, one issuing calls at one token row (16 operand columns, 128 tensor-memory columns per CTA) and the other
+    at eight (128 operand columns, 256 tensor-memory columns): CTAs of both kernels share SMs; results as in isolation."""
+    shapes = [(4096, 4096), (1024, 11008), (2816, 1024)]
+    calls = {m: [[make_layer(3, 400 + 10 * m + 3 * c + j, n, k, m, rows=sample_rows(n, c + j, 100)) for j, (n, k) in enumerate(shapes)]
+                 for c in range(4)] for m in (1, 8)}
+    batches = {m: [mxq.LinearBatch(layers) for layers in calls[m]] for m in calls}
+    ws = {m: mxq.new_workspace(max(b.workspace_bytes() for b in batches[m])) for m in calls}
+    for m in calls:
+        for b in batches[m]:
+            b.run(ws[m])
+    torch.cuda.synchronize()
+    ref = {m: [[lay["out"].clone() for lay in layers] for layers in calls[m]] for m in calls}
+    streams = {1: torch.cuda.Stream(), 8: torch.cuda.Stream()}
+    for _ in range(3):
+        for m in calls:
+            for layers in calls[m]:
+                for lay in layers:
+                    lay["out"].fill_(float("nan"))
+        torch.cuda.synchronize()
+        for c in range(4):
+            for m in (1, 8):
+                batches[m][c].run(ws[m], stream=streams[m])
+        torch.cuda.synchronize()
+        for m in calls:
+            for layers, outs in zip(calls[m], ref[m]):
+                for lay, want in zip(layers, outs):
+                    assert torch.equal(lay["out"], want)
+    for m in calls:
+        for j, lay in enumerate(calls[m][0]):
+            check_layer(lay, "side by side, layer %d M=%d" % (j, m))
+
+
 def test_grouped_calls_are_not_spread_over_streams():
     """The CTAs of a call of several groups wait for one another, so the whole grid must be resident: the helper that
     issues independent calls on several streams refuses such calls (on one stream they are fine)."""

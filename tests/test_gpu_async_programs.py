@@ -135,3 +135,16 @@ def test_a_program_on_the_7b_widths(m, only_own_kernels):
         for idx, (a, b) in enumerate(zip(ref, got)):
             assert torch.equal(a, b), "M=%d: item %d of the final state differs without synchronisation (attempt %d)" % (m, idx, attempt)
     assert mxq.mxq_linear_device_status() == 0
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+@pytest.mark.parametrize("m", [1, 2, 3, 4, 5, 8, 9, 16])
+def test_programs_of_the_librarys_own_kernels_only(m, seed):
+    """Every call overlaps the one before it: the hardest ordering case, at every kernel choice the token count selects."""
+    prog = Program(m, 5000 + 10 * m + seed, steps=32, widths=(4096, 11008), kinds=("lin", "res", "swi", "down", "accept", "recast"))
+    ref = prog.run(sync=True)
+    for attempt in range(2):
+        got = prog.run(sync=False)
+        for idx, (a, b) in enumerate(zip(ref, got)):
+            assert torch.equal(a, b), "M=%d seed %d: item %d of the final state differs without synchronisation (attempt %d)" % (m, seed, idx, attempt)
+    assert mxq.mxq_linear_device_status() == 0

@@ -24,6 +24,11 @@ pytestmark = pytest.mark.gpu
 V = 3000   # a small vocabulary for the fused verification
 
 
+def same_bits(a, b):
+    """Equality of the stored bytes (a NaN equals itself: long programs may overflow BF16, which is no ordering matter)."""
+    return torch.equal(a.contiguous().view(torch.uint8), b.contiguous().view(torch.uint8))
+
+
 class Program:
     def __init__(self, m, seed, steps=40, widths=(1024, 1408), kinds=("lin", "res", "swi", "down", "bf16", "recast", "accept", "batch")):
         """widths: the two activation widths A (hidden) and B (feed-forward), both multiples of 128.  kinds: the calls
@@ -33,10 +38,12 @@ class Program:
         rng = random.Random(seed)
         dev = "cuda"
         cast = lambda w: list(mxq.mxq_quantize(w))
-        self.src_aa = [synth.weight(3, 800 + i, A, A, device=dev) for i in range(3)]    # BF16 sources, also the BF16-weight layers
+        # (weights a quarter of the benchmark's size, so that forty layers on top of one another stay inside BF16)
+        small = lambda cfg, idx, n, k: synth.weight(cfg, idx, n, k, device=dev) * 0.25
+        self.src_aa = [small(3, 800 + i, A, A) for i in range(3)]    # BF16 sources, also the BF16-weight layers
         self.w_aa = [cast(w) for w in self.src_aa]                                       # [codes, scales], re-cast in place by "recast"
-        self.w_ba = [cast(synth.weight(3, 810 + i, 2 * B, A, device=dev)) for i in range(2)]
-        self.w_ab = [cast(synth.weight(3, 820 + i, A, B, device=dev)) for i in range(2)]
+        self.w_ba = [cast(small(3, 810 + i, 2 * B, A)) for i in range(2)]
+        self.w_ab = [cast(small(3, 820 + i, A, B)) for i in range(2)]
         self.head = cast(synth.weight(4, 830, V, A, device=dev))
         self.h0 = [synth.normal_bf16((m, A), 1.0, 840 + i, dev) for i in range(4)]
         self.g0 = [synth.normal_bf16((m, B), 1.0, 850 + i, dev) for i in range(2)]
@@ -57,6 +64,7 @@ class Program:
                 j = (j + 1) % 4          # the output may be the residual (k), never the input
             self.ops.append((kind, i, j, k, rng.randrange(3), rng.randrange(2)))
         self.batch_ws = None
+        self.batches = {}
 
     def reset(self):
         for t, t0 in zip(self.h + self.g, self.h0 + self.g0):
@@ -86,6 +94,25 @@ class Program:
                 mxq.mxq_quantize(self.src_aa[(r3 + 1) % 3], codes=self.w_aa[r3][0], scales=self.w_aa[r3][1])
             elif kind == "accept":
                 seen.append(mxq.mxq_lm_head_accept(h[j], *self.head, self.draft, workspace=self.ws_head))
+            elif kind in ("batch_direct", "batch_groups"):
+                # the batch call writing straight into the shared buffers: no torch kernel anywhere near it
+                a_, b_ = (j + 1) % 4, (j + 2) % 4          # two outputs that are not the input h[j]
+                if kind == "batch_direct":   # three independent layers (none reads what another writes)
+                    lays = [dict(x=h[j], codes=self.w_aa[r3][0], scales=self.w_aa[r3][1], out=h[a_]),
+                            dict(x=g[1 - r2], codes=self.w_ab[r2][0], scales=self.w_ab[r2][1], out=h[b_], epilogue="residual", residual=h[b_]),
+                            dict(x=h[j], codes=self.w_ba[r2][0], scales=self.w_ba[r2][1], out=g[r2], epilogue="swiglu")]
+                else:                        # a dependent chain in three groups: o + residual -> gate/up -> down + residual
+                    lays = [dict(x=h[j], codes=self.w_aa[r3][0], scales=self.w_aa[r3][1], out=h[a_], epilogue="residual", residual=h[(j + 3) % 4]),
+                            dict(x=h[a_], codes=self.w_ba[r2][0], scales=self.w_ba[r2][1], out=g[r2], epilogue="swiglu", depends=True),
+                            dict(x=g[r2], codes=self.w_ab[r2][0], scales=self.w_ab[r2][1], out=h[b_], epilogue="residual", residual=h[a_], depends=True)]
+                key = (kind, j, r3, r2)
+                if key not in self.batches:
+                    self.batches[key] = mxq.LinearBatch(lays)
+                    need = self.batches[key].workspace_bytes()
+                    if self.batch_ws is None or self.batch_ws.numel() < need:
+                        torch.cuda.synchronize()
+                        self.batch_ws = mxq.new_workspace(need)
+                self.batches[key].run(self.batch_ws)
             else:   # three independent layers in one launch, reading what earlier calls left
                 outs = [torch.empty((self.m, A), dtype=torch.bfloat16, device="cuda") for _ in range(2)] + \
                        [torch.empty((self.m, B), dtype=torch.bfloat16, device="cuda")]
@@ -116,7 +143,7 @@ def test_a_program_of_calls_without_synchronisation(m, seed):
     for attempt in range(3):
         got = prog.run(sync=False)
         for idx, (a, b) in enumerate(zip(ref, got)):
-            assert torch.equal(a, b), "M=%d seed %d: item %d of the final state differs without synchronisation (attempt %d)" % (m, seed, idx, attempt)
+            assert same_bits(a, b), "M=%d seed %d: item %d of the final state differs without synchronisation (attempt %d)" % (m, seed, idx, attempt)
     assert mxq.mxq_linear_device_status() == 0
 
 
@@ -133,7 +160,7 @@ def test_a_program_on_the_7b_widths(m, only_own_kernels):
     for attempt in range(3):
         got = prog.run(sync=False)
         for idx, (a, b) in enumerate(zip(ref, got)):
-            assert torch.equal(a, b), "M=%d: item %d of the final state differs without synchronisation (attempt %d)" % (m, idx, attempt)
+            assert same_bits(a, b), "M=%d: item %d of the final state differs without synchronisation (attempt %d)" % (m, idx, attempt)
     assert mxq.mxq_linear_device_status() == 0
 
 
@@ -141,10 +168,11 @@ def test_a_program_on_the_7b_widths(m, only_own_kernels):
 @pytest.mark.parametrize("m", [1, 2, 3, 4, 5, 8, 9, 16])
 def test_programs_of_the_librarys_own_kernels_only(m, seed):
     """Every call overlaps the one before it: the hardest ordering case, at every kernel choice the token count selects."""
-    prog = Program(m, 5000 + 10 * m + seed, steps=32, widths=(4096, 11008), kinds=("lin", "res", "swi", "down", "accept", "recast"))
+    prog = Program(m, 5000 + 10 * m + seed, steps=32, widths=(4096, 11008), kinds=("lin", "res", "swi", "down", "accept", "recast", "batch_direct", "batch_groups"))
     ref = prog.run(sync=True)
+    assert all(bool(torch.isfinite(t.float()).all()) for t in ref[:6]), "the program's values ran away: not a useful case"
     for attempt in range(2):
         got = prog.run(sync=False)
         for idx, (a, b) in enumerate(zip(ref, got)):
-            assert torch.equal(a, b), "M=%d seed %d: item %d of the final state differs without synchronisation (attempt %d)" % (m, seed, idx, attempt)
+            assert same_bits(a, b), "M=%d seed %d: item %d of the final state differs without synchronisation (attempt %d)" % (m, seed, idx, attempt)
     assert mxq.mxq_linear_device_status() == 0

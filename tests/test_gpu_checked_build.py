@@ -63,9 +63,9 @@ def test_the_ordinary_build_says_so():
 SELECTION = ("ragged or small or windows or token_operand or workspace or config1 or config2 or wide_range or many_tiles "
              "or in_place or composed or aligned or without_a_tcgen05 or epilogues or far_below or cannot_be_rewritten "
              "or does_not_cover or ring_depths or sixty_four or dependent_groups_in_one_call or outside_the_tensor_core or two_passes "
-             "or chain")
+             "or chain or program")
 FILES = ["tests/test_gpu_linear.py", "tests/test_gpu_epilogues.py", "tests/test_gpu_lm_head_accept.py", "tests/test_gpu_linear_batch.py",
-         "tests/test_gpu_linear_bf16.py", "tests/test_gpu_chain.py"]
+         "tests/test_gpu_linear_bf16.py", "tests/test_gpu_chain.py", "tests/test_gpu_async_programs.py"]
 
 
 def test_ragged_and_tiny_shapes_touch_nothing_outside_their_buffers():

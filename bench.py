@@ -164,7 +164,10 @@ class LinearPass:
             self.info = self.batches[0].info()
         else:
             ws_bytes = max([mxq.mxq_linear_workspace_bytes(m, n, k) for _, n, k, _, _ in mats] + [16])
-            self.ws = mxq.new_workspace(ws_bytes, device)
+            self.nstreams = max(1, min(streams, len(mats)))
+            self.wss = [mxq.new_workspace(ws_bytes, device) for _ in range(self.nstreams)]
+            self.ws = self.wss[0]
+            self.side = [torch.cuda.Stream(device=device) for _ in range(self.nstreams)] if self.nstreams > 1 else []
             self.launches = len(mats)
         self.graph = None
         self.stream = torch.cuda.Stream(device=device)
@@ -182,8 +185,21 @@ class LinearPass:
         if self.batches is not None:
             self.calls.run(self.stream)
             return
-        for (_, n, k, codes, scales), y in zip(self.mats, self.y):
-            self.mxq.mxq_linear(self.x[k], codes, scales, out=y, workspace=self.ws)
+        if not self.side:
+            for (_, n, k, codes, scales), y in zip(self.mats, self.y):
+                self.mxq.mxq_linear(self.x[k], codes, scales, out=y, workspace=self.ws)
+            return
+        # the independent calls round-robin on several streams, a workspace each, between a fork and a join
+        fork = torch.cuda.Event()
+        fork.record(self.stream)
+        for s_ in self.side:
+            s_.wait_event(fork)
+        for i, ((_, n, k, codes, scales), y) in enumerate(zip(self.mats, self.y)):
+            self.mxq.mxq_linear(self.x[k], codes, scales, out=y, workspace=self.wss[i % self.nstreams], stream=self.side[i % self.nstreams])
+        for s_ in self.side:
+            join = torch.cuda.Event()
+            join.record(s_)
+            self.stream.wait_event(join)
 
     def step(self):
         if self.graph is not None:
@@ -424,7 +440,7 @@ def run_ours(args):
         todo = [(head, per_call, streams)]
         for name, pc, ns in (("batch_%d_layer_sets_per_call" % nper, per_call, 1), ("batch_4_layer_sets_per_call_%d_streams" % streams, 4 * n7, streams),
                              ("batch_4_layer_sets_per_call", 4 * n7, 1), ("batch_1_layer_set_per_call_%d_streams" % streams, n7, streams),
-                             ("batch_1_layer_set_per_call", n7, 1), ("separate_calls", 0, 1)):
+                             ("batch_1_layer_set_per_call", n7, 1), ("separate_calls_%d_streams" % streams, 0, streams), ("separate_calls", 0, 1)):
             if (pc, ns) != (per_call, streams) and pc <= n7 * args.layers and name not in [t_[0] for t_ in todo] and (ns == 1 or streams > 1):
                 todo.append((name, pc, ns))
         for name, pc, ns in todo:

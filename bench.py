@@ -6,8 +6,9 @@ draft-token pass over the linear projections of ``--layers`` (default 32) distin
 layers -- q/k/v/o 4096x4096, gate/up 11008x4096, down 4096x11008 -- i.e. 224 independent layer
 problems per step, streaming 3.44 GB of MXFP4 weights (far larger than the 126 MB L2, so every
 step reads HBM).  They run through mxq_linear_batch, ``--layers-per-call`` (default 8) layer
-sets = 56 layers per launch; the same step with four and with one layer set per launch and as 224
-separate mxq_linear calls is timed beside it (``extra.routes``).  Weights are synthetic (Student-t, seeded), direct-cast on the device by
+sets = 56 layers per launch, the step's independent calls issued round-robin on ``--streams``
+(default 2) CUDA streams with a workspace each; the same step on one stream, with four and with one
+layer set per launch and as 224 separate mxq_linear calls is timed beside it (``extra.routes``).  Weights are synthetic (Student-t, seeded), direct-cast on the device by
 mxq_quantize before timing; the offline cast and the greedy-accept step are timed separately and
 reported under "extra".
 

@@ -341,6 +341,27 @@ def time_graph(fn, iters: int, warmup: int = 3):
     return e0.elapsed_time(e1) * 1e-3 / iters
 
 
+def round_robin(calls, nstreams: int):
+    """fn() that issues the independent `calls` (each takes the stream to run on) round-robin on `nstreams` streams between a
+    fork from and a join to the current stream: a call then starts in the SMs the other stream's call leaves, without
+    waiting for it to drain."""
+    side = [torch.cuda.Stream() for _ in range(nstreams)]
+
+    def fn():
+        cur = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(cur)
+        for s_ in side:
+            s_.wait_event(fork)
+        for i, call in enumerate(calls):
+            call(side[i % nstreams])
+        for s_ in side:
+            join = torch.cuda.Event()
+            join.record(s_)
+            cur.wait_event(join)
+    return fn
+
+
 def cpu_baseline_leg(m: int, budget_s: float = 15.0):
     """The oracle, as it stands, on one 7B layer set (host cores of this machine)."""
     import numpy as np
@@ -783,7 +804,12 @@ def run_ours(args):
         tq = time_graph(q, 10) / 4
         extra["quantize"] = {"gbs": 11008 * 4096 * 2.53125 / tq / 1e9, "us_per_call": tq * 1e6, "shape": "11008x4096",
                              "frac_of_peak": 11008 * 4096 * 2.53125 / tq / 1e9 / peaks["hbm_gbs"]}
-        del w, ws_
+        # the same casts, which are independent of one another, round-robin on two streams (outputs of their own)
+        outs2 = [(torch.empty_like(codes), torch.empty_like(scales)) for _ in ws_]
+        tq2 = time_graph(round_robin([(lambda st_, w_=w_, o_=o_: mxq.mxq_quantize(w_, o_[0], o_[1], stream=st_)) for w_, o_ in zip(ws_, outs2)], 2), 10) / 4
+        extra["quantize"]["two_streams"] = {"gbs": 11008 * 4096 * 2.53125 / tq2 / 1e9, "us_per_call": tq2 * 1e6,
+                                            "frac_of_peak": 11008 * 4096 * 2.53125 / tq2 / 1e9 / peaks["hbm_gbs"]}
+        del w, ws_, outs2
         # config 5: the direct cast of all 40 layers of a 13B-shaped model (12.69 G weights, 25.4 GB of BF16 in, 6.7 GB
         # out), every matrix resident, one replayed graph of the 280 casts
         try:
@@ -799,6 +825,10 @@ def run_ours(args):
             weights13 = sum(w_.numel() for w_ in w13)
             extra["quantize_13b"] = {"ms_per_sweep": t13 * 1e3, "weights": weights13, "gbs": weights13 * 2.53125 / t13 / 1e9,
                                      "frac_of_peak": weights13 * 2.53125 / t13 / 1e9 / peaks["hbm_gbs"], "matrices": len(w13)}
+            t13b = time_graph(round_robin([(lambda st_, w_=w_, c_=c_, s_=s_: mxq.mxq_quantize(w_, c_, s_, stream=st_))
+                                           for w_, c_, s_ in zip(w13, c13, s13)], 2), 3)
+            extra["quantize_13b"]["two_streams"] = {"ms_per_sweep": t13b * 1e3, "gbs": weights13 * 2.53125 / t13b / 1e9,
+                                                    "frac_of_peak": weights13 * 2.53125 / t13b / 1e9 / peaks["hbm_gbs"]}
             del w13, c13, s13
         except torch.OutOfMemoryError as e:   # (a GPU with less memory than the 32 GB this leg holds)
             extra["quantize_13b"] = {"skipped": str(e)[:80]}

@@ -837,6 +837,14 @@ def run_ours(args):
         ws2 = mxq.new_workspace(mxq.mxq_accept_workspace_bytes(250, 17, 32000), device)
         ta = time_graph(lambda: mxq.mxq_greedy_accept(lg, draft, workspace=ws2), 20)
         extra["greedy_accept"] = {"gbs": lg.numel() * 4 / ta / 1e9, "us_per_call": ta * 1e6, "shape": "250x17x32000 f32"}
+        # two such batches, independent of each other, on two streams (logits, workspace and outputs of their own)
+        lg_b, draft_b, _, _ = synth.accept_trials(250, 16, 17, 32000, seed=2, device=device)
+        ws2b = mxq.new_workspace(mxq.mxq_accept_workspace_bytes(250, 17, 32000), device)
+        outs_a = [tuple(torch.empty(250, dtype=torch.int32, device=device) for _ in range(2)) for _ in range(2)]
+        ta2 = time_graph(round_robin([lambda st_: mxq.mxq_greedy_accept(lg, draft, workspace=ws2, stream=st_, out=outs_a[0]),
+                                      lambda st_: mxq.mxq_greedy_accept(lg_b, draft_b, workspace=ws2b, stream=st_, out=outs_a[1])], 2), 20) / 2
+        extra["greedy_accept"]["two_streams"] = {"gbs": lg.numel() * 4 / ta2 / 1e9, "us_per_call": ta2 * 1e6}
+        del lg_b, draft_b
         del lg
 
     cpu = None

@@ -280,16 +280,22 @@ def mxq_linear_host(x_host: torch.Tensor, codes: torch.Tensor, scales: torch.Ten
            "mxq_linear_host")
 
 
-def mxq_greedy_accept(logits: torch.Tensor, draft: torch.Tensor, workspace: torch.Tensor = None, stream=None):
-    """logits [B,R,V] (fp32 or bf16), draft [B,T] int32 -> (accept_len [B], next_token [B]) int32."""
+def mxq_greedy_accept(logits: torch.Tensor, draft: torch.Tensor, workspace: torch.Tensor = None, stream=None, out=None):
+    """logits [B,R,V] (fp32 or bf16), draft [B,T] int32 -> (accept_len [B], next_token [B]) int32.  ``out``: optional
+    pair of int32 [B] tensors to write into (pass them when the call runs on another stream than the current one)."""
     b, r, v = logits.shape
     t = draft.shape[1]
     if workspace is None:
         workspace = new_workspace(mxq_accept_workspace_bytes(b, r, v), logits.device)
-    g = torch.empty(b, dtype=torch.int32, device=logits.device)
-    nxt = torch.empty(b, dtype=torch.int32, device=logits.device)
+    if out is None:
+        g = torch.empty(b, dtype=torch.int32, device=logits.device)
+        nxt = torch.empty(b, dtype=torch.int32, device=logits.device)
+    else:
+        g, nxt = out
+        if tuple(g.shape) != (b,) or tuple(nxt.shape) != (b,):
+            raise ValueError("out must be two int32 tensors of shape [B]")
     _check(lib().mxq_greedy_accept(_dev(logits, logits.dtype, "logits"), _dt(logits.dtype), b, r, v,
-                                   _dev(draft, torch.int32, "draft"), t, g.data_ptr(), nxt.data_ptr(),
+                                   _dev(draft, torch.int32, "draft"), t, _dev(g, torch.int32, "accept_len"), _dev(nxt, torch.int32, "next_token"),
                                    _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)),
            "mxq_greedy_accept")
     return g, nxt

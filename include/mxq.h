@@ -284,7 +284,7 @@ int mxq_linear_swiglu(const void *X_bf16, int M, const uint8_t *codes, const uin
 
 /* Several layers in ONE launch (Sec. III-B: a draft step is bound by the stream of its weights; Sec. III-D-2: the
  * operators of a layer fused around its linear layers).  A decoder layer is seven small matrices, and a kernel launch
- * per matrix costs more than its 1.4-3.7 us of weight traffic; here one persistent grid (one CTA per SM) walks all
+ * per matrix costs more than its 1.4-3.7 us of weight traffic; here one persistent grid (two CTAs per SM) walks all
  * the layers of the call with one uninterrupted stream of weights, the token rows of every distinct X are rewritten as
  * tensor-core operands once, and tiles that fall into two CTAs' shares are summed in a fixed order.
  *   descs   HOST array of `count` (1..MXQ_MAX_BATCH) descriptors, read during the call only.  Per layer:
@@ -337,7 +337,7 @@ int mxq_linear_batch(const mxq_linear_desc *descs, int count, int M, void *works
  * [0] launches of the persistent kernel (1; 2 for 9..16 token rows, the rest then describes the first), 0 if the
  * layers would run one by one; [1] CTAs; [2] ring slots per
  * CTA; [3] dynamic shared memory bytes; [4] columns of the token operand; [5] units of work (128 rows x 256 k);
- * [6] tensor-memory columns per CTA. */
+ * [6] tensor-memory columns per CTA; [7] accumulator slots in tensor memory. */
 int mxq_linear_batch_info(const mxq_linear_desc *descs, int count, int M, int32_t *info);
 
 /* Test hook for the bounded waits of mxq_linear_batch: the NEXT call of mxq_linear_batch (one-shot) leaves out the weight
